@@ -1,0 +1,255 @@
+"""CPU oracle for the group-wise mixed-precision weight-only linear layer.
+
+TEST INFRASTRUCTURE ONLY.  This file is the plain, slow, obviously-correct
+statement of what the CUDA library must compute.  It shares no code with the
+CUDA path and must never be imported by it: only the tests, the smoke check and
+the CPU-baseline leg of the benchmark may call it.
+
+Notation follows the paper: the weight is w in R^{n x m} (here N x K, groups of
+g = 128 consecutive input columns, Algorithm 1 slices w[:, b:b+beta]), x in
+R^{t x m} (here M x K), N-bar is the target average bit-width.
+
+Everything floating point is fp64 computed from fp16-exact inputs unless a line
+says otherwise.
+
+Pinned (tests/test_oracle_*.py): bit budget, quantizer closed forms and brute
+force, packing positions, dequantisation single-rounding, linear layer special
+cases.  Parity unpinned: nothing in this file (the paper's perplexity / accuracy
+/ token-per-second tables are not reproduced at all).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+GROUP = 128
+
+# A b-bit code is stored as slices (lo, w): slice value = (q >> lo) & (2^w - 1).
+# This is the storage format's definition, restated here independently.
+CODE_SLICES = {1: ((0, 1),), 2: ((0, 2),), 3: ((0, 2), (2, 1)), 4: ((0, 4),)}
+
+
+# --------------------------------------------------------------------------- salience / bit map
+def group_salience(W16: np.ndarray, act_norm: np.ndarray, g: int = GROUP, power: int = 2) -> np.ndarray:
+    """Group salience S_j = sum_{k in group j} a_k^power * sum_n w[n,k]^2.
+
+    Diagonal form of Definition 1 / Theorem 1 (Sec. 3.2.1): the salience of a
+    column is proportional to its squared weights times the squared activation
+    norm of that input channel.  Alg. 2 (SBA, first step) averages it per group;
+    sum and average rank groups identically because groups have equal size.
+    """
+    W = W16.astype(np.float64)
+    a = np.asarray(act_norm).astype(np.float64)
+    N, K = W.shape
+    assert K % g == 0 and a.shape == (K,)
+    col = (W * W).sum(axis=0) * a**power
+    return col.reshape(K // g, g).sum(axis=1)
+
+
+def allocate_bits(salience: np.ndarray, avg_bits: int, p: int | None = None) -> np.ndarray:
+    """Bit-width per group under the constraint |G_{N-1}| = |G_{N+1}| (Eq. 4).
+
+    Groups are ranked by salience (descending; equal salience: lower index first).
+    The p most salient groups get N-bar+1 bits, the p least salient N-bar-1, the
+    rest N-bar.  p defaults to floor(G/4), the fixed ratio of the benchmark
+    workloads (the paper searches p with a KL objective, Alg. 2).
+    """
+    S = np.asarray(salience, dtype=np.float64)
+    G = S.shape[0]
+    if p is None:
+        p = G // 4
+    assert 0 <= 2 * p <= G
+    order = sorted(range(G), key=lambda j: (-S[j], j))
+    bits = np.full(G, avg_bits, dtype=np.uint8)
+    for j in order[:p]:
+        bits[j] = avg_bits + 1
+    for j in order[G - p:] if p > 0 else []:
+        bits[j] = avg_bits - 1
+    return bits
+
+
+# --------------------------------------------------------------------------- quantizer (Eq. 1)
+def quantize_minmax(W16: np.ndarray, bits: np.ndarray, g: int = GROUP):
+    """Asymmetric min-max uniform quantizer of Eq. 1, per (row, group).
+
+        s = (w_max - w_min) / (2^b - 1),  z = -round(w_min / s),
+        q = clamp(round(w / s) + z, 0, 2^b - 1)
+
+    Readings where the paper is silent: round = round-half-to-even; the range
+    always contains 0 (w_min <= 0 <= w_max) so that z lies in [0, 2^b - 1]; the
+    scale is rounded to fp16 (stored format) *before* z and q are computed; a
+    zero scale becomes 1; a scale beyond the fp16 range becomes 65504.
+
+    Returns codes uint8 [N][K], scales fp16 [G][N], zeros fp16 [G][N].
+    """
+    N, K = W16.shape
+    G = K // g
+    assert K % g == 0 and len(bits) == G
+    codes = np.zeros((N, K), dtype=np.uint8)
+    scales = np.zeros((G, N), dtype=np.float16)
+    zeros = np.zeros((G, N), dtype=np.float16)
+    for j in range(G):
+        b = int(bits[j])
+        levels = float(2**b - 1)
+        w = W16[:, j * g:(j + 1) * g].astype(np.float64)
+        lo = np.minimum(w.min(axis=1), 0.0)
+        hi = np.maximum(w.max(axis=1), 0.0)
+        with np.errstate(over="ignore"):
+            s16 = ((hi - lo) / levels).astype(np.float16)
+        s16[np.isinf(s16)] = np.float16(65504.0)
+        s16[s16 == 0] = np.float16(1.0)
+        s = s16.astype(np.float64)
+        z = np.clip(-np.rint(lo / s), 0.0, levels)
+        q = np.clip(np.rint(w / s[:, None]) + z[:, None], 0.0, levels)
+        codes[:, j * g:(j + 1) * g] = q.astype(np.uint8)
+        scales[j] = s16
+        zeros[j] = z.astype(np.float16)
+    return codes, scales, zeros
+
+
+def quantize_sign_alpha_1bit(W16: np.ndarray, g: int = GROUP):
+    """Eq. 2 for one-bit groups: w_b = sign(w) (sign(0) = +1), alpha = mean |w|.
+
+    Expressed in the deployed (scale, zero, code) form: q = [w >= 0], z = 1/2,
+    s = fp16(2 alpha), so that s (q - z) = +-alpha.  Returned with the layouts of
+    quantize_minmax, every group at one bit.
+    """
+    N, K = W16.shape
+    G = K // g
+    w = W16.astype(np.float64).reshape(N, G, g)
+    alpha = np.abs(w).mean(axis=2)
+    codes = (w >= 0).astype(np.uint8).reshape(N, K)
+    scales = (2.0 * alpha).astype(np.float16).T.copy()
+    zeros = np.full((G, N), 0.5, dtype=np.float16)
+    return codes, scales, zeros
+
+
+# --------------------------------------------------------------------------- dequantisation
+def _expand_group_param(p: np.ndarray, g: int) -> np.ndarray:
+    """[G][N] per-(group,row) parameter -> [N][K] per-element."""
+    return np.repeat(np.asarray(p).T, g, axis=1)
+
+
+def dequant_f64(codes, scales, zeros, g: int = GROUP) -> np.ndarray:
+    """w-hat = s (q - z), exact in fp64 (the closed-form inverse inside Eq. 5)."""
+    s = _expand_group_param(scales, g).astype(np.float64)
+    z = _expand_group_param(zeros, g).astype(np.float64)
+    return s * (codes.astype(np.float64) - z)
+
+
+def dequant_f16(codes, scales, zeros, g: int = GROUP) -> np.ndarray:
+    """fp16 materialisation: fp16_rn( f32(s) *_f32 ( f32(q) -_f32 f32(z) ) ).
+
+    For integer or half-integer z both fp32 operations are exact, so this is the
+    correctly rounded fp16 value of s (q - z).
+    """
+    s = _expand_group_param(scales, g).astype(np.float32)
+    z = _expand_group_param(zeros, g).astype(np.float32)
+    d = codes.astype(np.float32) - z
+    with np.errstate(over="ignore"):
+        return (s * d).astype(np.float16)
+
+
+# --------------------------------------------------------------------------- linear layer
+def linear_f64(x16, codes, scales, zeros, g: int = GROUP) -> np.ndarray:
+    """y_ref = x @ W-hat^T with exact (unrounded) dequantised weights, fp64."""
+    return x16.astype(np.float64) @ dequant_f64(codes, scales, zeros, g).T
+
+
+def linear_rows_f64(x16, codes, scales, zeros, rows, g: int = GROUP) -> np.ndarray:
+    """y_ref[:, rows] only (for sampled checks of large layers)."""
+    rows = np.asarray(rows)
+    return linear_f64(x16, codes[rows], np.asarray(scales)[:, rows], np.asarray(zeros)[:, rows], g)
+
+
+# --------------------------------------------------------------------------- storage format
+def packed_bytes(N: int, K: int, bits, g: int = GROUP) -> int:
+    """N*K*b-bar/8: groups are stored back to back without padding (App. B.2)."""
+    assert K % g == 0 and len(bits) == K // g
+    return 16 * N * int(np.asarray(bits, dtype=np.int64).sum())
+
+
+def _unit_word_index(N, bits_prefix, b, t, unit, lane, half):
+    """Index (in 32-bit words) of one word of the packed buffer.
+
+    Group at byte 16*N*B_j; inside it the 16-row tile t at t*256*b; inside that
+    the 256-byte unit `unit`; inside that lane L at 8*L; word `half` (0: even row,
+    1: odd row) at 4*half.
+    """
+    byte = 16 * N * bits_prefix + t * 256 * b + 256 * unit + 8 * lane + 4 * half
+    return byte // 4
+
+
+def pack(codes: np.ndarray, bits, g: int = GROUP) -> np.ndarray:
+    """Pack codes [N][K] into the sliced bit-plane format; returns uint8 bytes.
+
+    Format (g = 128, N a multiple of 16).  B_j = sum_{i<j} b_i.  Group j holds,
+    for each 16-row tile t, b_j units of 256 bytes.  The code of group width b is
+    cut into slices (lo, w) listed in CODE_SLICES[b]; a slice of width w owns w
+    consecutive units.  A unit is 32 lanes x 8 bytes; lane L = 4*gq + c
+    (gq = 0..7, c = 0..3) holds two little-endian 32-bit words, word 0 for row
+    16t + 2gq and word 1 for row 16t + 2gq + 1.  Word (row r, slice (lo, w),
+    unit u of the slice, c) has 32/w fields; field f occupies bits [w f, w f + w)
+    and stores slice (lo, w) of q[r, 128 j + 32 c + (32/w) u + f].
+    """
+    codes = np.asarray(codes, dtype=np.uint8)
+    N, K = codes.shape
+    G = K // g
+    assert g == 128 and K % g == 0 and N % 16 == 0 and len(bits) == G
+    out = np.zeros(packed_bytes(N, K, bits, g) // 4, dtype=np.uint32)
+    rows = np.arange(N)
+    t, r = rows // 16, rows % 16
+    gq, half = r // 2, r % 2
+    prefix = 0
+    for j in range(G):
+        b = int(bits[j])
+        q = codes[:, j * g:(j + 1) * g].astype(np.uint32)
+        assert int(q.max(initial=0)) < 2**b, "code out of range for its group width"
+        unit_base = 0
+        for (lo, w) in CODE_SLICES[b]:
+            nf = 32 // w
+            for u in range(w):
+                for c in range(4):
+                    word = np.zeros(N, dtype=np.uint32)
+                    for f in range(nf):
+                        k = 32 * c + nf * u + f
+                        word |= ((q[:, k] >> np.uint32(lo)) & np.uint32(2**w - 1)) << np.uint32(w * f)
+                    idx = _unit_word_index(N, prefix, b, t, unit_base + u, 4 * gq + c, half)
+                    out[idx] = word
+            unit_base += w
+        prefix += b
+    return out.view(np.uint8)
+
+
+def unpack(packed: np.ndarray, N: int, K: int, bits, g: int = GROUP) -> np.ndarray:
+    """Inverse of pack: bytes -> codes uint8 [N][K]."""
+    G = K // g
+    words = np.ascontiguousarray(packed).view(np.uint32)
+    assert words.size * 4 == packed_bytes(N, K, bits, g)
+    codes = np.zeros((N, K), dtype=np.uint8)
+    rows = np.arange(N)
+    t, r = rows // 16, rows % 16
+    gq, half = r // 2, r % 2
+    prefix = 0
+    for j in range(G):
+        b = int(bits[j])
+        unit_base = 0
+        for (lo, w) in CODE_SLICES[b]:
+            nf = 32 // w
+            for u in range(w):
+                for c in range(4):
+                    word = words[_unit_word_index(N, prefix, b, t, unit_base + u, 4 * gq + c, half)]
+                    for f in range(nf):
+                        k = j * g + 32 * c + nf * u + f
+                        v = (word >> np.uint32(w * f)) & np.uint32(2**w - 1)
+                        codes[:, k] |= (v << np.uint32(lo)).astype(np.uint8)
+            unit_base += w
+        prefix += b
+    return codes
+
+
+# --------------------------------------------------------------------------- convenience
+def make_layer(W16, act_norm, avg_bits: int, g: int = GROUP, p: int | None = None):
+    """Salience -> bit map -> quantizer, the pipeline of the benchmark configs."""
+    bits = allocate_bits(group_salience(W16, act_norm, g), avg_bits, p)
+    codes, scales, zeros = quantize_minmax(W16, bits, g)
+    return bits, codes, scales, zeros
