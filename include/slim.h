@@ -1,0 +1,140 @@
+/* slim.h -- C ABI of the B200 (sm_100a) group-wise mixed-precision weight-only linear layer.
+ *
+ * The layer is y = x * W^T with W stored quantised: the input dimension K is cut into groups of
+ * g = 128 consecutive columns (Algorithm 1 of the SliM-LLM paper slices w[:, b:b+beta]); group j
+ * carries one bit-width b_j in {1,2,3,4} (Salience-Determined Bit Allocation, Sec. 3.2.2) and every
+ * (row, group) pair carries an fp16 scale s and an fp16 zero point z.  A stored code q dequantises
+ * as w = s * (q - z) (inverse of Eq. 1, written out inside Eq. 5).
+ *
+ * Conventions
+ *   N = output features (rows of W), K = input features (columns of W), M = tokens (rows of x),
+ *   G = K / g groups.  All matrices are dense row-major:
+ *     x       fp16  [M][K]        device
+ *     y       fp16  [M][N]        device
+ *     scales  fp16  [G][N]        device   (N contiguous)
+ *     zeros   fp16  [G][N]        device   (any fp16 value; integers for Eq. 1, 0.5 for Eq. 2)
+ *     codes   uint8 [N][K]        device   (unpacked codes, code < 2^b_j)
+ *     bits    uint8 [G]           HOST     (read during the call; values 1..4)
+ *     packed  bytes               device   (format below, slim_packed_bytes() bytes)
+ *   "device" pointers must be 16-byte aligned and are owned by the caller, who keeps them alive
+ *   until the work enqueued on `stream` has finished.  No function allocates device memory,
+ *   none synchronises unless it says so, and all work is enqueued on `stream` (a cudaStream_t
+ *   passed as void*; NULL is the legacy default stream).  Calls never throw; they return a status.
+ *
+ * Limits: g must be 128; K a multiple of 128 with at most 256 groups; N a multiple of 16;
+ * N = 0 or M = 0 is a successful no-op.  Anything else returns an error status and enqueues nothing.
+ *
+ * Packed format ("sliced bit planes", version SLIM_FORMAT_VERSION).  Groups are stored back to
+ * back without padding, as the paper's deployment format does (App. B.2), so the buffer holds
+ * exactly N*K*avg_bits/8 bytes.  With B_j = b_0 + ... + b_{j-1}:
+ *   - group j starts at byte 16*N*B_j and holds, for each tile t of 16 consecutive rows, b_j
+ *     units of 256 bytes (tile t at offset t*256*b_j inside the group);
+ *   - a b-bit code is cut into slices (lo, w): b=1 -> (0,1); b=2 -> (0,2); b=3 -> (0,2),(2,1);
+ *     b=4 -> (0,4); slice value = (q >> lo) & (2^w - 1).  A slice of width w owns w consecutive
+ *     units, slices in the order listed;
+ *   - a unit is 32 lanes x 8 bytes.  Lane L = 4*gq + c (gq = 0..7, c = 0..3) holds two
+ *     little-endian 32-bit words: word 0 belongs to row 16t + 2gq, word 1 to row 16t + 2gq + 1;
+ *   - the word of (row r, slice (lo,w), unit u of that slice, c) has 32/w fields of w bits; field f
+ *     (bits [w*f, w*f + w)) stores the slice of q[r][128*j + 32*c + (32/w)*u + f].
+ */
+#ifndef SLIM_H_
+#define SLIM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SLIM_FORMAT_VERSION 2
+#define SLIM_GROUP 128
+#define SLIM_MAX_GROUPS 256
+#define SLIM_GEMV_MAX_M 16
+
+enum {
+    SLIM_OK = 0,
+    SLIM_ERR_INVALID_ARG = -1, /* null pointer, negative size, bit-width outside 1..4, M out of range */
+    SLIM_ERR_UNSUPPORTED = -2, /* g != 128, K % 128 != 0, N % 16 != 0, more than 256 groups */
+    SLIM_ERR_ALIGNMENT = -3,   /* a device pointer is not 16-byte aligned */
+    SLIM_ERR_WORKSPACE = -4,   /* workspace missing or smaller than slim_workspace_bytes() */
+    SLIM_ERR_CUDA = -5,        /* a CUDA runtime call failed; see slim_last_cuda_error() */
+    SLIM_ERR_TIMEOUT = -6      /* a device-side wait gave up (reported by slim_workspace_status) */
+};
+
+/* Library / format version: (SLIM_FORMAT_VERSION << 16) | build number. */
+int slim_version(void);
+/* Static, NUL-terminated description of a status code. */
+const char* slim_status_string(int status);
+/* cudaError_t value of the most recent failing CUDA call made by this library on the calling
+ * thread's process (0 if none). */
+int slim_last_cuda_error(void);
+
+/* Size of the packed buffer, N*K*avg_bits/8 bytes ("no additional padding", App. B.2). */
+int slim_packed_bytes(int N, int K, int g, const uint8_t* bits_host, size_t* out_bytes);
+
+/* Scratch size for slim_mpq_gemv / slim_mpq_gemm with these shapes on the current device
+ * (split-K partial sums, tile counters, one status word).  Always at least 256. */
+int slim_workspace_bytes(int M, int N, int K, int g, const uint8_t* bits_host, size_t* out_bytes);
+
+/* Zeroes the control part of a workspace (status word and tile counters).  Must be enqueued
+ * once after allocating a workspace, before its first use; the kernels leave it zeroed. */
+int slim_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronises `stream`, reads and clears the workspace status word.  Returns SLIM_OK, or
+ * SLIM_ERR_TIMEOUT if a kernel using this workspace abandoned a bounded wait (its output is
+ * then undefined), or SLIM_ERR_CUDA. */
+int slim_workspace_status(void* workspace, void* stream);
+
+/* Packs unpacked codes into the format above (the storage step of App. B.2: "packs the weights
+ * ... into integer-compressed representations based on the precision of different groups").
+ * Integer work, deterministic; codes with bits above b_j set are masked to b_j bits. */
+int slim_pack_weights(const uint8_t* codes, const uint8_t* bits_host, void* packed,
+                      int N, int K, int g, void* stream);
+
+/* Materialises W-hat as fp16 [N][K]:  W[n][k] = fp16_rn( f32(s) * ( f32(q) - f32(z) ) ) with both
+ * fp32 operations rounded to nearest (for integer or half-integer z this is the correctly rounded
+ * s*(q-z), the dequantisation of Eq. 1 / Eq. 5).  Bit-exact and deterministic. */
+int slim_dequant(const void* packed, const uint8_t* bits_host, const void* scales, const void* zeros,
+                 void* W, int N, int K, int g, void* stream);
+
+/* Decode path, 1 <= M <= 16:  y = x * W-hat^T, fp32 accumulation, fp16 output (the paper's
+ * inference kernel, App. B.2: group-by-group dequantisation and dot product with the shared
+ * activation).  Streams the packed slices once; HBM-bound.  Results are deterministic for a
+ * given (shape, device).  x with Inf/NaN gives unspecified y.  `workspace` may be NULL only if
+ * slim_workspace_bytes() reported 256 or less... it never does; pass a workspace. */
+int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host,
+                  const void* scales, const void* zeros, void* y,
+                  int M, int N, int K, int g,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* Batched / prefill path, M > 16: same contract, tensor-core (tcgen05) kernel. */
+int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* bits_host,
+                  const void* scales, const void* zeros, void* y,
+                  int M, int N, int K, int g,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---- producing the inputs of the layer (the steps right before packing) ------------------- */
+
+/* Group salience S_j = sum_{k in group j} a_k^2 * sum_n W[n][k]^2 (diagonal form of Definition 1 /
+ * Theorem 1; first step of SBA in Algorithm 2).  W fp16 [N][K] device, act_norm fp32 [K] device,
+ * salience fp64 [G] device.  fp64 accumulation in a fixed order. */
+int slim_group_salience(const void* W, const float* act_norm, double* salience,
+                        int N, int K, int g, void* stream);
+
+/* Host-only.  Bit-width per group under |G_{N-1}| = |G_{N+1}| = p (Eq. 4): the p most salient
+ * groups get avg_bits+1, the p least salient avg_bits-1, the rest avg_bits; equal salience ranks
+ * the lower index higher.  p < 0 selects floor(G/4).  avg_bits in {2,3}. */
+int slim_allocate_bits(const double* salience_host, int G, int avg_bits, int p, uint8_t* bits_host_out);
+
+/* Asymmetric min-max quantizer of Eq. 1 per (row, group), in fp64 from the fp16 weights:
+ * range extended to contain 0, s rounded to fp16 first (0 -> 1, overflow -> 65504),
+ * z = clamp(-rint(lo/s)), q = clamp(rint(w/s) + z), rint = round-half-to-even.
+ * W fp16 [N][K]; codes uint8 [N][K]; scales, zeros fp16 [G][N]; all device. */
+int slim_quantize_minmax(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
+                         int N, int K, int g, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLIM_H_ */

@@ -98,7 +98,7 @@ def quantize_minmax(W16: np.ndarray, bits: np.ndarray, g: int = GROUP):
         s16[np.isinf(s16)] = np.float16(65504.0)
         s16[s16 == 0] = np.float16(1.0)
         s = s16.astype(np.float64)
-        z = np.clip(-np.rint(lo / s), 0.0, levels)
+        z = np.clip(-np.rint(lo / s), 0.0, levels) + 0.0   # an unsigned integer: -0.0 is stored as +0
         q = np.clip(np.rint(w / s[:, None]) + z[:, None], 0.0, levels)
         codes[:, j * g:(j + 1) * g] = q.astype(np.uint8)
         scales[j] = s16

@@ -1,0 +1,226 @@
+"""Thin ctypes binding of the C ABI declared in include/slim.h.
+
+Argument marshalling only: every function checks dtypes/devices, takes raw device
+pointers from torch tensors and the current CUDA stream, and calls the entry point
+of the same name.  There is no fallback: if the CUDA library has not been built
+the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+from .build import LIB_PATH
+
+GROUP = 128
+GEMV_MAX_M = 16
+
+_lib = None
+
+
+class SlimError(RuntimeError):
+    def __init__(self, fn: str, status: int, text: str, cuda_error: int):
+        super().__init__(f"{fn} failed: {text} (status {status}, cuda error {cuda_error})")
+        self.status = status
+        self.cuda_error = cuda_error
+
+
+def lib():
+    """Loads libslim_b200.so (built by paper_2405_14917_b200.build.build())."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"CUDA library not built: {LIB_PATH} is missing; run "
+                               "`python -m paper_2405_14917_b200.build` (there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.slim_version.restype = i
+        L.slim_version.argtypes = []
+        L.slim_status_string.restype = ctypes.c_char_p
+        L.slim_status_string.argtypes = [i]
+        L.slim_last_cuda_error.restype = i
+        L.slim_last_cuda_error.argtypes = []
+        sigs = {
+            "slim_packed_bytes": [i, i, i, vp, ctypes.POINTER(sz)],
+            "slim_workspace_bytes": [i, i, i, i, vp, ctypes.POINTER(sz)],
+            "slim_workspace_init": [vp, sz, vp],
+            "slim_workspace_status": [vp, vp],
+            "slim_pack_weights": [vp, vp, vp, i, i, i, vp],
+            "slim_dequant": [vp, vp, vp, vp, vp, i, i, i, vp],
+            "slim_mpq_gemv": [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp],
+            "slim_mpq_gemm": [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp],
+            "slim_group_salience": [vp, vp, vp, i, i, i, vp],
+            "slim_allocate_bits": [vp, i, i, i, vp],
+            "slim_quantize_minmax": [vp, vp, vp, vp, vp, i, i, i, vp],
+        }
+        for name, args in sigs.items():
+            fn = getattr(L, name)
+            fn.restype = i
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def _check(fn: str, status: int):
+    if status != 0:
+        L = lib()
+        raise SlimError(fn, status, L.slim_status_string(status).decode(), L.slim_last_cuda_error())
+
+
+def _bits(bits) -> np.ndarray:
+    b = np.ascontiguousarray(np.asarray(bits), dtype=np.uint8)
+    assert b.ndim == 1
+    return b
+
+
+def _bp(b: np.ndarray):
+    return b.ctypes.data_as(ctypes.c_void_p)
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of dtype {dtype}")
+    return t.data_ptr()
+
+
+def _stream(t: torch.Tensor) -> int:
+    return torch.cuda.current_stream(t.device).cuda_stream
+
+
+def version() -> int:
+    return lib().slim_version()
+
+
+def packed_bytes(N: int, K: int, bits, g: int = GROUP) -> int:
+    b = _bits(bits)
+    out = ctypes.c_size_t(0)
+    _check("slim_packed_bytes", lib().slim_packed_bytes(N, K, g, _bp(b), ctypes.byref(out)))
+    return out.value
+
+
+def workspace_bytes(M: int, N: int, K: int, bits, g: int = GROUP) -> int:
+    b = _bits(bits)
+    out = ctypes.c_size_t(0)
+    _check("slim_workspace_bytes", lib().slim_workspace_bytes(M, N, K, g, _bp(b), ctypes.byref(out)))
+    return out.value
+
+
+def workspace_init(workspace: torch.Tensor) -> None:
+    p = _dev(workspace, torch.uint8, "workspace")
+    _check("slim_workspace_init", lib().slim_workspace_init(p, workspace.numel(), _stream(workspace)))
+
+
+def workspace_status(workspace: torch.Tensor) -> None:
+    """Synchronises; raises SlimError(SLIM_ERR_TIMEOUT) if a kernel gave up a bounded wait."""
+    p = _dev(workspace, torch.uint8, "workspace")
+    _check("slim_workspace_status", lib().slim_workspace_status(p, _stream(workspace)))
+
+
+def new_workspace(M: int, N: int, K: int, bits, device="cuda") -> torch.Tensor:
+    """Allocates (torch) and initialises a workspace large enough for this shape."""
+    ws = torch.empty(workspace_bytes(M, N, K, bits), dtype=torch.uint8, device=device)
+    workspace_init(ws)
+    return ws
+
+
+def pack_weights(codes: torch.Tensor, bits, packed: torch.Tensor | None = None) -> torch.Tensor:
+    b = _bits(bits)
+    N, K = codes.shape
+    if packed is None:
+        packed = torch.empty(packed_bytes(N, K, b), dtype=torch.uint8, device=codes.device)
+    _check("slim_pack_weights", lib().slim_pack_weights(_dev(codes, torch.uint8, "codes"), _bp(b),
+                                                        _dev(packed, torch.uint8, "packed"), N, K, GROUP, _stream(codes)))
+    return packed
+
+
+def dequant(packed: torch.Tensor, bits, scales: torch.Tensor, zeros: torch.Tensor, N: int, K: int,
+            out: torch.Tensor | None = None) -> torch.Tensor:
+    b = _bits(bits)
+    if out is None:
+        out = torch.empty((N, K), dtype=torch.float16, device=packed.device)
+    _check("slim_dequant", lib().slim_dequant(_dev(packed, torch.uint8, "packed"), _bp(b),
+                                              _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
+                                              _dev(out, torch.float16, "W"), N, K, GROUP, _stream(packed)))
+    return out
+
+
+def _linear(fn_name: str, x, packed, bits, scales, zeros, N, workspace, out):
+    b = _bits(bits)
+    M, K = x.shape
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float16, device=x.device)
+    wp = _dev(workspace, torch.uint8, "workspace") if workspace is not None else None
+    wb = workspace.numel() if workspace is not None else 0
+    fn = getattr(lib(), fn_name)
+    _check(fn_name, fn(_dev(x, torch.float16, "x"), _dev(packed, torch.uint8, "packed"), _bp(b),
+                       _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
+                       _dev(out, torch.float16, "y"), M, N, K, GROUP, wp, wb, _stream(x)))
+    return out
+
+
+def mpq_gemv(x, packed, bits, scales, zeros, N: int, workspace, out=None) -> torch.Tensor:
+    """y = x W-hat^T for 1 <= M <= 16 (decode path)."""
+    return _linear("slim_mpq_gemv", x, packed, bits, scales, zeros, N, workspace, out)
+
+
+def mpq_gemm(x, packed, bits, scales, zeros, N: int, workspace, out=None) -> torch.Tensor:
+    """y = x W-hat^T for M > 16 (batched tensor-core path)."""
+    return _linear("slim_mpq_gemm", x, packed, bits, scales, zeros, N, workspace, out)
+
+
+def group_salience(W: torch.Tensor, act_norm: torch.Tensor) -> torch.Tensor:
+    N, K = W.shape
+    out = torch.empty(K // GROUP, dtype=torch.float64, device=W.device)
+    _check("slim_group_salience", lib().slim_group_salience(_dev(W, torch.float16, "W"), _dev(act_norm, torch.float32, "act_norm"),
+                                                            _dev(out, torch.float64, "salience"), N, K, GROUP, _stream(W)))
+    return out
+
+
+def allocate_bits(salience, avg_bits: int, p: int = -1) -> np.ndarray:
+    s = np.ascontiguousarray(np.asarray(salience), dtype=np.float64)
+    out = np.zeros(s.shape[0], dtype=np.uint8)
+    _check("slim_allocate_bits", lib().slim_allocate_bits(s.ctypes.data_as(ctypes.c_void_p), s.shape[0], avg_bits, p, _bp(out)))
+    return out
+
+
+def quantize_minmax(W: torch.Tensor, bits):
+    b = _bits(bits)
+    N, K = W.shape
+    G = K // GROUP
+    codes = torch.empty((N, K), dtype=torch.uint8, device=W.device)
+    scales = torch.empty((G, N), dtype=torch.float16, device=W.device)
+    zeros = torch.empty((G, N), dtype=torch.float16, device=W.device)
+    _check("slim_quantize_minmax", lib().slim_quantize_minmax(_dev(W, torch.float16, "W"), _bp(b), _dev(codes, torch.uint8, "codes"),
+                                                              _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
+                                                              N, K, GROUP, _stream(W)))
+    return codes, scales, zeros
+
+
+class QuantLinear:
+    """One quantised layer resident on the device: packed codes, scales, zeros, bit map."""
+
+    def __init__(self, packed, bits, scales, zeros, N: int, K: int):
+        self.packed, self.bits, self.scales, self.zeros, self.N, self.K = packed, _bits(bits), scales, zeros, N, K
+
+    @classmethod
+    def from_weight(cls, W: torch.Tensor, act_norm: torch.Tensor, avg_bits: int, p: int = -1) -> "QuantLinear":
+        """Salience -> bit allocation -> Eq. 1 quantizer -> packing, all on the device."""
+        N, K = W.shape
+        sal = group_salience(W, act_norm).cpu().numpy()
+        bits = allocate_bits(sal, avg_bits, p)
+        codes, scales, zeros = quantize_minmax(W, bits)
+        return cls(pack_weights(codes, bits), bits, scales, zeros, N, K)
+
+    def workspace_bytes(self, M: int) -> int:
+        return workspace_bytes(M, self.N, self.K, self.bits)
+
+    def forward(self, x: torch.Tensor, workspace: torch.Tensor, out=None) -> torch.Tensor:
+        fn = mpq_gemv if x.shape[0] <= GEMV_MAX_M else mpq_gemm
+        return fn(x, self.packed, self.bits, self.scales, self.zeros, self.N, workspace, out)
+
+    def algorithmic_bytes(self, M: int) -> int:
+        G = self.K // GROUP
+        return self.packed.numel() + 2 * 2 * G * self.N + G + 2 * M * self.K + 2 * M * self.N

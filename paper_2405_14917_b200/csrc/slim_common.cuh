@@ -1,0 +1,44 @@
+// Shared host-side helpers of the CUDA library: argument validation, the group table that
+// every kernel receives by value, and the last-CUDA-error slot.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/slim.h"
+
+namespace slim {
+
+// Group table passed by value in kernel parameters (the paper's "additional array" of group
+// bit-widths plus the "cumulative calculations" that give each group's start, App. B.2).
+struct GroupTable {
+    int G;
+    uint16_t prefix[SLIM_MAX_GROUPS + 1];  // prefix[j] = b_0 + ... + b_{j-1}
+    uint8_t bits[SLIM_MAX_GROUPS];
+};
+
+void set_cuda_error(cudaError_t e);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Validates shape arguments and fills the table.  Returns SLIM_OK or an error status.
+int make_group_table(int N, int K, int g, const uint8_t* bits_host, GroupTable* out);
+
+#define SLIM_CUDA_TRY(expr)                                    \
+    do {                                                       \
+        cudaError_t _e = (expr);                               \
+        if (_e != cudaSuccess) {                               \
+            ::slim::set_cuda_error(_e);                        \
+            return SLIM_ERR_CUDA;                              \
+        }                                                      \
+    } while (0)
+
+// Slice table of a b-bit code: number of slices, and (lo, w, first unit) of each.
+__host__ __device__ inline int slice_count(int b) { return b == 3 ? 2 : 1; }
+__host__ __device__ inline int slice_lo(int b, int s) { return (b == 3 && s == 1) ? 2 : 0; }
+__host__ __device__ inline int slice_w(int b, int s) { return b == 3 ? (s == 0 ? 2 : 1) : b; }
+__host__ __device__ inline int slice_unit0(int b, int s) { return (b == 3 && s == 1) ? 2 : 0; }
+
+}  // namespace slim

@@ -1,0 +1,120 @@
+// Producing the layer's inputs on the device: group salience (first step of SBA) and the
+// asymmetric min-max quantizer of Eq. 1.  fp64 arithmetic from fp16 weights, fixed summation
+// order, so the outputs are reproducible bit for bit.
+#include "slim_common.cuh"
+
+namespace slim {
+
+// One block per group.  Thread (ph, cp) owns column pair cp (2 columns) and rows ph, ph+4, ...
+// Column sums of squares are accumulated in fp64 in ascending row order per phase, the four
+// phases are added in order, then the 128 columns are weighted by a_k^2 and summed in order.
+__global__ void __launch_bounds__(256) salience_kernel(const __half* __restrict__ W, const float* __restrict__ act_norm,
+                                                       double* __restrict__ salience, int N, int K) {
+    const int j = blockIdx.x;
+    const int cp = threadIdx.x & 63, ph = threadIdx.x >> 6;
+    const __half2* base = reinterpret_cast<const __half2*>(W + static_cast<size_t>(SLIM_GROUP) * j) + cp;
+    double s0 = 0.0, s1 = 0.0;
+    for (int n = ph; n < N; n += 4) {
+        const float2 v = __half22float2(base[static_cast<size_t>(n) * (K / 2)]);
+        s0 += static_cast<double>(v.x) * static_cast<double>(v.x);
+        s1 += static_cast<double>(v.y) * static_cast<double>(v.y);
+    }
+    __shared__ double part[4][SLIM_GROUP];
+    part[ph][2 * cp] = s0;
+    part[ph][2 * cp + 1] = s1;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double total = 0.0;
+        for (int k = 0; k < SLIM_GROUP; ++k) {
+            const double col = ((part[0][k] + part[1][k]) + part[2][k]) + part[3][k];
+            const double a = static_cast<double>(act_norm[SLIM_GROUP * j + k]);
+            total += a * a * col;
+        }
+        salience[j] = total;
+    }
+}
+
+__device__ __forceinline__ unsigned short double_to_half_bits_rn(double v) {
+    unsigned short h;
+    asm("cvt.rn.f16.f64 %0, %1;" : "=h"(h) : "d"(v));
+    return h;
+}
+
+// One warp per (row, group): lane l owns columns 4l..4l+3 of the group.
+__global__ void __launch_bounds__(256) quantize_minmax_kernel(const __half* __restrict__ W, uint8_t* __restrict__ codes,
+                                                              __half* __restrict__ scales, __half* __restrict__ zeros,
+                                                              int N, int K, GroupTable gt) {
+    const long long warp = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    const int G = gt.G;
+    if (warp >= static_cast<long long>(N) * G) return;
+    const int n = static_cast<int>(warp / G), j = static_cast<int>(warp % G);
+    const size_t off = static_cast<size_t>(n) * K + SLIM_GROUP * j + 4 * lane;
+    const uint2 raw = *reinterpret_cast<const uint2*>(W + off);
+    const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+    const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+    const float w[4] = {f01.x, f01.y, f23.x, f23.y};
+    float lo = fminf(fminf(w[0], w[1]), fminf(w[2], w[3]));
+    float hi = fmaxf(fmaxf(w[0], w[1]), fmaxf(w[2], w[3]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    lo = fminf(lo, 0.0f);
+    hi = fmaxf(hi, 0.0f);
+    const int b = gt.bits[j];
+    const double levels = static_cast<double>((1 << b) - 1);
+    unsigned short sbits = double_to_half_bits_rn((static_cast<double>(hi) - static_cast<double>(lo)) / levels);
+    if ((sbits & 0x7fffu) == 0x7c00u) sbits = 0x7bffu;  // beyond fp16 range -> 65504
+    if ((sbits & 0x7fffu) == 0u) sbits = 0x3c00u;       // zero scale -> 1
+    const __half s16 = __ushort_as_half(sbits);
+    const double s = static_cast<double>(__half2float(s16));
+    const double z = fmin(fmax(-rint(static_cast<double>(lo) / s), 0.0), levels);
+    uint32_t out = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const double q = fmin(fmax(rint(static_cast<double>(w[i]) / s) + z, 0.0), levels);
+        out |= static_cast<uint32_t>(static_cast<int>(q)) << (8 * i);
+    }
+    *reinterpret_cast<uint32_t*>(codes + off) = out;
+    if (lane == 0) {
+        scales[static_cast<size_t>(j) * N + n] = s16;
+        zeros[static_cast<size_t>(j) * N + n] = __float2half_rn(static_cast<float>(z));
+    }
+}
+
+}  // namespace slim
+
+extern "C" {
+
+int slim_group_salience(const void* W, const float* act_norm, double* salience, int N, int K, int g, void* stream) {
+    if (N < 0 || K < 0) return SLIM_ERR_INVALID_ARG;
+    if (g != SLIM_GROUP || K % SLIM_GROUP != 0 || K / SLIM_GROUP > SLIM_MAX_GROUPS) return SLIM_ERR_UNSUPPORTED;
+    if (K == 0) return SLIM_OK;
+    if (W == nullptr || act_norm == nullptr || salience == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (!slim::aligned16(W) || !slim::aligned16(act_norm) || !slim::aligned16(salience)) return SLIM_ERR_ALIGNMENT;
+    slim::salience_kernel<<<K / SLIM_GROUP, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const __half*>(W), act_norm, salience, N, K);
+    SLIM_CUDA_TRY(cudaGetLastError());
+    return SLIM_OK;
+}
+
+int slim_quantize_minmax(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
+                         int N, int K, int g, void* stream) {
+    slim::GroupTable gt;
+    const int st = slim::make_group_table(N, K, g, bits_host, &gt);
+    if (st != SLIM_OK) return st;
+    if (N == 0 || K == 0) return SLIM_OK;
+    if (W == nullptr || codes == nullptr || scales == nullptr || zeros == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (!slim::aligned16(W) || !slim::aligned16(codes) || !slim::aligned16(scales) || !slim::aligned16(zeros))
+        return SLIM_ERR_ALIGNMENT;
+    const long long warps = static_cast<long long>(N) * gt.G;
+    const unsigned grid = static_cast<unsigned>((warps + 7) / 8);
+    slim::quantize_minmax_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const __half*>(W), codes, static_cast<__half*>(scales), static_cast<__half*>(zeros), N, K, gt);
+    SLIM_CUDA_TRY(cudaGetLastError());
+    return SLIM_OK;
+}
+
+}  // extern "C"

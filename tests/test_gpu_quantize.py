@@ -1,0 +1,70 @@
+"""GPU parity: salience, bit allocation and the Eq. 1 quantizer against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import slim_oracle as orc
+from paper_2405_14917_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _slim():
+    from paper_2405_14917_b200 import binding
+    return binding
+
+
+@pytest.mark.parametrize("N,K,avg", [(64, 512, 2), (1024, 4096, 2), (272, 11008, 3), (512, 5120, 3)])
+def test_salience_bits_and_quantizer_match_oracle(N, K, avg):
+    slim = _slim()
+    seed = wl.layer_seed("test", f"quant-{N}x{K}", avg)
+    W = wl.make_weight(seed, N, K)
+    a = wl.make_act_norms(seed, K)
+    sal_ref = orc.group_salience(W, a)
+    sal = slim.group_salience(torch.from_numpy(W).cuda(), torch.from_numpy(a).cuda()).cpu().numpy()
+    assert np.allclose(sal, sal_ref, rtol=1e-12, atol=0)
+    bits_ref = orc.allocate_bits(sal_ref, avg)
+    bits = slim.allocate_bits(sal, avg)
+    # the ranking is decided in fp64 on both sides; a different map is only acceptable on a near-tie
+    if not (bits == bits_ref).all():
+        diff = np.flatnonzero(bits != bits_ref)
+        order = np.sort(sal_ref)
+        gaps = np.min(np.abs(sal_ref[diff][:, None] - np.delete(order, 0)[None, :]), axis=1)
+        assert (gaps <= 1e-11 * sal_ref[diff]).all(), "bit maps differ without a salience tie"
+    assert int(bits.astype(int).sum()) == avg * (K // 128)
+    codes, scales, zeros = slim.quantize_minmax(torch.from_numpy(W).cuda(), bits_ref)
+    c_ref, s_ref, z_ref = orc.quantize_minmax(W, bits_ref)
+    assert (scales.cpu().numpy().view(np.uint16) == s_ref.view(np.uint16)).all()
+    assert (zeros.cpu().numpy().view(np.uint16) == z_ref.view(np.uint16)).all()
+    assert (codes.cpu().numpy() == c_ref).all()
+
+
+def test_quantizer_edge_groups():
+    """All-positive, all-negative, constant-zero, huge-range and tiny-range groups."""
+    slim = _slim()
+    rng = np.random.default_rng(3)
+    N, K = 16, 640
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float16)
+    W[:, 0:128] = np.abs(W[:, 0:128])
+    W[:, 128:256] = -np.abs(W[:, 128:256])
+    W[:, 256:384] = 0
+    W[:, 384:512] = np.clip(rng.standard_normal((N, 128)) * 3e4, -6e4, 6e4).astype(np.float16)   # range beyond fp16 for 1 bit
+    W[:, 512:640] = (rng.standard_normal((N, 128)) * 1e-7).astype(np.float16)  # subnormal weights
+    for bits in ([1, 2, 3, 1, 4], [4, 3, 2, 1, 1], [2, 2, 2, 2, 2]):
+        bits = np.array(bits, dtype=np.uint8)
+        c_ref, s_ref, z_ref = orc.quantize_minmax(W, bits)
+        codes, scales, zeros = slim.quantize_minmax(torch.from_numpy(W).cuda(), bits)
+        assert (scales.cpu().numpy().view(np.uint16) == s_ref.view(np.uint16)).all()
+        assert (zeros.cpu().numpy().view(np.uint16) == z_ref.view(np.uint16)).all()
+        assert (codes.cpu().numpy() == c_ref).all()
+
+
+def test_allocate_bits_host_matches_oracle_on_ties_and_p():
+    slim = _slim()
+    rng = np.random.default_rng(5)
+    for G in (4, 32, 86, 108, 224):
+        S = rng.integers(0, 6, G).astype(np.float64)   # many ties
+        for avg in (2, 3):
+            assert (slim.allocate_bits(S, avg) == orc.allocate_bits(S, avg)).all()
+            for p in (0, 1, G // 2):
+                assert (slim.allocate_bits(S, avg, p) == orc.allocate_bits(S, avg, p)).all()

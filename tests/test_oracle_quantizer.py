@@ -28,6 +28,7 @@ def test_hand_worked_cases(case):
     codes, scales, zeros = orc.quantize_minmax(W, np.array([b], dtype=np.uint8))
     assert scales.dtype == np.float16 and zeros.dtype == np.float16
     assert float(scales[0, 0]) == s and float(zeros[0, 0]) == z
+    assert not np.signbit(zeros).any()   # the zero point is an unsigned integer: never -0
     assert float(scales[0, 1]) == s and float(zeros[0, 1]) == z
     assert codes[0].tolist() == [qs[i % len(ws)] for i in range(128)]
     assert codes[1].tolist() == codes[0].tolist()[::-1]
