@@ -1,0 +1,375 @@
+"""Benchmark of the group-wise mixed-precision weight-only linear layer on B200.
+
+Default workload: the LLaMA-7B decode layer set at M = 1, average 2 bits (bit-widths {1,2,3} per
+group of 128 input columns): q/k/v/o 4096x4096, gate/up 11008x4096, down 4096x11008 for all 32
+blocks, 224 distinct layers (1.83 GB of packed weights, scales and zeros, far larger than L2).
+One step = one pass over all 224 layers, replayed from a CUDA graph.  The metric is achieved
+GB/s over the algorithmic bytes (packed codes + fp16 scales and zeros + bit map + x + y).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints one JSON line (rank 0).  With N > 1 every rank runs an independent replica of the
+workload on its own GPU (no data-path collective); the value is the sum over ranks divided by
+the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2405_14917_b200 import workloads as wl  # noqa: E402
+
+METRIC = "mixed-precision dequant GEMV GB/s at M=1 (LLaMA-7B layer set, avg 2-bit, g=128)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of the GEMV kernel per launch from one ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), keyed by the sha256 of the kernel source it was taken from.  A kernel
+# that has changed since reports null.
+NCU_TRAFFIC = {
+    # "sha256 of csrc/slim_gemv.cu": {"layer": "NxK", "traffic_bytes": ..., "algorithmic_bytes": ...}
+}
+
+
+def workload_spec(name: str):
+    if name == "llama7b-decode-avg2":
+        return dict(model="llama-7b", avg_bits=2, M=1, n_blocks=wl.N_BLOCKS["llama-7b"])
+    if name == "llama7b-decode-avg3":
+        return dict(model="llama-7b", avg_bits=3, M=1, n_blocks=wl.N_BLOCKS["llama-7b"])
+    if name == "llama7b-block-avg2":      # one block only (small case for profiling)
+        return dict(model="llama-7b", avg_bits=2, M=1, n_blocks=4)
+    raise SystemExit(f"unknown workload {name}")
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            time.sleep(0.3)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [t.strip() for t in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for nm, v in zip(names, f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nm)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle legs
+def _oracle_layers(spec, n_layers):
+    """First n_layers layers of the sweep, generated and quantised on the host by the oracle."""
+    from oracle import slim_oracle as orc
+    out = []
+    for (name, blk, N, K, seed) in wl.model_layers(spec["model"], spec["n_blocks"]):
+        if len(out) >= n_layers:
+            break
+        W = wl.make_weight(seed, N, K)
+        a = wl.make_act_norms(seed, K)
+        bits, codes, scales, zeros = orc.make_layer(W, a, spec["avg_bits"])
+        out.append(dict(name=name, N=N, K=K, bits=bits, codes=codes, scales=scales, zeros=zeros,
+                        x=wl.make_x(seed, spec["M"], K)))
+    return out
+
+
+def _time_oracle(layers, rows_of_first=None):
+    """Runs the plain-C oracle once over `layers` (optionally only the first rows of the first
+    layer).  Returns (seconds, algorithmic bytes, threads)."""
+    from oracle import slim_oracle_c as oc
+    total_bytes, threads = 0, 1
+    t0 = time.perf_counter()
+    for L in layers:
+        codes, scales, zeros, N = L["codes"], L["scales"], L["zeros"], L["N"]
+        if rows_of_first is not None:
+            N = rows_of_first
+            codes, scales, zeros = codes[:N], np.ascontiguousarray(scales[:, :N]), np.ascontiguousarray(zeros[:, :N])
+        _, threads = oc.linear_f64(L["x"], codes, scales, zeros)
+        total_bytes += wl.algorithmic_bytes(L["x"].shape[0], N, L["K"], L["bits"])
+    return time.perf_counter() - t0, total_bytes, threads
+
+
+def cpu_baseline(spec, budget_s=12.0):
+    """The oracle as it stands on the host cores, over the first block's layers (bounded)."""
+    from oracle import slim_oracle_c as oc
+    oc.build()
+    layers = _oracle_layers(spec, 7)
+    _time_oracle(layers[:1], rows_of_first=256)   # load the library, touch the code
+    secs, nbytes, reps, threads = 0.0, 0, 0, 1
+    while secs < budget_s and reps < 8:
+        s, b, threads = _time_oracle(layers)
+        secs, nbytes, reps = secs + s, nbytes + b, reps + 1
+    return {"value": nbytes / secs / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"block 0 of the sweep (7 layers, {nbytes // reps / 1e6:.1f} MB algorithmic) x {reps} passes, "
+                      f"plain-C fp64 dequantise-then-dot, OpenMP over rows, {secs:.1f} s"}
+
+
+def run_reference(args, spec):
+    """--impl reference: the CPU oracle, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import slim_oracle_c as oc
+    oc.build()
+    steps = args.steps if args.steps is not None else 5
+    warmup = args.warmup if args.warmup is not None else 1
+    layers = _oracle_layers(spec, 7)
+    # calibrate on 256 rows of the first layer, then size the per-step sample for ~100 s in total
+    t_cal, _, threads = _time_oracle(layers[:1], rows_of_first=256)
+    t_cal, _, threads = _time_oracle(layers[:1], rows_of_first=256)
+    per_row = t_cal / 256
+    budget = 100.0 / max(steps + warmup, 1)
+    block_rows = sum(L["N"] * L["K"] for L in layers) / layers[0]["K"]
+    if per_row * block_rows <= budget:
+        sample, rows, what = layers, None, "block 0 of the sweep (7 layers)"
+    else:
+        rows = int(min(layers[0]["N"], max(16, budget / per_row))) // 16 * 16
+        rows = max(rows, 16)
+        sample, what = layers[:1], f"first {rows} output rows of layer q, block 0"
+    for _ in range(warmup):
+        _time_oracle(sample, rows)
+    secs, nbytes = 0.0, 0
+    for _ in range(steps):
+        s, b, threads = _time_oracle(sample, rows)
+        secs, nbytes = secs + s, nbytes + b
+    value = nbytes / secs / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": 1e3 * secs / steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "M": spec["M"], "avg_bits": spec["avg_bits"], "g": wl.GROUP},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": what + "; plain-C fp64 dequantise-then-dot, OpenMP over rows"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+def build_layers(spec, device, rank):
+    """Quantises the whole sweep on the device through the library: salience, bit allocation,
+    Eq. 1 quantizer, packing.  Returns the resident layers."""
+    import torch
+    from paper_2405_14917_b200 import binding as slim
+    layers = []
+    for (name, blk, N, K, seed) in wl.model_layers(spec["model"], spec["n_blocks"]):
+        W, a = wl.make_weight_and_norms_device(seed + (rank,), N, K, device)
+        layers.append(slim.QuantLinear.from_weight(W, a, spec["avg_bits"]))
+        del W, a
+    torch.cuda.synchronize()
+    return layers
+
+
+def run_ours(args, spec):
+    import torch
+    import torch.distributed as dist
+    from paper_2405_14917_b200 import binding as slim
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    steps = args.steps if args.steps is not None else 2000
+    warmup = max(args.warmup if args.warmup is not None else 20, 3)
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    slim.lib()   # fails loudly if the CUDA library is missing
+
+    layers = build_layers(spec, device, rank)
+    M = spec["M"]
+    alg_bytes = sum(L.algorithmic_bytes(M) for L in layers)
+
+    # all activations of the sweep in one buffer, all outputs in another
+    x_off = np.cumsum([0] + [M * L.K for L in layers])
+    y_off = np.cumsum([0] + [M * L.N for L in layers])
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(1234 + rank)
+    x_host = torch.randn(int(x_off[-1]), generator=gen, dtype=torch.float32).to(torch.float16).pin_memory()
+    y_host = torch.empty(int(y_off[-1]), dtype=torch.float16).pin_memory()
+    x_dev = x_host.to(device)
+    y_dev = torch.zeros(int(y_off[-1]), dtype=torch.float16, device=device)
+    ws = torch.zeros(max(L.workspace_bytes(M) for L in layers), dtype=torch.uint8, device=device)
+    slim.workspace_init(ws)
+    xs = [x_dev[x_off[i]:x_off[i + 1]].view(M, L.K) for i, L in enumerate(layers)]
+    ys = [y_dev[y_off[i]:y_off[i + 1]].view(M, L.N) for i, L in enumerate(layers)]
+
+    def sweep():
+        for L, x, y in zip(layers, xs, ys):
+            L.forward(x, ws, out=y)
+
+    # capture one sweep in a CUDA graph (launch-bound otherwise: ~1.4 us of HBM time per layer)
+    side = torch.cuda.Stream(device)
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        sweep()
+        sweep()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        sweep()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(step_fn, n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(n):
+            step_fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    def step_device():
+        graph.replay()
+
+    def step_e2e():
+        x_dev.copy_(x_host, non_blocking=True)
+        graph.replay()
+        y_host.copy_(y_dev, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for _ in range(warmup):
+        step_device()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms = timed(step_device, steps)
+    clocks = sampler.stop() if rank == 0 else None
+    slim.workspace_status(ws)
+
+    e2e_steps = max(steps // 4, 3)
+    for _ in range(3):
+        step_e2e()
+    ms_e2e = timed(step_e2e, e2e_steps)
+    slim.workspace_status(ws)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    value = world * alg_bytes * steps / (ms * 1e-3) / 1e9
+    e2e_value = world * alg_bytes * e2e_steps / (ms_e2e * 1e-3) / 1e9
+    peak, peak_kind = measured_hbm_peak()
+    n_launch = len(layers)
+    per_launch_us = 1e3 * ms / steps / n_launch
+    achieved = alg_bytes / n_launch / (per_launch_us * 1e-6) / 1e9
+    sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2405_14917_b200", "csrc", "slim_gemv.cu"), "rb").read()).hexdigest()
+    traffic = NCU_TRAFFIC.get(sha)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f16 (exact fp8-split products on mma.sync, f32 accumulate)", "data": "synthetic",
+        "config": {"workload": args.workload, "layers": n_launch, "M": M, "avg_bits": spec["avg_bits"], "g": wl.GROUP,
+                   "algorithmic_bytes_per_step": alg_bytes, "l2": "distinct layers, 1.8 GB per step >> L2",
+                   "launch": "CUDA graph of one launch per layer, programmatic dependent launch",
+                   "parallelism": f"replicas x{world}"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": peak_kind, "kernel": "gemv_kernel", "avg_launch_us": per_launch_us,
+                     "algorithmic_bytes_per_launch": alg_bytes / n_launch,
+                     "traffic": traffic["traffic_bytes"] if traffic else None,
+                     "frac_of_nominal_8000": achieved / 8000.0},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 2),
+                "d2h_bytes_per_step": int(y_host.numel() * 2), "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
+        "gpu_launches": steps * n_launch,
+        "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(spec)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama7b-decode-avg2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    spec = workload_spec(args.workload)
+    if args.impl == "reference":
+        run_reference(args, spec)
+    else:
+        run_ours(args, spec)
+
+
+if __name__ == "__main__":
+    main()

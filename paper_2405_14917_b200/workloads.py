@@ -87,3 +87,22 @@ def algorithmic_bytes(M: int, N: int, K: int, bits) -> int:
     G = K // GROUP
     assert bits.shape == (G,)
     return int(N * GROUP * int(bits.sum()) // 8 + 2 * 2 * G * N + G + 2 * M * K + 2 * M * N)
+
+
+def make_weight_and_norms_device(seed: tuple, N: int, K: int, device, outlier_frac: float = 0.01,
+                                 outlier_gain: float = 10.0, sigma: float = 0.02):
+    """Same recipe as make_weight / make_act_norms, drawn on the device with torch's seeded generator.
+
+    Used where hundreds of full-size layers are needed (billions of draws); the values differ
+    from the NumPy streams but follow the same distributions.  Returns (W fp16 [N][K], a fp32 [K]).
+    """
+    import torch
+    gen = torch.Generator(device=device)
+    gen.manual_seed(int(np.random.SeedSequence(list(seed)).generate_state(1, dtype=np.uint64)[0] >> 1))
+    w = torch.randn((N, K), generator=gen, device=device, dtype=torch.float32) * sigma
+    n_out = int(round(outlier_frac * K))
+    if n_out > 0:
+        cols = torch.randperm(K, generator=gen, device=device)[:n_out]
+        w[:, cols] *= outlier_gain
+    a = torch.exp(torch.randn(K, generator=gen, device=device, dtype=torch.float32))
+    return w.to(torch.float16), a
