@@ -333,7 +333,7 @@ def run_ours(args, spec):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f16 (exact fp8-split products on mma.sync, f32 accumulate)", "data": "synthetic",
+        "dtype": "f16 (mma.sync m16n8k16 on raw code fields, f32 accumulate)", "data": "synthetic",
         "config": {"workload": args.workload, "layers": n_launch, "M": M, "avg_bits": spec["avg_bits"], "g": wl.GROUP,
                    "algorithmic_bytes_per_step": alg_bytes, "l2": "distinct layers, 1.8 GB per step >> L2",
                    "launch": "CUDA graph of one launch per layer, programmatic dependent launch",

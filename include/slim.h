@@ -108,6 +108,12 @@ int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host,
                   int M, int N, int K, int g,
                   void* workspace, size_t workspace_bytes, void* stream);
 
+/* Host-only introspection: the launch plan slim_mpq_gemv uses for this shape on the current device
+ * (148 SMs assumed when no device is present).  out6 = {16-row tiles per CTA, k-slices =
+ * cluster size, row blocks, dynamic shared memory bytes, 8-token MMA tiles, groups per chunk}.
+ * grid = k-slices x row blocks, 8 warps per CTA. */
+int slim_gemv_plan(int M, int N, int K, int g, const uint8_t* bits_host, int* out6);
+
 /* Batched / prefill path, M > 16: same contract, tensor-core (tcgen05) kernel. */
 int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* bits_host,
                   const void* scales, const void* zeros, void* y,

@@ -52,6 +52,7 @@ def lib():
             "slim_dequant": [vp, vp, vp, vp, vp, i, i, i, vp],
             "slim_mpq_gemv": [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp],
             "slim_mpq_gemm": [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp],
+            "slim_gemv_plan": [i, i, i, i, vp, vp],
             "slim_group_salience": [vp, vp, vp, i, i, i, vp],
             "slim_allocate_bits": [vp, i, i, i, vp],
             "slim_quantize_minmax": [vp, vp, vp, vp, vp, i, i, i, vp],
@@ -106,6 +107,14 @@ def workspace_bytes(M: int, N: int, K: int, bits, g: int = GROUP) -> int:
     out = ctypes.c_size_t(0)
     _check("slim_workspace_bytes", lib().slim_workspace_bytes(M, N, K, g, _bp(b), ctypes.byref(out)))
     return out.value
+
+
+def gemv_plan(M: int, N: int, K: int, bits, g: int = GROUP) -> dict:
+    """Launch plan of slim_mpq_gemv for this shape (host-only)."""
+    b = _bits(bits)
+    out = (ctypes.c_int * 6)()
+    _check("slim_gemv_plan", lib().slim_gemv_plan(M, N, K, g, _bp(b), ctypes.cast(out, ctypes.c_void_p)))
+    return dict(zip(("tiles_per_cta", "k_slices", "row_blocks", "smem_bytes", "n_tiles", "groups_per_chunk"), list(out)))
 
 
 def workspace_init(workspace: torch.Tensor) -> None:

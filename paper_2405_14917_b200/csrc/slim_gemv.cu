@@ -1,44 +1,45 @@
 // slim_mpq_gemv: decode path (1 <= M <= 16) of the mixed-precision linear layer, sm_100a.
 //
 // The kernel streams the packed slices exactly once (HBM-bound) and does the dot products on
-// the tensor cores without ever materialising fp16 weights:
+// the tensor cores (mma.sync m16n8k16, fp16 x fp16 -> fp32) without materialising fp16 weights:
 //
-//  * A operand = raw code slices.  A byte whose low nibble holds a code field v (v <= 15) and
-//    whose high nibble is zero is, read as FP8 E4M3, exactly v * 2^-9 (subnormals and the first
-//    binade are linear in the bit pattern).  So one AND isolates the same field of four weights
-//    and yields four ready-to-use E4M3 operands; fields in the high nibble need one shift first.
-//    The position of a field inside the nibble (bit 0..3) multiplies its value by a power of two.
-//  * B operand = activations.  Each fp16 x[m][k] is split exactly into four E5M2 pieces (3
-//    significant bits each, 4 x 3 >= 11); the four pieces of a token occupy four columns of the
-//    m16n8k32 tile, so one n-tile serves two tokens.  While staging, each piece is multiplied by
-//    the power of two that undoes the field position and slice offset of the weight it will meet,
-//    and by a per-token power of two 2^S that centres the token's range in E5M2.
-//  * mma.sync.m16n8k32.e4m3.e5m2 accumulates the exact products in fp32.  Per (row, group) the
-//    group partial D is folded as acc += s * (D - z * sum_k x_k), which is s * sum_k x_k (q_k - z).
-//  * At the end the piece columns of a token are added and scaled by 2^(9-S).
+//  * A operand = raw code slices.  A 16-bit half whose exponent and sign bits are zero and whose
+//    mantissa holds a code field v at bit position pos is the subnormal v * 2^(pos-24), exactly.
+//    A slice word keeps the fields of columns f and f + nf/2 sixteen bits apart, so ONE AND
+//    yields a ready-to-use half2 operand (two weights); fields above mantissa bit 9 need the word
+//    shifted right once first.
+//  * B operand = activations, staged once per CTA in fragment order: x[m][k] * 2^(S + lo - pos),
+//    where pos undoes the field position of the weight it will meet, lo is the slice's offset
+//    inside the code, and 2^S (per token and chunk, from max|x|) lifts the values to the top of the
+//    fp16 range so that the small ones keep their bits.
+//  * The MMA accumulates the exact products in fp32.  Per (row, group) the group partial D is
+//    folded as acc += s * (D - z * sum_k x_k), which is s * sum_k x_k (q_k - z); the chunk's
+//    2^(24-S) is undone when the chunk is added to the running sum.
 //
-// Work split: grid = (row blocks of 128*T rows) x (SK contiguous group ranges).  Each of the 8
-// warps of a CTA owns T 16-row tiles and walks the CTA's group range; for one group its T tiles
-// are one contiguous run of the packed buffer, fetched with one bulk async copy (plus two small
-// ones for scales and zeros) into a warp-private ring of stages guarded by mbarriers.  Split-K
-// partials go to the workspace; the last CTA of a row block (atomic ticket) adds them in a fixed
-// order, so results are deterministic.
-//
-// The kernel is launched with programmatic stream serialisation: it issues its first weight
-// copies, lets the next kernel start, and only then waits for the previous kernel before it
-// touches x, y or the workspace.  Back-to-back layers therefore overlap their weight streams.
+// Work split.  A layer is smaller than, or comparable to, the bytes HBM must keep in flight, and
+// a warp's instruction stream is the critical path, so the kernel spreads a layer over as many
+// warps as possible and is built around latency:
+//  * grid = (CS k-slices) x (row blocks of T 16-row tiles); the CS CTAs of one row block form a
+//    thread-block cluster.  Warp w of a CTA owns tile w % T and takes every (8/T)-th group of the
+//    CTA's range, so x is staged once for T tiles; the range is walked in chunks of GC groups
+//    (one chunk for decode-sized inputs).
+//  * Every warp issues the weight, scale and zero bytes of its groups of the first chunk as
+//    16-byte cp.async copies in its first instructions; chunk c+1 is in flight while chunk c is
+//    consumed.
+//  * The kernel is launched with programmatic stream serialisation: after issuing the copies it
+//    lets the next kernel start (whose copies then overlap this kernel's arithmetic) and only
+//    then waits for the previous kernel before it touches x or y.
+//  * Partial sums are added across warps in shared memory and across the cluster through
+//    distributed shared memory, both in a fixed order (deterministic); no global scratch.
 #include "slim_common.cuh"
 
 #include <cstring>
 
 namespace slim {
 
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
-constexpr int kMaxSplit = 64;
-constexpr int kMaxStages = 8;
+constexpr int kMaxWarps = 8;
+constexpr int kMaxCluster = 8;
 constexpr int kWsHeader = 256;              // status word + padding
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct GemvParams {
     const __half* x;
@@ -46,61 +47,43 @@ struct GemvParams {
     const __half* scales;
     const __half* zeros;
     __half* y;
-    float* partials;        // [SK][M][N] fp32 (workspace)
-    unsigned int* counters; // [row blocks] (workspace)
-    unsigned int* status;   // workspace status word
     int M, N, K;
-    int SK;
-    int nstage;
-    int stage_bytes;        // bytes of one ring stage (weights of T tiles at the widest group + scales + zeros)
-    int w_stage_bytes;      // offset of the scales inside a stage
-    int max_groups;         // widest group range of any split (sizes the x staging area)
-    int max_slots;          // most slices in any group range
-    uint16_t kbegin[kMaxSplit + 1];
+    int CS;                 // k-slices (= cluster size)
+    int W;                  // warps per CTA
+    int T;                  // 16-row tiles per CTA (divides W)
+    int GC;                 // groups per chunk
+    int region_bytes;       // landing buffer of one chunk (largest chunk, all T tiles)
+    int max_slots;          // most slices in any chunk
+    int two_bufs;           // some k-slice has more than one chunk: weights and raw x are double-buffered
+    uint16_t kbegin[kMaxCluster + 1];
     GroupTable gt;
 };
 
 // ------------------------------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_timer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait: gives up after kWaitLimitNs and reports false (the caller flags the error and
-// stops consuming; nothing ever spins without a limit).
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_timer_ns();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - t0 > kWaitLimitNs) return false;
-    }
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ float2 ld_cluster_f32x2(uint32_t local_addr, uint32_t rank) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(remote) : "memory");
+    return v;
+}
 
 __device__ __forceinline__ uint2 lds64(uint32_t addr) {
     uint2 v;
@@ -113,26 +96,28 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
     return v;
 }
 
-// D += A(e4m3, 16x32) * B(e5m2, 32x8), fp32 accumulate.
-__device__ __forceinline__ void mma_e4m3_e5m2(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint2 b) {
+// D += A(f16, 16x16, row) * B(f16, 16x8, col), fp32 accumulate.
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint2 b) {
     asm volatile(
-        "mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e5m2.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b.x), "r"(b.y));
 }
 
 // ------------------------------------------------------------------------------------------ slice geometry
-// Field p (0 .. 8/W-1) of every byte of a slice word, isolated in the low nibble of its byte.
-// `sh` is the word shifted right by 4 (computed once per word by the caller).
+// A word of a width-w slice has nf = 32/w fields; pair p (0 <= p < nf/2) is fields p and p + nf/2,
+// which sit 16 bits apart.  Pairs whose field ends above mantissa bit 9 are taken from the word
+// shifted right by pair_shift(w).
+__host__ __device__ constexpr int pair_shift(int w) { return w == 4 ? 8 : 10; }
+__host__ __device__ constexpr bool pair_direct(int w, int p) { return w * p + w <= 10; }
+// Bit position of pair p inside each half after the optional shift: the operand is v * 2^(pos-24).
+__host__ __device__ constexpr int pair_pos(int w, int p) { return pair_direct(w, p) ? w * p : w * p - pair_shift(w); }
+
 template <int W>
-__device__ __forceinline__ uint32_t field(uint32_t word, uint32_t sh, int p) {
-    constexpr int kPerNibble = 4 / W;                     // fields that fit in one nibble
-    constexpr uint32_t kMask = 0x01010101u * ((1u << W) - 1u);
-    const uint32_t src = (p < kPerNibble) ? word : sh;
-    return src & (kMask << (W * (p % kPerNibble)));
+__device__ __forceinline__ uint32_t pair(uint32_t word, uint32_t sh, int p) {
+    constexpr uint32_t kMask = 0x00010001u * ((1u << W) - 1u);
+    return (pair_direct(W, p) ? word : sh) & (kMask << pair_pos(W, p));
 }
-// Bit position of field p inside its nibble after the optional shift: its value is scaled by 2^pos.
-__host__ __device__ __forceinline__ int field_pos(int w, int p) { return w * (p % (4 / w)); }
 
 template <int V> struct WidthTag { static constexpr int value = V; };
 using W1 = WidthTag<1>;
@@ -141,338 +126,326 @@ using W4 = WidthTag<4>;
 
 // ------------------------------------------------------------------------------------------ shared memory map
 struct SmemMap {
-    uint32_t mbar;     // kWarps * nstage * 8
-    uint32_t sexp;     // int[16]: per-token power-of-two exponent S
-    uint32_t xslot;    // uint16[max_groups + 1]: first staging slot of each group of the range
-    uint32_t sx;       // float[max_groups][8*NT]: 2^(S-9) * sum_k x (piece-0 columns only)
-    uint32_t xraw;     // half[M][max_groups*128]
-    uint32_t xs;       // [slots][4 mma][NT][32 lanes][8 B]
-    uint32_t ring;     // kWarps * nstage * stage_bytes
+    uint32_t smax;     // uint32[2][16]: per-token max |x| bits over the chunk (double-buffered)
+    uint32_t xslot;    // uint16[GC + 1]: first staging slot of each group of the chunk
+    uint32_t sx;       // float[GC][16]: 2^(S-24) * sum_k x per (group, token)
+    uint32_t red;      // float[W][M][16]: per-warp partial outputs, then [M][16] in place of warp 0
+    uint32_t xraw;     // half[2][M][GC*128] (double-buffered)
+    uint32_t xs;       // [slots][8 mma][M tokens][4 lanes] x 8 B: B fragments
+    uint32_t wbuf;     // [2][region_bytes]: packed slices, scales, zeros of the chunk
     uint32_t total;
 };
 __host__ __device__ inline uint32_t align_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
-__host__ __device__ inline SmemMap make_smem_map(int NT, int M, int nstage, int stage_bytes, int max_groups, int max_slots) {
+__host__ __device__ inline SmemMap make_smem_map(int M, int W, int GC, int region_bytes, int max_slots, bool two_bufs) {
     SmemMap m;
     uint32_t o = 0;
-    m.mbar = o;  o += kWarps * kMaxStages * 8;
-    m.sexp = o;  o += 64;
-    m.xslot = o; o += align_up(2 * (max_groups + 1), 16);
-    m.sx = o;    o += align_up(4 * max_groups * 8 * NT, 16);
-    m.xraw = o;  o += align_up(2 * M * max_groups * SLIM_GROUP, 16);
+    m.smax = o;  o += 128;
+    m.xslot = o; o += align_up(2 * (GC + 1), 16);
+    m.sx = o;    o += 64u * GC;
+    m.red = o;   o += 64u * W * M;
+    m.xraw = o;  o += (two_bufs ? 2u : 1u) * (256u * M * GC);
     o = align_up(o, 128);
-    m.xs = o;    o += static_cast<uint32_t>(max_slots) * 4 * NT * 256;
+    m.xs = o;    o += static_cast<uint32_t>(max_slots) * 8 * M * 32;
     o = align_up(o, 128);
-    m.ring = o;  o += static_cast<uint32_t>(kWarps) * nstage * stage_bytes;
+    m.wbuf = o;  o += (two_bufs ? 2u : 1u) * region_bytes;
     m.total = o;
     return m;
 }
 
 // ------------------------------------------------------------------------------------------ kernel
-template <int NT, int T>
-__global__ void __launch_bounds__(kThreads, 2) gemv_kernel(const __grid_constant__ GemvParams p) {
+template <int NT>   // 8-token MMA tiles: 1 (M <= 8) or 2
+__global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_constant__ GemvParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
-    const SmemMap sm = make_smem_map(NT, p.M, p.nstage, p.stage_bytes, p.max_groups, p.max_slots);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int W = p.W, T = p.T, KW = W / T, nthreads = W * 32;
     const int gq = lane >> 2, c = lane & 3;
-    const int rb = blockIdx.x, ks = blockIdx.y;
-    const int N = p.N, M = p.M;
+    const int ks = blockIdx.x, rb = blockIdx.y;
+    const int N = p.N, M = p.M, GC = p.GC;
     const int g0 = p.kbegin[ks], g1 = p.kbegin[ks + 1];
     const int ng = g1 - g0;
+    const int n_chunks = (ng + GC - 1) / GC;
+    const SmemMap sm = make_smem_map(M, W, GC, p.region_bytes, p.max_slots, p.two_bufs != 0);
+    const uint32_t xraw_stride = 256u * M * GC;                   // bytes per xraw buffer
+    const int tw = warp % T, kw = warp / T;                       // this warp's tile of the CTA and k-way
+    const int tile = rb * T + tw;
+    const bool active = tile < (N >> 4);
 
-    const int tiles_total = N >> 4;
-    const int tile0 = (rb * kWarps + warp) * T;
-    const int tw = min(T, tiles_total - tile0);            // tiles this warp owns (<= 0: none)
-    const bool active = tw > 0;
-
-    const uint32_t my_bar = sbase + sm.mbar + warp * kMaxStages * 8;
-    const uint32_t my_ring = sbase + sm.ring + static_cast<uint32_t>(warp) * p.nstage * p.stage_bytes;
-
-    // ---- producer side: one chunk = (this warp's tiles, one group): weights, scales, zeros
-    auto issue_chunk = [&](int it) {
-        const int j = g0 + it;
-        const int b = p.gt.bits[j];
-        const int st = it % p.nstage;
-        const uint32_t bar = my_bar + st * 8;
-        const uint32_t dst = my_ring + st * p.stage_bytes;
-        const uint32_t wbytes = static_cast<uint32_t>(tw) * 256u * b;
-        const uint32_t sbytes = static_cast<uint32_t>(tw) * 32u;
-        mbar_expect_tx(bar, wbytes + 2 * sbytes);
-        bulk_g2s(dst, p.packed + 16ull * N * p.gt.prefix[j] + static_cast<size_t>(tile0) * 256 * b, wbytes, bar);
-        bulk_g2s(dst + p.w_stage_bytes, p.scales + static_cast<size_t>(j) * N + 16 * tile0, sbytes, bar);
-        bulk_g2s(dst + p.w_stage_bytes + T * 32, p.zeros + static_cast<size_t>(j) * N + 16 * tile0, sbytes, bar);
+    // Layout of a chunk buffer: group after group, inside a group the T tiles one after another,
+    // each as its slices followed by 32 bytes of scales and 32 bytes of zeros.
+    auto item_addr = [&](uint32_t buf, int ja, int j, int b) -> uint32_t {
+        return buf + T * (256u * (p.gt.prefix[j] - p.gt.prefix[ja]) + 64u * (j - ja)) + tw * (256u * b + 64u);
     };
-
-    if (lane == 0) {
-        for (int s = 0; s < p.nstage; ++s) mbar_init(my_bar + s * 8, 1);
-        fence_barrier_init();
-        fence_proxy_async();
-        if (active) {
-            const int pre = min(p.nstage, ng);
-            for (int it = 0; it < pre; ++it) issue_chunk(it);
-        }
-    }
-    __syncwarp();
-
-    // Weights are in flight; let the next kernel begin its own prefetch, then wait until the
-    // previous kernel has finished before x, y or the workspace are touched.
-    pdl_launch_dependents();
-    pdl_wait();
-
-    // ---- stage x for this group range ---------------------------------------------------------
-    const int kr = ng * SLIM_GROUP;                           // columns in this range
-    {
-        // raw copy + per-token max exponent; warp `warp` serves tokens warp, warp + 8
-        for (int m = warp; m < M; m += kWarps) {
-            const __half2* src = reinterpret_cast<const __half2*>(p.x + static_cast<size_t>(m) * p.K + g0 * SLIM_GROUP);
-            uint32_t mx = 0;
-            for (int i = lane; i < kr / 2; i += 32) {
-                const uint32_t v = *reinterpret_cast<const uint32_t*>(src + i);
-                *reinterpret_cast<uint32_t*>(smem + sm.xraw + (static_cast<size_t>(m) * kr + 2 * i) * 2) = v;
-                mx = max(mx, max(v & 0x7fffu, (v >> 16) & 0x7fffu));
-            }
-            mx = __reduce_max_sync(0xffffffffu, mx);
-            if (lane == 0) {
-                const int e = max(static_cast<int>(mx >> 10), 1);   // biased exponent of the largest |x| (Inf/NaN: 31)
-                reinterpret_cast<int*>(smem + sm.sexp)[m] = (mx == 0) ? 0 : 27 - e;  // max|x| * 2^S in [2^12, 2^13)
-            }
-        }
-        if (tid == 0) {
-            uint16_t* xslot = reinterpret_cast<uint16_t*>(smem + sm.xslot);
-            int slot = 0;
-            for (int i = 0; i < ng; ++i) { xslot[i] = static_cast<uint16_t>(slot); slot += slice_count(p.gt.bits[g0 + i]); }
-            xslot[ng] = static_cast<uint16_t>(slot);
-        }
-        // zero the staging area (columns of absent tokens must read as 0) and the sums
-        const int nslots_max = p.max_slots;
-        uint4* z4 = reinterpret_cast<uint4*>(smem + sm.xs);
-        for (int i = tid; i < nslots_max * 4 * NT * 16; i += kThreads) z4[i] = make_uint4(0, 0, 0, 0);
-        float* sx = reinterpret_cast<float*>(smem + sm.sx);
-        for (int i = tid; i < ng * 8 * NT; i += kThreads) sx[i] = 0.f;
-    }
-    __syncthreads();
-    {
-        const uint16_t* xslot = reinterpret_cast<const uint16_t*>(smem + sm.xslot);
-        const int* sexp = reinterpret_cast<const int*>(smem + sm.sexp);
-        const __half* xraw = reinterpret_cast<const __half*>(smem + sm.xraw);
-        // one item = (token m, local group i, column kk): split x into 4 e5m2 pieces and scatter them
-        const int items = M * kr;
-        for (int it = tid; it < items; it += kThreads) {
-            const int m = it / kr, rem = it - m * kr;
-            const int i = rem >> 7, kk = rem & 127;
-            const int b = p.gt.bits[g0 + i];
-            const float xf = __half2float(xraw[static_cast<size_t>(m) * kr + rem]);
-            const int S = sexp[m];
-            const int nt = m >> 1, colbase = 4 * (m & 1);
-            const int cc = kk >> 5, r32 = kk & 31;
-            const int ns = slice_count(b);
-            for (int s = 0; s < ns; ++s) {
-                const int w = slice_w(b, s), lo = slice_lo(b, s);
-                const int nf = 32 / w, per_byte = 8 / w;
-                const int u = r32 / nf, f = r32 % nf;
-                const int bt = f / per_byte, pp = f % per_byte;
-                const int mi = u * (4 / w) + (pp >> 1), reg = pp & 1;
-                const int e = S + lo - field_pos(w, pp);
-                float v = xf * __int_as_float((127 + e) << 23);
-                uint8_t* dst = smem + sm.xs + ((static_cast<size_t>(xslot[i] + s) * 4 + mi) * NT + nt) * 256 + reg * 4 + bt;
-#pragma unroll
-                for (int pc = 0; pc < 4; ++pc) {
-                    const float piece = __uint_as_float(__float_as_uint(v) & 0xffe00000u);  // top 3 significant bits
-                    v -= piece;                                                           // exact
-                    const uint16_t hb = __half_as_ushort(__float2half_rz(piece));
-                    dst[((colbase + pc) * 4 + cc) * 8] = static_cast<uint8_t>(hb >> 8);   // e5m2 = high byte of fp16
+    // weights, scales and zeros of this warp's items of chunk `ch` -> buffer ch & 1
+    auto issue_weights = [&](int ch) {
+        if (active && ch < n_chunks) {
+            const int ja = g0 + ch * GC, jb = min(g1, ja + GC);
+            const uint32_t buf = sbase + sm.wbuf + (ch & 1) * p.region_bytes;
+            for (int j = ja + kw; j < jb; j += KW) {
+                const int b = p.gt.bits[j];
+                const uint32_t dst = item_addr(buf, ja, j, b);
+                const uint8_t* src = p.packed + 16ull * N * p.gt.prefix[j] + static_cast<size_t>(tile) * 256 * b;
+                if (lane < 16 * b) cp_async16(dst + 16 * lane, src + 16 * lane);
+                if (lane + 32 < 16 * b) cp_async16(dst + 16 * (lane + 32), src + 16 * (lane + 32));
+                if (lane < 4) {
+                    const __half* sz = (lane < 2 ? p.scales : p.zeros) + static_cast<size_t>(j) * N + 16 * tile + 8 * (lane & 1);
+                    cp_async16(dst + 256 * b + 16 * lane, sz);
                 }
             }
         }
-        // per (token, group): 2^(S-9) * sum_k x, 8 lanes per sum, fixed order
-        float* sx = reinterpret_cast<float*>(smem + sm.sx);
-        const int sums = M * ng;
-        for (int qb = warp * 4; qb < sums; qb += kThreads / 8) {     // warp-uniform trip count
-            const int q = qb + (lane >> 3), l8 = lane & 7;
-            const bool valid = q < sums;
-            const int m = valid ? q / ng : 0, i = valid ? q - m * ng : 0;
-            const __half* src = xraw + static_cast<size_t>(m) * kr + i * SLIM_GROUP + 16 * l8;
-            float acc = 0.f;
-#pragma unroll
-            for (int k = 0; k < 16; ++k) acc += __half2float(src[k]);
-            acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-            acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-            acc += __shfl_xor_sync(0xffffffffu, acc, 4);
-            if (valid && l8 == 0) sx[i * 8 * NT + (m >> 1) * 8 + 4 * (m & 1)] = acc * __int_as_float((127 + sexp[m] - 9) << 23);
+        cp_async_commit();
+    };
+    // raw activations of chunk `ch` (all tokens) -> xraw buffer ch & 1
+    auto issue_x = [&](int ch) {
+        if (ch < n_chunks) {
+            const int ja = g0 + ch * GC, cg = min(g1, ja + GC) - ja;
+            const int per_tok = cg * 16;                                   // 16-byte pieces per token
+            const uint32_t dst0 = sbase + sm.xraw + (ch & 1) * xraw_stride;
+            for (int m = 0; m < M; ++m)
+                for (int q = tid; q < per_tok; q += nthreads)
+                    cp_async16(dst0 + (m * GC * SLIM_GROUP + 8 * q) * 2, p.x + static_cast<size_t>(m) * p.K + ja * SLIM_GROUP + 8 * q);
         }
-    }
-    __syncthreads();
+        cp_async_commit();
+    };
 
-    // ---- main loop ------------------------------------------------------------------------------
-    float acc[T][NT][4];
-#pragma unroll
-    for (int t = 0; t < T; ++t)
-#pragma unroll
-        for (int n = 0; n < NT; ++n)
-#pragma unroll
-            for (int r = 0; r < 4; ++r) acc[t][n][r] = 0.f;
+    // ---- put the first chunk in flight --------------------------------------------------------------
+    issue_weights(0);
+    // Let the next kernel begin its own copies, then wait until the previous kernel has finished
+    // before x or y are touched.
+    pdl_launch_dependents();
+    pdl_wait();
+    issue_x(0);
 
-    bool timed_out = false;
-    int consumed = 0;   // chunks whose barrier phase has been observed
-    if (active) {
-        const uint16_t* xslot = reinterpret_cast<const uint16_t*>(smem + sm.xslot);
-        constexpr bool kCacheB = (NT <= 2);
-        for (int it = 0; it < ng; ++it) {
-            const int st = it % p.nstage;
-            if (!mbar_wait_bounded(my_bar + st * 8, (it / p.nstage) & 1)) { timed_out = true; break; }
-            consumed = it + 1;
-            const int b = p.gt.bits[g0 + it];
-            const uint32_t stage = my_ring + st * p.stage_bytes;
-            const uint32_t xs_slot0 = sbase + sm.xs + static_cast<uint32_t>(xslot[it]) * 4 * NT * 256;
+    uint32_t* smax = reinterpret_cast<uint32_t*>(smem + sm.smax);
+    if (tid < 32) smax[tid] = 0;
+    for (int i = tid; i < 16 * GC; i += nthreads) reinterpret_cast<float*>(smem + sm.sx)[i] = 0.f;   // absent tokens read 0
+    // per-token exponent S of a chunk: max|x| * 2^S lies in [2^13, 2^14) (Inf/NaN: the top binade)
+    auto token_exp = [&](int ch, int m) -> int {
+        const uint32_t mx = smax[(ch & 1) * 16 + m];
+        return mx == 0 ? 0 : 28 - max(static_cast<int>(mx >> 10), 1);
+    };
 
-            float d[T][NT][4];
+    float accf[NT][4];
 #pragma unroll
-            for (int t = 0; t < T; ++t)
+    for (int n = 0; n < NT; ++n)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) accf[n][r] = 0.f;
+
+    for (int ch = 0; ch < n_chunks; ++ch) {
+        const int ja = g0 + ch * GC, cg = min(g1, ja + GC) - ja;
+        const int kc = GC * SLIM_GROUP;                                   // xraw row stride (halves)
+        const __half* xraw = reinterpret_cast<const __half*>(smem + sm.xraw + (ch & 1) * xraw_stride);
+        uint16_t* xslot = reinterpret_cast<uint16_t*>(smem + sm.xslot);
+
+        cp_async_wait_all();             // x and weights of this chunk have landed (this thread's copies)
+        __syncthreads();                 // ... everybody's; and the previous chunk is fully consumed
+        issue_weights(ch + 1);           // into the buffer the previous chunk has left
+        // ---- per-token max |x| of the chunk, slot table ---------------------------------------------
+        {
+            const int per_tok = cg * 16;
+            for (int m = 0; m < M; ++m) {
+                uint32_t mx = 0;
+                for (int q = tid; q < per_tok; q += nthreads) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(xraw + m * kc + 8 * q);
+                    const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) mx = max(mx, max(wv[t] & 0x7fffu, (wv[t] >> 16) & 0x7fffu));
+                }
+                mx = __reduce_max_sync(0xffffffffu, mx);
+                if (lane == 0 && mx != 0) atomicMax(smax + (ch & 1) * 16 + m, mx);
+            }
+            if (tid == nthreads - 1) {
+                int slot = 0;
+                for (int i = 0; i < cg; ++i) { xslot[i] = static_cast<uint16_t>(slot); slot += slice_count(p.gt.bits[ja + i]); }
+                xslot[cg] = static_cast<uint16_t>(slot);
+            }
+            if (tid < 16) smax[((ch + 1) & 1) * 16 + tid] = 0;        // for the next chunk
+        }
+        __syncthreads();
+        // ---- activations in B-fragment order; group sums -----------------------------------------------
+        {
+            // One task = (group i, slice s, mma mi, lane column cc) of a token: the four activations that
+            // meet one lane's two B registers.
+            float* sx = reinterpret_cast<float*>(smem + sm.sx);
+            for (int m = 0; m < M; ++m) {
+                const int S = token_exp(ch, m);
+                for (int t = tid; t < cg * 64; t += nthreads) {
+                    const int cc = t & 3, mi = (t >> 2) & 7, s = (t >> 5) & 1, i = t >> 6;
+                    const int b = p.gt.bits[ja + i];
+                    if (s >= slice_count(b)) continue;
+                    const int w = slice_w(b, s), lo = slice_lo(b, s);
+                    const int lg = w >> 1;                          // log2(w) for w in {1,2,4}
+                    const int nf = 32 >> lg;                        // fields per word; 8/w MMAs per unit
+                    const int u = mi >> (3 - lg), ii = mi & ((8 >> lg) - 1);
+                    const __half* xg = xraw + m * kc + i * SLIM_GROUP + 32 * cc + nf * u + 2 * ii;
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(xg));               // pairs 2ii, 2ii+1: first field
+                    const float2 g = __half22float2(*reinterpret_cast<const __half2*>(xg + (nf >> 1)));   // ... second field
+                    const float sc0 = __int_as_float((127 + S + lo - pair_pos(w, 2 * ii)) << 23);
+                    const float sc1 = __int_as_float((127 + S + lo - pair_pos(w, 2 * ii + 1)) << 23);
+                    const __half2 b0 = __floats2half2_rn(f.x * sc0, g.x * sc0);
+                    const __half2 b1 = __floats2half2_rn(f.y * sc1, g.y * sc1);
+                    *reinterpret_cast<uint2*>(smem + sm.xs + (((static_cast<size_t>(xslot[i] + s) * 8 + mi) * M + m) * 4 + cc) * 8) =
+                        make_uint2(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1));
+                }
+                // per group: 2^(S-24) * sum_k x; 8 lanes per sum, fixed order
+                for (int qb = warp * 4; qb < cg; qb += nthreads / 8) {       // warp-uniform trip count
+                    const int i = qb + (lane >> 3), l8 = lane & 7;
+                    float acc = 0.f;
+                    if (i < cg) {
+                        const __half* src = xraw + m * kc + i * SLIM_GROUP + 16 * l8;
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) acc += __half2float(src[k]);
+                    }
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+                    if (i < cg && l8 == 0) sx[i * 16 + m] = acc * __int_as_float((127 + S - 24) << 23);
+                }
+            }
+        }
+        issue_x(ch + 1);
+        __syncthreads();
+
+        // ---- this warp's tile against its groups of the chunk --------------------------------------------
+        if (active) {
+            float acc[NT][4];
+#pragma unroll
+            for (int n = 0; n < NT; ++n)
+#pragma unroll
+                for (int r = 0; r < 4; ++r) acc[n][r] = 0.f;
+            const uint32_t buf = sbase + sm.wbuf + (ch & 1) * p.region_bytes;
+            for (int it = kw; it < cg; it += KW) {
+                const int b = p.gt.bits[ja + it];
+                const uint32_t item = item_addr(buf, ja, ja + it, b);
+                const uint32_t xs_slot0 = sbase + sm.xs + static_cast<uint32_t>(xslot[it]) * 8 * M * 32;
+
+                float d[NT][4];
 #pragma unroll
                 for (int n = 0; n < NT; ++n)
 #pragma unroll
-                    for (int r = 0; r < 4; ++r) d[t][n][r] = 0.f;
+                    for (int r = 0; r < 4; ++r) d[n][r] = 0.f;
 
-            // one slice of width W starting at unit `unit0`, activations in staging slot `xs_slot`
-            auto run_slice = [&](auto wtag, int unit0, uint32_t xs_slot) {
-                constexpr int W = decltype(wtag)::value;
-                constexpr int MPU = 4 / W;                  // MMAs per unit
-                uint2 bf[kCacheB ? 4 : 1][kCacheB ? NT : 1];
-                if constexpr (kCacheB) {
+                // one slice of width WD starting at unit `unit0`, activations in staging slot `xs_slot`
+                auto run_slice = [&](auto wtag, int unit0, uint32_t xs_slot) {
+                    constexpr int WD = decltype(wtag)::value;
+                    constexpr int MPU = 8 / WD;                 // MMAs per unit
 #pragma unroll
-                    for (int mi = 0; mi < 4; ++mi)
+                    for (int u = 0; u < WD; ++u) {
+                        const uint2 wd = lds64(item + 256 * (unit0 + u) + 8 * lane);
+                        const uint32_t shx = wd.x >> pair_shift(WD), shy = wd.y >> pair_shift(WD);
 #pragma unroll
-                        for (int n = 0; n < NT; ++n) bf[mi][n] = lds64(xs_slot + ((mi * NT + n) * 32 + lane) * 8);
-                }
+                        for (int ii = 0; ii < MPU; ++ii) {
+                            const uint32_t a0 = pair<WD>(wd.x, shx, 2 * ii), a1 = pair<WD>(wd.y, shy, 2 * ii);
+                            const uint32_t a2 = pair<WD>(wd.x, shx, 2 * ii + 1), a3 = pair<WD>(wd.y, shy, 2 * ii + 1);
+                            const int mi = u * MPU + ii;
 #pragma unroll
-                for (int t = 0; t < T; ++t) {
-                    if (t < tw) {
-#pragma unroll
-                        for (int u = 0; u < W; ++u) {
-                            const uint2 wd = lds64(stage + t * 256 * b + 256 * (unit0 + u) + 8 * lane);
-                            const uint32_t sha = wd.x >> 4, shb = wd.y >> 4;
-#pragma unroll
-                            for (int ii = 0; ii < MPU; ++ii) {
-                                const uint32_t a0 = field<W>(wd.x, sha, 2 * ii), a1 = field<W>(wd.y, shb, 2 * ii);
-                                const uint32_t a2 = field<W>(wd.x, sha, 2 * ii + 1), a3 = field<W>(wd.y, shb, 2 * ii + 1);
-                                const int mi = u * MPU + ii;
-#pragma unroll
-                                for (int n = 0; n < NT; ++n) {
-                                    const uint2 bv = kCacheB ? bf[kCacheB ? mi : 0][kCacheB ? n : 0]
-                                                             : lds64(xs_slot + ((mi * NT + n) * 32 + lane) * 8);
-                                    mma_e4m3_e5m2(d[t][n], a0, a1, a2, a3, bv);
-                                }
+                            for (int n = 0; n < NT; ++n) {
+                                const int m = 8 * n + gq;
+                                uint2 bv = make_uint2(0u, 0u);
+                                if (m < M) bv = lds64(xs_slot + ((mi * M + m) * 4 + c) * 8);
+                                mma_f16(d[n], a0, a1, a2, a3, bv);
                             }
                         }
                     }
+                };
+                switch (b) {
+                    case 1: run_slice(W1{}, 0, xs_slot0); break;
+                    case 2: run_slice(W2{}, 0, xs_slot0); break;
+                    case 3: run_slice(W2{}, 0, xs_slot0); run_slice(W1{}, 2, xs_slot0 + 8 * M * 32); break;
+                    default: run_slice(W4{}, 0, xs_slot0); break;
                 }
-            };
-            switch (b) {
-                case 1: run_slice(W1{}, 0, xs_slot0); break;
-                case 2: run_slice(W2{}, 0, xs_slot0); break;
-                case 3: run_slice(W2{}, 0, xs_slot0); run_slice(W1{}, 2, xs_slot0 + 4 * NT * 256); break;
-                default: run_slice(W4{}, 0, xs_slot0); break;
-            }
 
-            // fold the group: acc += s * (D - z * sum_x)
-            const uint32_t sxa = sbase + sm.sx + (it * 8 * NT + 2 * c) * 4;
+                // fold the group: acc += s * (D - z * sum_x); rows 2gq, 2gq+1, tokens 8n+2c, 8n+2c+1
+                const uint32_t s2 = lds32(item + 256 * b + gq * 4);
+                const uint32_t z2 = lds32(item + 256 * b + 32 + gq * 4);
+                const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
+                const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
+                const uint32_t sxa = sbase + sm.sx + (it * 16 + 2 * c) * 4;
 #pragma unroll
-            for (int t = 0; t < T; ++t) {
-                if (t < tw) {
-                    const uint32_t s2 = lds32(stage + p.w_stage_bytes + t * 32 + gq * 4);
-                    const uint32_t z2 = lds32(stage + p.w_stage_bytes + T * 32 + t * 32 + gq * 4);
-                    const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
-                    const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
-#pragma unroll
-                    for (int n = 0; n < NT; ++n) {
-                        const uint2 sxr = lds64(sxa + n * 32);
-                        const float sx0 = __uint_as_float(sxr.x), sx1 = __uint_as_float(sxr.y);
-                        acc[t][n][0] = fmaf(sf.x, fmaf(-zf.x, sx0, d[t][n][0]), acc[t][n][0]);
-                        acc[t][n][1] = fmaf(sf.x, fmaf(-zf.x, sx1, d[t][n][1]), acc[t][n][1]);
-                        acc[t][n][2] = fmaf(sf.y, fmaf(-zf.y, sx0, d[t][n][2]), acc[t][n][2]);
-                        acc[t][n][3] = fmaf(sf.y, fmaf(-zf.y, sx1, d[t][n][3]), acc[t][n][3]);
-                    }
+                for (int n = 0; n < NT; ++n) {
+                    const uint2 sxr = lds64(sxa + n * 32);
+                    const float sx0 = __uint_as_float(sxr.x), sx1 = __uint_as_float(sxr.y);
+                    acc[n][0] = fmaf(sf.x, fmaf(-zf.x, sx0, d[n][0]), acc[n][0]);
+                    acc[n][1] = fmaf(sf.x, fmaf(-zf.x, sx1, d[n][1]), acc[n][1]);
+                    acc[n][2] = fmaf(sf.y, fmaf(-zf.y, sx0, d[n][2]), acc[n][2]);
+                    acc[n][3] = fmaf(sf.y, fmaf(-zf.y, sx1, d[n][3]), acc[n][3]);
                 }
             }
-            // the stage is free again: refill it with the chunk nstage groups ahead
-            __syncwarp();
-            if (lane == 0 && it + p.nstage < ng) {
-                fence_proxy_async();
-                issue_chunk(it + p.nstage);
+            // undo the chunk's activation scaling
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+                const int m0 = 8 * n + 2 * c;
+                const float back0 = m0 < M ? __int_as_float((127 + 24 - token_exp(ch, m0)) << 23) : 0.f;
+                const float back1 = m0 + 1 < M ? __int_as_float((127 + 24 - token_exp(ch, m0 + 1)) << 23) : 0.f;
+                accf[n][0] = fmaf(acc[n][0], back0, accf[n][0]);
+                accf[n][1] = fmaf(acc[n][1], back1, accf[n][1]);
+                accf[n][2] = fmaf(acc[n][2], back0, accf[n][2]);
+                accf[n][3] = fmaf(acc[n][3], back1, accf[n][3]);
             }
-        }
-        if (timed_out) {
-            // leave nothing in flight: every issued chunk either lands or its wait runs out as well
-            if (lane == 0) {
-                atomicOr(p.status, 1u);
-                const int issued = min(ng, consumed + p.nstage);
-                for (int it = consumed; it < issued; ++it)
-                    (void)mbar_wait_bounded(my_bar + (it % p.nstage) * 8, (it / p.nstage) & 1);
-            }
-            __syncwarp();
         }
     }
 
-    // ---- combine the piece columns of each token, scale back, write -------------------------------
-    const int* sexp = reinterpret_cast<const int*>(smem + sm.sexp);
-    const bool direct = (p.SK == 1);
+    // ---- add the partial sums of the warps that share a tile (fixed order) ---------------------------
+    float* red = reinterpret_cast<float*>(smem + sm.red);      // [W][M][16], warp = kw * T + tw
 #pragma unroll
-    for (int t = 0; t < T; ++t) {
-#pragma unroll
-        for (int n = 0; n < NT; ++n) {
-            float va = acc[t][n][0] + acc[t][n][1];    // row 2gq,   columns 2c, 2c+1
-            float vb = acc[t][n][2] + acc[t][n][3];    // row 2gq+1
-            va += __shfl_xor_sync(0xffffffffu, va, 1);
-            vb += __shfl_xor_sync(0xffffffffu, vb, 1);
-            const int m = 2 * n + (c >> 1);
-            if (active && t < tw && (c & 1) == 0 && m < M) {
-                const float back = __int_as_float((127 + 9 - sexp[m]) << 23);
-                va *= back;
-                vb *= back;
-                const int row = 16 * (tile0 + t) + 2 * gq;
-                if (direct) {
-                    *reinterpret_cast<__half2*>(p.y + static_cast<size_t>(m) * N + row) = __floats2half2_rn(va, vb);
-                } else {
-                    *reinterpret_cast<float2*>(p.partials + (static_cast<size_t>(ks) * M + m) * N + row) = make_float2(va, vb);
-                }
-            }
+    for (int n = 0; n < NT; ++n) {
+        const int m0 = 8 * n + 2 * c;
+        if (m0 < M) *reinterpret_cast<float2*>(red + (warp * M + m0) * 16 + 2 * gq) = make_float2(accf[n][0], accf[n][2]);
+        if (m0 + 1 < M) *reinterpret_cast<float2*>(red + (warp * M + m0 + 1) * 16 + 2 * gq) = make_float2(accf[n][1], accf[n][3]);
+    }
+    __syncthreads();
+    const bool direct = (p.CS == 1);
+    const int pairs = T * M * 8;                                // e = (tile of the CTA, token, row pair)
+    auto out_ptr = [&](int e) -> __half2* {
+        const int t = e / (M * 8), rem = e - t * (M * 8);
+        const int row = 16 * (rb * T + t) + 2 * (rem & 7);
+        return row < N ? reinterpret_cast<__half2*>(p.y + static_cast<size_t>(rem >> 3) * N + row) : nullptr;
+    };
+    for (int e = tid; e < pairs; e += nthreads) {
+        float2 sum = make_float2(0.f, 0.f);
+        for (int k = 0; k < KW; ++k) {
+            const float2 v = *reinterpret_cast<const float2*>(red + k * T * M * 16 + 2 * e);
+            sum.x += v.x;
+            sum.y += v.y;
+        }
+        if (direct) {
+            __half2* dst = out_ptr(e);
+            if (dst != nullptr) *dst = __floats2half2_rn(sum.x, sum.y);
+        } else {
+            *reinterpret_cast<float2*>(red + 2 * e) = sum;      // CTA partial in place of k-way 0 (read by this thread only)
         }
     }
     if (direct) return;
 
-    // ---- split-K: the last CTA of this row block adds the partials in split order ------------------
-    __shared__ unsigned int s_ticket;
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_ticket = atomicAdd(p.counters + rb, 1u);
-    __syncthreads();
-    if (s_ticket != static_cast<unsigned int>(p.SK - 1)) return;
-    __threadfence();
-    const int row0 = rb * kWarps * T * 16;
-    const int nrows = min(kWarps * T * 16, N - row0);
-    for (int i = tid; i < M * (nrows / 2); i += kThreads) {
-        const int m = i / (nrows / 2), r2 = i - m * (nrows / 2);
-        const size_t off = static_cast<size_t>(m) * N + row0 + 2 * r2;
-        float2 sum = make_float2(0.f, 0.f);
-        for (int s = 0; s < p.SK; ++s) {
-            const float2 v = __ldcg(reinterpret_cast<const float2*>(p.partials + static_cast<size_t>(s) * M * N + off));
-            sum.x += v.x;
-            sum.y += v.y;
+    // ---- split-K: add the partials of the cluster's CTAs in rank order ------------------------------
+    cluster_sync_all();
+    {
+        const uint32_t rank = cluster_ctarank();
+        const int share = (pairs + p.CS - 1) / p.CS;
+        const int e1 = min(pairs, static_cast<int>(rank + 1) * share);
+        for (int e = rank * share + tid; e < e1; e += nthreads) {
+            const uint32_t addr = sbase + sm.red + 8 * e;
+            float2 sum = make_float2(0.f, 0.f);
+            for (int s = 0; s < p.CS; ++s) {
+                const float2 v = ld_cluster_f32x2(addr, s);
+                sum.x += v.x;
+                sum.y += v.y;
+            }
+            __half2* dst = out_ptr(e);
+            if (dst != nullptr) *dst = __floats2half2_rn(sum.x, sum.y);
         }
-        *reinterpret_cast<__half2*>(p.y + off) = __floats2half2_rn(sum.x, sum.y);
     }
-    if (tid == 0) p.counters[rb] = 0;   // leave the counter ready for the next call
+    cluster_sync_all();   // nobody leaves while a peer may still read its partials
 }
 
 // ------------------------------------------------------------------------------------------ host side
 struct GemvPlan {
-    int NT, T, SK, RB;
-    int nstage, stage_bytes, w_stage_bytes;
-    int max_groups, max_slots;
+    int NT, W, T, CS, GC;
+    int region_bytes, max_groups, max_slots;
+    bool two_bufs;
     uint32_t smem_bytes;
-    uint16_t kbegin[kMaxSplit + 1];
-    size_t counters_bytes, partial_bytes;
+    uint16_t kbegin[kMaxCluster + 1];
 };
 
 static int device_sm_count() {
@@ -487,89 +460,107 @@ static int device_sm_count() {
     return cached[dev];
 }
 
-// Deterministic launch plan for (M, N, K, bit map) on the current device.
-static void plan_gemv(int M, int N, const GroupTable& gt, GemvPlan* pl) {
+// k-slice boundaries at the groups where the running bit count crosses i/cs of the total.
+static void split_groups(const GroupTable& gt, int cs, GemvPlan* pl) {
     const int G = gt.G;
-    const int need_nt = (M + 1) / 2;
-    pl->NT = need_nt <= 1 ? 1 : need_nt <= 2 ? 2 : need_nt <= 4 ? 4 : 8;
-    pl->T = pl->NT <= 2 ? 2 : 1;
-    const int rows_per_cta = kWarps * pl->T * 16;
-    pl->RB = (N + rows_per_cta - 1) / rows_per_cta;
-    int bmax = 1;
-    for (int j = 0; j < G; ++j) bmax = bmax > gt.bits[j] ? bmax : gt.bits[j];
-    pl->w_stage_bytes = pl->T * 256 * bmax;
-    pl->stage_bytes = static_cast<int>(align_up(pl->w_stage_bytes + 2 * pl->T * 32, 128));
-
-    const int sms = device_sm_count();
-    int sk = sms / (pl->RB > 0 ? pl->RB : 1);
-    if (sk < 1) sk = 1;
-    if (sk > G) sk = G;
-    if (sk > kMaxSplit) sk = kMaxSplit;
-    const uint32_t smem_budget = 100 * 1024;   // two CTAs per SM: the next layer's CTA co-resides
-    for (;; ++sk) {
-        // boundaries at the group where the running bit count crosses i/sk of the total
-        const int total = gt.prefix[G];
-        pl->kbegin[0] = 0;
-        int j = 0;
-        for (int i = 1; i < sk; ++i) {
-            const int target = (total * i + sk / 2) / sk;
-            while (j < G && gt.prefix[j] < target) ++j;
-            if (j <= pl->kbegin[i - 1]) j = pl->kbegin[i - 1] + 1;   // every split gets at least one group
-            if (j > G - (sk - i)) j = G - (sk - i);
-            pl->kbegin[i] = static_cast<uint16_t>(j);
-        }
-        pl->kbegin[sk] = static_cast<uint16_t>(G);
-        int mg = 0, ms = 0;
-        for (int i = 0; i < sk; ++i) {
-            const int a = pl->kbegin[i], b = pl->kbegin[i + 1];
-            int slots = 0;
-            for (int q = a; q < b; ++q) slots += slice_count(gt.bits[q]);
-            mg = mg > (b - a) ? mg : (b - a);
-            ms = ms > slots ? ms : slots;
-        }
-        pl->max_groups = mg;
-        pl->max_slots = ms;
-        const SmemMap fixed = make_smem_map(pl->NT, M, 0, 0, mg, ms);
-        const uint32_t ring_min = static_cast<uint32_t>(kWarps) * 2 * pl->stage_bytes;
-        if (fixed.total + ring_min <= smem_budget || sk >= G || sk >= kMaxSplit) {
-            const uint32_t avail = smem_budget > fixed.total ? smem_budget - fixed.total : 0;
-            int ns = static_cast<int>(avail / (static_cast<uint32_t>(kWarps) * pl->stage_bytes));
-            if (ns > kMaxStages) ns = kMaxStages;
-            if (ns > mg) ns = mg;
-            if (ns < 2) ns = mg < 2 ? 1 : 2;
-            pl->nstage = ns;
-            pl->smem_bytes = make_smem_map(pl->NT, M, ns, pl->stage_bytes, mg, ms).total;
-            break;
-        }
+    const int total = gt.prefix[G];
+    pl->kbegin[0] = 0;
+    int j = 0;
+    for (int i = 1; i < cs; ++i) {
+        const int target = (total * i + cs / 2) / cs;
+        while (j < G && gt.prefix[j] < target) ++j;
+        if (j <= pl->kbegin[i - 1]) j = pl->kbegin[i - 1] + 1;   // every slice gets at least one group
+        if (j > G - (cs - i)) j = G - (cs - i);
+        pl->kbegin[i] = static_cast<uint16_t>(j);
     }
-    pl->SK = sk;
-    pl->counters_bytes = align_up(4u * static_cast<uint32_t>(N / 128 + 1), 256);
-    pl->partial_bytes = sk > 1 ? static_cast<size_t>(sk) * M * N * sizeof(float) : 0;
+    pl->kbegin[cs] = static_cast<uint16_t>(G);
+    int mg = 0;
+    for (int i = 0; i < cs; ++i) mg = mg > (pl->kbegin[i + 1] - pl->kbegin[i]) ? mg : (pl->kbegin[i + 1] - pl->kbegin[i]);
+    pl->max_groups = mg;
+    pl->CS = cs;
 }
 
-template <int NT, int T>
+// Sizes that depend on the chunk length: the largest chunk in bytes and in slices.
+static void size_chunks(const GroupTable& gt, int gc, GemvPlan* pl) {
+    int ms = 0, mb = 0;
+    for (int i = 0; i < pl->CS; ++i)
+        for (int a = pl->kbegin[i]; a < pl->kbegin[i + 1]; a += gc) {
+            const int b = a + gc < pl->kbegin[i + 1] ? a + gc : pl->kbegin[i + 1];
+            int slots = 0;
+            for (int q = a; q < b; ++q) slots += slice_count(gt.bits[q]);
+            const int bytes = 256 * (gt.prefix[b] - gt.prefix[a]) + 64 * (b - a);
+            ms = ms > slots ? ms : slots;
+            mb = mb > bytes ? mb : bytes;
+        }
+    pl->GC = gc;
+    pl->max_slots = ms;
+    pl->region_bytes = mb * pl->T;
+    pl->two_bufs = pl->max_groups > gc;
+}
+
+// Deterministic launch plan for (M, N, K, bit map) on the current device.  x is staged once per
+// CTA, so a CTA takes as many tiles (up to 8, one per warp) as still leaves two CTAs per SM; the
+// k-range is cut so that a warp sees about four groups (its instruction stream is the critical
+// path) and further while the grid is smaller than two CTAs per SM; chunks
+// are as long as shared memory allows while CTAs of consecutive layers can still share an SM.
+// Returns false if a single group does not fit (cannot happen within the documented limits).
+static bool plan_gemv(int M, int N, const GroupTable& gt, GemvPlan* pl) {
+    const int G = gt.G;
+    pl->NT = M <= 8 ? 1 : 2;
+    pl->W = kMaxWarps;
+    const int sms = device_sm_count();
+    const int tiles = N / 16;
+    const int cs_max = G < kMaxCluster ? G : kMaxCluster;
+    int T = kMaxWarps;
+    while (T > 1 && ((tiles + T - 1) / T) * cs_max < 2 * sms) T >>= 1;
+    pl->T = T;
+    const int rb = (tiles + T - 1) / T;
+    int cs = (G * T / kMaxWarps + 3) / 4;
+    if (cs < 1) cs = 1;
+    if (cs > cs_max) cs = cs_max;
+    while (cs < cs_max && rb * cs < 2 * sms) ++cs;
+    split_groups(gt, cs, pl);
+    // up to two chunks under 48 KB if possible, else the fewest chunks under 100 KB (two CTAs
+    // per SM), else whatever fits
+    const uint32_t budgets[3] = {48 * 1024, 100 * 1024, 220 * 1024};
+    for (int bi = 0; bi < 3; ++bi)
+        for (int nc = 1; nc <= (bi == 0 && pl->max_groups > 2 ? 2 : pl->max_groups); ++nc) {
+            size_chunks(gt, (pl->max_groups + nc - 1) / nc, pl);
+            const uint32_t need = make_smem_map(M, pl->W, pl->GC, pl->region_bytes, pl->max_slots, pl->two_bufs).total;
+            if (need > budgets[bi]) continue;
+            pl->smem_bytes = need;
+            return true;
+        }
+    return false;
+}
+
+template <int NT>
 static cudaError_t launch_gemv(const GemvParams& prm, const GemvPlan& pl, cudaStream_t stream) {
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        e = cudaFuncSetAttribute(gemv_kernel<NT, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        e = cudaFuncSetAttribute(gemv_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(static_cast<unsigned>(pl.RB), static_cast<unsigned>(pl.SK), 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.gridDim = dim3(static_cast<unsigned>(pl.CS), static_cast<unsigned>((prm.N / 16 + pl.T - 1) / pl.T), 1);
+    cfg.blockDim = dim3(static_cast<unsigned>(pl.W * 32), 1, 1);
     cfg.dynamicSmemBytes = pl.smem_bytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = static_cast<unsigned>(pl.CS);
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_kernel<NT, T>, prm);
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, gemv_kernel<NT>, prm);
 }
 
 }  // namespace slim
@@ -581,20 +572,26 @@ int slim_workspace_bytes(int M, int N, int K, int g, const uint8_t* bits_host, s
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;
-    size_t bytes = slim::kWsHeader + slim::align_up(4u * static_cast<uint32_t>(N / 128 + 1), 256);
-    if (M >= 1 && M <= SLIM_GEMV_MAX_M && N > 0 && K > 0) {
-        slim::GemvPlan pl;
-        slim::plan_gemv(M, N, gt, &pl);
-        bytes += pl.partial_bytes;
-    }
-    *out_bytes = bytes;
+    *out_bytes = slim::kWsHeader;
+    return SLIM_OK;
+}
+
+int slim_gemv_plan(int M, int N, int K, int g, const uint8_t* bits_host, int* out6) {
+    if (out6 == nullptr || M < 1 || M > SLIM_GEMV_MAX_M) return SLIM_ERR_INVALID_ARG;
+    slim::GroupTable gt;
+    const int st = slim::make_group_table(N, K, g, bits_host, &gt);
+    if (st != SLIM_OK) return st;
+    if (N == 0 || K == 0) return SLIM_ERR_INVALID_ARG;
+    slim::GemvPlan pl;
+    if (!slim::plan_gemv(M, N, gt, &pl)) return SLIM_ERR_UNSUPPORTED;
+    out6[0] = pl.T; out6[1] = pl.CS; out6[2] = (N / 16 + pl.T - 1) / pl.T; out6[3] = static_cast<int>(pl.smem_bytes);
+    out6[4] = pl.NT; out6[5] = pl.GC;
     return SLIM_OK;
 }
 
 int slim_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
     if (workspace == nullptr || workspace_bytes < slim::kWsHeader) return SLIM_ERR_WORKSPACE;
     if (!slim::aligned16(workspace)) return SLIM_ERR_ALIGNMENT;
-    // control region = header + counters; zeroing the whole workspace is simplest and always safe
     SLIM_CUDA_TRY(cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)));
     return SLIM_OK;
 }
@@ -630,12 +627,11 @@ int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host, c
     if (x == nullptr || packed == nullptr || scales == nullptr || zeros == nullptr) return SLIM_ERR_INVALID_ARG;
     if (!slim::aligned16(x) || !slim::aligned16(packed) || !slim::aligned16(scales) || !slim::aligned16(zeros))
         return SLIM_ERR_ALIGNMENT;
+    if (workspace == nullptr || workspace_bytes < slim::kWsHeader) return SLIM_ERR_WORKSPACE;
+    if (!slim::aligned16(workspace)) return SLIM_ERR_ALIGNMENT;
 
     slim::GemvPlan pl;
-    slim::plan_gemv(M, N, gt, &pl);
-    const size_t need = slim::kWsHeader + pl.counters_bytes + pl.partial_bytes;
-    if (workspace == nullptr || workspace_bytes < need) return SLIM_ERR_WORKSPACE;
-    if (!slim::aligned16(workspace)) return SLIM_ERR_ALIGNMENT;
+    if (!slim::plan_gemv(M, N, gt, &pl)) return SLIM_ERR_UNSUPPORTED;
 
     slim::GemvParams prm;
     memset(&prm, 0, sizeof prm);
@@ -644,25 +640,20 @@ int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host, c
     prm.scales = static_cast<const __half*>(scales);
     prm.zeros = static_cast<const __half*>(zeros);
     prm.y = static_cast<__half*>(y);
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
-    prm.status = reinterpret_cast<unsigned int*>(ws);
-    prm.counters = reinterpret_cast<unsigned int*>(ws + slim::kWsHeader);
-    prm.partials = reinterpret_cast<float*>(ws + slim::kWsHeader + pl.counters_bytes);
     prm.M = M; prm.N = N; prm.K = K;
-    prm.SK = pl.SK;
-    prm.nstage = pl.nstage;
-    prm.stage_bytes = pl.stage_bytes;
-    prm.w_stage_bytes = pl.w_stage_bytes;
-    prm.max_groups = pl.max_groups;
+    prm.CS = pl.CS;
+    prm.W = pl.W;
+    prm.T = pl.T;
+    prm.GC = pl.GC;
+    prm.region_bytes = pl.region_bytes;
     prm.max_slots = pl.max_slots;
+    prm.two_bufs = pl.two_bufs ? 1 : 0;
     memcpy(prm.kbegin, pl.kbegin, sizeof prm.kbegin);
     prm.gt = gt;
 
     cudaError_t e;
-    if (pl.NT == 1) e = slim::launch_gemv<1, 2>(prm, pl, s);
-    else if (pl.NT == 2) e = slim::launch_gemv<2, 2>(prm, pl, s);
-    else if (pl.NT == 4) e = slim::launch_gemv<4, 1>(prm, pl, s);
-    else e = slim::launch_gemv<8, 1>(prm, pl, s);
+    if (pl.NT == 1) e = slim::launch_gemv<1>(prm, pl, s);
+    else e = slim::launch_gemv<2>(prm, pl, s);
     SLIM_CUDA_TRY(e);
     return SLIM_OK;
 }
