@@ -1,7 +1,531 @@
-// slim_mpq_gemm: batched path (M > 16).  Placeholder until the tcgen05 kernel lands.
+// slim_mpq_gemm: batched / prefill path (M > 16) of the mixed-precision linear layer, sm_100a.
+//
+// y^T = W-hat * x^T on the 5th-generation tensor cores.  The weight rows are the M dimension of
+// the MMA (128 per CTA), the tokens its N dimension (TOK = 128 or 256 per tile):
+//
+//  * A operand = dequantised weights, fp16, written by eight dequant warps straight into tensor
+//    memory with tcgen05.st (thread = weight row, 32-bit column = two consecutive k); no shared
+//    memory round trip and no swizzled layout to reproduce.  One stage = one group of 128 k.
+//  * B operand = activations, x[tokens][k], brought by TMA into 128-byte-swizzled K-major shared
+//    memory tiles (two boxes of 64 k per group).
+//  * D = fp32 accumulator in tensor memory, 128 lanes x TOK columns; tcgen05.mma kind::f16 is
+//    issued by one thread, eight K=16 steps per group, and tcgen05.commit hands the stages back.
+//  * Epilogue warps read D with tcgen05.ld and store y as fp16.
+//
+// Dequantisation: a code field is moved to mantissa bits [6,10) of a half whose exponent makes it
+// 16 + q (ulp 1/64); one HSUB2 removes 16 + z exactly for every zero point that is a multiple of
+// 1/64 in [-16, 16) (all integer and half-integer zero points of Eq. 1 / Eq. 2), one HMUL2 applies
+// the scale with a single rounding, so the operand equals the fp16 weight slim_dequant produces.
+// Other zero points are rounded to the nearest 1/64.
+//
+// Warp roles (448 threads): warp 0 producer (TMA + bulk copies of packed slices, scales, zeros),
+// warp 1 MMA issuer and tensor-memory allocator, warps 2-9 dequant, warps 10-13 epilogue.
+// Persistent CTAs walk the (token tile, row block) tiles; every wait on an mbarrier is bounded
+// and reports through the workspace status word instead of spinning forever.
 #include "slim_common.cuh"
 
-extern "C" int slim_mpq_gemm(const void*, const void*, const uint8_t*, const void*, const void*, void*,
-                             int, int, int, int, void*, size_t, void*) {
-    return SLIM_ERR_UNSUPPORTED;
+#include <cuda.h>
+#include <cstring>
+
+namespace slim {
+
+constexpr int kGemmThreads = 448;
+constexpr int kRowsPerCta = 128;
+constexpr int kNA = 4;                      // tensor-memory stages of A (64 columns each)
+constexpr int kNP = 3;                      // shared-memory stages of packed slices
+constexpr int kPStageBytes = 8192 + 512;    // 128 rows x 128 k x 4 bits, + scales + zeros
+constexpr int kTmemCols = 512;
+constexpr int kTmemAcol = 256;              // A stages start here; D occupies [0, TOK)
+constexpr unsigned long long kGemmWaitNs = 2000000000ull;
+
+struct GemmParams {
+    const uint8_t* packed;
+    const __half* scales;
+    const __half* zeros;
+    __half* y;
+    unsigned int* status;
+    int M, N, K;
+    int row_blocks, tok_tiles;
+    GroupTable gt;
+};
+
+// ------------------------------------------------------------------------------------------ PTX helpers
+namespace g {
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Gives up when the limit passes or when another role has raised `abort`.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort != 0) return false;
+        if (global_timer_ns() - t0 > kGemmWaitNs) { *abort = 1; return false; }
+    }
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem descriptor]; fp16 inputs, fp32 accumulate.
+__device__ __forceinline__ void umma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %6, %7, %8}, p;\n}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
+}
+
+// 32 lanes x 32 columns of 32-bit: thread = lane, register j = column j.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
+}  // namespace g
+
+// ------------------------------------------------------------------------------------------ dequantisation
+// Everything below works on one "c-word set": the slice words of one weight row that cover 32
+// consecutive k, and produces the 16 tensor-memory columns (k, k+1 pairs) of those 32 weights.
+constexpr uint32_t kMagic16 = 0x4C004C00u;   // half2(16, 16): ulp 1/64, mantissa bit 6 is 1.0
+
+struct DqRow {
+    __half2 zc;   // (16 + z, 16 + z)
+    __half2 s;    // (s, s)
+};
+// v holds two fields at mantissa bits [6,10) under the exponent of 16: returns s * (q - z) twice.
+__device__ __forceinline__ uint32_t dq_pair(uint32_t v, const DqRow& r) {
+    const __half2 h = __hmul2(__hsub2(*reinterpret_cast<const __half2*>(&v), r.zc), r.s);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ uint32_t lo_halves(uint32_t a, uint32_t b) { return g::prmt(a, b, 0x5410u); }
+__device__ __forceinline__ uint32_t hi_halves(uint32_t a, uint32_t b) { return g::prmt(a, b, 0x7632u); }
+
+// Logical shift, left if s > 0 (s is a constant after unrolling).
+__device__ __forceinline__ uint32_t shift_to(uint32_t v, int s) { return s >= 0 ? v << s : v >> (-s); }
+
+// Fields of width W: F = 16/W pairs (f, f + F) per word; H[f] = (w[k0+f], w[k0+f+F]).  The word
+// covers 2F consecutive k; its F columns are (H[2j].lo, H[2j+1].lo) for j < F/2 and the hi halves
+// for the rest.  If HIGH, X carries a third code bit: bit f of its low/high half belongs to pair f.
+template <int W, int F, bool HIGH>
+__device__ __forceinline__ void decode_word(uint32_t word, uint32_t X, const DqRow& r, uint32_t* cols) {
+    constexpr uint32_t kMask = (0x00010001u * ((1u << W) - 1u)) << 6;
+    uint32_t H[F];
+#pragma unroll
+    for (int f = 0; f < F; ++f) {
+        uint32_t v = (shift_to(word, 6 - W * f) & kMask) | kMagic16;
+        if (HIGH) v |= shift_to(X, 8 - f) & 0x01000100u;
+        H[f] = dq_pair(v, r);
+    }
+#pragma unroll
+    for (int j = 0; j < F / 2; ++j) {
+        cols[j] = lo_halves(H[2 * j], H[2 * j + 1]);
+        cols[F / 2 + j] = hi_halves(H[2 * j], H[2 * j + 1]);
+    }
+}
+
+// words[u] = word of unit u for this row and this 32-k range.  cols[16].
+template <int B>
+__device__ __forceinline__ void decode_cword(const uint32_t (&words)[4], const DqRow& r, uint32_t* cols) {
+    if constexpr (B == 1) {
+        decode_word<1, 16, false>(words[0], 0u, r, cols);
+    } else if constexpr (B == 2) {
+        decode_word<2, 8, false>(words[0], 0u, r, cols);
+        decode_word<2, 8, false>(words[1], 0u, r, cols + 8);
+    } else if constexpr (B == 3) {
+        // the 1-bit slice word holds k = bit index; bytes 2u and 2u+1 line up with the pairs of unit u
+        decode_word<2, 8, true>(words[0], g::prmt(words[2], 0u, 0x4140u), r, cols);
+        decode_word<2, 8, true>(words[1], g::prmt(words[2], 0u, 0x4342u), r, cols + 8);
+    } else {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) decode_word<4, 4, false>(words[u], 0u, r, cols + 4 * u);
+    }
+}
+
+// ------------------------------------------------------------------------------------------ kernel
+template <int TOK> struct GemmCfg {
+    static constexpr int NX = TOK == 256 ? 3 : 4;            // shared-memory stages of x
+    static constexpr int XBOX = TOK * 128;                   // bytes of one TMA box: TOK rows x 64 k
+    static constexpr int XSTAGE = 2 * XBOX;                  // one group: 128 k
+    static constexpr int OFF_P = NX * XSTAGE;
+    static constexpr int OFF_BAR = OFF_P + kNP * kPStageBytes;
+    static constexpr int NBAR = 2 * NX + 2 * kNP + 2 * kNA + 2;
+    static constexpr int OFF_MISC = OFF_BAR + 8 * NBAR;      // tensor-memory base, abort flag
+    static constexpr int SMEM = OFF_MISC + 16 + 1024;        // + slack to align the base to 1024
+};
+
+// Shared-memory matrix descriptor of a K-major, 128-byte-swizzled operand: rows of 128 bytes,
+// groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t sw128_kmajor_desc(uint32_t smem_addr) {
+    return static_cast<uint64_t>((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+template <int TOK>
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ CUtensorMap x_map,
+                                                               const __grid_constant__ GemmParams p) {
+    using C = GemmCfg<TOK>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t sbase = (g::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (sbase - g::smem_u32(smem_raw));
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t bar0 = sbase + C::OFF_BAR;
+    auto x_full = [&](int s) { return bar0 + 8 * s; };
+    auto x_empty = [&](int s) { return bar0 + 8 * (C::NX + s); };
+    auto p_full = [&](int s) { return bar0 + 8 * (2 * C::NX + s); };
+    auto p_empty = [&](int s) { return bar0 + 8 * (2 * C::NX + kNP + s); };
+    auto a_full = [&](int s) { return bar0 + 8 * (2 * C::NX + 2 * kNP + s); };
+    auto a_empty = [&](int s) { return bar0 + 8 * (2 * C::NX + 2 * kNP + kNA + s); };
+    const uint32_t d_full = bar0 + 8 * (2 * C::NX + 2 * kNP + 2 * kNA);
+    const uint32_t d_empty = d_full + 8;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OFF_MISC);
+    volatile int* abort = reinterpret_cast<volatile int*>(smem + C::OFF_MISC + 4);
+
+    if (tid == 0) {
+        for (int s = 0; s < C::NX; ++s) { g::mbar_init(x_full(s), 1); g::mbar_init(x_empty(s), 1); }
+        for (int s = 0; s < kNP; ++s) { g::mbar_init(p_full(s), 1); g::mbar_init(p_empty(s), 8); }
+        for (int s = 0; s < kNA; ++s) { g::mbar_init(a_full(s), 8); g::mbar_init(a_empty(s), 1); }
+        g::mbar_init(d_full, 1);
+        g::mbar_init(d_empty, 4);
+        *abort = 0;
+        g::fence_barrier_init();
+        g::fence_proxy_async();
+    }
+    if (warp == 1) {
+        g::tmem_alloc(g::smem_u32(tmem_slot), kTmemCols);
+        g::tmem_relinquish();
+    }
+    g::tc_fence_before();
+    __syncthreads();
+    g::tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const int G = p.gt.G, N = p.N;
+    const int total_tiles = p.row_blocks * p.tok_tiles;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            int sx = 0, sp = 0;
+            uint32_t phx = 0, php = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int rb = tile % p.row_blocks, mt = tile / p.row_blocks;
+                const int tiles_here = min(8, (N >> 4) - 8 * rb);
+                for (int j = 0; j < G && ok; ++j) {
+                    // activations of the group
+                    if (!g::mbar_wait(x_empty(sx), phx ^ 1u, abort)) { ok = false; break; }
+                    g::mbar_expect_tx(x_full(sx), C::XSTAGE);
+                    g::tma_load_2d(sbase + sx * C::XSTAGE, &x_map, SLIM_GROUP * j, mt * TOK, x_full(sx));
+                    g::tma_load_2d(sbase + sx * C::XSTAGE + C::XBOX, &x_map, SLIM_GROUP * j + 64, mt * TOK, x_full(sx));
+                    if (++sx == C::NX) { sx = 0; phx ^= 1u; }
+                    // packed slices, scales, zeros of the row block
+                    if (!g::mbar_wait(p_empty(sp), php ^ 1u, abort)) { ok = false; break; }
+                    const int b = p.gt.bits[j];
+                    const uint32_t wbytes = static_cast<uint32_t>(tiles_here) * 256u * b, sbytes = static_cast<uint32_t>(tiles_here) * 32u;
+                    const uint32_t dst = sbase + C::OFF_P + sp * kPStageBytes;
+                    g::mbar_expect_tx(p_full(sp), wbytes + 2 * sbytes);
+                    g::bulk_g2s(dst, p.packed + 16ull * N * p.gt.prefix[j] + static_cast<size_t>(8 * rb) * 256 * b, wbytes, p_full(sp));
+                    g::bulk_g2s(dst + 8192, p.scales + static_cast<size_t>(j) * N + kRowsPerCta * rb, sbytes, p_full(sp));
+                    g::bulk_g2s(dst + 8192 + 256, p.zeros + static_cast<size_t>(j) * N + kRowsPerCta * rb, sbytes, p_full(sp));
+                    if (++sp == kNP) { sp = 0; php ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // leave no copy in flight: wait (bounded) for the last phase issued to every stage
+                auto drain = [&](uint32_t bar, uint32_t parity) {
+                    const unsigned long long t0 = g::global_timer_ns();
+                    while (!g::mbar_try_wait(bar, parity) && g::global_timer_ns() - t0 < 1000000ull) { }
+                };
+                for (int s = 0; s < C::NX; ++s) drain(x_full(s), s < sx ? phx : phx ^ 1u);
+                for (int s = 0; s < kNP; ++s) drain(p_full(s), s < sp ? php : php ^ 1u);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(TOK >> 3) << 17) | (static_cast<uint32_t>(kRowsPerCta >> 4) << 24);
+            int sx = 0, sa = 0;
+            uint32_t phx = 0, pha = 0, phd = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                if (!g::mbar_wait(d_empty, phd ^ 1u, abort)) { ok = false; break; }   // epilogue has drained D
+                g::tc_fence_after();
+                for (int j = 0; j < G; ++j) {
+                    if (!g::mbar_wait(x_full(sx), phx, abort) || !g::mbar_wait(a_full(sa), pha, abort)) { ok = false; break; }
+                    g::tc_fence_after();
+                    const uint32_t xs = sbase + sx * C::XSTAGE;
+                    const uint32_t a_t = tmem + kTmemAcol + 64 * sa;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t bdesc = sw128_kmajor_desc(xs + (ks >> 2) * C::XBOX + (ks & 3) * 32);
+                        g::umma_f16_ts(tmem, a_t + 8 * ks, bdesc, idesc, (j | ks) != 0 ? 1u : 0u);
+                    }
+                    g::tc_commit(x_empty(sx));
+                    g::tc_commit(a_empty(sa));
+                    if (++sx == C::NX) { sx = 0; phx ^= 1u; }
+                    if (++sa == kNA) { sa = 0; pha ^= 1u; }
+                }
+                if (ok) g::tc_commit(d_full);
+                phd ^= 1u;
+            }
+        }
+    } else if (warp < 10) {
+        // ------------------------------------------------------------------ dequant warps
+        const int q = warp & 3, kh = (warp - 2) >> 2;           // tensor-memory lane quarter, k half of the group
+        const int r = 32 * q + lane;                            // row inside the block
+        const int t = r >> 4, gq = (r & 15) >> 1, half = r & 1;
+        int sp = 0, sa = 0;
+        uint32_t php = 0, pha = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            const int rb = tile % p.row_blocks;
+            const bool row_ok = kRowsPerCta * rb + r < N;
+            for (int j = 0; j < G; ++j) {
+                if (!g::mbar_wait(p_full(sp), php, abort)) { ok = false; break; }
+                const int b = p.gt.bits[j];
+                const uint32_t stage = sbase + C::OFF_P + sp * kPStageBytes;
+                uint32_t w0[4] = {0, 0, 0, 0}, w1[4] = {0, 0, 0, 0};   // words of units 0..3 for the two 32-k ranges
+                DqRow row;
+                row.zc = __float2half2_rn(16.f);
+                row.s = __float2half2_rn(0.f);
+                if (row_ok) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (u < b) {
+                            const uint4 v = g::lds128(stage + t * 256 * b + 256 * u + 8 * (4 * gq + 2 * kh));
+                            w0[u] = half ? v.y : v.x;
+                            w1[u] = half ? v.w : v.z;
+                        }
+                    }
+                    const __half s = *reinterpret_cast<const __half*>(smem + C::OFF_P + sp * kPStageBytes + 8192 + 2 * r);
+                    const __half z = *reinterpret_cast<const __half*>(smem + C::OFF_P + sp * kPStageBytes + 8192 + 256 + 2 * r);
+                    row.s = __half2half2(s);
+                    row.zc = __half2half2(__hadd(__float2half_rn(16.f), z));
+                }
+                __syncwarp();
+                if (lane == 0) g::mbar_arrive(p_empty(sp));
+                if (++sp == kNP) { sp = 0; php ^= 1u; }
+
+                uint32_t cols[32];
+                switch (b) {
+                    case 1: decode_cword<1>(w0, row, cols); decode_cword<1>(w1, row, cols + 16); break;
+                    case 2: decode_cword<2>(w0, row, cols); decode_cword<2>(w1, row, cols + 16); break;
+                    case 3: decode_cword<3>(w0, row, cols); decode_cword<3>(w1, row, cols + 16); break;
+                    default: decode_cword<4>(w0, row, cols); decode_cword<4>(w1, row, cols + 16); break;
+                }
+                if (!g::mbar_wait(a_empty(sa), pha ^ 1u, abort)) { ok = false; break; }
+                g::tc_fence_after();
+                g::tmem_st32(tmem + (static_cast<uint32_t>(32 * q) << 16) + kTmemAcol + 64 * sa + 32 * kh, cols);
+                g::tc_wait_st();
+                g::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) g::mbar_arrive(a_full(sa));
+                if (++sa == kNA) { sa = 0; pha ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int q = warp & 3;
+        uint32_t phd = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            const int rb = tile % p.row_blocks, mt = tile / p.row_blocks;
+            const int n = kRowsPerCta * rb + 32 * q + lane;
+            if (!g::mbar_wait(d_full, phd, abort)) { ok = false; break; }
+            g::tc_fence_after();
+#pragma unroll 1
+            for (int cc = 0; cc < TOK / 32; ++cc) {
+                uint32_t v[32];
+                g::tmem_ld32(tmem + (static_cast<uint32_t>(32 * q) << 16) + 32 * cc, v);
+                g::tc_wait_ld();
+                const int m0 = mt * TOK + 32 * cc;
+                if (n < N) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (m0 + i < p.M) p.y[static_cast<size_t>(m0 + i) * N + n] = __float2half_rn(__uint_as_float(v[i]));
+                }
+            }
+            g::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) g::mbar_arrive(d_empty);
+            phd ^= 1u;
+        }
+    }
+
+    __syncthreads();
+    if (tid == 0 && *abort != 0) atomicOr(p.status, 1u);
+    if (warp == 1) {
+        g::tc_fence_after();
+        g::tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// Tensor map of x [M][K] fp16: boxes of 64 k x tok rows, 128-byte swizzle, rows past M read as 0.
+static bool make_x_map(CUtensorMap* map, const void* x, int M, int K, int tok) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (enc == nullptr) return false;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(M)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * sizeof(__half)};
+    const cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(tok)};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int gemm_sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    return n;
+}
+
+template <int TOK>
+static cudaError_t launch_gemm(const CUtensorMap& map, const GemmParams& prm, cudaStream_t stream) {
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        e = cudaFuncSetAttribute(gemm_kernel<TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<TOK>::SMEM);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    const int tiles = prm.row_blocks * prm.tok_tiles;
+    const int sms = gemm_sm_count();
+    const int grid = tiles < sms ? tiles : sms;
+    gemm_kernel<TOK><<<grid, kGemmThreads, GemmCfg<TOK>::SMEM, stream>>>(map, prm);
+    return cudaGetLastError();
+}
+
+}  // namespace slim
+
+extern "C" int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* bits_host, const void* scales, const void* zeros,
+                             void* y, int M, int N, int K, int g, void* workspace, size_t workspace_bytes, void* stream) {
+    if (M < 0) return SLIM_ERR_INVALID_ARG;
+    if (M > 0 && M <= SLIM_GEMV_MAX_M) return SLIM_ERR_INVALID_ARG;     // the decode path serves these
+    slim::GroupTable gt;
+    const int st = slim::make_group_table(N, K, g, bits_host, &gt);
+    if (st != SLIM_OK) return st;
+    if (M == 0 || N == 0) return SLIM_OK;
+    if (y == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (!slim::aligned16(y)) return SLIM_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (K == 0) {
+        SLIM_CUDA_TRY(cudaMemsetAsync(y, 0, static_cast<size_t>(M) * N * sizeof(__half), s));
+        return SLIM_OK;
+    }
+    if (x == nullptr || packed == nullptr || scales == nullptr || zeros == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (!slim::aligned16(x) || !slim::aligned16(packed) || !slim::aligned16(scales) || !slim::aligned16(zeros))
+        return SLIM_ERR_ALIGNMENT;
+    if (workspace == nullptr || workspace_bytes < 256) return SLIM_ERR_WORKSPACE;
+    if (!slim::aligned16(workspace)) return SLIM_ERR_ALIGNMENT;
+
+    const int tok = M <= 128 ? 128 : 256;
+    CUtensorMap map;
+    if (!slim::make_x_map(&map, x, M, K, tok)) {
+        slim::set_cuda_error(cudaErrorUnknown);
+        return SLIM_ERR_CUDA;
+    }
+    slim::GemmParams prm;
+    memset(&prm, 0, sizeof prm);
+    prm.packed = static_cast<const uint8_t*>(packed);
+    prm.scales = static_cast<const __half*>(scales);
+    prm.zeros = static_cast<const __half*>(zeros);
+    prm.y = static_cast<__half*>(y);
+    prm.status = static_cast<unsigned int*>(workspace);
+    prm.M = M; prm.N = N; prm.K = K;
+    prm.row_blocks = (N + slim::kRowsPerCta - 1) / slim::kRowsPerCta;
+    prm.tok_tiles = (M + tok - 1) / tok;
+    prm.gt = gt;
+    const cudaError_t e = tok == 128 ? slim::launch_gemm<128>(map, prm, s) : slim::launch_gemm<256>(map, prm, s);
+    SLIM_CUDA_TRY(e);
+    return SLIM_OK;
 }
