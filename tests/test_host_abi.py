@@ -1,0 +1,106 @@
+"""CPU-only checks of the C-ABI library: it builds, loads, exports every declared symbol, and its
+host-side logic (argument validation, sizes, bit allocation, launch plans) behaves as declared.
+No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import slim_oracle as orc
+from paper_2405_14917_b200 import build as cuda_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def slim():
+    cuda_build.build()
+    from paper_2405_14917_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "slim.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(slim_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(slim):
+    names = _declared_symbols()
+    assert {"slim_pack_weights", "slim_dequant", "slim_mpq_gemv", "slim_mpq_gemm"} <= set(names)
+    L = ctypes.CDLL(cuda_build.LIB_PATH)
+    for n in names:
+        assert hasattr(L, n), f"{n} is declared in slim.h but not exported"
+
+
+def test_version_and_status_strings(slim):
+    assert slim.version() >> 16 == 2
+    L = slim.lib()
+    for code in range(0, -7, -1):
+        assert L.slim_status_string(code).decode() not in ("", "unknown status")
+    assert L.slim_status_string(-99).decode() == "unknown status"
+
+
+def test_packed_bytes_is_unpadded(slim):
+    """N*K*avg_bits/8 exactly: groups are stored back to back (App. B.2)."""
+    for N, K, avg in [(4096, 4096, 2), (11008, 4096, 3), (4096, 11008, 2), (16, 128, 3)]:
+        G = K // 128
+        p = G // 4
+        bits = np.full(G, avg, np.uint8)
+        bits[:p] = avg + 1
+        bits[G - p:] = avg - 1
+        assert slim.packed_bytes(N, K, bits) == N * K * avg // 8 == orc.packed_bytes(N, K, bits)
+
+
+def test_shape_and_argument_errors(slim):
+    bits = np.array([2, 2], np.uint8)
+    out = ctypes.c_size_t(0)
+    L = slim.lib()
+    bp = bits.ctypes.data_as(ctypes.c_void_p)
+    assert L.slim_packed_bytes(16, 256, 64, bp, ctypes.byref(out)) == -2      # g != 128
+    assert L.slim_packed_bytes(16, 200, 128, bp, ctypes.byref(out)) == -2     # K % 128
+    assert L.slim_packed_bytes(24, 256, 128, bp, ctypes.byref(out)) == -2     # N % 16
+    assert L.slim_packed_bytes(16, 256, 128, None, ctypes.byref(out)) == -1   # no bit map
+    bad = np.array([2, 5], np.uint8)
+    assert L.slim_packed_bytes(16, 256, 128, bad.ctypes.data_as(ctypes.c_void_p), ctypes.byref(out)) == -1
+    big = np.full(257, 2, np.uint8)
+    assert L.slim_packed_bytes(16, 257 * 128, 128, big.ctypes.data_as(ctypes.c_void_p), ctypes.byref(out)) == -2
+    # the linear entry points validate before touching the device: null pointers and M ranges
+    assert L.slim_mpq_gemv(None, None, bp, None, None, None, 17, 16, 256, 128, None, 0, None) == -1
+    assert L.slim_mpq_gemm(None, None, bp, None, None, None, 16, 16, 256, 128, None, 0, None) == -1
+    assert L.slim_mpq_gemv(None, None, bp, None, None, None, 1, 16, 256, 128, None, 0, None) == -1   # y missing
+    assert L.slim_mpq_gemv(None, None, bp, None, None, None, 0, 16, 256, 128, None, 0, None) == 0    # M = 0: no-op
+
+
+def test_allocate_bits_matches_oracle_and_budget(slim):
+    rng = np.random.default_rng(11)
+    for G in (4, 32, 86, 108, 224):
+        for avg in (2, 3):
+            S = rng.lognormal(size=G)
+            b = slim.allocate_bits(S, avg)
+            assert (b == orc.allocate_bits(S, avg)).all()
+            assert int(b.astype(int).sum()) == avg * G                       # the average-bit budget is exact
+            assert (b == avg + 1).sum() == (b == avg - 1).sum() == G // 4
+            T = rng.integers(0, 4, G).astype(np.float64)                     # ties: lower index ranks higher
+            assert (slim.allocate_bits(T, avg) == orc.allocate_bits(T, avg)).all()
+
+
+def test_gemv_plan_invariants(slim):
+    rng = np.random.default_rng(3)
+    for (N, K, avg, M) in [(4096, 4096, 2, 1), (11008, 4096, 2, 1), (4096, 11008, 2, 1), (1024, 8192, 2, 16),
+                           (28672, 8192, 2, 1), (8192, 28672, 2, 16), (16, 128, 2, 1), (272, 1408, 3, 9), (4096, 32768, 3, 16)]:
+        G = K // 128
+        bits = np.full(G, avg, np.uint8)
+        bits[: G // 4] = avg + 1
+        bits[G - G // 4:] = avg - 1
+        rng.shuffle(bits)
+        pl = slim.gemv_plan(M, N, K, bits)
+        assert pl["tiles_per_cta"] in (1, 2, 4, 8)
+        assert 1 <= pl["k_slices"] <= min(8, G)
+        assert pl["row_blocks"] * pl["tiles_per_cta"] >= N // 16
+        assert pl["smem_bytes"] <= 227 * 1024
+        assert pl["n_tiles"] == (1 if M <= 8 else 2)
+        assert 1 <= pl["groups_per_chunk"] <= G
