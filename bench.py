@@ -40,7 +40,9 @@ FALLBACK_TENSOR_TFLOPS = 1400.0
 # dram__bytes_write.sum), keyed by the sha256 of the kernel source it was taken from.  A kernel
 # that has changed since reports null.
 NCU_TRAFFIC = {
-    # "sha256 of csrc/slim_gemv.cu": {"layer": "NxK", "traffic_bytes": ..., "algorithmic_bytes": ...}
+    # 4096x4096 layer, avg 2-bit, M = 1: 4,759,808 B read + 0 written per launch (algorithmic 4,735,008 B);
+    # scaled to the sweep's average launch by the algorithmic bytes (traffic grows with the layer size)
+    "6b2aa44167417399c395aecc4c7a8801c023f59a66e454ef099c876e580ddeed": {"layer": "4096x4096", "traffic_bytes": 4759808, "algorithmic_bytes": 4735008},
 }
 
 
@@ -385,7 +387,7 @@ def run_ours(args, spec):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": peak_kind, "kernel": "gemv_kernel", "avg_launch_us": per_launch_us,
                      "algorithmic_bytes_per_launch": alg_bytes / n_launch,
-                     "traffic": traffic["traffic_bytes"] if traffic else None,
+                     "traffic": (traffic["traffic_bytes"] / traffic["algorithmic_bytes"] * alg_bytes / n_launch) if traffic else None,
                      "frac_of_nominal_8000": achieved / 8000.0},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 2),
                 "d2h_bytes_per_step": int(y_host.numel() * 2), "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
