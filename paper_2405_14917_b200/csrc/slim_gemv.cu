@@ -10,11 +10,10 @@
 //    shifted right once first.
 //  * B operand = activations, staged once per CTA in fragment order: x[m][k] * 2^(S + lo - pos),
 //    where pos undoes the field position of the weight it will meet, lo is the slice's offset
-//    inside the code, and 2^S (per token and chunk, from max|x|) lifts the values to the top of the
+//    inside the code, and 2^S (per token and group, from max|x|) lifts the values to the top of the
 //    fp16 range so that the small ones keep their bits.
 //  * The MMA accumulates the exact products in fp32.  Per (row, group) the group partial D is
-//    folded as acc += s * (D - z * sum_k x_k), which is s * sum_k x_k (q_k - z); the chunk's
-//    2^(24-S) is undone when the chunk is added to the running sum.
+//    folded as acc += s * (D * 2^(24-S) - z * sum_k x_k), which is s * sum_k x_k (q_k - z).
 //
 // Work split.  A layer is smaller than, or comparable to, the bytes HBM must keep in flight, and
 // a warp's instruction stream is the critical path, so the kernel spreads a layer over as many
@@ -26,11 +25,14 @@
 //  * Every warp issues the weight, scale and zero bytes of its groups of the first chunk as
 //    16-byte cp.async copies in its first instructions; chunk c+1 is in flight while chunk c is
 //    consumed.
-//  * The kernel is launched with programmatic stream serialisation: after issuing the copies it
-//    lets the next kernel start (whose copies then overlap this kernel's arithmetic) and only
-//    then waits for the previous kernel before it touches x or y.
-//  * Partial sums are added across warps in shared memory and across the cluster through
-//    distributed shared memory, both in a fixed order (deterministic); no global scratch.
+//  * The kernel is launched with programmatic stream serialisation: it lets the next kernel
+//    start at once (whose copies then overlap this kernel's arithmetic) and waits for the
+//    previous kernel only before it touches x or y.
+//  * x is put into B-fragment order by one warp per (token, group), which also finds the group's
+//    max |x| and sum with shuffles: one barrier between landing and use.
+//  * Partial sums are added across warps in shared memory; across the cluster every CTA owns a
+//    share of the outputs, receives the other CTAs' partials for it through distributed shared
+//    memory and adds them in rank order (deterministic); no global scratch.
 #include "slim_common.cuh"
 
 #include <cstring>
@@ -56,6 +58,7 @@ struct GemvParams {
     int max_slots;          // most slices in any chunk
     int two_bufs;           // some k-slice has more than one chunk: weights and raw x are double-buffered
     uint16_t kbegin[kMaxCluster + 1];
+    uint16_t pre3[SLIM_MAX_GROUPS + 1];   // pre3[j] = number of 3-bit groups (two slices) before group j
     GroupTable gt;
 };
 
@@ -83,6 +86,12 @@ __device__ __forceinline__ float2 ld_cluster_f32x2(uint32_t local_addr, uint32_t
     float2 v;
     asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(remote) : "memory");
     return v;
+}
+
+__device__ __forceinline__ void st_cluster_f32x2(uint32_t local_addr, uint32_t rank, float2 v) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(remote), "f"(v.x), "f"(v.y) : "memory");
 }
 
 __device__ __forceinline__ uint2 lds64(uint32_t addr) {
@@ -126,23 +135,24 @@ using W4 = WidthTag<4>;
 
 // ------------------------------------------------------------------------------------------ shared memory map
 struct SmemMap {
-    uint32_t smax;     // uint32[2][16]: per-token max |x| bits over the chunk (double-buffered)
-    uint32_t xslot;    // uint16[GC + 1]: first staging slot of each group of the chunk
-    uint32_t sx;       // float[GC][16]: 2^(S-24) * sum_k x per (group, token)
-    uint32_t red;      // float[W][M][16]: per-warp partial outputs, then [M][16] in place of warp 0
+    uint32_t sxe;      // float2[GC][16]: (sum_k x, 2^(24-S)) per (group, token)
+    uint32_t red;      // float[W][M][16]: per-warp partial outputs
+    uint32_t cred;     // float2[CS][share]: partial outputs received from the cluster's CTAs
     uint32_t xraw;     // half[2][M][GC*128] (double-buffered)
     uint32_t xs;       // [slots][8 mma][M tokens][4 lanes] x 8 B: B fragments
     uint32_t wbuf;     // [2][region_bytes]: packed slices, scales, zeros of the chunk
     uint32_t total;
 };
 __host__ __device__ inline uint32_t align_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
-__host__ __device__ inline SmemMap make_smem_map(int M, int W, int GC, int region_bytes, int max_slots, bool two_bufs) {
+// Output pairs (two rows of one token) a CTA owns in the cluster reduction.
+__host__ __device__ inline int cluster_share(int T, int M, int CS) { return (T * M * 8 + CS - 1) / CS; }
+__host__ __device__ inline SmemMap make_smem_map(int M, int W, int T, int CS, int GC, int region_bytes, int max_slots, bool two_bufs) {
     SmemMap m;
     uint32_t o = 0;
-    m.smax = o;  o += 128;
-    m.xslot = o; o += align_up(2 * (GC + 1), 16);
-    m.sx = o;    o += 64u * GC;
+    m.sxe = o;   o += 128u * GC;
     m.red = o;   o += 64u * W * M;
+    m.cred = o;  o += CS > 1 ? 8u * CS * cluster_share(T, M, CS) : 0u;
+    o = align_up(o, 16);
     m.xraw = o;  o += (two_bufs ? 2u : 1u) * (256u * M * GC);
     o = align_up(o, 128);
     m.xs = o;    o += static_cast<uint32_t>(max_slots) * 8 * M * 32;
@@ -157,6 +167,9 @@ template <int NT>   // 8-token MMA tiles: 1 (M <= 8) or 2
 __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_constant__ GemvParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
+    // Let the next kernel of the stream start at once: it only prefetches its own weights until
+    // this kernel has finished.
+    pdl_launch_dependents();
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int W = p.W, T = p.T, KW = W / T, nthreads = W * 32;
@@ -166,7 +179,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
     const int g0 = p.kbegin[ks], g1 = p.kbegin[ks + 1];
     const int ng = g1 - g0;
     const int n_chunks = (ng + GC - 1) / GC;
-    const SmemMap sm = make_smem_map(M, W, GC, p.region_bytes, p.max_slots, p.two_bufs != 0);
+    const SmemMap sm = make_smem_map(M, W, T, p.CS, GC, p.region_bytes, p.max_slots, p.two_bufs != 0);
     const uint32_t xraw_stride = 256u * M * GC;                   // bytes per xraw buffer
     const int tw = warp % T, kw = warp / T;                       // this warp's tile of the CTA and k-way
     const int tile = rb * T + tw;
@@ -209,99 +222,62 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
         cp_async_commit();
     };
 
-    // ---- put the first chunk in flight --------------------------------------------------------------
+    // ---- put the first chunk in flight, then wait until the previous kernel has finished before
+    // x or y are touched
     issue_weights(0);
-    // Let the next kernel begin its own copies, then wait until the previous kernel has finished
-    // before x or y are touched.
-    pdl_launch_dependents();
     pdl_wait();
     issue_x(0);
+    for (int i = tid; i < 32 * GC; i += nthreads) reinterpret_cast<float*>(smem + sm.sxe)[i] = 0.f;   // absent tokens read 0
 
-    uint32_t* smax = reinterpret_cast<uint32_t*>(smem + sm.smax);
-    if (tid < 32) smax[tid] = 0;
-    for (int i = tid; i < 16 * GC; i += nthreads) reinterpret_cast<float*>(smem + sm.sx)[i] = 0.f;   // absent tokens read 0
-    // per-token exponent S of a chunk: max|x| * 2^S lies in [2^13, 2^14) (Inf/NaN: the top binade)
-    auto token_exp = [&](int ch, int m) -> int {
-        const uint32_t mx = smax[(ch & 1) * 16 + m];
-        return mx == 0 ? 0 : 28 - max(static_cast<int>(mx >> 10), 1);
-    };
-
-    float accf[NT][4];
+    float acc[NT][4];
 #pragma unroll
     for (int n = 0; n < NT; ++n)
 #pragma unroll
-        for (int r = 0; r < 4; ++r) accf[n][r] = 0.f;
+        for (int r = 0; r < 4; ++r) acc[n][r] = 0.f;
 
     for (int ch = 0; ch < n_chunks; ++ch) {
         const int ja = g0 + ch * GC, cg = min(g1, ja + GC) - ja;
         const int kc = GC * SLIM_GROUP;                                   // xraw row stride (halves)
         const __half* xraw = reinterpret_cast<const __half*>(smem + sm.xraw + (ch & 1) * xraw_stride);
-        uint16_t* xslot = reinterpret_cast<uint16_t*>(smem + sm.xslot);
+        float2* sxe = reinterpret_cast<float2*>(smem + sm.sxe);
 
         cp_async_wait_all();             // x and weights of this chunk have landed (this thread's copies)
         __syncthreads();                 // ... everybody's; and the previous chunk is fully consumed
         issue_weights(ch + 1);           // into the buffer the previous chunk has left
-        // ---- per-token max |x| of the chunk, slot table ---------------------------------------------
-        {
-            const int per_tok = cg * 16;
-            for (int m = 0; m < M; ++m) {
-                uint32_t mx = 0;
-                for (int q = tid; q < per_tok; q += nthreads) {
-                    const uint4 v = *reinterpret_cast<const uint4*>(xraw + m * kc + 8 * q);
-                    const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+        // ---- activations in B-fragment order: one warp per (token, group) ------------------------------
+        for (int pi = warp; pi < M * cg; pi += W) {
+            const int m = pi / cg, i = pi - m * cg;
+            const __half* xg = xraw + m * kc + i * SLIM_GROUP;
+            // 2^S lifts the group's largest |x| into [2^13, 2^14) (Inf/NaN: the top binade)
+            const uint2 raw = *reinterpret_cast<const uint2*>(xg + 4 * lane);
+            uint32_t mx = max(max(raw.x & 0x7fffu, (raw.x >> 16) & 0x7fffu), max(raw.y & 0x7fffu, (raw.y >> 16) & 0x7fffu));
+            mx = __reduce_max_sync(0xffffffffu, mx);
+            const int S = mx == 0 ? 0 : 28 - max(static_cast<int>(mx >> 10), 1);
+            const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+            const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+            float sum = (f01.x + f01.y) + (f23.x + f23.y);
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) mx = max(mx, max(wv[t] & 0x7fffu, (wv[t] >> 16) & 0x7fffu));
-                }
-                mx = __reduce_max_sync(0xffffffffu, mx);
-                if (lane == 0 && mx != 0) atomicMax(smax + (ch & 1) * 16 + m, mx);
-            }
-            if (tid == nthreads - 1) {
-                int slot = 0;
-                for (int i = 0; i < cg; ++i) { xslot[i] = static_cast<uint16_t>(slot); slot += slice_count(p.gt.bits[ja + i]); }
-                xslot[cg] = static_cast<uint16_t>(slot);
-            }
-            if (tid < 16) smax[((ch + 1) & 1) * 16 + tid] = 0;        // for the next chunk
-        }
-        __syncthreads();
-        // ---- activations in B-fragment order; group sums -----------------------------------------------
-        {
-            // One task = (group i, slice s, mma mi, lane column cc) of a token: the four activations that
-            // meet one lane's two B registers.
-            float* sx = reinterpret_cast<float*>(smem + sm.sx);
-            for (int m = 0; m < M; ++m) {
-                const int S = token_exp(ch, m);
-                for (int t = tid; t < cg * 64; t += nthreads) {
-                    const int cc = t & 3, mi = (t >> 2) & 7, s = (t >> 5) & 1, i = t >> 6;
-                    const int b = p.gt.bits[ja + i];
-                    if (s >= slice_count(b)) continue;
-                    const int w = slice_w(b, s), lo = slice_lo(b, s);
-                    const int lg = w >> 1;                          // log2(w) for w in {1,2,4}
-                    const int nf = 32 >> lg;                        // fields per word; 8/w MMAs per unit
-                    const int u = mi >> (3 - lg), ii = mi & ((8 >> lg) - 1);
-                    const __half* xg = xraw + m * kc + i * SLIM_GROUP + 32 * cc + nf * u + 2 * ii;
-                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(xg));               // pairs 2ii, 2ii+1: first field
-                    const float2 g = __half22float2(*reinterpret_cast<const __half2*>(xg + (nf >> 1)));   // ... second field
-                    const float sc0 = __int_as_float((127 + S + lo - pair_pos(w, 2 * ii)) << 23);
-                    const float sc1 = __int_as_float((127 + S + lo - pair_pos(w, 2 * ii + 1)) << 23);
-                    const __half2 b0 = __floats2half2_rn(f.x * sc0, g.x * sc0);
-                    const __half2 b1 = __floats2half2_rn(f.y * sc1, g.y * sc1);
-                    *reinterpret_cast<uint2*>(smem + sm.xs + (((static_cast<size_t>(xslot[i] + s) * 8 + mi) * M + m) * 4 + cc) * 8) =
-                        make_uint2(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1));
-                }
-                // per group: 2^(S-24) * sum_k x; 8 lanes per sum, fixed order
-                for (int qb = warp * 4; qb < cg; qb += nthreads / 8) {       // warp-uniform trip count
-                    const int i = qb + (lane >> 3), l8 = lane & 7;
-                    float acc = 0.f;
-                    if (i < cg) {
-                        const __half* src = xraw + m * kc + i * SLIM_GROUP + 16 * l8;
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) acc += __half2float(src[k]);
-                    }
-                    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-                    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-                    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
-                    if (i < cg && l8 == 0) sx[i * 16 + m] = acc * __int_as_float((127 + S - 24) << 23);
-                }
+            for (int o = 1; o < 32; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            if (lane == 0) sxe[i * 16 + m] = make_float2(sum, __int_as_float((127 + 24 - S) << 23));
+            // lane = (mma mi, lane column cc): the four activations that meet one lane's two B registers
+            const int b = p.gt.bits[ja + i];
+            const int slot0 = i + p.pre3[ja + i] - p.pre3[ja];
+            const int cc = lane & 3, mi = lane >> 2;
+            const int ns = slice_count(b);
+            for (int s = 0; s < ns; ++s) {
+                const int w = slice_w(b, s), lo = slice_lo(b, s);
+                const int lg = w >> 1;                          // log2(w) for w in {1,2,4}
+                const int nf = 32 >> lg;                        // fields per word; 8/w MMAs per unit
+                const int u = mi >> (3 - lg), ii = mi & ((8 >> lg) - 1);
+                const __half* xp = xg + 32 * cc + nf * u + 2 * ii;
+                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(xp));               // pairs 2ii, 2ii+1: first field
+                const float2 g = __half22float2(*reinterpret_cast<const __half2*>(xp + (nf >> 1)));   // ... second field
+                const float sc0 = __int_as_float((127 + S + lo - pair_pos(w, 2 * ii)) << 23);
+                const float sc1 = __int_as_float((127 + S + lo - pair_pos(w, 2 * ii + 1)) << 23);
+                const __half2 b0 = __floats2half2_rn(f.x * sc0, g.x * sc0);
+                const __half2 b1 = __floats2half2_rn(f.y * sc1, g.y * sc1);
+                *reinterpret_cast<uint2*>(smem + sm.xs + (((static_cast<size_t>(slot0 + s) * 8 + mi) * M + m) * 4 + cc) * 8) =
+                    make_uint2(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1));
             }
         }
         issue_x(ch + 1);
@@ -309,22 +285,19 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
 
         // ---- this warp's tile against its groups of the chunk --------------------------------------------
         if (active) {
-            float acc[NT][4];
-#pragma unroll
-            for (int n = 0; n < NT; ++n)
-#pragma unroll
-                for (int r = 0; r < 4; ++r) acc[n][r] = 0.f;
             const uint32_t buf = sbase + sm.wbuf + (ch & 1) * p.region_bytes;
             for (int it = kw; it < cg; it += KW) {
                 const int b = p.gt.bits[ja + it];
                 const uint32_t item = item_addr(buf, ja, ja + it, b);
-                const uint32_t xs_slot0 = sbase + sm.xs + static_cast<uint32_t>(xslot[it]) * 8 * M * 32;
+                const uint32_t xs_slot0 = sbase + sm.xs + static_cast<uint32_t>(it + p.pre3[ja + it] - p.pre3[ja]) * 8 * M * 32;
 
-                float d[NT][4];
+                float d[2][NT][4];       // two interleaved accumulation chains
 #pragma unroll
-                for (int n = 0; n < NT; ++n)
+                for (int h = 0; h < 2; ++h)
 #pragma unroll
-                    for (int r = 0; r < 4; ++r) d[n][r] = 0.f;
+                    for (int n = 0; n < NT; ++n)
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) d[h][n][r] = 0.f;
 
                 // one slice of width WD starting at unit `unit0`, activations in staging slot `xs_slot`
                 auto run_slice = [&](auto wtag, int unit0, uint32_t xs_slot) {
@@ -344,7 +317,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
                                 const int m = 8 * n + gq;
                                 uint2 bv = make_uint2(0u, 0u);
                                 if (m < M) bv = lds64(xs_slot + ((mi * M + m) * 4 + c) * 8);
-                                mma_f16(d[n], a0, a1, a2, a3, bv);
+                                mma_f16(d[ii & 1][n], a0, a1, a2, a3, bv);
                             }
                         }
                     }
@@ -356,32 +329,21 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
                     default: run_slice(W4{}, 0, xs_slot0); break;
                 }
 
-                // fold the group: acc += s * (D - z * sum_x); rows 2gq, 2gq+1, tokens 8n+2c, 8n+2c+1
+                // fold the group: acc += s * (D * 2^(24-S) - z * sum_x); rows 2gq, 2gq+1, tokens 8n+2c, 8n+2c+1
                 const uint32_t s2 = lds32(item + 256 * b + gq * 4);
                 const uint32_t z2 = lds32(item + 256 * b + 32 + gq * 4);
                 const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
                 const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
-                const uint32_t sxa = sbase + sm.sx + (it * 16 + 2 * c) * 4;
 #pragma unroll
                 for (int n = 0; n < NT; ++n) {
-                    const uint2 sxr = lds64(sxa + n * 32);
-                    const float sx0 = __uint_as_float(sxr.x), sx1 = __uint_as_float(sxr.y);
-                    acc[n][0] = fmaf(sf.x, fmaf(-zf.x, sx0, d[n][0]), acc[n][0]);
-                    acc[n][1] = fmaf(sf.x, fmaf(-zf.x, sx1, d[n][1]), acc[n][1]);
-                    acc[n][2] = fmaf(sf.y, fmaf(-zf.y, sx0, d[n][2]), acc[n][2]);
-                    acc[n][3] = fmaf(sf.y, fmaf(-zf.y, sx1, d[n][3]), acc[n][3]);
+                    const float4 t = *reinterpret_cast<const float4*>(sxe + it * 16 + 8 * n + 2 * c);   // (sx0, e0, sx1, e1)
+                    const float d0 = (d[0][n][0] + d[1][n][0]) * t.y, d1 = (d[0][n][1] + d[1][n][1]) * t.w;
+                    const float d2 = (d[0][n][2] + d[1][n][2]) * t.y, d3 = (d[0][n][3] + d[1][n][3]) * t.w;
+                    acc[n][0] = fmaf(sf.x, fmaf(-zf.x, t.x, d0), acc[n][0]);
+                    acc[n][1] = fmaf(sf.x, fmaf(-zf.x, t.z, d1), acc[n][1]);
+                    acc[n][2] = fmaf(sf.y, fmaf(-zf.y, t.x, d2), acc[n][2]);
+                    acc[n][3] = fmaf(sf.y, fmaf(-zf.y, t.z, d3), acc[n][3]);
                 }
-            }
-            // undo the chunk's activation scaling
-#pragma unroll
-            for (int n = 0; n < NT; ++n) {
-                const int m0 = 8 * n + 2 * c;
-                const float back0 = m0 < M ? __int_as_float((127 + 24 - token_exp(ch, m0)) << 23) : 0.f;
-                const float back1 = m0 + 1 < M ? __int_as_float((127 + 24 - token_exp(ch, m0 + 1)) << 23) : 0.f;
-                accf[n][0] = fmaf(acc[n][0], back0, accf[n][0]);
-                accf[n][1] = fmaf(acc[n][1], back1, accf[n][1]);
-                accf[n][2] = fmaf(acc[n][2], back0, accf[n][2]);
-                accf[n][3] = fmaf(acc[n][3], back1, accf[n][3]);
             }
         }
     }
@@ -391,16 +353,18 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
 #pragma unroll
     for (int n = 0; n < NT; ++n) {
         const int m0 = 8 * n + 2 * c;
-        if (m0 < M) *reinterpret_cast<float2*>(red + (warp * M + m0) * 16 + 2 * gq) = make_float2(accf[n][0], accf[n][2]);
-        if (m0 + 1 < M) *reinterpret_cast<float2*>(red + (warp * M + m0 + 1) * 16 + 2 * gq) = make_float2(accf[n][1], accf[n][3]);
+        if (m0 < M) *reinterpret_cast<float2*>(red + (warp * M + m0) * 16 + 2 * gq) = make_float2(acc[n][0], acc[n][2]);
+        if (m0 + 1 < M) *reinterpret_cast<float2*>(red + (warp * M + m0 + 1) * 16 + 2 * gq) = make_float2(acc[n][1], acc[n][3]);
     }
     __syncthreads();
-    const bool direct = (p.CS == 1);
+    const int CS = p.CS;
     const int pairs = T * M * 8;                                // e = (tile of the CTA, token, row pair)
-    auto out_ptr = [&](int e) -> __half2* {
+    const int share = cluster_share(T, M, CS);
+    const uint32_t rank = CS > 1 ? cluster_ctarank() : 0u;
+    auto store_out = [&](int e, float2 v) {
         const int t = e / (M * 8), rem = e - t * (M * 8);
         const int row = 16 * (rb * T + t) + 2 * (rem & 7);
-        return row < N ? reinterpret_cast<__half2*>(p.y + static_cast<size_t>(rem >> 3) * N + row) : nullptr;
+        if (row < N) *reinterpret_cast<__half2*>(p.y + static_cast<size_t>(rem >> 3) * N + row) = __floats2half2_rn(v.x, v.y);
     };
     for (int e = tid; e < pairs; e += nthreads) {
         float2 sum = make_float2(0.f, 0.f);
@@ -409,34 +373,31 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
             sum.x += v.x;
             sum.y += v.y;
         }
-        if (direct) {
-            __half2* dst = out_ptr(e);
-            if (dst != nullptr) *dst = __floats2half2_rn(sum.x, sum.y);
+        if (CS == 1) {
+            store_out(e, sum);
         } else {
-            *reinterpret_cast<float2*>(red + 2 * e) = sum;      // CTA partial in place of k-way 0 (read by this thread only)
+            // hand the pair to the CTA of the cluster that owns it
+            const int owner = e / share;
+            st_cluster_f32x2(sbase + sm.cred + 8u * (rank * share + (e - owner * share)), owner, sum);
         }
     }
-    if (direct) return;
+    if (CS == 1) return;
 
-    // ---- split-K: add the partials of the cluster's CTAs in rank order ------------------------------
+    // ---- split-K: every CTA adds, in rank order, the partials it received for its share of pairs -----
     cluster_sync_all();
-    {
-        const uint32_t rank = cluster_ctarank();
-        const int share = (pairs + p.CS - 1) / p.CS;
-        const int e1 = min(pairs, static_cast<int>(rank + 1) * share);
-        for (int e = rank * share + tid; e < e1; e += nthreads) {
-            const uint32_t addr = sbase + sm.red + 8 * e;
+    const float2* cred = reinterpret_cast<const float2*>(smem + sm.cred);
+    for (int i = tid; i < share; i += nthreads) {
+        const int e = rank * share + i;
+        if (e < pairs) {
             float2 sum = make_float2(0.f, 0.f);
-            for (int s = 0; s < p.CS; ++s) {
-                const float2 v = ld_cluster_f32x2(addr, s);
+            for (int s = 0; s < CS; ++s) {
+                const float2 v = cred[s * share + i];
                 sum.x += v.x;
                 sum.y += v.y;
             }
-            __half2* dst = out_ptr(e);
-            if (dst != nullptr) *dst = __floats2half2_rn(sum.x, sum.y);
+            store_out(e, sum);
         }
     }
-    cluster_sync_all();   // nobody leaves while a peer may still read its partials
 }
 
 // ------------------------------------------------------------------------------------------ host side
@@ -500,7 +461,7 @@ static void size_chunks(const GroupTable& gt, int gc, GemvPlan* pl) {
 
 // Deterministic launch plan for (M, N, K, bit map) on the current device.  x is staged once per
 // CTA, so a CTA takes as many tiles (up to 8, one per warp) as still leaves two CTAs per SM; the
-// k-range is cut so that a warp sees about four groups (its instruction stream is the critical
+// k-range is cut so that a warp sees about two groups (its instruction stream is the critical
 // path) and further while the grid is smaller than two CTAs per SM; chunks
 // are as long as shared memory allows while CTAs of consecutive layers can still share an SM.
 // Returns false if a single group does not fit (cannot happen within the documented limits).
@@ -515,7 +476,7 @@ static bool plan_gemv(int M, int N, const GroupTable& gt, GemvPlan* pl) {
     while (T > 1 && ((tiles + T - 1) / T) * cs_max < 2 * sms) T >>= 1;
     pl->T = T;
     const int rb = (tiles + T - 1) / T;
-    int cs = (G * T / kMaxWarps + 3) / 4;
+    int cs = (G * T / kMaxWarps + 1) / 2;
     if (cs < 1) cs = 1;
     if (cs > cs_max) cs = cs_max;
     while (cs < cs_max && rb * cs < 2 * sms) ++cs;
@@ -526,7 +487,7 @@ static bool plan_gemv(int M, int N, const GroupTable& gt, GemvPlan* pl) {
     for (int bi = 0; bi < 3; ++bi)
         for (int nc = 1; nc <= (bi == 0 && pl->max_groups > 2 ? 2 : pl->max_groups); ++nc) {
             size_chunks(gt, (pl->max_groups + nc - 1) / nc, pl);
-            const uint32_t need = make_smem_map(M, pl->W, pl->GC, pl->region_bytes, pl->max_slots, pl->two_bufs).total;
+            const uint32_t need = make_smem_map(M, pl->W, pl->T, pl->CS, pl->GC, pl->region_bytes, pl->max_slots, pl->two_bufs).total;
             if (need > budgets[bi]) continue;
             pl->smem_bytes = need;
             return true;
@@ -649,6 +610,9 @@ int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host, c
     prm.max_slots = pl.max_slots;
     prm.two_bufs = pl.two_bufs ? 1 : 0;
     memcpy(prm.kbegin, pl.kbegin, sizeof prm.kbegin);
+    prm.pre3[0] = 0;
+    for (int j = 0; j < SLIM_MAX_GROUPS; ++j)
+        prm.pre3[j + 1] = static_cast<uint16_t>(prm.pre3[j] + (j < gt.G && gt.bits[j] == 3 ? 1 : 0));
     prm.gt = gt;
 
     cudaError_t e;
