@@ -73,12 +73,16 @@ int slim_last_cuda_error(void);
 /* Size of the packed buffer, N*K*avg_bits/8 bytes ("no additional padding", App. B.2). */
 int slim_packed_bytes(int N, int K, int g, const uint8_t* bits_host, size_t* out_bytes);
 
-/* Scratch size for slim_mpq_gemv / slim_mpq_gemm with these shapes on the current device
- * (split-K partial sums, tile counters, one status word).  Always at least 256. */
+/* Scratch size for slim_mpq_gemv / slim_mpq_gemm with these shapes on the current device.
+ * Always at least 256 (one status word).  slim_mpq_gemv needs no more.  slim_mpq_gemm asks for
+ * flags and fp32 partial tiles (128 KB per SM) when it would split tiles across CTAs (stream-K:
+ * shapes whose tile count leaves the last wave of CTAs mostly idle); given a smaller workspace
+ * (at least 256 bytes) it falls back to whole tiles per CTA and uses no scratch. */
 int slim_workspace_bytes(int M, int N, int K, int g, const uint8_t* bits_host, size_t* out_bytes);
 
-/* Zeroes the control part of a workspace (status word and tile counters).  Must be enqueued
- * once after allocating a workspace, before its first use; the kernels leave it zeroed. */
+/* Zeroes a workspace (status word, stream-K flags).  Must be enqueued once after allocating a
+ * workspace, before its first use; the kernels leave the flags zeroed.  Calls that share a
+ * workspace must be ordered on one stream. */
 int slim_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
 /* Synchronises `stream`, reads and clears the workspace status word.  Returns SLIM_OK, or
@@ -101,8 +105,8 @@ int slim_dequant(const void* packed, const uint8_t* bits_host, const void* scale
 /* Decode path, 1 <= M <= 16:  y = x * W-hat^T, fp32 accumulation, fp16 output (the paper's
  * inference kernel, App. B.2: group-by-group dequantisation and dot product with the shared
  * activation).  Streams the packed slices once; HBM-bound.  Results are deterministic for a
- * given (shape, device).  x with Inf/NaN gives unspecified y.  `workspace` may be NULL only if
- * slim_workspace_bytes() reported 256 or less... it never does; pass a workspace. */
+ * given (shape, device).  x with Inf/NaN gives unspecified y.  `workspace` must be at least 256
+ * bytes (the kernel itself keeps its partial sums in shared memory). */
 int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host,
                   const void* scales, const void* zeros, void* y,
                   int M, int N, int K, int g,
@@ -114,7 +118,9 @@ int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host,
  * grid = k-slices x row blocks, 8 warps per CTA. */
 int slim_gemv_plan(int M, int N, int K, int g, const uint8_t* bits_host, int* out6);
 
-/* Batched / prefill path, M > 16: same contract, tensor-core (tcgen05) kernel. */
+/* Batched / prefill path, M > 16: same contract, tensor-core (tcgen05) kernel.  Zero points that
+ * are multiples of 1/64 in [-16, 16) (every zero point Eq. 1 or Eq. 2 produces) are applied exactly,
+ * others are rounded to the nearest 1/64.  Deterministic for a given (shape, device, workspace size). */
 int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* bits_host,
                   const void* scales, const void* zeros, void* y,
                   int M, int N, int K, int g,

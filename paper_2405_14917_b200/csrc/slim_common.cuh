@@ -23,6 +23,9 @@ void set_cuda_error(cudaError_t e);
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Scratch bytes slim_mpq_gemm wants for (M, N) on the current device (256 when it needs none).
+size_t gemm_workspace_bytes(int M, int N, int G);
+
 // Validates shape arguments and fills the table.  Returns SLIM_OK or an error status.
 int make_group_table(int N, int K, int g, const uint8_t* bits_host, GroupTable* out);
 

@@ -44,10 +44,17 @@ struct GemmParams {
     const __half* zeros;
     __half* y;
     unsigned int* status;
+    unsigned int* flags;     // [grid]: "partial of this CTA is ready" (stream-K only; zero between launches)
+    float* partials;         // [grid][TOK][128] fp32 (stream-K only)
     int M, N, K;
     int row_blocks, tok_tiles;
+    int stream_k;            // 1: CTAs take equal shares of (tile, group) units; 0: whole tiles
     GroupTable gt;
 };
+
+constexpr int kGemmWsFlags = 256;            // byte offset of the flags in the workspace
+constexpr int kGemmMaxGrid = 256;
+constexpr int kGemmWsPartials = kGemmWsFlags + 4 * kGemmMaxGrid;
 
 // ------------------------------------------------------------------------------------------ PTX helpers
 namespace g {
@@ -271,6 +278,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
 
     const int G = p.gt.G, N = p.N;
     const int total_tiles = p.row_blocks * p.tok_tiles;
+    // This CTA's contiguous range [u0, u1) of (tile, group) units, unit = tile * G + group,
+    // tile = token tile * row_blocks + row block.  Without stream-K the range is whole tiles.
+    auto range_begin = [&](int cta) -> long long {
+        return p.stream_k ? (static_cast<long long>(cta) * total_tiles * G) / gridDim.x
+                          : ((static_cast<long long>(cta) * total_tiles) / gridDim.x) * G;
+    };
+    const long long u0 = range_begin(blockIdx.x), u1 = range_begin(blockIdx.x + 1);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
@@ -278,10 +292,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
             int sx = 0, sp = 0;
             uint32_t phx = 0, php = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (long long u = u0; u < u1 && ok;) {
+                const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
+                const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
+                u += ge - gb;
                 const int rb = tile % p.row_blocks, mt = tile / p.row_blocks;
                 const int tiles_here = min(8, (N >> 4) - 8 * rb);
-                for (int j = 0; j < G && ok; ++j) {
+                for (int j = gb; j < ge && ok; ++j) {
                     // activations of the group
                     if (!g::mbar_wait(x_empty(sx), phx ^ 1u, abort)) { ok = false; break; }
                     g::mbar_expect_tx(x_full(sx), C::XSTAGE);
@@ -317,10 +334,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
             int sx = 0, sa = 0;
             uint32_t phx = 0, pha = 0, phd = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (long long u = u0; u < u1 && ok;) {
+                const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
+                const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
+                u += ge - gb;
                 if (!g::mbar_wait(d_empty, phd ^ 1u, abort)) { ok = false; break; }   // epilogue has drained D
                 g::tc_fence_after();
-                for (int j = 0; j < G; ++j) {
+                for (int j = gb; j < ge; ++j) {
                     if (!g::mbar_wait(x_full(sx), phx, abort) || !g::mbar_wait(a_full(sa), pha, abort)) { ok = false; break; }
                     g::tc_fence_after();
                     const uint32_t xs = sbase + sx * C::XSTAGE;
@@ -328,7 +348,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint64_t bdesc = sw128_kmajor_desc(xs + (ks >> 2) * C::XBOX + (ks & 3) * 32);
-                        g::umma_f16_ts(tmem, a_t + 8 * ks, bdesc, idesc, (j | ks) != 0 ? 1u : 0u);
+                        g::umma_f16_ts(tmem, a_t + 8 * ks, bdesc, idesc, (j > gb || ks != 0) ? 1u : 0u);
                     }
                     g::tc_commit(x_empty(sx));
                     g::tc_commit(a_empty(sa));
@@ -347,10 +367,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         int sp = 0, sa = 0;
         uint32_t php = 0, pha = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (long long u = u0; u < u1 && ok;) {
+            const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
+            const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
+            u += ge - gb;
             const int rb = tile % p.row_blocks;
             const bool row_ok = kRowsPerCta * rb + r < N;
-            for (int j = 0; j < G; ++j) {
+            for (int j = gb; j < ge; ++j) {
                 if (!g::mbar_wait(p_full(sp), php, abort)) { ok = false; break; }
                 const int b = p.gt.bits[j];
                 const uint32_t stage = sbase + C::OFF_P + sp * kPStageBytes;
@@ -395,30 +418,105 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
+        // A segment that covers its whole tile is stored as fp16.  With stream-K a tile may be cut:
+        // the CTA whose segment does not start the tile leaves its fp32 partial in its workspace
+        // slot and raises its flag; the CTA that starts the tile (it reaches that segment last, the
+        // others reach theirs first) waits for those flags, adds the partials in CTA order and
+        // stores the tile.
         const int q = warp & 3;
+        const int et = tid - 320;                               // 0..127 among the epilogue threads
         uint32_t phd = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        auto epi_sync = [] { asm volatile("bar.sync 1, 128;" ::: "memory"); };
+        for (long long u = u0; u < u1 && ok;) {
+            const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
+            const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
+            u += ge - gb;
             const int rb = tile % p.row_blocks, mt = tile / p.row_blocks;
             const int n = kRowsPerCta * rb + 32 * q + lane;
+            const bool is_partial = gb > 0;
+            // peers: the CTAs after this one, up to the one that ends the tile (CTAs with an empty
+            // range take no part)
+            int npeer = 0;
+            if (!is_partial && ge < G) {
+                for (int pc = blockIdx.x + 1; pc < static_cast<int>(gridDim.x); ++pc) {
+                    ++npeer;
+                    if (range_begin(pc + 1) >= static_cast<long long>(tile + 1) * G) break;
+                }
+            }
+            auto peer_active = [&](int k) { return range_begin(blockIdx.x + k) < range_begin(blockIdx.x + k + 1); };
             if (!g::mbar_wait(d_full, phd, abort)) { ok = false; break; }
             g::tc_fence_after();
+            if (npeer > 0) {
+                if (et == 0) {
+                    const unsigned long long t0 = g::global_timer_ns();
+                    for (int k = 1; k <= npeer; ++k) {
+                        if (!peer_active(k)) continue;
+                        volatile unsigned int* f = p.flags + blockIdx.x + k;
+                        while (*f == 0u) {
+                            if (*abort != 0 || g::global_timer_ns() - t0 > kGemmWaitNs) { *abort = 1; break; }
+                        }
+                    }
+                    __threadfence();
+                }
+                epi_sync();
+                if (*abort != 0) { ok = false; break; }
+            }
+            // slot layout [token][row]: a warp touches 32 consecutive floats per access
+            float* my_slot = p.partials + static_cast<size_t>(blockIdx.x) * (TOK * kRowsPerCta) + 32 * q + lane;
+            if (is_partial) {
 #pragma unroll 1
-            for (int cc = 0; cc < TOK / 32; ++cc) {
-                uint32_t v[32];
-                g::tmem_ld32(tmem + (static_cast<uint32_t>(32 * q) << 16) + 32 * cc, v);
-                g::tc_wait_ld();
-                const int m0 = mt * TOK + 32 * cc;
-                if (n < N) {
+                for (int cc = 0; cc < TOK / 32; ++cc) {
+                    uint32_t v[32];
+                    g::tmem_ld32(tmem + (static_cast<uint32_t>(32 * q) << 16) + 32 * cc, v);
+                    g::tc_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (m0 + i < p.M) p.y[static_cast<size_t>(m0 + i) * N + n] = __float2half_rn(__uint_as_float(v[i]));
+                    for (int i = 0; i < 32; ++i) my_slot[(32 * cc + i) * kRowsPerCta] = __uint_as_float(v[i]);
+                }
+            } else {
+                // sum of the peers' partials for one 32-token chunk, in CTA order
+                auto peer_sum = [&](int cc, float (&t)[32]) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) t[i] = 0.f;
+                    for (int k = 1; k <= npeer; ++k) {
+                        if (!peer_active(k)) continue;
+                        const float* slot = p.partials + static_cast<size_t>(blockIdx.x + k) * (TOK * kRowsPerCta) + 32 * q + lane;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) t[i] += __ldcg(slot + (32 * cc + i) * kRowsPerCta);
+                    }
+                };
+                float t[32];
+                if (npeer > 0) peer_sum(0, t);
+#pragma unroll 1
+                for (int cc = 0; cc < TOK / 32; ++cc) {
+                    uint32_t v[32];
+                    g::tmem_ld32(tmem + (static_cast<uint32_t>(32 * q) << 16) + 32 * cc, v);
+                    g::tc_wait_ld();
+                    if (npeer > 0) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + t[i]);
+                        if (cc + 1 < TOK / 32) peer_sum(cc + 1, t);     // in flight while this chunk is stored
+                    }
+                    const int m0 = mt * TOK + 32 * cc;
+                    if (n < N) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (m0 + i < p.M) p.y[static_cast<size_t>(m0 + i) * N + n] = __float2half_rn(__uint_as_float(v[i]));
+                    }
                 }
             }
             g::tc_fence_before();
             __syncwarp();
             if (lane == 0) g::mbar_arrive(d_empty);
             phd ^= 1u;
+            if (is_partial) {
+                __threadfence();
+                epi_sync();
+                if (et == 0) { __threadfence(); *(volatile unsigned int*)(p.flags + blockIdx.x) = 1u; }
+            } else if (npeer > 0) {
+                epi_sync();                                     // everyone has read the peers' slots
+                if (et < npeer) p.flags[blockIdx.x + 1 + et] = 0u;   // ready for the next launch (unused ones are 0 already)
+            }
         }
     }
 
@@ -467,8 +565,39 @@ static int gemm_sm_count() {
     return n;
 }
 
+// Launch shape shared by the entry point and the workspace query.  Stream-K (equal shares of
+// (tile, group) units per CTA, partial tiles combined through the workspace) is used when it is
+// predicted to beat whole tiles, whose last wave may leave most SMs idle.
+struct GemmPlan {
+    int tok, row_blocks, tok_tiles, grid, stream_k;
+    size_t workspace_bytes;
+};
+static GemmPlan plan_gemm(int M, int N, int G) {
+    GemmPlan pl;
+    pl.tok = M <= 128 ? 128 : 256;
+    pl.row_blocks = (N + kRowsPerCta - 1) / kRowsPerCta;
+    pl.tok_tiles = (M + pl.tok - 1) / pl.tok;
+    const int tiles = pl.row_blocks * pl.tok_tiles;
+    int sms = gemm_sm_count();
+    if (sms > kGemmMaxGrid) sms = kGemmMaxGrid;
+    pl.grid = tiles < sms ? tiles : sms;
+    const int waves = (tiles + sms - 1) / sms;
+    (void)waves;
+    pl.stream_k = 0;
+    // time in units of one group: whole tiles take waves * G; equal shares take units / SMs plus
+    // about two dozen groups' worth of draining, storing and re-reading a partial tile (measured)
+    const long long units = static_cast<long long>(tiles) * G;
+    if (units >= 8ll * sms && static_cast<double>(units) / sms + 24.0 < 0.95 * static_cast<double>(waves) * G) {
+        pl.stream_k = 1;
+        pl.grid = sms;
+    }
+    pl.workspace_bytes = pl.stream_k ? kGemmWsPartials + static_cast<size_t>(pl.grid) * pl.tok * kRowsPerCta * sizeof(float) : 256;
+    return pl;
+}
+size_t gemm_workspace_bytes(int M, int N, int G) { return plan_gemm(M, N, G).workspace_bytes; }
+
 template <int TOK>
-static cudaError_t launch_gemm(const CUtensorMap& map, const GemmParams& prm, cudaStream_t stream) {
+static cudaError_t launch_gemm(const CUtensorMap& map, const GemmParams& prm, int grid, cudaStream_t stream) {
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -478,9 +607,6 @@ static cudaError_t launch_gemm(const CUtensorMap& map, const GemmParams& prm, cu
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    const int tiles = prm.row_blocks * prm.tok_tiles;
-    const int sms = gemm_sm_count();
-    const int grid = tiles < sms ? tiles : sms;
     gemm_kernel<TOK><<<grid, kGemmThreads, GemmCfg<TOK>::SMEM, stream>>>(map, prm);
     return cudaGetLastError();
 }
@@ -508,7 +634,13 @@ extern "C" int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* b
     if (workspace == nullptr || workspace_bytes < 256) return SLIM_ERR_WORKSPACE;
     if (!slim::aligned16(workspace)) return SLIM_ERR_ALIGNMENT;
 
-    const int tok = M <= 128 ? 128 : 256;
+    slim::GemmPlan pl = slim::plan_gemm(M, N, gt.G);
+    if (pl.stream_k && workspace_bytes < pl.workspace_bytes) {   // small workspace: whole tiles, no scratch
+        pl.stream_k = 0;
+        const int tiles = pl.row_blocks * pl.tok_tiles;
+        if (pl.grid > tiles) pl.grid = tiles;
+    }
+    const int tok = pl.tok;
     CUtensorMap map;
     if (!slim::make_x_map(&map, x, M, K, tok)) {
         slim::set_cuda_error(cudaErrorUnknown);
@@ -522,10 +654,13 @@ extern "C" int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* b
     prm.y = static_cast<__half*>(y);
     prm.status = static_cast<unsigned int*>(workspace);
     prm.M = M; prm.N = N; prm.K = K;
-    prm.row_blocks = (N + slim::kRowsPerCta - 1) / slim::kRowsPerCta;
-    prm.tok_tiles = (M + tok - 1) / tok;
+    prm.flags = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(workspace) + slim::kGemmWsFlags);
+    prm.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + slim::kGemmWsPartials);
+    prm.row_blocks = pl.row_blocks;
+    prm.tok_tiles = pl.tok_tiles;
+    prm.stream_k = pl.stream_k;
     prm.gt = gt;
-    const cudaError_t e = tok == 128 ? slim::launch_gemm<128>(map, prm, s) : slim::launch_gemm<256>(map, prm, s);
+    const cudaError_t e = tok == 128 ? slim::launch_gemm<128>(map, prm, pl.grid, s) : slim::launch_gemm<256>(map, prm, pl.grid, s);
     SLIM_CUDA_TRY(e);
     return SLIM_OK;
 }

@@ -533,7 +533,7 @@ int slim_workspace_bytes(int M, int N, int K, int g, const uint8_t* bits_host, s
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;
-    *out_bytes = slim::kWsHeader;
+    *out_bytes = (M > SLIM_GEMV_MAX_M && N > 0) ? slim::gemm_workspace_bytes(M, N, gt.G) : static_cast<size_t>(slim::kWsHeader);
     return SLIM_OK;
 }
 

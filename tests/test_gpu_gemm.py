@@ -79,6 +79,28 @@ def test_13b_shapes_full_size_sampled_rows(N, K, M):
     assert np.isfinite(y.astype(np.float64)).all()
 
 
+def test_stream_k_and_whole_tile_paths_agree():
+    """A shape whose tile count leaves the last wave half empty takes the stream-K path when the
+    workspace is large enough and whole tiles when it is not; both must match the oracle."""
+    slim = _slim()
+    L = oracle_layer(5120, 13824, 3, 512)         # 40 row blocks x 2 token tiles = 80 tiles on 148 SMs
+    assert slim.workspace_bytes(512, 5120, 13824, L["bits"]) > 1 << 20
+    packed = torch.from_numpy(orc.pack(L["codes"], L["bits"])).cuda()
+    sc, zp, x = (torch.from_numpy(L[k]).cuda() for k in ("scales", "zeros", "x"))
+    big = slim.new_workspace(512, 5120, 13824, L["bits"])
+    small = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    ys = []
+    for ws in (big, small, big):                   # the large workspace is used twice: its flags must be reusable
+        ys.append(slim.mpq_gemm(x, packed, L["bits"], sc, zp, 5120, ws).cpu().numpy())
+        slim.workspace_status(ws)
+    rows = np.unique(np.concatenate([[0, 127, 128, 5119], np.random.default_rng(2).integers(0, 5120, 100)]))
+    y_ref = orc.linear_rows_f64(L["x"], L["codes"], L["scales"], L["zeros"], rows)
+    for y in ys:
+        check_output(y[:, rows], y_ref, "5120x13824 M=512")
+    assert (ys[0].view(np.uint16) == ys[2].view(np.uint16)).all()
+    assert np.abs(ys[0].astype(np.float64) - ys[1].astype(np.float64)).max() <= 2e-3 * np.abs(ys[1].astype(np.float64)).max()
+
+
 def test_argument_errors_are_statuses():
     slim = _slim()
     L = oracle_layer(128, 256, 2, 1)
