@@ -59,7 +59,8 @@ enum {
     SLIM_ERR_ALIGNMENT = -3,   /* a device pointer is not 16-byte aligned */
     SLIM_ERR_WORKSPACE = -4,   /* workspace missing or smaller than slim_workspace_bytes() */
     SLIM_ERR_CUDA = -5,        /* a CUDA runtime call failed; see slim_last_cuda_error() */
-    SLIM_ERR_TIMEOUT = -6      /* a device-side wait gave up (reported by slim_workspace_status) */
+    SLIM_ERR_TIMEOUT = -6,     /* a device-side wait gave up (reported by slim_workspace_status) */
+    SLIM_ERR_STATIC_SCRATCH = -7 /* slim_mpq_gemm_static: the shape needs more than the built-in scratch */
 };
 
 /* Library / format version: (SLIM_FORMAT_VERSION << 16) | build number. */
@@ -125,6 +126,32 @@ int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* bits_host,
                   const void* scales, const void* zeros, void* y,
                   int M, int N, int K, int g,
                   void* workspace, size_t workspace_bytes, void* stream);
+
+/* slim_mpq_gemm for callers that must not allocate device memory.  (The paper has no counterpart
+ * of this entry point; it exists for deployment.)  Typical callers: the enqueue callback of an
+ * inference-engine plugin, which is handed input and output pointers and a stream and nothing
+ * else, and serving loops whose memory budget was handed out at start-up, where a cudaMalloc would
+ * stall every stream of the device or fail late.  Such callers have no workspace to pass.
+ *
+ * Same arithmetic and arguments as slim_mpq_gemm, except that the scratch (status word, stream-K
+ * flags and fp32 partial tiles) is a fixed array inside the library: SLIM_STATIC_SCRATCH_MAX bytes
+ * of device memory on every GPU that loads the library, held until the process exits.  The call
+ * allocates and frees nothing.  A shape that would need more scratch on the current device (only
+ * possible on a GPU with more than 148 SMs) returns SLIM_ERR_STATIC_SCRATCH and enqueues nothing.
+ *
+ * All calls on a device share that array.  Each call first clears the control words on `stream`,
+ * then runs; two calls whose kernels can overlap on the GPU (different streams, no ordering) race
+ * on it and give undefined results, so keep the calls of a device on one stream or order them.
+ * The first call on each device looks up the array's device address (a driver query, no
+ * allocation); make that first call outside any stream capture.
+ *
+ * status_out: optional device pointer to one 32-bit word (4-byte aligned, may be NULL).  After
+ * the call's work completes it holds 0, or 1 if a device-side wait gave up (y is then undefined);
+ * it plays the part slim_workspace_status plays for a caller-owned workspace. */
+#define SLIM_STATIC_SCRATCH_MAX (1280 + 148 * 256 * 128 * 4)
+int slim_mpq_gemm_static(const void* x, const void* packed, const uint8_t* bits_host,
+                         const void* scales, const void* zeros, void* y,
+                         int M, int N, int K, int g, unsigned int* status_out, void* stream);
 
 /* ---- producing the inputs of the layer (the steps right before packing) ------------------- */
 

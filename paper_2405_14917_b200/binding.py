@@ -53,6 +53,7 @@ def lib():
             "slim_mpq_gemv": [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp],
             "slim_mpq_gemm": [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp],
             "slim_gemv_plan": [i, i, i, i, vp, vp],
+            "slim_mpq_gemm_static": [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, vp],
             "slim_group_salience": [vp, vp, vp, i, i, i, vp],
             "slim_allocate_bits": [vp, i, i, i, vp],
             "slim_quantize_minmax": [vp, vp, vp, vp, vp, i, i, i, vp],
@@ -178,6 +179,22 @@ def mpq_gemv(x, packed, bits, scales, zeros, N: int, workspace, out=None) -> tor
 def mpq_gemm(x, packed, bits, scales, zeros, N: int, workspace, out=None) -> torch.Tensor:
     """y = x W-hat^T for M > 16 (batched tensor-core path)."""
     return _linear("slim_mpq_gemm", x, packed, bits, scales, zeros, N, workspace, out)
+
+
+def mpq_gemm_static(x, packed, bits, scales, zeros, N: int, out: torch.Tensor, status: torch.Tensor | None = None) -> torch.Tensor:
+    """slim_mpq_gemm without a caller workspace: the library's built-in scratch array is used.
+
+    For callers that may not allocate device memory, so `out` (fp16 [M][N]) and the optional
+    `status` (one int32 word on the device) must be passed in; nothing is allocated here either.
+    Calls on one device share the scratch: keep them on one stream.
+    """
+    b = _bits(bits)
+    M, K = x.shape
+    sp = _dev(status, torch.int32, "status") if status is not None else None
+    _check("slim_mpq_gemm_static", lib().slim_mpq_gemm_static(
+        _dev(x, torch.float16, "x"), _dev(packed, torch.uint8, "packed"), _bp(b), _dev(scales, torch.float16, "scales"),
+        _dev(zeros, torch.float16, "zeros"), _dev(out, torch.float16, "y"), M, N, K, GROUP, sp, _stream(x)))
+    return out
 
 
 def group_salience(W: torch.Tensor, act_norm: torch.Tensor) -> torch.Tensor:

@@ -49,6 +49,7 @@ const char* slim_status_string(int status) {
         case SLIM_ERR_WORKSPACE: return "workspace missing or too small";
         case SLIM_ERR_CUDA: return "CUDA runtime error";
         case SLIM_ERR_TIMEOUT: return "device-side wait timed out";
+        case SLIM_ERR_STATIC_SCRATCH: return "shape needs more scratch than the library's built-in array holds";
         default: return "unknown status";
     }
 }

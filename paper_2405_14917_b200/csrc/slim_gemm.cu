@@ -664,3 +664,44 @@ extern "C" int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* b
     SLIM_CUDA_TRY(e);
     return SLIM_OK;
 }
+
+// ------------------------------------------------------------------------------------------ no-allocation variant
+// Built-in scratch for slim_mpq_gemm_static: the control words plus one fp32 partial tile per CTA
+// of a 148-SM device.  It lives in every GPU that loads the library, for the life of the process.
+static_assert(SLIM_STATIC_SCRATCH_MAX == slim::kGemmWsPartials + 148 * 256 * slim::kRowsPerCta * 4, "scratch size");
+static __device__ __align__(256) unsigned char g_static_scratch[SLIM_STATIC_SCRATCH_MAX];
+
+extern "C" int slim_mpq_gemm_static(const void* x, const void* packed, const uint8_t* bits_host, const void* scales,
+                                    const void* zeros, void* y, int M, int N, int K, int g,
+                                    unsigned int* status_out, void* stream) {
+    if (M < 0 || (M > 0 && M <= SLIM_GEMV_MAX_M)) return SLIM_ERR_INVALID_ARG;
+    slim::GroupTable gt;
+    const int st = slim::make_group_table(N, K, g, bits_host, &gt);
+    if (st != SLIM_OK) return st;
+    if (status_out != nullptr && (reinterpret_cast<uintptr_t>(status_out) & 3u) != 0) return SLIM_ERR_ALIGNMENT;
+    if (M == 0 || N == 0 || K == 0)   // nothing needs scratch: the ordinary entry point handles these
+        return slim_mpq_gemm(x, packed, bits_host, scales, zeros, y, M, N, K, g, nullptr, 0, stream);
+    // what this shape wants on this device; more than the array holds is refused, never truncated
+    if (slim::gemm_workspace_bytes(M, N, gt.G) > static_cast<size_t>(SLIM_STATIC_SCRATCH_MAX)) return SLIM_ERR_STATIC_SCRATCH;
+
+    // Device address of the array, looked up once per device (the array's name is only a
+    // host-side handle here and must not be handed to a kernel).
+    static void* scratch_ptr[64] = {nullptr};
+    int dev = 0;
+    SLIM_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return SLIM_ERR_UNSUPPORTED;
+    if (scratch_ptr[dev] == nullptr) {
+        void* ptr = nullptr;
+        SLIM_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        scratch_ptr[dev] = ptr;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the array keeps what the last call left: the status word and the flags must start at zero
+    SLIM_CUDA_TRY(cudaMemsetAsync(scratch_ptr[dev], 0, slim::kGemmWsPartials, s));
+    const int rc = slim_mpq_gemm(x, packed, bits_host, scales, zeros, y, M, N, K, g, scratch_ptr[dev],
+                                 SLIM_STATIC_SCRATCH_MAX, stream);
+    if (rc != SLIM_OK) return rc;
+    if (status_out != nullptr)
+        SLIM_CUDA_TRY(cudaMemcpyAsync(status_out, scratch_ptr[dev], sizeof(unsigned int), cudaMemcpyDeviceToDevice, s));
+    return SLIM_OK;
+}

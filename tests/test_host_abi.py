@@ -39,7 +39,7 @@ def test_library_exports_every_declared_symbol(slim):
 def test_version_and_status_strings(slim):
     assert slim.version() >> 16 == 2
     L = slim.lib()
-    for code in range(0, -7, -1):
+    for code in range(0, -8, -1):
         assert L.slim_status_string(code).decode() not in ("", "unknown status")
     assert L.slim_status_string(-99).decode() == "unknown status"
 
