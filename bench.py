@@ -40,9 +40,9 @@ FALLBACK_TENSOR_TFLOPS = 1400.0
 # dram__bytes_write.sum), keyed by the sha256 of the kernel source it was taken from.  A kernel
 # that has changed since reports null.
 NCU_TRAFFIC = {
-    # 4096x4096 layer, avg 2-bit, M = 1: 4,759,808 B read + 0 written per launch (algorithmic 4,735,008 B);
+    # 4096x4096 layer, avg 2-bit, M = 1: 4,755,200 B read + 0 written per launch (algorithmic 4,735,008 B);
     # scaled to the sweep's average launch by the algorithmic bytes (traffic grows with the layer size)
-    "6b2aa44167417399c395aecc4c7a8801c023f59a66e454ef099c876e580ddeed": {"layer": "4096x4096", "traffic_bytes": 4759808, "algorithmic_bytes": 4735008},
+    "b224ffa6096f3c804842f14517aae781ba1a60137dc5da479ed292a207368224": {"layer": "4096x4096", "traffic_bytes": 4755200, "algorithmic_bytes": 4735008},
 }
 
 
@@ -55,6 +55,13 @@ def workload_spec(name: str):
         return dict(model="llama-7b", avg_bits=2, M=1, n_blocks=4)
     if name.startswith("llama13b-prefill-avg3-m"):    # batched tensor-core path, two blocks (14 layers)
         return dict(model="llama-13b", avg_bits=3, M=int(name.rsplit("m", 1)[1]), n_blocks=2)
+    # other decode configurations: <model>-decode-avg<bits>-m<M>[-blocks<n>], model in llama7b / llama70b
+    import re
+    m = re.fullmatch(r"(llama7b|llama70b)-decode-avg([23])-m(\d+)(?:-blocks(\d+))?", name)
+    if m:
+        model = {"llama7b": "llama-7b", "llama70b": "llama-2-70b"}[m.group(1)]
+        blocks = int(m.group(4)) if m.group(4) else (wl.N_BLOCKS[model] if model == "llama-7b" else 8)
+        return dict(model=model, avg_bits=int(m.group(2)), M=int(m.group(3)), n_blocks=blocks)
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -377,11 +384,13 @@ def run_ours(args, spec):
     sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2405_14917_b200", "csrc", "slim_gemv.cu"), "rb").read()).hexdigest()
     traffic = NCU_TRAFFIC.get(sha)
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "metric": METRIC if args.workload == "llama7b-decode-avg2" else
+                  f"mixed-precision dequant GEMV GB/s at M={M} ({spec['model']} layer set, avg {spec['avg_bits']}-bit, g=128)",
+        "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f16 (mma.sync m16n8k16 on raw code fields, f32 accumulate)", "data": "synthetic",
         "config": {"workload": args.workload, "layers": n_launch, "M": M, "avg_bits": spec["avg_bits"], "g": wl.GROUP,
-                   "algorithmic_bytes_per_step": alg_bytes, "l2": "distinct layers, 1.8 GB per step >> L2",
+                   "algorithmic_bytes_per_step": alg_bytes, "l2": f"distinct layers, {alg_bytes / 1e9:.2f} GB per step >> L2",
                    "launch": "CUDA graph of one launch per layer, programmatic dependent launch",
                    "parallelism": f"replicas x{world}"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
