@@ -42,7 +42,7 @@ FALLBACK_TENSOR_TFLOPS = 1400.0
 NCU_TRAFFIC = {
     # 4096x4096 layer, avg 2-bit, M = 1: 4,755,200 B read + 0 written per launch (algorithmic 4,735,008 B);
     # scaled to the sweep's average launch by the algorithmic bytes (traffic grows with the layer size)
-    "b224ffa6096f3c804842f14517aae781ba1a60137dc5da479ed292a207368224": {"layer": "4096x4096", "traffic_bytes": 4755200, "algorithmic_bytes": 4735008},
+    "4b06a5d5b512621bbe525cb3d0c66822ff452c130a671af895469c10fb834593": {"layer": "4096x4096", "traffic_bytes": 4755200, "algorithmic_bytes": 4735008},
 }
 
 

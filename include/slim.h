@@ -75,7 +75,9 @@ int slim_last_cuda_error(void);
 int slim_packed_bytes(int N, int K, int g, const uint8_t* bits_host, size_t* out_bytes);
 
 /* Scratch size for slim_mpq_gemv / slim_mpq_gemm with these shapes on the current device.
- * Always at least 256 (one status word).  slim_mpq_gemv needs no more.  slim_mpq_gemm asks for
+ * Always at least 256 (one status word).  slim_mpq_gemv needs no more up to three tokens; from
+ * four tokens on it asks for room to put x into tensor-core fragment order once (a few bytes
+ * per element of x) and, given less, lets every thread block do that for itself.  slim_mpq_gemm asks for
  * flags and fp32 partial tiles (128 KB per SM) when it would split tiles across CTAs (stream-K:
  * shapes whose tile count leaves the last wave of CTAs mostly idle); given a smaller workspace
  * (at least 256 bytes) it falls back to whole tiles per CTA and uses no scratch. */

@@ -42,6 +42,7 @@ namespace slim {
 constexpr int kMaxWarps = 8;
 constexpr int kMaxCluster = 8;
 constexpr int kWsHeader = 256;              // status word + padding
+constexpr int kPreStageMinM = 4;            // from this many tokens on, x is put into fragment order by a kernel of its own
 
 struct GemvParams {
     const __half* x;
@@ -49,6 +50,8 @@ struct GemvParams {
     const __half* scales;
     const __half* zeros;
     __half* y;
+    const uint8_t* xs_g;    // pre-staged B fragments [slot][8 mma][M][4 lanes] x 8 B (pre-staged mode)
+    const float2* sxe_g;    // pre-staged (sum_k x, 2^(24-S)) [G][16] (pre-staged mode)
     int M, N, K;
     int CS;                 // k-slices (= cluster size)
     int W;                  // warps per CTA
@@ -146,24 +149,84 @@ struct SmemMap {
 __host__ __device__ inline uint32_t align_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
 // Output pairs (two rows of one token) a CTA owns in the cluster reduction.
 __host__ __device__ inline int cluster_share(int T, int M, int CS) { return (T * M * 8 + CS - 1) / CS; }
-__host__ __device__ inline SmemMap make_smem_map(int M, int W, int T, int CS, int GC, int region_bytes, int max_slots, bool two_bufs) {
+// `pre`: x arrives already in fragment order (no raw x; fragments and sums double-buffered instead).
+__host__ __device__ inline SmemMap make_smem_map(int M, int W, int T, int CS, int GC, int region_bytes, int max_slots, bool two_bufs,
+                                                 bool pre) {
     SmemMap m;
     uint32_t o = 0;
-    m.sxe = o;   o += 128u * GC;
+    m.sxe = o;   o += (pre && two_bufs ? 2u : 1u) * 128u * GC;
     m.red = o;   o += 64u * W * M;
     m.cred = o;  o += CS > 1 ? 8u * CS * cluster_share(T, M, CS) : 0u;
     o = align_up(o, 16);
-    m.xraw = o;  o += (two_bufs ? 2u : 1u) * (256u * M * GC);
+    m.xraw = o;  o += pre ? 0u : (two_bufs ? 2u : 1u) * (256u * M * GC);
     o = align_up(o, 128);
-    m.xs = o;    o += static_cast<uint32_t>(max_slots) * 8 * M * 32;
+    m.xs = o;    o += (pre && two_bufs ? 2u : 1u) * static_cast<uint32_t>(max_slots) * 8 * M * 32;
     o = align_up(o, 128);
     m.wbuf = o;  o += (two_bufs ? 2u : 1u) * region_bytes;
     m.total = o;
     return m;
 }
 
-// ------------------------------------------------------------------------------------------ kernel
-template <int NT>   // 8-token MMA tiles: 1 (M <= 8) or 2
+// ------------------------------------------------------------------------------------------ kernels
+// Puts the 128 activations of one (token m, group) into B-fragment order for every slice of the
+// group (lane = (mma mi, lane column cc) -> the four activations that meet that lane's two B
+// registers) and returns the group's (sum_k x, 2^(24-S)) in lane 0.  xg: the group's 128 halves
+// (shared or global); xs_slot0: first fragment slot of the group (shared or global).
+__device__ __forceinline__ float2 stage_group(const __half* xg, uint8_t* xs_slot0, int b, int m, int M, int lane) {
+    // 2^S lifts the group's largest |x| into [2^13, 2^14) (Inf/NaN: the top binade)
+    const uint2 raw = *reinterpret_cast<const uint2*>(xg + 4 * lane);
+    uint32_t mx = max(max(raw.x & 0x7fffu, (raw.x >> 16) & 0x7fffu), max(raw.y & 0x7fffu, (raw.y >> 16) & 0x7fffu));
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    const int S = mx == 0 ? 0 : 28 - max(static_cast<int>(mx >> 10), 1);
+    const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+    const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+    float sum = (f01.x + f01.y) + (f23.x + f23.y);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const int cc = lane & 3, mi = lane >> 2;
+    const int ns = slice_count(b);
+    for (int s = 0; s < ns; ++s) {
+        const int w = slice_w(b, s), lo = slice_lo(b, s);
+        const int lg = w >> 1;                          // log2(w) for w in {1,2,4}
+        const int nf = 32 >> lg;                        // fields per word; 8/w MMAs per unit
+        const int u = mi >> (3 - lg), ii = mi & ((8 >> lg) - 1);
+        const __half* xp = xg + 32 * cc + nf * u + 2 * ii;
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(xp));               // pairs 2ii, 2ii+1: first field
+        const float2 g = __half22float2(*reinterpret_cast<const __half2*>(xp + (nf >> 1)));   // ... second field
+        const float sc0 = __int_as_float((127 + S + lo - pair_pos(w, 2 * ii)) << 23);
+        const float sc1 = __int_as_float((127 + S + lo - pair_pos(w, 2 * ii + 1)) << 23);
+        const __half2 b0 = __floats2half2_rn(f.x * sc0, g.x * sc0);
+        const __half2 b1 = __floats2half2_rn(f.y * sc1, g.y * sc1);
+        *reinterpret_cast<uint2*>(xs_slot0 + (((static_cast<size_t>(s) * 8 + mi) * M + m) * 4 + cc) * 8) =
+            make_uint2(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1));
+    }
+    return make_float2(sum, __int_as_float((127 + 24 - S) << 23));
+}
+
+// Pre-staging kernel (M >= kPreStageMinM): one warp per (token, group) writes the fragments and
+// sums of the whole x to global scratch once, instead of every row block repeating the work.
+struct StageParams {
+    const __half* x;
+    uint8_t* xs_g;
+    float2* sxe_g;
+    int M, K, G;
+    uint16_t pre3[SLIM_MAX_GROUPS + 1];
+    uint8_t bits[SLIM_MAX_GROUPS];
+};
+__global__ void __launch_bounds__(256) gemv_stage_x_kernel(const __grid_constant__ StageParams p) {
+    pdl_launch_dependents();
+    pdl_wait();                                          // x may come from the previous kernel
+    const int lane = threadIdx.x & 31;
+    const int pi = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (pi >= p.M * p.G) return;
+    const int m = pi / p.G, j = pi - m * p.G;
+    const float2 r = stage_group(p.x + static_cast<size_t>(m) * p.K + j * SLIM_GROUP,
+                                 p.xs_g + static_cast<size_t>(j + p.pre3[j]) * 8 * p.M * 32, p.bits[j], m, p.M, lane);
+    if (lane == 0) p.sxe_g[j * 16 + m] = r;
+    if (m == 0 && lane < 16 && lane >= p.M) p.sxe_g[j * 16 + lane] = make_float2(0.f, 1.f);   // absent tokens read 0
+}
+
+template <int NT, bool PRE>   // NT 8-token MMA tiles: 1 (M <= 8) or 2; PRE: x arrives pre-staged
 __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_constant__ GemvParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
@@ -179,7 +242,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
     const int g0 = p.kbegin[ks], g1 = p.kbegin[ks + 1];
     const int ng = g1 - g0;
     const int n_chunks = (ng + GC - 1) / GC;
-    const SmemMap sm = make_smem_map(M, W, T, p.CS, GC, p.region_bytes, p.max_slots, p.two_bufs != 0);
+    const SmemMap sm = make_smem_map(M, W, T, p.CS, GC, p.region_bytes, p.max_slots, p.two_bufs != 0, PRE);
+    const uint32_t xs_stride = static_cast<uint32_t>(p.max_slots) * 8 * M * 32;   // bytes per fragment buffer (pre-staged mode)
     const uint32_t xraw_stride = 256u * M * GC;                   // bytes per xraw buffer
     const int tw = warp % T, kw = warp / T;                       // this warp's tile of the CTA and k-way
     const int tile = rb * T + tw;
@@ -211,7 +275,18 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
     };
     // raw activations of chunk `ch` (all tokens) -> xraw buffer ch & 1
     auto issue_x = [&](int ch) {
-        if (ch < n_chunks) {
+        if (PRE && ch < n_chunks) {
+            // fragments and sums of the chunk, already in their final order
+            const int ja = g0 + ch * GC, jb = min(g1, ja + GC);
+            const int s0 = ja + p.pre3[ja], s1 = jb + p.pre3[jb];
+            const int n16 = (s1 - s0) * 16 * M;                            // 16-byte pieces of the fragments
+            const uint32_t dst = sbase + sm.xs + (ch & 1) * xs_stride;
+            const uint8_t* src = p.xs_g + static_cast<size_t>(s0) * 8 * M * 32;
+            for (int q = tid; q < n16; q += nthreads) cp_async16(dst + 16 * q, src + 16 * q);
+            const uint32_t dsx = sbase + sm.sxe + (ch & 1) * 128u * GC;
+            for (int q = tid; q < (jb - ja) * 8; q += nthreads)
+                cp_async16(dsx + 16 * q, reinterpret_cast<const uint8_t*>(p.sxe_g + ja * 16) + 16 * q);
+        } else if (ch < n_chunks) {
             const int ja = g0 + ch * GC, cg = min(g1, ja + GC) - ja;
             const int per_tok = cg * 16;                                   // 16-byte pieces per token
             const uint32_t dst0 = sbase + sm.xraw + (ch & 1) * xraw_stride;
@@ -227,7 +302,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
     issue_weights(0);
     pdl_wait();
     issue_x(0);
-    for (int i = tid; i < 32 * GC; i += nthreads) reinterpret_cast<float*>(smem + sm.sxe)[i] = 0.f;   // absent tokens read 0
+    if (!PRE)
+        for (int i = tid; i < 32 * GC; i += nthreads) reinterpret_cast<float*>(smem + sm.sxe)[i] = 0.f;   // absent tokens read 0
 
     float acc[NT][4];
 #pragma unroll
@@ -239,49 +315,26 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
         const int ja = g0 + ch * GC, cg = min(g1, ja + GC) - ja;
         const int kc = GC * SLIM_GROUP;                                   // xraw row stride (halves)
         const __half* xraw = reinterpret_cast<const __half*>(smem + sm.xraw + (ch & 1) * xraw_stride);
-        float2* sxe = reinterpret_cast<float2*>(smem + sm.sxe);
+        float2* sxe = reinterpret_cast<float2*>(smem + sm.sxe + (PRE ? (ch & 1) * 128u * GC : 0u));
+        const uint32_t xs_buf = sbase + sm.xs + (PRE ? (ch & 1) * xs_stride : 0u);
 
         cp_async_wait_all();             // x and weights of this chunk have landed (this thread's copies)
         __syncthreads();                 // ... everybody's; and the previous chunk is fully consumed
         issue_weights(ch + 1);           // into the buffer the previous chunk has left
-        // ---- activations in B-fragment order: one warp per (token, group) ------------------------------
-        for (int pi = warp; pi < M * cg; pi += W) {
-            const int m = pi / cg, i = pi - m * cg;
-            const __half* xg = xraw + m * kc + i * SLIM_GROUP;
-            // 2^S lifts the group's largest |x| into [2^13, 2^14) (Inf/NaN: the top binade)
-            const uint2 raw = *reinterpret_cast<const uint2*>(xg + 4 * lane);
-            uint32_t mx = max(max(raw.x & 0x7fffu, (raw.x >> 16) & 0x7fffu), max(raw.y & 0x7fffu, (raw.y >> 16) & 0x7fffu));
-            mx = __reduce_max_sync(0xffffffffu, mx);
-            const int S = mx == 0 ? 0 : 28 - max(static_cast<int>(mx >> 10), 1);
-            const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
-            const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
-            float sum = (f01.x + f01.y) + (f23.x + f23.y);
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            if (lane == 0) sxe[i * 16 + m] = make_float2(sum, __int_as_float((127 + 24 - S) << 23));
-            // lane = (mma mi, lane column cc): the four activations that meet one lane's two B registers
-            const int b = p.gt.bits[ja + i];
-            const int slot0 = i + p.pre3[ja + i] - p.pre3[ja];
-            const int cc = lane & 3, mi = lane >> 2;
-            const int ns = slice_count(b);
-            for (int s = 0; s < ns; ++s) {
-                const int w = slice_w(b, s), lo = slice_lo(b, s);
-                const int lg = w >> 1;                          // log2(w) for w in {1,2,4}
-                const int nf = 32 >> lg;                        // fields per word; 8/w MMAs per unit
-                const int u = mi >> (3 - lg), ii = mi & ((8 >> lg) - 1);
-                const __half* xp = xg + 32 * cc + nf * u + 2 * ii;
-                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(xp));               // pairs 2ii, 2ii+1: first field
-                const float2 g = __half22float2(*reinterpret_cast<const __half2*>(xp + (nf >> 1)));   // ... second field
-                const float sc0 = __int_as_float((127 + S + lo - pair_pos(w, 2 * ii)) << 23);
-                const float sc1 = __int_as_float((127 + S + lo - pair_pos(w, 2 * ii + 1)) << 23);
-                const __half2 b0 = __floats2half2_rn(f.x * sc0, g.x * sc0);
-                const __half2 b1 = __floats2half2_rn(f.y * sc1, g.y * sc1);
-                *reinterpret_cast<uint2*>(smem + sm.xs + (((static_cast<size_t>(slot0 + s) * 8 + mi) * M + m) * 4 + cc) * 8) =
-                    make_uint2(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1));
+        if (PRE) {
+            issue_x(ch + 1);             // its fragments and sums too
+        } else {
+            // ---- activations in B-fragment order: one warp per (token, group) --------------------------
+            for (int pi = warp; pi < M * cg; pi += W) {
+                const int m = pi / cg, i = pi - m * cg;
+                const int slot0 = i + p.pre3[ja + i] - p.pre3[ja];
+                const float2 r = stage_group(xraw + m * kc + i * SLIM_GROUP, smem + sm.xs + static_cast<size_t>(slot0) * 8 * M * 32,
+                                             p.gt.bits[ja + i], m, M, lane);
+                if (lane == 0) sxe[i * 16 + m] = r;
             }
+            issue_x(ch + 1);
+            __syncthreads();
         }
-        issue_x(ch + 1);
-        __syncthreads();
 
         // ---- this warp's tile against its groups of the chunk --------------------------------------------
         if (active) {
@@ -289,7 +342,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
             for (int it = kw; it < cg; it += KW) {
                 const int b = p.gt.bits[ja + it];
                 const uint32_t item = item_addr(buf, ja, ja + it, b);
-                const uint32_t xs_slot0 = sbase + sm.xs + static_cast<uint32_t>(it + p.pre3[ja + it] - p.pre3[ja]) * 8 * M * 32;
+                const uint32_t xs_slot0 = xs_buf + static_cast<uint32_t>(it + p.pre3[ja + it] - p.pre3[ja]) * 8 * M * 32;
 
                 float d[2][NT][4];       // two interleaved accumulation chains
 #pragma unroll
@@ -405,6 +458,7 @@ struct GemvPlan {
     int NT, W, T, CS, GC;
     int region_bytes, max_groups, max_slots;
     bool two_bufs;
+    bool pre;                // x pre-staged in global scratch
     uint32_t smem_bytes;
     uint16_t kbegin[kMaxCluster + 1];
 };
@@ -465,8 +519,9 @@ static void size_chunks(const GroupTable& gt, int gc, GemvPlan* pl) {
 // path) and further while the grid is smaller than two CTAs per SM; chunks
 // are as long as shared memory allows while CTAs of consecutive layers can still share an SM.
 // Returns false if a single group does not fit (cannot happen within the documented limits).
-static bool plan_gemv(int M, int N, const GroupTable& gt, GemvPlan* pl) {
+static bool plan_gemv(int M, int N, const GroupTable& gt, bool pre, GemvPlan* pl) {
     const int G = gt.G;
+    pl->pre = pre;
     pl->NT = M <= 8 ? 1 : 2;
     pl->W = kMaxWarps;
     const int sms = device_sm_count();
@@ -487,7 +542,7 @@ static bool plan_gemv(int M, int N, const GroupTable& gt, GemvPlan* pl) {
     for (int bi = 0; bi < 3; ++bi)
         for (int nc = 1; nc <= (bi == 0 && pl->max_groups > 2 ? 2 : pl->max_groups); ++nc) {
             size_chunks(gt, (pl->max_groups + nc - 1) / nc, pl);
-            const uint32_t need = make_smem_map(M, pl->W, pl->T, pl->CS, pl->GC, pl->region_bytes, pl->max_slots, pl->two_bufs).total;
+            const uint32_t need = make_smem_map(M, pl->W, pl->T, pl->CS, pl->GC, pl->region_bytes, pl->max_slots, pl->two_bufs, pl->pre).total;
             if (need > budgets[bi]) continue;
             pl->smem_bytes = need;
             return true;
@@ -495,14 +550,37 @@ static bool plan_gemv(int M, int N, const GroupTable& gt, GemvPlan* pl) {
     return false;
 }
 
-template <int NT>
+// Scratch layout of the pre-staged mode: header, then sums [G][16] float2, then fragments.
+static size_t prestage_sxe_offset() { return kWsHeader; }
+static size_t prestage_xs_offset(int G) { return kWsHeader + static_cast<size_t>(G) * 128; }
+static size_t prestage_bytes(int M, const GroupTable& gt) {
+    int slots = gt.G;
+    for (int j = 0; j < gt.G; ++j) slots += gt.bits[j] == 3 ? 1 : 0;
+    return prestage_xs_offset(gt.G) + static_cast<size_t>(slots) * 8 * M * 32;
+}
+
+static cudaError_t launch_stage_x(const StageParams& sp, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(static_cast<unsigned>((sp.M * sp.G + 7) / 8), 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemv_stage_x_kernel, sp);
+}
+
+template <int NT, bool PRE>
 static cudaError_t launch_gemv(const GemvParams& prm, const GemvPlan& pl, cudaStream_t stream) {
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        e = cudaFuncSetAttribute(gemv_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        e = cudaFuncSetAttribute(gemv_kernel<NT, PRE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
@@ -521,7 +599,7 @@ static cudaError_t launch_gemv(const GemvParams& prm, const GemvPlan& pl, cudaSt
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, gemv_kernel<NT>, prm);
+    return cudaLaunchKernelEx(&cfg, gemv_kernel<NT, PRE>, prm);
 }
 
 }  // namespace slim
@@ -533,7 +611,9 @@ int slim_workspace_bytes(int M, int N, int K, int g, const uint8_t* bits_host, s
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;
-    *out_bytes = (M > SLIM_GEMV_MAX_M && N > 0) ? slim::gemm_workspace_bytes(M, N, gt.G) : static_cast<size_t>(slim::kWsHeader);
+    if (M > SLIM_GEMV_MAX_M && N > 0) *out_bytes = slim::gemm_workspace_bytes(M, N, gt.G);
+    else if (M >= slim::kPreStageMinM && N > 0 && K > 0) *out_bytes = slim::prestage_bytes(M, gt);
+    else *out_bytes = slim::kWsHeader;
     return SLIM_OK;
 }
 
@@ -544,7 +624,7 @@ int slim_gemv_plan(int M, int N, int K, int g, const uint8_t* bits_host, int* ou
     if (st != SLIM_OK) return st;
     if (N == 0 || K == 0) return SLIM_ERR_INVALID_ARG;
     slim::GemvPlan pl;
-    if (!slim::plan_gemv(M, N, gt, &pl)) return SLIM_ERR_UNSUPPORTED;
+    if (!slim::plan_gemv(M, N, gt, M >= slim::kPreStageMinM, &pl)) return SLIM_ERR_UNSUPPORTED;
     out6[0] = pl.T; out6[1] = pl.CS; out6[2] = (N / 16 + pl.T - 1) / pl.T; out6[3] = static_cast<int>(pl.smem_bytes);
     out6[4] = pl.NT; out6[5] = pl.GC;
     return SLIM_OK;
@@ -591,8 +671,11 @@ int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host, c
     if (workspace == nullptr || workspace_bytes < slim::kWsHeader) return SLIM_ERR_WORKSPACE;
     if (!slim::aligned16(workspace)) return SLIM_ERR_ALIGNMENT;
 
+    // From kPreStageMinM tokens on, a small kernel puts x into fragment order once, in the
+    // workspace; with a workspace too small for that every CTA stages its own part of x.
+    const bool pre = M >= slim::kPreStageMinM && workspace_bytes >= slim::prestage_bytes(M, gt);
     slim::GemvPlan pl;
-    if (!slim::plan_gemv(M, N, gt, &pl)) return SLIM_ERR_UNSUPPORTED;
+    if (!slim::plan_gemv(M, N, gt, pre, &pl)) return SLIM_ERR_UNSUPPORTED;
 
     slim::GemvParams prm;
     memset(&prm, 0, sizeof prm);
@@ -616,8 +699,23 @@ int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host, c
     prm.gt = gt;
 
     cudaError_t e;
-    if (pl.NT == 1) e = slim::launch_gemv<1>(prm, pl, s);
-    else e = slim::launch_gemv<2>(prm, pl, s);
+    if (pre) {
+        uint8_t* ws = static_cast<uint8_t*>(workspace);
+        slim::StageParams sp;
+        memset(&sp, 0, sizeof sp);
+        sp.x = prm.x;
+        sp.sxe_g = reinterpret_cast<float2*>(ws + slim::prestage_sxe_offset());
+        sp.xs_g = ws + slim::prestage_xs_offset(gt.G);
+        sp.M = M; sp.K = K; sp.G = gt.G;
+        memcpy(sp.pre3, prm.pre3, sizeof sp.pre3);
+        memcpy(sp.bits, gt.bits, sizeof sp.bits);
+        prm.xs_g = sp.xs_g;
+        prm.sxe_g = sp.sxe_g;
+        SLIM_CUDA_TRY(slim::launch_stage_x(sp, s));
+        e = pl.NT == 1 ? slim::launch_gemv<1, true>(prm, pl, s) : slim::launch_gemv<2, true>(prm, pl, s);
+    } else {
+        e = pl.NT == 1 ? slim::launch_gemv<1, false>(prm, pl, s) : slim::launch_gemv<2, false>(prm, pl, s);
+    }
     SLIM_CUDA_TRY(e);
     return SLIM_OK;
 }

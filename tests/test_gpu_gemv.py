@@ -103,6 +103,23 @@ def test_config_shapes_full_size_sampled_rows(N, K, avg, M):
     assert np.isfinite(y.astype(np.float64)).all()
 
 
+@pytest.mark.parametrize("M", [4, 8, 16])
+def test_small_workspace_stages_x_inside_the_kernel(M):
+    """From four tokens on x is put into fragment order by a kernel of its own, in the workspace;
+    with a 256-byte workspace every CTA stages x itself.  Both paths must match the oracle."""
+    slim = _slim()
+    L = oracle_layer(1024, 2048, 3, M)
+    assert slim.workspace_bytes(M, 1024, 2048, L["bits"]) > 256
+    packed = torch.from_numpy(orc.pack(L["codes"], L["bits"])).cuda()
+    sc, zp, x = (torch.from_numpy(L[k]).cuda() for k in ("scales", "zeros", "x"))
+    y_ref = orc.linear_f64(L["x"], L["codes"], L["scales"], L["zeros"])
+    big = slim.new_workspace(M, 1024, 2048, L["bits"])
+    small = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    for ws in (big, small, big):
+        y = slim.mpq_gemv(x, packed, L["bits"], sc, zp, 1024, ws).cpu().numpy()
+        check_output(y, y_ref, f"M={M} workspace {ws.numel()} B")
+
+
 def test_argument_errors_are_statuses():
     slim = _slim()
     L = oracle_layer(128, 256, 2, 1)
