@@ -14,7 +14,7 @@ says otherwise.
 
 Pinned (tests/test_oracle_*.py): bit budget, quantizer closed forms and brute
 force, packing positions, dequantisation single-rounding, linear layer special
-cases.  Parity unpinned: nothing in this file (the paper's perplexity / accuracy
+cases, the SQC line search (brute force, never worse than tau = 1, exact grids).  Parity unpinned: nothing in this file (the paper's perplexity / accuracy
 / token-per-second tables are not reproduced at all).
 """
 from __future__ import annotations
@@ -104,6 +104,84 @@ def quantize_minmax(W16: np.ndarray, bits: np.ndarray, g: int = GROUP):
         scales[j] = s16
         zeros[j] = z.astype(np.float16)
     return codes, scales, zeros
+
+
+def sqc_tau_grid(lam: float = 0.1, n: int = 50) -> np.ndarray:
+    """Calibration candidates of SQC (Sec. 3.3): [1 - lam, 1 + lam] cut into 2n slices.
+
+    Reading: the 2n candidates are the left ends of the slices, tau_i = 1 - lam + i * lam / n for
+    i = 0 .. 2n-1, so tau = 1 (the plain min-max quantizer) is candidate n.
+    """
+    return 1.0 - lam + np.arange(2 * n, dtype=np.float64) * (lam / n)
+
+
+def salient_mask_3sigma(W16: np.ndarray, g: int = GROUP) -> np.ndarray:
+    """3-sigma mask of Sec. 3.3 per (row, group): w < mu - 3 sigma or w > mu + 3 sigma, with mu and
+    sigma the mean and (population) standard deviation of the group's 128 weights."""
+    N, K = W16.shape
+    w = W16.astype(np.float64).reshape(N, K // g, g)
+    mu = w.mean(axis=2, keepdims=True)
+    sd = w.std(axis=2, keepdims=True)
+    return ((w < mu - 3.0 * sd) | (w > mu + 3.0 * sd)).reshape(N, K)
+
+
+def quantize_sqc(W16: np.ndarray, bits: np.ndarray, g: int = GROUP, lam: float = 0.1, n: int = 50):
+    """Salience-Weighted Quantizer Calibration, function SQC of Algorithm 2, per (row, group).
+
+    For every candidate tau: Delta = tau (w_max - w_min) / (2^b - 1), z = -round(tau w_min / Delta),
+    fake-quantise the salient and the non-salient part of the group with the shared (Delta, z) and
+    keep the candidate with the smallest L_s + L_us (first one on ties: the comparison is strict).
+    Storage readings as in quantize_minmax: the range contains 0, Delta is rounded to fp16 before z,
+    the codes and the losses are computed, a zero Delta becomes 1, z is clamped to [0, 2^b - 1].
+    Losses are fp64 sums of squared errors taken in column order.
+
+    Returns codes uint8 [N][K], scales fp16 [G][N], zeros fp16 [G][N], tau index int32 [G][N],
+    loss fp64 [G][N] (= L_s + L_us of the chosen candidate), salient loss fp64 [G][N] (L_s of it).
+    """
+    N, K = W16.shape
+    G = K // g
+    assert K % g == 0 and len(bits) == G
+    taus = sqc_tau_grid(lam, n)
+    mask = salient_mask_3sigma(W16, g)
+    codes = np.zeros((N, K), dtype=np.uint8)
+    scales = np.zeros((G, N), dtype=np.float16)
+    zeros = np.zeros((G, N), dtype=np.float16)
+    tau_idx = np.zeros((G, N), dtype=np.int32)
+    loss = np.zeros((G, N), dtype=np.float64)
+    loss_s = np.zeros((G, N), dtype=np.float64)
+    for j in range(G):
+        b = int(bits[j])
+        levels = float(2**b - 1)
+        w = W16[:, j * g:(j + 1) * g].astype(np.float64)
+        ms = mask[:, j * g:(j + 1) * g]
+        lo = np.minimum(w.min(axis=1), 0.0)
+        hi = np.maximum(w.max(axis=1), 0.0)
+        best = np.full(N, np.inf)
+        for ti, tau in enumerate(taus):
+            with np.errstate(over="ignore"):
+                s16 = (tau * (hi - lo) / levels).astype(np.float16)
+            s16[np.isinf(s16)] = np.float16(65504.0)
+            s16[s16 == 0] = np.float16(1.0)
+            s = s16.astype(np.float64)
+            z = np.clip(-np.rint(tau * lo / s), 0.0, levels) + 0.0
+            q = np.clip(np.rint(w / s[:, None]) + z[:, None], 0.0, levels)
+            err = w - s[:, None] * (q - z[:, None])
+            sq = err * err
+            L_s = np.zeros(N)
+            L_us = np.zeros(N)
+            for k in range(g):                       # column order, so that every implementation can follow it
+                L_s = L_s + np.where(ms[:, k], sq[:, k], 0.0)
+                L_us = L_us + np.where(ms[:, k], 0.0, sq[:, k])
+            total = L_s + L_us
+            take = total < best
+            best = np.where(take, total, best)
+            codes[take, j * g:(j + 1) * g] = q[take].astype(np.uint8)
+            scales[j, take] = s16[take]
+            zeros[j, take] = z[take].astype(np.float16)
+            tau_idx[j, take] = ti
+            loss[j, take] = total[take]
+            loss_s[j, take] = L_s[take]
+    return codes, scales, zeros, tau_idx, loss, loss_s
 
 
 def quantize_sign_alpha_1bit(W16: np.ndarray, g: int = GROUP):
