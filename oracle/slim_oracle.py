@@ -117,12 +117,22 @@ def sqc_tau_grid(lam: float = 0.1, n: int = 50) -> np.ndarray:
 
 def salient_mask_3sigma(W16: np.ndarray, g: int = GROUP) -> np.ndarray:
     """3-sigma mask of Sec. 3.3 per (row, group): w < mu - 3 sigma or w > mu + 3 sigma, with mu and
-    sigma the mean and (population) standard deviation of the group's 128 weights."""
+    sigma the mean and (population) standard deviation of the group's 128 weights.  Both sums run
+    in column order (the paper fixes no order; a fixed one lets every implementation agree on
+    which elements sit exactly at the threshold)."""
     N, K = W16.shape
     w = W16.astype(np.float64).reshape(N, K // g, g)
-    mu = w.mean(axis=2, keepdims=True)
-    sd = w.std(axis=2, keepdims=True)
-    return ((w < mu - 3.0 * sd) | (w > mu + 3.0 * sd)).reshape(N, K)
+    tot = np.zeros((N, K // g))
+    for k in range(g):
+        tot = tot + w[:, :, k]
+    mu = tot / g
+    var = np.zeros((N, K // g))
+    for k in range(g):
+        d = w[:, :, k] - mu
+        var = var + d * d
+    sd = np.sqrt(var / g)
+    lo, hi = (mu - 3.0 * sd)[:, :, None], (mu + 3.0 * sd)[:, :, None]
+    return ((w < lo) | (w > hi)).reshape(N, K)
 
 
 def quantize_sqc(W16: np.ndarray, bits: np.ndarray, g: int = GROUP, lam: float = 0.1, n: int = 50):
