@@ -245,6 +245,78 @@ def build_layers(spec, device, rank):
     return layers
 
 
+def run_sqc(args):
+    """--workload sqc-llama7b-block: Salience-Weighted Quantizer Calibration (Algorithm 2) of the seven
+    layers of one LLaMA-7B block (202 M weights, avg 2-bit map, lambda = 0.1, n = 50) per step."""
+    import torch
+    from paper_2405_14917_b200 import binding as slim
+    steps = args.steps if args.steps is not None else 20
+    warmup = max(args.warmup if args.warmup is not None else 3, 3)
+    torch.cuda.set_device(0)
+    slim.lib()
+    layers = []
+    for (name, blk, N, K, seed) in wl.model_layers("llama-7b", 1):
+        W, a = wl.make_weight_and_norms_device(seed, N, K, "cuda")
+        bits = slim.allocate_bits(slim.group_salience(W, a).cpu().numpy(), 2)
+        layers.append((W, bits, W.cpu().pin_memory()))
+    weights = sum(W.numel() for W, _, _ in layers)
+
+    def step_device():
+        for W, bits, _ in layers:
+            slim.quantize_sqc(W, bits)
+
+    outs_host = [(torch.empty(W.shape, dtype=torch.uint8).pin_memory(),
+                  torch.empty((W.shape[1] // 128, W.shape[0]), dtype=torch.float16).pin_memory(),
+                  torch.empty((W.shape[1] // 128, W.shape[0]), dtype=torch.float16).pin_memory()) for W, _, _ in layers]
+
+    def step_e2e():
+        for (W, bits, Wh), (ch, sh, zh) in zip(layers, outs_host):
+            W.copy_(Wh, non_blocking=True)
+            codes, scales, zeros, _ = slim.quantize_sqc(W, bits)
+            ch.copy_(codes, non_blocking=True); sh.copy_(scales, non_blocking=True); zh.copy_(zeros, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    def timed(fn, k):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(k):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    for _ in range(warmup):
+        step_device()
+    sampler = ClockSampler(0)
+    sampler.start()
+    ms = timed(step_device, steps)
+    clocks = sampler.stop()
+    for _ in range(3):
+        step_e2e()
+    e2e_steps = max(steps // 4, 3)
+    ms_e2e = timed(step_e2e, e2e_steps)
+    value = weights * steps / (ms * 1e-3) / 1e9
+    # fp64 work: 2n = 100 candidates per weight, 10 fp64 operations each (divide, round, add, min, max,
+    # subtract, multiply, subtract, multiply, add); peak = 148 SMs x 64 fp64 lanes x 1.965 GHz
+    ops = 100 * 10 * weights
+    achieved = ops * steps / (ms * 1e-3) / 1e12
+    peak = 148 * 64 * 1.965e9 / 1e12
+    line = {"metric": "SQC calibration throughput (LLaMA-7B block, 2n = 100 candidates, g=128)", "value": value,
+            "unit": "Gweight/s", "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": ms / steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "layers": len(layers), "weights_per_step": weights, "lambda": 0.1, "n": 50,
+                       "l2": "404 MB of fp16 weights per step > L2"},
+            "roofline": {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "Tinstr/s (fp64 lanes)", "frac": achieved / peak,
+                         "peak_kind": "derived: 148 SMs x 64 fp64 lanes x 1.965 GHz", "kernel": "quantize_sqc_kernel",
+                         "avg_launch_us": 1e3 * ms / steps / len(layers), "traffic": None},
+            "e2e": {"value": weights * e2e_steps / (ms_e2e * 1e-3) / 1e9, "unit": "Gweight/s",
+                    "h2d_bytes_per_step": 2 * weights, "d2h_bytes_per_step": weights + 4 * weights // 128 * 1,
+                    "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
+            "gpu_launches": steps * len(layers), "clocks": clocks}
+    print(json.dumps(line), flush=True)
+
+
 def finish_gemm_line(args, spec, layers, world, steps, warmup, ms, e2e_steps, ms_e2e, x_host, y_host, clocks):
     """JSON line of a batched (M > 16) workload: TFLOP/s against the dense fp16 tensor peak."""
     M = spec["M"]
@@ -419,6 +491,9 @@ def main():
     ap.add_argument("--workload", default="llama7b-decode-avg2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.workload == "sqc-llama7b-block" and args.impl != "reference":
+        run_sqc(args)
+        return
     spec = workload_spec(args.workload)
     if args.impl == "reference":
         run_reference(args, spec)

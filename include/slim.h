@@ -175,6 +175,18 @@ int slim_allocate_bits(const double* salience_host, int G, int avg_bits, int p, 
 int slim_quantize_minmax(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
                          int N, int K, int g, void* stream);
 
+/* Salience-Weighted Quantizer Calibration (Sec. 3.3, Eq. 5; function SQC of Algorithm 2), per
+ * (row, group): for tau_i = 1 - lambda + i * lambda / n, i = 0 .. 2n-1, the quantizer
+ * Delta = tau (w_max - w_min) / (2^b - 1), z = -round(tau w_min / Delta) is tried on the group and
+ * the candidate with the smallest squared error (salient part, outside mu +- 3 sigma, plus the
+ * rest; first candidate on ties) is kept, so the salient and the other weights share one scale
+ * and one zero point.  Same storage conventions as slim_quantize_minmax (range extended to 0,
+ * Delta rounded to fp16 first, z clamped to the code range); fp64 arithmetic with column-order
+ * sums, so the result is reproducible bit for bit.  tau_index int32 [G][N] (device) receives the
+ * chosen i and may be NULL.  The paper uses lambda = 0.1, n = 50; n <= 64. */
+int slim_quantize_sqc(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
+                      int* tau_index, int N, int K, int g, double lambda, int n, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -53,6 +53,7 @@ def lib():
             "slim_mpq_gemv": [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp],
             "slim_mpq_gemm": [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp],
             "slim_gemv_plan": [i, i, i, i, vp, vp],
+            "slim_quantize_sqc": [vp, vp, vp, vp, vp, vp, i, i, i, ctypes.c_double, i, vp],
             "slim_mpq_gemm_static": [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, vp],
             "slim_group_salience": [vp, vp, vp, i, i, i, vp],
             "slim_allocate_bits": [vp, i, i, i, vp],
@@ -223,6 +224,21 @@ def quantize_minmax(W: torch.Tensor, bits):
                                                               _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
                                                               N, K, GROUP, _stream(W)))
     return codes, scales, zeros
+
+
+def quantize_sqc(W: torch.Tensor, bits, lam: float = 0.1, n: int = 50):
+    """SQC line search (Algorithm 2) on the device.  Returns codes, scales, zeros, tau index."""
+    b = _bits(bits)
+    N, K = W.shape
+    G = K // GROUP
+    codes = torch.empty((N, K), dtype=torch.uint8, device=W.device)
+    scales = torch.empty((G, N), dtype=torch.float16, device=W.device)
+    zeros = torch.empty((G, N), dtype=torch.float16, device=W.device)
+    tau = torch.empty((G, N), dtype=torch.int32, device=W.device)
+    _check("slim_quantize_sqc", lib().slim_quantize_sqc(_dev(W, torch.float16, "W"), _bp(b), _dev(codes, torch.uint8, "codes"),
+                                                        _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
+                                                        _dev(tau, torch.int32, "tau_index"), N, K, GROUP, float(lam), int(n), _stream(W)))
+    return codes, scales, zeros, tau
 
 
 class QuantLinear:

@@ -118,3 +118,139 @@ int slim_quantize_minmax(const void* W, const uint8_t* bits_host, uint8_t* codes
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------ SQC
+// Salience-Weighted Quantizer Calibration (Sec. 3.3, Eq. 5; function SQC of Algorithm 2).
+// One warp per (row, group): the 128 weights sit in shared memory as fp64, every lane evaluates
+// the candidates tau_i with i = lane, lane + 32, ... one after another, walking the columns in
+// order, so that every loss is the same fp64 sum a sequential program would form.  Every fp64
+// operation is an explicit round-to-nearest intrinsic: nothing may be contracted into an FMA.
+namespace slim {
+
+constexpr int kSqcWarps = 4;
+
+struct SqcBest {
+    double loss;
+    int idx;
+};
+
+__global__ void __launch_bounds__(kSqcWarps * 32) quantize_sqc_kernel(const __half* __restrict__ W, uint8_t* __restrict__ codes,
+                                                                       __half* __restrict__ scales, __half* __restrict__ zeros,
+                                                                       int* __restrict__ tau_index, int N, int K, double lambda,
+                                                                       int n_half, GroupTable gt) {
+    __shared__ double sw[kSqcWarps][SLIM_GROUP];
+    const int lane = threadIdx.x & 31, wl = threadIdx.x >> 5;
+    const long long pair = static_cast<long long>(blockIdx.x) * kSqcWarps + wl;
+    const int G = gt.G;
+    if (pair >= static_cast<long long>(N) * G) return;
+    const int n = static_cast<int>(pair / G), j = static_cast<int>(pair % G);
+    const size_t off = static_cast<size_t>(n) * K + SLIM_GROUP * j + 4 * lane;
+    const uint2 raw = *reinterpret_cast<const uint2*>(W + off);
+    const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+    const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+    const float w4[4] = {f01.x, f01.y, f23.x, f23.y};
+    float lo = fminf(fminf(w4[0], w4[1]), fminf(w4[2], w4[3]));
+    float hi = fmaxf(fmaxf(w4[0], w4[1]), fmaxf(w4[2], w4[3]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    const double dlo = static_cast<double>(fminf(lo, 0.0f)), dhi = static_cast<double>(fmaxf(hi, 0.0f));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) sw[wl][4 * lane + i] = static_cast<double>(w4[i]);
+    __syncwarp();
+    const double* w = sw[wl];
+
+    // 3-sigma mask: mean and population standard deviation, both sums in column order
+    double tot = 0.0;
+#pragma unroll 4
+    for (int k = 0; k < SLIM_GROUP; ++k) tot = __dadd_rn(tot, w[k]);
+    const double mu = __ddiv_rn(tot, static_cast<double>(SLIM_GROUP));
+    double var = 0.0;
+#pragma unroll 4
+    for (int k = 0; k < SLIM_GROUP; ++k) {
+        const double d = __dsub_rn(w[k], mu);
+        var = __dadd_rn(var, __dmul_rn(d, d));
+    }
+    const double sd = __dsqrt_rn(__ddiv_rn(var, static_cast<double>(SLIM_GROUP)));
+    const double t_lo = __dsub_rn(mu, __dmul_rn(3.0, sd)), t_hi = __dadd_rn(mu, __dmul_rn(3.0, sd));
+
+    const int b = gt.bits[j];
+    const double levels = static_cast<double>((1 << b) - 1);
+    const double tau0 = __dsub_rn(1.0, lambda), step = __ddiv_rn(lambda, static_cast<double>(n_half));
+    const double range = __dsub_rn(dhi, dlo);
+
+    // scale (fp16 bits) and zero point of candidate i
+    auto candidate = [&](int i, double* s_out, double* z_out) -> unsigned short {
+        const double tau = __dadd_rn(tau0, __dmul_rn(static_cast<double>(i), step));
+        unsigned short sbits = double_to_half_bits_rn(__ddiv_rn(__dmul_rn(tau, range), levels));
+        if ((sbits & 0x7fffu) == 0x7c00u) sbits = 0x7bffu;  // beyond fp16 range -> 65504
+        if ((sbits & 0x7fffu) == 0u) sbits = 0x3c00u;       // zero scale -> 1
+        const double s = static_cast<double>(__half2float(__ushort_as_half(sbits)));
+        *s_out = s;
+        *z_out = fmin(fmax(-rint(__ddiv_rn(__dmul_rn(tau, dlo), s)), 0.0), levels) + 0.0;
+        return sbits;
+    };
+
+    SqcBest best{__longlong_as_double(0x7ff0000000000000ll), 0x7fffffff};
+    for (int i = lane; i < 2 * n_half; i += 32) {
+        double s, z;
+        (void)candidate(i, &s, &z);
+        double Ls = 0.0, Lus = 0.0;
+#pragma unroll 2
+        for (int k = 0; k < SLIM_GROUP; ++k) {
+            const double wk = w[k];
+            const double q = fmin(fmax(__dadd_rn(rint(__ddiv_rn(wk, s)), z), 0.0), levels);
+            const double e = __dsub_rn(wk, __dmul_rn(s, __dsub_rn(q, z)));
+            const double sq = __dmul_rn(e, e);
+            if (wk < t_lo || wk > t_hi) Ls = __dadd_rn(Ls, sq);
+            else Lus = __dadd_rn(Lus, sq);
+        }
+        const double total = __dadd_rn(Ls, Lus);
+        if (total < best.loss) { best.loss = total; best.idx = i; }   // strict: the first candidate wins ties
+    }
+    // smallest loss over the warp, smallest index among equals
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const double ol = __shfl_xor_sync(0xffffffffu, best.loss, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, best.idx, o);
+        if (ol < best.loss || (ol == best.loss && oi < best.idx)) { best.loss = ol; best.idx = oi; }
+    }
+    double s, z;
+    const unsigned short sbits = candidate(best.idx, &s, &z);
+    uint32_t out = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const double q = fmin(fmax(__dadd_rn(rint(__ddiv_rn(static_cast<double>(w4[i]), s)), z), 0.0), levels);
+        out |= static_cast<uint32_t>(static_cast<int>(q)) << (8 * i);
+    }
+    *reinterpret_cast<uint32_t*>(codes + off) = out;
+    if (lane == 0) {
+        scales[static_cast<size_t>(j) * N + n] = __ushort_as_half(sbits);
+        zeros[static_cast<size_t>(j) * N + n] = __float2half_rn(static_cast<float>(z));
+        if (tau_index != nullptr) tau_index[static_cast<size_t>(j) * N + n] = best.idx;
+    }
+}
+
+}  // namespace slim
+
+extern "C" int slim_quantize_sqc(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
+                                 int* tau_index, int N, int K, int g, double lambda, int n, void* stream) {
+    slim::GroupTable gt;
+    const int st = slim::make_group_table(N, K, g, bits_host, &gt);
+    if (st != SLIM_OK) return st;
+    if (!(lambda >= 0.0 && lambda < 1.0) || n < 1 || n > 64) return SLIM_ERR_INVALID_ARG;
+    if (N == 0 || K == 0) return SLIM_OK;
+    if (W == nullptr || codes == nullptr || scales == nullptr || zeros == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (!slim::aligned16(W) || !slim::aligned16(codes) || !slim::aligned16(scales) || !slim::aligned16(zeros) ||
+        (tau_index != nullptr && !slim::aligned16(tau_index)))
+        return SLIM_ERR_ALIGNMENT;
+    const long long pairs = static_cast<long long>(N) * gt.G;
+    const unsigned grid = static_cast<unsigned>((pairs + slim::kSqcWarps - 1) / slim::kSqcWarps);
+    slim::quantize_sqc_kernel<<<grid, slim::kSqcWarps * 32, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const __half*>(W), codes, static_cast<__half*>(scales), static_cast<__half*>(zeros), tau_index, N, K,
+        lambda, n, gt);
+    SLIM_CUDA_TRY(cudaGetLastError());
+    return SLIM_OK;
+}

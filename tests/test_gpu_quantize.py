@@ -68,3 +68,40 @@ def test_allocate_bits_host_matches_oracle_on_ties_and_p():
             assert (slim.allocate_bits(S, avg) == orc.allocate_bits(S, avg)).all()
             for p in (0, 1, G // 2):
                 assert (slim.allocate_bits(S, avg, p) == orc.allocate_bits(S, avg, p)).all()
+
+
+@pytest.mark.parametrize("N,K,bits", [(48, 1024, [1, 2, 3, 4, 2, 3, 1, 4]), (272, 512, [2, 3, 3, 2]), (64, 11008, None)])
+def test_sqc_line_search_matches_oracle_bit_for_bit(N, K, bits):
+    """slim_quantize_sqc (function SQC of Algorithm 2): codes, scales, zero points and the chosen
+    candidate must equal the oracle's; both sides decide in fp64 with column-order sums."""
+    slim = _slim()
+    seed = wl.layer_seed("test", f"sqc-{N}x{K}", 0)
+    W = wl.make_weight(seed, N, K)
+    if bits is None:
+        bits = orc.allocate_bits(orc.group_salience(W, wl.make_act_norms(seed, K)), 2)
+    bits = np.asarray(bits, dtype=np.uint8)
+    c_ref, s_ref, z_ref, t_ref, _, _ = orc.quantize_sqc(W, bits)
+    codes, scales, zeros, tau = slim.quantize_sqc(torch.from_numpy(W).cuda(), bits)
+    assert (tau.cpu().numpy() == t_ref).all()
+    assert (scales.cpu().numpy().view(np.uint16) == s_ref.view(np.uint16)).all()
+    assert (zeros.cpu().numpy().view(np.uint16) == z_ref.view(np.uint16)).all()
+    assert (codes.cpu().numpy() == c_ref).all()
+
+
+def test_sqc_edge_groups_and_other_grids():
+    slim = _slim()
+    rng = np.random.default_rng(13)
+    N, K = 16, 512
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float16)
+    W[:, 0:128] = np.abs(W[:, 0:128])          # all positive
+    W[:, 128:256] = 0                          # constant zero
+    W[:, 256:384] = (rng.standard_normal((N, 128)) * 1e-7).astype(np.float16)   # subnormal weights
+    W[:, 400] = np.float16(3.0)                # one strong outlier
+    for bits, lam, n in ([[1, 2, 3, 4], 0.1, 50], [[4, 3, 2, 1], 0.25, 10], [[2, 2, 2, 2], 0.0, 1]):
+        bits = np.array(bits, dtype=np.uint8)
+        c_ref, s_ref, z_ref, t_ref, _, _ = orc.quantize_sqc(W, bits, lam=lam, n=n)
+        codes, scales, zeros, tau = slim.quantize_sqc(torch.from_numpy(W).cuda(), bits, lam=lam, n=n)
+        assert (tau.cpu().numpy() == t_ref).all()
+        assert (scales.cpu().numpy().view(np.uint16) == s_ref.view(np.uint16)).all()
+        assert (zeros.cpu().numpy().view(np.uint16) == z_ref.view(np.uint16)).all()
+        assert (codes.cpu().numpy() == c_ref).all()
