@@ -1,16 +1,21 @@
 // slim_mpq_gemm: batched / prefill path (M > 16) of the mixed-precision linear layer, sm_100a.
 //
-// y^T = W-hat * x^T on the 5th-generation tensor cores.  The weight rows are the M dimension of
-// the MMA (128 per CTA), the tokens its N dimension (TOK = 128 or 256 per tile):
+// y^T = W-hat * x^T on the 5th-generation tensor cores, two CTAs (one cluster, two SMs) per MMA.
+// The weight rows are the M dimension of the MMA (256 per pair, 128 per CTA), the tokens its N
+// dimension (TOK = 128 or 256 per tile):
 //
-//  * A operand = dequantised weights, fp16, written by eight dequant warps straight into tensor
-//    memory with tcgen05.st (thread = weight row, 32-bit column = two consecutive k); no shared
-//    memory round trip and no swizzled layout to reproduce.  One stage = one group of 128 k.
-//  * B operand = activations, x[tokens][k], brought by TMA into 128-byte-swizzled K-major shared
-//    memory tiles (two boxes of 64 k per group).
-//  * D = fp32 accumulator in tensor memory, 128 lanes x TOK columns; tcgen05.mma kind::f16 is
-//    issued by one thread, eight K=16 steps per group, and tcgen05.commit hands the stages back.
-//  * Epilogue warps read D with tcgen05.ld and store y as fp16.
+//  * A operand = dequantised weights, fp16, written by eight dequant warps of each CTA straight
+//    into that CTA's tensor memory with tcgen05.st (thread = weight row, 32-bit column = two
+//    consecutive k); no shared memory round trip and no swizzled layout to reproduce.  One stage
+//    = one group of 128 k.
+//  * B operand = activations, x[tokens][k].  Each CTA brings HALF of the tile's tokens by TMA into
+//    128-byte-swizzled K-major shared memory (two boxes of 64 k per group); the pair's MMA reads
+//    both halves, so every SM pulls half the activation bytes a single-CTA tile would need and
+//    the freed shared memory buys deeper pipelines.
+//  * D = fp32 accumulator in tensor memory, 128 lanes x TOK columns per CTA; tcgen05.mma
+//    cta_group::2 kind::f16 is issued by one thread of the leader CTA (cluster rank 0), eight
+//    K=16 steps per group, and a multicast tcgen05.commit hands the stages back to both CTAs.
+//  * Epilogue warps of each CTA read their D with tcgen05.ld and store y as fp16.
 //
 // Dequantisation: a code field is moved to mantissa bits [6,10) of a half whose exponent makes it
 // 16 + q (ulp 1/64); one HSUB2 removes 16 + z exactly for every zero point that is a multiple of
@@ -18,10 +23,12 @@
 // the scale with a single rounding, so the operand equals the fp16 weight slim_dequant produces.
 // Other zero points are rounded to the nearest 1/64.
 //
-// Warp roles (448 threads): warp 0 producer (TMA + bulk copies of packed slices, scales, zeros),
-// warp 1 MMA issuer and tensor-memory allocator, warps 2-9 dequant, warps 10-13 epilogue.
-// Persistent CTAs walk the (token tile, row block) tiles; every wait on an mbarrier is bounded
-// and reports through the workspace status word instead of spinning forever.
+// Warp roles (448 threads per CTA): warp 0 producer (TMA + bulk copies of packed slices, scales,
+// zeros), warp 1 MMA issuer in the leader / "my half of x has landed" relay in the other CTA,
+// and tensor-memory allocator in both, warps 2-9 dequant, warps 10-13 epilogue.  Persistent
+// clusters walk the (token tile, 256-row block) tiles; every wait on an mbarrier or a flag is
+// bounded and reports through the workspace status word instead of spinning forever, and no CTA
+// leaves before its partner has stopped signalling it.
 #include "slim_common.cuh"
 
 #include <cuda.h>
@@ -31,8 +38,8 @@ namespace slim {
 
 constexpr int kGemmThreads = 448;
 constexpr int kRowsPerCta = 128;
+constexpr int kRowsPerPair = 2 * kRowsPerCta;
 constexpr int kNA = 4;                      // tensor-memory stages of A (64 columns each)
-constexpr int kNP = 3;                      // shared-memory stages of packed slices
 constexpr int kPStageBytes = 8192 + 512;    // 128 rows x 128 k x 4 bits, + scales + zeros
 constexpr int kTmemCols = 512;
 constexpr int kTmemAcol = 256;              // A stages start here; D occupies [0, TOK)
@@ -47,8 +54,8 @@ struct GemmParams {
     unsigned int* flags;     // [grid]: "partial of this CTA is ready" (stream-K only; zero between launches)
     float* partials;         // [grid][TOK][128] fp32 (stream-K only)
     int M, N, K;
-    int row_blocks, tok_tiles;
-    int stream_k;            // 1: CTAs take equal shares of (tile, group) units; 0: whole tiles
+    int row_blocks, tok_tiles;   // 256-row blocks, TOK-token tiles
+    int stream_k;            // 1: clusters take equal shares of (tile, group) units; 0: whole tiles
     GroupTable gt;
 };
 
@@ -60,6 +67,20 @@ constexpr int kGemmWsPartials = kGemmWsFlags + 4 * kGemmMaxGrid;
 namespace g {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
@@ -69,6 +90,13 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// arrive on a barrier of any CTA of the cluster (address from map_to_cta)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -94,6 +122,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (global_timer_ns() - t0 > kGemmWaitNs) { *abort = 1; return false; }
     }
 }
+// The same for a wait that is known to be long (a whole tile): one lane polls, with a pause
+// between tries, so the waiting warp leaves the issue slots to the warps that work.
+__device__ __forceinline__ bool mbar_wait_long(uint32_t bar, uint32_t parity, volatile int* abort) {
+    bool ok = true;
+    if ((threadIdx.x & 31) == 0) {
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(bar, parity)) {
+            __nanosleep(128);
+            if (*abort != 0) { ok = false; break; }
+            if (global_timer_ns() - t0 > kGemmWaitNs) { *abort = 1; ok = false; break; }
+        }
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (ok) ok = mbar_wait(bar, parity, abort);  // every lane observes the completed phase itself
+    return ok;
+}
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -106,26 +150,31 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
                  ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 
+// Tensor memory of the CTA pair: one warp of EACH CTA executes these together.
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
 }
-__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// When the pair's MMAs issued so far have completed, arrive on the barrier at this shared-memory
+// offset in both CTAs of the pair.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem descriptor]; fp16 inputs, fp32 accumulate.
+// D[tmem] (+)= A[tmem] * B[smem descriptor] over the CTA pair: 256 weight rows (128 from each
+// CTA's tensor memory) x TOK tokens (half from each CTA's shared memory); fp16 in, fp32 accumulate.
 __device__ __forceinline__ void umma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-        " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %6, %7, %8}, p;\n}\n"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
+        " tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
 // 32 lanes x 32 columns of 32-bit: thread = lane, register j = column j.
@@ -220,12 +269,14 @@ __device__ __forceinline__ void decode_cword(const uint32_t (&words)[4], const D
 
 // ------------------------------------------------------------------------------------------ kernel
 template <int TOK> struct GemmCfg {
-    static constexpr int NX = TOK == 256 ? 3 : 4;            // shared-memory stages of x
-    static constexpr int XBOX = TOK * 128;                   // bytes of one TMA box: TOK rows x 64 k
+    static constexpr int HALF = TOK / 2;                     // tokens this CTA brings
+    static constexpr int NX = TOK == 256 ? 5 : 8;            // shared-memory stages of x
+    static constexpr int NP = TOK == 256 ? 6 : 8;            // shared-memory stages of packed slices
+    static constexpr int XBOX = HALF * 128;                  // bytes of one TMA box: HALF rows x 64 k
     static constexpr int XSTAGE = 2 * XBOX;                  // one group: 128 k
     static constexpr int OFF_P = NX * XSTAGE;
-    static constexpr int OFF_BAR = OFF_P + kNP * kPStageBytes;
-    static constexpr int NBAR = 2 * NX + 2 * kNP + 2 * kNA + 2;
+    static constexpr int OFF_BAR = OFF_P + NP * kPStageBytes;
+    static constexpr int NBAR = 3 * NX + 2 * NP + 2 * kNA + 2;
     static constexpr int OFF_MISC = OFF_BAR + 8 * NBAR;      // tensor-memory base, abort flag
     static constexpr int SMEM = OFF_MISC + 16 + 1024;        // + slack to align the base to 1024
 };
@@ -237,32 +288,36 @@ __device__ __forceinline__ uint64_t sw128_kmajor_desc(uint32_t smem_addr) {
 }
 
 template <int TOK>
-__global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ CUtensorMap x_map,
-                                                               const __grid_constant__ GemmParams p) {
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ GemmParams p) {
     using C = GemmCfg<TOK>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (g::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (sbase - g::smem_u32(smem_raw));
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int rank = static_cast<int>(g::cluster_ctarank());     // 0 = leader of the pair
     const uint32_t bar0 = sbase + C::OFF_BAR;
+    // barriers of this CTA
     auto x_full = [&](int s) { return bar0 + 8 * s; };
     auto x_empty = [&](int s) { return bar0 + 8 * (C::NX + s); };
-    auto p_full = [&](int s) { return bar0 + 8 * (2 * C::NX + s); };
-    auto p_empty = [&](int s) { return bar0 + 8 * (2 * C::NX + kNP + s); };
-    auto a_full = [&](int s) { return bar0 + 8 * (2 * C::NX + 2 * kNP + s); };
-    auto a_empty = [&](int s) { return bar0 + 8 * (2 * C::NX + 2 * kNP + kNA + s); };
-    const uint32_t d_full = bar0 + 8 * (2 * C::NX + 2 * kNP + 2 * kNA);
-    const uint32_t d_empty = d_full + 8;
+    auto p_full = [&](int s) { return bar0 + 8 * (3 * C::NX + s); };
+    auto p_empty = [&](int s) { return bar0 + 8 * (3 * C::NX + C::NP + s); };
+    auto a_empty = [&](int s) { return bar0 + 8 * (3 * C::NX + 2 * C::NP + kNA + s); };
+    const uint32_t d_full = bar0 + 8 * (3 * C::NX + 2 * C::NP + 2 * kNA);
+    // barriers that live in the leader only: the other CTA reaches them through the cluster window
+    auto xp_full = [&](int s) { return bar0 + 8 * (2 * C::NX + s); };               // partner's half of x has landed
+    auto a_full = [&](int s) { return bar0 + 8 * (3 * C::NX + 2 * C::NP + s); };    // 16 dequant warps of the pair
+    const uint32_t d_empty = d_full + 8;                                            // 8 epilogue warps of the pair
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OFF_MISC);
     volatile int* abort = reinterpret_cast<volatile int*>(smem + C::OFF_MISC + 4);
 
     if (tid == 0) {
-        for (int s = 0; s < C::NX; ++s) { g::mbar_init(x_full(s), 1); g::mbar_init(x_empty(s), 1); }
-        for (int s = 0; s < kNP; ++s) { g::mbar_init(p_full(s), 1); g::mbar_init(p_empty(s), 8); }
-        for (int s = 0; s < kNA; ++s) { g::mbar_init(a_full(s), 8); g::mbar_init(a_empty(s), 1); }
+        for (int s = 0; s < C::NX; ++s) { g::mbar_init(x_full(s), 1); g::mbar_init(x_empty(s), 1); g::mbar_init(xp_full(s), 1); }
+        for (int s = 0; s < C::NP; ++s) { g::mbar_init(p_full(s), 1); g::mbar_init(p_empty(s), 8); }
+        for (int s = 0; s < kNA; ++s) { g::mbar_init(a_full(s), 16); g::mbar_init(a_empty(s), 1); }
         g::mbar_init(d_full, 1);
-        g::mbar_init(d_empty, 4);
+        g::mbar_init(d_empty, 8);
         *abort = 0;
         g::fence_barrier_init();
         g::fence_proxy_async();
@@ -272,19 +327,20 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         g::tmem_relinquish();
     }
     g::tc_fence_before();
-    __syncthreads();
+    g::cluster_sync_all();          // both CTAs' barriers exist before either signals the other
     g::tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
     const int G = p.gt.G, N = p.N;
     const int total_tiles = p.row_blocks * p.tok_tiles;
-    // This CTA's contiguous range [u0, u1) of (tile, group) units, unit = tile * G + group,
-    // tile = token tile * row_blocks + row block.  Without stream-K the range is whole tiles.
-    auto range_begin = [&](int cta) -> long long {
-        return p.stream_k ? (static_cast<long long>(cta) * total_tiles * G) / gridDim.x
-                          : ((static_cast<long long>(cta) * total_tiles) / gridDim.x) * G;
+    const int cl = blockIdx.x >> 1, ncl = gridDim.x >> 1;
+    // This pair's contiguous range [u0, u1) of (tile, group) units, unit = tile * G + group,
+    // tile = token tile * row_blocks + 256-row block.  Without stream-K the range is whole tiles.
+    auto range_begin = [&](int c) -> long long {
+        return p.stream_k ? (static_cast<long long>(c) * total_tiles * G) / ncl
+                          : ((static_cast<long long>(c) * total_tiles) / ncl) * G;
     };
-    const long long u0 = range_begin(blockIdx.x), u1 = range_begin(blockIdx.x + 1);
+    const long long u0 = range_begin(cl), u1 = range_begin(cl + 1);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
@@ -296,41 +352,51 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                 const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
                 const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
                 u += ge - gb;
-                const int rb = tile % p.row_blocks, mt = tile / p.row_blocks;
-                const int tiles_here = min(8, (N >> 4) - 8 * rb);
+                const int rb = 2 * (tile % p.row_blocks) + rank, mt = tile / p.row_blocks;   // my 128-row block
+                const int tiles_here = max(0, min(8, (N >> 4) - 8 * rb));
                 for (int j = gb; j < ge && ok; ++j) {
-                    // activations of the group
+                    // my half of the group's activations
                     if (!g::mbar_wait(x_empty(sx), phx ^ 1u, abort)) { ok = false; break; }
                     g::mbar_expect_tx(x_full(sx), C::XSTAGE);
-                    g::tma_load_2d(sbase + sx * C::XSTAGE, &x_map, SLIM_GROUP * j, mt * TOK, x_full(sx));
-                    g::tma_load_2d(sbase + sx * C::XSTAGE + C::XBOX, &x_map, SLIM_GROUP * j + 64, mt * TOK, x_full(sx));
+                    g::tma_load_2d(sbase + sx * C::XSTAGE, &x_map, SLIM_GROUP * j, mt * TOK + rank * C::HALF, x_full(sx));
+                    g::tma_load_2d(sbase + sx * C::XSTAGE + C::XBOX, &x_map, SLIM_GROUP * j + 64, mt * TOK + rank * C::HALF, x_full(sx));
                     if (++sx == C::NX) { sx = 0; phx ^= 1u; }
-                    // packed slices, scales, zeros of the row block
+                    // packed slices, scales, zeros of my rows
                     if (!g::mbar_wait(p_empty(sp), php ^ 1u, abort)) { ok = false; break; }
-                    const int b = p.gt.bits[j];
-                    const uint32_t wbytes = static_cast<uint32_t>(tiles_here) * 256u * b, sbytes = static_cast<uint32_t>(tiles_here) * 32u;
-                    const uint32_t dst = sbase + C::OFF_P + sp * kPStageBytes;
-                    g::mbar_expect_tx(p_full(sp), wbytes + 2 * sbytes);
-                    g::bulk_g2s(dst, p.packed + 16ull * N * p.gt.prefix[j] + static_cast<size_t>(8 * rb) * 256 * b, wbytes, p_full(sp));
-                    g::bulk_g2s(dst + 8192, p.scales + static_cast<size_t>(j) * N + kRowsPerCta * rb, sbytes, p_full(sp));
-                    g::bulk_g2s(dst + 8192 + 256, p.zeros + static_cast<size_t>(j) * N + kRowsPerCta * rb, sbytes, p_full(sp));
-                    if (++sp == kNP) { sp = 0; php ^= 1u; }
+                    if (tiles_here > 0) {
+                        const int b = p.gt.bits[j];
+                        const uint32_t wbytes = static_cast<uint32_t>(tiles_here) * 256u * b, sbytes = static_cast<uint32_t>(tiles_here) * 32u;
+                        const uint32_t dst = sbase + C::OFF_P + sp * kPStageBytes;
+                        g::mbar_expect_tx(p_full(sp), wbytes + 2 * sbytes);
+                        g::bulk_g2s(dst, p.packed + 16ull * N * p.gt.prefix[j] + static_cast<size_t>(8 * rb) * 256 * b, wbytes, p_full(sp));
+                        g::bulk_g2s(dst + 8192, p.scales + static_cast<size_t>(j) * N + kRowsPerCta * rb, sbytes, p_full(sp));
+                        g::bulk_g2s(dst + 8192 + 256, p.zeros + static_cast<size_t>(j) * N + kRowsPerCta * rb, sbytes, p_full(sp));
+                    } else {
+                        g::mbar_arrive(p_full(sp));             // no row of mine exists: nothing to bring
+                    }
+                    if (++sp == C::NP) { sp = 0; php ^= 1u; }
                 }
             }
-            if (!ok) {
+            if (ok) {
+                // every x stage has been handed back: no commit of the leader is still on its way here
+                for (int s = 0; s < C::NX && ok; ++s) {
+                    ok = g::mbar_wait(x_empty(sx), phx ^ 1u, abort);
+                    if (++sx == C::NX) { sx = 0; phx ^= 1u; }
+                }
+            } else {
                 // leave no copy in flight: wait (bounded) for the last phase issued to every stage
                 auto drain = [&](uint32_t bar, uint32_t parity) {
                     const unsigned long long t0 = g::global_timer_ns();
                     while (!g::mbar_try_wait(bar, parity) && g::global_timer_ns() - t0 < 1000000ull) { }
                 };
                 for (int s = 0; s < C::NX; ++s) drain(x_full(s), s < sx ? phx : phx ^ 1u);
-                for (int s = 0; s < kNP; ++s) drain(p_full(s), s < sp ? php : php ^ 1u);
+                for (int s = 0; s < C::NP; ++s) drain(p_full(s), s < sp ? php : php ^ 1u);
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(TOK >> 3) << 17) | (static_cast<uint32_t>(kRowsPerCta >> 4) << 24);
+        if (lane == 0 && rank == 0) {
+            // -------------------------------------------------------------- MMA issuer (leader)
+            constexpr uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(TOK >> 3) << 17) | (static_cast<uint32_t>(kRowsPerPair >> 4) << 24);
             int sx = 0, sa = 0;
             uint32_t phx = 0, pha = 0, phd = 0;
             bool ok = true;
@@ -338,10 +404,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                 const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
                 const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
                 u += ge - gb;
-                if (!g::mbar_wait(d_empty, phd ^ 1u, abort)) { ok = false; break; }   // epilogue has drained D
+                if (!g::mbar_wait(d_empty, phd ^ 1u, abort)) { ok = false; break; }   // both epilogues have drained D
                 g::tc_fence_after();
                 for (int j = gb; j < ge; ++j) {
-                    if (!g::mbar_wait(x_full(sx), phx, abort) || !g::mbar_wait(a_full(sa), pha, abort)) { ok = false; break; }
+                    if (!g::mbar_wait(x_full(sx), phx, abort) || !g::mbar_wait(xp_full(sx), phx, abort) ||
+                        !g::mbar_wait(a_full(sa), pha, abort)) { ok = false; break; }
                     g::tc_fence_after();
                     const uint32_t xs = sbase + sx * C::XSTAGE;
                     const uint32_t a_t = tmem + kTmemAcol + 64 * sa;
@@ -350,13 +417,24 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                         const uint64_t bdesc = sw128_kmajor_desc(xs + (ks >> 2) * C::XBOX + (ks & 3) * 32);
                         g::umma_f16_ts(tmem, a_t + 8 * ks, bdesc, idesc, (j > gb || ks != 0) ? 1u : 0u);
                     }
-                    g::tc_commit(x_empty(sx));
-                    g::tc_commit(a_empty(sa));
+                    g::tc_commit_pair(x_empty(sx));
+                    g::tc_commit_pair(a_empty(sa));
                     if (++sx == C::NX) { sx = 0; phx ^= 1u; }
                     if (++sa == kNA) { sa = 0; pha ^= 1u; }
                 }
-                if (ok) g::tc_commit(d_full);
+                if (ok) g::tc_commit_pair(d_full);
                 phd ^= 1u;
+            }
+        } else if (lane == 0) {
+            // -------------------------------------------------------------- relay (other CTA)
+            // tells the leader that this CTA's half of a group's activations is in shared memory
+            int sx = 0;
+            uint32_t phx = 0;
+            bool ok = true;
+            for (long long u = u0; u < u1 && ok; ++u) {
+                if (!g::mbar_wait(x_full(sx), phx, abort)) { ok = false; break; }
+                g::mbar_arrive_cluster(g::map_to_cta(xp_full(sx), 0));
+                if (++sx == C::NX) { sx = 0; phx ^= 1u; }
             }
         }
     } else if (warp < 10) {
@@ -367,11 +445,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
         int sp = 0, sa = 0;
         uint32_t php = 0, pha = 0;
         bool ok = true;
+        const uint32_t a_full_leader = g::map_to_cta(a_full(0), 0);
         for (long long u = u0; u < u1 && ok;) {
             const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
             const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
             u += ge - gb;
-            const int rb = tile % p.row_blocks;
+            const int rb = 2 * (tile % p.row_blocks) + rank;
             const bool row_ok = kRowsPerCta * rb + r < N;
             for (int j = gb; j < ge; ++j) {
                 if (!g::mbar_wait(p_full(sp), php, abort)) { ok = false; break; }
@@ -397,7 +476,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                 }
                 __syncwarp();
                 if (lane == 0) g::mbar_arrive(p_empty(sp));
-                if (++sp == kNP) { sp = 0; php ^= 1u; }
+                if (++sp == C::NP) { sp = 0; php ^= 1u; }
 
                 uint32_t cols[32];
                 switch (b) {
@@ -412,47 +491,54 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                 g::tc_wait_st();
                 g::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) g::mbar_arrive(a_full(sa));
+                if (lane == 0) g::mbar_arrive_cluster(a_full_leader + 8 * sa);
                 if (++sa == kNA) { sa = 0; pha ^= 1u; }
             }
+        }
+        // every A stage has been handed back: no commit of the leader is still on its way here
+        for (int s = 0; s < kNA && ok; ++s) {
+            ok = g::mbar_wait(a_empty(sa), pha ^ 1u, abort);
+            if (++sa == kNA) { sa = 0; pha ^= 1u; }
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
         // A segment that covers its whole tile is stored as fp16.  With stream-K a tile may be cut:
-        // the CTA whose segment does not start the tile leaves its fp32 partial in its workspace
-        // slot and raises its flag; the CTA that starts the tile (it reaches that segment last, the
-        // others reach theirs first) waits for those flags, adds the partials in CTA order and
-        // stores the tile.
+        // a pair whose segment does not start the tile leaves its fp32 partials in its CTAs'
+        // workspace slots and raises their flags; the pair that starts the tile (it reaches that
+        // segment last, the others reach theirs first) waits for those flags, adds the partials in
+        // pair order and stores the tile.  Each CTA deals with the CTAs of the same rank, which
+        // hold the same 128 rows.
         const int q = warp & 3;
         const int et = tid - 320;                               // 0..127 among the epilogue threads
         uint32_t phd = 0;
         bool ok = true;
+        const uint32_t d_empty_leader = g::map_to_cta(d_empty, 0);
         auto epi_sync = [] { asm volatile("bar.sync 1, 128;" ::: "memory"); };
         for (long long u = u0; u < u1 && ok;) {
             const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
             const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
             u += ge - gb;
-            const int rb = tile % p.row_blocks, mt = tile / p.row_blocks;
+            const int rb = 2 * (tile % p.row_blocks) + rank, mt = tile / p.row_blocks;
             const int n = kRowsPerCta * rb + 32 * q + lane;
             const bool is_partial = gb > 0;
-            // peers: the CTAs after this one, up to the one that ends the tile (CTAs with an empty
-            // range take no part)
+            // peers: the pairs after this one, up to the one that ends the tile (pairs with an empty
+            // range take no part); peer k is CTA blockIdx.x + 2k
             int npeer = 0;
             if (!is_partial && ge < G) {
-                for (int pc = blockIdx.x + 1; pc < static_cast<int>(gridDim.x); ++pc) {
+                for (int pc = cl + 1; pc < ncl; ++pc) {
                     ++npeer;
                     if (range_begin(pc + 1) >= static_cast<long long>(tile + 1) * G) break;
                 }
             }
-            auto peer_active = [&](int k) { return range_begin(blockIdx.x + k) < range_begin(blockIdx.x + k + 1); };
-            if (!g::mbar_wait(d_full, phd, abort)) { ok = false; break; }
+            auto peer_active = [&](int k) { return range_begin(cl + k) < range_begin(cl + k + 1); };
+            if (!g::mbar_wait_long(d_full, phd, abort)) { ok = false; break; }
             g::tc_fence_after();
             if (npeer > 0) {
                 if (et == 0) {
                     const unsigned long long t0 = g::global_timer_ns();
                     for (int k = 1; k <= npeer; ++k) {
                         if (!peer_active(k)) continue;
-                        volatile unsigned int* f = p.flags + blockIdx.x + k;
+                        volatile unsigned int* f = p.flags + blockIdx.x + 2 * k;
                         while (*f == 0u) {
                             if (*abort != 0 || g::global_timer_ns() - t0 > kGemmWaitNs) { *abort = 1; break; }
                         }
@@ -480,7 +566,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                     for (int i = 0; i < 32; ++i) t[i] = 0.f;
                     for (int k = 1; k <= npeer; ++k) {
                         if (!peer_active(k)) continue;
-                        const float* slot = p.partials + static_cast<size_t>(blockIdx.x + k) * (TOK * kRowsPerCta) + 32 * q + lane;
+                        const float* slot = p.partials + static_cast<size_t>(blockIdx.x + 2 * k) * (TOK * kRowsPerCta) + 32 * q + lane;
 #pragma unroll
                         for (int i = 0; i < 32; ++i) t[i] += __ldcg(slot + (32 * cc + i) * kRowsPerCta);
                     }
@@ -507,7 +593,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
             }
             g::tc_fence_before();
             __syncwarp();
-            if (lane == 0) g::mbar_arrive(d_empty);
+            if (lane == 0) g::mbar_arrive_cluster(d_empty_leader);
             phd ^= 1u;
             if (is_partial) {
                 __threadfence();
@@ -515,12 +601,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                 if (et == 0) { __threadfence(); *(volatile unsigned int*)(p.flags + blockIdx.x) = 1u; }
             } else if (npeer > 0) {
                 epi_sync();                                     // everyone has read the peers' slots
-                if (et < npeer) p.flags[blockIdx.x + 1 + et] = 0u;   // ready for the next launch (unused ones are 0 already)
+                if (et < npeer) p.flags[blockIdx.x + 2 * (1 + et)] = 0u;   // ready for the next launch (unused ones are 0 already)
             }
         }
     }
 
-    __syncthreads();
+    // nobody leaves, and the pair's tensor memory stays, until both CTAs are through
+    g::tc_fence_before();
+    g::cluster_sync_all();
     if (tid == 0 && *abort != 0) atomicOr(p.status, 1u);
     if (warp == 1) {
         g::tc_fence_after();
@@ -545,13 +633,13 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// Tensor map of x [M][K] fp16: boxes of 64 k x tok rows, 128-byte swizzle, rows past M read as 0.
-static bool make_x_map(CUtensorMap* map, const void* x, int M, int K, int tok) {
+// Tensor map of x [M][K] fp16: boxes of 64 k x `rows` tokens, 128-byte swizzle, rows past M read as 0.
+static bool make_x_map(CUtensorMap* map, const void* x, int M, int K, int rows) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (enc == nullptr) return false;
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(M)};
     const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * sizeof(__half)};
-    const cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(tok)};
+    const cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(rows)};
     const cuuint32_t estr[2] = {1u, 1u};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -565,9 +653,37 @@ static int gemm_sm_count() {
     return n;
 }
 
+// CTA pairs that can be resident at once (the stream-K hand-over needs all of them running).
+template <int TOK>
+static int max_resident_pairs() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (cached[dev] == 0) {
+        if (cudaFuncSetAttribute(gemm_kernel<TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<TOK>::SMEM) != cudaSuccess) return 0;
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3(2 * gemm_sm_count(), 1, 1);
+        cfg.blockDim = dim3(kGemmThreads, 1, 1);
+        cfg.dynamicSmemBytes = GemmCfg<TOK>::SMEM;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel<TOK>, &cfg) != cudaSuccess || n <= 0) {
+            cudaGetLastError();
+            return 0;
+        }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 // Launch shape shared by the entry point and the workspace query.  Stream-K (equal shares of
-// (tile, group) units per CTA, partial tiles combined through the workspace) is used when it is
-// predicted to beat whole tiles, whose last wave may leave most SMs idle.
+// (tile, group) units per CTA pair, partial tiles combined through the workspace) is used when it
+// is predicted to beat whole tiles, whose last wave may leave most SMs idle.
 struct GemmPlan {
     int tok, row_blocks, tok_tiles, grid, stream_k;
     size_t workspace_bytes;
@@ -575,21 +691,25 @@ struct GemmPlan {
 static GemmPlan plan_gemm(int M, int N, int G) {
     GemmPlan pl;
     pl.tok = M <= 128 ? 128 : 256;
-    pl.row_blocks = (N + kRowsPerCta - 1) / kRowsPerCta;
+    pl.row_blocks = (N + kRowsPerPair - 1) / kRowsPerPair;
     pl.tok_tiles = (M + pl.tok - 1) / pl.tok;
     const int tiles = pl.row_blocks * pl.tok_tiles;
-    int sms = gemm_sm_count();
-    if (sms > kGemmMaxGrid) sms = kGemmMaxGrid;
-    pl.grid = tiles < sms ? tiles : sms;
-    const int waves = (tiles + sms - 1) / sms;
-    (void)waves;
+    int pairs = gemm_sm_count() / 2;
+    const int resident = pl.tok == 128 ? max_resident_pairs<128>() : max_resident_pairs<256>();
+    if (resident > 0 && pairs > resident) pairs = resident;
+    if (pairs > kGemmMaxGrid / 2) pairs = kGemmMaxGrid / 2;
+    if (pairs < 1) pairs = 1;
+    const int npairs = tiles < pairs ? tiles : pairs;
+    const int waves = (tiles + pairs - 1) / pairs;
+    pl.grid = 2 * npairs;
     pl.stream_k = 0;
-    // time in units of one group: whole tiles take waves * G; equal shares take units / SMs plus
+    // time in units of one group: whole tiles take waves * G; equal shares take units / pairs plus
     // about two dozen groups' worth of draining, storing and re-reading a partial tile (measured)
     const long long units = static_cast<long long>(tiles) * G;
-    if (units >= 8ll * sms && static_cast<double>(units) / sms + 24.0 < 0.95 * static_cast<double>(waves) * G) {
+    if (resident > 0 && units >= 8ll * pairs &&
+        static_cast<double>(units) / pairs + 24.0 < 0.95 * static_cast<double>(waves) * G) {
         pl.stream_k = 1;
-        pl.grid = sms;
+        pl.grid = 2 * pairs;
     }
     pl.workspace_bytes = pl.stream_k ? kGemmWsPartials + static_cast<size_t>(pl.grid) * pl.tok * kRowsPerCta * sizeof(float) : 256;
     return pl;
@@ -607,7 +727,7 @@ static cudaError_t launch_gemm(const CUtensorMap& map, const GemmParams& prm, in
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    gemm_kernel<TOK><<<grid, kGemmThreads, GemmCfg<TOK>::SMEM, stream>>>(map, prm);
+    gemm_kernel<TOK><<<grid, kGemmThreads, GemmCfg<TOK>::SMEM, stream>>>(map, prm);   // clusters of 2: see the kernel
     return cudaGetLastError();
 }
 
@@ -638,11 +758,11 @@ extern "C" int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* b
     if (pl.stream_k && workspace_bytes < pl.workspace_bytes) {   // small workspace: whole tiles, no scratch
         pl.stream_k = 0;
         const int tiles = pl.row_blocks * pl.tok_tiles;
-        if (pl.grid > tiles) pl.grid = tiles;
+        if (pl.grid > 2 * tiles) pl.grid = 2 * tiles;
     }
     const int tok = pl.tok;
     CUtensorMap map;
-    if (!slim::make_x_map(&map, x, M, K, tok)) {
+    if (!slim::make_x_map(&map, x, M, K, tok / 2)) {
         slim::set_cuda_error(cudaErrorUnknown);
         return SLIM_ERR_CUDA;
     }
