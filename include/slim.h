@@ -122,8 +122,8 @@ int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host,
 int slim_gemv_plan(int M, int N, int K, int g, const uint8_t* bits_host, int* out6);
 
 /* Batched / prefill path, M > 16: same contract, tensor-core (tcgen05) kernel.  Zero points that
- * are multiples of 1/64 in [-16, 16) (every zero point Eq. 1 or Eq. 2 produces) are applied exactly,
- * others are rounded to the nearest 1/64.  Deterministic for a given (shape, device, workspace size). */
+ * are multiples of 1/16 in [-16, 16) (every zero point Eq. 1 or Eq. 2 produces) are applied exactly,
+ * others are rounded (to the nearest 1/16 at worst).  Deterministic for a given (shape, device, workspace size). */
 int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* bits_host,
                   const void* scales, const void* zeros, void* y,
                   int M, int N, int K, int g,

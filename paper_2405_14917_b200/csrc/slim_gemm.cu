@@ -4,7 +4,7 @@
 // The weight rows are the M dimension of the MMA (256 per pair, 128 per CTA), the tokens its N
 // dimension (TOK = 128 or 256 per tile):
 //
-//  * A operand = dequantised weights, fp16, written by eight dequant warps of each CTA straight
+//  * A operand = dequantised weights, fp16, written by the dequant warps of each CTA straight
 //    into that CTA's tensor memory with tcgen05.st (thread = weight row, 32-bit column = two
 //    consecutive k); no shared memory round trip and no swizzled layout to reproduce.  One stage
 //    = one group of 128 k.
@@ -17,15 +17,16 @@
 //    K=16 steps per group, and a multicast tcgen05.commit hands the stages back to both CTAs.
 //  * Epilogue warps of each CTA read their D with tcgen05.ld and store y as fp16.
 //
-// Dequantisation: a code field is moved to mantissa bits [6,10) of a half whose exponent makes it
-// 16 + q (ulp 1/64); one HSUB2 removes 16 + z exactly for every zero point that is a multiple of
-// 1/64 in [-16, 16) (all integer and half-integer zero points of Eq. 1 / Eq. 2), one HMUL2 applies
-// the scale with a single rounding, so the operand equals the fp16 weight slim_dequant produces.
-// Other zero points are rounded to the nearest 1/64.
+// Dequantisation: a code field is left in mantissa bits [6,10) of the half 1024; one HFMA2 with
+// constants that hold the zero point turns it into q - z exactly for every zero point that is a
+// multiple of 1/16 in [-16, 16) (all integer and half-integer zero points of Eq. 1 / Eq. 2), one
+// HMUL2 applies the scale with a single rounding, so the operand equals the fp16 weight
+// slim_dequant produces.  Other zero points are rounded (to the nearest 1/16 at worst).
 //
-// Warp roles (448 threads per CTA): warp 0 producer (TMA + bulk copies of packed slices, scales,
-// zeros), warp 1 MMA issuer in the leader / "my half of x has landed" relay in the other CTA,
-// and tensor-memory allocator in both, warps 2-9 dequant, warps 10-13 epilogue.  Persistent
+// Warp roles (23 warps per CTA): warp 0 producer of activations (TMA); warp 1 MMA issuer in the
+// leader / "my half of x has landed" relay in the other CTA, and tensor-memory allocator in both;
+// warps 2-17 dequant, two sets of eight that take alternate groups; warps 18-21 epilogue; warp 22
+// producer of packed slices, scales and zeros (bulk copies).  Persistent
 // clusters walk the (token tile, 256-row block) tiles; every wait on an mbarrier or a flag is
 // bounded and reports through the workspace status word instead of spinning forever, and no CTA
 // leaves before its partner has stopped signalling it.
@@ -36,12 +37,17 @@
 
 namespace slim {
 
-constexpr int kGemmThreads = 448;
+constexpr int kDqWarps = 16;                // dequant warps: sets of 8 that take the pipeline stages in turn
+constexpr int kWarpEpi = 2 + kDqWarps;      // first of the four epilogue warps
+constexpr int kWarpPacked = kWarpEpi + 4;   // producer of packed slices
+constexpr int kGemmThreads = 32 * (kWarpPacked + 1);
 constexpr int kRowsPerCta = 128;
 constexpr int kRowsPerPair = 2 * kRowsPerCta;
-constexpr int kNA = 4;                      // tensor-memory stages of A (64 columns each)
+constexpr int kGPS = 2;                     // groups per pipeline stage: one round of barriers serves this many
+constexpr int kNS = 4 / kGPS;               // pipeline stages: a shared-memory slot of x + 64 tensor-memory columns of A per group
 constexpr int kPStageBytes = 8192 + 512;    // 128 rows x 128 k x 4 bits, + scales + zeros
 constexpr int kTmemCols = 512;
+constexpr int kEpiCols = 16;                // accumulator columns (tokens) the epilogue handles at a time
 constexpr int kTmemAcol = 256;              // A stages start here; D occupies [0, TOK)
 constexpr unsigned long long kGemmWaitNs = 2000000000ull;
 
@@ -122,6 +128,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (global_timer_ns() - t0 > kGemmWaitNs) { *abort = 1; return false; }
     }
 }
+// The same by a whole warp: its lanes go on, or give up, together.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort));
+}
 // The same for a wait that is known to be long (a whole tile): one lane polls, with a pause
 // between tries, so the waiting warp leaves the issue slots to the warps that work.
 __device__ __forceinline__ bool mbar_wait_long(uint32_t bar, uint32_t parity, volatile int* abort) {
@@ -135,8 +145,13 @@ __device__ __forceinline__ bool mbar_wait_long(uint32_t bar, uint32_t parity, vo
         }
     }
     ok = __shfl_sync(0xffffffffu, ok, 0);
-    if (ok) ok = mbar_wait(bar, parity, abort);  // every lane observes the completed phase itself
+    if (ok) ok = mbar_wait_warp(bar, parity, abort);  // every lane observes the completed phase itself
     return ok;
+}
+// After a failure: wait, for a millisecond at most, until the copies issued to a stage have landed.
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+    const unsigned long long t0 = global_timer_ns();
+    while (!mbar_try_wait(bar, parity) && global_timer_ns() - t0 < 1000000ull) { }
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -187,6 +202,20 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
           "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
           "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]) : "memory");
 }
+// 32 lanes x 16 columns
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
@@ -212,35 +241,71 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 // ------------------------------------------------------------------------------------------ dequantisation
 // Everything below works on one "c-word set": the slice words of one weight row that cover 32
 // consecutive k, and produces the 16 tensor-memory columns (k, k+1 pairs) of those 32 weights.
-constexpr uint32_t kMagic16 = 0x4C004C00u;   // half2(16, 16): ulp 1/64, mantissa bit 6 is 1.0
+//
+// A code field q left at mantissa bit p under the exponent of 1024 is the half 1024 + q * 2^p, so
+//     fma(v, 2^-p, -(2^(10-p) + z)) = q - z
+// with no rounding whenever q - z is a half; the product with the scale then rounds once, like
+// slim_dequant.  Positions 6..9 keep the constant 2^(10-p) + z below 32, where a half resolves
+// 1/64.  One shifted copy of a slice word therefore serves every field that lands in bits [6,10):
+// four 1-bit fields, two 2-bit fields or one 4-bit field; both halves of the word at once.
+constexpr uint32_t kMagic1024 = 0x64006400u;            // half2(1024, 1024): ulp 1
+
+__device__ __forceinline__ __half2 as_half2(uint32_t v) { return *reinterpret_cast<const __half2*>(&v); }
+__device__ __forceinline__ uint32_t as_u32(__half2 h) { return *reinterpret_cast<const uint32_t*>(&h); }
+// half2(2^e, 2^e), -14 <= e <= 15
+__device__ __forceinline__ __half2 pow2_h2(int e) { return as_half2(0x00010001u * (static_cast<uint32_t>(e + 15) << 10)); }
 
 struct DqRow {
-    __half2 zc;   // (16 + z, 16 + z)
-    __half2 s;    // (s, s)
+    __half2 s;        // (s, s)
+    __half2 add[4];   // -(constant of position i + z), see the decoders
 };
-// v holds two fields at mantissa bits [6,10) under the exponent of 16: returns s * (q - z) twice.
-__device__ __forceinline__ uint32_t dq_pair(uint32_t v, const DqRow& r) {
-    const __half2 h = __hmul2(__hsub2(*reinterpret_cast<const __half2*>(&v), r.zc), r.s);
-    return *reinterpret_cast<const uint32_t*>(&h);
-}
 __device__ __forceinline__ uint32_t lo_halves(uint32_t a, uint32_t b) { return g::prmt(a, b, 0x5410u); }
 __device__ __forceinline__ uint32_t hi_halves(uint32_t a, uint32_t b) { return g::prmt(a, b, 0x7632u); }
 
 // Logical shift, left if s > 0 (s is a constant after unrolling).
 __device__ __forceinline__ uint32_t shift_to(uint32_t v, int s) { return s >= 0 ? v << s : v >> (-s); }
 
+// Constants of a row for groups of B bits.  Position i of a copy holds a field at bit 6 + W*i
+// (W = field width of the slice: 1, 2, 2, 4 for B = 1..4).  For B = 3 the third bit of pair f
+// comes from a copy of the 1-bit slice at bit 6 + (f & 3) and enters through a second fma as
+// 4 * bit + 2^(6 - (f & 3)); that constant is taken off in advance with the first one.
+template <int B>
+__device__ __forceinline__ void row_constants(__half s, __half z, DqRow& r) {
+    r.s = __half2half2(s);
+    const __half2 z2 = __half2half2(z);
+    constexpr int W = B == 3 ? 2 : B;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float c = 0.f;
+        if (B == 3) c = static_cast<float>(1 << (4 - 2 * (i & 1))) + static_cast<float>(1 << (6 - i));
+        else if (W * i < 4) c = static_cast<float>(1 << (4 - W * i));
+        r.add[i] = __hsub2(__float2half2_rn(-c), z2);
+    }
+}
+
 // Fields of width W: F = 16/W pairs (f, f + F) per word; H[f] = (w[k0+f], w[k0+f+F]).  The word
 // covers 2F consecutive k; its F columns are (H[2j].lo, H[2j+1].lo) for j < F/2 and the hi halves
 // for the rest.  If HIGH, X carries a third code bit: bit f of its low/high half belongs to pair f.
 template <int W, int F, bool HIGH>
 __device__ __forceinline__ void decode_word(uint32_t word, uint32_t X, const DqRow& r, uint32_t* cols) {
-    constexpr uint32_t kMask = (0x00010001u * ((1u << W) - 1u)) << 6;
+    constexpr int PER = 4 / W;                                   // fields of one half served by one copy
+    constexpr uint32_t kField = 0x00010001u * ((1u << W) - 1u);
     uint32_t H[F];
 #pragma unroll
-    for (int f = 0; f < F; ++f) {
-        uint32_t v = (shift_to(word, 6 - W * f) & kMask) | kMagic16;
-        if (HIGH) v |= shift_to(X, 8 - f) & 0x01000100u;
-        H[f] = dq_pair(v, r);
+    for (int c = 0; c < F / PER; ++c) {
+        const uint32_t copy = shift_to(word, 6 - 4 * c);
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const int f = PER * c + i, pos = 6 + W * i;
+            const uint32_t v = (copy & (kField << pos)) | kMagic1024;
+            __half2 t = __hfma2(as_half2(v), pow2_h2(-pos), r.add[HIGH ? (f & 3) : i]);
+            if (HIGH) {
+                const int xpos = 6 + (f & 3);
+                const uint32_t vb = (shift_to(X, 6 - 4 * (f >> 2)) & (0x00010001u << xpos)) | kMagic1024;
+                t = __hfma2(as_half2(vb), pow2_h2(2 - xpos), t);
+            }
+            H[f] = as_u32(__hmul2(t, r.s));
+        }
     }
 #pragma unroll
     for (int j = 0; j < F / 2; ++j) {
@@ -270,13 +335,12 @@ __device__ __forceinline__ void decode_cword(const uint32_t (&words)[4], const D
 // ------------------------------------------------------------------------------------------ kernel
 template <int TOK> struct GemmCfg {
     static constexpr int HALF = TOK / 2;                     // tokens this CTA brings
-    static constexpr int NX = TOK == 256 ? 5 : 8;            // shared-memory stages of x
-    static constexpr int NP = TOK == 256 ? 6 : 8;            // shared-memory stages of packed slices
+    static constexpr int NP = 8;                             // shared-memory stages of packed slices
     static constexpr int XBOX = HALF * 128;                  // bytes of one TMA box: HALF rows x 64 k
     static constexpr int XSTAGE = 2 * XBOX;                  // one group: 128 k
-    static constexpr int OFF_P = NX * XSTAGE;
+    static constexpr int OFF_P = kNS * kGPS * XSTAGE;
     static constexpr int OFF_BAR = OFF_P + NP * kPStageBytes;
-    static constexpr int NBAR = 3 * NX + 2 * NP + 2 * kNA + 2;
+    static constexpr int NBAR = 3 * kNS + 2 * NP + 2;
     static constexpr int OFF_MISC = OFF_BAR + 8 * NBAR;      // tensor-memory base, abort flag
     static constexpr int SMEM = OFF_MISC + 16 + 1024;        // + slack to align the base to 1024
 };
@@ -298,24 +362,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rank = static_cast<int>(g::cluster_ctarank());     // 0 = leader of the pair
     const uint32_t bar0 = sbase + C::OFF_BAR;
-    // barriers of this CTA
-    auto x_full = [&](int s) { return bar0 + 8 * s; };
-    auto x_empty = [&](int s) { return bar0 + 8 * (C::NX + s); };
-    auto p_full = [&](int s) { return bar0 + 8 * (3 * C::NX + s); };
-    auto p_empty = [&](int s) { return bar0 + 8 * (3 * C::NX + C::NP + s); };
-    auto a_empty = [&](int s) { return bar0 + 8 * (3 * C::NX + 2 * C::NP + kNA + s); };
-    const uint32_t d_full = bar0 + 8 * (3 * C::NX + 2 * C::NP + 2 * kNA);
-    // barriers that live in the leader only: the other CTA reaches them through the cluster window
-    auto xp_full = [&](int s) { return bar0 + 8 * (2 * C::NX + s); };               // partner's half of x has landed
-    auto a_full = [&](int s) { return bar0 + 8 * (3 * C::NX + 2 * C::NP + s); };    // 16 dequant warps of the pair
-    const uint32_t d_empty = d_full + 8;                                            // 8 epilogue warps of the pair
+    // Barriers of this CTA.  Stage s is ready for the MMA when `full(s)` of the LEADER completes:
+    // 16 dequant warps of the pair have written A, the leader's half of x has landed (its TMA
+    // signals that barrier directly) and the other CTA's relay has reported its half (which lands
+    // on that CTA's `xl_full(s)`).  One multicast commit on `empty(s)` gives the stage back to the
+    // x producers and dequant warps of both CTAs.
+    auto xl_full = [&](int s) { return bar0 + 8 * s; };
+    auto full = [&](int s) { return bar0 + 8 * (kNS + s); };
+    auto empty = [&](int s) { return bar0 + 8 * (2 * kNS + s); };
+    auto p_full = [&](int s) { return bar0 + 8 * (3 * kNS + s); };
+    auto p_empty = [&](int s) { return bar0 + 8 * (3 * kNS + C::NP + s); };
+    const uint32_t d_full = bar0 + 8 * (3 * kNS + 2 * C::NP);
+    const uint32_t d_empty = d_full + 8;                 // leader's: 8 epilogue warps of the pair
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OFF_MISC);
     volatile int* abort = reinterpret_cast<volatile int*>(smem + C::OFF_MISC + 4);
 
     if (tid == 0) {
-        for (int s = 0; s < C::NX; ++s) { g::mbar_init(x_full(s), 1); g::mbar_init(x_empty(s), 1); g::mbar_init(xp_full(s), 1); }
+        for (int s = 0; s < kNS; ++s) { g::mbar_init(xl_full(s), 1); g::mbar_init(full(s), 18); g::mbar_init(empty(s), 1); }
         for (int s = 0; s < C::NP; ++s) { g::mbar_init(p_full(s), 1); g::mbar_init(p_empty(s), 8); }
-        for (int s = 0; s < kNA; ++s) { g::mbar_init(a_full(s), 16); g::mbar_init(a_empty(s), 1); }
         g::mbar_init(d_full, 1);
         g::mbar_init(d_empty, 8);
         *abort = 0;
@@ -343,62 +407,80 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
     const long long u0 = range_begin(cl), u1 = range_begin(cl + 1);
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ producer
+        // ------------------------------------------------------------------ producer of activations
         if (lane == 0) {
-            int sx = 0, sp = 0;
-            uint32_t phx = 0, php = 0;
+            int sx = 0;
+            uint32_t phx = 0;
             bool ok = true;
             for (long long u = u0; u < u1 && ok;) {
                 const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
                 const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
                 u += ge - gb;
-                const int rb = 2 * (tile % p.row_blocks) + rank, mt = tile / p.row_blocks;   // my 128-row block
+                const int m0 = (tile / p.row_blocks) * TOK + rank * C::HALF;     // my half of the token tile
+                for (int j = gb; j < ge; j += kGPS) {
+                    const int ng = min(kGPS, ge - j);                            // groups of this stage
+                    if (!g::mbar_wait(empty(sx), phx ^ 1u, abort)) { ok = false; break; }
+                    const uint32_t bar = rank == 0 ? full(sx) : xl_full(sx);
+                    g::mbar_expect_tx(bar, ng * C::XSTAGE);
+                    for (int i = 0; i < 2 * ng; ++i)                            // boxes of 64 k
+                        g::tma_load_2d(sbase + sx * kGPS * C::XSTAGE + i * C::XBOX, &x_map, SLIM_GROUP * j + 64 * i, m0, bar);
+                    if (++sx == kNS) { sx = 0; phx ^= 1u; }
+                }
+            }
+            if (ok) {
+                // every stage has been handed back: no commit of the leader is still on its way here
+                for (int s = 0; s < kNS && ok; ++s) {
+                    ok = g::mbar_wait(empty(sx), phx ^ 1u, abort);
+                    if (++sx == kNS) { sx = 0; phx ^= 1u; }
+                }
+            } else {
+                // leave no copy in flight: wait (bounded) for the last phase issued to every stage
+                for (int s = 0; s < kNS; ++s) g::mbar_drain(rank == 0 ? full(s) : xl_full(s), s < sx ? phx : phx ^ 1u);
+            }
+        }
+    } else if (warp == kWarpPacked) {
+        // ------------------------------------------------------------------ producer of packed slices, scales, zeros
+        // three lanes, one bulk copy each per group
+        if (lane < 3) {
+            int sp = 0;
+            uint32_t php = 0;
+            bool ok = true;
+            for (long long u = u0; u < u1 && ok;) {
+                const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
+                const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
+                u += ge - gb;
+                const int rb = 2 * (tile % p.row_blocks) + rank;                 // my 128-row block
                 const int tiles_here = max(0, min(8, (N >> 4) - 8 * rb));
-                for (int j = gb; j < ge && ok; ++j) {
-                    // my half of the group's activations
-                    if (!g::mbar_wait(x_empty(sx), phx ^ 1u, abort)) { ok = false; break; }
-                    g::mbar_expect_tx(x_full(sx), C::XSTAGE);
-                    g::tma_load_2d(sbase + sx * C::XSTAGE, &x_map, SLIM_GROUP * j, mt * TOK + rank * C::HALF, x_full(sx));
-                    g::tma_load_2d(sbase + sx * C::XSTAGE + C::XBOX, &x_map, SLIM_GROUP * j + 64, mt * TOK + rank * C::HALF, x_full(sx));
-                    if (++sx == C::NX) { sx = 0; phx ^= 1u; }
-                    // packed slices, scales, zeros of my rows
-                    if (!g::mbar_wait(p_empty(sp), php ^ 1u, abort)) { ok = false; break; }
+                const uint32_t sbytes = static_cast<uint32_t>(tiles_here) * 32u;
+                const __half* sz = (lane == 1 ? p.scales : p.zeros) + kRowsPerCta * rb;
+                for (int j = gb; j < ge; ++j) {
+                    // the three lanes go on, or give up, together
+                    if (!__all_sync(0x7u, g::mbar_wait(p_empty(sp), php ^ 1u, abort))) { ok = false; break; }
                     if (tiles_here > 0) {
-                        const int b = p.gt.bits[j];
-                        const uint32_t wbytes = static_cast<uint32_t>(tiles_here) * 256u * b, sbytes = static_cast<uint32_t>(tiles_here) * 32u;
+                        const uint32_t b = p.gt.bits[j];
+                        const uint32_t wbytes = static_cast<uint32_t>(tiles_here) * 256u * b;
                         const uint32_t dst = sbase + C::OFF_P + sp * kPStageBytes;
-                        g::mbar_expect_tx(p_full(sp), wbytes + 2 * sbytes);
-                        g::bulk_g2s(dst, p.packed + 16ull * N * p.gt.prefix[j] + static_cast<size_t>(8 * rb) * 256 * b, wbytes, p_full(sp));
-                        g::bulk_g2s(dst + 8192, p.scales + static_cast<size_t>(j) * N + kRowsPerCta * rb, sbytes, p_full(sp));
-                        g::bulk_g2s(dst + 8192 + 256, p.zeros + static_cast<size_t>(j) * N + kRowsPerCta * rb, sbytes, p_full(sp));
-                    } else {
+                        if (lane == 0) g::mbar_expect_tx(p_full(sp), wbytes + 2 * sbytes);
+                        __syncwarp(0x7u);
+                        if (lane == 0)
+                            g::bulk_g2s(dst, p.packed + 16ull * N * p.gt.prefix[j] + static_cast<size_t>(8 * rb) * 256 * b, wbytes, p_full(sp));
+                        else
+                            g::bulk_g2s(dst + 8192 + 256 * (lane - 1), sz + static_cast<size_t>(j) * N, sbytes, p_full(sp));
+                    } else if (lane == 0) {
                         g::mbar_arrive(p_full(sp));             // no row of mine exists: nothing to bring
                     }
                     if (++sp == C::NP) { sp = 0; php ^= 1u; }
                 }
             }
-            if (ok) {
-                // every x stage has been handed back: no commit of the leader is still on its way here
-                for (int s = 0; s < C::NX && ok; ++s) {
-                    ok = g::mbar_wait(x_empty(sx), phx ^ 1u, abort);
-                    if (++sx == C::NX) { sx = 0; phx ^= 1u; }
-                }
-            } else {
-                // leave no copy in flight: wait (bounded) for the last phase issued to every stage
-                auto drain = [&](uint32_t bar, uint32_t parity) {
-                    const unsigned long long t0 = g::global_timer_ns();
-                    while (!g::mbar_try_wait(bar, parity) && g::global_timer_ns() - t0 < 1000000ull) { }
-                };
-                for (int s = 0; s < C::NX; ++s) drain(x_full(s), s < sx ? phx : phx ^ 1u);
-                for (int s = 0; s < C::NP; ++s) drain(p_full(s), s < sp ? php : php ^ 1u);
-            }
+            if (!ok)
+                for (int s = 0; s < C::NP; ++s) g::mbar_drain(p_full(s), s < sp ? php : php ^ 1u);
         }
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
             // -------------------------------------------------------------- MMA issuer (leader)
             constexpr uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(TOK >> 3) << 17) | (static_cast<uint32_t>(kRowsPerPair >> 4) << 24);
-            int sx = 0, sa = 0;
-            uint32_t phx = 0, pha = 0, phd = 0;
+            int st = 0;
+            uint32_t ph = 0, phd = 0;
             bool ok = true;
             for (long long u = u0; u < u1 && ok;) {
                 const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
@@ -406,21 +488,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
                 u += ge - gb;
                 if (!g::mbar_wait(d_empty, phd ^ 1u, abort)) { ok = false; break; }   // both epilogues have drained D
                 g::tc_fence_after();
-                for (int j = gb; j < ge; ++j) {
-                    if (!g::mbar_wait(x_full(sx), phx, abort) || !g::mbar_wait(xp_full(sx), phx, abort) ||
-                        !g::mbar_wait(a_full(sa), pha, abort)) { ok = false; break; }
+                for (int j = gb; j < ge; j += kGPS) {
+                    const int nk = 8 * min(kGPS, ge - j);                        // K = 16 steps of this stage
+                    if (!g::mbar_wait(full(st), ph, abort)) { ok = false; break; }
                     g::tc_fence_after();
-                    const uint32_t xs = sbase + sx * C::XSTAGE;
-                    const uint32_t a_t = tmem + kTmemAcol + 64 * sa;
+                    const uint32_t xs = sbase + st * kGPS * C::XSTAGE;
+                    const uint32_t a_t = tmem + kTmemAcol + 64 * kGPS * st;
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint64_t bdesc = sw128_kmajor_desc(xs + (ks >> 2) * C::XBOX + (ks & 3) * 32);
-                        g::umma_f16_ts(tmem, a_t + 8 * ks, bdesc, idesc, (j > gb || ks != 0) ? 1u : 0u);
+                    for (int ks = 0; ks < 8 * kGPS; ++ks) {
+                        if (ks < nk) {
+                            const uint64_t bdesc = sw128_kmajor_desc(xs + (ks >> 2) * C::XBOX + (ks & 3) * 32);
+                            g::umma_f16_ts(tmem, a_t + 8 * ks, bdesc, idesc, (j > gb || ks != 0) ? 1u : 0u);
+                        }
                     }
-                    g::tc_commit_pair(x_empty(sx));
-                    g::tc_commit_pair(a_empty(sa));
-                    if (++sx == C::NX) { sx = 0; phx ^= 1u; }
-                    if (++sa == kNA) { sa = 0; pha ^= 1u; }
+                    g::tc_commit_pair(empty(st));
+                    if (++st == kNS) { st = 0; ph ^= 1u; }
                 }
                 if (ok) g::tc_commit_pair(d_full);
                 phd ^= 1u;
@@ -431,76 +513,97 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
             int sx = 0;
             uint32_t phx = 0;
             bool ok = true;
-            for (long long u = u0; u < u1 && ok; ++u) {
-                if (!g::mbar_wait(x_full(sx), phx, abort)) { ok = false; break; }
-                g::mbar_arrive_cluster(g::map_to_cta(xp_full(sx), 0));
-                if (++sx == C::NX) { sx = 0; phx ^= 1u; }
+            for (long long u = u0; u < u1 && ok;) {
+                const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
+                const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
+                u += ge - gb;
+                for (int j = gb; j < ge; j += kGPS) {
+                    if (!g::mbar_wait(xl_full(sx), phx, abort)) { ok = false; break; }
+                    g::mbar_arrive_cluster(g::map_to_cta(full(sx), 0));
+                    if (++sx == kNS) { sx = 0; phx ^= 1u; }
+                }
             }
         }
-    } else if (warp < 10) {
+    } else if (warp < kWarpEpi) {
         // ------------------------------------------------------------------ dequant warps
-        const int q = warp & 3, kh = (warp - 2) >> 2;           // tensor-memory lane quarter, k half of the group
+        // Warp = (tensor-memory lane quarter, k half of the group, set).  The two sets take
+        // alternate groups, so the fixed latencies of one group (barriers, shared-memory loads,
+        // tensor-memory store) overlap with the arithmetic of the next.
+        static_assert((kNS & (kNS - 1)) == 0 && (C::NP & (C::NP - 1)) == 0, "stage counters use masks");
+        constexpr int kSets = kDqWarps / 8;
+        const int q = warp & 3, kh = ((warp - 2) >> 2) & 1, set = (warp - 2) >> 3;
         const int r = 32 * q + lane;                            // row inside the block
         const int t = r >> 4, gq = (r & 15) >> 1, half = r & 1;
-        int sp = 0, sa = 0;
-        uint32_t php = 0, pha = 0;
         bool ok = true;
-        const uint32_t a_full_leader = g::map_to_cta(a_full(0), 0);
+        const uint32_t full_leader = g::map_to_cta(full(0), 0);
+        int si = 0, gi = 0;                                     // running numbers of the stage and of the group in this CTA's range
         for (long long u = u0; u < u1 && ok;) {
             const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
             const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
             u += ge - gb;
             const int rb = 2 * (tile % p.row_blocks) + rank;
             const bool row_ok = kRowsPerCta * rb + r < N;
-            for (int j = gb; j < ge; ++j) {
-                if (!g::mbar_wait(p_full(sp), php, abort)) { ok = false; break; }
-                const int b = p.gt.bits[j];
-                const uint32_t stage = sbase + C::OFF_P + sp * kPStageBytes;
-                uint32_t w0[4] = {0, 0, 0, 0}, w1[4] = {0, 0, 0, 0};   // words of units 0..3 for the two 32-k ranges
-                DqRow row;
-                row.zc = __float2half2_rn(16.f);
-                row.s = __float2half2_rn(0.f);
-                if (row_ok) {
+            for (int j = gb; j < ge && ok; j += kGPS, ++si) {
+                const int ng = min(kGPS, ge - j);                                // groups of this stage
+                const int g0 = gi;
+                gi += ng;
+                if (si % kSets != set) continue;
+                const int sa = si & (kNS - 1);
+                const uint32_t pha = (si / kNS) & 1;
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        if (u < b) {
-                            const uint4 v = g::lds128(stage + t * 256 * b + 256 * u + 8 * (4 * gq + 2 * kh));
-                            w0[u] = half ? v.y : v.x;
-                            w1[u] = half ? v.w : v.z;
+                for (int i = 0; i < kGPS; ++i) {
+                    if (i >= ng) break;
+                    const int sp = (g0 + i) & (C::NP - 1);
+                    const uint32_t php = ((g0 + i) / C::NP) & 1;
+                    if (!g::mbar_wait_warp(p_full(sp), php, abort)) { ok = false; break; }
+                    const int b = p.gt.bits[j + i];
+                    const uint32_t stage = sbase + C::OFF_P + sp * kPStageBytes;
+                    uint32_t w0[4] = {0, 0, 0, 0}, w1[4] = {0, 0, 0, 0};   // words of units 0..3 for the two 32-k ranges
+                    __half sc = __float2half_rn(0.f), zp = sc;             // rows past N: weight 0
+                    if (row_ok) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if (u < b) {
+                                const uint4 v = g::lds128(stage + t * 256 * b + 256 * u + 8 * (4 * gq + 2 * kh));
+                                w0[u] = half ? v.y : v.x;
+                                w1[u] = half ? v.w : v.z;
+                            }
                         }
+                        sc = *reinterpret_cast<const __half*>(smem + C::OFF_P + sp * kPStageBytes + 8192 + 2 * r);
+                        zp = *reinterpret_cast<const __half*>(smem + C::OFF_P + sp * kPStageBytes + 8192 + 256 + 2 * r);
                     }
-                    const __half s = *reinterpret_cast<const __half*>(smem + C::OFF_P + sp * kPStageBytes + 8192 + 2 * r);
-                    const __half z = *reinterpret_cast<const __half*>(smem + C::OFF_P + sp * kPStageBytes + 8192 + 256 + 2 * r);
-                    row.s = __half2half2(s);
-                    row.zc = __half2half2(__hadd(__float2half_rn(16.f), z));
-                }
-                __syncwarp();
-                if (lane == 0) g::mbar_arrive(p_empty(sp));
-                if (++sp == C::NP) { sp = 0; php ^= 1u; }
+                    __syncwarp();
+                    if (lane == 0) g::mbar_arrive(p_empty(sp));
 
-                uint32_t cols[32];
-                switch (b) {
-                    case 1: decode_cword<1>(w0, row, cols); decode_cword<1>(w1, row, cols + 16); break;
-                    case 2: decode_cword<2>(w0, row, cols); decode_cword<2>(w1, row, cols + 16); break;
-                    case 3: decode_cword<3>(w0, row, cols); decode_cword<3>(w1, row, cols + 16); break;
-                    default: decode_cword<4>(w0, row, cols); decode_cword<4>(w1, row, cols + 16); break;
+                    const uint32_t a_t = tmem + (static_cast<uint32_t>(32 * q) << 16) + kTmemAcol + 64 * (kGPS * sa + i) + 32 * kh;
+                    uint32_t cols[16];
+                    DqRow row;
+                    // first 32 k of my half, then (the stage's columns are free by now) the other 32
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t (&w)[4] = h == 0 ? w0 : w1;
+                        switch (b) {
+                            case 1: if (h == 0) row_constants<1>(sc, zp, row); decode_cword<1>(w, row, cols); break;
+                            case 2: if (h == 0) row_constants<2>(sc, zp, row); decode_cword<2>(w, row, cols); break;
+                            case 3: if (h == 0) row_constants<3>(sc, zp, row); decode_cword<3>(w, row, cols); break;
+                            default: if (h == 0) row_constants<4>(sc, zp, row); decode_cword<4>(w, row, cols); break;
+                        }
+                        if (h == 0 && i == 0) {
+                            if (!g::mbar_wait_warp(empty(sa), pha ^ 1u, abort)) { ok = false; break; }
+                            g::tc_fence_after();
+                        }
+                        g::tmem_st16(a_t + 16 * h, cols);
+                    }
+                    if (!ok) break;
                 }
-                if (!g::mbar_wait(a_empty(sa), pha ^ 1u, abort)) { ok = false; break; }
-                g::tc_fence_after();
-                g::tmem_st32(tmem + (static_cast<uint32_t>(32 * q) << 16) + kTmemAcol + 64 * sa + 32 * kh, cols);
+                if (!ok) break;
                 g::tc_wait_st();
                 g::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) g::mbar_arrive_cluster(a_full_leader + 8 * sa);
-                if (++sa == kNA) { sa = 0; pha ^= 1u; }
+                if (lane == 0) g::mbar_arrive_cluster(full_leader + 8 * sa);
             }
         }
-        // every A stage has been handed back: no commit of the leader is still on its way here
-        for (int s = 0; s < kNA && ok; ++s) {
-            ok = g::mbar_wait(a_empty(sa), pha ^ 1u, abort);
-            if (++sa == kNA) { sa = 0; pha ^= 1u; }
-        }
-    } else {
+    } else if (warp < kWarpPacked) {
         // ------------------------------------------------------------------ epilogue warps
         // A segment that covers its whole tile is stored as fp16.  With stream-K a tile may be cut:
         // a pair whose segment does not start the tile leaves its fp32 partials in its CTAs'
@@ -509,7 +612,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
         // pair order and stores the tile.  Each CTA deals with the CTAs of the same rank, which
         // hold the same 128 rows.
         const int q = warp & 3;
-        const int et = tid - 320;                               // 0..127 among the epilogue threads
+        const int et = tid - 32 * kWarpEpi;                     // 0..127 among the epilogue threads
         uint32_t phd = 0;
         bool ok = true;
         const uint32_t d_empty_leader = g::map_to_cta(d_empty, 0);
@@ -552,41 +655,41 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
             float* my_slot = p.partials + static_cast<size_t>(blockIdx.x) * (TOK * kRowsPerCta) + 32 * q + lane;
             if (is_partial) {
 #pragma unroll 1
-                for (int cc = 0; cc < TOK / 32; ++cc) {
-                    uint32_t v[32];
-                    g::tmem_ld32(tmem + (static_cast<uint32_t>(32 * q) << 16) + 32 * cc, v);
+                for (int cc = 0; cc < TOK / kEpiCols; ++cc) {
+                    uint32_t v[kEpiCols];
+                    g::tmem_ld16(tmem + (static_cast<uint32_t>(32 * q) << 16) + kEpiCols * cc, v);
                     g::tc_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) my_slot[(32 * cc + i) * kRowsPerCta] = __uint_as_float(v[i]);
+                    for (int i = 0; i < kEpiCols; ++i) my_slot[(kEpiCols * cc + i) * kRowsPerCta] = __uint_as_float(v[i]);
                 }
             } else {
-                // sum of the peers' partials for one 32-token chunk, in CTA order
-                auto peer_sum = [&](int cc, float (&t)[32]) {
+                // sum of the peers' partials for one chunk of tokens, in CTA order
+                auto peer_sum = [&](int cc, float (&t)[kEpiCols]) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) t[i] = 0.f;
+                    for (int i = 0; i < kEpiCols; ++i) t[i] = 0.f;
                     for (int k = 1; k <= npeer; ++k) {
                         if (!peer_active(k)) continue;
                         const float* slot = p.partials + static_cast<size_t>(blockIdx.x + 2 * k) * (TOK * kRowsPerCta) + 32 * q + lane;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) t[i] += __ldcg(slot + (32 * cc + i) * kRowsPerCta);
+                        for (int i = 0; i < kEpiCols; ++i) t[i] += __ldcg(slot + (kEpiCols * cc + i) * kRowsPerCta);
                     }
                 };
-                float t[32];
+                float t[kEpiCols];
                 if (npeer > 0) peer_sum(0, t);
 #pragma unroll 1
-                for (int cc = 0; cc < TOK / 32; ++cc) {
-                    uint32_t v[32];
-                    g::tmem_ld32(tmem + (static_cast<uint32_t>(32 * q) << 16) + 32 * cc, v);
+                for (int cc = 0; cc < TOK / kEpiCols; ++cc) {
+                    uint32_t v[kEpiCols];
+                    g::tmem_ld16(tmem + (static_cast<uint32_t>(32 * q) << 16) + kEpiCols * cc, v);
                     g::tc_wait_ld();
                     if (npeer > 0) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + t[i]);
-                        if (cc + 1 < TOK / 32) peer_sum(cc + 1, t);     // in flight while this chunk is stored
+                        for (int i = 0; i < kEpiCols; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + t[i]);
+                        if (cc + 1 < TOK / kEpiCols) peer_sum(cc + 1, t);     // in flight while this chunk is stored
                     }
-                    const int m0 = mt * TOK + 32 * cc;
+                    const int m0 = mt * TOK + kEpiCols * cc;
                     if (n < N) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
+                        for (int i = 0; i < kEpiCols; ++i)
                             if (m0 + i < p.M) p.y[static_cast<size_t>(m0 + i) * N + n] = __float2half_rn(__uint_as_float(v[i]));
                     }
                 }
