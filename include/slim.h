@@ -155,6 +155,61 @@ int slim_mpq_gemm_static(const void* x, const void* packed, const uint8_t* bits_
                          const void* scales, const void* zeros, void* y,
                          int M, int N, int K, int g, unsigned int* status_out, void* stream);
 
+/* ---- layer-set launch of the decode path --------------------------------------------------- */
+
+/* Several INDEPENDENT layers of the decode path (1 <= M <= 16 each) in one launch: the q/k/v or
+ * gate/up projections that share an input, or a sweep over a model's layers.  (The paper launches
+ * its kernel per layer, App. B.2; a decode-sized layer is too small to keep HBM busy on its own,
+ * so the set is walked by persistent CTAs that stream the packed slices of one 128-row block after
+ * another through a ring of shared-memory slots, with no pause between layers.)  No layer of a set
+ * may read what another layer of the same set writes.
+ *
+ * Every layer gets the y = x * W-hat^T of slim_mpq_gemv (same products, fp32 accumulation in a
+ * different order, fp16 output); the results are deterministic for a given (set, device).
+ * N > 0 a multiple of 16, K > 0 a multiple of 128. */
+typedef struct slim_layer {
+    const void* x;             /* device fp16 [M][K] */
+    const void* packed;        /* device, packed codes of the layer */
+    const void* scales;        /* device fp16 [G][N] */
+    const void* zeros;         /* device fp16 [G][N] */
+    void* y;                   /* device fp16 [M][N] */
+    const uint8_t* bits_host;  /* host [K/g] */
+    int M, N, K;
+} slim_layer;
+
+/* Filled by slim_gemv_set_plan, read by slim_mpq_gemv_set; plain data owned by the caller. */
+typedef struct slim_gemv_set_info {
+    int n_layers;
+    int grid;              /* persistent CTAs */
+    int n_slots;           /* ring slots per CTA */
+    int slot_bytes;
+    int token_tiles;       /* 8-token MMA tiles: 1 or 2 */
+    int stage_tasks;       /* (layer, token, group) triples of the set */
+    int n_items;           /* 128-row blocks of the set */
+    int max_bits;          /* widest group of the set */
+    size_t plan_bytes;
+    size_t workspace_bytes;
+} slim_gemv_set_info;
+
+/* Host-only.  Sizes of the device plan buffer and of the workspace a set needs on the current
+ * device.  The workspace holds the status word and, per layer, its activations in tensor-core
+ * fragment order. */
+int slim_gemv_set_bytes(const slim_layer* layers_host, int n_layers, int g,
+                        size_t* plan_bytes, size_t* workspace_bytes);
+
+/* Validates the set, lays the work out over the device's SMs and writes the plan (layer
+ * descriptors, item ranges of every CTA) into `plan` (device, 16-byte aligned, plan_bytes from
+ * slim_gemv_set_bytes) with copies enqueued on `stream`; fills *info.  layers_host and the bit
+ * maps are read during the call only.  The plan stays valid while the layers' pointers do. */
+int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g,
+                       void* plan, size_t plan_bytes, slim_gemv_set_info* info, void* stream);
+
+/* Runs the set: one small kernel puts every layer's activations into fragment order in the
+ * workspace, one persistent kernel computes all layers.  `workspace` as for slim_mpq_gemv
+ * (zeroed once with slim_workspace_init; slim_workspace_status reports a device-side time-out). */
+int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- producing the inputs of the layer (the steps right before packing) ------------------- */
 
 /* Group salience S_j = sum_{k in group j} a_k^2 * sum_n W[n][k]^2 (diagonal form of Definition 1 /

@@ -58,6 +58,9 @@ def lib():
             "slim_group_salience": [vp, vp, vp, i, i, i, vp],
             "slim_allocate_bits": [vp, i, i, i, vp],
             "slim_quantize_minmax": [vp, vp, vp, vp, vp, i, i, i, vp],
+            "slim_gemv_set_bytes": [vp, i, i, ctypes.POINTER(sz), ctypes.POINTER(sz)],
+            "slim_gemv_set_plan": [vp, i, i, vp, sz, vp, vp],
+            "slim_mpq_gemv_set": [vp, vp, vp, sz, vp],
         }
         for name, args in sigs.items():
             fn = getattr(L, name)
@@ -239,6 +242,65 @@ def quantize_sqc(W: torch.Tensor, bits, lam: float = 0.1, n: int = 50):
                                                         _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
                                                         _dev(tau, torch.int32, "tau_index"), N, K, GROUP, float(lam), int(n), _stream(W)))
     return codes, scales, zeros, tau
+
+
+class _Layer(ctypes.Structure):
+    """struct slim_layer"""
+    _fields_ = [("x", ctypes.c_void_p), ("packed", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("zeros", ctypes.c_void_p),
+                ("y", ctypes.c_void_p), ("bits_host", ctypes.c_void_p), ("M", ctypes.c_int), ("N", ctypes.c_int), ("K", ctypes.c_int)]
+
+
+class _SetInfo(ctypes.Structure):
+    """struct slim_gemv_set_info"""
+    _fields_ = [("n_layers", ctypes.c_int), ("grid", ctypes.c_int), ("n_slots", ctypes.c_int), ("slot_bytes", ctypes.c_int),
+                ("token_tiles", ctypes.c_int), ("stage_tasks", ctypes.c_int), ("n_items", ctypes.c_int), ("max_bits", ctypes.c_int),
+                ("plan_bytes", ctypes.c_size_t), ("workspace_bytes", ctypes.c_size_t)]
+
+
+class LayerSet:
+    """Several independent decode-path layers run by one launch (slim_gemv_set_plan / slim_mpq_gemv_set).
+
+    entries: sequence of (layer: QuantLinear, x: fp16 CUDA [M][K], y: fp16 CUDA [M][N]).  The plan
+    and the workspace are torch tensors owned by this object; the tensors of the entries are kept
+    alive with it."""
+
+    def __init__(self, entries, g: int = GROUP):
+        entries = list(entries)
+        if not entries:
+            raise ValueError("a layer set needs at least one layer")
+        self._keep = entries
+        self._bits = [_bits(L.bits) for (L, _, _) in entries]
+        arr = (_Layer * len(entries))()
+        for k, (L, x, y) in enumerate(entries):
+            M = x.shape[0]
+            if tuple(x.shape) != (M, L.K) or tuple(y.shape) != (M, L.N):
+                raise ValueError(f"layer {k}: x must be [M][{L.K}] and y [M][{L.N}]")
+            arr[k] = _Layer(_dev(x, torch.float16, "x"), _dev(L.packed, torch.uint8, "packed"), _dev(L.scales, torch.float16, "scales"),
+                            _dev(L.zeros, torch.float16, "zeros"), _dev(y, torch.float16, "y"), self._bits[k].ctypes.data,
+                            M, L.N, L.K)
+        self._arr = arr
+        device = entries[0][1].device
+        pb, wb = ctypes.c_size_t(0), ctypes.c_size_t(0)
+        _check("slim_gemv_set_bytes", lib().slim_gemv_set_bytes(ctypes.cast(arr, ctypes.c_void_p), len(entries), g,
+                                                              ctypes.byref(pb), ctypes.byref(wb)))
+        self.plan = torch.empty(pb.value, dtype=torch.uint8, device=device)
+        self.workspace = torch.empty(max(wb.value, 256), dtype=torch.uint8, device=device)
+        workspace_init(self.workspace)
+        self._info = _SetInfo()
+        _check("slim_gemv_set_plan", lib().slim_gemv_set_plan(ctypes.cast(arr, ctypes.c_void_p), len(entries), g, self.plan.data_ptr(),
+                                                            self.plan.numel(), ctypes.addressof(self._info), _stream(self.plan)))
+
+    @property
+    def info(self) -> dict:
+        return {name: getattr(self._info, name) for name, _ in _SetInfo._fields_}
+
+    def run(self) -> None:
+        """Enqueues the set on the current stream: y of every entry is overwritten."""
+        _check("slim_mpq_gemv_set", lib().slim_mpq_gemv_set(ctypes.addressof(self._info), self.plan.data_ptr(), self.workspace.data_ptr(),
+                                                          self.workspace.numel(), _stream(self.plan)))
+
+    def check(self) -> None:
+        workspace_status(self.workspace)
 
 
 class QuantLinear:

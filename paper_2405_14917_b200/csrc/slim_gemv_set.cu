@@ -1,0 +1,558 @@
+// slim_mpq_gemv_set: the decode path (1 <= M <= 16) over a set of independent layers, sm_100a.
+//
+// A decode-sized layer holds fewer bytes than HBM must keep in flight, so a launch per layer
+// leaves the memory system idle while kernels start, stage x and reduce.  Here the whole set is
+// one stream of work items for persistent CTAs:
+//
+//  * item = (layer, block of 128 rows = 8 tiles of 16), the full K of the layer.  The items of
+//    the set are cut into one contiguous range per CTA, balanced by packed bytes, on the host.
+//  * x is put into B-fragment order once per layer by a small kernel (one warp per token and
+//    group; the routine slim_mpq_gemv uses) and kept in the workspace; every item re-reads its
+//    fragments from L2.
+//  * a producer warp walks the CTA's items group by group and brings, per group, the slices of the
+//    8 tiles (one contiguous piece of the packed buffer), their scales and zeros, the group's
+//    fragments and its (sum_k x, 2^(24-S)) into the next slot of a shared-memory ring with
+//    cp.async.bulk; mbarriers hand the slots back and forth.  The ring never drains between items
+//    or layers, so HBM always has the ring's worth of bytes in flight per CTA.
+//  * consumer warp w owns tile w of the item: per group one pass of mma.sync m16n8k16 over raw
+//    code fields (subnormal-mantissa operands, see slim_gemv_dev.cuh / slim_gemv.cu) and the fold
+//    acc += s * (D * 2^(24-S) - z * sum_k x); after the last group it stores its 16 rows.  A warp
+//    walks the whole K itself: no partial sums, no reduction between warps or CTAs.
+//
+// Every wait on an mbarrier is bounded and reports through the workspace status word.
+#include "slim_gemv_dev.cuh"
+
+#include <cstring>
+
+namespace slim {
+
+constexpr int kSetConsumers = 8;                       // consumer warps = tiles of an item
+constexpr int kSetProducers = 2;                       // producer warps: they take the groups in turn
+constexpr int kSetThreads = 32 * (kSetConsumers + kSetProducers);
+constexpr int kSetRowsPerItem = 16 * kSetConsumers;
+constexpr int kSetMaxSlots = 32;
+constexpr int kSetHeader = 16;                         // slot header: bit-width of the group
+constexpr unsigned long long kSetWaitNs = 2000000000ull;
+
+// Device-side description of one layer (lives in the plan buffer).
+struct SetLayer {
+    const __half* x;
+    const uint8_t* packed;
+    const __half* scales;
+    const __half* zeros;
+    __half* y;
+    size_t x_off;          // workspace offset of the layer's staged activations, group after group:
+                           // (sum_k x, 2^(24-S)) float2[16], then the fragments [slice][8 mma][M][4 lanes] x 8 B
+    size_t pad0;
+    int M, N, K, G;
+    int item0, n_items;    // this layer's items in the set's numbering
+    int task0;             // first (token, group) staging task of the layer
+    int pad;
+    uint16_t prefix[SLIM_MAX_GROUPS + 1];
+    uint16_t pre3[SLIM_MAX_GROUPS + 1];   // 3-bit groups (two slices) before group j
+    uint8_t bits[SLIM_MAX_GROUPS];
+    uint8_t pad2[4];
+};
+static_assert(sizeof(SetLayer) % 16 == 0, "descriptors are copied and read in 16-byte pieces");
+
+// Plan buffer: int item_begin[grid + 1] (padded to kSetPlanHeader bytes), then the descriptors.
+constexpr int kSetMaxGrid = 1023;
+constexpr size_t kSetPlanHeader = 4096;
+
+struct SetParams {
+    const int* item_begin;
+    const SetLayer* layers;
+    uint8_t* ws;                           // workspace: status word, then the layers' fragments and sums
+    int n_layers, n_slots, slot_bytes;
+    int off_s, off_z, off_e, off_x;        // offsets inside a slot (weights start at kSetHeader)
+};
+
+// ------------------------------------------------------------------------------------------ mbarrier helpers
+namespace sb {
+__device__ __forceinline__ void init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up when the limit passes or when another role has raised `abort`.
+__device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+    if (try_wait(bar, parity)) return true;
+    const unsigned long long t0 = timer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (try_wait(bar, parity)) return true;
+        if (*abort != 0) return false;
+        if (timer_ns() - t0 > kSetWaitNs) { *abort = 1; return false; }
+    }
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+}  // namespace sb
+
+// ------------------------------------------------------------------------------------------ activation staging
+// Byte offset of group j inside a layer's staged activations (pre3 = 3-bit groups before j).
+__host__ __device__ inline size_t staged_group_offset(int j, int pre3, int M) {
+    return 128u * static_cast<size_t>(j) + 256u * static_cast<size_t>(M) * static_cast<size_t>(j + pre3);
+}
+// One warp per (layer, token, group): fragments and sums of the whole set, once.
+__global__ void __launch_bounds__(256) gemv_set_stage_kernel(const SetLayer* __restrict__ layers, uint8_t* ws, int n_layers, int n_tasks) {
+    const int lane = threadIdx.x & 31;
+    const int task = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (task >= n_tasks) return;
+    int lo = 0, hi = n_layers - 1;                       // last layer whose task0 <= task
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (layers[mid].task0 <= task) lo = mid; else hi = mid - 1;
+    }
+    const SetLayer& L = layers[lo];
+    const int pi = task - L.task0;
+    const int m = pi / L.G, j = pi - m * L.G;
+    uint8_t* grp = ws + L.x_off + staged_group_offset(j, L.pre3[j], L.M);
+    float2* sxe = reinterpret_cast<float2*>(grp);
+    const float2 r = stage_group(L.x + static_cast<size_t>(m) * L.K + j * SLIM_GROUP, grp + 128, L.bits[j], m, L.M, lane);
+    if (lane == 0) sxe[m] = r;
+    if (m == 0 && lane < 16 && lane >= L.M) sxe[lane] = make_float2(0.f, 1.f);   // absent tokens read 0
+}
+
+// ------------------------------------------------------------------------------------------ the persistent kernel
+constexpr uint32_t kSetOffAbort = 16 * kSetMaxSlots;          // after the full and empty barriers
+constexpr uint32_t kSetOffDesc = 1024;                        // the producer's copy of its layer's descriptor
+constexpr uint32_t kSetOffRing = (kSetOffDesc + kSetProducers * sizeof(SetLayer) + 127) / 128 * 128;
+
+template <int NT>   // 8-token MMA tiles: 1 (every M <= 8) or 2
+__global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_constant__ SetParams p) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    const uint32_t sbase = smem_u32(smem);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    auto full = [&](int s) { return sbase + 8u * s; };
+    auto empty = [&](int s) { return sbase + 8u * (kSetMaxSlots + s); };
+    volatile int* abort = reinterpret_cast<volatile int*>(smem + kSetOffAbort);
+    const uint32_t ring = sbase + kSetOffRing;
+
+    if (tid == 0) {
+        for (int s = 0; s < p.n_slots; ++s) { sb::init(full(s), 1); sb::init(empty(s), kSetConsumers); }
+        *abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    const int i0 = p.item_begin[blockIdx.x], i1 = p.item_begin[blockIdx.x + 1];
+    if (i0 < i1) {
+        int l = 0;                                        // layer of item i0
+        {
+            int lo = 0, hi = p.n_layers - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (p.layers[mid].item0 <= i0) lo = mid; else hi = mid - 1;
+            }
+            l = lo;
+        }
+        if (warp >= kSetConsumers) {
+            // -------------------------------------------------------------- producers
+            // producer warp w takes the groups whose running number is w modulo the number of producers
+            const int pw = warp - kSetConsumers;
+            uint8_t* desc = smem + kSetOffDesc + pw * sizeof(SetLayer);
+            const SetLayer* D = reinterpret_cast<const SetLayer*>(desc);
+            int have = -1;                                // layer whose descriptor is in shared memory
+            // ring position of the next group this warp fills: it advances by the number of producers
+            int s = pw;
+            uint32_t ph = 0;
+            uint32_t cnt = 0;                             // running number of the group in this CTA's range
+            bool ok = true;
+            for (int i = i0; i < i1 && ok; ++i) {
+                while (i >= p.layers[l].item0 + p.layers[l].n_items) ++l;
+                if (have != l) {
+                    const uint4* src = reinterpret_cast<const uint4*>(p.layers + l);
+                    uint4* dst = reinterpret_cast<uint4*>(desc);
+                    for (int q = lane; q < static_cast<int>(sizeof(SetLayer) / 16); q += 32) dst[q] = src[q];
+                    __syncwarp();
+                    have = l;
+                }
+                const int rb = i - D->item0, N = D->N, M = D->M, G = D->G;
+                const int tiles_here = min(kSetConsumers, (N >> 4) - kSetConsumers * rb);
+                // lane 0 brings the slices, lanes 1 and 2 scales and zeros, lane 3 the staged activations
+                const uint8_t* base = lane == 0 ? D->packed
+                                    : lane == 1 ? reinterpret_cast<const uint8_t*>(D->scales + kSetRowsPerItem * rb)
+                                    : lane == 2 ? reinterpret_cast<const uint8_t*>(D->zeros + kSetRowsPerItem * rb)
+                                                : p.ws + D->x_off;
+                const uint32_t dst_off = lane == 0 ? kSetHeader : lane == 1 ? p.off_s : lane == 2 ? p.off_z : p.off_e;
+                const uint32_t szb = static_cast<uint32_t>(tiles_here) * 32u;
+                int j = static_cast<int>((static_cast<uint32_t>(pw) + kSetProducers - cnt % kSetProducers) % kSetProducers);
+                cnt += static_cast<uint32_t>(G);
+                for (; j < G; j += kSetProducers) {
+                    // the lanes go on, or give up, together
+                    if (!__all_sync(0xffffffffu, sb::wait(empty(s), ph ^ 1u, abort))) { ok = false; break; }
+                    const uint32_t b = D->bits[j];
+                    const uint32_t wbytes = static_cast<uint32_t>(tiles_here) * 256u * b;
+                    const uint32_t xbytes = 128u + static_cast<uint32_t>(slice_count(b)) * 256u * M;
+                    const uint32_t slot = ring + static_cast<uint32_t>(s) * p.slot_bytes;
+                    if (lane == 0) {
+                        asm volatile("st.shared.u32 [%0], %1;" ::"r"(slot), "r"(b) : "memory");
+                        sb::expect_tx(full(s), wbytes + 2 * szb + xbytes);
+                    }
+                    const size_t off = lane == 0 ? 16ull * N * D->prefix[j] + static_cast<size_t>(kSetConsumers * rb) * 256 * b
+                                     : lane == 3 ? staged_group_offset(j, D->pre3[j], M)
+                                                 : 2ull * static_cast<size_t>(j) * N;
+                    const uint32_t bytes = lane == 0 ? wbytes : lane == 3 ? xbytes : szb;
+                    __syncwarp();
+                    if (lane < 4) sb::bulk_g2s(slot + dst_off, base + off, bytes, full(s));
+                    s += kSetProducers;
+                    if (s >= p.n_slots) { s -= p.n_slots; ph ^= 1u; }
+                }
+            }
+            if (!ok && lane == 0) {
+                // leave no copy in flight: give what was issued a millisecond to land
+                const unsigned long long t0 = sb::timer_ns();
+                while (sb::timer_ns() - t0 < 1000000ull) { }
+            }
+        } else {
+            // -------------------------------------------------------------- consumer: tile `warp` of every item
+            const int gq = lane >> 2, c = lane & 3;
+            int s = 0;                                    // ring position of the next group
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int i = i0; i < i1 && ok; ++i) {
+                while (i >= p.layers[l].item0 + p.layers[l].n_items) ++l;
+                const SetLayer& L = p.layers[l];
+                const int rb = i - L.item0, N = L.N, M = L.M, G = L.G;
+                const int tile = kSetConsumers * rb + warp;
+                const bool active = tile < (N >> 4);
+                float acc[NT][4];
+#pragma unroll
+                for (int n = 0; n < NT; ++n)
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) acc[n][r] = 0.f;
+
+                for (int j = 0; j < G; ++j) {
+                    if (!__all_sync(0xffffffffu, sb::wait(full(s), ph, abort))) { ok = false; break; }
+                    const uint32_t slot = ring + static_cast<uint32_t>(s) * p.slot_bytes;
+                    if (active) {
+                        const int b = static_cast<int>(lds32(slot));
+                        const uint32_t item = slot + kSetHeader + static_cast<uint32_t>(warp) * 256u * b;
+                        const uint32_t xs_slot0 = slot + p.off_x;
+                        constexpr int CH = NT == 1 ? 4 : 2;      // interleaved accumulation chains
+                        float d[CH][NT][4];
+#pragma unroll
+                        for (int h = 0; h < CH; ++h)
+#pragma unroll
+                            for (int n = 0; n < NT; ++n)
+#pragma unroll
+                                for (int r = 0; r < 4; ++r) d[h][n][r] = 0.f;
+
+                        // one slice of width WD starting at unit `unit0`, activations in fragment slot `xs_slot`
+                        auto run_slice = [&](auto wtag, int unit0, uint32_t xs_slot) {
+                            constexpr int WD = decltype(wtag)::value;
+                            constexpr int MPU = 8 / WD;                 // MMAs per unit
+#pragma unroll
+                            for (int u = 0; u < WD; ++u) {
+                                const uint2 wd = lds64(item + 256 * (unit0 + u) + 8 * lane);
+                                const uint32_t shx = wd.x >> pair_shift(WD), shy = wd.y >> pair_shift(WD);
+#pragma unroll
+                                for (int ii = 0; ii < MPU; ++ii) {
+                                    const uint32_t a0 = pair<WD>(wd.x, shx, 2 * ii), a1 = pair<WD>(wd.y, shy, 2 * ii);
+                                    const uint32_t a2 = pair<WD>(wd.x, shx, 2 * ii + 1), a3 = pair<WD>(wd.y, shy, 2 * ii + 1);
+                                    const int mi = u * MPU + ii;
+#pragma unroll
+                                    for (int n = 0; n < NT; ++n) {
+                                        const int m = 8 * n + gq;
+                                        uint2 bv = make_uint2(0u, 0u);
+                                        if (m < M) bv = lds64(xs_slot + ((mi * M + m) * 4 + c) * 8);
+                                        mma_f16(d[(u * MPU + ii) & (CH - 1)][n], a0, a1, a2, a3, bv);
+                                    }
+                                }
+                            }
+                        };
+                        switch (b) {
+                            case 1: run_slice(W1{}, 0, xs_slot0); break;
+                            case 2: run_slice(W2{}, 0, xs_slot0); break;
+                            case 3: run_slice(W2{}, 0, xs_slot0); run_slice(W1{}, 2, xs_slot0 + 8 * M * 32); break;
+                            default: run_slice(W4{}, 0, xs_slot0); break;
+                        }
+
+                        // fold the group: acc += s * (D * 2^(24-S) - z * sum_x); rows 2gq, 2gq+1, tokens 8n+2c, 8n+2c+1
+                        const uint32_t s2 = lds32(slot + p.off_s + warp * 32 + gq * 4);
+                        const uint32_t z2 = lds32(slot + p.off_z + warp * 32 + gq * 4);
+                        const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
+                        const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
+                        const float2* sxe = reinterpret_cast<const float2*>(smem + (slot - sbase) + p.off_e);
+#pragma unroll
+                        for (int n = 0; n < NT; ++n) {
+                            const float4 t = *reinterpret_cast<const float4*>(sxe + 8 * n + 2 * c);   // (sx0, e0, sx1, e1)
+                            float dd[4];
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) {
+                                dd[r] = d[0][n][r] + d[1][n][r];
+                                if (CH == 4) dd[r] += d[2][n][r] + d[3][n][r];
+                            }
+                            const float d0 = dd[0] * t.y, d1 = dd[1] * t.w, d2 = dd[2] * t.y, d3 = dd[3] * t.w;
+                            acc[n][0] = fmaf(sf.x, fmaf(-zf.x, t.x, d0), acc[n][0]);
+                            acc[n][1] = fmaf(sf.x, fmaf(-zf.x, t.z, d1), acc[n][1]);
+                            acc[n][2] = fmaf(sf.y, fmaf(-zf.y, t.x, d2), acc[n][2]);
+                            acc[n][3] = fmaf(sf.y, fmaf(-zf.y, t.z, d3), acc[n][3]);
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) sb::arrive(empty(s));
+                    if (++s == p.n_slots) { s = 0; ph ^= 1u; }
+                }
+                // ---- this warp's 16 rows of the item: rows 2gq, 2gq+1 of tokens 8n+2c, 8n+2c+1
+                if (active && ok) {
+                    __half* yrow = L.y + 16 * tile + 2 * gq;
+#pragma unroll
+                    for (int n = 0; n < NT; ++n) {
+                        const int m0 = 8 * n + 2 * c;
+                        if (m0 < M) *reinterpret_cast<__half2*>(yrow + static_cast<size_t>(m0) * N) = __floats2half2_rn(acc[n][0], acc[n][2]);
+                        if (m0 + 1 < M) *reinterpret_cast<__half2*>(yrow + static_cast<size_t>(m0 + 1) * N) = __floats2half2_rn(acc[n][1], acc[n][3]);
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (tid == 0 && *abort != 0) atomicOr(reinterpret_cast<unsigned int*>(p.ws), 1u);
+}
+
+// ------------------------------------------------------------------------------------------ host side
+// What the whole set fixes: token tiles, slot geometry, ring depth, grid, sizes.
+struct SetGeometry {
+    int nt, bmax, mmax;
+    int off_s, off_z, off_e, off_x, slot_bytes;
+    int n_slots, grid, ctas_per_sm;
+    size_t smem_bytes;
+    long long n_items, n_tasks;
+    unsigned long long total_cost;     // packed + scale + zero bytes of the set
+    size_t ws_bytes;
+};
+
+static size_t align_to(size_t v, size_t a) { return (v + a - 1) / a * a; }
+// Workspace of one layer: per group the sums and the fragments of its slices.
+static size_t layer_ws_bytes(int M, const GroupTable& gt) {
+    int slots = gt.G;
+    for (int j = 0; j < gt.G; ++j) slots += gt.bits[j] == 3 ? 1 : 0;
+    return align_to(static_cast<size_t>(gt.G) * 128 + static_cast<size_t>(slots) * 256 * M, 128);
+}
+static unsigned long long item_cost(int tiles_here, const GroupTable& gt) {
+    return static_cast<unsigned long long>(tiles_here) * (256ull * gt.prefix[gt.G] + 64ull * gt.G);
+}
+
+static int set_sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    return n;
+}
+
+// First pass over the set: validation of the shapes and everything that depends on all layers.
+static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeometry* sg) {
+    if (layers == nullptr || n_layers < 1 || sg == nullptr) return SLIM_ERR_INVALID_ARG;
+    memset(sg, 0, sizeof *sg);
+    sg->ws_bytes = 256;
+    for (int l = 0; l < n_layers; ++l) {
+        const slim_layer& L = layers[l];
+        if (L.M < 1 || L.M > SLIM_GEMV_MAX_M) return SLIM_ERR_INVALID_ARG;
+        GroupTable gt;
+        const int st = make_group_table(L.N, L.K, g, L.bits_host, &gt);
+        if (st != SLIM_OK) return st;
+        if (L.N == 0 || L.K == 0) return SLIM_ERR_INVALID_ARG;
+        for (int j = 0; j < gt.G; ++j) sg->bmax = sg->bmax > gt.bits[j] ? sg->bmax : gt.bits[j];
+        sg->mmax = sg->mmax > L.M ? sg->mmax : L.M;
+        const int items = (L.N + kSetRowsPerItem - 1) / kSetRowsPerItem;
+        sg->n_items += items;
+        sg->n_tasks += static_cast<long long>(L.M) * gt.G;
+        for (int rb = 0; rb < items; ++rb) {
+            const int th = (L.N >> 4) - kSetConsumers * rb;
+            sg->total_cost += item_cost(th < kSetConsumers ? th : kSetConsumers, gt);
+        }
+        sg->ws_bytes += layer_ws_bytes(L.M, gt);
+    }
+    if (sg->n_items > 0x3fffffff || sg->n_tasks > 0x3fffffff) return SLIM_ERR_UNSUPPORTED;
+    sg->nt = sg->mmax <= 8 ? 1 : 2;
+    sg->off_s = kSetHeader + kSetConsumers * 256 * sg->bmax;
+    sg->off_z = sg->off_s + kSetConsumers * 32;
+    sg->off_e = sg->off_z + kSetConsumers * 32;
+    sg->off_x = sg->off_e + 128;
+    // a 3-bit group brings the fragments of two slices (a set whose widest group has 4 bits may hold one)
+    sg->slot_bytes = static_cast<int>(align_to(static_cast<size_t>(sg->off_x) + (sg->bmax >= 3 ? 2 : 1) * 256 * sg->mmax, 128));
+    // two CTAs per SM when each still gets at least 8 slots, else one
+    const size_t per_sm = 224 * 1024;
+    sg->ctas_per_sm = 2;
+    size_t budget = per_sm / 2 - 1024 - kSetOffRing;          // 1 KB per CTA is reserved by the system
+    if (budget / sg->slot_bytes < 8) { sg->ctas_per_sm = 1; budget = per_sm - 1024 - kSetOffRing; }
+    size_t slots = budget / sg->slot_bytes;
+    if (slots > kSetMaxSlots) slots = kSetMaxSlots;
+    if (slots < 2) return SLIM_ERR_UNSUPPORTED;
+    sg->n_slots = static_cast<int>(slots);
+    sg->smem_bytes = kSetOffRing + slots * sg->slot_bytes;
+    long long grid = static_cast<long long>(set_sm_count()) * sg->ctas_per_sm;
+    if (grid > kSetMaxGrid) grid = kSetMaxGrid;
+    if (grid > sg->n_items) grid = sg->n_items;
+    sg->grid = static_cast<int>(grid);
+    return SLIM_OK;
+}
+
+static size_t set_plan_bytes(int n_layers) { return kSetPlanHeader + static_cast<size_t>(n_layers) * sizeof(SetLayer); }
+
+template <int NT>
+static cudaError_t launch_set(const SetParams& prm, int grid, size_t smem, cudaStream_t stream) {
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        e = cudaFuncSetAttribute(gemv_set_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    gemv_set_kernel<NT><<<grid, kSetThreads, smem, stream>>>(prm);
+    return cudaGetLastError();
+}
+
+}  // namespace slim
+
+extern "C" {
+
+int slim_gemv_set_bytes(const slim_layer* layers_host, int n_layers, int g, size_t* plan_bytes, size_t* workspace_bytes) {
+    if (plan_bytes == nullptr || workspace_bytes == nullptr) return SLIM_ERR_INVALID_ARG;
+    slim::SetGeometry sg;
+    const int st = slim::set_geometry(layers_host, n_layers, g, &sg);
+    if (st != SLIM_OK) return st;
+    *plan_bytes = slim::set_plan_bytes(n_layers);
+    *workspace_bytes = sg.ws_bytes;
+    return SLIM_OK;
+}
+
+int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void* plan, size_t plan_bytes,
+                       slim_gemv_set_info* info, void* stream) {
+    if (info == nullptr || plan == nullptr) return SLIM_ERR_INVALID_ARG;
+    slim::SetGeometry sg;
+    const int st = slim::set_geometry(layers_host, n_layers, g, &sg);
+    if (st != SLIM_OK) return st;
+    if (!slim::aligned16(plan)) return SLIM_ERR_ALIGNMENT;
+    if (plan_bytes < slim::set_plan_bytes(n_layers)) return SLIM_ERR_WORKSPACE;
+    for (int l = 0; l < n_layers; ++l) {
+        const slim_layer& L = layers_host[l];
+        if (L.x == nullptr || L.packed == nullptr || L.scales == nullptr || L.zeros == nullptr || L.y == nullptr)
+            return SLIM_ERR_INVALID_ARG;
+        if (!slim::aligned16(L.x) || !slim::aligned16(L.packed) || !slim::aligned16(L.scales) || !slim::aligned16(L.zeros) ||
+            !slim::aligned16(L.y))
+            return SLIM_ERR_ALIGNMENT;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* plan_dev = static_cast<uint8_t*>(plan);
+
+    // Second pass: descriptors, and the first item of every CTA (equal shares of the set's bytes).
+    // The copies below read host memory that goes out of scope: pageable sources are staged
+    // before cudaMemcpyAsync returns.
+    static_assert((slim::kSetMaxGrid + 1) * sizeof(int) <= slim::kSetPlanHeader, "item ranges fit the plan header");
+    int item_begin[slim::kSetMaxGrid + 1];
+    int next_cta = 1;
+    item_begin[0] = 0;
+    unsigned long long cost = 0;
+    int item = 0, task = 0;
+    size_t ws_off = 256;
+    for (int l = 0; l < n_layers; ++l) {
+        const slim_layer& L = layers_host[l];
+        slim::GroupTable gt;
+        slim::make_group_table(L.N, L.K, g, L.bits_host, &gt);
+        slim::SetLayer d;
+        memset(&d, 0, sizeof d);
+        d.x = static_cast<const __half*>(L.x);
+        d.packed = static_cast<const uint8_t*>(L.packed);
+        d.scales = static_cast<const __half*>(L.scales);
+        d.zeros = static_cast<const __half*>(L.zeros);
+        d.y = static_cast<__half*>(L.y);
+        d.M = L.M; d.N = L.N; d.K = L.K; d.G = gt.G;
+        d.item0 = item;
+        d.n_items = (L.N + slim::kSetRowsPerItem - 1) / slim::kSetRowsPerItem;
+        d.task0 = task;
+        d.x_off = ws_off;
+        ws_off += slim::layer_ws_bytes(L.M, gt);
+        memcpy(d.prefix, gt.prefix, sizeof d.prefix);
+        memcpy(d.bits, gt.bits, sizeof d.bits);
+        d.pre3[0] = 0;
+        for (int j = 0; j < SLIM_MAX_GROUPS; ++j)
+            d.pre3[j + 1] = static_cast<uint16_t>(d.pre3[j] + (j < gt.G && gt.bits[j] == 3 ? 1 : 0));
+        SLIM_CUDA_TRY(cudaMemcpyAsync(plan_dev + slim::kSetPlanHeader + static_cast<size_t>(l) * sizeof d, &d, sizeof d,
+                                      cudaMemcpyHostToDevice, s));
+        for (int rb = 0; rb < d.n_items; ++rb, ++item) {
+            // CTA c starts at the first item at which the bytes before it reach c/grid of the total
+            while (next_cta < sg.grid && cost * sg.grid >= sg.total_cost * static_cast<unsigned long long>(next_cta))
+                item_begin[next_cta++] = item;
+            const int th = (L.N >> 4) - slim::kSetConsumers * rb;
+            cost += slim::item_cost(th < slim::kSetConsumers ? th : slim::kSetConsumers, gt);
+        }
+        task += L.M * gt.G;
+    }
+    while (next_cta <= sg.grid) item_begin[next_cta++] = item;
+    SLIM_CUDA_TRY(cudaMemcpyAsync(plan_dev, item_begin, static_cast<size_t>(sg.grid + 1) * sizeof(int), cudaMemcpyHostToDevice, s));
+
+    memset(info, 0, sizeof *info);
+    info->n_layers = n_layers;
+    info->grid = sg.grid;
+    info->n_slots = sg.n_slots;
+    info->slot_bytes = sg.slot_bytes;
+    info->token_tiles = sg.nt;
+    info->stage_tasks = task;
+    info->n_items = item;
+    info->max_bits = sg.bmax;
+    info->plan_bytes = slim::set_plan_bytes(n_layers);
+    info->workspace_bytes = sg.ws_bytes;
+    return SLIM_OK;
+}
+
+
+int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* workspace, size_t workspace_bytes, void* stream) {
+    if (info == nullptr || plan == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (info->n_layers < 1 || info->grid < 1 || info->grid > slim::kSetMaxGrid || info->n_slots < 2 ||
+        info->n_slots > slim::kSetMaxSlots || info->slot_bytes < 128 || info->slot_bytes % 128 != 0 ||
+        (info->token_tiles != 1 && info->token_tiles != 2) || info->max_bits < 1 || info->max_bits > 4 || info->stage_tasks < 1)
+        return SLIM_ERR_INVALID_ARG;
+    const size_t smem = slim::kSetOffRing + static_cast<size_t>(info->n_slots) * info->slot_bytes;
+    if (smem > 224 * 1024) return SLIM_ERR_INVALID_ARG;
+    if (!slim::aligned16(plan)) return SLIM_ERR_ALIGNMENT;
+    if (workspace == nullptr || workspace_bytes < info->workspace_bytes || workspace_bytes < 256) return SLIM_ERR_WORKSPACE;
+    if (!slim::aligned16(workspace)) return SLIM_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    slim::SetParams prm;
+    memset(&prm, 0, sizeof prm);
+    prm.item_begin = static_cast<const int*>(plan);
+    prm.layers = reinterpret_cast<const slim::SetLayer*>(static_cast<const uint8_t*>(plan) + slim::kSetPlanHeader);
+    prm.ws = static_cast<uint8_t*>(workspace);
+    prm.n_layers = info->n_layers;
+    prm.n_slots = info->n_slots;
+    prm.slot_bytes = info->slot_bytes;
+    prm.off_s = slim::kSetHeader + slim::kSetConsumers * 256 * info->max_bits;
+    prm.off_z = prm.off_s + slim::kSetConsumers * 32;
+    prm.off_e = prm.off_z + slim::kSetConsumers * 32;
+    prm.off_x = prm.off_e + 128;
+    if (prm.off_x + (info->max_bits >= 3 ? 2 : 1) * 256 * (info->token_tiles == 1 ? 1 : 9) > info->slot_bytes) return SLIM_ERR_INVALID_ARG;
+
+    slim::gemv_set_stage_kernel<<<(info->stage_tasks + 7) / 8, 256, 0, s>>>(prm.layers, prm.ws, info->n_layers, info->stage_tasks);
+    SLIM_CUDA_TRY(cudaGetLastError());
+    const cudaError_t e = info->token_tiles == 1 ? slim::launch_set<1>(prm, info->grid, smem, s) : slim::launch_set<2>(prm, info->grid, smem, s);
+    SLIM_CUDA_TRY(e);
+    return SLIM_OK;
+}
+
+}  // extern "C"

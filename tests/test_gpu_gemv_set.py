@@ -1,0 +1,132 @@
+"""GPU parity: the layer-set launch of the decode path (slim_gemv_set_plan / slim_mpq_gemv_set)
+against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import slim_oracle as orc
+from tests.helpers import check_output, oracle_layer
+
+pytestmark = pytest.mark.gpu
+
+
+def _slim():
+    from paper_2405_14917_b200 import binding
+    return binding
+
+
+def _device_layer(L):
+    slim = _slim()
+    packed = torch.from_numpy(orc.pack(L["codes"], L["bits"])).cuda()
+    return slim.QuantLinear(packed, L["bits"], torch.from_numpy(L["scales"]).cuda(), torch.from_numpy(L["zeros"]).cuda(), L["N"], L["K"])
+
+
+def _run_set(layers):
+    """layers: oracle dicts.  Returns the list of y (numpy) the set launch produced."""
+    slim = _slim()
+    entries = []
+    for L in layers:
+        x = torch.from_numpy(L["x"]).cuda()
+        y = torch.full((L["M"], L["N"]), float("nan"), dtype=torch.float16, device="cuda")
+        entries.append((_device_layer(L), x, y))
+    s = slim.LayerSet(entries)
+    s.run()
+    s.check()
+    return [y.cpu().numpy() for (_, _, y) in entries], s
+
+
+def _check_all(layers, ys, what):
+    for k, (L, y) in enumerate(zip(layers, ys)):
+        y_ref = orc.linear_f64(L["x"], L["codes"], L["scales"], L["zeros"])
+        check_output(y, y_ref, f"{what}: layer {k} ({L['N']}x{L['K']} M={L['M']})")
+
+
+def test_mixed_shapes_one_token():
+    # several tiles, a ragged last row block (272 = 2 * 128 + 16), one to eleven groups
+    layers = [oracle_layer(512, 1024, 2, 1, block=0), oracle_layer(272, 1408, 3, 1, block=1),
+              oracle_layer(128, 128, 2, 1, block=2), oracle_layer(16, 256, 3, 1, block=3),
+              oracle_layer(1040, 512, 2, 1, block=4)]
+    ys, s = _run_set(layers)
+    _check_all(layers, ys, "one token")
+    assert s.info["n_items"] == 4 + 3 + 1 + 1 + 9
+
+
+@pytest.mark.parametrize("Ms", [(1, 2, 3), (4, 8, 5), (16, 9, 1), (16, 16, 16)])
+def test_mixed_token_counts(Ms):
+    layers = [oracle_layer(384, 768, 2, Ms[0], block=0), oracle_layer(144, 1280, 3, Ms[1], block=1),
+              oracle_layer(256, 256, 2, Ms[2], block=2)]
+    ys, _ = _run_set(layers)
+    _check_all(layers, ys, f"Ms={Ms}")
+
+
+@pytest.mark.parametrize("bits", [[1] * 8, [2] * 8, [3] * 8, [4] * 8, [1, 4, 2, 3, 3, 1, 4, 2], [3], [2, 1]])
+def test_adversarial_bit_maps(bits):
+    layers = [oracle_layer(144, 128 * len(bits), 2, M, bits=bits, block=M) for M in (1, 4)]
+    ys, _ = _run_set(layers)
+    _check_all(layers, ys, f"bits={bits}")
+
+
+def test_many_layers_more_items_than_ctas_and_repeatable():
+    # 60 layers x 9 row blocks = 540 items: every CTA of a 148-SM device walks across layer boundaries
+    layers = [oracle_layer(1136, 384, 2 + (k & 1), 1, block=k) for k in range(60)]
+    ys, s = _run_set(layers)
+    _check_all(layers, ys, "many layers")
+    assert s.info["n_items"] == 60 * 9
+    ys2, _ = _run_set(layers)
+    for a, b in zip(ys, ys2):
+        assert (a.view(np.uint16) == b.view(np.uint16)).all(), "two runs of the same set differ"
+
+
+def test_one_hot_x_returns_dequantised_columns():
+    L = oracle_layer(256, 1024, 2, 1)
+    What = orc.dequant_f64(L["codes"], L["scales"], L["zeros"])
+    layers = []
+    cols = (0, 1, 31, 32, 127, 128, 500, 1023)
+    for k in cols:
+        Lk = dict(L)
+        x = np.zeros((1, 1024), dtype=np.float16)
+        x[0, k] = 1.0
+        Lk["x"] = x
+        layers.append(Lk)
+    ys, _ = _run_set(layers)
+    for k, y in zip(cols, ys):
+        want = What[:, k].astype(np.float16)   # exact column, rounded once to fp16
+        assert (y[0].view(np.uint16) == want.view(np.uint16)).all(), f"column {k}"
+
+
+def test_half_integer_zero_points_and_zero_x():
+    L = oracle_layer(128, 512, 3, 2)
+    Lh = dict(L)
+    Lh["zeros"] = (L["zeros"].astype(np.float32) + 0.5).astype(np.float16)
+    L0 = dict(L)
+    L0["x"] = np.zeros((2, 512), np.float16)
+    ys, _ = _run_set([Lh, L0])
+    check_output(ys[0], orc.linear_f64(Lh["x"], Lh["codes"], Lh["scales"], Lh["zeros"]), "half-integer zeros")
+    assert (ys[1] == 0).all()
+
+
+def test_agrees_with_the_single_layer_entry_point():
+    slim = _slim()
+    L = oracle_layer(4096, 4096, 2, 1, seed_name="set-vs-single")
+    ys, _ = _run_set([L])
+    dl = _device_layer(L)
+    ws = slim.new_workspace(1, L["N"], L["K"], L["bits"])
+    y1 = slim.mpq_gemv(torch.from_numpy(L["x"]).cuda(), dl.packed, L["bits"], dl.scales, dl.zeros, L["N"], ws).cpu().numpy()
+    y_ref = orc.linear_f64(L["x"], L["codes"], L["scales"], L["zeros"])
+    check_output(ys[0], y_ref, "set launch, 4096x4096")
+    # two summation orders of the same products: both within the oracle's tolerance of each other
+    assert np.abs(ys[0].astype(np.float64) - y1.astype(np.float64)).max() <= 5e-3 * np.abs(y_ref).max()
+
+
+def test_rejects_bad_sets():
+    slim = _slim()
+    L = oracle_layer(128, 256, 2, 1)
+    dl = _device_layer(L)
+    x = torch.from_numpy(L["x"]).cuda()
+    with pytest.raises(ValueError):
+        slim.LayerSet([])
+    with pytest.raises(ValueError):
+        slim.LayerSet([(dl, x, torch.empty(1, 64, dtype=torch.float16, device="cuda"))])
+    x17 = torch.zeros(17, 256, dtype=torch.float16, device="cuda")
+    with pytest.raises(slim.SlimError):
+        slim.LayerSet([(dl, x17, torch.empty(17, 128, dtype=torch.float16, device="cuda"))])

@@ -104,3 +104,36 @@ def test_gemv_plan_invariants(slim):
         assert pl["smem_bytes"] <= 227 * 1024
         assert pl["n_tiles"] == (1 if M <= 8 else 2)
         assert 1 <= pl["groups_per_chunk"] <= G
+
+
+def _set_bytes(slim, shapes, g=128):
+    """shapes: list of (M, N, K, bits).  Returns (status, plan_bytes, workspace_bytes)."""
+    arr = (slim._Layer * max(len(shapes), 1))()
+    keep = []
+    for k, (M, N, K, bits) in enumerate(shapes):
+        b = np.asarray(bits, dtype=np.uint8)
+        keep.append(b)
+        arr[k] = slim._Layer(0, 0, 0, 0, 0, b.ctypes.data, M, N, K)
+    pb, wb = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    st = slim.lib().slim_gemv_set_bytes(ctypes.cast(arr, ctypes.c_void_p), len(shapes), g, ctypes.byref(pb), ctypes.byref(wb))
+    return st, pb.value, wb.value
+
+
+def test_layer_set_sizes_and_argument_errors(slim):
+    ok = [(1, 256, 512, [2, 3, 1, 2]), (4, 144, 256, [3, 3])]
+    st, pb, wb = _set_bytes(slim, ok)
+    assert st == 0
+    # plan: item ranges of the CTAs, then one descriptor per layer; it grows by a fixed step per layer
+    st2, pb2, _ = _set_bytes(slim, ok + [(1, 128, 128, [2])])
+    assert st2 == 0 and pb2 > pb and (pb2 - pb) % 16 == 0
+    # workspace: status header + per layer the sums [G][16] float2 and the fragments of every slice
+    want = 256 + (4 * 128 + (4 + 1) * 8 * 1 * 32) + (2 * 128 + (2 + 2) * 8 * 4 * 32)
+    assert wb == want
+    assert _set_bytes(slim, [])[0] == -1                                  # empty set
+    assert _set_bytes(slim, [(0, 256, 512, [2] * 4)])[0] == -1            # no token
+    assert _set_bytes(slim, [(17, 256, 512, [2] * 4)])[0] == -1           # the batched path serves these
+    assert _set_bytes(slim, [(1, 256, 512, [2, 5, 2, 2])])[0] == -1       # bit-width out of range
+    assert _set_bytes(slim, [(1, 250, 512, [2] * 4)])[0] == -2            # N not a multiple of 16
+    assert _set_bytes(slim, [(1, 256, 500, [2] * 4)])[0] == -2            # K not a multiple of 128
+    assert _set_bytes(slim, [(1, 256, 0, [])])[0] == -1                   # empty reduction
+    assert _set_bytes(slim, ok, g=64)[0] == -2                            # group size
