@@ -187,6 +187,8 @@ typedef struct slim_gemv_set_info {
     int stage_tasks;       /* (layer, token, group) triples of the set */
     int n_items;           /* 128-row blocks of the set */
     int max_bits;          /* widest group of the set */
+    int max_tokens;        /* largest M of the set */
+    int reserved;
     size_t plan_bytes;
     size_t workspace_bytes;
 } slim_gemv_set_info;

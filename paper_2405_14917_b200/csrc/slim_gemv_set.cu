@@ -31,6 +31,7 @@ constexpr int kSetProducers = 2;                       // producer warps: they t
 constexpr int kSetThreads = 32 * (kSetConsumers + kSetProducers);
 constexpr int kSetRowsPerItem = 16 * kSetConsumers;
 constexpr int kSetMaxSlots = 32;
+constexpr int kSetCtasPerSm = 2;                       // resident CTAs per SM the plan aims at
 constexpr int kSetHeader = 16;                         // slot header: bit-width of the group
 constexpr unsigned long long kSetWaitNs = 2000000000ull;
 
@@ -133,12 +134,22 @@ __global__ void __launch_bounds__(256) gemv_set_stage_kernel(const SetLayer* __r
     if (m == 0 && lane < 16 && lane >= L.M) sxe[lane] = make_float2(0.f, 1.f);   // absent tokens read 0
 }
 
+// D = A * B with a zero accumulator input: starts an accumulation chain without clearing registers first.
+__device__ __forceinline__ void mma_f16_first(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint2 b) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b.x), "r"(b.y), "f"(0.f));
+}
+
 // ------------------------------------------------------------------------------------------ the persistent kernel
 constexpr uint32_t kSetOffAbort = 16 * kSetMaxSlots;          // after the full and empty barriers
 constexpr uint32_t kSetOffDesc = 1024;                        // the producer's copy of its layer's descriptor
 constexpr uint32_t kSetOffRing = (kSetOffDesc + kSetProducers * sizeof(SetLayer) + 127) / 128 * 128;
 
-template <int NT>   // 8-token MMA tiles: 1 (every M <= 8) or 2
+// NT: 8-token MMA tiles, 1 (every M <= 8) or 2.  ONE: every layer has a single token; then only
+// column 0 of the MMA results is ever used, so every lane feeds token 0's fragment and folds token 0.
+template <int NT, bool ONE>
 __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_constant__ SetParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
@@ -251,18 +262,13 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                         const uint32_t item = slot + kSetHeader + static_cast<uint32_t>(warp) * 256u * b;
                         const uint32_t xs_slot0 = slot + p.off_x;
                         constexpr int CH = NT == 1 ? 4 : 2;      // interleaved accumulation chains
-                        float d[CH][NT][4];
-#pragma unroll
-                        for (int h = 0; h < CH; ++h)
-#pragma unroll
-                            for (int n = 0; n < NT; ++n)
-#pragma unroll
-                                for (int r = 0; r < 4; ++r) d[h][n][r] = 0.f;
+                        float d[CH][NT][4];      // every chain is started by an MMA with a zero accumulator
 
                         // one slice of width WD starting at unit `unit0`, activations in fragment slot `xs_slot`
-                        auto run_slice = [&](auto wtag, int unit0, uint32_t xs_slot) {
+                        auto run_slice = [&](auto wtag, auto first_tag, int unit0, uint32_t xs_slot) {
                             constexpr int WD = decltype(wtag)::value;
                             constexpr int MPU = 8 / WD;                 // MMAs per unit
+                            constexpr bool FIRST = decltype(first_tag)::value != 0;   // the group's first slice
 #pragma unroll
                             for (int u = 0; u < WD; ++u) {
                                 const uint2 wd = lds64(item + 256 * (unit0 + u) + 8 * lane);
@@ -276,17 +282,19 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                                     for (int n = 0; n < NT; ++n) {
                                         const int m = 8 * n + gq;
                                         uint2 bv = make_uint2(0u, 0u);
-                                        if (m < M) bv = lds64(xs_slot + ((mi * M + m) * 4 + c) * 8);
-                                        mma_f16(d[(u * MPU + ii) & (CH - 1)][n], a0, a1, a2, a3, bv);
+                                        if (ONE) bv = lds64(xs_slot + (mi * 4 + c) * 8);
+                                        else if (m < M) bv = lds64(xs_slot + ((mi * M + m) * 4 + c) * 8);
+                                        if (FIRST && mi < CH) mma_f16_first(d[mi & (CH - 1)][n], a0, a1, a2, a3, bv);
+                                        else mma_f16(d[mi & (CH - 1)][n], a0, a1, a2, a3, bv);
                                     }
                                 }
                             }
                         };
                         switch (b) {
-                            case 1: run_slice(W1{}, 0, xs_slot0); break;
-                            case 2: run_slice(W2{}, 0, xs_slot0); break;
-                            case 3: run_slice(W2{}, 0, xs_slot0); run_slice(W1{}, 2, xs_slot0 + 8 * M * 32); break;
-                            default: run_slice(W4{}, 0, xs_slot0); break;
+                            case 1: run_slice(W1{}, WidthTag<1>{}, 0, xs_slot0); break;
+                            case 2: run_slice(W2{}, WidthTag<1>{}, 0, xs_slot0); break;
+                            case 3: run_slice(W2{}, WidthTag<1>{}, 0, xs_slot0); run_slice(W1{}, WidthTag<0>{}, 2, xs_slot0 + 8 * M * 32); break;
+                            default: run_slice(W4{}, WidthTag<1>{}, 0, xs_slot0); break;
                         }
 
                         // fold the group: acc += s * (D * 2^(24-S) - z * sum_x); rows 2gq, 2gq+1, tokens 8n+2c, 8n+2c+1
@@ -295,6 +303,13 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                         const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
                         const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
                         const float2* sxe = reinterpret_cast<const float2*>(smem + (slot - sbase) + p.off_e);
+                        if (ONE) {
+                            const float2 t = sxe[0];                                       // (sum_k x, 2^(24-S)) of token 0
+                            const float e0 = (d[0][0][0] + d[1][0][0]) + (d[2 % CH][0][0] + d[3 % CH][0][0]);
+                            const float e2 = (d[0][0][2] + d[1][0][2]) + (d[2 % CH][0][2] + d[3 % CH][0][2]);
+                            acc[0][0] = fmaf(sf.x, fmaf(-zf.x, t.x, e0 * t.y), acc[0][0]);
+                            acc[0][2] = fmaf(sf.y, fmaf(-zf.y, t.x, e2 * t.y), acc[0][2]);
+                        } else
 #pragma unroll
                         for (int n = 0; n < NT; ++n) {
                             const float4 t = *reinterpret_cast<const float4*>(sxe + 8 * n + 2 * c);   // (sx0, e0, sx1, e1)
@@ -318,6 +333,9 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                 // ---- this warp's 16 rows of the item: rows 2gq, 2gq+1 of tokens 8n+2c, 8n+2c+1
                 if (active && ok) {
                     __half* yrow = L.y + 16 * tile + 2 * gq;
+                    if (ONE) {
+                        if (c == 0) *reinterpret_cast<__half2*>(yrow) = __floats2half2_rn(acc[0][0], acc[0][2]);
+                    } else
 #pragma unroll
                     for (int n = 0; n < NT; ++n) {
                         const int m0 = 8 * n + 2 * c;
@@ -393,11 +411,13 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     sg->off_x = sg->off_e + 128;
     // a 3-bit group brings the fragments of two slices (a set whose widest group has 4 bits may hold one)
     sg->slot_bytes = static_cast<int>(align_to(static_cast<size_t>(sg->off_x) + (sg->bmax >= 3 ? 2 : 1) * 256 * sg->mmax, 128));
-    // two CTAs per SM when each still gets at least 8 slots, else one
+    // as many CTAs per SM (kSetCtasPerSm at most) as still leaves each a ring of 8 slots
     const size_t per_sm = 224 * 1024;
-    sg->ctas_per_sm = 2;
-    size_t budget = per_sm / 2 - 1024 - kSetOffRing;          // 1 KB per CTA is reserved by the system
-    if (budget / sg->slot_bytes < 8) { sg->ctas_per_sm = 1; budget = per_sm - 1024 - kSetOffRing; }
+    size_t budget = 0;
+    for (sg->ctas_per_sm = kSetCtasPerSm; sg->ctas_per_sm >= 1; --sg->ctas_per_sm) {
+        budget = per_sm / sg->ctas_per_sm - 1024 - kSetOffRing;   // 1 KB per CTA is reserved by the system
+        if (budget / sg->slot_bytes >= 8 || sg->ctas_per_sm == 1) break;
+    }
     size_t slots = budget / sg->slot_bytes;
     if (slots > kSetMaxSlots) slots = kSetMaxSlots;
     if (slots < 2) return SLIM_ERR_UNSUPPORTED;
@@ -412,18 +432,18 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
 
 static size_t set_plan_bytes(int n_layers) { return kSetPlanHeader + static_cast<size_t>(n_layers) * sizeof(SetLayer); }
 
-template <int NT>
+template <int NT, bool ONE>
 static cudaError_t launch_set(const SetParams& prm, int grid, size_t smem, cudaStream_t stream) {
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        e = cudaFuncSetAttribute(gemv_set_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        e = cudaFuncSetAttribute(gemv_set_kernel<NT, ONE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    gemv_set_kernel<NT><<<grid, kSetThreads, smem, stream>>>(prm);
+    gemv_set_kernel<NT, ONE><<<grid, kSetThreads, smem, stream>>>(prm);
     return cudaGetLastError();
 }
 
@@ -515,6 +535,7 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
     info->stage_tasks = task;
     info->n_items = item;
     info->max_bits = sg.bmax;
+    info->max_tokens = sg.mmax;
     info->plan_bytes = slim::set_plan_bytes(n_layers);
     info->workspace_bytes = sg.ws_bytes;
     return SLIM_OK;
@@ -525,7 +546,8 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     if (info == nullptr || plan == nullptr) return SLIM_ERR_INVALID_ARG;
     if (info->n_layers < 1 || info->grid < 1 || info->grid > slim::kSetMaxGrid || info->n_slots < 2 ||
         info->n_slots > slim::kSetMaxSlots || info->slot_bytes < 128 || info->slot_bytes % 128 != 0 ||
-        (info->token_tiles != 1 && info->token_tiles != 2) || info->max_bits < 1 || info->max_bits > 4 || info->stage_tasks < 1)
+        (info->token_tiles != 1 && info->token_tiles != 2) || info->max_tokens < 1 || info->max_tokens > 8 * info->token_tiles ||
+        info->max_bits < 1 || info->max_bits > 4 || info->stage_tasks < 1)
         return SLIM_ERR_INVALID_ARG;
     const size_t smem = slim::kSetOffRing + static_cast<size_t>(info->n_slots) * info->slot_bytes;
     if (smem > 224 * 1024) return SLIM_ERR_INVALID_ARG;
@@ -546,11 +568,13 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     prm.off_z = prm.off_s + slim::kSetConsumers * 32;
     prm.off_e = prm.off_z + slim::kSetConsumers * 32;
     prm.off_x = prm.off_e + 128;
-    if (prm.off_x + (info->max_bits >= 3 ? 2 : 1) * 256 * (info->token_tiles == 1 ? 1 : 9) > info->slot_bytes) return SLIM_ERR_INVALID_ARG;
+    if (prm.off_x + (info->max_bits >= 3 ? 2 : 1) * 256 * info->max_tokens > info->slot_bytes) return SLIM_ERR_INVALID_ARG;
 
     slim::gemv_set_stage_kernel<<<(info->stage_tasks + 7) / 8, 256, 0, s>>>(prm.layers, prm.ws, info->n_layers, info->stage_tasks);
     SLIM_CUDA_TRY(cudaGetLastError());
-    const cudaError_t e = info->token_tiles == 1 ? slim::launch_set<1>(prm, info->grid, smem, s) : slim::launch_set<2>(prm, info->grid, smem, s);
+    const cudaError_t e = info->max_tokens == 1 ? slim::launch_set<1, true>(prm, info->grid, smem, s)
+                        : info->token_tiles == 1 ? slim::launch_set<1, false>(prm, info->grid, smem, s)
+                                                 : slim::launch_set<2, false>(prm, info->grid, smem, s);
     SLIM_CUDA_TRY(e);
     return SLIM_OK;
 }
