@@ -185,10 +185,10 @@ typedef struct slim_gemv_set_info {
     int slot_bytes;
     int token_tiles;       /* 8-token MMA tiles: 1 or 2 */
     int stage_tasks;       /* (layer, token, group) triples of the set */
-    int n_items;           /* 128-row blocks of the set */
+    int n_items;           /* row blocks (work items) of the set */
     int max_bits;          /* widest group of the set */
     int max_tokens;        /* largest M of the set */
-    int reserved;
+    int tiles_per_warp;    /* 16-row tiles a consumer warp owns: an item is 128 rows times this */
     size_t plan_bytes;
     size_t workspace_bytes;
 } slim_gemv_set_info;

@@ -26,10 +26,9 @@
 
 namespace slim {
 
-constexpr int kSetConsumers = 8;                       // consumer warps = tiles of an item
+constexpr int kSetConsumers = 8;                       // consumer warps; each owns TPW (1 or 2) tiles of an item
 constexpr int kSetProducers = 2;                       // producer warps: they take the groups in turn
 constexpr int kSetThreads = 32 * (kSetConsumers + kSetProducers);
-constexpr int kSetRowsPerItem = 16 * kSetConsumers;
 constexpr int kSetMaxSlots = 32;
 constexpr int kSetCtasPerSm = 2;                       // resident CTAs per SM the plan aims at
 constexpr int kSetHeader = 16;                         // slot header: bit-width of the group
@@ -149,7 +148,9 @@ constexpr uint32_t kSetOffRing = (kSetOffDesc + kSetProducers * sizeof(SetLayer)
 
 // NT: 8-token MMA tiles, 1 (every M <= 8) or 2.  ONE: every layer has a single token; then only
 // column 0 of the MMA results is ever used, so every lane feeds token 0's fragment and folds token 0.
-template <int NT, bool ONE>
+// TPW: 16-row tiles per consumer warp (an item is 8 * TPW tiles); two tiles share the fragment loads and
+// the per-group bookkeeping.
+template <int NT, bool ONE, int TPW>
 __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_constant__ SetParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
@@ -158,6 +159,7 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
     auto empty = [&](int s) { return sbase + 8u * (kSetMaxSlots + s); };
     volatile int* abort = reinterpret_cast<volatile int*>(smem + kSetOffAbort);
     const uint32_t ring = sbase + kSetOffRing;
+    constexpr int TPI = kSetConsumers * TPW;                  // tiles per item
 
     if (tid == 0) {
         for (int s = 0; s < p.n_slots; ++s) { sb::init(full(s), 1); sb::init(empty(s), kSetConsumers); }
@@ -200,11 +202,11 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                     have = l;
                 }
                 const int rb = i - D->item0, N = D->N, M = D->M, G = D->G;
-                const int tiles_here = min(kSetConsumers, (N >> 4) - kSetConsumers * rb);
+                const int tiles_here = min(TPI, (N >> 4) - TPI * rb);
                 // lane 0 brings the slices, lanes 1 and 2 scales and zeros, lane 3 the staged activations
                 const uint8_t* base = lane == 0 ? D->packed
-                                    : lane == 1 ? reinterpret_cast<const uint8_t*>(D->scales + kSetRowsPerItem * rb)
-                                    : lane == 2 ? reinterpret_cast<const uint8_t*>(D->zeros + kSetRowsPerItem * rb)
+                                    : lane == 1 ? reinterpret_cast<const uint8_t*>(D->scales + 16 * TPI * rb)
+                                    : lane == 2 ? reinterpret_cast<const uint8_t*>(D->zeros + 16 * TPI * rb)
                                                 : p.ws + D->x_off;
                 const uint32_t dst_off = lane == 0 ? kSetHeader : lane == 1 ? p.off_s : lane == 2 ? p.off_z : p.off_e;
                 const uint32_t szb = static_cast<uint32_t>(tiles_here) * 32u;
@@ -221,7 +223,7 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                         asm volatile("st.shared.u32 [%0], %1;" ::"r"(slot), "r"(b) : "memory");
                         sb::expect_tx(full(s), wbytes + 2 * szb + xbytes);
                     }
-                    const size_t off = lane == 0 ? 16ull * N * D->prefix[j] + static_cast<size_t>(kSetConsumers * rb) * 256 * b
+                    const size_t off = lane == 0 ? 16ull * N * D->prefix[j] + static_cast<size_t>(TPI * rb) * 256 * b
                                      : lane == 3 ? staged_group_offset(j, D->pre3[j], M)
                                                  : 2ull * static_cast<size_t>(j) * N;
                     const uint32_t bytes = lane == 0 ? wbytes : lane == 3 ? xbytes : szb;
@@ -246,23 +248,27 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                 while (i >= p.layers[l].item0 + p.layers[l].n_items) ++l;
                 const SetLayer& L = p.layers[l];
                 const int rb = i - L.item0, N = L.N, M = L.M, G = L.G;
-                const int tile = kSetConsumers * rb + warp;
-                const bool active = tile < (N >> 4);
-                float acc[NT][4];
+                const int tile0 = TPI * rb + TPW * warp;                  // this warp's first tile of the layer
+                const int n_act = min(TPW, (N >> 4) - tile0);              // its tiles that exist (<= 0: none)
+                float acc[TPW][NT][4];
 #pragma unroll
-                for (int n = 0; n < NT; ++n)
+                for (int t = 0; t < TPW; ++t)
 #pragma unroll
-                    for (int r = 0; r < 4; ++r) acc[n][r] = 0.f;
+                    for (int n = 0; n < NT; ++n)
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) acc[t][n][r] = 0.f;
 
                 for (int j = 0; j < G; ++j) {
                     if (!__all_sync(0xffffffffu, sb::wait(full(s), ph, abort))) { ok = false; break; }
                     const uint32_t slot = ring + static_cast<uint32_t>(s) * p.slot_bytes;
-                    if (active) {
+                    if (n_act > 0) {
                         const int b = static_cast<int>(lds32(slot));
-                        const uint32_t item = slot + kSetHeader + static_cast<uint32_t>(warp) * 256u * b;
+                        // tile t of the warp: its slices follow each other.  For a tile past the end of the
+                        // layer the slot holds stale bytes: its accumulators are computed and never stored.
+                        const uint32_t item0 = slot + kSetHeader + static_cast<uint32_t>(TPW * warp) * 256u * b;
                         const uint32_t xs_slot0 = slot + p.off_x;
-                        constexpr int CH = NT == 1 ? 4 : 2;      // interleaved accumulation chains
-                        float d[CH][NT][4];      // every chain is started by an MMA with a zero accumulator
+                        constexpr int CH = NT == 1 ? (TPW == 1 ? 4 : 2) : 2;     // interleaved accumulation chains
+                        float d[TPW][CH][NT][4];      // every chain is started by an MMA with a zero accumulator
 
                         // one slice of width WD starting at unit `unit0`, activations in fragment slot `xs_slot`
                         auto run_slice = [&](auto wtag, auto first_tag, int unit0, uint32_t xs_slot) {
@@ -271,12 +277,17 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                             constexpr bool FIRST = decltype(first_tag)::value != 0;   // the group's first slice
 #pragma unroll
                             for (int u = 0; u < WD; ++u) {
-                                const uint2 wd = lds64(item + 256 * (unit0 + u) + 8 * lane);
-                                const uint32_t shx = wd.x >> pair_shift(WD), shy = wd.y >> pair_shift(WD);
+                                uint2 wd[TPW];
+                                uint32_t shx[TPW], shy[TPW];
+#pragma unroll
+                                for (int t = 0; t < TPW; ++t) {
+                                    const uint32_t item = item0 + t * 256u * b;
+                                    wd[t] = lds64(item + 256 * (unit0 + u) + 8 * lane);
+                                    shx[t] = wd[t].x >> pair_shift(WD);
+                                    shy[t] = wd[t].y >> pair_shift(WD);
+                                }
 #pragma unroll
                                 for (int ii = 0; ii < MPU; ++ii) {
-                                    const uint32_t a0 = pair<WD>(wd.x, shx, 2 * ii), a1 = pair<WD>(wd.y, shy, 2 * ii);
-                                    const uint32_t a2 = pair<WD>(wd.x, shx, 2 * ii + 1), a3 = pair<WD>(wd.y, shy, 2 * ii + 1);
                                     const int mi = u * MPU + ii;
 #pragma unroll
                                     for (int n = 0; n < NT; ++n) {
@@ -284,8 +295,13 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                                         uint2 bv = make_uint2(0u, 0u);
                                         if (ONE) bv = lds64(xs_slot + (mi * 4 + c) * 8);
                                         else if (m < M) bv = lds64(xs_slot + ((mi * M + m) * 4 + c) * 8);
-                                        if (FIRST && mi < CH) mma_f16_first(d[mi & (CH - 1)][n], a0, a1, a2, a3, bv);
-                                        else mma_f16(d[mi & (CH - 1)][n], a0, a1, a2, a3, bv);
+#pragma unroll
+                                        for (int t = 0; t < TPW; ++t) {
+                                            const uint32_t a0 = pair<WD>(wd[t].x, shx[t], 2 * ii), a1 = pair<WD>(wd[t].y, shy[t], 2 * ii);
+                                            const uint32_t a2 = pair<WD>(wd[t].x, shx[t], 2 * ii + 1), a3 = pair<WD>(wd[t].y, shy[t], 2 * ii + 1);
+                                            if (FIRST && mi < CH) mma_f16_first(d[t][mi & (CH - 1)][n], a0, a1, a2, a3, bv);
+                                            else mma_f16(d[t][mi & (CH - 1)][n], a0, a1, a2, a3, bv);
+                                        }
                                     }
                                 }
                             }
@@ -298,49 +314,62 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                         }
 
                         // fold the group: acc += s * (D * 2^(24-S) - z * sum_x); rows 2gq, 2gq+1, tokens 8n+2c, 8n+2c+1
-                        const uint32_t s2 = lds32(slot + p.off_s + warp * 32 + gq * 4);
-                        const uint32_t z2 = lds32(slot + p.off_z + warp * 32 + gq * 4);
-                        const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
-                        const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
                         const float2* sxe = reinterpret_cast<const float2*>(smem + (slot - sbase) + p.off_e);
-                        if (ONE) {
-                            const float2 t = sxe[0];                                       // (sum_k x, 2^(24-S)) of token 0
-                            const float e0 = (d[0][0][0] + d[1][0][0]) + (d[2 % CH][0][0] + d[3 % CH][0][0]);
-                            const float e2 = (d[0][0][2] + d[1][0][2]) + (d[2 % CH][0][2] + d[3 % CH][0][2]);
-                            acc[0][0] = fmaf(sf.x, fmaf(-zf.x, t.x, e0 * t.y), acc[0][0]);
-                            acc[0][2] = fmaf(sf.y, fmaf(-zf.y, t.x, e2 * t.y), acc[0][2]);
-                        } else
 #pragma unroll
-                        for (int n = 0; n < NT; ++n) {
-                            const float4 t = *reinterpret_cast<const float4*>(sxe + 8 * n + 2 * c);   // (sx0, e0, sx1, e1)
-                            float dd[4];
+                        for (int t = 0; t < TPW; ++t) {
+                            const int tt = TPW * warp + t;                             // tile inside the item
+                            const uint32_t s2 = lds32(slot + p.off_s + tt * 32 + gq * 4);
+                            const uint32_t z2 = lds32(slot + p.off_z + tt * 32 + gq * 4);
+                            const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
+                            const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
+                            if (ONE) {
+                                const float2 tk = sxe[0];                                  // (sum_k x, 2^(24-S)) of token 0
+                                float e0 = d[t][0][0][0] + d[t][1][0][0], e2 = d[t][0][0][2] + d[t][1][0][2];
+                                if (CH == 4) {
+                                    e0 += d[t][2 % CH][0][0] + d[t][3 % CH][0][0];
+                                    e2 += d[t][2 % CH][0][2] + d[t][3 % CH][0][2];
+                                }
+                                acc[t][0][0] = fmaf(sf.x, fmaf(-zf.x, tk.x, e0 * tk.y), acc[t][0][0]);
+                                acc[t][0][2] = fmaf(sf.y, fmaf(-zf.y, tk.x, e2 * tk.y), acc[t][0][2]);
+                            } else {
 #pragma unroll
-                            for (int r = 0; r < 4; ++r) {
-                                dd[r] = d[0][n][r] + d[1][n][r];
-                                if (CH == 4) dd[r] += d[2][n][r] + d[3][n][r];
+                                for (int n = 0; n < NT; ++n) {
+                                    const float4 tk = *reinterpret_cast<const float4*>(sxe + 8 * n + 2 * c);   // (sx0, e0, sx1, e1)
+                                    float dd[4];
+#pragma unroll
+                                    for (int r = 0; r < 4; ++r) {
+                                        dd[r] = d[t][0][n][r] + d[t][1][n][r];
+                                        if (CH == 4) dd[r] += d[t][2 % CH][n][r] + d[t][3 % CH][n][r];
+                                    }
+                                    const float d0 = dd[0] * tk.y, d1 = dd[1] * tk.w, d2 = dd[2] * tk.y, d3 = dd[3] * tk.w;
+                                    acc[t][n][0] = fmaf(sf.x, fmaf(-zf.x, tk.x, d0), acc[t][n][0]);
+                                    acc[t][n][1] = fmaf(sf.x, fmaf(-zf.x, tk.z, d1), acc[t][n][1]);
+                                    acc[t][n][2] = fmaf(sf.y, fmaf(-zf.y, tk.x, d2), acc[t][n][2]);
+                                    acc[t][n][3] = fmaf(sf.y, fmaf(-zf.y, tk.z, d3), acc[t][n][3]);
+                                }
                             }
-                            const float d0 = dd[0] * t.y, d1 = dd[1] * t.w, d2 = dd[2] * t.y, d3 = dd[3] * t.w;
-                            acc[n][0] = fmaf(sf.x, fmaf(-zf.x, t.x, d0), acc[n][0]);
-                            acc[n][1] = fmaf(sf.x, fmaf(-zf.x, t.z, d1), acc[n][1]);
-                            acc[n][2] = fmaf(sf.y, fmaf(-zf.y, t.x, d2), acc[n][2]);
-                            acc[n][3] = fmaf(sf.y, fmaf(-zf.y, t.z, d3), acc[n][3]);
                         }
                     }
                     __syncwarp();
                     if (lane == 0) sb::arrive(empty(s));
                     if (++s == p.n_slots) { s = 0; ph ^= 1u; }
                 }
-                // ---- this warp's 16 rows of the item: rows 2gq, 2gq+1 of tokens 8n+2c, 8n+2c+1
-                if (active && ok) {
-                    __half* yrow = L.y + 16 * tile + 2 * gq;
-                    if (ONE) {
-                        if (c == 0) *reinterpret_cast<__half2*>(yrow) = __floats2half2_rn(acc[0][0], acc[0][2]);
-                    } else
+                // ---- this warp's rows of the item: rows 2gq, 2gq+1 of tokens 8n+2c, 8n+2c+1 of every tile
+                if (ok) {
 #pragma unroll
-                    for (int n = 0; n < NT; ++n) {
-                        const int m0 = 8 * n + 2 * c;
-                        if (m0 < M) *reinterpret_cast<__half2*>(yrow + static_cast<size_t>(m0) * N) = __floats2half2_rn(acc[n][0], acc[n][2]);
-                        if (m0 + 1 < M) *reinterpret_cast<__half2*>(yrow + static_cast<size_t>(m0 + 1) * N) = __floats2half2_rn(acc[n][1], acc[n][3]);
+                    for (int t = 0; t < TPW; ++t) {
+                        if (t >= n_act) break;
+                        __half* yrow = L.y + 16 * (tile0 + t) + 2 * gq;
+                        if (ONE) {
+                            if (c == 0) *reinterpret_cast<__half2*>(yrow) = __floats2half2_rn(acc[t][0][0], acc[t][0][2]);
+                        } else {
+#pragma unroll
+                            for (int n = 0; n < NT; ++n) {
+                                const int m0 = 8 * n + 2 * c;
+                                if (m0 < M) *reinterpret_cast<__half2*>(yrow + static_cast<size_t>(m0) * N) = __floats2half2_rn(acc[t][n][0], acc[t][n][2]);
+                                if (m0 + 1 < M) *reinterpret_cast<__half2*>(yrow + static_cast<size_t>(m0 + 1) * N) = __floats2half2_rn(acc[t][n][1], acc[t][n][3]);
+                            }
+                        }
                     }
                 }
             }
@@ -353,7 +382,7 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
 // ------------------------------------------------------------------------------------------ host side
 // What the whole set fixes: token tiles, slot geometry, ring depth, grid, sizes.
 struct SetGeometry {
-    int nt, bmax, mmax;
+    int nt, bmax, mmax, tpw;           // tpw: tiles per consumer warp (2 when every layer has one token)
     int off_s, off_z, off_e, off_x, slot_bytes;
     int n_slots, grid, ctas_per_sm;
     size_t smem_bytes;
@@ -385,6 +414,10 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     if (layers == nullptr || n_layers < 1 || sg == nullptr) return SLIM_ERR_INVALID_ARG;
     memset(sg, 0, sizeof *sg);
     sg->ws_bytes = 256;
+    sg->tpw = 2;
+    for (int l = 0; l < n_layers; ++l)
+        if (layers[l].M != 1) sg->tpw = 1;
+    const int tpi = kSetConsumers * sg->tpw;          // tiles per item
     for (int l = 0; l < n_layers; ++l) {
         const slim_layer& L = layers[l];
         if (L.M < 1 || L.M > SLIM_GEMV_MAX_M) return SLIM_ERR_INVALID_ARG;
@@ -394,29 +427,29 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
         if (L.N == 0 || L.K == 0) return SLIM_ERR_INVALID_ARG;
         for (int j = 0; j < gt.G; ++j) sg->bmax = sg->bmax > gt.bits[j] ? sg->bmax : gt.bits[j];
         sg->mmax = sg->mmax > L.M ? sg->mmax : L.M;
-        const int items = (L.N + kSetRowsPerItem - 1) / kSetRowsPerItem;
+        const int items = ((L.N >> 4) + tpi - 1) / tpi;
         sg->n_items += items;
         sg->n_tasks += static_cast<long long>(L.M) * gt.G;
         for (int rb = 0; rb < items; ++rb) {
-            const int th = (L.N >> 4) - kSetConsumers * rb;
-            sg->total_cost += item_cost(th < kSetConsumers ? th : kSetConsumers, gt);
+            const int th = (L.N >> 4) - tpi * rb;
+            sg->total_cost += item_cost(th < tpi ? th : tpi, gt);
         }
         sg->ws_bytes += layer_ws_bytes(L.M, gt);
     }
     if (sg->n_items > 0x3fffffff || sg->n_tasks > 0x3fffffff) return SLIM_ERR_UNSUPPORTED;
     sg->nt = sg->mmax <= 8 ? 1 : 2;
-    sg->off_s = kSetHeader + kSetConsumers * 256 * sg->bmax;
-    sg->off_z = sg->off_s + kSetConsumers * 32;
-    sg->off_e = sg->off_z + kSetConsumers * 32;
+    sg->off_s = kSetHeader + tpi * 256 * sg->bmax;
+    sg->off_z = sg->off_s + tpi * 32;
+    sg->off_e = sg->off_z + tpi * 32;
     sg->off_x = sg->off_e + 128;
     // a 3-bit group brings the fragments of two slices (a set whose widest group has 4 bits may hold one)
     sg->slot_bytes = static_cast<int>(align_to(static_cast<size_t>(sg->off_x) + (sg->bmax >= 3 ? 2 : 1) * 256 * sg->mmax, 128));
-    // as many CTAs per SM (kSetCtasPerSm at most) as still leaves each a ring of 8 slots
+    // as many CTAs per SM (kSetCtasPerSm at most) as still leaves each a ring of 6 slots
     const size_t per_sm = 224 * 1024;
     size_t budget = 0;
     for (sg->ctas_per_sm = kSetCtasPerSm; sg->ctas_per_sm >= 1; --sg->ctas_per_sm) {
         budget = per_sm / sg->ctas_per_sm - 1024 - kSetOffRing;   // 1 KB per CTA is reserved by the system
-        if (budget / sg->slot_bytes >= 8 || sg->ctas_per_sm == 1) break;
+        if (budget / sg->slot_bytes >= 6 || sg->ctas_per_sm == 1) break;
     }
     size_t slots = budget / sg->slot_bytes;
     if (slots > kSetMaxSlots) slots = kSetMaxSlots;
@@ -432,18 +465,18 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
 
 static size_t set_plan_bytes(int n_layers) { return kSetPlanHeader + static_cast<size_t>(n_layers) * sizeof(SetLayer); }
 
-template <int NT, bool ONE>
+template <int NT, bool ONE, int TPW>
 static cudaError_t launch_set(const SetParams& prm, int grid, size_t smem, cudaStream_t stream) {
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        e = cudaFuncSetAttribute(gemv_set_kernel<NT, ONE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        e = cudaFuncSetAttribute(gemv_set_kernel<NT, ONE, TPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    gemv_set_kernel<NT, ONE><<<grid, kSetThreads, smem, stream>>>(prm);
+    gemv_set_kernel<NT, ONE, TPW><<<grid, kSetThreads, smem, stream>>>(prm);
     return cudaGetLastError();
 }
 
@@ -503,7 +536,8 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
         d.y = static_cast<__half*>(L.y);
         d.M = L.M; d.N = L.N; d.K = L.K; d.G = gt.G;
         d.item0 = item;
-        d.n_items = (L.N + slim::kSetRowsPerItem - 1) / slim::kSetRowsPerItem;
+        const int tpi = slim::kSetConsumers * sg.tpw;
+        d.n_items = ((L.N >> 4) + tpi - 1) / tpi;
         d.task0 = task;
         d.x_off = ws_off;
         ws_off += slim::layer_ws_bytes(L.M, gt);
@@ -518,8 +552,8 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
             // CTA c starts at the first item at which the bytes before it reach c/grid of the total
             while (next_cta < sg.grid && cost * sg.grid >= sg.total_cost * static_cast<unsigned long long>(next_cta))
                 item_begin[next_cta++] = item;
-            const int th = (L.N >> 4) - slim::kSetConsumers * rb;
-            cost += slim::item_cost(th < slim::kSetConsumers ? th : slim::kSetConsumers, gt);
+            const int th = (L.N >> 4) - tpi * rb;
+            cost += slim::item_cost(th < tpi ? th : tpi, gt);
         }
         task += L.M * gt.G;
     }
@@ -536,6 +570,7 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
     info->n_items = item;
     info->max_bits = sg.bmax;
     info->max_tokens = sg.mmax;
+    info->tiles_per_warp = sg.tpw;
     info->plan_bytes = slim::set_plan_bytes(n_layers);
     info->workspace_bytes = sg.ws_bytes;
     return SLIM_OK;
@@ -547,6 +582,7 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     if (info->n_layers < 1 || info->grid < 1 || info->grid > slim::kSetMaxGrid || info->n_slots < 2 ||
         info->n_slots > slim::kSetMaxSlots || info->slot_bytes < 128 || info->slot_bytes % 128 != 0 ||
         (info->token_tiles != 1 && info->token_tiles != 2) || info->max_tokens < 1 || info->max_tokens > 8 * info->token_tiles ||
+        info->tiles_per_warp != (info->max_tokens == 1 ? 2 : 1) ||
         info->max_bits < 1 || info->max_bits > 4 || info->stage_tasks < 1)
         return SLIM_ERR_INVALID_ARG;
     const size_t smem = slim::kSetOffRing + static_cast<size_t>(info->n_slots) * info->slot_bytes;
@@ -564,17 +600,18 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     prm.n_layers = info->n_layers;
     prm.n_slots = info->n_slots;
     prm.slot_bytes = info->slot_bytes;
-    prm.off_s = slim::kSetHeader + slim::kSetConsumers * 256 * info->max_bits;
-    prm.off_z = prm.off_s + slim::kSetConsumers * 32;
-    prm.off_e = prm.off_z + slim::kSetConsumers * 32;
+    const int tpi = slim::kSetConsumers * info->tiles_per_warp;
+    prm.off_s = slim::kSetHeader + tpi * 256 * info->max_bits;
+    prm.off_z = prm.off_s + tpi * 32;
+    prm.off_e = prm.off_z + tpi * 32;
     prm.off_x = prm.off_e + 128;
     if (prm.off_x + (info->max_bits >= 3 ? 2 : 1) * 256 * info->max_tokens > info->slot_bytes) return SLIM_ERR_INVALID_ARG;
 
     slim::gemv_set_stage_kernel<<<(info->stage_tasks + 7) / 8, 256, 0, s>>>(prm.layers, prm.ws, info->n_layers, info->stage_tasks);
     SLIM_CUDA_TRY(cudaGetLastError());
-    const cudaError_t e = info->max_tokens == 1 ? slim::launch_set<1, true>(prm, info->grid, smem, s)
-                        : info->token_tiles == 1 ? slim::launch_set<1, false>(prm, info->grid, smem, s)
-                                                 : slim::launch_set<2, false>(prm, info->grid, smem, s);
+    const cudaError_t e = info->max_tokens == 1 ? slim::launch_set<1, true, 2>(prm, info->grid, smem, s)
+                        : info->token_tiles == 1 ? slim::launch_set<1, false, 1>(prm, info->grid, smem, s)
+                                                 : slim::launch_set<2, false, 1>(prm, info->grid, smem, s);
     SLIM_CUDA_TRY(e);
     return SLIM_OK;
 }
