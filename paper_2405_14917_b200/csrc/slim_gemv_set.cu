@@ -416,7 +416,7 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     sg->ws_bytes = 256;
     sg->tpw = 2;
     for (int l = 0; l < n_layers; ++l)
-        if (layers[l].M != 1) sg->tpw = 1;
+        if (layers[l].M > 8) sg->tpw = 1;
     const int tpi = kSetConsumers * sg->tpw;          // tiles per item
     for (int l = 0; l < n_layers; ++l) {
         const slim_layer& L = layers[l];
@@ -582,7 +582,7 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     if (info->n_layers < 1 || info->grid < 1 || info->grid > slim::kSetMaxGrid || info->n_slots < 2 ||
         info->n_slots > slim::kSetMaxSlots || info->slot_bytes < 128 || info->slot_bytes % 128 != 0 ||
         (info->token_tiles != 1 && info->token_tiles != 2) || info->max_tokens < 1 || info->max_tokens > 8 * info->token_tiles ||
-        info->tiles_per_warp != (info->max_tokens == 1 ? 2 : 1) ||
+        info->tiles_per_warp != (info->max_tokens <= 8 ? 2 : 1) ||
         info->max_bits < 1 || info->max_bits > 4 || info->stage_tasks < 1)
         return SLIM_ERR_INVALID_ARG;
     const size_t smem = slim::kSetOffRing + static_cast<size_t>(info->n_slots) * info->slot_bytes;
@@ -610,7 +610,7 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     slim::gemv_set_stage_kernel<<<(info->stage_tasks + 7) / 8, 256, 0, s>>>(prm.layers, prm.ws, info->n_layers, info->stage_tasks);
     SLIM_CUDA_TRY(cudaGetLastError());
     const cudaError_t e = info->max_tokens == 1 ? slim::launch_set<1, true, 2>(prm, info->grid, smem, s)
-                        : info->token_tiles == 1 ? slim::launch_set<1, false, 1>(prm, info->grid, smem, s)
+                        : info->token_tiles == 1 ? slim::launch_set<1, false, 2>(prm, info->grid, smem, s)
                                                  : slim::launch_set<2, false, 1>(prm, info->grid, smem, s);
     SLIM_CUDA_TRY(e);
     return SLIM_OK;
