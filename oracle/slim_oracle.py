@@ -14,7 +14,8 @@ says otherwise.
 
 Pinned (tests/test_oracle_*.py): bit budget, quantizer closed forms and brute
 force, packing positions, dequantisation single-rounding, linear layer special
-cases, the SQC line search (brute force, never worse than tau = 1, exact grids).  Parity unpinned: nothing in this file (the paper's perplexity / accuracy
+cases, the SQC line search (brute force, never worse than tau = 1, exact grids), the SBA search
+(library KL, shift invariance, constructed optima, budget).  Parity unpinned: nothing in this file (the paper's perplexity / accuracy
 / token-per-second tables are not reproduced at all).
 """
 from __future__ import annotations
@@ -333,6 +334,59 @@ def unpack(packed: np.ndarray, N: int, K: int, bits, g: int = GROUP) -> np.ndarr
             unit_base += w
         prefix += b
     return codes
+
+
+# --------------------------------------------------------------------------- SBA search (Algorithm 2, func SBA)
+def softmax_kl(y_ref: np.ndarray, y_q: np.ndarray) -> np.ndarray:
+    """D_kl( softmax(y_ref[t]) || softmax(y_q[t]) ) for every token row t, natural logarithm.
+
+    The objective of Eq. 4 compares the layer outputs x w^T and x w-hat^T; the appendix on the
+    evaluation function of SBA turns each output into a probability distribution with a softmax
+    first.  The softmax runs over the output features of one token; one value per token is
+    returned.  Written as the definition: p = exp(y - logsumexp(y)), sum_n p_n (log p_n - log q_n).
+    """
+    a = np.asarray(y_ref, dtype=np.float64)
+    b = np.asarray(y_q, dtype=np.float64)
+    out = np.empty(a.shape[0], dtype=np.float64)
+    for t in range(a.shape[0]):
+        la = a[t] - a[t].max()
+        lb = b[t] - b[t].max()
+        log_p = la - np.log(np.exp(la).sum())
+        log_q = lb - np.log(np.exp(lb).sum())
+        out[t] = float((np.exp(log_p) * (log_p - log_q)).sum())
+    return out
+
+
+def sba_search(W16: np.ndarray, x16: np.ndarray, act_norm: np.ndarray, avg_bits: int, g: int = GROUP,
+               include_uniform: bool = True):
+    """Salience-Determined Bit Allocation, func SBA of Algorithm 2 (Sec. 3.2.2, Eq. 4).
+
+    Groups are ranked by salience; for p = 0 (uniform; the loop of Algorithm 2 starts at 1, the
+    appendix on the search names the uniform map as one end of the range), 1, ..., floor(G/2) the p
+    most salient groups get N-bar+1 bits and the p least salient N-bar-1 (the double pointer), the
+    weight is fake-quantised with the quantizer of Eq. 1 under that map, and the candidate's error
+    is the KL divergence between the softmax of the full-precision output x w^T and of x w-hat^T,
+    averaged over the calibration tokens.  The first p with the smallest error wins (Algorithm 2
+    compares with '<').  Returns (p_star, bits[G], errors[list over the candidates p]).
+    """
+    W = W16.astype(np.float64)
+    x = x16.astype(np.float64)
+    S = group_salience(W16, act_norm, g)
+    G = S.shape[0]
+    y_f = x @ W.T
+    first = 0 if include_uniform else 1
+    errors = []
+    for p in range(first, G // 2 + 1):
+        bits = allocate_bits(S, avg_bits, p)
+        codes, scales, zeros = quantize_minmax(W16, bits, g)
+        y_q = linear_f64(x16, codes, scales, zeros, g)
+        errors.append(float(softmax_kl(y_f, y_q).mean()))
+    best = 0
+    for i in range(1, len(errors)):
+        if errors[i] < errors[best]:
+            best = i
+    p_star = first + best
+    return p_star, allocate_bits(S, avg_bits, p_star), errors
 
 
 # --------------------------------------------------------------------------- convenience
