@@ -244,6 +244,34 @@ int slim_quantize_minmax(const void* W, const uint8_t* bits_host, uint8_t* codes
 int slim_quantize_sqc(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
                       int* tau_index, int N, int K, int g, double lambda, int n, void* stream);
 
+/* ---- Salience-Determined Bit Allocation (func SBA of Algorithm 2, Sec. 3.2.2, Eq. 4) --------- */
+
+/* y = x * W^T in full precision: x fp16 [M][K], W fp16 [N][K], y fp32 [M][N] (device), fp32
+ * accumulation in k order.  The reference output "x w_f^T" of Eq. 4.  K a multiple of 32. */
+int slim_dense_linear(const void* x, const void* W, float* y, int M, int N, int K, void* stream);
+
+/* kl[t] = D_kl( softmax(y_ref[t]) || softmax(y_q[t]) ) for every token t (natural logarithm, softmax
+ * over the N outputs of the token; the error measure of SBA, appendix on its evaluation function).
+ * y_ref fp32 [M][N], y_q fp16 [M][N], kl fp64 [M], all device; fp64 arithmetic, fixed reduction order. */
+int slim_softmax_kl(const float* y_ref, const void* y_q, double* kl, int M, int N, void* stream);
+
+/* Host-only: bytes of workspace slim_sba_search needs (scratch of the layer calls, codes, scales, zeros,
+ * packed buffer, both outputs, one error per candidate and token). */
+int slim_sba_workspace_bytes(int M, int N, int K, int g, int avg_bits, size_t* out_bytes);
+
+/* The search: groups ranked by salience (slim_group_salience; equal salience: lower index first);
+ * for p = 0 (only if include_uniform), 1, ..., floor(G/2) the p most salient groups get avg_bits+1
+ * bits and the p least salient avg_bits-1, the weight is quantised with slim_quantize_minmax under
+ * that map, packed, and x * W-hat^T is computed by slim_mpq_gemv / slim_mpq_gemm; the candidate's
+ * error is the mean over the M calibration tokens of slim_softmax_kl against slim_dense_linear(x, W).
+ * The first p with the smallest error wins (Algorithm 2 compares with '<').
+ * W fp16 [N][K], x fp16 [M][K], act_norm fp32 [K]: device.  workspace: device, 256-byte aligned.
+ * Outputs on the HOST: *p_star, bits_host_out[G], errors_host[candidates] (may be NULL).
+ * The call synchronises `stream` (it returns results to the host).  avg_bits in {2, 3}. */
+int slim_sba_search(const void* W, const void* x, const float* act_norm, int M, int N, int K, int g, int avg_bits,
+                    int include_uniform, void* workspace, size_t workspace_bytes,
+                    int* p_star_host, uint8_t* bits_host_out, double* errors_host, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -61,6 +61,10 @@ def lib():
             "slim_gemv_set_bytes": [vp, i, i, ctypes.POINTER(sz), ctypes.POINTER(sz)],
             "slim_gemv_set_plan": [vp, i, i, vp, sz, vp, vp],
             "slim_mpq_gemv_set": [vp, vp, vp, sz, vp],
+            "slim_dense_linear": [vp, vp, vp, i, i, i, vp],
+            "slim_softmax_kl": [vp, vp, vp, i, i, vp],
+            "slim_sba_workspace_bytes": [i, i, i, i, i, ctypes.POINTER(sz)],
+            "slim_sba_search": [vp, vp, vp, i, i, i, i, i, i, vp, sz, vp, vp, vp, vp],
         }
         for name, args in sigs.items():
             fn = getattr(L, name)
@@ -242,6 +246,51 @@ def quantize_sqc(W: torch.Tensor, bits, lam: float = 0.1, n: int = 50):
                                                         _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
                                                         _dev(tau, torch.int32, "tau_index"), N, K, GROUP, float(lam), int(n), _stream(W)))
     return codes, scales, zeros, tau
+
+
+def dense_linear(x: torch.Tensor, W: torch.Tensor) -> torch.Tensor:
+    """y = x W^T in full precision (fp16 in, fp32 accumulate and out): the reference output of SBA."""
+    M, K = x.shape
+    N = W.shape[0]
+    y = torch.empty((M, N), dtype=torch.float32, device=x.device)
+    _check("slim_dense_linear", lib().slim_dense_linear(_dev(x, torch.float16, "x"), _dev(W, torch.float16, "W"),
+                                                        _dev(y, torch.float32, "y"), M, N, K, _stream(x)))
+    return y
+
+
+def softmax_kl(y_ref: torch.Tensor, y_q: torch.Tensor) -> torch.Tensor:
+    """KL divergence between softmax(y_ref[t]) and softmax(y_q[t]) per token t (fp64)."""
+    M, N = y_ref.shape
+    kl = torch.empty(M, dtype=torch.float64, device=y_ref.device)
+    _check("slim_softmax_kl", lib().slim_softmax_kl(_dev(y_ref, torch.float32, "y_ref"), _dev(y_q, torch.float16, "y_q"),
+                                                    _dev(kl, torch.float64, "kl"), M, N, _stream(y_ref)))
+    return kl
+
+
+def sba_workspace_bytes(M: int, N: int, K: int, avg_bits: int, g: int = GROUP) -> int:
+    out = ctypes.c_size_t(0)
+    _check("slim_sba_workspace_bytes", lib().slim_sba_workspace_bytes(M, N, K, g, avg_bits, ctypes.byref(out)))
+    return out.value
+
+
+def sba_search(W: torch.Tensor, x: torch.Tensor, act_norm: torch.Tensor, avg_bits: int, include_uniform: bool = True,
+               workspace: torch.Tensor | None = None):
+    """Salience-Determined Bit Allocation search (func SBA of Algorithm 2) on the device.
+    Returns (p_star, bits[G] (numpy), errors (numpy, one per candidate p))."""
+    N, K = W.shape
+    M = x.shape[0]
+    G = K // GROUP
+    if workspace is None:
+        workspace = torch.empty(sba_workspace_bytes(M, N, K, avg_bits), dtype=torch.uint8, device=W.device)
+    p_star = ctypes.c_int(-1)
+    bits = np.zeros(G, dtype=np.uint8)
+    errors = np.zeros(G // 2 + 1 - (0 if include_uniform else 1), dtype=np.float64)
+    _check("slim_sba_search", lib().slim_sba_search(_dev(W, torch.float16, "W"), _dev(x, torch.float16, "x"),
+                                                    _dev(act_norm, torch.float32, "act_norm"), M, N, K, GROUP, avg_bits,
+                                                    1 if include_uniform else 0, _dev(workspace, torch.uint8, "workspace"),
+                                                    workspace.numel(), ctypes.addressof(p_star), bits.ctypes.data,
+                                                    errors.ctypes.data, _stream(W)))
+    return p_star.value, bits, errors
 
 
 class _Layer(ctypes.Structure):
