@@ -232,6 +232,12 @@ int slim_allocate_bits(const double* salience_host, int G, int avg_bits, int p, 
 int slim_quantize_minmax(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
                          int N, int K, int g, void* stream);
 
+/* slim_quantize_minmax with the binarisation of Eq. 2 for the one-bit groups: q = [w >= 0]
+ * (sign(0) = +1), alpha = mean |w| of the (row, group), stored as s = fp16(2 alpha), z = 1/2, so
+ * that s (q - z) = +-alpha.  Groups of two or more bits use Eq. 1 as above.  Same layouts. */
+int slim_quantize_minmax_sign1(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
+                               int N, int K, int g, void* stream);
+
 /* Salience-Weighted Quantizer Calibration (Sec. 3.3, Eq. 5; function SQC of Algorithm 2), per
  * (row, group): for tau_i = 1 - lambda + i * lambda / n, i = 0 .. 2n-1, the quantizer
  * Delta = tau (w_max - w_min) / (2^b - 1), z = -round(tau w_min / Delta) is tried on the group and

@@ -212,6 +212,19 @@ def quantize_sign_alpha_1bit(W16: np.ndarray, g: int = GROUP):
     return codes, scales, zeros
 
 
+def quantize_minmax_sign1(W16: np.ndarray, bits: np.ndarray, g: int = GROUP):
+    """Eq. 1 for the groups of two or more bits, Eq. 2 (sign, alpha) for the one-bit groups: the
+    quantizer the paper describes "when converted to 1-bit" (Sec. 3.1), in the deployed layouts."""
+    bits = np.asarray(bits, dtype=np.uint8)
+    codes, scales, zeros = quantize_minmax(W16, bits, g)
+    c1, s1, z1 = quantize_sign_alpha_1bit(W16, g)
+    for j in np.nonzero(bits == 1)[0]:
+        codes[:, g * j:g * (j + 1)] = c1[:, g * j:g * (j + 1)]
+        scales[j] = s1[j]
+        zeros[j] = z1[j]
+    return codes, scales, zeros
+
+
 # --------------------------------------------------------------------------- dequantisation
 def _expand_group_param(p: np.ndarray, g: int) -> np.ndarray:
     """[G][N] per-(group,row) parameter -> [N][K] per-element."""

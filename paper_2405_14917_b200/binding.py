@@ -58,6 +58,7 @@ def lib():
             "slim_group_salience": [vp, vp, vp, i, i, i, vp],
             "slim_allocate_bits": [vp, i, i, i, vp],
             "slim_quantize_minmax": [vp, vp, vp, vp, vp, i, i, i, vp],
+            "slim_quantize_minmax_sign1": [vp, vp, vp, vp, vp, i, i, i, vp],
             "slim_gemv_set_bytes": [vp, i, i, ctypes.POINTER(sz), ctypes.POINTER(sz)],
             "slim_gemv_set_plan": [vp, i, i, vp, sz, vp, vp],
             "slim_mpq_gemv_set": [vp, vp, vp, sz, vp],
@@ -220,16 +221,20 @@ def allocate_bits(salience, avg_bits: int, p: int = -1) -> np.ndarray:
     return out
 
 
-def quantize_minmax(W: torch.Tensor, bits):
+def quantize_minmax(W: torch.Tensor, bits, one_bit: str = "minmax"):
+    """Eq. 1 per (row, group); one_bit="sign_alpha" binarises the one-bit groups with Eq. 2 instead."""
+    if one_bit not in ("minmax", "sign_alpha"):
+        raise ValueError("one_bit must be 'minmax' or 'sign_alpha'")
+    fn_name = "slim_quantize_minmax" if one_bit == "minmax" else "slim_quantize_minmax_sign1"
     b = _bits(bits)
     N, K = W.shape
     G = K // GROUP
     codes = torch.empty((N, K), dtype=torch.uint8, device=W.device)
     scales = torch.empty((G, N), dtype=torch.float16, device=W.device)
     zeros = torch.empty((G, N), dtype=torch.float16, device=W.device)
-    _check("slim_quantize_minmax", lib().slim_quantize_minmax(_dev(W, torch.float16, "W"), _bp(b), _dev(codes, torch.uint8, "codes"),
-                                                              _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
-                                                              N, K, GROUP, _stream(W)))
+    _check(fn_name, getattr(lib(), fn_name)(_dev(W, torch.float16, "W"), _bp(b), _dev(codes, torch.uint8, "codes"),
+                                            _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
+                                            N, K, GROUP, _stream(W)))
     return codes, scales, zeros
 
 

@@ -40,10 +40,12 @@ __device__ __forceinline__ unsigned short double_to_half_bits_rn(double v) {
     return h;
 }
 
-// One warp per (row, group): lane l owns columns 4l..4l+3 of the group.
+// One warp per (row, group): lane l owns columns 4l..4l+3 of the group.  With sign_alpha != 0 the
+// one-bit groups are binarised as in Eq. 2 (q = [w >= 0], alpha = mean |w|, stored as s = 2 alpha,
+// z = 1/2 so that s (q - z) = +-alpha); all other groups, and all groups otherwise, use Eq. 1.
 __global__ void __launch_bounds__(256) quantize_minmax_kernel(const __half* __restrict__ W, uint8_t* __restrict__ codes,
                                                               __half* __restrict__ scales, __half* __restrict__ zeros,
-                                                              int N, int K, GroupTable gt) {
+                                                              int N, int K, int sign_alpha, GroupTable gt) {
     const long long warp = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     const int G = gt.G;
@@ -64,6 +66,22 @@ __global__ void __launch_bounds__(256) quantize_minmax_kernel(const __half* __re
     lo = fminf(lo, 0.0f);
     hi = fmaxf(hi, 0.0f);
     const int b = gt.bits[j];
+    if (sign_alpha != 0 && b == 1) {
+        // the sum of 128 fp16 magnitudes is exact in fp64, whatever the order
+        double sum = (fabs(static_cast<double>(w[0])) + fabs(static_cast<double>(w[1]))) +
+                     (fabs(static_cast<double>(w[2])) + fabs(static_cast<double>(w[3])));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        uint32_t out = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) out |= (w[i] >= 0.0f ? 1u : 0u) << (8 * i);
+        *reinterpret_cast<uint32_t*>(codes + off) = out;
+        if (lane == 0) {
+            scales[static_cast<size_t>(j) * N + n] = __ushort_as_half(double_to_half_bits_rn(sum / 64.0));   // 2 * mean
+            zeros[static_cast<size_t>(j) * N + n] = __float2half_rn(0.5f);
+        }
+        return;
+    }
     const double levels = static_cast<double>((1 << b) - 1);
     unsigned short sbits = double_to_half_bits_rn((static_cast<double>(hi) - static_cast<double>(lo)) / levels);
     if ((sbits & 0x7fffu) == 0x7c00u) sbits = 0x7bffu;  // beyond fp16 range -> 65504
@@ -100,8 +118,8 @@ int slim_group_salience(const void* W, const float* act_norm, double* salience, 
     return SLIM_OK;
 }
 
-int slim_quantize_minmax(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
-                         int N, int K, int g, void* stream) {
+static int quantize_minmax_impl(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
+                                int N, int K, int g, int sign_alpha, void* stream) {
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;
@@ -112,9 +130,20 @@ int slim_quantize_minmax(const void* W, const uint8_t* bits_host, uint8_t* codes
     const long long warps = static_cast<long long>(N) * gt.G;
     const unsigned grid = static_cast<unsigned>((warps + 7) / 8);
     slim::quantize_minmax_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const __half*>(W), codes, static_cast<__half*>(scales), static_cast<__half*>(zeros), N, K, gt);
+        static_cast<const __half*>(W), codes, static_cast<__half*>(scales), static_cast<__half*>(zeros), N, K, sign_alpha, gt);
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;
+}
+
+
+int slim_quantize_minmax(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
+                         int N, int K, int g, void* stream) {
+    return quantize_minmax_impl(W, bits_host, codes, scales, zeros, N, K, g, 0, stream);
+}
+
+int slim_quantize_minmax_sign1(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
+                               int N, int K, int g, void* stream) {
+    return quantize_minmax_impl(W, bits_host, codes, scales, zeros, N, K, g, 1, stream);
 }
 
 }  // extern "C"

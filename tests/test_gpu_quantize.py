@@ -105,3 +105,35 @@ def test_sqc_edge_groups_and_other_grids():
         assert (scales.cpu().numpy().view(np.uint16) == s_ref.view(np.uint16)).all()
         assert (zeros.cpu().numpy().view(np.uint16) == z_ref.view(np.uint16)).all()
         assert (codes.cpu().numpy() == c_ref).all()
+
+
+@pytest.mark.parametrize("N,K,M", [(272, 1536, 1), (512, 1024, 5), (256, 2048, 40)])
+def test_eq2_one_bit_groups_end_to_end(N, K, M):
+    """Eq. 2 for the one-bit groups: quantizer bit-exact against the oracle, then the packed layer through every
+    entry point of the hot path (z = 1/2) against the fp64 oracle."""
+    from tests.helpers import check_output
+    slim = _slim()
+    seed = wl.layer_seed("test", f"sign1-{N}x{K}", M)
+    W, a, x = wl.make_weight(seed, N, K), wl.make_act_norms(seed, K), wl.make_x(seed, M, K)
+    bits = orc.allocate_bits(orc.group_salience(W, a), 2)
+    assert (bits == 1).sum() == K // 128 // 4
+    codes, scales, zeros = slim.quantize_minmax(torch.from_numpy(W).cuda(), bits, one_bit="sign_alpha")
+    c_ref, s_ref, z_ref = orc.quantize_minmax_sign1(W, bits)
+    assert (codes.cpu().numpy() == c_ref).all()
+    assert (scales.cpu().numpy().view(np.uint16) == s_ref.view(np.uint16)).all()
+    assert (zeros.cpu().numpy().view(np.uint16) == z_ref.view(np.uint16)).all()
+    packed = slim.pack_weights(codes, bits)
+    What = slim.dequant(packed, bits, scales, zeros, N, K).cpu().numpy()
+    assert (What.view(np.uint16) == orc.dequant_f16(c_ref, s_ref, z_ref).view(np.uint16)).all()
+    y_ref = orc.linear_f64(x, c_ref, s_ref, z_ref)
+    xd = torch.from_numpy(x).cuda()
+    layer = slim.QuantLinear(packed, bits, scales, zeros, N, K)
+    ws = slim.new_workspace(M, N, K, bits)
+    check_output(layer.forward(xd, ws).cpu().numpy(), y_ref, f"Eq. 2 groups, M={M}")
+    slim.workspace_status(ws)
+    if M <= 16:
+        y = torch.empty(M, N, dtype=torch.float16, device="cuda")
+        s = slim.LayerSet([(layer, xd, y)])
+        s.run()
+        s.check()
+        check_output(y.cpu().numpy(), y_ref, f"Eq. 2 groups, layer set, M={M}")

@@ -5,6 +5,7 @@ import numpy as np
 import pytest
 
 from oracle import slim_oracle as orc
+from paper_2405_14917_b200 import workloads as wl
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "eq1_hand_cases.txt")
 
@@ -132,3 +133,23 @@ def test_sign_alpha_binarisation_eq2():
     a1 = 127.0 / 128.0
     assert What[1, 0] == pytest.approx(a1, rel=2**-11) and What[1, 0] > 0
     assert (What[1, 1:] < 0).all()
+
+
+def test_mixed_quantizer_takes_eq2_only_for_one_bit_groups():
+    seed = wl.layer_seed("test", "sign1", 0)
+    W = wl.make_weight(seed, 24, 768)
+    bits = np.array([1, 2, 3, 1, 2, 1], dtype=np.uint8)
+    codes, scales, zeros = orc.quantize_minmax_sign1(W, bits)
+    c0, s0, z0 = orc.quantize_minmax(W, bits)
+    c1, s1, z1 = orc.quantize_sign_alpha_1bit(W)
+    for j, b in enumerate(bits):
+        cols = slice(128 * j, 128 * j + 128)
+        src = (c1, s1, z1) if b == 1 else (c0, s0, z0)
+        assert (codes[:, cols] == src[0][:, cols]).all() and (scales[j] == src[1][j]).all() and (zeros[j] == src[2][j]).all()
+    # Eq. 2: the dequantised one-bit groups are +-alpha with alpha = mean |w| (rounded once to fp16 as 2 alpha)
+    What = orc.dequant_f64(codes, scales, zeros)
+    w = W.astype(np.float64)
+    for j in np.nonzero(bits == 1)[0]:
+        cols = slice(128 * j, 128 * j + 128)
+        alpha = np.float16(2 * np.abs(w[:, cols]).mean(axis=1)).astype(np.float64) / 2
+        assert (What[:, cols] == np.where(w[:, cols] >= 0, alpha[:, None], -alpha[:, None])).all()
