@@ -42,12 +42,13 @@ struct SetLayer {
     const __half* zeros;
     __half* y;
     size_t x_off;          // workspace offset of the layer's staged activations, group after group:
-                           // (sum_k x, 2^(24-S)) float2[16], then the fragments [slice][8 mma][M][4 lanes] x 8 B
+                           // (sum_k x, 2^(24-S)) float2[16], then the fragments [slice][8 mma][MP][4 lanes] x 8 B
     size_t pad0;
     int M, N, K, G;
     int item0, n_items;    // this layer's items in the set's numbering
     int task0;             // first (token, group) staging task of the layer
-    int pad;
+    int MP;                // tokens in the staged layout: 1 if every layer of the set has one token, else 8 or 16
+                           // for the whole set (absent tokens are staged as zeros, so the kernel reads without a test)
     uint16_t prefix[SLIM_MAX_GROUPS + 1];
     uint16_t pre3[SLIM_MAX_GROUPS + 1];   // 3-bit groups (two slices) before group j
     uint8_t bits[SLIM_MAX_GROUPS];
@@ -125,11 +126,18 @@ __global__ void __launch_bounds__(256) gemv_set_stage_kernel(const SetLayer* __r
     }
     const SetLayer& L = layers[lo];
     const int pi = task - L.task0;
-    const int m = pi / L.G, j = pi - m * L.G;
-    uint8_t* grp = ws + L.x_off + staged_group_offset(j, L.pre3[j], L.M);
+    const int m = pi / L.G, j = pi - m * L.G;        // m < MP
+    uint8_t* grp = ws + L.x_off + staged_group_offset(j, L.pre3[j], L.MP);
     float2* sxe = reinterpret_cast<float2*>(grp);
-    const float2 r = stage_group(L.x + static_cast<size_t>(m) * L.K + j * SLIM_GROUP, grp + 128, L.bits[j], m, L.M, lane);
-    if (lane == 0) sxe[m] = r;
+    if (m < L.M) {
+        const float2 r = stage_group(L.x + static_cast<size_t>(m) * L.K + j * SLIM_GROUP, grp + 128, L.bits[j], m, L.MP, lane);
+        if (lane == 0) sxe[m] = r;
+    } else {
+        // a token the layer does not have: zero fragments in every slice of the group
+        const int cc = lane & 3, mi = lane >> 2;
+        for (int sl = 0; sl < slice_count(L.bits[j]); ++sl)
+            *reinterpret_cast<uint2*>(grp + 128 + (((static_cast<size_t>(sl) * 8 + mi) * L.MP + m) * 4 + cc) * 8) = make_uint2(0u, 0u);
+    }
     if (m == 0 && lane < 16 && lane >= L.M) sxe[lane] = make_float2(0.f, 1.f);   // absent tokens read 0
 }
 
@@ -160,6 +168,7 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
     volatile int* abort = reinterpret_cast<volatile int*>(smem + kSetOffAbort);
     const uint32_t ring = sbase + kSetOffRing;
     constexpr int TPI = kSetConsumers * TPW;                  // tiles per item
+    constexpr int MPK = ONE ? 1 : 8 * NT;                     // tokens in the staged layout
 
     if (tid == 0) {
         for (int s = 0; s < p.n_slots; ++s) { sb::init(full(s), 1); sb::init(empty(s), kSetConsumers); }
@@ -201,7 +210,7 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                     __syncwarp();
                     have = l;
                 }
-                const int rb = i - D->item0, N = D->N, M = D->M, G = D->G;
+                const int rb = i - D->item0, N = D->N, MP = D->MP, G = D->G;
                 const int tiles_here = min(TPI, (N >> 4) - TPI * rb);
                 // lane 0 brings the slices, lanes 1 and 2 scales and zeros, lane 3 the staged activations
                 const uint8_t* base = lane == 0 ? D->packed
@@ -217,14 +226,14 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                     if (!__all_sync(0xffffffffu, sb::wait(empty(s), ph ^ 1u, abort))) { ok = false; break; }
                     const uint32_t b = D->bits[j];
                     const uint32_t wbytes = static_cast<uint32_t>(tiles_here) * 256u * b;
-                    const uint32_t xbytes = 128u + static_cast<uint32_t>(slice_count(b)) * 256u * M;
+                    const uint32_t xbytes = 128u + static_cast<uint32_t>(slice_count(b)) * 256u * MP;
                     const uint32_t slot = ring + static_cast<uint32_t>(s) * p.slot_bytes;
                     if (lane == 0) {
                         asm volatile("st.shared.u32 [%0], %1;" ::"r"(slot), "r"(b) : "memory");
                         sb::expect_tx(full(s), wbytes + 2 * szb + xbytes);
                     }
                     const size_t off = lane == 0 ? 16ull * N * D->prefix[j] + static_cast<size_t>(TPI * rb) * 256 * b
-                                     : lane == 3 ? staged_group_offset(j, D->pre3[j], M)
+                                     : lane == 3 ? staged_group_offset(j, D->pre3[j], MP)
                                                  : 2ull * static_cast<size_t>(j) * N;
                     const uint32_t bytes = lane == 0 ? wbytes : lane == 3 ? xbytes : szb;
                     __syncwarp();
@@ -291,10 +300,8 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                                     const int mi = u * MPU + ii;
 #pragma unroll
                                     for (int n = 0; n < NT; ++n) {
-                                        const int m = 8 * n + gq;
-                                        uint2 bv = make_uint2(0u, 0u);
-                                        if (ONE) bv = lds64(xs_slot + (mi * 4 + c) * 8);
-                                        else if (m < M) bv = lds64(xs_slot + ((mi * M + m) * 4 + c) * 8);
+                                        // fragment of token 8n + gq (tokens the layer lacks are staged as zeros)
+                                        const uint2 bv = lds64(xs_slot + ((mi * MPK + (ONE ? 0 : 8 * n + gq)) * 4 + c) * 8);
 #pragma unroll
                                         for (int t = 0; t < TPW; ++t) {
                                             const uint32_t a0 = pair<WD>(wd[t].x, shx[t], 2 * ii), a1 = pair<WD>(wd[t].y, shy[t], 2 * ii);
@@ -309,7 +316,7 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                         switch (b) {
                             case 1: run_slice(W1{}, WidthTag<1>{}, 0, xs_slot0); break;
                             case 2: run_slice(W2{}, WidthTag<1>{}, 0, xs_slot0); break;
-                            case 3: run_slice(W2{}, WidthTag<1>{}, 0, xs_slot0); run_slice(W1{}, WidthTag<0>{}, 2, xs_slot0 + 8 * M * 32); break;
+                            case 3: run_slice(W2{}, WidthTag<1>{}, 0, xs_slot0); run_slice(W1{}, WidthTag<0>{}, 2, xs_slot0 + 8 * MPK * 32); break;
                             default: run_slice(W4{}, WidthTag<1>{}, 0, xs_slot0); break;
                         }
 
@@ -382,7 +389,7 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
 // ------------------------------------------------------------------------------------------ host side
 // What the whole set fixes: token tiles, slot geometry, ring depth, grid, sizes.
 struct SetGeometry {
-    int nt, bmax, mmax, tpw;           // tpw: tiles per consumer warp (2 when every layer has one token)
+    int nt, bmax, mmax, tpw, mpad;     // tpw: tiles per consumer warp; mpad: tokens in the staged layout
     int off_s, off_z, off_e, off_x, slot_bytes;
     int n_slots, grid, ctas_per_sm;
     size_t smem_bytes;
@@ -414,9 +421,9 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     if (layers == nullptr || n_layers < 1 || sg == nullptr) return SLIM_ERR_INVALID_ARG;
     memset(sg, 0, sizeof *sg);
     sg->ws_bytes = 256;
-    sg->tpw = 2;
-    for (int l = 0; l < n_layers; ++l)
-        if (layers[l].M > 8) sg->tpw = 1;
+    for (int l = 0; l < n_layers; ++l) sg->mmax = sg->mmax > layers[l].M ? sg->mmax : layers[l].M;
+    sg->tpw = sg->mmax > 8 ? 1 : 2;
+    sg->mpad = sg->mmax <= 1 ? 1 : (sg->mmax <= 8 ? 8 : 16);
     const int tpi = kSetConsumers * sg->tpw;          // tiles per item
     for (int l = 0; l < n_layers; ++l) {
         const slim_layer& L = layers[l];
@@ -426,15 +433,14 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
         if (st != SLIM_OK) return st;
         if (L.N == 0 || L.K == 0) return SLIM_ERR_INVALID_ARG;
         for (int j = 0; j < gt.G; ++j) sg->bmax = sg->bmax > gt.bits[j] ? sg->bmax : gt.bits[j];
-        sg->mmax = sg->mmax > L.M ? sg->mmax : L.M;
         const int items = ((L.N >> 4) + tpi - 1) / tpi;
         sg->n_items += items;
-        sg->n_tasks += static_cast<long long>(L.M) * gt.G;
+        sg->n_tasks += static_cast<long long>(sg->mpad) * gt.G;
         for (int rb = 0; rb < items; ++rb) {
             const int th = (L.N >> 4) - tpi * rb;
             sg->total_cost += item_cost(th < tpi ? th : tpi, gt);
         }
-        sg->ws_bytes += layer_ws_bytes(L.M, gt);
+        sg->ws_bytes += layer_ws_bytes(sg->mpad, gt);
     }
     if (sg->n_items > 0x3fffffff || sg->n_tasks > 0x3fffffff) return SLIM_ERR_UNSUPPORTED;
     sg->nt = sg->mmax <= 8 ? 1 : 2;
@@ -443,7 +449,7 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     sg->off_e = sg->off_z + tpi * 32;
     sg->off_x = sg->off_e + 128;
     // a 3-bit group brings the fragments of two slices (a set whose widest group has 4 bits may hold one)
-    sg->slot_bytes = static_cast<int>(align_to(static_cast<size_t>(sg->off_x) + (sg->bmax >= 3 ? 2 : 1) * 256 * sg->mmax, 128));
+    sg->slot_bytes = static_cast<int>(align_to(static_cast<size_t>(sg->off_x) + (sg->bmax >= 3 ? 2 : 1) * 256 * sg->mpad, 128));
     // as many CTAs per SM (kSetCtasPerSm at most) as still leaves each a ring of 6 slots
     const size_t per_sm = 224 * 1024;
     size_t budget = 0;
@@ -535,12 +541,13 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
         d.zeros = static_cast<const __half*>(L.zeros);
         d.y = static_cast<__half*>(L.y);
         d.M = L.M; d.N = L.N; d.K = L.K; d.G = gt.G;
+        d.MP = sg.mpad;
         d.item0 = item;
         const int tpi = slim::kSetConsumers * sg.tpw;
         d.n_items = ((L.N >> 4) + tpi - 1) / tpi;
         d.task0 = task;
         d.x_off = ws_off;
-        ws_off += slim::layer_ws_bytes(L.M, gt);
+        ws_off += slim::layer_ws_bytes(sg.mpad, gt);
         memcpy(d.prefix, gt.prefix, sizeof d.prefix);
         memcpy(d.bits, gt.bits, sizeof d.bits);
         d.pre3[0] = 0;
@@ -555,7 +562,7 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
             const int th = (L.N >> 4) - tpi * rb;
             cost += slim::item_cost(th < tpi ? th : tpi, gt);
         }
-        task += L.M * gt.G;
+        task += sg.mpad * gt.G;
     }
     while (next_cta <= sg.grid) item_begin[next_cta++] = item;
     SLIM_CUDA_TRY(cudaMemcpyAsync(plan_dev, item_begin, static_cast<size_t>(sg.grid + 1) * sizeof(int), cudaMemcpyHostToDevice, s));
@@ -605,7 +612,7 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     prm.off_z = prm.off_s + tpi * 32;
     prm.off_e = prm.off_z + tpi * 32;
     prm.off_x = prm.off_e + 128;
-    if (prm.off_x + (info->max_bits >= 3 ? 2 : 1) * 256 * info->max_tokens > info->slot_bytes) return SLIM_ERR_INVALID_ARG;
+    if (prm.off_x + (info->max_bits >= 3 ? 2 : 1) * 256 * (info->max_tokens == 1 ? 1 : 8 * info->token_tiles) > info->slot_bytes) return SLIM_ERR_INVALID_ARG;
 
     slim::gemv_set_stage_kernel<<<(info->stage_tasks + 7) / 8, 256, 0, s>>>(prm.layers, prm.ws, info->n_layers, info->stage_tasks);
     SLIM_CUDA_TRY(cudaGetLastError());

@@ -126,9 +126,12 @@ def test_layer_set_sizes_and_argument_errors(slim):
     # plan: item ranges of the CTAs, then one descriptor per layer; it grows by a fixed step per layer
     st2, pb2, _ = _set_bytes(slim, ok + [(1, 128, 128, [2])])
     assert st2 == 0 and pb2 > pb and (pb2 - pb) % 16 == 0
-    # workspace: status header + per layer the sums [G][16] float2 and the fragments of every slice
-    want = 256 + (4 * 128 + (4 + 1) * 8 * 1 * 32) + (2 * 128 + (2 + 2) * 8 * 4 * 32)
+    # workspace: status header + per layer the sums [G][16] float2 and the fragments of every slice; the set has a
+    # layer with more than one token, so every layer is staged eight tokens wide (absent tokens as zeros)
+    want = 256 + (4 * 128 + (4 + 1) * 8 * 8 * 32) + (2 * 128 + (2 + 2) * 8 * 8 * 32)
     assert wb == want
+    assert _set_bytes(slim, [(1, 256, 512, [2, 3, 1, 2])])[2] == 256 + (4 * 128 + (4 + 1) * 8 * 1 * 32)      # one token: as is
+    assert _set_bytes(slim, [(9, 256, 512, [2, 3, 1, 2])])[2] == 256 + (4 * 128 + (4 + 1) * 8 * 16 * 32)     # sixteen wide
     assert _set_bytes(slim, [])[0] == -1                                  # empty set
     assert _set_bytes(slim, [(0, 256, 512, [2] * 4)])[0] == -1            # no token
     assert _set_bytes(slim, [(17, 256, 512, [2] * 4)])[0] == -1           # the batched path serves these
