@@ -131,3 +131,31 @@ def test_rejects_bad_sets():
     x17 = torch.zeros(17, 256, dtype=torch.float16, device="cuda")
     with pytest.raises(slim.SlimError):
         slim.LayerSet([(dl, x17, torch.empty(17, 128, dtype=torch.float16, device="cuda"))])
+
+
+def test_llama7b_shapes_full_size_in_the_benchmark_configuration():
+    """Full-size LLaMA-7B layers (q, gate, down shapes) as one set that is larger than the persistent grid, so that
+    CTAs walk several items and cross layer boundaries as in the benchmark's sweep; the oracle computes sampled rows."""
+    slim = _slim()
+    shapes = [(4096, 4096), (11008, 4096), (4096, 11008)]
+    base = [oracle_layer(N, K, 2, 1, seed_name="set-full", block=i) for i, (N, K) in enumerate(shapes)]
+    dev = [_device_layer(L) for L in base]
+    entries, meta = [], []
+    rng = np.random.default_rng(2405)
+    for rep in range(12):
+        for L, dl in zip(base, dev):
+            x = rng.normal(0, 1, (1, L["K"])).astype(np.float16)
+            y = torch.full((1, L["N"]), float("nan"), dtype=torch.float16, device="cuda")
+            entries.append((dl, torch.from_numpy(x).cuda(), y))
+            meta.append((L, x))
+    s = slim.LayerSet(entries)
+    assert s.info["n_items"] > 2 * s.info["grid"]
+    s.run()
+    s.check()
+    for k, ((L, x), (_, _, y)) in enumerate(zip(meta, entries)):
+        y = y.cpu().numpy()
+        assert np.isfinite(y.astype(np.float64)).all(), f"entry {k}"
+        N = L["N"]
+        rows = np.unique(np.concatenate([[0, 1, 15, 16, 255, 256, N - 1], rng.integers(0, N, 120)]))
+        y_ref = orc.linear_rows_f64(x, L["codes"], L["scales"], L["zeros"], rows)
+        check_output(y[:, rows], y_ref, f"entry {k}: {N}x{L['K']}")
