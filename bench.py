@@ -49,6 +49,13 @@ NCU_TRAFFIC = {
 }
 
 
+# DRAM bytes (read + written) of the 14 gemm_kernel launches of one step of llama13b-prefill-avg3-m2048, from one ncu
+# capture of dram__bytes_read.sum and dram__bytes_write.sum; keyed by the SHA-256 of slim_gemm.cu at capture time
+NCU_TRAFFIC_GEMM = {
+    "1a98f6bdbcf5c7c1c57790e2a1ed836e1474feb538dcafefdc70f951cd97623b": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1119355392 + 232290560},
+}
+
+
 def workload_spec(name: str):
     if name == "llama7b-decode-avg2":
         return dict(model="llama-7b", avg_bits=2, M=1, n_blocks=wl.N_BLOCKS["llama-7b"])
@@ -404,6 +411,9 @@ def finish_gemm_line(args, spec, layers, world, steps, warmup, ms, e2e_steps, ms
     n_launch = len(layers)
     per_launch_us = 1e3 * ms / steps / n_launch
     achieved = flops / n_launch / (per_launch_us * 1e-6) / 1e12
+    sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2405_14917_b200", "csrc", "slim_gemm.cu"), "rb").read()).hexdigest()
+    cap = NCU_TRAFFIC_GEMM.get(sha)
+    traffic = cap["traffic_bytes"] / cap["launches"] if cap and cap["workload"] == args.workload and cap["launches"] == n_launch else None
     line = {
         "metric": f"mixed-precision dequant GEMM TFLOP/s at M={M} (LLaMA-13B layer shapes, avg 3-bit, g=128)",
         "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warmup,
@@ -414,7 +424,7 @@ def finish_gemm_line(args, spec, layers, world, steps, warmup, ms, e2e_steps, ms
                    "launch": "CUDA graph of one launch per layer", "parallelism": f"replicas x{world}"},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_kind": peak_kind, "kernel": "gemm_kernel", "avg_launch_us": per_launch_us,
-                     "flops_per_launch": flops / n_launch, "traffic": None, "frac_of_nominal_2250": achieved / 2250.0},
+                     "flops_per_launch": flops / n_launch, "traffic": traffic, "frac_of_nominal_2250": achieved / 2250.0},
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": int(x_host.numel() * 2),
                 "d2h_bytes_per_step": int(y_host.numel() * 2), "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
         "gpu_launches": steps * n_launch,
