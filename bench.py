@@ -306,20 +306,21 @@ def run_sba(args):
     e2e_steps = max(steps // 2, 3)
     ms_e2e = timed(step_e2e, e2e_steps)
     value = candidates * steps / (ms * 1e-3)
-    # dominant kernel: quantize_minmax_kernel, once per candidate: reads W (2 B per weight), writes codes (1 B)
-    # and scales, zeros (4 B per 128 weights); charged with the whole step (packing, layer call, KL included)
-    bytes_q = weight_visits * (3 + 4 / 128)
-    achieved = bytes_q * steps / (ms * 1e-3) / 1e9
-    peak, peak_kind = measured_hbm_peak()
+    # dominant kernel (31 % of the device time in the ncu launch list): gemm_kernel<128>, the hot path evaluating a
+    # candidate on the 128 calibration tokens, 2 M N K FLOPs each; charged with the whole step (quantizer, packing,
+    # KL and the host loop included)
+    flops = 2.0 * M * weight_visits
+    achieved = flops * steps / (ms * 1e-3) / 1e12
+    peak, peak_kind = measured_tensor_peak()
     line = {"metric": "SBA search: candidate bit maps evaluated per second (LLaMA-7B block, avg 2-bit, 128 tokens)",
             "value": value, "unit": "candidates/s", "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": ms / steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64 quantizer and KL, f16 tensor-core layer calls", "data": "synthetic",
             "config": {"workload": args.workload, "layers": len(layers), "candidates_per_step": candidates, "tokens": M,
                        "l2": "404 MB of fp16 weights per step > L2"},
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_kind": peak_kind, "kernel": "quantize_minmax_kernel",
-                         "avg_launch_us": 1e3 * ms / steps / candidates, "algorithmic_bytes_per_launch": bytes_q / candidates,
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                         "peak_kind": peak_kind, "kernel": "gemm_kernel",
+                         "avg_launch_us": 1e3 * ms / steps / candidates, "flops_per_launch": flops / candidates,
                          "traffic": None},
             "e2e": {"value": candidates * e2e_steps / (ms_e2e * 1e-3), "unit": "candidates/s",
                     "h2d_bytes_per_step": int(sum(2 * W.numel() + 2 * x.numel() for W, x, *_ in layers)),

@@ -232,6 +232,12 @@ int slim_allocate_bits(const double* salience_host, int G, int avg_bits, int p, 
 int slim_quantize_minmax(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
                          int N, int K, int g, void* stream);
 
+/* slim_quantize_minmax restricted to the groups listed in groups_host[n_groups] (host, distinct
+ * indices): only their columns of `codes` and their rows of `scales` and `zeros` are written,
+ * under bits_host.  Used by the SBA search, whose consecutive candidates differ in two groups. */
+int slim_quantize_minmax_groups(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
+                                int N, int K, int g, const int* groups_host, int n_groups, void* stream);
+
 /* slim_quantize_minmax with the binarisation of Eq. 2 for the one-bit groups: q = [w >= 0]
  * (sign(0) = +1), alpha = mean |w| of the (row, group), stored as s = fp16(2 alpha), z = 1/2, so
  * that s (q - z) = +-alpha.  Groups of two or more bits use Eq. 1 as above.  Same layouts. */
@@ -253,7 +259,7 @@ int slim_quantize_sqc(const void* W, const uint8_t* bits_host, uint8_t* codes, v
 /* ---- Salience-Determined Bit Allocation (func SBA of Algorithm 2, Sec. 3.2.2, Eq. 4) --------- */
 
 /* y = x * W^T in full precision: x fp16 [M][K], W fp16 [N][K], y fp32 [M][N] (device), fp32
- * accumulation in k order.  The reference output "x w_f^T" of Eq. 4.  K a multiple of 32. */
+ * accumulation (tensor cores).  The reference output "x w_f^T" of Eq. 4.  K a multiple of 32. */
 int slim_dense_linear(const void* x, const void* W, float* y, int M, int N, int K, void* stream);
 
 /* kl[t] = D_kl( softmax(y_ref[t]) || softmax(y_q[t]) ) for every token t (natural logarithm, softmax

@@ -59,6 +59,7 @@ def lib():
             "slim_allocate_bits": [vp, i, i, i, vp],
             "slim_quantize_minmax": [vp, vp, vp, vp, vp, i, i, i, vp],
             "slim_quantize_minmax_sign1": [vp, vp, vp, vp, vp, i, i, i, vp],
+            "slim_quantize_minmax_groups": [vp, vp, vp, vp, vp, i, i, i, vp, i, vp],
             "slim_gemv_set_bytes": [vp, i, i, ctypes.POINTER(sz), ctypes.POINTER(sz)],
             "slim_gemv_set_plan": [vp, i, i, vp, sz, vp, vp],
             "slim_mpq_gemv_set": [vp, vp, vp, sz, vp],
@@ -236,6 +237,16 @@ def quantize_minmax(W: torch.Tensor, bits, one_bit: str = "minmax"):
                                             _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
                                             N, K, GROUP, _stream(W)))
     return codes, scales, zeros
+
+
+def quantize_minmax_groups(W: torch.Tensor, bits, groups, codes: torch.Tensor, scales: torch.Tensor, zeros: torch.Tensor) -> None:
+    """Re-quantises (Eq. 1) only the listed groups under `bits`, in place in codes / scales / zeros."""
+    b = _bits(bits)
+    gl = np.ascontiguousarray(np.asarray(groups), dtype=np.int32)
+    N, K = W.shape
+    _check("slim_quantize_minmax_groups", lib().slim_quantize_minmax_groups(
+        _dev(W, torch.float16, "W"), _bp(b), _dev(codes, torch.uint8, "codes"), _dev(scales, torch.float16, "scales"),
+        _dev(zeros, torch.float16, "zeros"), N, K, GROUP, gl.ctypes.data, int(gl.size), _stream(W)))
 
 
 def quantize_sqc(W: torch.Tensor, bits, lam: float = 0.1, n: int = 50):

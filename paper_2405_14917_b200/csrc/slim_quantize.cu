@@ -3,30 +3,51 @@
 // order, so the outputs are reproducible bit for bit.
 #include "slim_common.cuh"
 
+#include <cstring>
+
 namespace slim {
 
-// One block per group.  Thread (ph, cp) owns column pair cp (2 columns) and rows ph, ph+4, ...
+// One cluster of kSalCluster blocks per group; block r of the cluster owns the r-th slice of the
+// rows.  Thread (ph, cp) owns column pair cp (2 columns) and rows ph, ph+4, ... of the slice.
 // Column sums of squares are accumulated in fp64 in ascending row order per phase, the four
-// phases are added in order, then the 128 columns are weighted by a_k^2 and summed in order.
-__global__ void __launch_bounds__(256) salience_kernel(const __half* __restrict__ W, const float* __restrict__ act_norm,
-                                                       double* __restrict__ salience, int N, int K) {
-    const int j = blockIdx.x;
+// phases are added in order, the blocks' sums are added in rank order by block 0 (which receives
+// them through distributed shared memory), then the 128 columns are weighted by a_k^2 and summed
+// in order: a fixed order, so the result is reproducible.
+constexpr int kSalCluster = 8;
+
+__global__ void __cluster_dims__(kSalCluster, 1, 1) __launch_bounds__(256)
+salience_kernel(const __half* __restrict__ W, const float* __restrict__ act_norm, double* __restrict__ salience, int N, int K) {
+    const int j = blockIdx.x / kSalCluster, r = blockIdx.x % kSalCluster;     // group, rank in the cluster
     const int cp = threadIdx.x & 63, ph = threadIdx.x >> 6;
+    const int rows = (N + kSalCluster - 1) / kSalCluster;
+    const int n0 = r * rows, n1 = min(N, n0 + rows);
     const __half2* base = reinterpret_cast<const __half2*>(W + static_cast<size_t>(SLIM_GROUP) * j) + cp;
     double s0 = 0.0, s1 = 0.0;
-    for (int n = ph; n < N; n += 4) {
+    for (int n = n0 + ph; n < n1; n += 4) {
         const float2 v = __half22float2(base[static_cast<size_t>(n) * (K / 2)]);
         s0 += static_cast<double>(v.x) * static_cast<double>(v.x);
         s1 += static_cast<double>(v.y) * static_cast<double>(v.y);
     }
     __shared__ double part[4][SLIM_GROUP];
+    __shared__ double from_rank[kSalCluster][SLIM_GROUP];        // used in block 0 of the cluster
     part[ph][2 * cp] = s0;
     part[ph][2 * cp + 1] = s1;
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (threadIdx.x < SLIM_GROUP) {
+        const int k = threadIdx.x;
+        const double col = ((part[0][k] + part[1][k]) + part[2][k]) + part[3][k];
+        // hand the slice's column sum to block 0
+        uint32_t remote;
+        const uint32_t local = static_cast<uint32_t>(__cvta_generic_to_shared(&from_rank[r][k]));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(0));
+        asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(remote), "d"(col) : "memory");
+    }
+    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    if (r == 0 && threadIdx.x == 0) {
         double total = 0.0;
         for (int k = 0; k < SLIM_GROUP; ++k) {
-            const double col = ((part[0][k] + part[1][k]) + part[2][k]) + part[3][k];
+            double col = 0.0;
+            for (int q = 0; q < kSalCluster; ++q) col += from_rank[q][k];
             const double a = static_cast<double>(act_norm[SLIM_GROUP * j + k]);
             total += a * a * col;
         }
@@ -40,17 +61,39 @@ __device__ __forceinline__ unsigned short double_to_half_bits_rn(double v) {
     return h;
 }
 
+// Groups a launch of the quantizer is restricted to (n = 0: all groups).
+struct GroupSubset {
+    int n;
+    uint8_t idx[SLIM_MAX_GROUPS];
+};
+
+// rint(w / s) for fp16-exact w and s > 0 without a division per weight: t = w * (1/s) is within a few
+// ulps of the quotient, and the quotient of two fp16 numbers that is not exactly half-way between
+// two integers stays farther than 2^-13 from it (its denominator has at most 11 bits; |w/s| < 2^6
+// here), so rint(t) is rint(w/s) unless t sits within 1e-6 of a half-integer, which can only be an
+// exact tie and goes to the even neighbour as rint does.
+__device__ __forceinline__ double rint_quotient(double w, double inv_s) {
+    const double t = w * inv_s;
+    const double k = rint(t);
+    if (fabs(fabs(t - k) - 0.5) < 1e-6) {
+        const double m = rint(t - 0.5);                   // the integer below the tie
+        return fmod(m, 2.0) == 0.0 ? m : m + 1.0;
+    }
+    return k;
+}
+
 // One warp per (row, group): lane l owns columns 4l..4l+3 of the group.  With sign_alpha != 0 the
 // one-bit groups are binarised as in Eq. 2 (q = [w >= 0], alpha = mean |w|, stored as s = 2 alpha,
 // z = 1/2 so that s (q - z) = +-alpha); all other groups, and all groups otherwise, use Eq. 1.
 __global__ void __launch_bounds__(256) quantize_minmax_kernel(const __half* __restrict__ W, uint8_t* __restrict__ codes,
                                                               __half* __restrict__ scales, __half* __restrict__ zeros,
-                                                              int N, int K, int sign_alpha, GroupTable gt) {
+                                                              int N, int K, int sign_alpha, GroupSubset sub, GroupTable gt) {
     const long long warp = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    const int G = gt.G;
+    const int G = sub.n > 0 ? sub.n : gt.G;              // groups this launch quantises
     if (warp >= static_cast<long long>(N) * G) return;
-    const int n = static_cast<int>(warp / G), j = static_cast<int>(warp % G);
+    const int n = static_cast<int>(warp / G);
+    const int j = sub.n > 0 ? sub.idx[warp % G] : static_cast<int>(warp % G);
     const size_t off = static_cast<size_t>(n) * K + SLIM_GROUP * j + 4 * lane;
     const uint2 raw = *reinterpret_cast<const uint2*>(W + off);
     const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
@@ -89,10 +132,11 @@ __global__ void __launch_bounds__(256) quantize_minmax_kernel(const __half* __re
     const __half s16 = __ushort_as_half(sbits);
     const double s = static_cast<double>(__half2float(s16));
     const double z = fmin(fmax(-rint(static_cast<double>(lo) / s), 0.0), levels);
+    const double inv_s = 1.0 / s;
     uint32_t out = 0;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const double q = fmin(fmax(rint(static_cast<double>(w[i]) / s) + z, 0.0), levels);
+        const double q = fmin(fmax(rint_quotient(static_cast<double>(w[i]), inv_s) + z, 0.0), levels);
         out |= static_cast<uint32_t>(static_cast<int>(q)) << (8 * i);
     }
     *reinterpret_cast<uint32_t*>(codes + off) = out;
@@ -112,14 +156,14 @@ int slim_group_salience(const void* W, const float* act_norm, double* salience, 
     if (K == 0) return SLIM_OK;
     if (W == nullptr || act_norm == nullptr || salience == nullptr) return SLIM_ERR_INVALID_ARG;
     if (!slim::aligned16(W) || !slim::aligned16(act_norm) || !slim::aligned16(salience)) return SLIM_ERR_ALIGNMENT;
-    slim::salience_kernel<<<K / SLIM_GROUP, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+    slim::salience_kernel<<<slim::kSalCluster * (K / SLIM_GROUP), 256, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const __half*>(W), act_norm, salience, N, K);
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;
 }
 
 static int quantize_minmax_impl(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
-                                int N, int K, int g, int sign_alpha, void* stream) {
+                                int N, int K, int g, int sign_alpha, const int* groups_host, int n_groups, void* stream) {
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;
@@ -127,10 +171,21 @@ static int quantize_minmax_impl(const void* W, const uint8_t* bits_host, uint8_t
     if (W == nullptr || codes == nullptr || scales == nullptr || zeros == nullptr) return SLIM_ERR_INVALID_ARG;
     if (!slim::aligned16(W) || !slim::aligned16(codes) || !slim::aligned16(scales) || !slim::aligned16(zeros))
         return SLIM_ERR_ALIGNMENT;
-    const long long warps = static_cast<long long>(N) * gt.G;
+    slim::GroupSubset sub;
+    memset(&sub, 0, sizeof sub);
+    if (groups_host != nullptr) {
+        if (n_groups < 0 || n_groups > gt.G) return SLIM_ERR_INVALID_ARG;
+        if (n_groups == 0) return SLIM_OK;
+        for (int i = 0; i < n_groups; ++i) {
+            if (groups_host[i] < 0 || groups_host[i] >= gt.G) return SLIM_ERR_INVALID_ARG;
+            sub.idx[i] = static_cast<uint8_t>(groups_host[i]);
+        }
+        sub.n = n_groups;
+    }
+    const long long warps = static_cast<long long>(N) * (sub.n > 0 ? sub.n : gt.G);
     const unsigned grid = static_cast<unsigned>((warps + 7) / 8);
     slim::quantize_minmax_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const __half*>(W), codes, static_cast<__half*>(scales), static_cast<__half*>(zeros), N, K, sign_alpha, gt);
+        static_cast<const __half*>(W), codes, static_cast<__half*>(scales), static_cast<__half*>(zeros), N, K, sign_alpha, sub, gt);
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;
 }
@@ -138,12 +193,18 @@ static int quantize_minmax_impl(const void* W, const uint8_t* bits_host, uint8_t
 
 int slim_quantize_minmax(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
                          int N, int K, int g, void* stream) {
-    return quantize_minmax_impl(W, bits_host, codes, scales, zeros, N, K, g, 0, stream);
+    return quantize_minmax_impl(W, bits_host, codes, scales, zeros, N, K, g, 0, nullptr, 0, stream);
+}
+
+int slim_quantize_minmax_groups(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
+                                int N, int K, int g, const int* groups_host, int n_groups, void* stream) {
+    if (groups_host == nullptr) return SLIM_ERR_INVALID_ARG;
+    return quantize_minmax_impl(W, bits_host, codes, scales, zeros, N, K, g, 0, groups_host, n_groups, stream);
 }
 
 int slim_quantize_minmax_sign1(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
                                int N, int K, int g, void* stream) {
-    return quantize_minmax_impl(W, bits_host, codes, scales, zeros, N, K, g, 1, stream);
+    return quantize_minmax_impl(W, bits_host, codes, scales, zeros, N, K, g, 1, nullptr, 0, stream);
 }
 
 }  // extern "C"

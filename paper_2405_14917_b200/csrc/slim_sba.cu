@@ -5,8 +5,9 @@
 // the KL divergence between softmax(x w^T) and softmax(x w-hat^T), averaged over the calibration
 // tokens; the first p with the smallest error wins.  Every step runs in this library's kernels:
 //   salience            slim_group_salience            (first step of func SBA)
-//   x w^T               dense_linear_kernel            (fp16 in, fp32 accumulate and out; once)
-//   quantise, pack      slim_quantize_minmax, slim_pack_weights
+//   x w^T               dense_linear_kernel            (fp16 in, fp32 accumulate on mma.sync, fp32 out; once)
+//   quantise, pack      slim_quantize_minmax (first candidate), slim_quantize_minmax_groups (the two groups
+//                       that change from one candidate to the next), slim_pack_weights
 //   x w-hat^T           slim_mpq_gemv / slim_mpq_gemm  (the hot path itself evaluates the candidate)
 //   error               softmax_kl_kernel              (fp64, fixed reduction order)
 // The host only ranks the G saliences, loops over p and takes the minimum of G/2 + 1 numbers.
@@ -17,57 +18,54 @@
 namespace slim {
 
 // ------------------------------------------------------------------------------------------ x w^T, full precision
-// y[m][n] = sum_k x[m][k] * W[n][k], fp32 accumulation in k order.  64 tokens x 64 rows per block,
-// 16 x 16 threads, 4 x 4 outputs per thread, k in steps of 32 through shared memory.
+// y[m][n] = sum_k x[m][k] * W[n][k]: fp16 operands, fp32 accumulation on the tensor cores
+// (mma.sync m16n8k16; it runs once per layer).  A block of four warps takes 64 tokens x 64 rows, warp w
+// the tokens 16w .. 16w+15; operand fragments are read straight from global memory (x and W are
+// both k-contiguous, which is what the row x column fragment layouts want).
 constexpr int kDenseTile = 64;
-constexpr int kDenseK = 32;
+constexpr int kDenseK = 32;      // K must be a multiple of this
 
-__global__ void __launch_bounds__(256) dense_linear_kernel(const __half* __restrict__ x, const __half* __restrict__ W,
+__global__ void __launch_bounds__(128) dense_linear_kernel(const __half* __restrict__ x, const __half* __restrict__ W,
                                                            float* __restrict__ y, int M, int N, int K) {
-    __shared__ float xs[kDenseK][kDenseTile + 1];
-    __shared__ float ws[kDenseK][kDenseTile + 1];
-    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-    const int m0 = blockIdx.y * kDenseTile, n0 = blockIdx.x * kDenseTile;
-    float acc[4][4];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int gq = lane >> 2, c = lane & 3;
+    const int m0 = blockIdx.y * kDenseTile + 16 * warp, n0 = blockIdx.x * kDenseTile;
+    // rows past the ends are clamped for the loads and masked at the store
+    const int ma = min(m0 + gq, M - 1), mb = min(m0 + gq + 8, M - 1);
+    const uint32_t* xa = reinterpret_cast<const uint32_t*>(x + static_cast<size_t>(ma) * K) + c;
+    const uint32_t* xb = reinterpret_cast<const uint32_t*>(x + static_cast<size_t>(mb) * K) + c;
+    const uint32_t* wr[8];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int t = 0; t < 8; ++t) wr[t] = reinterpret_cast<const uint32_t*>(W + static_cast<size_t>(min(n0 + 8 * t + gq, N - 1)) * K) + c;
+    float acc[8][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-    for (int k0 = 0; k0 < K; k0 += kDenseK) {
-        // 64 x 32 halves of each operand: 256 threads x 8 halves
-        const int r = threadIdx.x >> 2, c8 = (threadIdx.x & 3) * 8;
-        {
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (m0 + r < M) v = *reinterpret_cast<const uint4*>(x + static_cast<size_t>(m0 + r) * K + k0 + c8);
-            const __half* h = reinterpret_cast<const __half*>(&v);
+    for (int t = 0; t < 8; ++t)
 #pragma unroll
-            for (int i = 0; i < 8; ++i) xs[c8 + i][r] = __half2float(h[i]);
-            uint4 u = make_uint4(0u, 0u, 0u, 0u);
-            if (n0 + r < N) u = *reinterpret_cast<const uint4*>(W + static_cast<size_t>(n0 + r) * K + k0 + c8);
-            const __half* g = reinterpret_cast<const __half*>(&u);
+        for (int r = 0; r < 4; ++r) acc[t][r] = 0.f;
+    for (int k0 = 0; k0 < K; k0 += 16) {
+        const int o = k0 >> 1;                             // in 32-bit words
+        const uint32_t a0 = __ldg(xa + o), a1 = __ldg(xb + o), a2 = __ldg(xa + o + 4), a3 = __ldg(xb + o + 4);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) ws[c8 + i][r] = __half2float(g[i]);
+        for (int t = 0; t < 8; ++t) {
+            const uint32_t b0 = __ldg(wr[t] + o), b1 = __ldg(wr[t] + o + 4);
+            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                         : "+f"(acc[t][0]), "+f"(acc[t][1]), "+f"(acc[t][2]), "+f"(acc[t][3])
+                         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
         }
-        __syncthreads();
-#pragma unroll
-        for (int kk = 0; kk < kDenseK; ++kk) {
-            float a[4], b[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { a[i] = xs[kk][ty + 16 * i]; b[i] = ws[kk][tx + 16 * i]; }
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
-        }
-        __syncthreads();
     }
+    // D fragment: rows (tokens) gq and gq + 8, columns (weight rows) 2c and 2c + 1 of each 8-wide tile
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int t = 0; t < 8; ++t) {
+        const int n = n0 + 8 * t + 2 * c;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int m = m0 + ty + 16 * i, n = n0 + tx + 16 * j;
-            if (m < M && n < N) y[static_cast<size_t>(m) * N + n] = acc[i][j];
+        for (int h = 0; h < 2; ++h) {
+            const int m = m0 + gq + 8 * h;
+            if (m < M) {
+                if (n < N) y[static_cast<size_t>(m) * N + n] = acc[t][2 * h];
+                if (n + 1 < N) y[static_cast<size_t>(m) * N + n + 1] = acc[t][2 * h + 1];
+            }
         }
+    }
 }
 
 // ------------------------------------------------------------------------------------------ softmax + KL
@@ -172,7 +170,7 @@ int slim_dense_linear(const void* x, const void* W, float* y, int M, int N, int 
     if (!slim::aligned16(x) || !slim::aligned16(W) || !slim::aligned16(y)) return SLIM_ERR_ALIGNMENT;
     if (K % slim::kDenseK != 0) return SLIM_ERR_UNSUPPORTED;
     const dim3 grid((N + slim::kDenseTile - 1) / slim::kDenseTile, (M + slim::kDenseTile - 1) / slim::kDenseTile);
-    slim::dense_linear_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+    slim::dense_linear_kernel<<<grid, 128, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const __half*>(x), static_cast<const __half*>(W), y, M, N, K);
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;
@@ -225,12 +223,22 @@ int slim_sba_search(const void* W, const void* x, const float* act_norm, int M, 
     void* packed = ws + lay.packed;
     void* y_q = ws + lay.y_q;
     double* kl = reinterpret_cast<double*>(ws + lay.kl);
-    uint8_t bits[SLIM_MAX_GROUPS];
+    uint8_t bits[SLIM_MAX_GROUPS], prev[SLIM_MAX_GROUPS];
     for (int p = first; p <= G / 2; ++p) {
         st = slim_allocate_bits(sal, G, avg_bits, p, bits);
         if (st != SLIM_OK) return st;
-        st = slim_quantize_minmax(W, bits, codes, scales, zeros, N, K, g, stream);
+        if (p == first) {
+            st = slim_quantize_minmax(W, bits, codes, scales, zeros, N, K, g, stream);
+        } else {
+            // consecutive candidates differ in the two groups the double pointer has just passed: only those
+            // are quantised again, the codes, scales and zeros of all other groups stay
+            int changed[SLIM_MAX_GROUPS], n_changed = 0;
+            for (int j = 0; j < G; ++j)
+                if (bits[j] != prev[j]) changed[n_changed++] = j;
+            st = slim_quantize_minmax_groups(W, bits, codes, scales, zeros, N, K, g, changed, n_changed, stream);
+        }
         if (st != SLIM_OK) return st;
+        memcpy(prev, bits, sizeof prev);
         st = slim_pack_weights(codes, bits, packed, N, K, g, stream);
         if (st != SLIM_OK) return st;
         st = M <= SLIM_GEMV_MAX_M

@@ -137,3 +137,48 @@ def test_eq2_one_bit_groups_end_to_end(N, K, M):
         s.run()
         s.check()
         check_output(y.cpu().numpy(), y_ref, f"Eq. 2 groups, layer set, M={M}")
+
+
+@pytest.mark.parametrize("b", [1, 2, 3, 4])
+def test_quantizer_exact_ties_round_to_even(b):
+    """Weights exactly half-way between two grid points (w / s = k + 1/2): both sides must round to the even code."""
+    slim = _slim()
+    levels = 2 ** b - 1
+    s = 2.0 ** -6
+    rng = np.random.default_rng(b)
+    W = np.empty((32, 256), dtype=np.float16)
+    for n in range(32):
+        for j in range(2):
+            k = rng.integers(0, levels, 128)
+            w = (k + 0.5) * s                      # exact ties
+            w[0], w[1] = 0.0, levels * s           # the group's range is exactly [0, levels * s]: scale s, zero point 0
+            if n % 2:                              # every other row mirrored: negative range, zero point = levels
+                w = -w
+            W[n, 128 * j:128 * j + 128] = w
+    bits = np.array([b, b], dtype=np.uint8)
+    c_ref, s_ref, z_ref = orc.quantize_minmax(W, bits)
+    assert (s_ref.astype(np.float64) == s).all()
+    codes, scales, zeros = slim.quantize_minmax(torch.from_numpy(W).cuda(), bits)
+    assert (codes.cpu().numpy() == c_ref).all()
+    assert (scales.cpu().numpy().view(np.uint16) == s_ref.view(np.uint16)).all()
+    assert (zeros.cpu().numpy().view(np.uint16) == z_ref.view(np.uint16)).all()
+    # ties really occurred and went both ways
+    k_plus = (c_ref[0::2, 2:128].astype(np.int64) - np.floor(W[0::2, 2:128].astype(np.float64) / s)).ravel()
+    assert set(np.unique(k_plus)) <= {0, 1} and (len(set(np.unique(k_plus))) == 2 or b == 1)
+
+
+def test_requantising_a_subset_of_groups():
+    slim = _slim()
+    seed = wl.layer_seed("test", "quant-subset", 0)
+    W = wl.make_weight(seed, 272, 1024)
+    bits_a = np.array([2, 2, 2, 2, 2, 2, 2, 2], dtype=np.uint8)
+    bits_b = np.array([2, 3, 2, 2, 1, 2, 2, 4], dtype=np.uint8)
+    Wd = torch.from_numpy(W).cuda()
+    codes, scales, zeros = slim.quantize_minmax(Wd, bits_a)
+    slim.quantize_minmax_groups(Wd, bits_b, [7, 1, 4], codes, scales, zeros)
+    c_ref, s_ref, z_ref = orc.quantize_minmax(W, bits_b)       # groups 0, 2, 3, 5, 6 have the same width in both maps
+    assert (codes.cpu().numpy() == c_ref).all()
+    assert (scales.cpu().numpy().view(np.uint16) == s_ref.view(np.uint16)).all()
+    assert (zeros.cpu().numpy().view(np.uint16) == z_ref.view(np.uint16)).all()
+    with pytest.raises(slim.SlimError):
+        slim.quantize_minmax_groups(Wd, bits_b, [8], codes, scales, zeros)
