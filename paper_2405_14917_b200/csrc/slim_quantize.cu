@@ -287,11 +287,12 @@ __global__ void __launch_bounds__(kSqcWarps * 32) quantize_sqc_kernel(const __ha
     for (int i = lane; i < 2 * n_half; i += 32) {
         double s, z;
         (void)candidate(i, &s, &z);
+        const double inv_s = __ddiv_rn(1.0, s);           // |w / s| < 2^6 here too: see rint_quotient
         double Ls = 0.0, Lus = 0.0;
 #pragma unroll 2
         for (int k = 0; k < SLIM_GROUP; ++k) {
             const double wk = w[k];
-            const double q = fmin(fmax(__dadd_rn(rint(__ddiv_rn(wk, s)), z), 0.0), levels);
+            const double q = fmin(fmax(__dadd_rn(rint_quotient(wk, inv_s), z), 0.0), levels);
             const double e = __dsub_rn(wk, __dmul_rn(s, __dsub_rn(q, z)));
             const double sq = __dmul_rn(e, e);
             if (wk < t_lo || wk > t_hi) Ls = __dadd_rn(Ls, sq);
