@@ -159,3 +159,16 @@ def test_llama7b_shapes_full_size_in_the_benchmark_configuration():
         rows = np.unique(np.concatenate([[0, 1, 15, 16, 255, 256, N - 1], rng.integers(0, N, 120)]))
         y_ref = orc.linear_rows_f64(x, L["codes"], L["scales"], L["zeros"], rows)
         check_output(y[:, rows], y_ref, f"entry {k}: {N}x{L['K']}")
+
+
+def test_projections_that_share_one_input():
+    """q/k/v (and gate/up) of a block read the same activations: one set, one x tensor, three outputs."""
+    slim = _slim()
+    layers = [oracle_layer(384, 1024, 2, 2, seed_name="qkv", block=i) for i in range(3)]
+    x = torch.from_numpy(layers[0]["x"]).cuda()
+    entries = [(_device_layer(L), x, torch.empty(2, L["N"], dtype=torch.float16, device="cuda")) for L in layers]
+    s = slim.LayerSet(entries)
+    s.run()
+    s.check()
+    for L, (_, _, y) in zip(layers, entries):
+        check_output(y.cpu().numpy(), orc.linear_f64(layers[0]["x"], L["codes"], L["scales"], L["zeros"]), "shared x")
