@@ -40,9 +40,9 @@ FALLBACK_TENSOR_TFLOPS = 1400.0
 # dram__bytes_write.sum), keyed by the sha256 of the kernel source it was taken from.  A kernel
 # that has changed since reports null.
 NCU_TRAFFIC = {
-    # layer-set kernel, 4 blocks of the LLaMA-7B sweep (28 layers, avg 2-bit, M = 1): 228,475,392 B read +
-    # 5,545,472 B written per launch (algorithmic 228,297,816 B); scaled to the full sweep by the algorithmic bytes
-    "60b0f951c2676dd366a15020647a8d61618ad76f40a44aafcdd58a6b5f4a3554": {"layer": "4 blocks", "traffic_bytes": 234020864, "algorithmic_bytes": 228297816},
+    # layer-set kernel, 4 blocks of the LLaMA-7B sweep (28 layers, avg 2-bit, M = 1): 228,399,872 B read +
+    # 4,327,168 B written per launch (algorithmic 228,297,816 B); scaled to the full sweep by the algorithmic bytes
+    "047677bdb5be842f2b2a425ac2d281ada8638985fce6431a29f25bc392b12ecb": {"layer": "4 blocks", "traffic_bytes": 232727040, "algorithmic_bytes": 228297816},
     # 4096x4096 layer, avg 2-bit, M = 1: 4,755,200 B read + 0 written per launch (algorithmic 4,735,008 B);
     # scaled to the sweep's average launch by the algorithmic bytes (traffic grows with the layer size)
     "4b06a5d5b512621bbe525cb3d0c66822ff452c130a671af895469c10fb834593": {"layer": "4096x4096", "traffic_bytes": 4755200, "algorithmic_bytes": 4735008},
