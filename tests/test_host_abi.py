@@ -140,3 +140,26 @@ def test_layer_set_sizes_and_argument_errors(slim):
     assert _set_bytes(slim, [(1, 256, 500, [2] * 4)])[0] == -2            # K not a multiple of 128
     assert _set_bytes(slim, [(1, 256, 0, [])])[0] == -1                   # empty reduction
     assert _set_bytes(slim, ok, g=64)[0] == -2                            # group size
+
+
+def test_sba_workspace_and_quantizer_argument_errors(slim):
+    L = slim.lib()
+    out = ctypes.c_size_t(0)
+    assert L.slim_sba_workspace_bytes(128, 4096, 4096, 128, 2, ctypes.byref(out)) == 0
+    # codes + scales + zeros + widest packed buffer + both outputs + one error per candidate and token, at least
+    G = 32
+    least = 4096 * 4096 + 2 * (G * 4096 * 2) + 4096 * 4096 * 3 // 8 + 128 * 4096 * (4 + 2) + (G // 2 + 1) * 128 * 8
+    assert least <= out.value <= least + 32 * 1024 * 1024
+    assert L.slim_sba_workspace_bytes(128, 4096, 4096, 128, 4, ctypes.byref(out)) == -1      # average bit-width
+    assert L.slim_sba_workspace_bytes(0, 4096, 4096, 128, 2, ctypes.byref(out)) == -1        # no calibration token
+    assert L.slim_sba_workspace_bytes(128, 4096, 4000, 128, 2, ctypes.byref(out)) == -2      # K not a multiple of 128
+    assert L.slim_sba_workspace_bytes(128, 4096, 4096, 64, 2, ctypes.byref(out)) == -2       # group size
+    assert L.slim_sba_workspace_bytes(128, 4096, 4096, 128, 2, None) == -1
+    # nothing is launched for null pointers
+    bits = np.array([2, 2], dtype=np.uint8)
+    groups = np.array([0], dtype=np.int32)
+    assert L.slim_quantize_minmax_groups(None, bits.ctypes.data, None, None, None, 16, 256, 128, groups.ctypes.data, 1, None) == -1
+    assert L.slim_quantize_minmax_sign1(None, bits.ctypes.data, None, None, None, 16, 256, 128, None) == -1
+    assert L.slim_dense_linear(None, None, None, 4, 16, 128, None) == -1
+    assert L.slim_dense_linear(None, None, None, 0, 16, 128, None) == 0
+    assert L.slim_softmax_kl(None, None, None, 4, 16, None) == -1
