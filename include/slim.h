@@ -199,10 +199,12 @@ typedef struct slim_gemv_set_info {
 int slim_gemv_set_bytes(const slim_layer* layers_host, int n_layers, int g,
                         size_t* plan_bytes, size_t* workspace_bytes);
 
-/* Validates the set, lays the work out over the device's SMs and writes the plan (layer
- * descriptors, item ranges of every CTA) into `plan` (device, 16-byte aligned, plan_bytes from
+/* Validates the set, deals the work items to the persistent CTAs (heaviest item first, each to the
+ * CTA with the least work so far, so the CTAs finish together) and writes the plan (layer
+ * descriptors, every CTA's list of items) into `plan` (device, 16-byte aligned, plan_bytes from
  * slim_gemv_set_bytes) with copies enqueued on `stream`; fills *info.  layers_host and the bit
- * maps are read during the call only.  The plan stays valid while the layers' pointers do. */
+ * maps are read during the call only.  The plan stays valid while the layers' pointers do.
+ * SLIM_ERR_UNSUPPORTED if the host-side lists of the deal cannot be allocated. */
 int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g,
                        void* plan, size_t plan_bytes, slim_gemv_set_info* info, void* stream);
 

@@ -4,8 +4,9 @@
 // leaves the memory system idle while kernels start, stage x and reduce.  Here the whole set is
 // one stream of work items for persistent CTAs:
 //
-//  * item = (layer, block of 128 rows = 8 tiles of 16), the full K of the layer.  The items of
-//    the set are cut into one contiguous range per CTA, balanced by packed bytes, on the host.
+//  * item = (layer, block of 128 or 256 rows = 8 tiles of 16 per consumer warp's share), the full K
+//    of the layer.  The host deals the items to the CTAs, heaviest first, each to the CTA with the
+//    least work so far, and writes every CTA's list into the plan.
 //  * x is put into B-fragment order once per layer by a small kernel (one warp per token and
 //    group; the routine slim_mpq_gemv uses) and kept in the workspace; every item re-reads its
 //    fragments from L2.
@@ -22,7 +23,13 @@
 // Every wait on an mbarrier is bounded and reports through the workspace status word.
 #include "slim_gemv_dev.cuh"
 
+#include <algorithm>
 #include <cstring>
+#include <exception>
+#include <functional>
+#include <queue>
+#include <utility>
+#include <vector>
 
 namespace slim {
 
@@ -45,7 +52,7 @@ struct SetLayer {
                            // (sum_k x, 2^(24-S)) float2[16], then the fragments [slice][8 mma][MP][4 lanes] x 8 B
     size_t pad0;
     int M, N, K, G;
-    int item0, n_items;    // this layer's items in the set's numbering
+    int pad1[2];
     int task0;             // first (token, group) staging task of the layer
     int MP;                // tokens in the staged layout: 1 if every layer of the set has one token, else 8 or 16
                            // for the whole set (absent tokens are staged as zeros, so the kernel reads without a test)
@@ -56,13 +63,25 @@ struct SetLayer {
 };
 static_assert(sizeof(SetLayer) % 16 == 0, "descriptors are copied and read in 16-byte pieces");
 
-// Plan buffer: int item_begin[grid + 1] (padded to kSetPlanHeader bytes), then the descriptors.
+// One work item as the CTAs read it: what a consumer warp needs is here, so that it never waits for
+// the layer's descriptor.
+struct SetItem {
+    int layer, rb;         // layer of the set, row block inside the layer
+    int N, G;
+    __half* y;
+    int M, pad;
+};
+static_assert(sizeof(SetItem) == 32, "items are read as two 16-byte pieces");
+
+// Plan buffer: int item_begin[grid + 1] (padded to kSetPlanHeader bytes), the descriptors, then the
+// items in the order the CTAs take them: CTA c owns entries item_begin[c] .. item_begin[c + 1].
 constexpr int kSetMaxGrid = 1023;
 constexpr size_t kSetPlanHeader = 4096;
 
 struct SetParams {
     const int* item_begin;
     const SetLayer* layers;
+    const SetItem* items;
     uint8_t* ws;                           // workspace: status word, then the layers' fragments and sums
     int n_layers, n_slots, slot_bytes;
     int off_s, off_z, off_e, off_x;        // offsets inside a slot (weights start at kSetHeader)
@@ -180,15 +199,6 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
 
     const int i0 = p.item_begin[blockIdx.x], i1 = p.item_begin[blockIdx.x + 1];
     if (i0 < i1) {
-        int l = 0;                                        // layer of item i0
-        {
-            int lo = 0, hi = p.n_layers - 1;
-            while (lo < hi) {
-                const int mid = (lo + hi + 1) >> 1;
-                if (p.layers[mid].item0 <= i0) lo = mid; else hi = mid - 1;
-            }
-            l = lo;
-        }
         if (warp >= kSetConsumers) {
             // -------------------------------------------------------------- producers
             // producer warp w takes the groups whose running number is w modulo the number of producers
@@ -201,8 +211,10 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
             uint32_t ph = 0;
             uint32_t cnt = 0;                             // running number of the group in this CTA's range
             bool ok = true;
+            int l = p.items[i0].layer, rb = p.items[i0].rb;
             for (int i = i0; i < i1 && ok; ++i) {
-                while (i >= p.layers[l].item0 + p.layers[l].n_items) ++l;
+                // the next item's place is fetched while this one's groups are issued
+                const int l_next = i + 1 < i1 ? p.items[i + 1].layer : 0, rb_next = i + 1 < i1 ? p.items[i + 1].rb : 0;
                 if (have != l) {
                     const uint4* src = reinterpret_cast<const uint4*>(p.layers + l);
                     uint4* dst = reinterpret_cast<uint4*>(desc);
@@ -210,7 +222,7 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                     __syncwarp();
                     have = l;
                 }
-                const int rb = i - D->item0, N = D->N, MP = D->MP, G = D->G;
+                const int N = D->N, MP = D->MP, G = D->G;
                 const int tiles_here = min(TPI, (N >> 4) - TPI * rb);
                 // lane 0 brings the slices, lanes 1 and 2 scales and zeros, lane 3 the staged activations
                 const uint8_t* base = lane == 0 ? D->packed
@@ -241,6 +253,8 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                     s += kSetProducers;
                     if (s >= p.n_slots) { s -= p.n_slots; ph ^= 1u; }
                 }
+                l = l_next;
+                rb = rb_next;
             }
             if (!ok && lane == 0) {
                 // leave no copy in flight: give what was issued a millisecond to land
@@ -253,10 +267,16 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
             int s = 0;                                    // ring position of the next group
             uint32_t ph = 0;
             bool ok = true;
+            const int4* items4 = reinterpret_cast<const int4*>(p.items);
+            int4 it_a = items4[2 * i0], it_b = items4[2 * i0 + 1];   // (layer, rb, N, G), (y, M, -)
             for (int i = i0; i < i1 && ok; ++i) {
-                while (i >= p.layers[l].item0 + p.layers[l].n_items) ++l;
-                const SetLayer& L = p.layers[l];
-                const int rb = i - L.item0, N = L.N, M = L.M, G = L.G;
+                const int rb = it_a.y, N = it_a.z, G = it_a.w, M = it_b.z;
+                __half* const ybase = reinterpret_cast<__half*>((static_cast<unsigned long long>(static_cast<uint32_t>(it_b.y)) << 32) |
+                                                                static_cast<uint32_t>(it_b.x));
+                if (i + 1 < i1) {                                     // the next item arrives during this one's groups
+                    it_a = items4[2 * i + 2];
+                    it_b = items4[2 * i + 3];
+                }
                 const int tile0 = TPI * rb + TPW * warp;                  // this warp's first tile of the layer
                 const int n_act = min(TPW, (N >> 4) - tile0);              // its tiles that exist (<= 0: none)
                 float acc[TPW][NT][4];
@@ -366,7 +386,7 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
 #pragma unroll
                     for (int t = 0; t < TPW; ++t) {
                         if (t >= n_act) break;
-                        __half* yrow = L.y + 16 * (tile0 + t) + 2 * gq;
+                        __half* yrow = ybase + 16 * (tile0 + t) + 2 * gq;
                         if (ONE) {
                             if (c == 0) *reinterpret_cast<__half2*>(yrow) = __floats2half2_rn(acc[t][0][0], acc[t][0][2]);
                         } else {
@@ -394,7 +414,6 @@ struct SetGeometry {
     int n_slots, grid, ctas_per_sm;
     size_t smem_bytes;
     long long n_items, n_tasks;
-    unsigned long long total_cost;     // packed + scale + zero bytes of the set
     size_t ws_bytes;
 };
 
@@ -405,8 +424,15 @@ static size_t layer_ws_bytes(int M, const GroupTable& gt) {
     for (int j = 0; j < gt.G; ++j) slots += gt.bits[j] == 3 ? 1 : 0;
     return align_to(static_cast<size_t>(gt.G) * 128 + static_cast<size_t>(slots) * 256 * M, 128);
 }
+// Work of an item for the deal.  The kernel is bound by the instructions it issues, so a (tile, group)
+// weighs what a consumer warp issues for it: about 70 / 73 / 120 / 80 instructions at 1 / 2 / 3 / 4 bits
+// (counted in the kernel's loops: one AND per operand register, one MMA per four, the fragment loads and
+// the fold).
 static unsigned long long item_cost(int tiles_here, const GroupTable& gt) {
-    return static_cast<unsigned long long>(tiles_here) * (256ull * gt.prefix[gt.G] + 64ull * gt.G);
+    static const unsigned kGroupWork[5] = {0, 70, 73, 120, 80};
+    unsigned long long w = 0;
+    for (int j = 0; j < gt.G; ++j) w += kGroupWork[gt.bits[j]];
+    return w * static_cast<unsigned long long>(tiles_here);
 }
 
 static int set_sm_count() {
@@ -436,10 +462,6 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
         const int items = ((L.N >> 4) + tpi - 1) / tpi;
         sg->n_items += items;
         sg->n_tasks += static_cast<long long>(sg->mpad) * gt.G;
-        for (int rb = 0; rb < items; ++rb) {
-            const int th = (L.N >> 4) - tpi * rb;
-            sg->total_cost += item_cost(th < tpi ? th : tpi, gt);
-        }
         sg->ws_bytes += layer_ws_bytes(sg->mpad, gt);
     }
     if (sg->n_items > 0x3fffffff || sg->n_tasks > 0x3fffffff) return SLIM_ERR_UNSUPPORTED;
@@ -469,7 +491,9 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     return SLIM_OK;
 }
 
-static size_t set_plan_bytes(int n_layers) { return kSetPlanHeader + static_cast<size_t>(n_layers) * sizeof(SetLayer); }
+static size_t set_plan_bytes(int n_layers, long long n_items) {
+    return kSetPlanHeader + static_cast<size_t>(n_layers) * sizeof(SetLayer) + static_cast<size_t>(n_items) * sizeof(SetItem);
+}
 
 template <int NT, bool ONE, int TPW>
 static cudaError_t launch_set(const SetParams& prm, int grid, size_t smem, cudaStream_t stream) {
@@ -495,7 +519,7 @@ int slim_gemv_set_bytes(const slim_layer* layers_host, int n_layers, int g, size
     slim::SetGeometry sg;
     const int st = slim::set_geometry(layers_host, n_layers, g, &sg);
     if (st != SLIM_OK) return st;
-    *plan_bytes = slim::set_plan_bytes(n_layers);
+    *plan_bytes = slim::set_plan_bytes(n_layers, sg.n_items);
     *workspace_bytes = sg.ws_bytes;
     return SLIM_OK;
 }
@@ -507,7 +531,7 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
     const int st = slim::set_geometry(layers_host, n_layers, g, &sg);
     if (st != SLIM_OK) return st;
     if (!slim::aligned16(plan)) return SLIM_ERR_ALIGNMENT;
-    if (plan_bytes < slim::set_plan_bytes(n_layers)) return SLIM_ERR_WORKSPACE;
+    if (plan_bytes < slim::set_plan_bytes(n_layers, sg.n_items)) return SLIM_ERR_WORKSPACE;
     for (int l = 0; l < n_layers; ++l) {
         const slim_layer& L = layers_host[l];
         if (L.x == nullptr || L.packed == nullptr || L.scales == nullptr || L.zeros == nullptr || L.y == nullptr)
@@ -519,15 +543,16 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t* plan_dev = static_cast<uint8_t*>(plan);
 
-    // Second pass: descriptors, and the first item of every CTA (equal shares of the set's bytes).
-    // The copies below read host memory that goes out of scope: pageable sources are staged
-    // before cudaMemcpyAsync returns.
+    try {                       // the host-side lists may fail to allocate: reported as a status
+    // Second pass: descriptors and items.  The copies below read host memory that goes out of scope:
+    // pageable sources are staged before cudaMemcpyAsync returns.
     static_assert((slim::kSetMaxGrid + 1) * sizeof(int) <= slim::kSetPlanHeader, "item ranges fit the plan header");
-    int item_begin[slim::kSetMaxGrid + 1];
-    int next_cta = 1;
-    item_begin[0] = 0;
-    unsigned long long cost = 0;
-    int item = 0, task = 0;
+    std::vector<slim::SetItem> items;
+    std::vector<unsigned long long> cost;
+    items.reserve(static_cast<size_t>(sg.n_items));
+    cost.reserve(static_cast<size_t>(sg.n_items));
+    const int tpi = slim::kSetConsumers * sg.tpw;
+    int task = 0;
     size_t ws_off = 256;
     for (int l = 0; l < n_layers; ++l) {
         const slim_layer& L = layers_host[l];
@@ -542,9 +567,6 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
         d.y = static_cast<__half*>(L.y);
         d.M = L.M; d.N = L.N; d.K = L.K; d.G = gt.G;
         d.MP = sg.mpad;
-        d.item0 = item;
-        const int tpi = slim::kSetConsumers * sg.tpw;
-        d.n_items = ((L.N >> 4) + tpi - 1) / tpi;
         d.task0 = task;
         d.x_off = ws_off;
         ws_off += slim::layer_ws_bytes(sg.mpad, gt);
@@ -555,17 +577,44 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
             d.pre3[j + 1] = static_cast<uint16_t>(d.pre3[j] + (j < gt.G && gt.bits[j] == 3 ? 1 : 0));
         SLIM_CUDA_TRY(cudaMemcpyAsync(plan_dev + slim::kSetPlanHeader + static_cast<size_t>(l) * sizeof d, &d, sizeof d,
                                       cudaMemcpyHostToDevice, s));
-        for (int rb = 0; rb < d.n_items; ++rb, ++item) {
-            // CTA c starts at the first item at which the bytes before it reach c/grid of the total
-            while (next_cta < sg.grid && cost * sg.grid >= sg.total_cost * static_cast<unsigned long long>(next_cta))
-                item_begin[next_cta++] = item;
+        const int n_rb = ((L.N >> 4) + tpi - 1) / tpi;
+        for (int rb = 0; rb < n_rb; ++rb) {
             const int th = (L.N >> 4) - tpi * rb;
-            cost += slim::item_cost(th < tpi ? th : tpi, gt);
+            slim::SetItem it;
+            memset(&it, 0, sizeof it);
+            it.layer = l; it.rb = rb; it.N = L.N; it.G = gt.G; it.y = d.y; it.M = L.M;
+            items.push_back(it);
+            cost.push_back(slim::item_cost(th < tpi ? th : tpi, gt));
         }
         task += sg.mpad * gt.G;
     }
-    while (next_cta <= sg.grid) item_begin[next_cta++] = item;
+    // The deal: items by falling cost (equal costs in the set's order), each to the CTA that has the
+    // least so far (the lowest-numbered of equals).  Within a CTA the heavy items come first.
+    const int n_items = static_cast<int>(items.size());
+    std::vector<int> by_cost(n_items);
+    for (int i = 0; i < n_items; ++i) by_cost[i] = i;
+    std::stable_sort(by_cost.begin(), by_cost.end(), [&](int a, int b) { return cost[a] > cost[b]; });
+    typedef std::pair<unsigned long long, int> Load;                 // (work so far, CTA)
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load> > least;
+    for (int c = 0; c < sg.grid; ++c) least.push(Load(0ull, c));
+    std::vector<int> owner(n_items), count(sg.grid + 1, 0);
+    for (int k = 0; k < n_items; ++k) {
+        Load top = least.top();
+        least.pop();
+        owner[by_cost[k]] = top.second;
+        ++count[top.second + 1];
+        least.push(Load(top.first + cost[by_cost[k]], top.second));
+    }
+    int item_begin[slim::kSetMaxGrid + 1];
+    item_begin[0] = 0;
+    for (int c = 0; c < sg.grid; ++c) item_begin[c + 1] = item_begin[c] + count[c + 1];
+    std::vector<slim::SetItem> dealt(n_items);
+    std::vector<int> fill(item_begin, item_begin + sg.grid);
+    for (int k = 0; k < n_items; ++k) dealt[fill[owner[by_cost[k]]]++] = items[by_cost[k]];
     SLIM_CUDA_TRY(cudaMemcpyAsync(plan_dev, item_begin, static_cast<size_t>(sg.grid + 1) * sizeof(int), cudaMemcpyHostToDevice, s));
+    SLIM_CUDA_TRY(cudaMemcpyAsync(plan_dev + slim::kSetPlanHeader + static_cast<size_t>(n_layers) * sizeof(slim::SetLayer), dealt.data(),
+                                  static_cast<size_t>(n_items) * sizeof(slim::SetItem), cudaMemcpyHostToDevice, s));
+    const int item = n_items;
 
     memset(info, 0, sizeof *info);
     info->n_layers = n_layers;
@@ -578,8 +627,11 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
     info->max_bits = sg.bmax;
     info->max_tokens = sg.mmax;
     info->tiles_per_warp = sg.tpw;
-    info->plan_bytes = slim::set_plan_bytes(n_layers);
+    info->plan_bytes = slim::set_plan_bytes(n_layers, n_items);
     info->workspace_bytes = sg.ws_bytes;
+    } catch (const std::exception&) {
+        return SLIM_ERR_UNSUPPORTED;
+    }
     return SLIM_OK;
 }
 
@@ -603,6 +655,7 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     memset(&prm, 0, sizeof prm);
     prm.item_begin = static_cast<const int*>(plan);
     prm.layers = reinterpret_cast<const slim::SetLayer*>(static_cast<const uint8_t*>(plan) + slim::kSetPlanHeader);
+    prm.items = reinterpret_cast<const slim::SetItem*>(prm.layers + info->n_layers);
     prm.ws = static_cast<uint8_t*>(workspace);
     prm.n_layers = info->n_layers;
     prm.n_slots = info->n_slots;

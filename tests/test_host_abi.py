@@ -123,7 +123,7 @@ def test_layer_set_sizes_and_argument_errors(slim):
     ok = [(1, 256, 512, [2, 3, 1, 2]), (4, 144, 256, [3, 3])]
     st, pb, wb = _set_bytes(slim, ok)
     assert st == 0
-    # plan: item ranges of the CTAs, then one descriptor per layer; it grows by a fixed step per layer
+    # plan: item ranges of the CTAs, one descriptor per layer, one entry per work item
     st2, pb2, _ = _set_bytes(slim, ok + [(1, 128, 128, [2])])
     assert st2 == 0 and pb2 > pb and (pb2 - pb) % 16 == 0
     # workspace: status header + per layer the sums [G][16] float2 and the fragments of every slice; the set has a
