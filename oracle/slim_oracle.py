@@ -15,7 +15,8 @@ says otherwise.
 Pinned (tests/test_oracle_*.py): bit budget, quantizer closed forms and brute
 force, packing positions, dequantisation single-rounding, linear layer special
 cases, the SQC line search (brute force, never worse than tau = 1, exact grids), the SBA search
-(library KL, shift invariance, constructed optima, budget).  Parity unpinned: nothing in this file (the paper's perplexity / accuracy
+(library KL, shift invariance, constructed optima, budget), the GPTQ loop (column-by-column
+elimination, constrained least squares, H = I, proxy loss).  Parity unpinned: nothing in this file (the paper's perplexity / accuracy
 / token-per-second tables are not reproduced at all).
 """
 from __future__ import annotations
@@ -400,6 +401,76 @@ def sba_search(W16: np.ndarray, x16: np.ndarray, act_norm: np.ndarray, avg_bits:
             best = i
     p_star = first + best
     return p_star, allocate_bits(S, avg_bits, p_star), errors
+
+
+# --------------------------------------------------------------------------- GPTQ error compensation
+def gptq_hessian(x16: np.ndarray) -> np.ndarray:
+    """H = (1/P) sum_k x_k x_k^T over the P calibration tokens (Algorithm 1, first step), fp64 [K][K]."""
+    x = x16.astype(np.float64)
+    return x.T @ x / x.shape[0]
+
+
+def gptq_factor(H: np.ndarray, lam: float = 0.01):
+    """H_in = Cholesky((H + lambda I)^-1) (Algorithm 1, second step): the upper-triangular U with
+    U^T U = (H + lambda I)^-1.  Returns (U, dead).
+
+    Readings: lambda is relative to the mean diagonal of H (lambda_abs = lam * mean(diag H), the
+    convention of the GPTQ backbone the paper builds on), so the scale of H (the 1/P) does not matter;
+    an input channel that is zero in every token (`dead`) gets H_kk = 1 before damping and its weight
+    column is treated as zero by the caller.
+    """
+    import scipy.linalg
+    H = H.copy()
+    dead = np.diag(H) == 0
+    H[dead, dead] = 1.0
+    K = H.shape[0]
+    Hd = H + lam * np.mean(np.diag(H)) * np.eye(K)
+    U = scipy.linalg.cholesky(np.linalg.inv(Hd), lower=False)
+    return U, dead
+
+
+def gptq_quantize(W16: np.ndarray, x16: np.ndarray, bits, lam: float = 0.01, quantizer: str = "sqc", g: int = GROUP):
+    """Main loop of Algorithm 1 with a given bit map: group by group, quantise the CURRENT weights of
+    the group with SQC (or plain Eq. 1), then push the group's error onto the columns not yet
+    quantised:  E = (w_b - w-hat_b) / H_in[b, b]  (right division by the diagonal block),
+                w[:, after] -= E @ H_in[b, after].
+
+    Readings: the running weights are kept in fp64; the quantizer is given the group rounded to fp16
+    (its input type: the paper's weights are FP16) and returns fp16 scale and zero point, and the
+    error is taken against the exact s (q - z).  Returns (codes, scales, zeros, w_running) with the
+    layouts of quantize_minmax; w_running is the fp64 matrix after the last update.
+    """
+    bits = np.asarray(bits)
+    N, K = W16.shape
+    G = K // g
+    U, dead = gptq_factor(gptq_hessian(x16), lam)
+    w = W16.astype(np.float64).copy()
+    w[:, dead] = 0.0
+    codes = np.zeros((N, K), dtype=np.uint8)
+    scales = np.zeros((G, N), dtype=np.float16)
+    zeros = np.zeros((G, N), dtype=np.float16)
+    for j in range(G):
+        cols = slice(g * j, g * (j + 1))
+        wb16 = w[:, cols].astype(np.float16)
+        if quantizer == "sqc":
+            q, s, z = quantize_sqc(wb16, bits[j:j + 1], g)[:3]
+        elif quantizer == "minmax":
+            q, s, z = quantize_minmax(wb16, bits[j:j + 1], g)
+        else:
+            raise ValueError(quantizer)
+        codes[:, cols], scales[j], zeros[j] = q, s[0], z[0]
+        w_hat = s[0].astype(np.float64)[:, None] * (q.astype(np.float64) - z[0].astype(np.float64)[:, None])
+        delta = w[:, cols] - w_hat
+        # E U_bb = delta  (U_bb upper triangular)
+        E = np.linalg.solve(U[cols, cols].T, delta.T).T
+        w[:, g * (j + 1):] -= E @ U[cols, g * (j + 1):]
+    return codes, scales, zeros, w
+
+
+def gptq_proxy_loss(W16: np.ndarray, W_hat: np.ndarray, x16: np.ndarray) -> float:
+    """|| (w - w-hat) x^T ||_F^2 / P: the layer-output error the compensation minimises."""
+    d = (W16.astype(np.float64) - W_hat) @ x16.astype(np.float64).T
+    return float((d * d).sum() / x16.shape[0])
 
 
 # --------------------------------------------------------------------------- convenience

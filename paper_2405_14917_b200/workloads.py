@@ -73,6 +73,19 @@ def make_x(seed: tuple, M: int, K: int) -> np.ndarray:
     return _rng(seed, _STREAM_X, M).standard_normal((M, K), dtype=np.float32).astype(np.float16)
 
 
+def make_calibration_x(seed: tuple, T: int, K: int, rank: int = 16, mix: float = 0.7) -> np.ndarray:
+    """fp16 calibration activations [T][K] with correlated channels: every token is a mixture of
+    `rank` shared directions plus independent noise, scaled per channel by the lognormal activation
+    norms (so a few channels dominate, as in the outlier channels of LLM activations)."""
+    r = _rng(seed, _STREAM_X, 7000 + T)
+    basis = r.standard_normal((rank, K))
+    coeff = r.standard_normal((T, rank))
+    noise = r.standard_normal((T, K))
+    x = mix * (coeff @ basis) / np.sqrt(rank) + (1.0 - mix) * noise
+    x *= make_act_norms(seed, K).astype(np.float64)
+    return x.astype(np.float16)
+
+
 def model_layers(model: str, n_blocks: int | None = None):
     """Yield (layer name, block, N, K, seed) over n_blocks blocks of a model."""
     nb = N_BLOCKS[model] if n_blocks is None else n_blocks
