@@ -286,6 +286,36 @@ int slim_sba_search(const void* W, const void* x, const float* act_norm, int M, 
                     int include_uniform, void* workspace, size_t workspace_bytes,
                     int* p_star_host, uint8_t* bits_host_out, double* errors_host, void* stream);
 
+/* ---- GPTQ error compensation around the quantizer (Algorithm 1) ----------------------------- */
+
+/* Host-only: bytes of workspace for T calibration tokens and an N x K layer (two K x K fp64
+ * matrices, the fp64 running weights, one group of errors and of quantizer input and output).
+ * slim_gptq_factor alone needs the size for N = 0. */
+int slim_gptq_workspace_bytes(int T, int N, int K, int g, size_t* out_bytes);
+
+/* First two steps of Algorithm 1: H = (1/T) sum_t x_t x_t^T, then the upper-triangular U with
+ * U^T U = (H + lambda_abs I)^-1 (the Cholesky factor the algorithm calls H_in), obtained as the
+ * inverse of the factor R of H + lambda_abs I = R R^T.  lambda > 0 is relative to the mean
+ * diagonal: lambda_abs = lambda * mean(diag H) (the GPTQ convention; the scale of H then does not
+ * matter).  An input channel that is zero in every token gets H_kk = 1 and dead[k] = 1.
+ * x fp16 [T][K] device; U_out fp64 [K][K] device (lower triangle zero); dead_out uint8 [K] device
+ * or NULL; workspace 256-byte aligned.  fp64, fixed summation order. */
+int slim_gptq_factor(const void* x, int T, int K, double lambda, double* U_out, uint8_t* dead_out,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* Main loop of Algorithm 1 under the bit map bits_host[K/g]: for every group b in order, the
+ * CURRENT weights of the group, rounded once to fp16, are quantised with slim_quantize_sqc
+ * (use_sqc != 0; lambda 0.1, n 50) or slim_quantize_minmax; then
+ *     E = (w_b - s (q - z)) / U[b, b]      (right division by the diagonal block = times R[b, b]),
+ *     w[:, after b] -= E * U[b, after b].
+ * The running weights are fp64 (dead input channels start at zero).  W fp16 [N][K], x fp16 [T][K];
+ * codes uint8 [N][K], scales and zeros fp16 [G][N] as for slim_quantize_minmax; w_running fp64
+ * [N][K] receives the running weights after the last update and may be NULL.  All device.
+ * Deterministic.  The work is enqueued on `stream`; nothing is synchronised. */
+int slim_gptq_quantize(const void* W, const void* x, const uint8_t* bits_host, double lambda, int use_sqc,
+                       uint8_t* codes, void* scales, void* zeros, double* w_running,
+                       int N, int K, int T, int g, void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

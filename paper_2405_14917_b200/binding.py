@@ -67,6 +67,9 @@ def lib():
             "slim_softmax_kl": [vp, vp, vp, i, i, vp],
             "slim_sba_workspace_bytes": [i, i, i, i, i, ctypes.POINTER(sz)],
             "slim_sba_search": [vp, vp, vp, i, i, i, i, i, i, vp, sz, vp, vp, vp, vp],
+            "slim_gptq_workspace_bytes": [i, i, i, i, ctypes.POINTER(sz)],
+            "slim_gptq_factor": [vp, i, i, ctypes.c_double, vp, vp, vp, sz, vp],
+            "slim_gptq_quantize": [vp, vp, vp, ctypes.c_double, i, vp, vp, vp, vp, i, i, i, i, vp, sz, vp],
         }
         for name, args in sigs.items():
             fn = getattr(L, name)
@@ -307,6 +310,51 @@ def sba_search(W: torch.Tensor, x: torch.Tensor, act_norm: torch.Tensor, avg_bit
                                                     workspace.numel(), ctypes.addressof(p_star), bits.ctypes.data,
                                                     errors.ctypes.data, _stream(W)))
     return p_star.value, bits, errors
+
+
+def gptq_workspace_bytes(T: int, N: int, K: int, g: int = GROUP) -> int:
+    out = ctypes.c_size_t(0)
+    _check("slim_gptq_workspace_bytes", lib().slim_gptq_workspace_bytes(T, N, K, g, ctypes.byref(out)))
+    return out.value
+
+
+def gptq_factor(x: torch.Tensor, lam: float = 0.01, workspace: torch.Tensor | None = None):
+    """Second step of Algorithm 1 on the device: U (fp64 [K][K], upper triangular) with
+    U^T U = (H + lambda I)^-1 for H = x^T x / T, and the flags of the input channels that are zero in
+    every token.  Returns (U, dead)."""
+    T, K = x.shape
+    if workspace is None:
+        workspace = torch.empty(gptq_workspace_bytes(T, 0, K), dtype=torch.uint8, device=x.device)
+    U = torch.empty(K, K, dtype=torch.float64, device=x.device)
+    dead = torch.empty(K, dtype=torch.uint8, device=x.device)
+    _check("slim_gptq_factor", lib().slim_gptq_factor(_dev(x, torch.float16, "x"), T, K, float(lam), U.data_ptr(), dead.data_ptr(),
+                                                      _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(x)))
+    return U, dead
+
+
+def gptq_quantize(W: torch.Tensor, x: torch.Tensor, bits, lam: float = 0.01, quantizer: str = "sqc",
+                  workspace: torch.Tensor | None = None, return_running: bool = False):
+    """Main loop of Algorithm 1 under a given bit map: group by group, quantise the running weights
+    (SQC or Eq. 1) and push the group's error onto the columns still to come.  W fp16 [N][K], x fp16
+    [T][K] calibration tokens.  Returns (codes uint8 [N][K], scales fp16 [G][N], zeros fp16 [G][N])
+    and, if asked, the fp64 running weights after the last update."""
+    if quantizer not in ("sqc", "minmax"):
+        raise ValueError(quantizer)
+    N, K = W.shape
+    T = x.shape[0]
+    b = _bits(bits)
+    G = K // GROUP
+    if workspace is None:
+        workspace = torch.empty(gptq_workspace_bytes(T, N, K), dtype=torch.uint8, device=W.device)
+    codes = torch.empty(N, K, dtype=torch.uint8, device=W.device)
+    scales = torch.empty(G, N, dtype=torch.float16, device=W.device)
+    zeros = torch.empty(G, N, dtype=torch.float16, device=W.device)
+    running = torch.empty(N, K, dtype=torch.float64, device=W.device) if return_running else None
+    _check("slim_gptq_quantize", lib().slim_gptq_quantize(
+        _dev(W, torch.float16, "W"), _dev(x, torch.float16, "x"), _bp(b), float(lam), 1 if quantizer == "sqc" else 0,
+        codes.data_ptr(), scales.data_ptr(), zeros.data_ptr(), running.data_ptr() if return_running else None,
+        N, K, T, GROUP, _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(W)))
+    return (codes, scales, zeros, running) if return_running else (codes, scales, zeros)
 
 
 class _Layer(ctypes.Structure):

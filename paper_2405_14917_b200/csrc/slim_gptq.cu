@@ -1,0 +1,419 @@
+// GPTQ error compensation around the group quantizer (Algorithm 1), sm_100a, fp64 throughout.
+//
+//   H     = (1/P) sum_k x_k x_k^T                       gptq_hessian_kernel (upper tiles only)
+//   H    += lambda mean(diag H) I, dead channels         gptq_damp_kernel
+//   H     = R R^T, R upper triangular                    gptq_chol_{diag,panel,trail}_kernel, last block first
+//   U     = R^-1  (so U^T U = (H + lambda I)^-1: the Cholesky factor Algorithm 1 calls H_in)
+//                                                        gptq_inv_diag_kernel, gptq_inv_row_kernel
+//   per group b:  quantise fp16(w_b) with SQC or Eq. 1 (the library's quantizer kernels),
+//                 E = (w_b - w-hat_b) R_bb                gptq_error_kernel  (R_bb = U_bb^-1: no solve)
+//                 w[:, after] -= E U[b, after]            gptq_update_kernel
+//
+// Everything is a fixed-order fp64 sum, so a layer gives the same codes on every run.  The 64 x 64 x 16
+// register-tiled product below serves the four GEMM-shaped steps; the sequential parts (the factor of
+// a diagonal block, the triangular solves against it) run one thread per row or column.
+#include "slim_common.cuh"
+
+namespace slim {
+
+constexpr int kFB = 64;            // block of the factorisation
+constexpr int kFK = 16;            // depth of one shared-memory stage of the tile product
+constexpr int kFPad = kFB + 1;
+
+// ------------------------------------------------------------------------------------------ 64 x 64 tile product
+// acc[a][b] (rows 4 ty + a, columns 4 tx + b of the tile) += sum_k A(i, k) B(k, j); the operands of one
+// stage are put into As[k][i], Bs[k][j] by the two fill functors (called by all 256 threads with the
+// stage's first k), zero where the operand does not exist.
+template <class FillA, class FillB>
+__device__ __forceinline__ void tile_mac(double (&acc)[4][4], int klen, FillA fill_a, FillB fill_b,
+                                         double (*As)[kFPad], double (*Bs)[kFPad]) {
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    for (int k0 = 0; k0 < klen; k0 += kFK) {
+        fill_a(k0);
+        fill_b(k0);
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kFK; ++k) {
+            double a[4], b[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { a[e] = As[k][4 * ty + e]; b[e] = Bs[k][4 * tx + e]; }
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+#pragma unroll
+                for (int f = 0; f < 4; ++f) acc[e][f] = fma(a[e], b[f], acc[e][f]);
+        }
+        __syncthreads();
+    }
+}
+// Operand stored with the tile index contiguous: element (k, i) = src[k * ld + i].
+__device__ __forceinline__ void fill_k_major(double (*S)[kFPad], const double* src, size_t ld, int k0, int kmax) {
+    const int k = threadIdx.x >> 4, i = (threadIdx.x & 15) * 4;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) S[k][i + e] = k0 + k < kmax ? src[static_cast<size_t>(k0 + k) * ld + i + e] : 0.0;
+}
+__device__ __forceinline__ void fill_k_major_half(double (*S)[kFPad], const __half* src, size_t ld, int k0, int kmax) {
+    const int k = threadIdx.x >> 4, i = (threadIdx.x & 15) * 4;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+        S[k][i + e] = k0 + k < kmax ? static_cast<double>(__half2float(src[static_cast<size_t>(k0 + k) * ld + i + e])) : 0.0;
+}
+// Operand stored with k contiguous: element (i, k) = src[i * ld + k]; rows i >= imax do not exist.
+__device__ __forceinline__ void fill_i_major(double (*S)[kFPad], const double* src, size_t ld, int k0, int kmax, int imax) {
+    const int i = threadIdx.x >> 2, k = (threadIdx.x & 3) * 4;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+        S[k + e][i] = (k0 + k + e < kmax && i < imax) ? src[static_cast<size_t>(i) * ld + k0 + k + e] : 0.0;
+}
+
+// ------------------------------------------------------------------------------------------ Hessian
+// H[i][j] = (1/T) sum_t x[t][i] x[t][j] for the tiles on and above the diagonal (t ascending).
+__global__ void __launch_bounds__(256) gptq_hessian_kernel(const __half* __restrict__ x, double* __restrict__ H, int T, int K) {
+    const int bi = blockIdx.y, bj = blockIdx.x;
+    if (bj < bi) return;
+    __shared__ double As[kFK][kFPad], Bs[kFK][kFPad];
+    double acc[4][4] = {};
+    tile_mac(acc, T, [&](int k0) { fill_k_major_half(As, x + kFB * bi, K, k0, T); },
+             [&](int k0) { fill_k_major_half(Bs, x + kFB * bj, K, k0, T); }, As, Bs);
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const double inv = 1.0 / static_cast<double>(T);
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+#pragma unroll
+        for (int f = 0; f < 4; ++f)
+            H[static_cast<size_t>(kFB * bi + 4 * ty + e) * K + kFB * bj + 4 * tx + f] = acc[e][f] * inv;
+}
+
+// dead[k] = (H_kk == 0); such a channel gets H_kk = 1; then H_kk += lambda * mean(diag H).  One CTA.
+__global__ void __launch_bounds__(1024) gptq_damp_kernel(double* __restrict__ H, uint8_t* __restrict__ dead, int K, double lambda) {
+    __shared__ double part[1024];
+    double s = 0.0;
+    for (int k = threadIdx.x; k < K; k += 1024) {
+        double d = H[static_cast<size_t>(k) * K + k];
+        const bool z = d == 0.0;
+        dead[k] = z ? 1 : 0;
+        if (z) { d = 1.0; H[static_cast<size_t>(k) * K + k] = 1.0; }
+        s += d;
+    }
+    part[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 512; o > 0; o >>= 1) {
+        if (threadIdx.x < o) part[threadIdx.x] += part[threadIdx.x + o];
+        __syncthreads();
+    }
+    const double add = lambda * (part[0] / static_cast<double>(K));
+    for (int k = threadIdx.x; k < K; k += 1024) H[static_cast<size_t>(k) * K + k] += add;
+}
+
+// ------------------------------------------------------------------------------------------ H = R R^T, R upper
+// Diagonal block at b0: the unblocked recursion from the last column to the first,
+//   R_cc = sqrt(S_cc),  R_ic = S_ic / R_cc (i < c),  S_ij -= R_ic R_jc (i <= j < c),   in place.
+__global__ void __launch_bounds__(256) gptq_chol_diag_kernel(double* __restrict__ A, int K, int b0) {
+    __shared__ double S[kFB][kFPad];
+    double* blk = A + static_cast<size_t>(b0) * K + b0;
+    for (int e = threadIdx.x; e < kFB * kFB; e += 256) {
+        const int i = e >> 6, j = e & 63;
+        S[i][j] = j >= i ? blk[static_cast<size_t>(i) * K + j] : 0.0;
+    }
+    __syncthreads();
+    for (int c = kFB - 1; c >= 0; --c) {
+        const double d = sqrt(S[c][c]);
+        __syncthreads();
+        if (threadIdx.x < c) S[threadIdx.x][c] /= d;
+        else if (threadIdx.x == c) S[c][c] = d;
+        __syncthreads();
+        for (int e = threadIdx.x; e < c * c; e += 256) {
+            const int i = e / c, j = e - i * c;
+            if (j >= i) S[i][j] -= S[i][c] * S[j][c];
+        }
+        __syncthreads();
+    }
+    for (int e = threadIdx.x; e < kFB * kFB; e += 256) {
+        const int i = e >> 6, j = e & 63;
+        if (j >= i) blk[static_cast<size_t>(i) * K + j] = S[i][j];
+    }
+}
+
+// Panel above the diagonal block: X R_bb^T = A[I, b] row by row, column c from the last to the first:
+//   X_rc = (A_rc - sum_{c' > c} X_rc' R_cc') / R_cc.   One CTA per 64 rows, one thread per row.
+__global__ void __launch_bounds__(kFB) gptq_chol_panel_kernel(double* __restrict__ A, int K, int b0) {
+    __shared__ double X[kFB][kFPad];
+    const double* blk = A + static_cast<size_t>(b0) * K + b0;       // R_bb: every thread reads the same element
+    double* pan = A + static_cast<size_t>(kFB) * blockIdx.x * K + b0;
+    for (int e = threadIdx.x; e < kFB * kFB; e += kFB) {
+        const int i = e >> 6, j = e & 63;
+        X[i][j] = pan[static_cast<size_t>(i) * K + j];
+    }
+    __syncthreads();
+    const int r = threadIdx.x;
+    for (int c = kFB - 1; c >= 0; --c) {
+        double v = X[r][c];
+        for (int c2 = c + 1; c2 < kFB; ++c2) v -= X[r][c2] * blk[static_cast<size_t>(c) * K + c2];
+        X[r][c] = v / blk[static_cast<size_t>(c) * K + c];
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < kFB * kFB; e += kFB) {
+        const int i = e >> 6, j = e & 63;
+        pan[static_cast<size_t>(i) * K + j] = X[i][j];
+    }
+}
+
+// Trailing update: A[I, J] -= R[I, b] R[J, b]^T for the tiles I <= J in front of block b.
+__global__ void __launch_bounds__(256) gptq_chol_trail_kernel(double* __restrict__ A, int K, int b0) {
+    const int bi = blockIdx.y, bj = blockIdx.x;
+    if (bj < bi) return;
+    __shared__ double As[kFK][kFPad], Bs[kFK][kFPad];
+    double acc[4][4] = {};
+    const double* pi = A + static_cast<size_t>(kFB) * bi * K + b0;
+    const double* pj = A + static_cast<size_t>(kFB) * bj * K + b0;
+    tile_mac(acc, kFB, [&](int k0) { fill_i_major(As, pi, K, k0, kFB, kFB); },
+             [&](int k0) { fill_i_major(Bs, pj, K, k0, kFB, kFB); }, As, Bs);
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+#pragma unroll
+        for (int f = 0; f < 4; ++f)
+            A[static_cast<size_t>(kFB * bi + 4 * ty + e) * K + kFB * bj + 4 * tx + f] -= acc[e][f];
+}
+
+// ------------------------------------------------------------------------------------------ U = R^-1
+// Diagonal blocks: column j of U_bb by back substitution, u_i = (delta_ij - sum_{i < l <= j} R_il u_l) / R_ii.
+__global__ void __launch_bounds__(kFB) gptq_inv_diag_kernel(const double* __restrict__ R, double* __restrict__ U, int K) {
+    __shared__ double Ub[kFB][kFPad];
+    const size_t off = static_cast<size_t>(kFB) * blockIdx.x * K + static_cast<size_t>(kFB) * blockIdx.x;
+    for (int e = threadIdx.x; e < kFB * kFB; e += kFB) Ub[e >> 6][e & 63] = 0.0;
+    __syncthreads();
+    const int j = threadIdx.x;
+    for (int i = j; i >= 0; --i) {                       // lanes of a warp read the same R_il for l <= their j
+        double v = i == j ? 1.0 : 0.0;
+        for (int l = i + 1; l <= j; ++l) v -= R[off + static_cast<size_t>(i) * K + l] * Ub[l][j];
+        Ub[i][j] = v / R[off + static_cast<size_t>(i) * K + i];
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < kFB * kFB; e += kFB) {
+        const int i = e >> 6, j2 = e & 63;
+        U[off + static_cast<size_t>(i) * K + j2] = Ub[i][j2];
+    }
+}
+
+// Block row I, all J > I (the rows below I are complete): U[I, J] = -U_II sum_{I < L <= J} R[I, L] U[L, J].
+// The CTA first leaves the sum in U[I, J], then multiplies it by -U_II.
+__global__ void __launch_bounds__(256) gptq_inv_row_kernel(const double* R, double* U, int K, int I) {
+    const int J = I + 1 + blockIdx.x;
+    __shared__ double As[kFK][kFPad], Bs[kFK][kFPad];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    double acc[4][4] = {};
+    const double* a = R + static_cast<size_t>(kFB) * I * K + static_cast<size_t>(kFB) * (I + 1);        // R[I rows][k]
+    const double* b = U + static_cast<size_t>(kFB) * (I + 1) * K + static_cast<size_t>(kFB) * J;        // U[k][J columns]
+    const int klen = kFB * (J - I);
+    tile_mac(acc, klen, [&](int k0) { fill_i_major(As, a, K, k0, klen, kFB); },
+             [&](int k0) { fill_k_major(Bs, b, K, k0, klen); }, As, Bs);
+    double* out = U + static_cast<size_t>(kFB) * I * K + static_cast<size_t>(kFB) * J;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+#pragma unroll
+        for (int f = 0; f < 4; ++f) out[static_cast<size_t>(4 * ty + e) * K + 4 * tx + f] = acc[e][f];
+    __syncthreads();
+    double acc2[4][4] = {};
+    const double* uii = U + static_cast<size_t>(kFB) * I * K + static_cast<size_t>(kFB) * I;
+    tile_mac(acc2, kFB, [&](int k0) { fill_i_major(As, uii, K, k0, kFB, kFB); },
+             [&](int k0) { fill_k_major(Bs, out, K, k0, kFB); }, As, Bs);
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+#pragma unroll
+        for (int f = 0; f < 4; ++f) out[static_cast<size_t>(4 * ty + e) * K + 4 * tx + f] = -acc2[e][f];
+}
+
+// ------------------------------------------------------------------------------------------ the loop over the groups
+// Running weights: w = fp64(W), dead input channels zeroed.
+__global__ void __launch_bounds__(256) gptq_init_kernel(const __half* __restrict__ W, const uint8_t* __restrict__ dead,
+                                                        double* __restrict__ w, size_t total, int K) {
+    const size_t i = static_cast<size_t>(blockIdx.x) * 256 + threadIdx.x;
+    if (i >= total) return;
+    const int k = static_cast<int>(i % static_cast<size_t>(K));
+    w[i] = dead[k] ? 0.0 : static_cast<double>(__half2float(W[i]));
+}
+// The group's current weights rounded to fp16 (one rounding), [N][128]: the quantizer's input.
+__global__ void __launch_bounds__(256) gptq_round_kernel(const double* __restrict__ w, __half* __restrict__ wb, int N, int K, int c0) {
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= N * SLIM_GROUP) return;
+    const int n = i >> 7, c = i & 127;
+    wb[i] = __double2half(w[static_cast<size_t>(n) * K + c0 + c]);
+}
+// delta = w_b - s (q - z) for 16 rows per CTA, codes copied into the layer's array,
+// E[n][c] = sum_{c' <= c} delta[n][c'] R[c0 + c'][c0 + c]   (thread c, c' ascending).
+constexpr int kErrRows = 16;
+__global__ void __launch_bounds__(SLIM_GROUP) gptq_error_kernel(const double* __restrict__ w, const uint8_t* __restrict__ qb,
+                                                                const __half* __restrict__ s_row, const __half* __restrict__ z_row,
+                                                                const double* __restrict__ R, uint8_t* __restrict__ codes,
+                                                                double* __restrict__ E, int N, int K, int c0) {
+    __shared__ double delta[kErrRows][SLIM_GROUP];
+    const int c = threadIdx.x, n0 = kErrRows * blockIdx.x;
+    for (int r = 0; r < kErrRows; ++r) {
+        const int n = n0 + r;
+        double d = 0.0;
+        if (n < N) {
+            const uint8_t q = qb[static_cast<size_t>(n) * SLIM_GROUP + c];
+            codes[static_cast<size_t>(n) * K + c0 + c] = q;
+            const double sc = static_cast<double>(__half2float(s_row[n])), zp = static_cast<double>(__half2float(z_row[n]));
+            d = w[static_cast<size_t>(n) * K + c0 + c] - sc * (static_cast<double>(q) - zp);
+        }
+        delta[r][c] = d;
+    }
+    __syncthreads();
+    double acc[kErrRows];
+#pragma unroll
+    for (int r = 0; r < kErrRows; ++r) acc[r] = 0.0;
+    for (int c2 = 0; c2 <= c; ++c2) {
+        const double rv = R[static_cast<size_t>(c0 + c2) * K + c0 + c];
+#pragma unroll
+        for (int r = 0; r < kErrRows; ++r) acc[r] = fma(delta[r][c2], rv, acc[r]);
+    }
+    for (int r = 0; r < kErrRows; ++r)
+        if (n0 + r < N) E[static_cast<size_t>(n0 + r) * SLIM_GROUP + c] = acc[r];
+}
+// w[n][k] -= sum_c E[n][c] U[c0 + c][k] for the columns k >= k0 = c0 + 128 (c ascending).
+__global__ void __launch_bounds__(256) gptq_update_kernel(double* __restrict__ w, const double* __restrict__ E,
+                                                          const double* __restrict__ U, int N, int K, int c0) {
+    __shared__ double As[kFK][kFPad], Bs[kFK][kFPad];
+    const int n0 = kFB * blockIdx.y, k0 = c0 + SLIM_GROUP + kFB * blockIdx.x;
+    double acc[4][4] = {};
+    tile_mac(acc, SLIM_GROUP, [&](int kk) { fill_i_major(As, E + static_cast<size_t>(n0) * SLIM_GROUP, SLIM_GROUP, kk, SLIM_GROUP, N - n0); },
+             [&](int kk) { fill_k_major(Bs, U + static_cast<size_t>(c0) * K + k0, K, kk, SLIM_GROUP); }, As, Bs);
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int n = n0 + 4 * ty + e;
+        if (n >= N) continue;
+#pragma unroll
+        for (int f = 0; f < 4; ++f) w[static_cast<size_t>(n) * K + k0 + 4 * tx + f] -= acc[e][f];
+    }
+}
+
+// ------------------------------------------------------------------------------------------ host side
+struct GptqLayout {
+    size_t dead, R, U, w, E, wb, qb, total;
+};
+static size_t up256(size_t v) { return (v + 255) / 256 * 256; }
+static int gptq_layout(int T, int N, int K, int g, GptqLayout* lay) {
+    if (lay == nullptr || T < 1 || N < 0 || K < 1) return SLIM_ERR_INVALID_ARG;
+    if (g != SLIM_GROUP) return SLIM_ERR_UNSUPPORTED;
+    if (K % SLIM_GROUP != 0 || K / SLIM_GROUP > SLIM_MAX_GROUPS) return SLIM_ERR_UNSUPPORTED;
+    size_t off = 0;
+    lay->dead = off; off += up256(static_cast<size_t>(K));
+    lay->R = off; off += up256(static_cast<size_t>(K) * K * sizeof(double));
+    lay->U = off; off += up256(static_cast<size_t>(K) * K * sizeof(double));
+    lay->w = off; off += up256(static_cast<size_t>(N) * K * sizeof(double));
+    lay->E = off; off += up256(static_cast<size_t>(N) * SLIM_GROUP * sizeof(double));
+    lay->wb = off; off += up256(static_cast<size_t>(N) * SLIM_GROUP * sizeof(__half));
+    lay->qb = off; off += up256(static_cast<size_t>(N) * SLIM_GROUP);
+    lay->total = off;
+    return SLIM_OK;
+}
+
+// x -> U (and the dead-channel flags) inside the workspace.
+static int gptq_factor_into(const void* x, int T, int K, double lambda, uint8_t* ws, const GptqLayout& lay, cudaStream_t s) {
+    double* R = reinterpret_cast<double*>(ws + lay.R);
+    double* U = reinterpret_cast<double*>(ws + lay.U);
+    uint8_t* dead = ws + lay.dead;
+    const int nb = K / kFB;
+    gptq_hessian_kernel<<<dim3(nb, nb), 256, 0, s>>>(static_cast<const __half*>(x), R, T, K);
+    gptq_damp_kernel<<<1, 1024, 0, s>>>(R, dead, K, lambda);
+    for (int b = nb - 1; b >= 0; --b) {
+        gptq_chol_diag_kernel<<<1, 256, 0, s>>>(R, K, kFB * b);
+        if (b > 0) {
+            gptq_chol_panel_kernel<<<b, kFB, 0, s>>>(R, K, kFB * b);
+            gptq_chol_trail_kernel<<<dim3(b, b), 256, 0, s>>>(R, K, kFB * b);
+        }
+    }
+    SLIM_CUDA_TRY(cudaGetLastError());
+    SLIM_CUDA_TRY(cudaMemsetAsync(U, 0, static_cast<size_t>(K) * K * sizeof(double), s));
+    gptq_inv_diag_kernel<<<nb, kFB, 0, s>>>(R, U, K);
+    for (int I = nb - 2; I >= 0; --I) gptq_inv_row_kernel<<<nb - 1 - I, 256, 0, s>>>(R, U, K, I);
+    SLIM_CUDA_TRY(cudaGetLastError());
+    return SLIM_OK;
+}
+
+}  // namespace slim
+
+extern "C" {
+
+int slim_gptq_workspace_bytes(int T, int N, int K, int g, size_t* out_bytes) {
+    if (out_bytes == nullptr) return SLIM_ERR_INVALID_ARG;
+    slim::GptqLayout lay;
+    const int st = slim::gptq_layout(T, N, K, g, &lay);
+    if (st != SLIM_OK) return st;
+    *out_bytes = lay.total;
+    return SLIM_OK;
+}
+
+int slim_gptq_factor(const void* x, int T, int K, double lambda, double* U_out, uint8_t* dead_out,
+                     void* workspace, size_t workspace_bytes, void* stream) {
+    slim::GptqLayout lay;
+    const int st = slim::gptq_layout(T, 0, K, SLIM_GROUP, &lay);
+    if (st != SLIM_OK) return st;
+    if (!(lambda > 0.0) || x == nullptr || U_out == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (!slim::aligned16(x) || !slim::aligned16(U_out)) return SLIM_ERR_ALIGNMENT;
+    if (workspace == nullptr || workspace_bytes < lay.total) return SLIM_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SLIM_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const int st2 = slim::gptq_factor_into(x, T, K, lambda, ws, lay, s);
+    if (st2 != SLIM_OK) return st2;
+    SLIM_CUDA_TRY(cudaMemcpyAsync(U_out, ws + lay.U, static_cast<size_t>(K) * K * sizeof(double), cudaMemcpyDeviceToDevice, s));
+    if (dead_out != nullptr) SLIM_CUDA_TRY(cudaMemcpyAsync(dead_out, ws + lay.dead, static_cast<size_t>(K), cudaMemcpyDeviceToDevice, s));
+    return SLIM_OK;
+}
+
+int slim_gptq_quantize(const void* W, const void* x, const uint8_t* bits_host, double lambda, int use_sqc,
+                       uint8_t* codes, void* scales, void* zeros, double* w_running,
+                       int N, int K, int T, int g, void* workspace, size_t workspace_bytes, void* stream) {
+    slim::GptqLayout lay;
+    int st = slim::gptq_layout(T, N, K, g, &lay);
+    if (st != SLIM_OK) return st;
+    slim::GroupTable gt;
+    st = slim::make_group_table(N, K, g, bits_host, &gt);
+    if (st != SLIM_OK) return st;
+    if (!(lambda > 0.0)) return SLIM_ERR_INVALID_ARG;
+    if (N == 0) return SLIM_OK;
+    if (W == nullptr || x == nullptr || codes == nullptr || scales == nullptr || zeros == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (!slim::aligned16(W) || !slim::aligned16(x) || !slim::aligned16(codes) || !slim::aligned16(scales) || !slim::aligned16(zeros))
+        return SLIM_ERR_ALIGNMENT;
+    if (workspace == nullptr || workspace_bytes < lay.total) return SLIM_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SLIM_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    st = slim::gptq_factor_into(x, T, K, lambda, ws, lay, s);
+    if (st != SLIM_OK) return st;
+
+    const double* R = reinterpret_cast<const double*>(ws + lay.R);
+    const double* U = reinterpret_cast<const double*>(ws + lay.U);
+    double* w = reinterpret_cast<double*>(ws + lay.w);
+    double* E = reinterpret_cast<double*>(ws + lay.E);
+    __half* wb = reinterpret_cast<__half*>(ws + lay.wb);
+    uint8_t* qb = ws + lay.qb;
+    __half* sc = static_cast<__half*>(scales);
+    __half* zp = static_cast<__half*>(zeros);
+    const size_t total = static_cast<size_t>(N) * K;
+    slim::gptq_init_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, s>>>(static_cast<const __half*>(W), ws + lay.dead, w, total, K);
+    SLIM_CUDA_TRY(cudaGetLastError());
+    for (int j = 0; j < gt.G; ++j) {
+        const int c0 = SLIM_GROUP * j;
+        slim::gptq_round_kernel<<<(N * SLIM_GROUP + 255) / 256, 256, 0, s>>>(w, wb, N, K, c0);
+        SLIM_CUDA_TRY(cudaGetLastError());
+        const uint8_t b1[1] = {gt.bits[j]};
+        st = use_sqc ? slim_quantize_sqc(wb, b1, qb, sc + static_cast<size_t>(j) * N, zp + static_cast<size_t>(j) * N, nullptr,
+                                         N, SLIM_GROUP, g, 0.1, 50, stream)
+                     : slim_quantize_minmax(wb, b1, qb, sc + static_cast<size_t>(j) * N, zp + static_cast<size_t>(j) * N,
+                                            N, SLIM_GROUP, g, stream);
+        if (st != SLIM_OK) return st;
+        slim::gptq_error_kernel<<<(N + slim::kErrRows - 1) / slim::kErrRows, SLIM_GROUP, 0, s>>>(
+            w, qb, sc + static_cast<size_t>(j) * N, zp + static_cast<size_t>(j) * N, R, codes, E, N, K, c0);
+        if (j + 1 < gt.G)
+            slim::gptq_update_kernel<<<dim3((K - c0 - SLIM_GROUP) / slim::kFB, (N + slim::kFB - 1) / slim::kFB), 256, 0, s>>>(w, E, U, N, K, c0);
+        SLIM_CUDA_TRY(cudaGetLastError());
+    }
+    if (w_running != nullptr) SLIM_CUDA_TRY(cudaMemcpyAsync(w_running, w, total * sizeof(double), cudaMemcpyDeviceToDevice, s));
+    return SLIM_OK;
+}
+
+}  // extern "C"

@@ -163,3 +163,25 @@ def test_sba_workspace_and_quantizer_argument_errors(slim):
     assert L.slim_dense_linear(None, None, None, 4, 16, 128, None) == -1
     assert L.slim_dense_linear(None, None, None, 0, 16, 128, None) == 0
     assert L.slim_softmax_kl(None, None, None, 4, 16, None) == -1
+
+
+def test_gptq_workspace_and_argument_errors(slim):
+    def ws_bytes(T, N, K, g=128):
+        out = ctypes.c_size_t(0)
+        return slim.lib().slim_gptq_workspace_bytes(T, N, K, g, ctypes.byref(out)), out.value
+
+    st, b = ws_bytes(64, 256, 512)
+    # dead flags, two K x K fp64 matrices, the fp64 running weights, one group of errors (fp64), of quantizer input
+    # (fp16) and of codes, each rounded up to 256 bytes
+    assert st == 0 and b == 512 + 2 * 512 * 512 * 8 + 256 * 512 * 8 + 256 * 128 * (8 + 2 + 1)
+    assert ws_bytes(64, 0, 512)[1] == 512 + 2 * 512 * 512 * 8            # the factor alone
+    assert ws_bytes(0, 256, 512)[0] == -1                                 # no calibration token
+    assert ws_bytes(64, 256, 500)[0] == -2                                # K not a multiple of 128
+    assert ws_bytes(64, 256, 512, g=64)[0] == -2                          # group size
+    bits = np.array([2, 2, 2, 2], dtype=np.uint8)
+    L = slim.lib()
+    args = lambda lam, wsb: (256, 256, bits.ctypes.data, ctypes.c_double(lam), 1, 256, 256, 256, None, 256, 512, 64, 128, 256, wsb, None)
+    assert L.slim_gptq_quantize(*args(0.0, b)) == -1                      # the damping must be positive
+    assert L.slim_gptq_quantize(*args(0.01, b - 1)) == -4                 # workspace too small
+    assert L.slim_gptq_factor(256, 64, 512, ctypes.c_double(0.01), None, None, 256, b, None) == -1   # no output
+
