@@ -4,7 +4,7 @@
 //   H    += lambda mean(diag H) I, dead channels         gptq_damp_kernel
 //   H     = R R^T, R upper triangular                    gptq_chol_{diag,panel,trail}_kernel, last block first
 //   U     = R^-1  (so U^T U = (H + lambda I)^-1: the Cholesky factor Algorithm 1 calls H_in)
-//                                                        gptq_inv_diag_kernel, gptq_inv_row_kernel
+//                                                        gptq_inv_diag_kernel, gptq_inv_pair{1,2}_kernel (doubling)
 //   per group b:  quantise fp16(w_b) with SQC or Eq. 1 (the library's quantizer kernels),
 //                 E = (w_b - w-hat_b) R_bb                gptq_error_kernel  (R_bb = U_bb^-1: no solve)
 //                 w[:, after] -= E U[b, after]            gptq_update_kernel
@@ -195,32 +195,51 @@ __global__ void __launch_bounds__(kFB) gptq_inv_diag_kernel(const double* __rest
     }
 }
 
-// Block row I, all J > I (the rows below I are complete): U[I, J] = -U_II sum_{I < L <= J} R[I, L] U[L, J].
-// The CTA first leaves the sum in U[I, J], then multiplies it by -U_II.
-__global__ void __launch_bounds__(256) gptq_inv_row_kernel(const double* R, double* U, int K, int I) {
-    const int J = I + 1 + blockIdx.x;
+// Off-diagonal blocks by doubling: with the inverses of two neighbouring diagonal segments A (s x s at o) and
+// C (s2 x s2 at o + s) known, the block above C is  -A^-1 (B C^-1),  B = R[A rows, C columns].
+// First half: T = B C^-1, left in the unused mirror block U[C rows, A columns] (column tile j of the upper
+// triangular C^-1 has its nonzeros in k < 64 (j + 1)).
+__global__ void __launch_bounds__(256) gptq_inv_pair1_kernel(const double* R, double* U, int K, int s) {
+    const int o = 2 * s * blockIdx.z, s2 = min(s, K - o - s);
+    const int ti = blockIdx.y, tj = blockIdx.x;
+    if (s2 <= 0 || kFB * tj >= s2) return;
     __shared__ double As[kFK][kFPad], Bs[kFK][kFPad];
-    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     double acc[4][4] = {};
-    const double* a = R + static_cast<size_t>(kFB) * I * K + static_cast<size_t>(kFB) * (I + 1);        // R[I rows][k]
-    const double* b = U + static_cast<size_t>(kFB) * (I + 1) * K + static_cast<size_t>(kFB) * J;        // U[k][J columns]
-    const int klen = kFB * (J - I);
+    const double* a = R + static_cast<size_t>(o + kFB * ti) * K + o + s;                 // B[i][k]
+    const double* b = U + static_cast<size_t>(o + s) * K + o + s + kFB * tj;             // C^-1[k][j]
+    const int klen = kFB * (tj + 1);
     tile_mac(acc, klen, [&](int k0) { fill_i_major(As, a, K, k0, klen, kFB); },
              [&](int k0) { fill_k_major(Bs, b, K, k0, klen); }, As, Bs);
-    double* out = U + static_cast<size_t>(kFB) * I * K + static_cast<size_t>(kFB) * J;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    double* t = U + static_cast<size_t>(o + s + kFB * tj) * K + o + kFB * ti;            // T stored transposed: T^T[j][i]
 #pragma unroll
     for (int e = 0; e < 4; ++e)
 #pragma unroll
-        for (int f = 0; f < 4; ++f) out[static_cast<size_t>(4 * ty + e) * K + 4 * tx + f] = acc[e][f];
-    __syncthreads();
-    double acc2[4][4] = {};
-    const double* uii = U + static_cast<size_t>(kFB) * I * K + static_cast<size_t>(kFB) * I;
-    tile_mac(acc2, kFB, [&](int k0) { fill_i_major(As, uii, K, k0, kFB, kFB); },
-             [&](int k0) { fill_k_major(Bs, out, K, k0, kFB); }, As, Bs);
+        for (int f = 0; f < 4; ++f) t[static_cast<size_t>(4 * tx + f) * K + 4 * ty + e] = acc[e][f];
+}
+// Second half: U[A rows, C columns] = -A^-1 T (row tile i of the upper triangular A^-1 has its nonzeros in k >= 64 i).
+__global__ void __launch_bounds__(256) gptq_inv_pair2_kernel(double* U, int K, int s) {
+    const int o = 2 * s * blockIdx.z, s2 = min(s, K - o - s);
+    const int ti = blockIdx.y, tj = blockIdx.x;
+    if (s2 <= 0 || kFB * tj >= s2) return;
+    __shared__ double As[kFK][kFPad], Bs[kFK][kFPad];
+    double acc[4][4] = {};
+    const int kbeg = kFB * ti, klen = s - kbeg;
+    const double* a = U + static_cast<size_t>(o + kFB * ti) * K + o + kbeg;              // A^-1[i][k], k from kbeg
+    const double* b = U + static_cast<size_t>(o + s + kFB * tj) * K + o + kbeg;          // T^T[j][k]
+    tile_mac(acc, klen, [&](int k0) { fill_i_major(As, a, K, k0, klen, kFB); },
+             [&](int k0) { fill_i_major(Bs, b, K, k0, klen, kFB); }, As, Bs);
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    double* out = U + static_cast<size_t>(o + kFB * ti) * K + o + s + kFB * tj;
 #pragma unroll
     for (int e = 0; e < 4; ++e)
 #pragma unroll
-        for (int f = 0; f < 4; ++f) out[static_cast<size_t>(4 * ty + e) * K + 4 * tx + f] = -acc2[e][f];
+        for (int f = 0; f < 4; ++f) out[static_cast<size_t>(4 * ty + e) * K + 4 * tx + f] = -acc[e][f];
+}
+// The mirror blocks held T: the lower triangle goes back to zero.
+__global__ void __launch_bounds__(256) gptq_zero_lower_kernel(double* U, int K) {
+    const int i = blockIdx.y, j0 = blockIdx.x * 256 + threadIdx.x;
+    if (j0 < i) U[static_cast<size_t>(i) * K + j0] = 0.0;
 }
 
 // ------------------------------------------------------------------------------------------ the loop over the groups
@@ -328,7 +347,12 @@ static int gptq_factor_into(const void* x, int T, int K, double lambda, uint8_t*
     SLIM_CUDA_TRY(cudaGetLastError());
     SLIM_CUDA_TRY(cudaMemsetAsync(U, 0, static_cast<size_t>(K) * K * sizeof(double), s));
     gptq_inv_diag_kernel<<<nb, kFB, 0, s>>>(R, U, K);
-    for (int I = nb - 2; I >= 0; --I) gptq_inv_row_kernel<<<nb - 1 - I, 256, 0, s>>>(R, U, K, I);
+    for (int seg = kFB; seg < K; seg *= 2) {
+        const dim3 grid(seg / kFB, seg / kFB, (K + 2 * seg - 1) / (2 * seg));
+        gptq_inv_pair1_kernel<<<grid, 256, 0, s>>>(R, U, K, seg);
+        gptq_inv_pair2_kernel<<<grid, 256, 0, s>>>(U, K, seg);
+    }
+    gptq_zero_lower_kernel<<<dim3((K + 255) / 256, K), 256, 0, s>>>(U, K);
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;
 }
