@@ -463,7 +463,7 @@ def run_gptq(args):
     # trailing updates of the factorisation, block rows of the triangular inverse, pushes of the group errors
     tile = 2.0 * 64 * 64
     flops = (nb * (nb + 1) // 2) * tile * T
-    flops += sum(b * (b + 1) // 2 for b in range(1, nb)) * tile * 64
+    flops += sum(b * (b + 1) // 2 + b for b in range(1, nb)) * tile * 64      # trailing tiles and panel tiles
     seg = 64
     while seg < K:                                        # triangular inverse by doubling: T = B C^-1, then -A^-1 T
         for o in range(0, K, 2 * seg):
@@ -476,7 +476,7 @@ def run_gptq(args):
     achieved = flops * steps / (ms * 1e-3) / 1e12
     peak = 148 * 64 * 2 * 1.965e9 / 1e12
     levels = (nb - 1).bit_length()
-    launches = 2 + nb + 2 * (nb - 1) + 1 + 2 * levels + 1 + 1 + 4 * G - 1
+    launches = 2 + nb + 2 * (nb - 1) + 2 * levels + 1 + 1 + 4 * G - 1
     line = {"metric": "GPTQ error compensation with SQC (Algorithm 1): weights quantised per second (LLaMA-7B 4096x4096 layer, avg 2-bit, g=128)",
             "value": value, "unit": "Mweight/s", "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": ms / steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",

@@ -4,7 +4,7 @@
 //   H    += lambda mean(diag H) I, dead channels         gptq_damp_kernel
 //   H     = R R^T, R upper triangular                    gptq_chol_{diag,panel,trail}_kernel, last block first
 //   U     = R^-1  (so U^T U = (H + lambda I)^-1: the Cholesky factor Algorithm 1 calls H_in)
-//                                                        gptq_inv_diag_kernel, gptq_inv_pair{1,2}_kernel (doubling)
+//                                                        diagonal blocks with the factor, then gptq_inv_pair{1,2}_kernel (doubling)
 //   per group b:  quantise fp16(w_b) with SQC or Eq. 1 (the library's quantizer kernels),
 //                 E = (w_b - w-hat_b) R_bb                gptq_error_kernel  (R_bb = U_bb^-1: no solve)
 //                 w[:, after] -= E U[b, after]            gptq_update_kernel
@@ -18,12 +18,14 @@ namespace slim {
 
 constexpr int kFB = 64;            // block of the factorisation
 constexpr int kFK = 16;            // depth of one shared-memory stage of the tile product
-constexpr int kFPad = kFB + 1;
+constexpr int kFPad = kFB + 2;    // row stride of the staged operands: even, so that pairs of doubles stay 16-byte aligned
 
 // ------------------------------------------------------------------------------------------ 64 x 64 tile product
-// acc[a][b] (rows 4 ty + a, columns 4 tx + b of the tile) += sum_k A(i, k) B(k, j); the operands of one
-// stage are put into As[k][i], Bs[k][j] by the two fill functors (called by all 256 threads with the
-// stage's first k), zero where the operand does not exist.
+// acc[a][b] (rows tidx(ty, a), columns tidx(tx, b) of the tile) += sum_k A(i, k) B(k, j); the operands of
+// one stage are put into As[k][i], Bs[k][j] by the two fill functors (called by all 256 threads with the
+// stage's first k), zero where the operand does not exist.  A thread owns the index pairs (2t, 2t + 1) and
+// (32 + 2t, 33 + 2t), so that the 16 threads of a row read consecutive 16-byte pieces of shared memory.
+__device__ __forceinline__ int tidx(int t, int e) { return 2 * t + (e & 1) + 32 * (e >> 1); }
 template <class FillA, class FillB>
 __device__ __forceinline__ void tile_mac(double (&acc)[4][4], int klen, FillA fill_a, FillB fill_b,
                                          double (*As)[kFPad], double (*Bs)[kFPad]) {
@@ -34,9 +36,9 @@ __device__ __forceinline__ void tile_mac(double (&acc)[4][4], int klen, FillA fi
         __syncthreads();
 #pragma unroll
         for (int k = 0; k < kFK; ++k) {
-            double a[4], b[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) { a[e] = As[k][4 * ty + e]; b[e] = Bs[k][4 * tx + e]; }
+            const double2 a01 = *reinterpret_cast<const double2*>(&As[k][2 * ty]), a23 = *reinterpret_cast<const double2*>(&As[k][32 + 2 * ty]);
+            const double2 b01 = *reinterpret_cast<const double2*>(&Bs[k][2 * tx]), b23 = *reinterpret_cast<const double2*>(&Bs[k][32 + 2 * tx]);
+            const double a[4] = {a01.x, a01.y, a23.x, a23.y}, b[4] = {b01.x, b01.y, b23.x, b23.y};
 #pragma unroll
             for (int e = 0; e < 4; ++e)
 #pragma unroll
@@ -70,7 +72,7 @@ __device__ __forceinline__ void fill_i_major(double (*S)[kFPad], const double* s
 __global__ void __launch_bounds__(256) gptq_hessian_kernel(const __half* __restrict__ x, double* __restrict__ H, int T, int K) {
     const int bi = blockIdx.y, bj = blockIdx.x;
     if (bj < bi) return;
-    __shared__ double As[kFK][kFPad], Bs[kFK][kFPad];
+    __shared__ __align__(16) double As[kFK][kFPad], Bs[kFK][kFPad];
     double acc[4][4] = {};
     tile_mac(acc, T, [&](int k0) { fill_k_major_half(As, x + kFB * bi, K, k0, T); },
              [&](int k0) { fill_k_major_half(Bs, x + kFB * bj, K, k0, T); }, As, Bs);
@@ -80,7 +82,7 @@ __global__ void __launch_bounds__(256) gptq_hessian_kernel(const __half* __restr
     for (int e = 0; e < 4; ++e)
 #pragma unroll
         for (int f = 0; f < 4; ++f)
-            H[static_cast<size_t>(kFB * bi + 4 * ty + e) * K + kFB * bj + 4 * tx + f] = acc[e][f] * inv;
+            H[static_cast<size_t>(kFB * bi + tidx(ty, e)) * K + kFB * bj + tidx(tx, f)] = acc[e][f] * inv;
 }
 
 // dead[k] = (H_kk == 0); such a channel gets H_kk = 1; then H_kk += lambda * mean(diag H).  One CTA.
@@ -106,24 +108,28 @@ __global__ void __launch_bounds__(1024) gptq_damp_kernel(double* __restrict__ H,
 
 // ------------------------------------------------------------------------------------------ H = R R^T, R upper
 // Diagonal block at b0: the unblocked recursion from the last column to the first,
-//   R_cc = sqrt(S_cc),  R_ic = S_ic / R_cc (i < c),  S_ij -= R_ic R_jc (i <= j < c),   in place.
-__global__ void __launch_bounds__(256) gptq_chol_diag_kernel(double* __restrict__ A, int K, int b0) {
-    __shared__ double S[kFB][kFPad];
+//   R_cc = sqrt(S_cc),  R_ic = S_ic / R_cc (i < c),  S_ij -= R_ic R_jc (i <= j < c),   in place;
+// then its inverse (thread j: column j by back substitution, u_i = (delta_ij - sum_{l > i} R_il u_l) / R_ii,
+// held in registers), which is the diagonal block of U and turns the panel solve into a product.
+__global__ void __launch_bounds__(256) gptq_chol_diag_kernel(double* __restrict__ A, double* __restrict__ U, int K, int b0) {
+    __shared__ double S[kFB][kFB + 1];
     double* blk = A + static_cast<size_t>(b0) * K + b0;
     for (int e = threadIdx.x; e < kFB * kFB; e += 256) {
         const int i = e >> 6, j = e & 63;
         S[i][j] = j >= i ? blk[static_cast<size_t>(i) * K + j] : 0.0;
     }
     __syncthreads();
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     for (int c = kFB - 1; c >= 0; --c) {
         const double d = sqrt(S[c][c]);
         __syncthreads();
         if (threadIdx.x < c) S[threadIdx.x][c] /= d;
         else if (threadIdx.x == c) S[c][c] = d;
         __syncthreads();
-        for (int e = threadIdx.x; e < c * c; e += 256) {
-            const int i = e / c, j = e - i * c;
-            if (j >= i) S[i][j] -= S[i][c] * S[j][c];
+        for (int i = ty; i < c; i += 16) {
+            const double ric = S[i][c];
+            for (int j = tx; j < c; j += 16)
+                if (j >= i) S[i][j] -= ric * S[j][c];
         }
         __syncthreads();
     }
@@ -131,37 +137,45 @@ __global__ void __launch_bounds__(256) gptq_chol_diag_kernel(double* __restrict_
         const int i = e >> 6, j = e & 63;
         if (j >= i) blk[static_cast<size_t>(i) * K + j] = S[i][j];
     }
+    if (threadIdx.x < kFB) {
+        const int j = threadIdx.x;
+        double u[kFB];
+#pragma unroll
+        for (int i = kFB - 1; i >= 0; --i) {
+            double v0 = i == j ? 1.0 : 0.0, v1 = 0.0;          // rows below j stay zero: every u_l they meet is zero
+#pragma unroll
+            for (int l = i + 1; l < kFB; ++l) {
+                if ((l - i) & 1) v0 = fma(-S[i][l], u[l], v0);
+                else v1 = fma(-S[i][l], u[l], v1);
+            }
+            u[i] = (v0 + v1) / S[i][i];
+        }
+        double* ub = U + static_cast<size_t>(b0) * K + b0 + j;
+#pragma unroll
+        for (int i = 0; i < kFB; ++i) ub[static_cast<size_t>(i) * K] = u[i];
+    }
 }
 
-// Panel above the diagonal block: X R_bb^T = A[I, b] row by row, column c from the last to the first:
-//   X_rc = (A_rc - sum_{c' > c} X_rc' R_cc') / R_cc.   One CTA per 64 rows, one thread per row.
-__global__ void __launch_bounds__(kFB) gptq_chol_panel_kernel(double* __restrict__ A, int K, int b0) {
-    __shared__ double X[kFB][kFPad];
-    const double* blk = A + static_cast<size_t>(b0) * K + b0;       // R_bb: every thread reads the same element
+// Panel above the diagonal block: X R_bb^T = A[I, b], i.e. X = A[I, b] (R_bb^-1)^T, one 64 x 64 tile per CTA, in place.
+__global__ void __launch_bounds__(256) gptq_chol_panel_kernel(double* __restrict__ A, const double* __restrict__ U, int K, int b0) {
+    __shared__ __align__(16) double As[kFK][kFPad], Bs[kFK][kFPad];
     double* pan = A + static_cast<size_t>(kFB) * blockIdx.x * K + b0;
-    for (int e = threadIdx.x; e < kFB * kFB; e += kFB) {
-        const int i = e >> 6, j = e & 63;
-        X[i][j] = pan[static_cast<size_t>(i) * K + j];
-    }
-    __syncthreads();
-    const int r = threadIdx.x;
-    for (int c = kFB - 1; c >= 0; --c) {
-        double v = X[r][c];
-        for (int c2 = c + 1; c2 < kFB; ++c2) v -= X[r][c2] * blk[static_cast<size_t>(c) * K + c2];
-        X[r][c] = v / blk[static_cast<size_t>(c) * K + c];
-    }
-    __syncthreads();
-    for (int e = threadIdx.x; e < kFB * kFB; e += kFB) {
-        const int i = e >> 6, j = e & 63;
-        pan[static_cast<size_t>(i) * K + j] = X[i][j];
-    }
+    const double* rinv = U + static_cast<size_t>(b0) * K + b0;
+    double acc[4][4] = {};
+    tile_mac(acc, kFB, [&](int k0) { fill_i_major(As, pan, K, k0, kFB, kFB); },
+             [&](int k0) { fill_i_major(Bs, rinv, K, k0, kFB, kFB); }, As, Bs);
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+#pragma unroll
+        for (int f = 0; f < 4; ++f) pan[static_cast<size_t>(tidx(ty, e)) * K + tidx(tx, f)] = acc[e][f];
 }
 
 // Trailing update: A[I, J] -= R[I, b] R[J, b]^T for the tiles I <= J in front of block b.
 __global__ void __launch_bounds__(256) gptq_chol_trail_kernel(double* __restrict__ A, int K, int b0) {
     const int bi = blockIdx.y, bj = blockIdx.x;
     if (bj < bi) return;
-    __shared__ double As[kFK][kFPad], Bs[kFK][kFPad];
+    __shared__ __align__(16) double As[kFK][kFPad], Bs[kFK][kFPad];
     double acc[4][4] = {};
     const double* pi = A + static_cast<size_t>(kFB) * bi * K + b0;
     const double* pj = A + static_cast<size_t>(kFB) * bj * K + b0;
@@ -172,29 +186,10 @@ __global__ void __launch_bounds__(256) gptq_chol_trail_kernel(double* __restrict
     for (int e = 0; e < 4; ++e)
 #pragma unroll
         for (int f = 0; f < 4; ++f)
-            A[static_cast<size_t>(kFB * bi + 4 * ty + e) * K + kFB * bj + 4 * tx + f] -= acc[e][f];
+            A[static_cast<size_t>(kFB * bi + tidx(ty, e)) * K + kFB * bj + tidx(tx, f)] -= acc[e][f];
 }
 
 // ------------------------------------------------------------------------------------------ U = R^-1
-// Diagonal blocks: column j of U_bb by back substitution, u_i = (delta_ij - sum_{i < l <= j} R_il u_l) / R_ii.
-__global__ void __launch_bounds__(kFB) gptq_inv_diag_kernel(const double* __restrict__ R, double* __restrict__ U, int K) {
-    __shared__ double Ub[kFB][kFPad];
-    const size_t off = static_cast<size_t>(kFB) * blockIdx.x * K + static_cast<size_t>(kFB) * blockIdx.x;
-    for (int e = threadIdx.x; e < kFB * kFB; e += kFB) Ub[e >> 6][e & 63] = 0.0;
-    __syncthreads();
-    const int j = threadIdx.x;
-    for (int i = j; i >= 0; --i) {                       // lanes of a warp read the same R_il for l <= their j
-        double v = i == j ? 1.0 : 0.0;
-        for (int l = i + 1; l <= j; ++l) v -= R[off + static_cast<size_t>(i) * K + l] * Ub[l][j];
-        Ub[i][j] = v / R[off + static_cast<size_t>(i) * K + i];
-    }
-    __syncthreads();
-    for (int e = threadIdx.x; e < kFB * kFB; e += kFB) {
-        const int i = e >> 6, j2 = e & 63;
-        U[off + static_cast<size_t>(i) * K + j2] = Ub[i][j2];
-    }
-}
-
 // Off-diagonal blocks by doubling: with the inverses of two neighbouring diagonal segments A (s x s at o) and
 // C (s2 x s2 at o + s) known, the block above C is  -A^-1 (B C^-1),  B = R[A rows, C columns].
 // First half: T = B C^-1, left in the unused mirror block U[C rows, A columns] (column tile j of the upper
@@ -203,7 +198,7 @@ __global__ void __launch_bounds__(256) gptq_inv_pair1_kernel(const double* R, do
     const int o = 2 * s * blockIdx.z, s2 = min(s, K - o - s);
     const int ti = blockIdx.y, tj = blockIdx.x;
     if (s2 <= 0 || kFB * tj >= s2) return;
-    __shared__ double As[kFK][kFPad], Bs[kFK][kFPad];
+    __shared__ __align__(16) double As[kFK][kFPad], Bs[kFK][kFPad];
     double acc[4][4] = {};
     const double* a = R + static_cast<size_t>(o + kFB * ti) * K + o + s;                 // B[i][k]
     const double* b = U + static_cast<size_t>(o + s) * K + o + s + kFB * tj;             // C^-1[k][j]
@@ -215,14 +210,14 @@ __global__ void __launch_bounds__(256) gptq_inv_pair1_kernel(const double* R, do
 #pragma unroll
     for (int e = 0; e < 4; ++e)
 #pragma unroll
-        for (int f = 0; f < 4; ++f) t[static_cast<size_t>(4 * tx + f) * K + 4 * ty + e] = acc[e][f];
+        for (int f = 0; f < 4; ++f) t[static_cast<size_t>(tidx(tx, f)) * K + tidx(ty, e)] = acc[e][f];
 }
 // Second half: U[A rows, C columns] = -A^-1 T (row tile i of the upper triangular A^-1 has its nonzeros in k >= 64 i).
 __global__ void __launch_bounds__(256) gptq_inv_pair2_kernel(double* U, int K, int s) {
     const int o = 2 * s * blockIdx.z, s2 = min(s, K - o - s);
     const int ti = blockIdx.y, tj = blockIdx.x;
     if (s2 <= 0 || kFB * tj >= s2) return;
-    __shared__ double As[kFK][kFPad], Bs[kFK][kFPad];
+    __shared__ __align__(16) double As[kFK][kFPad], Bs[kFK][kFPad];
     double acc[4][4] = {};
     const int kbeg = kFB * ti, klen = s - kbeg;
     const double* a = U + static_cast<size_t>(o + kFB * ti) * K + o + kbeg;              // A^-1[i][k], k from kbeg
@@ -234,7 +229,7 @@ __global__ void __launch_bounds__(256) gptq_inv_pair2_kernel(double* U, int K, i
 #pragma unroll
     for (int e = 0; e < 4; ++e)
 #pragma unroll
-        for (int f = 0; f < 4; ++f) out[static_cast<size_t>(4 * ty + e) * K + 4 * tx + f] = -acc[e][f];
+        for (int f = 0; f < 4; ++f) out[static_cast<size_t>(tidx(ty, e)) * K + tidx(tx, f)] = -acc[e][f];
 }
 // The mirror blocks held T: the lower triangle goes back to zero.
 __global__ void __launch_bounds__(256) gptq_zero_lower_kernel(double* U, int K) {
@@ -293,7 +288,7 @@ __global__ void __launch_bounds__(SLIM_GROUP) gptq_error_kernel(const double* __
 // w[n][k] -= sum_c E[n][c] U[c0 + c][k] for the columns k >= k0 = c0 + 128 (c ascending).
 __global__ void __launch_bounds__(256) gptq_update_kernel(double* __restrict__ w, const double* __restrict__ E,
                                                           const double* __restrict__ U, int N, int K, int c0) {
-    __shared__ double As[kFK][kFPad], Bs[kFK][kFPad];
+    __shared__ __align__(16) double As[kFK][kFPad], Bs[kFK][kFPad];
     const int n0 = kFB * blockIdx.y, k0 = c0 + SLIM_GROUP + kFB * blockIdx.x;
     double acc[4][4] = {};
     tile_mac(acc, SLIM_GROUP, [&](int kk) { fill_i_major(As, E + static_cast<size_t>(n0) * SLIM_GROUP, SLIM_GROUP, kk, SLIM_GROUP, N - n0); },
@@ -301,10 +296,10 @@ __global__ void __launch_bounds__(256) gptq_update_kernel(double* __restrict__ w
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        const int n = n0 + 4 * ty + e;
+        const int n = n0 + tidx(ty, e);
         if (n >= N) continue;
 #pragma unroll
-        for (int f = 0; f < 4; ++f) w[static_cast<size_t>(n) * K + k0 + 4 * tx + f] -= acc[e][f];
+        for (int f = 0; f < 4; ++f) w[static_cast<size_t>(n) * K + k0 + tidx(tx, f)] -= acc[e][f];
     }
 }
 
@@ -337,16 +332,15 @@ static int gptq_factor_into(const void* x, int T, int K, double lambda, uint8_t*
     const int nb = K / kFB;
     gptq_hessian_kernel<<<dim3(nb, nb), 256, 0, s>>>(static_cast<const __half*>(x), R, T, K);
     gptq_damp_kernel<<<1, 1024, 0, s>>>(R, dead, K, lambda);
+    SLIM_CUDA_TRY(cudaMemsetAsync(U, 0, static_cast<size_t>(K) * K * sizeof(double), s));
     for (int b = nb - 1; b >= 0; --b) {
-        gptq_chol_diag_kernel<<<1, 256, 0, s>>>(R, K, kFB * b);
+        gptq_chol_diag_kernel<<<1, 256, 0, s>>>(R, U, K, kFB * b);
         if (b > 0) {
-            gptq_chol_panel_kernel<<<b, kFB, 0, s>>>(R, K, kFB * b);
+            gptq_chol_panel_kernel<<<b, 256, 0, s>>>(R, U, K, kFB * b);
             gptq_chol_trail_kernel<<<dim3(b, b), 256, 0, s>>>(R, K, kFB * b);
         }
     }
     SLIM_CUDA_TRY(cudaGetLastError());
-    SLIM_CUDA_TRY(cudaMemsetAsync(U, 0, static_cast<size_t>(K) * K * sizeof(double), s));
-    gptq_inv_diag_kernel<<<nb, kFB, 0, s>>>(R, U, K);
     for (int seg = kFB; seg < K; seg *= 2) {
         const dim3 grid(seg / kFB, seg / kFB, (K + 2 * seg - 1) / (2 * seg));
         gptq_inv_pair1_kernel<<<grid, 256, 0, s>>>(R, U, K, seg);
