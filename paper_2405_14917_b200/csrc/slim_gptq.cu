@@ -26,14 +26,24 @@ constexpr int kFPad = kFB + 2;    // row stride of the staged operands: even, so
 // stage's first k), zero where the operand does not exist.  A thread owns the index pairs (2t, 2t + 1) and
 // (32 + 2t, 33 + 2t), so that the 16 threads of a row read consecutive 16-byte pieces of shared memory.
 __device__ __forceinline__ int tidx(int t, int e) { return 2 * t + (e & 1) + 32 * (e >> 1); }
-template <class FillA, class FillB>
-__device__ __forceinline__ void tile_mac(double (&acc)[4][4], int klen, FillA fill_a, FillB fill_b,
+// An operand gives load(k0, r): the thread's four elements of the stage that starts at k0, from global
+// memory, and store(S, r): their places in the staged array.  The next stage is loaded into registers
+// while the current one is multiplied.
+template <class OpA, class OpB>
+__device__ __forceinline__ void tile_mac(double (&acc)[4][4], int klen, const OpA& opa, const OpB& opb,
                                          double (*As)[kFPad], double (*Bs)[kFPad]) {
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    double ra[4], rb[4];
+    opa.load(0, ra);
+    opb.load(0, rb);
     for (int k0 = 0; k0 < klen; k0 += kFK) {
-        fill_a(k0);
-        fill_b(k0);
+        OpA::store(As, ra);
+        OpB::store(Bs, rb);
         __syncthreads();
+        if (k0 + kFK < klen) {
+            opa.load(k0 + kFK, ra);
+            opb.load(k0 + kFK, rb);
+        }
 #pragma unroll
         for (int k = 0; k < kFK; ++k) {
             const double2 a01 = *reinterpret_cast<const double2*>(&As[k][2 * ty]), a23 = *reinterpret_cast<const double2*>(&As[k][32 + 2 * ty]);
@@ -47,25 +57,43 @@ __device__ __forceinline__ void tile_mac(double (&acc)[4][4], int klen, FillA fi
         __syncthreads();
     }
 }
-// Operand stored with the tile index contiguous: element (k, i) = src[k * ld + i].
-__device__ __forceinline__ void fill_k_major(double (*S)[kFPad], const double* src, size_t ld, int k0, int kmax) {
-    const int k = threadIdx.x >> 4, i = (threadIdx.x & 15) * 4;
+// Operand stored with the tile index contiguous: element (k, i) = src[k * ld + i], k < kmax.
+struct OpK {
+    const double* src; size_t ld; int kmax;
+    __device__ __forceinline__ void load(int k0, double (&r)[4]) const {
+        const int k = k0 + (threadIdx.x >> 4), i = (threadIdx.x & 15) * 4;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) S[k][i + e] = k0 + k < kmax ? src[static_cast<size_t>(k0 + k) * ld + i + e] : 0.0;
-}
-__device__ __forceinline__ void fill_k_major_half(double (*S)[kFPad], const __half* src, size_t ld, int k0, int kmax) {
-    const int k = threadIdx.x >> 4, i = (threadIdx.x & 15) * 4;
+        for (int e = 0; e < 4; ++e) r[e] = k < kmax ? src[static_cast<size_t>(k) * ld + i + e] : 0.0;
+    }
+    __device__ __forceinline__ static void store(double (*S)[kFPad], const double (&r)[4]) {
+        const int k = threadIdx.x >> 4, i = (threadIdx.x & 15) * 4;
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
-        S[k][i + e] = k0 + k < kmax ? static_cast<double>(__half2float(src[static_cast<size_t>(k0 + k) * ld + i + e])) : 0.0;
-}
-// Operand stored with k contiguous: element (i, k) = src[i * ld + k]; rows i >= imax do not exist.
-__device__ __forceinline__ void fill_i_major(double (*S)[kFPad], const double* src, size_t ld, int k0, int kmax, int imax) {
-    const int i = threadIdx.x >> 2, k = (threadIdx.x & 3) * 4;
+        for (int e = 0; e < 4; ++e) S[k][i + e] = r[e];
+    }
+};
+struct OpKHalf {
+    const __half* src; size_t ld; int kmax;
+    __device__ __forceinline__ void load(int k0, double (&r)[4]) const {
+        const int k = k0 + (threadIdx.x >> 4), i = (threadIdx.x & 15) * 4;
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
-        S[k + e][i] = (k0 + k + e < kmax && i < imax) ? src[static_cast<size_t>(i) * ld + k0 + k + e] : 0.0;
-}
+        for (int e = 0; e < 4; ++e) r[e] = k < kmax ? static_cast<double>(__half2float(src[static_cast<size_t>(k) * ld + i + e])) : 0.0;
+    }
+    __device__ __forceinline__ static void store(double (*S)[kFPad], const double (&r)[4]) { OpK::store(S, r); }
+};
+// Operand stored with k contiguous: element (i, k) = src[i * ld + k], k < kmax; rows i >= imax do not exist.
+struct OpI {
+    const double* src; size_t ld; int kmax, imax;
+    __device__ __forceinline__ void load(int k0, double (&r)[4]) const {
+        const int i = threadIdx.x >> 2, k = k0 + (threadIdx.x & 3) * 4;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) r[e] = (k + e < kmax && i < imax) ? src[static_cast<size_t>(i) * ld + k + e] : 0.0;
+    }
+    __device__ __forceinline__ static void store(double (*S)[kFPad], const double (&r)[4]) {
+        const int i = threadIdx.x >> 2, k = (threadIdx.x & 3) * 4;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) S[k + e][i] = r[e];
+    }
+};
 
 // ------------------------------------------------------------------------------------------ Hessian
 // H[i][j] = (1/T) sum_t x[t][i] x[t][j] for the tiles on and above the diagonal (t ascending).
@@ -74,8 +102,7 @@ __global__ void __launch_bounds__(256) gptq_hessian_kernel(const __half* __restr
     if (bj < bi) return;
     __shared__ __align__(16) double As[kFK][kFPad], Bs[kFK][kFPad];
     double acc[4][4] = {};
-    tile_mac(acc, T, [&](int k0) { fill_k_major_half(As, x + kFB * bi, K, k0, T); },
-             [&](int k0) { fill_k_major_half(Bs, x + kFB * bj, K, k0, T); }, As, Bs);
+    tile_mac(acc, T, OpKHalf{x + kFB * bi, static_cast<size_t>(K), T}, OpKHalf{x + kFB * bj, static_cast<size_t>(K), T}, As, Bs);
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     const double inv = 1.0 / static_cast<double>(T);
 #pragma unroll
@@ -119,20 +146,55 @@ __global__ void __launch_bounds__(256) gptq_chol_diag_kernel(double* __restrict_
         S[i][j] = j >= i ? blk[static_cast<size_t>(i) * K + j] : 0.0;
     }
     __syncthreads();
+    // the factor runs on registers: thread (ty, tx) owns rows ty + 16 a, columns tx + 16 b
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    __shared__ double col[kFB], diag;
+    double r[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) r[a][b] = S[ty + 16 * a][tx + 16 * b];
     for (int c = kFB - 1; c >= 0; --c) {
-        const double d = sqrt(S[c][c]);
-        __syncthreads();
-        if (threadIdx.x < c) S[threadIdx.x][c] /= d;
-        else if (threadIdx.x == c) S[c][c] = d;
-        __syncthreads();
-        for (int i = ty; i < c; i += 16) {
-            const double ric = S[i][c];
-            for (int j = tx; j < c; j += 16)
-                if (j >= i) S[i][j] -= ric * S[j][c];
+        const int cs = c >> 4, cl = c & 15;
+        if (ty == cl && tx == cl) {
+            double v = 0.0;
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+                if (a == cs) v = r[a][a];
+            diag = sqrt(v);
         }
         __syncthreads();
+        const double d = diag;
+        if (tx == cl) {
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                const int i = ty + 16 * a;
+                double v = 0.0;
+#pragma unroll
+                for (int b = 0; b < 4; ++b)
+                    if (b == cs) v = r[a][b];
+                v = i < c ? v / d : (i == c ? d : v);
+#pragma unroll
+                for (int b = 0; b < 4; ++b)
+                    if (b == cs) r[a][b] = v;
+                col[i] = v;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int i = ty + 16 * a, j = tx + 16 * b;
+                if (j < c && i <= j) r[a][b] -= col[i] * col[j];
+            }
     }
+    __syncthreads();
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) S[ty + 16 * a][tx + 16 * b] = r[a][b];
+    __syncthreads();
     for (int e = threadIdx.x; e < kFB * kFB; e += 256) {
         const int i = e >> 6, j = e & 63;
         if (j >= i) blk[static_cast<size_t>(i) * K + j] = S[i][j];
@@ -162,8 +224,7 @@ __global__ void __launch_bounds__(256) gptq_chol_panel_kernel(double* __restrict
     double* pan = A + static_cast<size_t>(kFB) * blockIdx.x * K + b0;
     const double* rinv = U + static_cast<size_t>(b0) * K + b0;
     double acc[4][4] = {};
-    tile_mac(acc, kFB, [&](int k0) { fill_i_major(As, pan, K, k0, kFB, kFB); },
-             [&](int k0) { fill_i_major(Bs, rinv, K, k0, kFB, kFB); }, As, Bs);
+    tile_mac(acc, kFB, OpI{pan, static_cast<size_t>(K), kFB, kFB}, OpI{rinv, static_cast<size_t>(K), kFB, kFB}, As, Bs);
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
 #pragma unroll
     for (int e = 0; e < 4; ++e)
@@ -179,8 +240,7 @@ __global__ void __launch_bounds__(256) gptq_chol_trail_kernel(double* __restrict
     double acc[4][4] = {};
     const double* pi = A + static_cast<size_t>(kFB) * bi * K + b0;
     const double* pj = A + static_cast<size_t>(kFB) * bj * K + b0;
-    tile_mac(acc, kFB, [&](int k0) { fill_i_major(As, pi, K, k0, kFB, kFB); },
-             [&](int k0) { fill_i_major(Bs, pj, K, k0, kFB, kFB); }, As, Bs);
+    tile_mac(acc, kFB, OpI{pi, static_cast<size_t>(K), kFB, kFB}, OpI{pj, static_cast<size_t>(K), kFB, kFB}, As, Bs);
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
 #pragma unroll
     for (int e = 0; e < 4; ++e)
@@ -203,8 +263,7 @@ __global__ void __launch_bounds__(256) gptq_inv_pair1_kernel(const double* R, do
     const double* a = R + static_cast<size_t>(o + kFB * ti) * K + o + s;                 // B[i][k]
     const double* b = U + static_cast<size_t>(o + s) * K + o + s + kFB * tj;             // C^-1[k][j]
     const int klen = kFB * (tj + 1);
-    tile_mac(acc, klen, [&](int k0) { fill_i_major(As, a, K, k0, klen, kFB); },
-             [&](int k0) { fill_k_major(Bs, b, K, k0, klen); }, As, Bs);
+    tile_mac(acc, klen, OpI{a, static_cast<size_t>(K), klen, kFB}, OpK{b, static_cast<size_t>(K), klen}, As, Bs);
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     double* t = U + static_cast<size_t>(o + s + kFB * tj) * K + o + kFB * ti;            // T stored transposed: T^T[j][i]
 #pragma unroll
@@ -222,8 +281,7 @@ __global__ void __launch_bounds__(256) gptq_inv_pair2_kernel(double* U, int K, i
     const int kbeg = kFB * ti, klen = s - kbeg;
     const double* a = U + static_cast<size_t>(o + kFB * ti) * K + o + kbeg;              // A^-1[i][k], k from kbeg
     const double* b = U + static_cast<size_t>(o + s + kFB * tj) * K + o + kbeg;          // T^T[j][k]
-    tile_mac(acc, klen, [&](int k0) { fill_i_major(As, a, K, k0, klen, kFB); },
-             [&](int k0) { fill_i_major(Bs, b, K, k0, klen, kFB); }, As, Bs);
+    tile_mac(acc, klen, OpI{a, static_cast<size_t>(K), klen, kFB}, OpI{b, static_cast<size_t>(K), klen, kFB}, As, Bs);
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     double* out = U + static_cast<size_t>(o + kFB * ti) * K + o + s + kFB * tj;
 #pragma unroll
@@ -291,8 +349,8 @@ __global__ void __launch_bounds__(256) gptq_update_kernel(double* __restrict__ w
     __shared__ __align__(16) double As[kFK][kFPad], Bs[kFK][kFPad];
     const int n0 = kFB * blockIdx.y, k0 = c0 + SLIM_GROUP + kFB * blockIdx.x;
     double acc[4][4] = {};
-    tile_mac(acc, SLIM_GROUP, [&](int kk) { fill_i_major(As, E + static_cast<size_t>(n0) * SLIM_GROUP, SLIM_GROUP, kk, SLIM_GROUP, N - n0); },
-             [&](int kk) { fill_k_major(Bs, U + static_cast<size_t>(c0) * K + k0, K, kk, SLIM_GROUP); }, As, Bs);
+    tile_mac(acc, SLIM_GROUP, OpI{E + static_cast<size_t>(n0) * SLIM_GROUP, SLIM_GROUP, SLIM_GROUP, N - n0},
+             OpK{U + static_cast<size_t>(c0) * K + k0, static_cast<size_t>(K), SLIM_GROUP}, As, Bs);
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
