@@ -178,7 +178,7 @@ constexpr uint32_t kSetOffRing = (kSetOffDesc + kSetProducers * sizeof(SetLayer)
 // TPW: 16-row tiles per consumer warp (an item is 8 * TPW tiles); two tiles share the fragment loads and
 // the per-group bookkeeping.
 template <int NT, bool ONE, int TPW>
-__global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_constant__ SetParams p) {
+__global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(const __grid_constant__ SetParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -350,7 +350,8 @@ __global__ void __launch_bounds__(kSetThreads) gemv_set_kernel(const __grid_cons
                             const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
                             const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
                             if (ONE) {
-                                const float2 tk = sxe[0];                                  // (sum_k x, 2^(24-S)) of token 0
+                                const uint2 tkw = lds64(slot + p.off_e);                   // (sum_k x, 2^(24-S)) of token 0
+                                const float2 tk = make_float2(__uint_as_float(tkw.x), __uint_as_float(tkw.y));
                                 float e0 = d[t][0][0][0] + d[t][1][0][0], e2 = d[t][0][0][2] + d[t][1][0][2];
                                 if (CH == 4) {
                                     e0 += d[t][2 % CH][0][0] + d[t][3 % CH][0][0];

@@ -199,23 +199,50 @@ __global__ void __launch_bounds__(256) gptq_chol_diag_kernel(double* __restrict_
         const int i = e >> 6, j = e & 63;
         if (j >= i) blk[static_cast<size_t>(i) * K + j] = S[i][j];
     }
-    if (threadIdx.x < kFB) {
-        const int j = threadIdx.x;
-        double u[kFB];
+    // The inverse, in place in S.  16 x 16 diagonal blocks by back substitution (thread = one column,
+    // u_i = (delta_ij - sum_{l > i} R_il u_l) / R_ii, in registers); then two doubling levels: for neighbouring
+    // segments A, C with known inverses the block above C becomes -A^-1 (B C^-1).  The lower triangle of S is
+    // zero, so the sums run over whole segments.
+    __shared__ double Tm[32][33];
+    {
+        const int o = threadIdx.x & 48, jl = threadIdx.x & 15;      // threads 0..63: column jl of the block at o
+        double u[16];
+        if (threadIdx.x < kFB) {
 #pragma unroll
-        for (int i = kFB - 1; i >= 0; --i) {
-            double v0 = i == j ? 1.0 : 0.0, v1 = 0.0;          // rows below j stay zero: every u_l they meet is zero
+            for (int i = 15; i >= 0; --i) {
+                double v = i == jl ? 1.0 : 0.0;                    // rows below the column's own stay zero
 #pragma unroll
-            for (int l = i + 1; l < kFB; ++l) {
-                if ((l - i) & 1) v0 = fma(-S[i][l], u[l], v0);
-                else v1 = fma(-S[i][l], u[l], v1);
+                for (int l = i + 1; l < 16; ++l) v = fma(-S[o + i][o + l], u[l], v);
+                u[i] = v / S[o + i][o + i];
             }
-            u[i] = (v0 + v1) / S[i][i];
         }
-        double* ub = U + static_cast<size_t>(b0) * K + b0 + j;
+        __syncthreads();                                           // every column has read R before any is replaced
+        if (threadIdx.x < kFB) {
 #pragma unroll
-        for (int i = 0; i < kFB; ++i) ub[static_cast<size_t>(i) * K] = u[i];
+            for (int i = 0; i < 16; ++i) S[o + i][o + jl] = u[i];
+        }
+        __syncthreads();
     }
+    for (int seg = 16; seg < kFB; seg *= 2) {
+        // T = B C^-1 for every pair of segments: pair at o = 2 seg p, B = S[o .. o+seg)[o+seg .. o+2seg)
+        const int per_pair = seg * seg, n_out = per_pair * (kFB / (2 * seg));
+        for (int e = threadIdx.x; e < n_out; e += 256) {
+            const int pr = e / per_pair, q = e - pr * per_pair, i = q / seg, j = q - i * seg, o = 2 * seg * pr;
+            double v = 0.0;
+            for (int k = 0; k < seg; ++k) v = fma(S[o + i][o + seg + k], S[o + seg + k][o + seg + j], v);
+            Tm[(seg == 16 ? 16 * pr : 0) + i][j] = v;
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < n_out; e += 256) {
+            const int pr = e / per_pair, q = e - pr * per_pair, i = q / seg, j = q - i * seg, o = 2 * seg * pr;
+            double v = 0.0;
+            for (int k = 0; k < seg; ++k) v = fma(S[o + i][o + k], Tm[(seg == 16 ? 16 * pr : 0) + k][j], v);
+            S[o + i][o + seg + j] = -v;
+        }
+        __syncthreads();
+    }
+    double* ub = U + static_cast<size_t>(b0) * K + b0;
+    for (int e = threadIdx.x; e < kFB * kFB; e += 256) ub[static_cast<size_t>(e >> 6) * K + (e & 63)] = S[e >> 6][e & 63];
 }
 
 // Panel above the diagonal block: X R_bb^T = A[I, b], i.e. X = A[I, b] (R_bb^-1)^T, one 64 x 64 tile per CTA, in place.
