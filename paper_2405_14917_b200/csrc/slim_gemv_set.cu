@@ -54,8 +54,9 @@ struct SetLayer {
     int M, N, K, G;
     int pad1[2];
     int task0;             // first (token, group) staging task of the layer
-    int MP;                // tokens in the staged layout: 1 if every layer of the set has one token, else 8 or 16
-                           // for the whole set (absent tokens are staged as zeros, so the kernel reads without a test)
+    int MP;                // 256-byte pieces per slice in the staged layout: 8 or 16 = tokens of the f16 fragments for the
+                           // whole set (absent tokens are staged as zeros, so the kernel reads without a test); 2 if every
+                           // layer of the set has one token: the 8-bit digit form (stage_group_i8)
     uint16_t prefix[SLIM_MAX_GROUPS + 1];
     uint16_t pre3[SLIM_MAX_GROUPS + 1];   // 3-bit groups (two slices) before group j
     uint8_t bits[SLIM_MAX_GROUPS];
@@ -133,6 +134,72 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 __host__ __device__ inline size_t staged_group_offset(int j, int pre3, int M) {
     return 128u * static_cast<size_t>(j) + 256u * static_cast<size_t>(M) * static_cast<size_t>(j + pre3);
 }
+// ---- single-token sets: activations as signed 8-bit digits, the packed words as unsigned bytes ----------
+// With one token seven of the eight MMA columns are free, and an integer MMA takes four codes per
+// operand register where the f16 MMA takes two.  So for M = 1 the group's activations become the
+// fixed-point X_k = rint(x_k 2^S) (|X| <= 2^14), and every MMA's B operand holds three signed base-256
+// digits of X_k 2^shift in columns 0..2 (column 3 zero; columns 4..7 repeat them).  The A operand is the
+// packed word ANDed with a byte-wise mask: byte value = field * 2^(w i) for the fields at position i of
+// their byte (w = slice width), and shift = lo + Pc - w i makes every product carry the same 2^Pc, so all
+// positions and both slices of a 3-bit group add up in one integer accumulator: exact.
+__host__ __device__ constexpr int i8_pc(int b) { return b == 1 ? 3 : (b == 4 ? 4 : 6); }
+// Column of the group that meets byte bb of the A register half h (k < 16 or k >= 16) of MMA mi, lane column c.
+__device__ __forceinline__ int i8_column(int w, int mi, int h, int bb, int c) {
+    return w == 2 ? 32 * c + 16 * h + 4 * bb + mi
+         : w == 1 ? 32 * c + 8 * bb + mi + 4 * h
+                  : 32 * c + 8 * (2 * (mi >> 1) + h) + 2 * bb + (mi & 1);
+}
+// Record of one group: (sum_k x, 2^(-S - Pc)) then, per slice, 4 MMAs x [4 columns][4 lanes] x 8 bytes.
+__device__ __forceinline__ void stage_group_i8(const __half* xg, uint8_t* rec, int b, int lane) {
+    const uint2 raw = *reinterpret_cast<const uint2*>(xg + 4 * lane);
+    uint32_t mx = max(max(raw.x & 0x7fffu, (raw.x >> 16) & 0x7fffu), max(raw.y & 0x7fffu, (raw.y >> 16) & 0x7fffu));
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    const int S = mx == 0 ? 0 : 28 - max(static_cast<int>(mx >> 10), 1);     // largest |x| 2^S in [2^13, 2^14)
+    const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+    const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+    float sum = (f01.x + f01.y) + (f23.x + f23.y);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const float up = __int_as_float((127 + S) << 23);
+    const int pc = i8_pc(b);
+    for (int sl = 0; sl < slice_count(b); ++sl) {
+        const int w = slice_w(b, sl), lo = slice_lo(b, sl);
+        for (int idx = lane; idx < 64; idx += 32) {
+            const int mi = idx >> 4, n = (idx >> 2) & 3, c = idx & 3;
+            const int pos = w == 4 ? (mi & 1) : mi;
+            const int shift = lo + pc - w * pos;
+            uint32_t word[2];
+            for (int h = 0; h < 2; ++h) {
+                uint32_t v4 = 0;
+                for (int bb = 0; bb < 4; ++bb) {
+                    const int X = __float2int_rn(__half2float(xg[i8_column(w, mi, h, bb, c)]) * up);
+                    const int V = X << shift;
+                    const int d0 = static_cast<int8_t>(V & 0xff), V1 = (V - d0) >> 8;
+                    const int d1 = static_cast<int8_t>(V1 & 0xff), d2 = (V1 - d1) >> 8;
+                    const int dig = n == 0 ? d2 : (n == 1 ? d1 : (n == 2 ? d0 : 0));
+                    v4 |= static_cast<uint32_t>(dig & 0xff) << (8 * bb);
+                }
+                word[h] = v4;
+            }
+            *reinterpret_cast<uint2*>(rec + 128 + sl * 512 + mi * 128 + (n * 4 + c) * 8) = make_uint2(word[0], word[1]);
+        }
+    }
+    if (lane == 0) *reinterpret_cast<float2*>(rec) = make_float2(sum, __int_as_float((127 - S - pc) << 23));
+}
+// D (+)= A(u8, 16x32, row) * B(s8, 32x8, col), s32 accumulate.
+__device__ __forceinline__ void mma_i8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint2 b) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b.x), "r"(b.y));
+}
+__device__ __forceinline__ void mma_i8_first(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint2 b) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b.x), "r"(b.y), "r"(0));
+}
+
 // One warp per (layer, token, group): fragments and sums of the whole set, once.
 __global__ void __launch_bounds__(256) gemv_set_stage_kernel(const SetLayer* __restrict__ layers, uint8_t* ws, int n_layers, int n_tasks) {
     const int lane = threadIdx.x & 31;
@@ -147,6 +214,10 @@ __global__ void __launch_bounds__(256) gemv_set_stage_kernel(const SetLayer* __r
     const int pi = task - L.task0;
     const int m = pi / L.G, j = pi - m * L.G;        // m < MP
     uint8_t* grp = ws + L.x_off + staged_group_offset(j, L.pre3[j], L.MP);
+    if (L.MP == 2) {                                     // single-token set: the 8-bit form (task m = 1 is idle)
+        if (m == 0) stage_group_i8(L.x + j * SLIM_GROUP, grp, L.bits[j], lane);
+        return;
+    }
     float2* sxe = reinterpret_cast<float2*>(grp);
     if (m < L.M) {
         const float2 r = stage_group(L.x + static_cast<size_t>(m) * L.K + j * SLIM_GROUP, grp + 128, L.bits[j], m, L.MP, lane);
@@ -296,6 +367,68 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                         // layer the slot holds stale bytes: its accumulators are computed and never stored.
                         const uint32_t item0 = slot + kSetHeader + static_cast<uint32_t>(TPW * warp) * 256u * b;
                         const uint32_t xs_slot0 = slot + p.off_x;
+                        if constexpr (ONE) {
+                            // ---- one token: integer MMAs on byte-masked words (see stage_group_i8)
+                            int di[TPW][2][4];                       // two accumulation chains per tile
+                            const uint32_t xs_lane = xs_slot0 + ((gq & 3) * 4 + c) * 8;
+                            // one slice of width WD starting at unit `unit0`, digits at `xs`
+                            auto run_pass = [&](auto wtag, auto first_tag, int unit0, uint32_t xs) {
+                                constexpr int WD = decltype(wtag)::value;
+                                constexpr bool FIRST = decltype(first_tag)::value != 0;
+                                constexpr uint32_t kByteMask = 0x01010101u * ((1u << WD) - 1u);
+                                constexpr int NW = WD == 4 ? 4 : 2;     // words per row the MMAs of the slice draw on
+                                uint2 wd[TPW][NW];
+#pragma unroll
+                                for (int t = 0; t < TPW; ++t) {
+                                    const uint32_t item = item0 + t * 256u * b + 256u * unit0 + 8u * lane;
+                                    wd[t][0] = lds64(item);
+                                    if (WD == 1) {
+                                        wd[t][1] = make_uint2(wd[t][0].x >> 4, wd[t][0].y >> 4);
+                                    } else {
+#pragma unroll
+                                        for (int u = 1; u < NW; ++u) wd[t][u] = lds64(item + 256u * u);
+                                    }
+                                }
+#pragma unroll
+                                for (int mi = 0; mi < 4; ++mi) {
+                                    const uint2 bv = lds64(xs + mi * 128);
+                                    const int pos = WD == 4 ? (mi & 1) : mi, w0 = WD == 4 ? 2 * (mi >> 1) : 0;
+                                    const uint32_t m = kByteMask << (WD * pos);
+#pragma unroll
+                                    for (int t = 0; t < TPW; ++t) {
+                                        const uint32_t a0 = wd[t][w0].x & m, a1 = wd[t][w0].y & m;
+                                        const uint32_t a2 = wd[t][w0 + 1].x & m, a3 = wd[t][w0 + 1].y & m;
+                                        if (FIRST && mi < 2) mma_i8_first(di[t][mi & 1], a0, a1, a2, a3, bv);
+                                        else mma_i8(di[t][mi & 1], a0, a1, a2, a3, bv);
+                                    }
+                                }
+                            };
+                            switch (b) {
+                                case 1: run_pass(W1{}, WidthTag<1>{}, 0, xs_lane); break;
+                                case 2: run_pass(W2{}, WidthTag<1>{}, 0, xs_lane); break;
+                                case 3: run_pass(W2{}, WidthTag<1>{}, 0, xs_lane); run_pass(W1{}, WidthTag<0>{}, 2, xs_lane + 512); break;
+                                default: run_pass(W4{}, WidthTag<1>{}, 0, xs_lane); break;
+                            }
+                            // fold: columns (0, 1) hold the high and middle digit sums, (2, 3) the low one and zero; lanes
+                            // with even c see the first pair, odd c the second.  acc += s (D 2^(-S-Pc) - z sum_x)
+                            const uint2 tkw = lds64(slot + p.off_e);
+                            const float2 tk = make_float2(__uint_as_float(tkw.x), __uint_as_float(tkw.y));
+                            const float ka = (c & 1) ? 1.f : 65536.f, kb = (c & 1) ? 0.f : 256.f;
+#pragma unroll
+                            for (int t = 0; t < TPW; ++t) {
+                                const int tt = TPW * warp + t;
+                                const uint32_t s2 = lds32(slot + p.off_s + tt * 32 + gq * 4);
+                                const uint32_t z2 = lds32(slot + p.off_z + tt * 32 + gq * 4);
+                                const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
+                                const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
+                                float r0 = fmaf(static_cast<float>(di[t][0][0] + di[t][1][0]), ka, static_cast<float>(di[t][0][1] + di[t][1][1]) * kb);
+                                float r1 = fmaf(static_cast<float>(di[t][0][2] + di[t][1][2]), ka, static_cast<float>(di[t][0][3] + di[t][1][3]) * kb);
+                                r0 += __shfl_xor_sync(0xffffffffu, r0, 1);
+                                r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
+                                acc[t][0][0] = fmaf(sf.x, fmaf(-zf.x, tk.x, r0 * tk.y), acc[t][0][0]);
+                                acc[t][0][2] = fmaf(sf.y, fmaf(-zf.y, tk.x, r1 * tk.y), acc[t][0][2]);
+                            }
+                        } else {
                         constexpr int CH = NT == 1 ? (TPW == 1 ? 4 : 2) : 2;     // interleaved accumulation chains
                         float d[TPW][CH][NT][4];      // every chain is started by an MMA with a zero accumulator
 
@@ -377,6 +510,7 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                                 }
                             }
                         }
+                        }
                     }
                     __syncwarp();
                     if (lane == 0) sb::arrive(empty(s));
@@ -450,7 +584,7 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     sg->ws_bytes = 256;
     for (int l = 0; l < n_layers; ++l) sg->mmax = sg->mmax > layers[l].M ? sg->mmax : layers[l].M;
     sg->tpw = sg->mmax > 8 ? 1 : 2;
-    sg->mpad = sg->mmax <= 1 ? 1 : (sg->mmax <= 8 ? 8 : 16);
+    sg->mpad = sg->mmax <= 1 ? 2 : (sg->mmax <= 8 ? 8 : 16);    // one token: the 8-bit digit form, 512 bytes per slice
     const int tpi = kSetConsumers * sg->tpw;          // tiles per item
     for (int l = 0; l < n_layers; ++l) {
         const slim_layer& L = layers[l];
@@ -473,12 +607,12 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     sg->off_x = sg->off_e + 128;
     // a 3-bit group brings the fragments of two slices (a set whose widest group has 4 bits may hold one)
     sg->slot_bytes = static_cast<int>(align_to(static_cast<size_t>(sg->off_x) + (sg->bmax >= 3 ? 2 : 1) * 256 * sg->mpad, 128));
-    // as many CTAs per SM (kSetCtasPerSm at most) as still leaves each a ring of 6 slots
+    // as many CTAs per SM (kSetCtasPerSm at most) as still leaves each a ring of 5 slots
     const size_t per_sm = 224 * 1024;
     size_t budget = 0;
     for (sg->ctas_per_sm = kSetCtasPerSm; sg->ctas_per_sm >= 1; --sg->ctas_per_sm) {
         budget = per_sm / sg->ctas_per_sm - 1024 - kSetOffRing;   // 1 KB per CTA is reserved by the system
-        if (budget / sg->slot_bytes >= 6 || sg->ctas_per_sm == 1) break;
+        if (budget / sg->slot_bytes >= 5 || sg->ctas_per_sm == 1) break;
     }
     size_t slots = budget / sg->slot_bytes;
     if (slots > kSetMaxSlots) slots = kSetMaxSlots;
@@ -666,7 +800,7 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     prm.off_z = prm.off_s + tpi * 32;
     prm.off_e = prm.off_z + tpi * 32;
     prm.off_x = prm.off_e + 128;
-    if (prm.off_x + (info->max_bits >= 3 ? 2 : 1) * 256 * (info->max_tokens == 1 ? 1 : 8 * info->token_tiles) > info->slot_bytes) return SLIM_ERR_INVALID_ARG;
+    if (prm.off_x + (info->max_bits >= 3 ? 2 : 1) * 256 * (info->max_tokens == 1 ? 2 : 8 * info->token_tiles) > info->slot_bytes) return SLIM_ERR_INVALID_ARG;
 
     slim::gemv_set_stage_kernel<<<(info->stage_tasks + 7) / 8, 256, 0, s>>>(prm.layers, prm.ws, info->n_layers, info->stage_tasks);
     SLIM_CUDA_TRY(cudaGetLastError());

@@ -130,7 +130,7 @@ def test_layer_set_sizes_and_argument_errors(slim):
     # layer with more than one token, so every layer is staged eight tokens wide (absent tokens as zeros)
     want = 256 + (4 * 128 + (4 + 1) * 8 * 8 * 32) + (2 * 128 + (2 + 2) * 8 * 8 * 32)
     assert wb == want
-    assert _set_bytes(slim, [(1, 256, 512, [2, 3, 1, 2])])[2] == 256 + (4 * 128 + (4 + 1) * 8 * 1 * 32)      # one token: as is
+    assert _set_bytes(slim, [(1, 256, 512, [2, 3, 1, 2])])[2] == 256 + (4 * 128 + (4 + 1) * 512)              # one token: 8-bit digit form
     assert _set_bytes(slim, [(9, 256, 512, [2, 3, 1, 2])])[2] == 256 + (4 * 128 + (4 + 1) * 8 * 16 * 32)     # sixteen wide
     assert _set_bytes(slim, [])[0] == -1                                  # empty set
     assert _set_bytes(slim, [(0, 256, 512, [2] * 4)])[0] == -1            # no token
