@@ -369,7 +369,8 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                         const uint32_t xs_slot0 = slot + p.off_x;
                         if constexpr (ONE) {
                             // ---- one token: integer MMAs on byte-masked words (see stage_group_i8)
-                            int di[TPW][2][4];                       // two accumulation chains per tile
+                            constexpr int CHI = 1;                   // accumulation chains per tile
+                            int di[TPW][CHI][4];
                             const uint32_t xs_lane = xs_slot0 + ((gq & 3) * 4 + c) * 8;
                             // one slice of width WD starting at unit `unit0`, digits at `xs`
                             auto run_pass = [&](auto wtag, auto first_tag, int unit0, uint32_t xs) {
@@ -398,8 +399,8 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                                     for (int t = 0; t < TPW; ++t) {
                                         const uint32_t a0 = wd[t][w0].x & m, a1 = wd[t][w0].y & m;
                                         const uint32_t a2 = wd[t][w0 + 1].x & m, a3 = wd[t][w0 + 1].y & m;
-                                        if (FIRST && mi < 2) mma_i8_first(di[t][mi & 1], a0, a1, a2, a3, bv);
-                                        else mma_i8(di[t][mi & 1], a0, a1, a2, a3, bv);
+                                        if (FIRST && mi < CHI) mma_i8_first(di[t][mi & (CHI - 1)], a0, a1, a2, a3, bv);
+                                        else mma_i8(di[t][mi & (CHI - 1)], a0, a1, a2, a3, bv);
                                     }
                                 }
                             };
@@ -409,25 +410,34 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                                 case 3: run_pass(W2{}, WidthTag<1>{}, 0, xs_lane); run_pass(W1{}, WidthTag<0>{}, 2, xs_lane + 512); break;
                                 default: run_pass(W4{}, WidthTag<1>{}, 0, xs_lane); break;
                             }
-                            // fold: columns (0, 1) hold the high and middle digit sums, (2, 3) the low one and zero; lanes
-                            // with even c see the first pair, odd c the second.  acc += s (D 2^(-S-Pc) - z sum_x)
+                            // fold: columns (0, 1) hold the high and middle digit sums, (2, 3) the low one and zero, (4..7)
+                            // repeat them; lanes with even c see a (high, middle) pair, odd c a (low, 0) pair.  Every lane
+                            // holds the sums of all the warp's tiles, so the lane pair c >> 1 folds tile c >> 1 only:
+                            // acc += s (D 2^(-S-Pc) - z sum_x)
+                            static_assert(TPW <= 2, "one lane pair per tile");
                             const uint2 tkw = lds64(slot + p.off_e);
-                            const float2 tk = make_float2(__uint_as_float(tkw.x), __uint_as_float(tkw.y));
-                            const float ka = (c & 1) ? 1.f : 65536.f, kb = (c & 1) ? 0.f : 256.f;
+                            const float sum_x = __uint_as_float(tkw.x), e = __uint_as_float(tkw.y);
+                            const float ka = (c & 1) ? e : 65536.f * e, kb = (c & 1) ? 0.f : 256.f * e;
+                            const int tsel = TPW == 2 ? (c >> 1) : 0;
+                            int dsel[4];
 #pragma unroll
-                            for (int t = 0; t < TPW; ++t) {
-                                const int tt = TPW * warp + t;
-                                const uint32_t s2 = lds32(slot + p.off_s + tt * 32 + gq * 4);
-                                const uint32_t z2 = lds32(slot + p.off_z + tt * 32 + gq * 4);
-                                const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
-                                const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
-                                float r0 = fmaf(static_cast<float>(di[t][0][0] + di[t][1][0]), ka, static_cast<float>(di[t][0][1] + di[t][1][1]) * kb);
-                                float r1 = fmaf(static_cast<float>(di[t][0][2] + di[t][1][2]), ka, static_cast<float>(di[t][0][3] + di[t][1][3]) * kb);
-                                r0 += __shfl_xor_sync(0xffffffffu, r0, 1);
-                                r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
-                                acc[t][0][0] = fmaf(sf.x, fmaf(-zf.x, tk.x, r0 * tk.y), acc[t][0][0]);
-                                acc[t][0][2] = fmaf(sf.y, fmaf(-zf.y, tk.x, r1 * tk.y), acc[t][0][2]);
+                            for (int r = 0; r < 4; ++r) {
+                                int v0 = di[0][0][r], v1 = di[TPW - 1][0][r];
+#pragma unroll
+                                for (int ch = 1; ch < CHI; ++ch) { v0 += di[0][ch][r]; v1 += di[TPW - 1][ch][r]; }
+                                dsel[r] = tsel ? v1 : v0;
                             }
+                            const int tt = TPW * warp + tsel;
+                            const uint32_t s2 = lds32(slot + p.off_s + tt * 32 + gq * 4);
+                            const uint32_t z2 = lds32(slot + p.off_z + tt * 32 + gq * 4);
+                            const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
+                            const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
+                            float r0 = fmaf(static_cast<float>(dsel[0]), ka, static_cast<float>(dsel[1]) * kb);
+                            float r1 = fmaf(static_cast<float>(dsel[2]), ka, static_cast<float>(dsel[3]) * kb);
+                            r0 += __shfl_xor_sync(0xffffffffu, r0, 1);
+                            r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
+                            acc[0][0][0] = fmaf(sf.x, fmaf(-zf.x, sum_x, r0), acc[0][0][0]);
+                            acc[0][0][2] = fmaf(sf.y, fmaf(-zf.y, sum_x, r1), acc[0][0][2]);
                         } else {
                         constexpr int CH = NT == 1 ? (TPW == 1 ? 4 : 2) : 2;     // interleaved accumulation chains
                         float d[TPW][CH][NT][4];      // every chain is started by an MMA with a zero accumulator
@@ -523,7 +533,8 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                         if (t >= n_act) break;
                         __half* yrow = ybase + 16 * (tile0 + t) + 2 * gq;
                         if (ONE) {
-                            if (c == 0) *reinterpret_cast<__half2*>(yrow) = __floats2half2_rn(acc[t][0][0], acc[t][0][2]);
+                            // the lane pair c >> 1 holds tile c >> 1 (in acc[0]); its even lane stores
+                            if (c == 2 * t) *reinterpret_cast<__half2*>(yrow) = __floats2half2_rn(acc[0][0][0], acc[0][0][2]);
                         } else {
 #pragma unroll
                             for (int n = 0; n < NT; ++n) {
