@@ -369,7 +369,7 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                         const uint32_t xs_slot0 = slot + p.off_x;
                         if constexpr (ONE) {
                             // ---- one token: integer MMAs on byte-masked words (see stage_group_i8)
-                            constexpr int CHI = 1;                   // accumulation chains per tile
+                            constexpr int CHI = 2;                   // accumulation chains per tile
                             int di[TPW][CHI][4];
                             const uint32_t xs_lane = xs_slot0 + ((gq & 3) * 4 + c) * 8;
                             // one slice of width WD starting at unit `unit0`, digits at `xs`
