@@ -40,9 +40,9 @@ FALLBACK_TENSOR_TFLOPS = 1400.0
 # dram__bytes_write.sum), keyed by the sha256 of the kernel source it was taken from.  A kernel
 # that has changed since reports null.
 NCU_TRAFFIC = {
-    # layer-set kernel, 4 blocks of the LLaMA-7B sweep (28 layers, avg 2-bit, M = 1): 228,306,944 B read +
-    # 4,196,864 B written per launch (algorithmic 228,297,816 B); scaled to the full sweep by the algorithmic bytes
-    "c3a6fafb9c2edd19d878709a54b3f6291e8bd701d97dd2c27447f0aabe38949a": {"layer": "4 blocks", "traffic_bytes": 232503808, "algorithmic_bytes": 228297816},
+    # layer-set kernel, 4 blocks of the LLaMA-7B sweep (28 layers, avg 2-bit, M = 1): 228,629,760 B read +
+    # 4,367,360 B written per launch (algorithmic 228,297,816 B); scaled to the full sweep by the algorithmic bytes
+    "e25960915e353f61dfff3a350b7b271bfc027a892e28cdcf869cb410ab6b1a0e": {"layer": "4 blocks", "traffic_bytes": 232997120, "algorithmic_bytes": 228297816},
     # 4096x4096 layer, avg 2-bit, M = 1: 4,755,200 B read + 0 written per launch (algorithmic 4,735,008 B);
     # scaled to the sweep's average launch by the algorithmic bytes (traffic grows with the layer size)
     "4b06a5d5b512621bbe525cb3d0c66822ff452c130a671af895469c10fb834593": {"layer": "4096x4096", "traffic_bytes": 4755200, "algorithmic_bytes": 4735008},
@@ -660,7 +660,8 @@ def run_ours(args, spec):
                   f"mixed-precision dequant GEMV GB/s at M={M} ({spec['model']} layer set, avg {spec['avg_bits']}-bit, g=128)",
         "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f16 (mma.sync m16n8k16 on raw code fields, f32 accumulate)", "data": "synthetic",
+        "dtype": ("s32 (mma.sync m16n8k32 u8 x s8: byte-masked code words against base-256 digits of fixed-point x; f32 fold)"
+                  if use_set and M == 1 else "f16 (mma.sync m16n8k16 on raw code fields, f32 accumulate)"), "data": "synthetic",
         "config": {"workload": args.workload, "layers": len(layers), "M": M, "avg_bits": spec["avg_bits"], "g": wl.GROUP,
                    "algorithmic_bytes_per_step": alg_bytes, "l2": f"distinct layers, {alg_bytes / 1e9:.2f} GB per step >> L2",
                    "launch": ("CUDA graph of the layer-set launch: one persistent kernel for the whole sweep "

@@ -150,7 +150,7 @@ __device__ __forceinline__ int i8_column(int w, int mi, int h, int bb, int c) {
                   : 32 * c + 8 * (2 * (mi >> 1) + h) + 2 * bb + (mi & 1);
 }
 // Record of one group: (sum_k x, 2^(-S - Pc)) then, per slice, 4 MMAs x [4 columns][4 lanes] x 8 bytes.
-__device__ __forceinline__ void stage_group_i8(const __half* xg, uint8_t* rec, int b, int lane) {
+__device__ __forceinline__ void stage_group_i8(const __half* xg, uint8_t* rec, int b, int lane, int* Xs) {
     const uint2 raw = *reinterpret_cast<const uint2*>(xg + 4 * lane);
     uint32_t mx = max(max(raw.x & 0x7fffu, (raw.x >> 16) & 0x7fffu), max(raw.y & 0x7fffu, (raw.y >> 16) & 0x7fffu));
     mx = __reduce_max_sync(0xffffffffu, mx);
@@ -162,6 +162,11 @@ __device__ __forceinline__ void stage_group_i8(const __half* xg, uint8_t* rec, i
     for (int o = 1; o < 32; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
     const float up = __int_as_float((127 + S) << 23);
     const int pc = i8_pc(b);
+    Xs[4 * lane + 0] = __float2int_rn(f01.x * up);       // the group's fixed-point activations, once
+    Xs[4 * lane + 1] = __float2int_rn(f01.y * up);
+    Xs[4 * lane + 2] = __float2int_rn(f23.x * up);
+    Xs[4 * lane + 3] = __float2int_rn(f23.y * up);
+    __syncwarp();
     for (int sl = 0; sl < slice_count(b); ++sl) {
         const int w = slice_w(b, sl), lo = slice_lo(b, sl);
         for (int idx = lane; idx < 64; idx += 32) {
@@ -172,7 +177,7 @@ __device__ __forceinline__ void stage_group_i8(const __half* xg, uint8_t* rec, i
             for (int h = 0; h < 2; ++h) {
                 uint32_t v4 = 0;
                 for (int bb = 0; bb < 4; ++bb) {
-                    const int X = __float2int_rn(__half2float(xg[i8_column(w, mi, h, bb, c)]) * up);
+                    const int X = Xs[i8_column(w, mi, h, bb, c)];
                     const int V = X << shift;
                     const int d0 = static_cast<int8_t>(V & 0xff), V1 = (V - d0) >> 8;
                     const int d1 = static_cast<int8_t>(V1 & 0xff), d2 = (V1 - d1) >> 8;
@@ -214,8 +219,9 @@ __global__ void __launch_bounds__(256) gemv_set_stage_kernel(const SetLayer* __r
     const int pi = task - L.task0;
     const int m = pi / L.G, j = pi - m * L.G;        // m < MP
     uint8_t* grp = ws + L.x_off + staged_group_offset(j, L.pre3[j], L.MP);
-    if (L.MP == 2) {                                     // single-token set: the 8-bit form (task m = 1 is idle)
-        if (m == 0) stage_group_i8(L.x + j * SLIM_GROUP, grp, L.bits[j], lane);
+    if (L.MP == 2) {                                     // single-token set: the 8-bit form, one task per group
+        __shared__ int Xs[8][SLIM_GROUP];
+        stage_group_i8(L.x + j * SLIM_GROUP, grp, L.bits[j], lane, Xs[threadIdx.x >> 5]);
         return;
     }
     float2* sxe = reinterpret_cast<float2*>(grp);
@@ -607,7 +613,7 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
         for (int j = 0; j < gt.G; ++j) sg->bmax = sg->bmax > gt.bits[j] ? sg->bmax : gt.bits[j];
         const int items = ((L.N >> 4) + tpi - 1) / tpi;
         sg->n_items += items;
-        sg->n_tasks += static_cast<long long>(sg->mpad) * gt.G;
+        sg->n_tasks += static_cast<long long>(sg->mpad == 2 ? 1 : sg->mpad) * gt.G;   // staging tasks: (token, group)
         sg->ws_bytes += layer_ws_bytes(sg->mpad, gt);
     }
     if (sg->n_items > 0x3fffffff || sg->n_tasks > 0x3fffffff) return SLIM_ERR_UNSUPPORTED;
@@ -732,7 +738,7 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
             items.push_back(it);
             cost.push_back(slim::item_cost(th < tpi ? th : tpi, gt));
         }
-        task += sg.mpad * gt.G;
+        task += (sg.mpad == 2 ? 1 : sg.mpad) * gt.G;
     }
     // The deal: items by falling cost (equal costs in the set's order), each to the CTA that has the
     // least so far (the lowest-numbered of equals).  Within a CTA the heavy items come first.
