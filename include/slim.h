@@ -169,7 +169,8 @@ int slim_mpq_gemm_static(const void* x, const void* packed, const uint8_t* bits_
  * A set in which EVERY layer has M = 1 runs on integer tensor-core instructions: per group of 128
  * columns x is first rounded to fixed point with 14 to 15 significant bits relative to the group's
  * largest |x_k| (error per element at most 2^-14 of that maximum, about 1e-4 of the output's norm);
- * the sums over the group are then exact.  Sets with more tokens multiply the fp16 x as it is.
+ * the sums over the group are then exact; x must be finite.  Sets with more tokens multiply the
+ * fp16 x as it is.
  * N > 0 a multiple of 16, K > 0 a multiple of 128. */
 typedef struct slim_layer {
     const void* x;             /* device fp16 [M][K] */
