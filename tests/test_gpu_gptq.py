@@ -19,7 +19,9 @@ def _layer(N, K, T, name="gptq-gpu", block=0):
     return wl.make_weight(seed, N, K), wl.make_calibration_x(seed, T, K)
 
 
-@pytest.mark.parametrize("K,T", [(128, 16), (256, 300), (512, 100), (1024, 1500)])
+# 384, 640 and 1408 columns: a number of 64-column blocks that is not a power of two (ragged last segments of the
+# doubling inverse)
+@pytest.mark.parametrize("K,T", [(128, 16), (256, 300), (384, 200), (512, 100), (640, 64), (1024, 1500), (1408, 700)])
 def test_factor_against_the_library_cholesky_of_the_inverse(K, T):
     slim = _slim()
     _, x = _layer(4, K, T)
@@ -47,7 +49,8 @@ def _check_quantize(W, x, bits, quantizer, lam=0.01):
 
 
 @pytest.mark.parametrize("N,K,T,bits", [(64, 512, 128, [2, 1, 3, 2]), (272, 1024, 300, [3, 2, 4, 3, 3, 2, 4, 3]),
-                                        (16, 128, 40, [2]), (130, 256, 64, [1, 3])])
+                                        (16, 128, 40, [2]), (130, 256, 64, [1, 3]), (48, 384, 500, [3, 2, 1]),
+                                        (32, 1408, 256, [2, 3, 1, 2, 3, 2, 2, 1, 3, 2, 2])])
 @pytest.mark.parametrize("quantizer", ["minmax", "sqc"])
 def test_quantize_matches_the_oracle(N, K, T, bits, quantizer):
     if N % 16:
