@@ -108,6 +108,23 @@ def test_llama7b_layer_full_size_on_sampled_rows():
     assert (got == c_ref).all(), f"{(got != c_ref).sum()} codes differ"
 
 
+def test_llama7b_down_projection_shape_on_sampled_rows():
+    """4096 x 11008 (172 blocks of 64 columns: ragged segments at several levels of the doubling inverse), SQC."""
+    slim = _slim()
+    N, K = 4096, 11008
+    seed = wl.layer_seed("llama-7b", "down_proj", 0)
+    W = wl.make_weight(seed, N, K)
+    x = wl.make_calibration_x(seed, 1024, K)
+    bits = orc.allocate_bits(orc.group_salience(W, wl.make_act_norms(seed, K)), 2)
+    codes, scales, zeros = slim.gptq_quantize(torch.from_numpy(W).cuda(), torch.from_numpy(x).cuda(), bits, 0.01, "sqc")
+    rows = np.array([0, 17, 2049, 4095])
+    c_ref, s_ref, z_ref, _ = orc.gptq_quantize(W[rows], x, bits, 0.01, "sqc")
+    assert (scales.cpu().numpy()[:, rows].view(np.uint16) == s_ref.view(np.uint16)).all()
+    assert (zeros.cpu().numpy()[:, rows].view(np.uint16) == z_ref.view(np.uint16)).all()
+    got = codes.cpu().numpy()[rows]
+    assert (got == c_ref).all(), f"{(got != c_ref).sum()} codes differ"
+
+
 def test_rejects_bad_arguments():
     slim = _slim()
     W, x = _layer(16, 256, 32)
