@@ -93,6 +93,14 @@ int slim_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
  * then undefined), or SLIM_ERR_CUDA. */
 int slim_workspace_status(void* workspace, void* stream);
 
+/* Self-test of the device-side time-out path.  (No counterpart in the paper: it exercises the status-word
+ * contract of this header.)  Enqueues one warp that waits, with the bounded wait the persistent kernels use, on a
+ * barrier that nothing ever signals; after limit_us microseconds (1 .. 100000) the wait gives up, the kernel sets
+ * the workspace status word the way a real time-out does, and returns by itself.  slim_workspace_status on that
+ * workspace then reports SLIM_ERR_TIMEOUT once and clears the word; the workspace stays usable.  `workspace` at
+ * least 256 bytes, 16-byte aligned. */
+int slim_selftest_wait_timeout(void* workspace, size_t workspace_bytes, unsigned int limit_us, void* stream);
+
 /* Packs unpacked codes into the format above (the storage step of App. B.2: "packs the weights
  * ... into integer-compressed representations based on the precision of different groups").
  * Integer work, deterministic; codes with bits above b_j set are masked to b_j bits. */
@@ -167,10 +175,12 @@ int slim_mpq_gemm_static(const void* x, const void* packed, const uint8_t* bits_
  * Every layer gets the y = x * W-hat^T of slim_mpq_gemv (same products, fp32 accumulation in a
  * different order, fp16 output); the results are deterministic for a given (set, device).
  * A set in which EVERY layer has M = 1 runs on integer tensor-core instructions: per group of 128
- * columns x is first rounded to fixed point with 14 to 15 significant bits relative to the group's
- * largest |x_k| (error per element at most 2^-14 of that maximum, about 1e-4 of the output's norm);
- * the sums over the group are then exact; x must be finite.  Sets with more tokens multiply the
- * fp16 x as it is.
+ * columns x is first rounded to fixed point with 22 bits relative to the group's largest |x_k|, so an
+ * fp16 activation within a factor 2^11 of that maximum is taken exactly and a smaller one with an error
+ * of at most 2^-22 of the maximum; the sums over the group are then exact.  Per output row n this adds at
+ * most  sum over groups of 2^-22 max|x_group| sum_{k in group} |w-hat[n][k]|  to the error of the fp16
+ * path (slim_mpq_gemv multiplies the fp16 x as it is); x must be finite.  Sets with more tokens multiply
+ * the fp16 x as it is.
  * N > 0 a multiple of 16, K > 0 a multiple of 128. */
 typedef struct slim_layer {
     const void* x;             /* device fp16 [M][K] */

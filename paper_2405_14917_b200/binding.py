@@ -48,6 +48,7 @@ def lib():
             "slim_workspace_bytes": [i, i, i, i, vp, ctypes.POINTER(sz)],
             "slim_workspace_init": [vp, sz, vp],
             "slim_workspace_status": [vp, vp],
+            "slim_selftest_wait_timeout": [vp, sz, ctypes.c_uint, vp],
             "slim_pack_weights": [vp, vp, vp, i, i, i, vp],
             "slim_dequant": [vp, vp, vp, vp, vp, i, i, i, vp],
             "slim_mpq_gemv": [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp],
@@ -140,6 +141,12 @@ def workspace_status(workspace: torch.Tensor) -> None:
     """Synchronises; raises SlimError(SLIM_ERR_TIMEOUT) if a kernel gave up a bounded wait."""
     p = _dev(workspace, torch.uint8, "workspace")
     _check("slim_workspace_status", lib().slim_workspace_status(p, _stream(workspace)))
+
+
+def selftest_wait_timeout(workspace: torch.Tensor, limit_us: int = 1000) -> None:
+    """Enqueues the kernel whose bounded wait runs out after limit_us microseconds (slim_selftest_wait_timeout)."""
+    p = _dev(workspace, torch.uint8, "workspace")
+    _check("slim_selftest_wait_timeout", lib().slim_selftest_wait_timeout(p, workspace.numel(), int(limit_us), _stream(workspace)))
 
 
 def new_workspace(M: int, N: int, K: int, bits, device="cuda") -> torch.Tensor:

@@ -32,6 +32,8 @@
 // leaves before its partner has stopped signalling it.
 #include "slim_common.cuh"
 
+#include <atomic>
+
 #include <cuda.h>
 #include <cstring>
 
@@ -617,6 +619,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
         bool ok = true;
         const uint32_t d_empty_leader = g::map_to_cta(d_empty, 0);
         auto epi_sync = [] { asm volatile("bar.sync 1, 128;" ::: "memory"); };
+        // barrier of the 128 epilogue threads that also ORs a flag: every thread gets the same answer, so the four
+        // warps leave, or go on to the next named barrier, together
+        auto epi_any = [](bool v) {
+            uint32_t r;
+            asm volatile("{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.or.pred p, 1, 128, q;\n selp.u32 %0, 1, 0, p;\n}\n"
+                         : "=r"(r) : "r"(static_cast<uint32_t>(v)) : "memory");
+            return r != 0;
+        };
         for (long long u = u0; u < u1 && ok;) {
             const int tile = static_cast<int>(u / G), gb = static_cast<int>(u - static_cast<long long>(tile) * G);
             const int ge = static_cast<int>(min(static_cast<long long>(G), gb + (u1 - u)));
@@ -634,7 +644,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
                 }
             }
             auto peer_active = [&](int k) { return range_begin(cl + k) < range_begin(cl + k + 1); };
-            if (!g::mbar_wait_long(d_full, phd, abort)) { ok = false; break; }
+            bool gave_up = !g::mbar_wait_long(d_full, phd, abort);
+            gave_up = epi_any(gave_up);          // named barriers may follow, now or in a later unit: decide once for all
+            if (gave_up) { ok = false; break; }
             g::tc_fence_after();
             if (npeer > 0) {
                 if (et == 0) {
@@ -648,8 +660,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
                     }
                     __threadfence();
                 }
-                epi_sync();
-                if (*abort != 0) { ok = false; break; }
+                if (epi_any(et == 0 && *abort != 0)) { ok = false; break; }   // thread 0's view of the flag, for everyone
             }
             // slot layout [token][row]: a warp touches 32 consecutive floats per access
             float* my_slot = p.partials + static_cast<size_t>(blockIdx.x) * (TOK * kRowsPerCta) + 32 * q + lane;
@@ -759,7 +770,7 @@ static int gemm_sm_count() {
 // CTA pairs that can be resident at once (the stream-K hand-over needs all of them running).
 template <int TOK>
 static int max_resident_pairs() {
-    static int cached[64] = {0};
+    static std::atomic<int> cached[64];       // zero-initialised; set-up is idempotent, so a race repeats it harmlessly
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
     if (cached[dev] == 0) {
@@ -821,7 +832,7 @@ size_t gemm_workspace_bytes(int M, int N, int G) { return plan_gemm(M, N, G).wor
 
 template <int TOK>
 static cudaError_t launch_gemm(const CUtensorMap& map, const GemmParams& prm, int grid, cudaStream_t stream) {
-    static bool attr_set[64] = {false};
+    static std::atomic<bool> attr_set[64];    // zero-initialised; set-up is idempotent, so a race repeats it harmlessly
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -902,29 +913,33 @@ extern "C" int slim_mpq_gemm_static(const void* x, const void* packed, const uin
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;
     if (status_out != nullptr && (reinterpret_cast<uintptr_t>(status_out) & 3u) != 0) return SLIM_ERR_ALIGNMENT;
-    if (M == 0 || N == 0 || K == 0)   // nothing needs scratch: the ordinary entry point handles these
-        return slim_mpq_gemm(x, packed, bits_host, scales, zeros, y, M, N, K, g, nullptr, 0, stream);
+    if (M == 0 || N == 0 || K == 0) {  // nothing needs scratch: the ordinary entry point handles these
+        const int rc0 = slim_mpq_gemm(x, packed, bits_host, scales, zeros, y, M, N, K, g, nullptr, 0, stream);
+        if (rc0 == SLIM_OK && status_out != nullptr)
+            SLIM_CUDA_TRY(cudaMemsetAsync(status_out, 0, sizeof(unsigned int), static_cast<cudaStream_t>(stream)));
+        return rc0;
+    }
     // what this shape wants on this device; more than the array holds is refused, never truncated
     if (slim::gemm_workspace_bytes(M, N, gt.G) > static_cast<size_t>(SLIM_STATIC_SCRATCH_MAX)) return SLIM_ERR_STATIC_SCRATCH;
 
     // Device address of the array, looked up once per device (the array's name is only a
     // host-side handle here and must not be handed to a kernel).
-    static void* scratch_ptr[64] = {nullptr};
+    static std::atomic<void*> scratch_ptr[64];   // zero-initialised; the look-up is idempotent
     int dev = 0;
     SLIM_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return SLIM_ERR_UNSUPPORTED;
-    if (scratch_ptr[dev] == nullptr) {
+    if (scratch_ptr[dev].load() == nullptr) {
         void* ptr = nullptr;
         SLIM_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
-        scratch_ptr[dev] = ptr;
+        scratch_ptr[dev].store(ptr);
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // the array keeps what the last call left: the status word and the flags must start at zero
-    SLIM_CUDA_TRY(cudaMemsetAsync(scratch_ptr[dev], 0, slim::kGemmWsPartials, s));
-    const int rc = slim_mpq_gemm(x, packed, bits_host, scales, zeros, y, M, N, K, g, scratch_ptr[dev],
+    SLIM_CUDA_TRY(cudaMemsetAsync(scratch_ptr[dev].load(), 0, slim::kGemmWsPartials, s));
+    const int rc = slim_mpq_gemm(x, packed, bits_host, scales, zeros, y, M, N, K, g, scratch_ptr[dev].load(),
                                  SLIM_STATIC_SCRATCH_MAX, stream);
     if (rc != SLIM_OK) return rc;
     if (status_out != nullptr)
-        SLIM_CUDA_TRY(cudaMemcpyAsync(status_out, scratch_ptr[dev], sizeof(unsigned int), cudaMemcpyDeviceToDevice, s));
+        SLIM_CUDA_TRY(cudaMemcpyAsync(status_out, scratch_ptr[dev].load(), sizeof(unsigned int), cudaMemcpyDeviceToDevice, s));
     return SLIM_OK;
 }

@@ -35,6 +35,8 @@
 //    memory and adds them in rank order (deterministic); no global scratch.
 #include "slim_gemv_dev.cuh"
 
+#include <atomic>
+
 #include <cstring>
 
 namespace slim {
@@ -194,6 +196,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
     // ---- put the first chunk in flight, then wait until the previous kernel has finished before
     // x or y are touched
     issue_weights(0);
+    if (p.CS > 1) cluster_arrive_relaxed();          // "this CTA runs": awaited before the first store into a peer's shared memory
     pdl_wait();
     issue_x(0);
     if (!PRE)
@@ -313,6 +316,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
         const int row = 16 * (rb * T + t) + 2 * (rem & 7);
         if (row < N) *reinterpret_cast<__half2*>(p.y + static_cast<size_t>(rem >> 3) * N + row) = __floats2half2_rn(v.x, v.y);
     };
+    if (CS > 1) cluster_wait();                       // every CTA of the cluster has started: its shared memory exists
     for (int e = tid; e < pairs; e += nthreads) {
         float2 sum = make_float2(0.f, 0.f);
         for (int k = 0; k < KW; ++k) {
@@ -358,7 +362,7 @@ struct GemvPlan {
 };
 
 static int device_sm_count() {
-    static int cached[64] = {0};
+    static std::atomic<int> cached[64];       // zero-initialised; set-up is idempotent, so a race repeats it harmlessly
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
     if (cached[dev] == 0) {
@@ -469,7 +473,7 @@ static cudaError_t launch_stage_x(const StageParams& sp, cudaStream_t stream) {
 
 template <int NT, bool PRE>
 static cudaError_t launch_gemv(const GemvParams& prm, const GemvPlan& pl, cudaStream_t stream) {
-    static bool attr_set[64] = {false};
+    static std::atomic<bool> attr_set[64];    // zero-initialised; set-up is idempotent, so a race repeats it harmlessly
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;

@@ -23,6 +23,8 @@
 // Every wait on an mbarrier is bounded and reports through the workspace status word.
 #include "slim_gemv_dev.cuh"
 
+#include <atomic>
+
 #include <algorithm>
 #include <cstring>
 #include <exception>
@@ -111,8 +113,8 @@ __device__ __forceinline__ unsigned long long timer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: gives up when the limit passes or when another role has raised `abort`.
-__device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+// Bounded wait: gives up when `limit_ns` has passed or when another role has raised `abort`.
+__device__ __forceinline__ bool wait_limit(uint32_t bar, uint32_t parity, volatile int* abort, unsigned long long limit_ns) {
     if (try_wait(bar, parity)) return true;
     const unsigned long long t0 = timer_ns();
     for (;;) {
@@ -120,8 +122,11 @@ __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, volatile int
         for (int i = 0; i < 32; ++i)
             if (try_wait(bar, parity)) return true;
         if (*abort != 0) return false;
-        if (timer_ns() - t0 > kSetWaitNs) { *abort = 1; return false; }
+        if (timer_ns() - t0 > limit_ns) { *abort = 1; return false; }
     }
+}
+__device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+    return wait_limit(bar, parity, abort, kSetWaitNs);
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -137,11 +142,12 @@ __host__ __device__ inline size_t staged_group_offset(int j, int pre3, int M) {
 // ---- single-token sets: activations as signed 8-bit digits, the packed words as unsigned bytes ----------
 // With one token seven of the eight MMA columns are free, and an integer MMA takes four codes per
 // operand register where the f16 MMA takes two.  So for M = 1 the group's activations become the
-// fixed-point X_k = rint(x_k 2^S) (|X| <= 2^14), and every MMA's B operand holds three signed base-256
-// digits of X_k 2^shift in columns 0..2 (column 3 zero; columns 4..7 repeat them).  The A operand is the
-// packed word ANDed with a byte-wise mask: byte value = field * 2^(w i) for the fields at position i of
-// their byte (w = slice width), and shift = lo + Pc - w i makes every product carry the same 2^Pc, so all
-// positions and both slices of a 3-bit group add up in one integer accumulator: exact.
+// fixed-point X_k = rint(x_k 2^S) (|X| < 2^22: an fp16 value within a factor 2^11 of the group's largest
+// is kept exactly), and every MMA's B operand holds the four signed base-256 digits of X_k 2^shift in
+// columns 0..3 (columns 4..7 repeat them).  The A operand is the packed word ANDed with a byte-wise
+// mask: byte value = field * 2^(w i) for the fields at position i of their byte (w = slice width), and
+// shift = lo + Pc - w i <= 8 makes every product carry the same 2^Pc, so all positions and both slices
+// of a 3-bit group add up in one set of integer accumulators (one per digit, each sum below 2^23: exact).
 __host__ __device__ constexpr int i8_pc(int b) { return b == 1 ? 3 : (b == 4 ? 4 : 6); }
 // Column of the group that meets byte bb of the A register half h (k < 16 or k >= 16) of MMA mi, lane column c.
 __device__ __forceinline__ int i8_column(int w, int mi, int h, int bb, int c) {
@@ -149,12 +155,12 @@ __device__ __forceinline__ int i8_column(int w, int mi, int h, int bb, int c) {
          : w == 1 ? 32 * c + 8 * bb + mi + 4 * h
                   : 32 * c + 8 * (2 * (mi >> 1) + h) + 2 * bb + (mi & 1);
 }
-// Record of one group: (sum_k x, 2^(-S - Pc)) then, per slice, 4 MMAs x [4 columns][4 lanes] x 8 bytes.
+// Record of one group: (sum_k x, 2^(-S - Pc)) then, per slice, 4 MMAs x [4 digits][4 lanes] x 8 bytes.
 __device__ __forceinline__ void stage_group_i8(const __half* xg, uint8_t* rec, int b, int lane, int* Xs) {
     const uint2 raw = *reinterpret_cast<const uint2*>(xg + 4 * lane);
     uint32_t mx = max(max(raw.x & 0x7fffu, (raw.x >> 16) & 0x7fffu), max(raw.y & 0x7fffu, (raw.y >> 16) & 0x7fffu));
     mx = __reduce_max_sync(0xffffffffu, mx);
-    const int S = mx == 0 ? 0 : 28 - max(static_cast<int>(mx >> 10), 1);     // largest |x| 2^S in [2^13, 2^14)
+    const int S = mx == 0 ? 0 : 36 - max(static_cast<int>(mx >> 10), 1);     // largest |x| 2^S in [2^21, 2^22)
     const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
     const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
     float sum = (f01.x + f01.y) + (f23.x + f23.y);
@@ -179,9 +185,10 @@ __device__ __forceinline__ void stage_group_i8(const __half* xg, uint8_t* rec, i
                 for (int bb = 0; bb < 4; ++bb) {
                     const int X = Xs[i8_column(w, mi, h, bb, c)];
                     const int V = X << shift;
-                    const int d0 = static_cast<int8_t>(V & 0xff), V1 = (V - d0) >> 8;
-                    const int d1 = static_cast<int8_t>(V1 & 0xff), d2 = (V1 - d1) >> 8;
-                    const int dig = n == 0 ? d2 : (n == 1 ? d1 : (n == 2 ? d0 : 0));
+                    const int d0 = static_cast<int8_t>(V & 0xff), V1 = (V - d0) >> 8;      // |V| < 2^30
+                    const int d1 = static_cast<int8_t>(V1 & 0xff), V2 = (V1 - d1) >> 8;
+                    const int d2 = static_cast<int8_t>(V2 & 0xff), d3 = (V2 - d2) >> 8;    // |d3| <= 64
+                    const int dig = n == 0 ? d3 : (n == 1 ? d2 : (n == 2 ? d1 : d0));
                     v4 |= static_cast<uint32_t>(dig & 0xff) << (8 * bb);
                 }
                 word[h] = v4;
@@ -416,14 +423,14 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                                 case 3: run_pass(W2{}, WidthTag<1>{}, 0, xs_lane); run_pass(W1{}, WidthTag<0>{}, 2, xs_lane + 512); break;
                                 default: run_pass(W4{}, WidthTag<1>{}, 0, xs_lane); break;
                             }
-                            // fold: columns (0, 1) hold the high and middle digit sums, (2, 3) the low one and zero, (4..7)
-                            // repeat them; lanes with even c see a (high, middle) pair, odd c a (low, 0) pair.  Every lane
+                            // fold: columns (0, 1) hold the sums of the two high digits, (2, 3) of the two low ones, (4..7)
+                            // repeat them; lanes with even c see the high pair, odd c the low pair.  Every lane
                             // holds the sums of all the warp's tiles, so the lane pair c >> 1 folds tile c >> 1 only:
                             // acc += s (D 2^(-S-Pc) - z sum_x)
                             static_assert(TPW <= 2, "one lane pair per tile");
                             const uint2 tkw = lds64(slot + p.off_e);
                             const float sum_x = __uint_as_float(tkw.x), e = __uint_as_float(tkw.y);
-                            const float ka = (c & 1) ? e : 65536.f * e, kb = (c & 1) ? 0.f : 256.f * e;
+                            const float ka = (c & 1) ? 256.f * e : 16777216.f * e, kb = (c & 1) ? e : 65536.f * e;
                             const int tsel = TPW == 2 ? (c >> 1) : 0;
                             int dsel[4];
 #pragma unroll
@@ -558,6 +565,25 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
     if (tid == 0 && *abort != 0) atomicOr(reinterpret_cast<unsigned int*>(p.ws), 1u);
 }
 
+// ------------------------------------------------------------------------------------------ self-test of the bounded wait
+// One warp waits, with the bounded wait of the persistent kernel, on an mbarrier that nobody arrives on.  When the
+// limit has passed it raises the abort flag and the kernel reports through the workspace status word exactly as
+// gemv_set_kernel does, then returns: the path a real time-out takes, without starving a real kernel.
+__global__ void __launch_bounds__(32) wait_selftest_kernel(uint8_t* ws, unsigned long long limit_ns) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        sb::init(b, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const bool ok = __all_sync(0xffffffffu, sb::wait_limit(b, 0, &abort_flag, limit_ns));
+    __syncwarp();
+    if (threadIdx.x == 0 && (!ok || abort_flag != 0)) atomicOr(reinterpret_cast<unsigned int*>(ws), 1u);
+}
+
 // ------------------------------------------------------------------------------------------ host side
 // What the whole set fixes: token tiles, slot geometry, ring depth, grid, sizes.
 struct SetGeometry {
@@ -649,7 +675,7 @@ static size_t set_plan_bytes(int n_layers, long long n_items) {
 
 template <int NT, bool ONE, int TPW>
 static cudaError_t launch_set(const SetParams& prm, int grid, size_t smem, cudaStream_t stream) {
-    static bool attr_set[64] = {false};
+    static std::atomic<bool> attr_set[64];    // zero-initialised; set-up is idempotent, so a race repeats it harmlessly
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -787,6 +813,16 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
     return SLIM_OK;
 }
 
+
+int slim_selftest_wait_timeout(void* workspace, size_t workspace_bytes, unsigned int limit_us, void* stream) {
+    if (workspace == nullptr || workspace_bytes < 256) return SLIM_ERR_WORKSPACE;
+    if (!slim::aligned16(workspace)) return SLIM_ERR_ALIGNMENT;
+    if (limit_us < 1 || limit_us > 100000) return SLIM_ERR_INVALID_ARG;
+    slim::wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint8_t*>(workspace),
+                                                                               1000ull * limit_us);
+    SLIM_CUDA_TRY(cudaGetLastError());
+    return SLIM_OK;
+}
 
 int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* workspace, size_t workspace_bytes, void* stream) {
     if (info == nullptr || plan == nullptr) return SLIM_ERR_INVALID_ARG;

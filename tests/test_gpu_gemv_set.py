@@ -177,7 +177,7 @@ def test_projections_that_share_one_input():
 def test_single_token_fixed_point_with_outlier_channels():
     """Single-token sets round x per group to fixed point relative to the group's largest |x|.  Outlier channels
     (a few activations 100 x the rest, as in LLM activations) and a group of tiny activations must stay within the
-    layer tolerance, and the error of a row must stay below 2^-14 max|x_group| sum|w-hat| per group."""
+    layer tolerance, and the error of a row must stay below 2^-22 max|x_group| sum|w-hat| per group."""
     L = oracle_layer(512, 1024, 2, 1, seed_name="set-outlier")
     rng = np.random.default_rng(11)
     x = rng.normal(0, 1, (1, 1024)).astype(np.float32)
@@ -191,7 +191,7 @@ def test_single_token_fixed_point_with_outlier_channels():
     check_output(ys[0], y_ref, "outlier channels")
     What = np.abs(orc.dequant_f64(L["codes"], L["scales"], L["zeros"]))
     xa = np.abs(L["x"].astype(np.float64))[0]
-    bound = sum(2.0 ** -14 * xa[128 * j:128 * j + 128].max() * What[:, 128 * j:128 * j + 128].sum(axis=1) for j in range(8))
+    bound = sum(2.0 ** -22 * xa[128 * j:128 * j + 128].max() * What[:, 128 * j:128 * j + 128].sum(axis=1) for j in range(8))
     err = np.abs(ys[0].astype(np.float64) - y_ref)[0]
     # + the fp16 rounding of y and the fp32 rounding of the running sum over the groups
     assert (err <= bound + 2.0 ** -10 * np.abs(y_ref[0]) + 1e-5 * np.abs(y_ref).max()).all()

@@ -41,8 +41,12 @@ def test_static_scratch_matches_workspace_entry_point_twice(N, K, M):
     status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
     for call in range(2):
         out.fill_(float("nan"))
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         slim.mpq_gemm_static(x, L.packed, L.bits, L.scales, L.zeros, N, out, status)
         torch.cuda.synchronize()
+        if call == 1:       # the first call on a device may make the driver load the module that holds the array
+            assert torch.cuda.mem_get_info()[0] >= free_before, "the call took device memory"
         assert int(status.item()) == 0, f"call {call}: a device-side wait gave up"
         got = out.cpu().numpy().astype(np.float64)
         assert np.isfinite(got).all(), f"call {call}"
