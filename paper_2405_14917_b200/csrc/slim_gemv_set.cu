@@ -88,6 +88,7 @@ struct SetParams {
     uint8_t* ws;                           // workspace: status word, then the layers' fragments and sums
     int n_layers, n_slots, slot_bytes;
     int off_s, off_z, off_e, off_x;        // offsets inside a slot (weights start at kSetHeader)
+    int one;                               // 1: a multiplier the compiler cannot fold, for selects done as integer multiply-adds
 };
 
 // ------------------------------------------------------------------------------------------ mbarrier helpers
@@ -184,7 +185,11 @@ __device__ __forceinline__ void stage_group_i8(const __half* xg, uint8_t* rec, i
                 uint32_t v4 = 0;
                 for (int bb = 0; bb < 4; ++bb) {
                     const int X = Xs[i8_column(w, mi, h, bb, c)];
-                    const int V = X << shift;
+                    int V = X << shift;
+                    // 2- and 4-bit slices: the MMA of the top field position takes the packed word as it is, i.e. every
+                    // field of the byte times that position's digit; the other positions subtract it again
+                    const int mi_top = w == 2 ? 3 : (mi | 1);
+                    if (w >= 2 && mi != mi_top) V -= Xs[i8_column(w, mi_top, h, bb, c)] << (lo + pc - w * (w == 2 ? 3 : 1));
                     const int d0 = static_cast<int8_t>(V & 0xff), V1 = (V - d0) >> 8;      // |V| < 2^30
                     const int d1 = static_cast<int8_t>(V1 & 0xff), V2 = (V1 - d1) >> 8;
                     const int d2 = static_cast<int8_t>(V2 & 0xff), d3 = (V2 - d2) >> 8;    // |d3| <= 64
@@ -250,6 +255,146 @@ __device__ __forceinline__ void mma_f16_first(float (&d)[4], uint32_t a0, uint32
         "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
         : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b.x), "r"(b.y), "f"(0.f));
+}
+
+
+// Slow path of a consumer's wait, kept out of line so that the loop around it stays small.
+__device__ __noinline__ bool wait_full_slow(uint32_t bar, uint32_t parity, volatile int* abort) {
+    return __all_sync(0xffffffffu, sb::wait(bar, parity, abort));
+}
+
+// Consumer warp of a single-token set: integer MMAs on byte-masked words (see stage_group_i8), then the fold
+// acc += s (D 2^(-S-Pc) - z sum_x) per (row, group).  The loop is bound by instruction dispatch, above all by the
+// half-rate integer/logic pipe, so everything that is not a mask runs on the multiply-add pipe: the two
+// accumulation chains of a tile are added, and the tile of this lane pair is selected, by integer multiply-adds
+// with 0 / 1 multipliers, and the integer sums become floats through the mantissa of 1.5 * 2^23.
+template <int TPW>
+__device__ __forceinline__ void consume_one(const SetParams& p, const uint32_t sbase, const uint32_t ring, volatile int* abort,
+                                            const int i0, const int i1, const int warp, const int lane) {
+    auto full = [&](int s) { return sbase + 8u * s; };
+    auto empty = [&](int s) { return sbase + 8u * (kSetMaxSlots + s); };
+    constexpr int TPI = kSetConsumers * TPW, CHI = 2;
+    static_assert(TPW <= 2, "one lane pair per tile");
+    const int gq = lane >> 2, c = lane & 3;
+    const int tsel = TPW == 2 ? (c >> 1) : 0;
+    const int m0 = tsel ? 0 : p.one, m1 = tsel ? p.one : 0;
+    // lanes with even c hold the sums of the two high digits, odd c of the two low ones
+    const float ma = (c & 1) ? 256.f : 16777216.f, mb = (c & 1) ? 1.f : 65536.f;
+    constexpr int kMagicBits = 0x4B400000;                 // 1.5 * 2^23: adding an integer |v| < 2^22 to these bits gives the float 12582912 + v
+    constexpr float kMagic = 12582912.f;
+    int s = 0;
+    uint32_t ph = 0;
+    bool ok = true;
+    const int4* items4 = reinterpret_cast<const int4*>(p.items);
+    int4 it_a = items4[2 * i0], it_b = items4[2 * i0 + 1];
+    for (int i = i0; i < i1 && ok; ++i) {
+        const int rb = it_a.y, N = it_a.z, G = it_a.w;
+        __half* const ybase = reinterpret_cast<__half*>((static_cast<unsigned long long>(static_cast<uint32_t>(it_b.y)) << 32) |
+                                                        static_cast<uint32_t>(it_b.x));
+        if (i + 1 < i1) {
+            it_a = items4[2 * i + 2];
+            it_b = items4[2 * i + 3];
+        }
+        const int tile0 = TPI * rb + TPW * warp;
+        const int n_act = min(TPW, (N >> 4) - tile0);
+        if (n_act <= 0) {
+            // a warp whose tiles lie past the end of the layer only hands the slots back
+            for (int j = 0; j < G; ++j) {
+                if (!__all_sync(0xffffffffu, sb::try_wait(full(s), ph)) && !wait_full_slow(full(s), ph, abort)) { ok = false; break; }
+                __syncwarp();
+                if (lane == 0) sb::arrive(empty(s));
+                if (++s == p.n_slots) { s = 0; ph ^= 1u; }
+            }
+            continue;
+        }
+        float acc0 = 0.f, acc2 = 0.f;
+        const uint32_t sz_lane = static_cast<uint32_t>((TPW * warp + tsel) * 32 + gq * 4);
+        const uint32_t x_lane = p.off_x + ((gq & 3) * 4 + c) * 8;
+        for (int j = 0; j < G; ++j) {
+            if (!__all_sync(0xffffffffu, sb::try_wait(full(s), ph)) && !wait_full_slow(full(s), ph, abort)) { ok = false; break; }
+            const uint32_t slot = ring + static_cast<uint32_t>(s) * p.slot_bytes;
+            const int b = static_cast<int>(lds32(slot));
+            // tile t of the warp: its slices follow each other.  For a tile past the end of the layer the slot holds
+            // stale bytes: its sums are computed and never stored.
+            const uint32_t item0 = slot + kSetHeader + static_cast<uint32_t>(TPW * warp) * 256u * b + 8u * lane;
+            const uint32_t xs_lane = slot + x_lane;
+            int di[TPW][CHI][4];
+            // one slice of width WD starting at unit `unit0`, digits at `xs`
+            auto run_pass = [&](auto wtag, auto first_tag, int unit0, uint32_t xs) {
+                constexpr int WD = decltype(wtag)::value;
+                constexpr bool FIRST = decltype(first_tag)::value != 0;
+                constexpr uint32_t kByteMask = 0x01010101u * ((1u << WD) - 1u);
+                constexpr int NW = WD == 4 ? 4 : 2;     // words per row the MMAs of the slice draw on
+                uint2 wd[TPW][NW];
+#pragma unroll
+                for (int t = 0; t < TPW; ++t) {
+                    const uint32_t item = item0 + t * 256u * b + 256u * unit0;
+                    wd[t][0] = lds64(item);
+                    if (WD == 1) {
+                        wd[t][1] = make_uint2(wd[t][0].x >> 4, wd[t][0].y >> 4);
+                    } else {
+#pragma unroll
+                        for (int u = 1; u < NW; ++u) wd[t][u] = lds64(item + 256u * u);
+                    }
+                }
+#pragma unroll
+                for (int mi = 0; mi < 4; ++mi) {
+                    const uint2 bv = lds64(xs + mi * 128);
+                    const int pos = WD == 4 ? (mi & 1) : mi, w0 = WD == 4 ? 2 * (mi >> 1) : 0;
+                    const uint32_t m = kByteMask << (WD * pos);
+                    // the top field position of a 2- or 4-bit slice takes the words unmasked (its digits are made for that)
+                    const bool top = (WD == 2 && mi == 3) || (WD == 4 && (mi & 1));
+#pragma unroll
+                    for (int t = 0; t < TPW; ++t) {
+                        const uint32_t a0 = top ? wd[t][w0].x : wd[t][w0].x & m, a1 = top ? wd[t][w0].y : wd[t][w0].y & m;
+                        const uint32_t a2 = top ? wd[t][w0 + 1].x : wd[t][w0 + 1].x & m, a3 = top ? wd[t][w0 + 1].y : wd[t][w0 + 1].y & m;
+                        if (FIRST && mi < CHI) mma_i8_first(di[t][mi & (CHI - 1)], a0, a1, a2, a3, bv);
+                        else mma_i8(di[t][mi & (CHI - 1)], a0, a1, a2, a3, bv);
+                    }
+                }
+            };
+            switch (b) {
+                case 2: run_pass(W2{}, WidthTag<1>{}, 0, xs_lane); break;
+                case 1: run_pass(W1{}, WidthTag<1>{}, 0, xs_lane); break;
+                case 3: run_pass(W2{}, WidthTag<1>{}, 0, xs_lane); run_pass(W1{}, WidthTag<0>{}, 2, xs_lane + 512); break;
+                default: run_pass(W4{}, WidthTag<1>{}, 0, xs_lane); break;
+            }
+            // fold.  Columns (0, 1) hold the sums of the two high digits, (2, 3) of the two low ones, (4..7) repeat
+            // them.  Every lane holds the sums of all the warp's tiles; the lane pair c >> 1 folds tile c >> 1.
+            const uint2 tkw = lds64(slot + p.off_e);
+            const uint32_t s2 = lds32(slot + p.off_s + sz_lane);
+            const uint32_t z2 = lds32(slot + p.off_z + sz_lane);
+            const float sum_x = __uint_as_float(tkw.x), e = __uint_as_float(tkw.y);
+            const float ka = ma * e, kb = mb * e;
+            float f[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                int v = kMagicBits;
+#pragma unroll
+                for (int ch = 0; ch < CHI; ++ch) v += di[0][ch][r] * m0 + di[TPW - 1][ch][r] * m1;
+                f[r] = __int_as_float(v) - kMagic;                        // exact
+            }
+            const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
+            const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
+            float r0 = fmaf(f[0], ka, f[1] * kb);
+            float r1 = fmaf(f[2], ka, f[3] * kb);
+            r0 += __shfl_xor_sync(0xffffffffu, r0, 1);
+            r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
+            acc0 = fmaf(sf.x, fmaf(-zf.x, sum_x, r0), acc0);
+            acc2 = fmaf(sf.y, fmaf(-zf.y, sum_x, r1), acc2);
+            __syncwarp();
+            if (lane == 0) sb::arrive(empty(s));
+            if (++s == p.n_slots) { s = 0; ph ^= 1u; }
+        }
+        if (ok) {
+#pragma unroll
+            for (int t = 0; t < TPW; ++t) {
+                if (t >= n_act) break;
+                __half* yrow = ybase + 16 * (tile0 + t) + 2 * gq;
+                if (c == 2 * t) *reinterpret_cast<__half2*>(yrow) = __floats2half2_rn(acc0, acc2);
+            }
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------ the persistent kernel
@@ -347,6 +492,9 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
             }
         } else {
             // -------------------------------------------------------------- consumer: tile `warp` of every item
+            if constexpr (ONE) {
+                consume_one<TPW>(p, sbase, ring, abort, i0, i1, warp, lane);
+            } else {
             const int gq = lane >> 2, c = lane & 3;
             int s = 0;                                    // ring position of the next group
             uint32_t ph = 0;
@@ -380,78 +528,7 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                         // layer the slot holds stale bytes: its accumulators are computed and never stored.
                         const uint32_t item0 = slot + kSetHeader + static_cast<uint32_t>(TPW * warp) * 256u * b;
                         const uint32_t xs_slot0 = slot + p.off_x;
-                        if constexpr (ONE) {
-                            // ---- one token: integer MMAs on byte-masked words (see stage_group_i8)
-                            constexpr int CHI = 2;                   // accumulation chains per tile
-                            int di[TPW][CHI][4];
-                            const uint32_t xs_lane = xs_slot0 + ((gq & 3) * 4 + c) * 8;
-                            // one slice of width WD starting at unit `unit0`, digits at `xs`
-                            auto run_pass = [&](auto wtag, auto first_tag, int unit0, uint32_t xs) {
-                                constexpr int WD = decltype(wtag)::value;
-                                constexpr bool FIRST = decltype(first_tag)::value != 0;
-                                constexpr uint32_t kByteMask = 0x01010101u * ((1u << WD) - 1u);
-                                constexpr int NW = WD == 4 ? 4 : 2;     // words per row the MMAs of the slice draw on
-                                uint2 wd[TPW][NW];
-#pragma unroll
-                                for (int t = 0; t < TPW; ++t) {
-                                    const uint32_t item = item0 + t * 256u * b + 256u * unit0 + 8u * lane;
-                                    wd[t][0] = lds64(item);
-                                    if (WD == 1) {
-                                        wd[t][1] = make_uint2(wd[t][0].x >> 4, wd[t][0].y >> 4);
-                                    } else {
-#pragma unroll
-                                        for (int u = 1; u < NW; ++u) wd[t][u] = lds64(item + 256u * u);
-                                    }
-                                }
-#pragma unroll
-                                for (int mi = 0; mi < 4; ++mi) {
-                                    const uint2 bv = lds64(xs + mi * 128);
-                                    const int pos = WD == 4 ? (mi & 1) : mi, w0 = WD == 4 ? 2 * (mi >> 1) : 0;
-                                    const uint32_t m = kByteMask << (WD * pos);
-#pragma unroll
-                                    for (int t = 0; t < TPW; ++t) {
-                                        const uint32_t a0 = wd[t][w0].x & m, a1 = wd[t][w0].y & m;
-                                        const uint32_t a2 = wd[t][w0 + 1].x & m, a3 = wd[t][w0 + 1].y & m;
-                                        if (FIRST && mi < CHI) mma_i8_first(di[t][mi & (CHI - 1)], a0, a1, a2, a3, bv);
-                                        else mma_i8(di[t][mi & (CHI - 1)], a0, a1, a2, a3, bv);
-                                    }
-                                }
-                            };
-                            switch (b) {
-                                case 1: run_pass(W1{}, WidthTag<1>{}, 0, xs_lane); break;
-                                case 2: run_pass(W2{}, WidthTag<1>{}, 0, xs_lane); break;
-                                case 3: run_pass(W2{}, WidthTag<1>{}, 0, xs_lane); run_pass(W1{}, WidthTag<0>{}, 2, xs_lane + 512); break;
-                                default: run_pass(W4{}, WidthTag<1>{}, 0, xs_lane); break;
-                            }
-                            // fold: columns (0, 1) hold the sums of the two high digits, (2, 3) of the two low ones, (4..7)
-                            // repeat them; lanes with even c see the high pair, odd c the low pair.  Every lane
-                            // holds the sums of all the warp's tiles, so the lane pair c >> 1 folds tile c >> 1 only:
-                            // acc += s (D 2^(-S-Pc) - z sum_x)
-                            static_assert(TPW <= 2, "one lane pair per tile");
-                            const uint2 tkw = lds64(slot + p.off_e);
-                            const float sum_x = __uint_as_float(tkw.x), e = __uint_as_float(tkw.y);
-                            const float ka = (c & 1) ? 256.f * e : 16777216.f * e, kb = (c & 1) ? e : 65536.f * e;
-                            const int tsel = TPW == 2 ? (c >> 1) : 0;
-                            int dsel[4];
-#pragma unroll
-                            for (int r = 0; r < 4; ++r) {
-                                int v0 = di[0][0][r], v1 = di[TPW - 1][0][r];
-#pragma unroll
-                                for (int ch = 1; ch < CHI; ++ch) { v0 += di[0][ch][r]; v1 += di[TPW - 1][ch][r]; }
-                                dsel[r] = tsel ? v1 : v0;
-                            }
-                            const int tt = TPW * warp + tsel;
-                            const uint32_t s2 = lds32(slot + p.off_s + tt * 32 + gq * 4);
-                            const uint32_t z2 = lds32(slot + p.off_z + tt * 32 + gq * 4);
-                            const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
-                            const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
-                            float r0 = fmaf(static_cast<float>(dsel[0]), ka, static_cast<float>(dsel[1]) * kb);
-                            float r1 = fmaf(static_cast<float>(dsel[2]), ka, static_cast<float>(dsel[3]) * kb);
-                            r0 += __shfl_xor_sync(0xffffffffu, r0, 1);
-                            r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
-                            acc[0][0][0] = fmaf(sf.x, fmaf(-zf.x, sum_x, r0), acc[0][0][0]);
-                            acc[0][0][2] = fmaf(sf.y, fmaf(-zf.y, sum_x, r1), acc[0][0][2]);
-                        } else {
+                        {
                         constexpr int CH = NT == 1 ? (TPW == 1 ? 4 : 2) : 2;     // interleaved accumulation chains
                         float d[TPW][CH][NT][4];      // every chain is started by an MMA with a zero accumulator
 
@@ -558,6 +635,7 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                         }
                     }
                 }
+            }
             }
         }
     }
@@ -848,6 +926,7 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     prm.n_layers = info->n_layers;
     prm.n_slots = info->n_slots;
     prm.slot_bytes = info->slot_bytes;
+    prm.one = 1;
     const int tpi = slim::kSetConsumers * info->tiles_per_warp;
     prm.off_s = slim::kSetHeader + tpi * 256 * info->max_bits;
     prm.off_z = prm.off_s + tpi * 32;
