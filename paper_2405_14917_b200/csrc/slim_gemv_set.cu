@@ -40,8 +40,17 @@ constexpr int kSetProducers = 2;                       // producer warps: they t
 constexpr int kSetThreads = 32 * (kSetConsumers + kSetProducers);
 constexpr int kSetMaxSlots = 32;
 constexpr int kSetCtasPerSm = 2;                       // resident CTAs per SM the plan aims at
-constexpr int kSetHeader = 16;                         // slot header: bit-width of the group
 constexpr unsigned long long kSetWaitNs = 2000000000ull;
+
+// Layout of a ring slot (tpi = 16-row tiles of a work item, mp = 256-byte pieces per slice of the staged
+// activations: 2 for single-token sets, else the 8 or 16 tokens of the set).  Everything but the packed slices has
+// a fixed size, so the slices come last and every other offset is a compile-time constant of the kernel:
+//   header (bit-width of the group) | scales | zeros | (sum_k x, scale) per token | activations of two slices | slices
+constexpr int kSlotOffS = 16;
+__host__ __device__ constexpr int slot_off_z(int tpi) { return kSlotOffS + 32 * tpi; }
+__host__ __device__ constexpr int slot_off_e(int tpi) { return kSlotOffS + 64 * tpi; }
+__host__ __device__ constexpr int slot_off_x(int tpi) { return slot_off_e(tpi) + 128; }
+__host__ __device__ constexpr int slot_off_w(int tpi, int mp) { return slot_off_x(tpi) + 2 * 256 * mp; }
 
 // Device-side description of one layer (lives in the plan buffer).
 struct SetLayer {
@@ -54,7 +63,7 @@ struct SetLayer {
                            // (sum_k x, 2^(24-S)) float2[16], then the fragments [slice][8 mma][MP][4 lanes] x 8 B
     size_t pad0;
     int M, N, K, G;
-    int pad1[2];
+    uint16_t count[4];     // groups of 1, 2, 3, 4 bits
     int task0;             // first (token, group) staging task of the layer
     int MP;                // 256-byte pieces per slice in the staged layout: 8 or 16 = tokens of the f16 fragments for the
                            // whole set (absent tokens are staged as zeros, so the kernel reads without a test); 2 if every
@@ -62,6 +71,7 @@ struct SetLayer {
     uint16_t prefix[SLIM_MAX_GROUPS + 1];
     uint16_t pre3[SLIM_MAX_GROUPS + 1];   // 3-bit groups (two slices) before group j
     uint8_t bits[SLIM_MAX_GROUPS];
+    uint8_t order[SLIM_MAX_GROUPS];       // the order in which the groups are streamed: by bit-width, then by index
     uint8_t pad2[4];
 };
 static_assert(sizeof(SetLayer) % 16 == 0, "descriptors are copied and read in 16-byte pieces");
@@ -72,7 +82,8 @@ struct SetItem {
     int layer, rb;         // layer of the set, row block inside the layer
     int N, G;
     __half* y;
-    int M, pad;
+    int M;
+    int counts;            // groups of 1, 2 and 3 bits, 9 bits each (the rest of G has 4): the groups arrive in that order
 };
 static_assert(sizeof(SetItem) == 32, "items are read as two 16-byte pieces");
 
@@ -87,7 +98,6 @@ struct SetParams {
     const SetItem* items;
     uint8_t* ws;                           // workspace: status word, then the layers' fragments and sums
     int n_layers, n_slots, slot_bytes;
-    int off_s, off_z, off_e, off_x;        // offsets inside a slot (weights start at kSetHeader)
     int one;                               // 1: a multiplier the compiler cannot fold, for selects done as integer multiply-adds
 };
 
@@ -101,6 +111,10 @@ __device__ __forceinline__ void expect_tx(uint32_t bar, uint32_t bytes) {
 }
 __device__ __forceinline__ void arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Arrive by the lanes whose flag is set, as one predicated instruction (no divergent branch around it).
+__device__ __forceinline__ void arrive_if(uint32_t bar, uint32_t flag) {
+    asm volatile("{\n .reg .pred p;\n setp.ne.u32 p, %1, 0;\n @p mbarrier.arrive.shared::cta.b64 _, [%0];\n}\n" ::"r"(bar), "r"(flag) : "memory");
 }
 __device__ __forceinline__ bool try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -274,6 +288,7 @@ __device__ __forceinline__ void consume_one(const SetParams& p, const uint32_t s
     auto full = [&](int s) { return sbase + 8u * s; };
     auto empty = [&](int s) { return sbase + 8u * (kSetMaxSlots + s); };
     constexpr int TPI = kSetConsumers * TPW, CHI = 2;
+    constexpr uint32_t kOffZ = slot_off_z(TPI), kOffE = slot_off_e(TPI), kOffX = slot_off_x(TPI), kOffW = slot_off_w(TPI, 2);
     static_assert(TPW <= 2, "one lane pair per tile");
     const int gq = lane >> 2, c = lane & 3;
     const int tsel = TPW == 2 ? (c >> 1) : 0;
@@ -282,16 +297,22 @@ __device__ __forceinline__ void consume_one(const SetParams& p, const uint32_t s
     const float ma = (c & 1) ? 256.f : 16777216.f, mb = (c & 1) ? 1.f : 65536.f;
     constexpr int kMagicBits = 0x4B400000;                 // 1.5 * 2^23: adding an integer |v| < 2^22 to these bits gives the float 12582912 + v
     constexpr float kMagic = 12582912.f;
+    const uint32_t lane0 = lane == 0 ? 1u : 0u;
+    const uint32_t slot_bytes = static_cast<uint32_t>(p.slot_bytes);
+    const int n_slots = p.n_slots;
+    const uint32_t sz_lane = static_cast<uint32_t>((TPW * warp + tsel) * 32 + gq * 4);
+    const uint32_t x_lane = kOffX + ((gq & 3) * 4 + c) * 8;
+    const uint32_t w_lane = kOffW + 8u * lane;
     int s = 0;
     uint32_t ph = 0;
     bool ok = true;
     const int4* items4 = reinterpret_cast<const int4*>(p.items);
-    int4 it_a = items4[2 * i0], it_b = items4[2 * i0 + 1];
+    int4 it_a = items4[2 * i0], it_b = items4[2 * i0 + 1];       // (layer, rb, N, G), (y, M, counts)
     for (int i = i0; i < i1 && ok; ++i) {
-        const int rb = it_a.y, N = it_a.z, G = it_a.w;
+        const int rb = it_a.y, N = it_a.z, G = it_a.w, counts = it_b.w;
         __half* const ybase = reinterpret_cast<__half*>((static_cast<unsigned long long>(static_cast<uint32_t>(it_b.y)) << 32) |
                                                         static_cast<uint32_t>(it_b.x));
-        if (i + 1 < i1) {
+        if (i + 1 < i1) {                                        // the next item arrives during this one's groups
             it_a = items4[2 * i + 2];
             it_b = items4[2 * i + 3];
         }
@@ -302,90 +323,95 @@ __device__ __forceinline__ void consume_one(const SetParams& p, const uint32_t s
             for (int j = 0; j < G; ++j) {
                 if (!__all_sync(0xffffffffu, sb::try_wait(full(s), ph)) && !wait_full_slow(full(s), ph, abort)) { ok = false; break; }
                 __syncwarp();
-                if (lane == 0) sb::arrive(empty(s));
-                if (++s == p.n_slots) { s = 0; ph ^= 1u; }
+                sb::arrive_if(empty(s), lane0);
+                if (++s == n_slots) { s = 0; ph ^= 1u; }
             }
             continue;
         }
         float acc0 = 0.f, acc2 = 0.f;
-        const uint32_t sz_lane = static_cast<uint32_t>((TPW * warp + tsel) * 32 + gq * 4);
-        const uint32_t x_lane = p.off_x + ((gq & 3) * 4 + c) * 8;
-        for (int j = 0; j < G; ++j) {
-            if (!__all_sync(0xffffffffu, sb::try_wait(full(s), ph)) && !wait_full_slow(full(s), ph, abort)) { ok = false; break; }
-            const uint32_t slot = ring + static_cast<uint32_t>(s) * p.slot_bytes;
-            const int b = static_cast<int>(lds32(slot));
-            // tile t of the warp: its slices follow each other.  For a tile past the end of the layer the slot holds
-            // stale bytes: its sums are computed and never stored.
-            const uint32_t item0 = slot + kSetHeader + static_cast<uint32_t>(TPW * warp) * 256u * b + 8u * lane;
-            const uint32_t xs_lane = slot + x_lane;
-            int di[TPW][CHI][4];
-            // one slice of width WD starting at unit `unit0`, digits at `xs`
-            auto run_pass = [&](auto wtag, auto first_tag, int unit0, uint32_t xs) {
-                constexpr int WD = decltype(wtag)::value;
-                constexpr bool FIRST = decltype(first_tag)::value != 0;
-                constexpr uint32_t kByteMask = 0x01010101u * ((1u << WD) - 1u);
-                constexpr int NW = WD == 4 ? 4 : 2;     // words per row the MMAs of the slice draw on
-                uint2 wd[TPW][NW];
-#pragma unroll
-                for (int t = 0; t < TPW; ++t) {
-                    const uint32_t item = item0 + t * 256u * b + 256u * unit0;
-                    wd[t][0] = lds64(item);
-                    if (WD == 1) {
-                        wd[t][1] = make_uint2(wd[t][0].x >> 4, wd[t][0].y >> 4);
-                    } else {
-#pragma unroll
-                        for (int u = 1; u < NW; ++u) wd[t][u] = lds64(item + 256u * u);
-                    }
-                }
-#pragma unroll
-                for (int mi = 0; mi < 4; ++mi) {
-                    const uint2 bv = lds64(xs + mi * 128);
-                    const int pos = WD == 4 ? (mi & 1) : mi, w0 = WD == 4 ? 2 * (mi >> 1) : 0;
-                    const uint32_t m = kByteMask << (WD * pos);
-                    // the top field position of a 2- or 4-bit slice takes the words unmasked (its digits are made for that)
-                    const bool top = (WD == 2 && mi == 3) || (WD == 4 && (mi & 1));
+
+        // The groups of an item arrive sorted by bit-width (the counts come with the item), so each width has a loop
+        // of its own and no group has to say what it is.  `n` groups of B bits: false if a wait gave up.
+        auto run_groups = [&](auto btag, int n) -> bool {
+            constexpr int B = decltype(btag)::value;
+            for (int k = 0; k < n; ++k) {
+                if (!__all_sync(0xffffffffu, sb::try_wait(full(s), ph)) && !wait_full_slow(full(s), ph, abort)) return false;
+                const uint32_t slot = ring + static_cast<uint32_t>(s) * slot_bytes;
+                // tile t of the warp: its slices follow each other.  For a tile past the end of the layer the slot holds
+                // stale bytes: its sums are computed and never stored.
+                const uint32_t item0 = slot + w_lane + static_cast<uint32_t>(TPW * warp) * (256u * B);
+                const uint32_t xs_lane = slot + x_lane;
+                int di[TPW][CHI][4];
+                // one slice of width WD starting at unit `unit0`, digits at `xs`
+                auto run_pass = [&](auto wtag, auto first_tag, int unit0, uint32_t xs) {
+                    constexpr int WD = decltype(wtag)::value;
+                    constexpr bool FIRST = decltype(first_tag)::value != 0;
+                    constexpr uint32_t kByteMask = 0x01010101u * ((1u << WD) - 1u);
+                    constexpr int NW = WD == 4 ? 4 : 2;     // words per row the MMAs of the slice draw on
+                    uint2 wd[TPW][NW];
 #pragma unroll
                     for (int t = 0; t < TPW; ++t) {
-                        const uint32_t a0 = top ? wd[t][w0].x : wd[t][w0].x & m, a1 = top ? wd[t][w0].y : wd[t][w0].y & m;
-                        const uint32_t a2 = top ? wd[t][w0 + 1].x : wd[t][w0 + 1].x & m, a3 = top ? wd[t][w0 + 1].y : wd[t][w0 + 1].y & m;
-                        if (FIRST && mi < CHI) mma_i8_first(di[t][mi & (CHI - 1)], a0, a1, a2, a3, bv);
-                        else mma_i8(di[t][mi & (CHI - 1)], a0, a1, a2, a3, bv);
+                        const uint32_t item = item0 + t * (256u * B) + 256u * unit0;
+                        wd[t][0] = lds64(item);
+                        if (WD == 1) {
+                            wd[t][1] = make_uint2(wd[t][0].x >> 4, wd[t][0].y >> 4);
+                        } else {
+#pragma unroll
+                            for (int u = 1; u < NW; ++u) wd[t][u] = lds64(item + 256u * u);
+                        }
                     }
+#pragma unroll
+                    for (int mi = 0; mi < 4; ++mi) {
+                        const uint2 bv = lds64(xs + mi * 128);
+                        const int pos = WD == 4 ? (mi & 1) : mi, w0 = WD == 4 ? 2 * (mi >> 1) : 0;
+                        const uint32_t m = kByteMask << (WD * pos);
+                        // the top field position of a 2- or 4-bit slice takes the words unmasked (its digits are made for that)
+                        const bool top = (WD == 2 && mi == 3) || (WD == 4 && (mi & 1));
+#pragma unroll
+                        for (int t = 0; t < TPW; ++t) {
+                            const uint32_t a0 = top ? wd[t][w0].x : wd[t][w0].x & m, a1 = top ? wd[t][w0].y : wd[t][w0].y & m;
+                            const uint32_t a2 = top ? wd[t][w0 + 1].x : wd[t][w0 + 1].x & m, a3 = top ? wd[t][w0 + 1].y : wd[t][w0 + 1].y & m;
+                            if (FIRST && mi < CHI) mma_i8_first(di[t][mi & (CHI - 1)], a0, a1, a2, a3, bv);
+                            else mma_i8(di[t][mi & (CHI - 1)], a0, a1, a2, a3, bv);
+                        }
+                    }
+                };
+                if (B == 1) run_pass(W1{}, WidthTag<1>{}, 0, xs_lane);
+                if (B == 2) run_pass(W2{}, WidthTag<1>{}, 0, xs_lane);
+                if (B == 3) { run_pass(W2{}, WidthTag<1>{}, 0, xs_lane); run_pass(W1{}, WidthTag<0>{}, 2, xs_lane + 512); }
+                if (B == 4) run_pass(W4{}, WidthTag<1>{}, 0, xs_lane);
+                // fold.  Columns (0, 1) hold the sums of the two high digits, (2, 3) of the two low ones, (4..7) repeat
+                // them.  Every lane holds the sums of all the warp's tiles; the lane pair c >> 1 folds tile c >> 1.
+                const uint2 tkw = lds64(slot + kOffE);
+                const uint32_t s2 = lds32(slot + kSlotOffS + sz_lane);
+                const uint32_t z2 = lds32(slot + kOffZ + sz_lane);
+                const float sum_x = __uint_as_float(tkw.x), e = __uint_as_float(tkw.y);
+                const float ka = ma * e, kb = mb * e;
+                float f[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    int v = kMagicBits;
+#pragma unroll
+                    for (int ch = 0; ch < CHI; ++ch) v += di[0][ch][r] * m0 + di[TPW - 1][ch][r] * m1;
+                    f[r] = __int_as_float(v) - kMagic;                        // exact
                 }
-            };
-            switch (b) {
-                case 2: run_pass(W2{}, WidthTag<1>{}, 0, xs_lane); break;
-                case 1: run_pass(W1{}, WidthTag<1>{}, 0, xs_lane); break;
-                case 3: run_pass(W2{}, WidthTag<1>{}, 0, xs_lane); run_pass(W1{}, WidthTag<0>{}, 2, xs_lane + 512); break;
-                default: run_pass(W4{}, WidthTag<1>{}, 0, xs_lane); break;
+                const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
+                const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
+                float r0 = fmaf(f[0], ka, f[1] * kb);
+                float r1 = fmaf(f[2], ka, f[3] * kb);
+                r0 += __shfl_xor_sync(0xffffffffu, r0, 1);
+                r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
+                acc0 = fmaf(sf.x, fmaf(-zf.x, sum_x, r0), acc0);
+                acc2 = fmaf(sf.y, fmaf(-zf.y, sum_x, r1), acc2);
+                __syncwarp();
+                sb::arrive_if(empty(s), lane0);
+                if (++s == n_slots) { s = 0; ph ^= 1u; }
             }
-            // fold.  Columns (0, 1) hold the sums of the two high digits, (2, 3) of the two low ones, (4..7) repeat
-            // them.  Every lane holds the sums of all the warp's tiles; the lane pair c >> 1 folds tile c >> 1.
-            const uint2 tkw = lds64(slot + p.off_e);
-            const uint32_t s2 = lds32(slot + p.off_s + sz_lane);
-            const uint32_t z2 = lds32(slot + p.off_z + sz_lane);
-            const float sum_x = __uint_as_float(tkw.x), e = __uint_as_float(tkw.y);
-            const float ka = ma * e, kb = mb * e;
-            float f[4];
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                int v = kMagicBits;
-#pragma unroll
-                for (int ch = 0; ch < CHI; ++ch) v += di[0][ch][r] * m0 + di[TPW - 1][ch][r] * m1;
-                f[r] = __int_as_float(v) - kMagic;                        // exact
-            }
-            const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
-            const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
-            float r0 = fmaf(f[0], ka, f[1] * kb);
-            float r1 = fmaf(f[2], ka, f[3] * kb);
-            r0 += __shfl_xor_sync(0xffffffffu, r0, 1);
-            r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
-            acc0 = fmaf(sf.x, fmaf(-zf.x, sum_x, r0), acc0);
-            acc2 = fmaf(sf.y, fmaf(-zf.y, sum_x, r1), acc2);
-            __syncwarp();
-            if (lane == 0) sb::arrive(empty(s));
-            if (++s == p.n_slots) { s = 0; ph ^= 1u; }
-        }
+            return true;
+        };
+        const int c1 = counts & 511, c2 = (counts >> 9) & 511, c3 = (counts >> 18) & 511;
+        ok = run_groups(WidthTag<1>{}, c1) && run_groups(WidthTag<2>{}, c2) && run_groups(WidthTag<3>{}, c3) &&
+             run_groups(WidthTag<4>{}, G - c1 - c2 - c3);
         if (ok) {
 #pragma unroll
             for (int t = 0; t < TPW; ++t) {
@@ -417,6 +443,8 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
     const uint32_t ring = sbase + kSetOffRing;
     constexpr int TPI = kSetConsumers * TPW;                  // tiles per item
     constexpr int MPK = ONE ? 1 : 8 * NT;                     // tokens in the staged layout
+    constexpr uint32_t kOffZ = slot_off_z(TPI), kOffE = slot_off_e(TPI), kOffX = slot_off_x(TPI);
+    constexpr uint32_t kOffW = slot_off_w(TPI, ONE ? 2 : 8 * NT);
 
     if (tid == 0) {
         for (int s = 0; s < p.n_slots; ++s) { sb::init(full(s), 1); sb::init(empty(s), kSetConsumers); }
@@ -458,13 +486,14 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                                     : lane == 1 ? reinterpret_cast<const uint8_t*>(D->scales + 16 * TPI * rb)
                                     : lane == 2 ? reinterpret_cast<const uint8_t*>(D->zeros + 16 * TPI * rb)
                                                 : p.ws + D->x_off;
-                const uint32_t dst_off = lane == 0 ? kSetHeader : lane == 1 ? p.off_s : lane == 2 ? p.off_z : p.off_e;
+                const uint32_t dst_off = lane == 0 ? kOffW : lane == 1 ? kSlotOffS : lane == 2 ? kOffZ : kOffE;
                 const uint32_t szb = static_cast<uint32_t>(tiles_here) * 32u;
-                int j = static_cast<int>((static_cast<uint32_t>(pw) + kSetProducers - cnt % kSetProducers) % kSetProducers);
+                int jj = static_cast<int>((static_cast<uint32_t>(pw) + kSetProducers - cnt % kSetProducers) % kSetProducers);
                 cnt += static_cast<uint32_t>(G);
-                for (; j < G; j += kSetProducers) {
+                for (; jj < G; jj += kSetProducers) {
                     // the lanes go on, or give up, together
                     if (!__all_sync(0xffffffffu, sb::wait(empty(s), ph ^ 1u, abort))) { ok = false; break; }
+                    const int j = D->order[jj];            // the groups are streamed sorted by bit-width
                     const uint32_t b = D->bits[j];
                     const uint32_t wbytes = static_cast<uint32_t>(tiles_here) * 256u * b;
                     const uint32_t xbytes = 128u + static_cast<uint32_t>(slice_count(b)) * 256u * MP;
@@ -526,8 +555,8 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                         const int b = static_cast<int>(lds32(slot));
                         // tile t of the warp: its slices follow each other.  For a tile past the end of the
                         // layer the slot holds stale bytes: its accumulators are computed and never stored.
-                        const uint32_t item0 = slot + kSetHeader + static_cast<uint32_t>(TPW * warp) * 256u * b;
-                        const uint32_t xs_slot0 = slot + p.off_x;
+                        const uint32_t item0 = slot + kOffW + static_cast<uint32_t>(TPW * warp) * 256u * b;
+                        const uint32_t xs_slot0 = slot + kOffX;
                         {
                         constexpr int CH = NT == 1 ? (TPW == 1 ? 4 : 2) : 2;     // interleaved accumulation chains
                         float d[TPW][CH][NT][4];      // every chain is started by an MMA with a zero accumulator
@@ -574,16 +603,16 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                         }
 
                         // fold the group: acc += s * (D * 2^(24-S) - z * sum_x); rows 2gq, 2gq+1, tokens 8n+2c, 8n+2c+1
-                        const float2* sxe = reinterpret_cast<const float2*>(smem + (slot - sbase) + p.off_e);
+                        const float2* sxe = reinterpret_cast<const float2*>(smem + (slot - sbase) + kOffE);
 #pragma unroll
                         for (int t = 0; t < TPW; ++t) {
                             const int tt = TPW * warp + t;                             // tile inside the item
-                            const uint32_t s2 = lds32(slot + p.off_s + tt * 32 + gq * 4);
-                            const uint32_t z2 = lds32(slot + p.off_z + tt * 32 + gq * 4);
+                            const uint32_t s2 = lds32(slot + kSlotOffS + tt * 32 + gq * 4);
+                            const uint32_t z2 = lds32(slot + kOffZ + tt * 32 + gq * 4);
                             const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
                             const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
                             if (ONE) {
-                                const uint2 tkw = lds64(slot + p.off_e);                   // (sum_k x, 2^(24-S)) of token 0
+                                const uint2 tkw = lds64(slot + kOffE);                   // (sum_k x, 2^(24-S)) of token 0
                                 const float2 tk = make_float2(__uint_as_float(tkw.x), __uint_as_float(tkw.y));
                                 float e0 = d[t][0][0][0] + d[t][1][0][0], e2 = d[t][0][0][2] + d[t][1][0][2];
                                 if (CH == 4) {
@@ -666,7 +695,7 @@ __global__ void __launch_bounds__(32) wait_selftest_kernel(uint8_t* ws, unsigned
 // What the whole set fixes: token tiles, slot geometry, ring depth, grid, sizes.
 struct SetGeometry {
     int nt, bmax, mmax, tpw, mpad;     // tpw: tiles per consumer warp; mpad: tokens in the staged layout
-    int off_s, off_z, off_e, off_x, slot_bytes;
+    int slot_bytes;
     int n_slots, grid, ctas_per_sm;
     size_t smem_bytes;
     long long n_items, n_tasks;
@@ -722,12 +751,7 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     }
     if (sg->n_items > 0x3fffffff || sg->n_tasks > 0x3fffffff) return SLIM_ERR_UNSUPPORTED;
     sg->nt = sg->mmax <= 8 ? 1 : 2;
-    sg->off_s = kSetHeader + tpi * 256 * sg->bmax;
-    sg->off_z = sg->off_s + tpi * 32;
-    sg->off_e = sg->off_z + tpi * 32;
-    sg->off_x = sg->off_e + 128;
-    // a 3-bit group brings the fragments of two slices (a set whose widest group has 4 bits may hold one)
-    sg->slot_bytes = static_cast<int>(align_to(static_cast<size_t>(sg->off_x) + (sg->bmax >= 3 ? 2 : 1) * 256 * sg->mpad, 128));
+    sg->slot_bytes = static_cast<int>(align_to(static_cast<size_t>(slot_off_w(tpi, sg->mpad)) + static_cast<size_t>(tpi) * 256 * sg->bmax, 128));
     // as many CTAs per SM (kSetCtasPerSm at most) as still leaves each a ring of 5 slots
     const size_t per_sm = 224 * 1024;
     size_t budget = 0;
@@ -831,6 +855,10 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
         d.pre3[0] = 0;
         for (int j = 0; j < SLIM_MAX_GROUPS; ++j)
             d.pre3[j + 1] = static_cast<uint16_t>(d.pre3[j] + (j < gt.G && gt.bits[j] == 3 ? 1 : 0));
+        int n_sorted = 0;                       // streaming order: by bit-width, then by index
+        for (int b = 1; b <= 4; ++b)
+            for (int j = 0; j < gt.G; ++j)
+                if (gt.bits[j] == b) { d.order[n_sorted++] = static_cast<uint8_t>(j); ++d.count[b - 1]; }
         SLIM_CUDA_TRY(cudaMemcpyAsync(plan_dev + slim::kSetPlanHeader + static_cast<size_t>(l) * sizeof d, &d, sizeof d,
                                       cudaMemcpyHostToDevice, s));
         const int n_rb = ((L.N >> 4) + tpi - 1) / tpi;
@@ -839,6 +867,7 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
             slim::SetItem it;
             memset(&it, 0, sizeof it);
             it.layer = l; it.rb = rb; it.N = L.N; it.G = gt.G; it.y = d.y; it.M = L.M;
+            it.counts = d.count[0] | (d.count[1] << 9) | (d.count[2] << 18);
             items.push_back(it);
             cost.push_back(slim::item_cost(th < tpi ? th : tpi, gt));
         }
@@ -928,11 +957,8 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     prm.slot_bytes = info->slot_bytes;
     prm.one = 1;
     const int tpi = slim::kSetConsumers * info->tiles_per_warp;
-    prm.off_s = slim::kSetHeader + tpi * 256 * info->max_bits;
-    prm.off_z = prm.off_s + tpi * 32;
-    prm.off_e = prm.off_z + tpi * 32;
-    prm.off_x = prm.off_e + 128;
-    if (prm.off_x + (info->max_bits >= 3 ? 2 : 1) * 256 * (info->max_tokens == 1 ? 2 : 8 * info->token_tiles) > info->slot_bytes) return SLIM_ERR_INVALID_ARG;
+    const int mp = info->max_tokens == 1 ? 2 : 8 * info->token_tiles;
+    if (slim::slot_off_w(tpi, mp) + tpi * 256 * info->max_bits > info->slot_bytes) return SLIM_ERR_INVALID_ARG;
 
     slim::gemv_set_stage_kernel<<<(info->stage_tasks + 7) / 8, 256, 0, s>>>(prm.layers, prm.ws, info->n_layers, info->stage_tasks);
     SLIM_CUDA_TRY(cudaGetLastError());
