@@ -163,7 +163,9 @@ __host__ __device__ inline size_t staged_group_offset(int j, int pre3, int M) {
 // mask: byte value = field * 2^(w i) for the fields at position i of their byte (w = slice width), and
 // shift = lo + Pc - w i <= 8 makes every product carry the same 2^Pc, so all positions and both slices
 // of a 3-bit group add up in one set of integer accumulators (one per digit, each sum below 2^23: exact).
-__host__ __device__ constexpr int i8_pc(int b) { return b == 1 ? 3 : (b == 4 ? 4 : 6); }
+__host__ __device__ constexpr int i8_pc(int b) { return b == 1 ? 7 : (b == 4 ? 4 : 6); }
+// Field position inside its byte that MMA mi meets in the A register half h, for a slice of width w.
+__host__ __device__ constexpr int i8_pos(int w, int mi, int h) { return w == 1 ? mi + 4 * h : (w == 4 ? (mi & 1) : mi); }
 // Column of the group that meets byte bb of the A register half h (k < 16 or k >= 16) of MMA mi, lane column c.
 __device__ __forceinline__ int i8_column(int w, int mi, int h, int bb, int c) {
     return w == 2 ? 32 * c + 16 * h + 4 * bb + mi
@@ -192,18 +194,16 @@ __device__ __forceinline__ void stage_group_i8(const __half* xg, uint8_t* rec, i
         const int w = slice_w(b, sl), lo = slice_lo(b, sl);
         for (int idx = lane; idx < 64; idx += 32) {
             const int mi = idx >> 4, n = (idx >> 2) & 3, c = idx & 3;
-            const int pos = w == 4 ? (mi & 1) : mi;
-            const int shift = lo + pc - w * pos;
             uint32_t word[2];
             for (int h = 0; h < 2; ++h) {
                 uint32_t v4 = 0;
+                // The MMA of a byte's top field position takes the packed word as it is, i.e. every field of the byte
+                // times that position's digit; the other positions subtract it again.
+                const int mi_top = w == 4 ? (mi | 1) : 3, h_top = w == 1 ? 1 : h;
+                const int pos = i8_pos(w, mi, h), pos_top = i8_pos(w, mi_top, h_top);
                 for (int bb = 0; bb < 4; ++bb) {
-                    const int X = Xs[i8_column(w, mi, h, bb, c)];
-                    int V = X << shift;
-                    // 2- and 4-bit slices: the MMA of the top field position takes the packed word as it is, i.e. every
-                    // field of the byte times that position's digit; the other positions subtract it again
-                    const int mi_top = w == 2 ? 3 : (mi | 1);
-                    if (w >= 2 && mi != mi_top) V -= Xs[i8_column(w, mi_top, h, bb, c)] << (lo + pc - w * (w == 2 ? 3 : 1));
+                    int V = Xs[i8_column(w, mi, h, bb, c)] << (lo + pc - w * pos);
+                    if (mi != mi_top || h != h_top) V -= Xs[i8_column(w, mi_top, h_top, bb, c)] << (lo + pc - w * pos_top);
                     const int d0 = static_cast<int8_t>(V & 0xff), V1 = (V - d0) >> 8;      // |V| < 2^30
                     const int d1 = static_cast<int8_t>(V1 & 0xff), V2 = (V1 - d1) >> 8;
                     const int d2 = static_cast<int8_t>(V2 & 0xff), d3 = (V2 - d2) >> 8;    // |d3| <= 64
@@ -347,30 +347,28 @@ __device__ __forceinline__ void consume_one(const SetParams& p, const uint32_t s
                     constexpr int WD = decltype(wtag)::value;
                     constexpr bool FIRST = decltype(first_tag)::value != 0;
                     constexpr uint32_t kByteMask = 0x01010101u * ((1u << WD) - 1u);
-                    constexpr int NW = WD == 4 ? 4 : 2;     // words per row the MMAs of the slice draw on
+                    constexpr int NW = WD;                  // 8-byte pieces (two rows' words) per lane that the MMAs of the slice draw on
                     uint2 wd[TPW][NW];
 #pragma unroll
                     for (int t = 0; t < TPW; ++t) {
                         const uint32_t item = item0 + t * (256u * B) + 256u * unit0;
-                        wd[t][0] = lds64(item);
-                        if (WD == 1) {
-                            wd[t][1] = make_uint2(wd[t][0].x >> 4, wd[t][0].y >> 4);
-                        } else {
 #pragma unroll
-                            for (int u = 1; u < NW; ++u) wd[t][u] = lds64(item + 256u * u);
-                        }
+                        for (int u = 0; u < NW; ++u) wd[t][u] = lds64(item + 256u * u);
                     }
 #pragma unroll
                     for (int mi = 0; mi < 4; ++mi) {
                         const uint2 bv = lds64(xs + mi * 128);
-                        const int pos = WD == 4 ? (mi & 1) : mi, w0 = WD == 4 ? 2 * (mi >> 1) : 0;
-                        const uint32_t m = kByteMask << (WD * pos);
-                        // the top field position of a 2- or 4-bit slice takes the words unmasked (its digits are made for that)
-                        const bool top = (WD == 2 && mi == 3) || (WD == 4 && (mi & 1));
+                        // registers (a0, a1) meet the MMA's k < 16, (a2, a3) its k >= 16: for a 1-bit slice field positions mi and
+                        // mi + 4 of the same word, else position mi (mi & 1 for 4 bits) of two consecutive words.  The top position of
+                        // a byte takes the word unmasked (its digits are made for that).
+                        const int w_lo = WD == 4 ? 2 * (mi >> 1) : 0, w_hi = WD == 1 ? 0 : w_lo + 1;
+                        const int pos_lo = i8_pos(WD, mi, 0), pos_hi = i8_pos(WD, mi, 1);
+                        const uint32_t m_lo = kByteMask << (WD * pos_lo), m_hi = kByteMask << (WD * pos_hi);
+                        const bool top_lo = WD * (pos_lo + 1) == 8, top_hi = WD * (pos_hi + 1) == 8;
 #pragma unroll
                         for (int t = 0; t < TPW; ++t) {
-                            const uint32_t a0 = top ? wd[t][w0].x : wd[t][w0].x & m, a1 = top ? wd[t][w0].y : wd[t][w0].y & m;
-                            const uint32_t a2 = top ? wd[t][w0 + 1].x : wd[t][w0 + 1].x & m, a3 = top ? wd[t][w0 + 1].y : wd[t][w0 + 1].y & m;
+                            const uint32_t a0 = top_lo ? wd[t][w_lo].x : wd[t][w_lo].x & m_lo, a1 = top_lo ? wd[t][w_lo].y : wd[t][w_lo].y & m_lo;
+                            const uint32_t a2 = top_hi ? wd[t][w_hi].x : wd[t][w_hi].x & m_hi, a3 = top_hi ? wd[t][w_hi].y : wd[t][w_hi].y & m_hi;
                             if (FIRST && mi < CHI) mma_i8_first(di[t][mi & (CHI - 1)], a0, a1, a2, a3, bv);
                             else mma_i8(di[t][mi & (CHI - 1)], a0, a1, a2, a3, bv);
                         }
