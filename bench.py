@@ -500,187 +500,399 @@ def run_gptq(args):
     print(json.dumps(line), flush=True)
 
 
-def finish_gemm_line(args, spec, layers, world, steps, warmup, ms, e2e_steps, ms_e2e, x_host, y_host, clocks):
-    """JSON line of a batched (M > 16) workload: TFLOP/s against the dense fp16 tensor peak."""
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_TENSOR_TFLOPS = 2250.0
+
+
+def measured_tensor_burst():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops"])
+    except Exception:
+        return 1590.0
+
+
+def _graph_of(fn, device):
+    """Captures fn() (already run twice on a side stream) in a CUDA graph."""
+    import torch
+    side = torch.cuda.Stream(device)
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        fn()
+        fn()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        fn()
+    torch.cuda.synchronize()
+    return graph
+
+
+class Timer:
+    """Device timing of blocks of exactly `steps` steps: barrier + synchronize on both sides, CUDA events on the
+    current stream, largest time over the ranks.  Blocks are repeated until `min_total_s` of timed work has run (a
+    handful of steps says little on a GPU whose clocks settle under its power limit after a few hundred ms)."""
+
+    def __init__(self, device, world):
+        self.device, self.world = device, world
+
+    def barrier(self):
+        import torch
+        import torch.distributed as dist
+        if self.world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def block(self, step_fn, steps):
+        import torch
+        from paper_2405_14917_b200 import replicas
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.barrier()
+        e0.record()
+        for _ in range(steps):
+            step_fn()
+        e1.record()
+        self.barrier()
+        return replicas.max_over_ranks(e0.elapsed_time(e1), self.device)
+
+    def blocks(self, step_fn, steps, min_total_s=1.0, min_blocks=1, max_blocks=400):
+        ms = [self.block(step_fn, steps)]
+        n = int(min(max_blocks, max(min_blocks, np.ceil(min_total_s * 1e3 / max(ms[0], 1e-3)))))
+        for _ in range(n - 1):                     # n follows from a number every rank has: the ranks agree on it
+            ms.append(self.block(step_fn, steps))
+        return ms
+
+
+def _timing_summary(ms_blocks, steps):
+    per = np.asarray(ms_blocks) / steps
+    return {"blocks": len(ms_blocks), "steps_per_block": steps, "ms_per_step_median": float(np.median(per)),
+            "ms_per_step_min": float(per.min()), "ms_per_step_max": float(per.max()), "timed_ms_total": float(np.sum(ms_blocks))}
+
+
+def decode_buffers(layers, M, device, seed):
+    """All activations of a sweep in one pinned host buffer and one device buffer, all outputs in another pair."""
+    import torch
+    x_off = np.cumsum([0] + [M * L.K for L in layers])
+    y_off = np.cumsum([0] + [M * L.N for L in layers])
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed)
+    x_host = torch.randn(int(x_off[-1]), generator=gen, dtype=torch.float32).to(torch.float16).pin_memory()
+    y_host = torch.empty(int(y_off[-1]), dtype=torch.float16).pin_memory()
+    x_dev = x_host.to(device)
+    y_dev = torch.zeros(int(y_off[-1]), dtype=torch.float16, device=device)
+    xs = [x_dev[x_off[i]:x_off[i + 1]].view(M, L.K) for i, L in enumerate(layers)]
+    ys = [y_dev[y_off[i]:y_off[i + 1]].view(M, L.N) for i, L in enumerate(layers)]
+    return x_host, y_host, x_dev, y_dev, xs, ys
+
+
+def decode_sweep(layers, M, device, launch, seed=1234):
+    """One pass over `layers` at M tokens as a CUDA graph.  launch: 'set' (one layer-set launch for everything),
+    'per-layer' (slim_mpq_gemv per layer) or 'decoder-order' (what a decoder can issue: per block the q/k/v
+    projections as a set of three on one x, o alone, gate/up as a set of two, down alone, in that order).
+    Returns (graph, objects to keep alive, launches of the dominant kernel per step, kernels per step, buffers)."""
+    import torch
+    from paper_2405_14917_b200 import binding as slim
+    bufs = decode_buffers(layers, M, device, seed)
+    x_host, y_host, x_dev, y_dev, xs, ys = bufs
+    ws = torch.zeros(max(L.workspace_bytes(M) for L in layers), dtype=torch.uint8, device=device)
+    slim.workspace_init(ws)
+    keep = [ws]
+    if launch == "set":
+        layer_set = slim.LayerSet(list(zip(layers, xs, ys)))
+        keep.append(layer_set)
+        run, checks, n_dom, n_kern = layer_set.run, [layer_set.check], 1, 2
+    elif launch == "per-layer":
+        def run():
+            for L, x, y in zip(layers, xs, ys):
+                L.forward(x, ws, out=y)
+        checks, n_dom, n_kern = [], len(layers), len(layers) * (2 if M >= 4 else 1)
+    else:
+        assert len(layers) % 7 == 0
+        calls, checks, n_kern = [], [], 0
+        for b0 in range(0, len(layers), 7):
+            q, k, v, o, gate, up, down = range(b0, b0 + 7)
+            qkv = slim.LayerSet([(layers[i], xs[q], ys[i]) for i in (q, k, v)])          # one input, three outputs
+            gu = slim.LayerSet([(layers[i], xs[gate], ys[i]) for i in (gate, up)])
+            keep += [qkv, gu]
+            checks += [qkv.check, gu.check]
+            calls += [qkv.run, (lambda i=o: layers[i].forward(xs[i], ws, out=ys[i])), gu.run,
+                      (lambda i=down: layers[i].forward(xs[i], ws, out=ys[i]))]
+            n_kern += 2 + 1 + 2 + 1 if M < 4 else 2 + 2 + 2 + 2
+
+        def run():
+            for c in calls:
+                c()
+        n_dom = len(calls)
+    graph = _graph_of(run, device)
+
+    def check():
+        slim.workspace_status(ws)
+        for c in checks:
+            c()
+    return graph, keep, n_dom, n_kern, bufs, check
+
+
+def decode_entry(name, layers, spec, device, timer, launch, steps, min_total_s, with_e2e=False, clock_gpu=None, warmup=5):
+    """Measures one decode configuration; returns the dict that goes into the JSON line."""
+    import torch
     M = spec["M"]
+    graph, keep, n_dom, n_kern, bufs, check = decode_sweep(layers, M, device, launch)
+    x_host, y_host, x_dev, y_dev, _, _ = bufs
+    alg_bytes = sum(L.algorithmic_bytes(M) for L in layers)
+    for _ in range(max(warmup, 3)):
+        graph.replay()
+    sampler = ClockSampler(clock_gpu) if clock_gpu is not None else None
+    if sampler:
+        sampler.start()
+    ms_blocks = timer.blocks(graph.replay, steps, min_total_s)
+    clocks = sampler.stop() if sampler else None
+    check()
+    tm = _timing_summary(ms_blocks, steps)
+    ms = tm["ms_per_step_median"]
+    value = timer.world * alg_bytes / (ms * 1e-3) / 1e9
+    peak, peak_kind = measured_hbm_peak()
+    per_launch_us = 1e3 * ms / n_dom
+    achieved = alg_bytes / n_dom / (per_launch_us * 1e-6) / 1e9
+    kernel = {"set": "gemv_set_kernel", "per-layer": "gemv_kernel", "decoder-order": "gemv_set_kernel + gemv_kernel"}[launch]
+    integer_form = M == 1 and launch != "per-layer"
+    out = {"name": name, "metric": f"mixed-precision dequant GEMV GB/s at M={M} ({spec['model']} layers, avg {spec['avg_bits']}-bit, g=128)",
+           "value": value, "unit": UNIT, "ms_per_step": ms, "timing": tm,
+           "dtype": ("s32 (mma.sync m16n8k32 u8 x s8: byte-masked code words against base-256 digits of fixed-point x; f32 fold)"
+                     if integer_form and launch == "set" else
+                     "s32 integer MMAs in the q/k/v and gate/up sets, f16 MMAs in the o and down calls" if integer_form else
+                     "f16 (mma.sync m16n8k16 on raw code fields, f32 accumulate)"),
+           "config": {"workload": name, "layers": len(layers), "M": M, "avg_bits": spec["avg_bits"], "g": wl.GROUP,
+                      "algorithmic_bytes_per_step": alg_bytes, "l2": f"distinct layers, {alg_bytes / 1e9:.2f} GB per step > L2",
+                      "launch": {"set": "CUDA graph of the layer-set launch: one persistent kernel for the whole sweep (plus one kernel that stages x)",
+                                 "per-layer": "CUDA graph of one slim_mpq_gemv launch per layer, programmatic dependent launch",
+                                 "decoder-order": "CUDA graph; per block: set(q, k, v) on one x, o, set(gate, up) on one x, down: the calls a decoder can issue, in its order"}[launch],
+                      "grouped_launch": launch != "per-layer"},
+           "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
+                        "kernel": kernel, "avg_launch_us": per_launch_us, "algorithmic_bytes_per_launch": alg_bytes / n_dom,
+                        "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS},
+           "gpu_launches_per_step": n_kern, "clocks": clocks}
+    if with_e2e:
+        def step_e2e():
+            x_dev.copy_(x_host, non_blocking=True)
+            graph.replay()
+            y_host.copy_(y_dev, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+        for _ in range(3):
+            step_e2e()
+        e2e_steps = max(steps // 4, 3)
+        ms_e2e = float(np.median(timer.blocks(step_e2e, e2e_steps, min_total_s / 4))) / e2e_steps
+        check()
+        out["e2e"] = {"value": timer.world * alg_bytes / (ms_e2e * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 2),
+                      "d2h_bytes_per_step": int(y_host.numel() * 2), "steps": e2e_steps, "ms_per_step": ms_e2e}
+    del graph, keep
+    return out
+
+
+def gemm_entry(name, layers, spec, device, timer, steps, min_total_s, with_e2e=False, clock_gpu=None, warmup=3):
+    """Measures one batched (M > 16) configuration: TFLOP/s against the dense fp16 tensor peak."""
+    import torch
+    from paper_2405_14917_b200 import binding as slim
+    M = spec["M"]
+    x_host, y_host, x_dev, y_dev, xs, ys = decode_buffers(layers, M, device, 4321)
+    ws = torch.zeros(max(L.workspace_bytes(M) for L in layers), dtype=torch.uint8, device=device)
+    slim.workspace_init(ws)
+
+    def run():
+        for L, x, y in zip(layers, xs, ys):
+            L.forward(x, ws, out=y)
+    graph = _graph_of(run, device)
+    for _ in range(max(warmup, 3)):
+        graph.replay()
+    sampler = ClockSampler(clock_gpu) if clock_gpu is not None else None
+    if sampler:
+        sampler.start()
+    ms_blocks = timer.blocks(graph.replay, steps, min_total_s)
+    clocks = sampler.stop() if sampler else None
+    slim.workspace_status(ws)
+    tm = _timing_summary(ms_blocks, steps)
+    ms = tm["ms_per_step_median"]
     flops = sum(2.0 * M * L.N * L.K for L in layers)
-    value = world * flops * steps / (ms * 1e-3) / 1e12
-    e2e_value = world * flops * e2e_steps / (ms_e2e * 1e-3) / 1e12
+    value = timer.world * flops / (ms * 1e-3) / 1e12
     peak, peak_kind = measured_tensor_peak()
     n_launch = len(layers)
-    per_launch_us = 1e3 * ms / steps / n_launch
+    per_launch_us = 1e3 * ms / n_launch
     achieved = flops / n_launch / (per_launch_us * 1e-6) / 1e12
     sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2405_14917_b200", "csrc", "slim_gemm.cu"), "rb").read()).hexdigest()
     cap = NCU_TRAFFIC_GEMM.get(sha)
-    traffic = cap["traffic_bytes"] / cap["launches"] if cap and cap["workload"] == args.workload and cap["launches"] == n_launch else None
-    line = {
-        "metric": f"mixed-precision dequant GEMM TFLOP/s at M={M} (LLaMA-13B layer shapes, avg 3-bit, g=128)",
-        "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warmup,
-        "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f16 (tcgen05 kind::f16, f32 accumulate)", "data": "synthetic",
-        "config": {"workload": args.workload, "layers": n_launch, "M": M, "avg_bits": spec["avg_bits"], "g": wl.GROUP,
-                   "flops_per_step": flops, "l2": "14 distinct layers, 258 MB of weights per step > L2",
-                   "launch": "CUDA graph of one launch per layer", "parallelism": f"replicas x{world}"},
-        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                     "peak_kind": peak_kind, "kernel": "gemm_kernel", "avg_launch_us": per_launch_us,
-                     "flops_per_launch": flops / n_launch, "traffic": traffic, "frac_of_nominal_2250": achieved / 2250.0},
-        "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": int(x_host.numel() * 2),
-                "d2h_bytes_per_step": int(y_host.numel() * 2), "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
-        "gpu_launches": steps * n_launch,
-        "clocks": clocks,
-    }
-    print(json.dumps(line), flush=True)
+    traffic = cap["traffic_bytes"] / cap["launches"] if cap and cap["workload"] == name and cap["launches"] == n_launch else None
+    out = {"name": name, "metric": f"mixed-precision dequant GEMM TFLOP/s at M={M} (LLaMA-13B layer shapes, avg 3-bit, g=128)",
+           "value": value, "unit": "TFLOP/s", "ms_per_step": ms, "timing": tm, "dtype": "f16 (tcgen05 kind::f16, f32 accumulate)",
+           "config": {"workload": name, "layers": n_launch, "M": M, "avg_bits": spec["avg_bits"], "g": wl.GROUP, "flops_per_step": flops,
+                      "l2": "14 distinct layers, 258 MB of weights per step > L2", "launch": "CUDA graph of one launch per layer"},
+           "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "peak_kind": peak_kind,
+                        "frac_of_burst": achieved / measured_tensor_burst(), "frac_of_nominal_2250": achieved / NOMINAL_TENSOR_TFLOPS,
+                        "kernel": "gemm_kernel", "avg_launch_us": per_launch_us, "flops_per_launch": flops / n_launch, "traffic": traffic},
+           "gpu_launches_per_step": n_launch, "clocks": clocks}
+    if with_e2e:
+        def step_e2e():
+            x_dev.copy_(x_host, non_blocking=True)
+            graph.replay()
+            y_host.copy_(y_dev, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+        for _ in range(3):
+            step_e2e()
+        e2e_steps = max(steps // 4, 3)
+        ms_e2e = float(np.median(timer.blocks(step_e2e, e2e_steps, min_total_s / 4))) / e2e_steps
+        slim.workspace_status(ws)
+        out["e2e"] = {"value": timer.world * flops / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": int(x_host.numel() * 2),
+                      "d2h_bytes_per_step": int(y_host.numel() * 2), "steps": e2e_steps, "ms_per_step": ms_e2e}
+    return out
+
+
+def single_layer_entry(layer, device, timer, copies=64):
+    """Config 1: one 4096 x 4096 layer at M = 1 through slim_mpq_gemv.  (a) latency of an isolated launch with a cold
+    L2 (a 256 MB buffer is overwritten before every call); (b) throughput over `copies` distinct copies of the layer
+    (303 MB > L2), one launch each, replayed from a CUDA graph; (c) the same copies as one layer-set launch."""
+    import torch
+    from paper_2405_14917_b200 import binding as slim
+    M = 1
+    clones = [slim.QuantLinear(layer.packed.clone(), layer.bits, layer.scales.clone(), layer.zeros.clone(), layer.N, layer.K) for _ in range(copies)]
+    alg = layer.algorithmic_bytes(M)
+    # (a)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    ws = slim.new_workspace(M, layer.N, layer.K, layer.bits)
+    x = torch.randn(M, layer.K, device=device).half()
+    y = torch.empty(M, layer.N, dtype=torch.float16, device=device)
+    lat = []
+    for i in range(40):
+        flush.fill_(i & 1)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        clones[i % copies].forward(x, ws, out=y)
+        e1.record()
+        torch.cuda.synchronize()
+        lat.append(e0.elapsed_time(e1) * 1e3)
+    slim.workspace_status(ws)
+    del flush
+    spec = dict(model="llama-7b", avg_bits=2, M=1)
+    per_layer = decode_entry("single-4096x4096-avg2-m1-rotating-per-layer", clones, spec, device, timer, "per-layer", 20, 0.3)
+    as_set = decode_entry("single-4096x4096-avg2-m1-rotating-set", clones, spec, device, timer, "set", 20, 0.3)
+    peak, _ = measured_hbm_peak()
+    return {"name": "single-4096x4096-avg2-m1", "metric": "one 4096 x 4096 layer, avg 2-bit, M = 1 (slim_mpq_gemv)",
+            "isolated_launch_us": {"median": float(np.median(lat[5:])), "min": float(np.min(lat[5:])), "max": float(np.max(lat[5:])),
+                                   "what": "one call timed with CUDA events around it, L2 flushed before every call, includes launch latency"},
+            "isolated_launch_gbs": alg / (float(np.median(lat[5:])) * 1e-6) / 1e9,
+            "ideal_us_at_measured_peak": alg / (peak * 1e9) * 1e6, "algorithmic_bytes": alg,
+            "rotating_copies": copies, "rotating_per_layer": per_layer, "rotating_set": as_set}
+
+
+def cpu_baseline_legs(spec):
+    """The oracle as it stands on the host cores: all cores (the reported baseline) and one core."""
+    base = cpu_baseline(spec, budget_s=10.0)
+    from oracle import slim_oracle_c as oc
+    layers = _oracle_layers(spec, 1)
+    L = layers[0]
+    rows = 512
+    codes, scales, zeros = L["codes"][:rows], np.ascontiguousarray(L["scales"][:, :rows]), np.ascontiguousarray(L["zeros"][:, :rows])
+    oc.linear_f64(L["x"], codes, scales, zeros, threads=1)
+    t0 = time.perf_counter()
+    reps = 0
+    while time.perf_counter() - t0 < 4.0:
+        oc.linear_f64(L["x"], codes, scales, zeros, threads=1)
+        reps += 1
+    dt = time.perf_counter() - t0
+    nbytes = wl.algorithmic_bytes(L["x"].shape[0], rows, L["K"], L["bits"]) * reps
+    oc.linear_f64(L["x"], codes, scales, zeros, threads=base["cores"])          # back to all cores
+    base["single_thread"] = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": 1,
+                             "sample": f"first {rows} output rows of layer q, block 0, x {reps} passes, {dt:.1f} s"}
+    return base
+
+
+def secondary_entries(args, device, timer, primary_layers, clock_gpu):
+    """The rest of the metric and of the configurations, each timed for about a second, for the same JSON line."""
+    import torch
+    out = []
+
+    def guarded(fn):
+        try:
+            out.append(fn())
+        except Exception as e:               # a secondary entry never takes the primary line down
+            out.append({"name": getattr(fn, "__name__", "entry"), "error": f"{type(e).__name__}: {e}"})
+        torch.cuda.empty_cache()
+
+    spec7 = workload_spec("llama7b-decode-avg2")
+    guarded(lambda: decode_entry("llama7b-decode-avg2-m1-per-layer", primary_layers, spec7, device, timer, "per-layer", 50, 0.5, clock_gpu=clock_gpu))
+    guarded(lambda: decode_entry("llama7b-decode-avg2-m1-decoder-order", primary_layers, spec7, device, timer, "decoder-order", 50, 0.5, clock_gpu=clock_gpu))
+    guarded(lambda: single_layer_entry(primary_layers[0], device, timer))
+    for wname in ("llama13b-prefill-avg3-m2048", "llama13b-prefill-avg3-m512"):
+        spec = workload_spec(wname)
+        layers13 = build_layers(spec, device, 0) if wname.endswith("m2048") else layers13
+        guarded(lambda: gemm_entry(wname, layers13, spec, device, timer, 20, 1.0, clock_gpu=clock_gpu))
+    del layers13
+    torch.cuda.empty_cache()
+    spec3 = workload_spec("llama7b-decode-avg3-m1-blocks8")
+    layers3 = build_layers(spec3, device, 0)
+    for M in (1, 4, 8, 16):
+        sp = dict(spec3, M=M)
+        guarded(lambda: decode_entry(f"llama7b-decode-avg3-m{M}-blocks8", layers3, sp, device, timer, "set", 50, 0.6, clock_gpu=clock_gpu))
+    del layers3
+    torch.cuda.empty_cache()
+    spec70 = workload_spec("llama70b-decode-avg2-m1")
+    layers70 = build_layers(spec70, device, 0)
+    for M in (1, 16):
+        sp = dict(spec70, M=M)
+        guarded(lambda: decode_entry(f"llama70b-decode-avg2-m{M}-blocks8", layers70, sp, device, timer, "set", 20, 0.6, clock_gpu=clock_gpu))
+    guarded(lambda: decode_entry("llama70b-decode-avg2-m1-blocks8-per-layer", layers70, dict(spec70, M=1), device, timer, "per-layer", 20, 0.5, clock_gpu=clock_gpu))
+    del layers70
+    torch.cuda.empty_cache()
+    return out
 
 
 def run_ours(args, spec):
     import torch
     import torch.distributed as dist
     from paper_2405_14917_b200 import binding as slim
-    from paper_2405_14917_b200 import replicas
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    steps = args.steps if args.steps is not None else (2000 if spec["M"] <= 16 else 300)
+    steps = args.steps if args.steps is not None else (200 if spec["M"] <= 16 else 50)
     warmup = max(args.warmup if args.warmup is not None else 20, 3)
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
     slim.lib()   # fails loudly if the CUDA library is missing
-
+    timer = Timer(device, world)
     layers = build_layers(spec, device, rank)
     M = spec["M"]
-    alg_bytes = sum(L.algorithmic_bytes(M) for L in layers)
-
-    # all activations of the sweep in one buffer, all outputs in another
-    x_off = np.cumsum([0] + [M * L.K for L in layers])
-    y_off = np.cumsum([0] + [M * L.N for L in layers])
-    gen = torch.Generator(device="cpu")
-    gen.manual_seed(1234 + rank)
-    x_host = torch.randn(int(x_off[-1]), generator=gen, dtype=torch.float32).to(torch.float16).pin_memory()
-    y_host = torch.empty(int(y_off[-1]), dtype=torch.float16).pin_memory()
-    x_dev = x_host.to(device)
-    y_dev = torch.zeros(int(y_off[-1]), dtype=torch.float16, device=device)
-    ws = torch.zeros(max(L.workspace_bytes(M) for L in layers), dtype=torch.uint8, device=device)
-    slim.workspace_init(ws)
-    xs = [x_dev[x_off[i]:x_off[i + 1]].view(M, L.K) for i, L in enumerate(layers)]
-    ys = [y_dev[y_off[i]:y_off[i + 1]].view(M, L.N) for i, L in enumerate(layers)]
-
-    use_set = M <= slim.GEMV_MAX_M and args.launch == "set"
-    layer_set = slim.LayerSet(list(zip(layers, xs, ys))) if use_set else None
-
-    def sweep():
-        if use_set:
-            layer_set.run()
-            return
-        for L, x, y in zip(layers, xs, ys):
-            L.forward(x, ws, out=y)
-
-    # capture one sweep in a CUDA graph (launch-bound otherwise: ~1.4 us of HBM time per layer)
-    side = torch.cuda.Stream(device)
-    side.wait_stream(torch.cuda.current_stream())
-    with torch.cuda.stream(side):
-        sweep()
-        sweep()
-    torch.cuda.current_stream().wait_stream(side)
-    torch.cuda.synchronize()
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph):
-        sweep()
-    torch.cuda.synchronize()
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def timed(step_fn, n):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        e0.record()
-        for _ in range(n):
-            step_fn()
-        e1.record()
-        barrier()
-        return replicas.max_over_ranks(e0.elapsed_time(e1), device)
-
-    def step_device():
-        graph.replay()
-
-    def step_e2e():
-        x_dev.copy_(x_host, non_blocking=True)
-        graph.replay()
-        y_host.copy_(y_dev, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
-
-    for _ in range(warmup):
-        step_device()
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    ms = timed(step_device, steps)
-    clocks = sampler.stop() if rank == 0 else None
-    slim.workspace_status(ws)
-    if use_set:
-        layer_set.check()
-
-    e2e_steps = max(steps // 4, 3)
-    for _ in range(3):
-        step_e2e()
-    ms_e2e = timed(step_e2e, e2e_steps)
-    slim.workspace_status(ws)
-    if use_set:
-        layer_set.check()
-
+    clock_gpu = local_rank if rank == 0 else None
+    launch = "set" if (M <= slim.GEMV_MAX_M and args.launch == "set") else "per-layer"
+    if M > slim.GEMV_MAX_M:
+        entry = gemm_entry(args.workload, layers, spec, device, timer, steps, args.min_seconds, with_e2e=True, clock_gpu=clock_gpu, warmup=warmup)
+    else:
+        entry = decode_entry(args.workload, layers, spec, device, timer, launch if args.launch != "decoder-order" else "decoder-order",
+                             steps, args.min_seconds, with_e2e=True, clock_gpu=clock_gpu, warmup=warmup)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
-
-    # launches of the dominant kernel per step: the persistent kernel once, or one kernel per layer
-    n_launch = 1 if use_set else len(layers)
-    per_launch_us = 1e3 * ms / steps / n_launch
-    if M > slim.GEMV_MAX_M:
-        finish_gemm_line(args, spec, layers, world, steps, warmup, ms, e2e_steps, ms_e2e, x_host, y_host, clocks)
-        if world > 1:
-            dist.destroy_process_group()
-        return
-    value = world * alg_bytes * steps / (ms * 1e-3) / 1e9
-    e2e_value = world * alg_bytes * e2e_steps / (ms_e2e * 1e-3) / 1e9
-    peak, peak_kind = measured_hbm_peak()
-    achieved = alg_bytes / n_launch / (per_launch_us * 1e-6) / 1e9
-    kernel_file = "slim_gemv_set.cu" if use_set else "slim_gemv.cu"
-    sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2405_14917_b200", "csrc", kernel_file), "rb").read()).hexdigest()
-    traffic = NCU_TRAFFIC.get(sha)
-    # the set launch also runs the small kernel that puts x into fragment order; its time is inside avg_launch_us
-    kernels_per_step = 2 if use_set else len(layers) * (2 if M >= 4 else 1)
-    line = {
-        "metric": METRIC if args.workload == "llama7b-decode-avg2" else
-                  f"mixed-precision dequant GEMV GB/s at M={M} ({spec['model']} layer set, avg {spec['avg_bits']}-bit, g=128)",
-        "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-        "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": ("s32 (mma.sync m16n8k32 u8 x s8: byte-masked code words against base-256 digits of fixed-point x; f32 fold)"
-                  if use_set and M == 1 else "f16 (mma.sync m16n8k16 on raw code fields, f32 accumulate)"), "data": "synthetic",
-        "config": {"workload": args.workload, "layers": len(layers), "M": M, "avg_bits": spec["avg_bits"], "g": wl.GROUP,
-                   "algorithmic_bytes_per_step": alg_bytes, "l2": f"distinct layers, {alg_bytes / 1e9:.2f} GB per step >> L2",
-                   "launch": ("CUDA graph of the layer-set launch: one persistent kernel for the whole sweep "
-                              "(plus one kernel that stages x)") if use_set else
-                             "CUDA graph of one launch per layer, programmatic dependent launch",
-                   "grouped_launch": bool(use_set),
-                   "parallelism": f"replicas x{world}"},
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": peak_kind, "kernel": "gemv_set_kernel" if use_set else "gemv_kernel", "avg_launch_us": per_launch_us,
-                     "algorithmic_bytes_per_launch": alg_bytes / n_launch,
-                     "traffic": (traffic["traffic_bytes"] / traffic["algorithmic_bytes"] * alg_bytes / n_launch) if traffic else None,
-                     "frac_of_nominal_8000": achieved / 8000.0},
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 2),
-                "d2h_bytes_per_step": int(y_host.numel() * 2), "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
-        "gpu_launches": steps * kernels_per_step,
-        "clocks": clocks,
-    }
+    tm = entry["timing"]
+    line = {"metric": METRIC if args.workload == "llama7b-decode-avg2" else entry["metric"],
+            "value": entry["value"], "unit": entry["unit"], "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": entry["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": entry["dtype"], "data": "synthetic",
+            "config": dict(entry["config"], parallelism=f"replicas x{world}",
+                           timing=f"median of {tm['blocks']} blocks of exactly {steps} steps each (barrier + synchronize around every block)"),
+            "timing": tm, "roofline": entry["roofline"], "e2e": entry["e2e"],
+            "gpu_launches": steps * tm["blocks"] * entry["gpu_launches_per_step"], "clocks": entry["clocks"]}
+    if M <= slim.GEMV_MAX_M and launch == "set":
+        sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2405_14917_b200", "csrc", "slim_gemv_set.cu"), "rb").read()).hexdigest()
+        traffic = NCU_TRAFFIC.get(sha)
+        line["roofline"]["traffic"] = (traffic["traffic_bytes"] / traffic["algorithmic_bytes"] * entry["roofline"]["algorithmic_bytes_per_launch"]) if traffic else None
+    elif "traffic" not in line["roofline"]:
+        line["roofline"]["traffic"] = None
+    if world == 1 and args.workload == "llama7b-decode-avg2" and not args.no_secondary:
+        line["secondary"] = secondary_entries(args, device, timer, layers, clock_gpu)
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(spec)
+        line["cpu_baseline"] = cpu_baseline_legs(spec) if M <= slim.GEMV_MAX_M else cpu_baseline(spec)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -694,8 +906,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama7b-decode-avg2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--launch", default="set", choices=["set", "per-layer"],
-                    help="decode workloads (M <= 16): the layer-set launch (one persistent kernel for the sweep) or one launch per layer")
+    ap.add_argument("--launch", default="set", choices=["set", "per-layer", "decoder-order"],
+                    help="decode workloads (M <= 16): the layer-set launch (one persistent kernel for the sweep), one launch per layer, "
+                         "or the calls a decoder can issue (per block: q/k/v as a set, o, gate/up as a set, down)")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="blocks of --steps steps are repeated until this much timed work has run; the median block is reported")
+    ap.add_argument("--no-secondary", action="store_true", help="default workload only: skip the other configurations of the same JSON line")
     args = ap.parse_args()
     if args.workload == "sqc-llama7b-block" and args.impl != "reference":
         run_sqc(args)
