@@ -61,7 +61,7 @@ struct SetLayer {
     __half* y;
     size_t x_off;          // workspace offset of the layer's staged activations, group after group:
                            // (sum_k x, 2^(24-S)) float2[16], then the fragments [slice][8 mma][MP][4 lanes] x 8 B
-    size_t pad0;
+    size_t part_off;       // workspace offset of the layer's fp32 partial outputs [split][M][N] (split > 1 only)
     int M, N, K, G;
     uint16_t count[4];     // groups of 1, 2, 3, 4 bits
     int task0;             // first (token, group) staging task of the layer
@@ -72,7 +72,8 @@ struct SetLayer {
     uint16_t pre3[SLIM_MAX_GROUPS + 1];   // 3-bit groups (two slices) before group j
     uint8_t bits[SLIM_MAX_GROUPS];
     uint8_t order[SLIM_MAX_GROUPS];       // the order in which the groups are streamed: by bit-width, then by index
-    uint8_t pad2[4];
+    uint8_t split;                        // parts the groups of a row block are cut into (1: whole K per item)
+    uint8_t pad2[3];
 };
 static_assert(sizeof(SetLayer) % 16 == 0, "descriptors are copied and read in 16-byte pieces");
 
@@ -80,11 +81,15 @@ static_assert(sizeof(SetLayer) % 16 == 0, "descriptors are copied and read in 16
 // the layer's descriptor.
 struct SetItem {
     int layer, rb;         // layer of the set, row block inside the layer
-    int N, G;
-    __half* y;
+    int N;
+    int range;             // the item's groups: positions [range & 0xffff, range >> 16) of the layer's streaming order
+    __half* y;             // the layer's y; for an item that covers part of the groups, the workspace offset of its fp32
+                           // partial output [M][N] instead
     int M;
-    int counts;            // groups of 1, 2 and 3 bits, 9 bits each (the rest of G has 4): the groups arrive in that order
+    int counts;            // the layer's groups of 1, 2 and 3 bits, 9 bits each (the rest has 4), i.e. where each width
+                           // starts in the streaming order; bit 30: partial item
 };
+constexpr int kItemPartial = 1 << 30;
 static_assert(sizeof(SetItem) == 32, "items are read as two 16-byte pieces");
 
 // Plan buffer: int item_begin[grid + 1] (padded to kSetPlanHeader bytes), the descriptors, then the
@@ -309,9 +314,9 @@ __device__ __forceinline__ void consume_one(const SetParams& p, const uint32_t s
     const int4* items4 = reinterpret_cast<const int4*>(p.items);
     int4 it_a = items4[2 * i0], it_b = items4[2 * i0 + 1];       // (layer, rb, N, G), (y, M, counts)
     for (int i = i0; i < i1 && ok; ++i) {
-        const int rb = it_a.y, N = it_a.z, G = it_a.w, counts = it_b.w;
-        __half* const ybase = reinterpret_cast<__half*>((static_cast<unsigned long long>(static_cast<uint32_t>(it_b.y)) << 32) |
-                                                        static_cast<uint32_t>(it_b.x));
+        const int rb = it_a.y, N = it_a.z, p0 = it_a.w & 0xffff, p1 = it_a.w >> 16, counts = it_b.w;
+        const int G = p1 - p0;                                   // groups of this item
+        const unsigned long long yword = (static_cast<unsigned long long>(static_cast<uint32_t>(it_b.y)) << 32) | static_cast<uint32_t>(it_b.x);
         if (i + 1 < i1) {                                        // the next item arrives during this one's groups
             it_a = items4[2 * i + 2];
             it_b = items4[2 * i + 3];
@@ -407,15 +412,20 @@ __device__ __forceinline__ void consume_one(const SetParams& p, const uint32_t s
             }
             return true;
         };
-        const int c1 = counts & 511, c2 = (counts >> 9) & 511, c3 = (counts >> 18) & 511;
-        ok = run_groups(WidthTag<1>{}, c1) && run_groups(WidthTag<2>{}, c2) && run_groups(WidthTag<3>{}, c3) &&
-             run_groups(WidthTag<4>{}, G - c1 - c2 - c3);
+        // the widths start at positions 0, e1, e2, e3 of the layer's streaming order; the item covers [p0, p1)
+        const int e1 = counts & 511, e2 = e1 + ((counts >> 9) & 511), e3 = e2 + ((counts >> 18) & 511);
+        auto part = [&](int a, int b) { return max(min(p1, b) - max(p0, a), 0); };
+        ok = run_groups(WidthTag<1>{}, part(0, e1)) && run_groups(WidthTag<2>{}, part(e1, e2)) &&
+             run_groups(WidthTag<3>{}, part(e2, e3)) && run_groups(WidthTag<4>{}, part(e3, 65535));
         if (ok) {
 #pragma unroll
             for (int t = 0; t < TPW; ++t) {
                 if (t >= n_act) break;
-                __half* yrow = ybase + 16 * (tile0 + t) + 2 * gq;
-                if (c == 2 * t) *reinterpret_cast<__half2*>(yrow) = __floats2half2_rn(acc0, acc2);
+                const int row = 16 * (tile0 + t) + 2 * gq;
+                if (c == 2 * t) {
+                    if (counts & kItemPartial) *reinterpret_cast<float2*>(reinterpret_cast<float*>(p.ws + yword) + row) = make_float2(acc0, acc2);
+                    else *reinterpret_cast<__half2*>(reinterpret_cast<__half*>(yword) + row) = __floats2half2_rn(acc0, acc2);
+                }
             }
         }
     }
@@ -466,10 +476,11 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
             uint32_t ph = 0;
             uint32_t cnt = 0;                             // running number of the group in this CTA's range
             bool ok = true;
-            int l = p.items[i0].layer, rb = p.items[i0].rb;
+            int l = p.items[i0].layer, rb = p.items[i0].rb, range = p.items[i0].range;
             for (int i = i0; i < i1 && ok; ++i) {
                 // the next item's place is fetched while this one's groups are issued
                 const int l_next = i + 1 < i1 ? p.items[i + 1].layer : 0, rb_next = i + 1 < i1 ? p.items[i + 1].rb : 0;
+                const int range_next = i + 1 < i1 ? p.items[i + 1].range : 0;
                 if (have != l) {
                     const uint4* src = reinterpret_cast<const uint4*>(p.layers + l);
                     uint4* dst = reinterpret_cast<uint4*>(desc);
@@ -477,7 +488,8 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                     __syncwarp();
                     have = l;
                 }
-                const int N = D->N, MP = D->MP, G = D->G;
+                const int N = D->N, MP = D->MP;
+                const int p0 = range & 0xffff, p1 = range >> 16;        // the item's positions in the streaming order
                 const int tiles_here = min(TPI, (N >> 4) - TPI * rb);
                 // lane 0 brings the slices, lanes 1 and 2 scales and zeros, lane 3 the staged activations
                 const uint8_t* base = lane == 0 ? D->packed
@@ -486,9 +498,9 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                                                 : p.ws + D->x_off;
                 const uint32_t dst_off = lane == 0 ? kOffW : lane == 1 ? kSlotOffS : lane == 2 ? kOffZ : kOffE;
                 const uint32_t szb = static_cast<uint32_t>(tiles_here) * 32u;
-                int jj = static_cast<int>((static_cast<uint32_t>(pw) + kSetProducers - cnt % kSetProducers) % kSetProducers);
-                cnt += static_cast<uint32_t>(G);
-                for (; jj < G; jj += kSetProducers) {
+                int jj = p0 + static_cast<int>((static_cast<uint32_t>(pw) + kSetProducers - cnt % kSetProducers) % kSetProducers);
+                cnt += static_cast<uint32_t>(p1 - p0);
+                for (; jj < p1; jj += kSetProducers) {
                     // the lanes go on, or give up, together
                     if (!__all_sync(0xffffffffu, sb::wait(empty(s), ph ^ 1u, abort))) { ok = false; break; }
                     const int j = D->order[jj];            // the groups are streamed sorted by bit-width
@@ -511,6 +523,7 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                 }
                 l = l_next;
                 rb = rb_next;
+                range = range_next;
             }
             if (!ok && lane == 0) {
                 // leave no copy in flight: give what was issued a millisecond to land
@@ -529,9 +542,9 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
             const int4* items4 = reinterpret_cast<const int4*>(p.items);
             int4 it_a = items4[2 * i0], it_b = items4[2 * i0 + 1];   // (layer, rb, N, G), (y, M, -)
             for (int i = i0; i < i1 && ok; ++i) {
-                const int rb = it_a.y, N = it_a.z, G = it_a.w, M = it_b.z;
-                __half* const ybase = reinterpret_cast<__half*>((static_cast<unsigned long long>(static_cast<uint32_t>(it_b.y)) << 32) |
-                                                                static_cast<uint32_t>(it_b.x));
+                const int rb = it_a.y, N = it_a.z, G = (it_a.w >> 16) - (it_a.w & 0xffff), M = it_b.z;
+                const bool partial = (it_b.w & kItemPartial) != 0;
+                const unsigned long long yword = (static_cast<unsigned long long>(static_cast<uint32_t>(it_b.y)) << 32) | static_cast<uint32_t>(it_b.x);
                 if (i + 1 < i1) {                                     // the next item arrives during this one's groups
                     it_a = items4[2 * i + 2];
                     it_b = items4[2 * i + 3];
@@ -581,7 +594,7 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
 #pragma unroll
                                     for (int n = 0; n < NT; ++n) {
                                         // fragment of token 8n + gq (tokens the layer lacks are staged as zeros)
-                                        const uint2 bv = lds64(xs_slot + ((mi * MPK + (ONE ? 0 : 8 * n + gq)) * 4 + c) * 8);
+                                        const uint2 bv = lds64(xs_slot + ((mi * MPK + 8 * n + gq) * 4 + c) * 8);
 #pragma unroll
                                         for (int t = 0; t < TPW; ++t) {
                                             const uint32_t a0 = pair<WD>(wd[t].x, shx[t], 2 * ii), a1 = pair<WD>(wd[t].y, shy[t], 2 * ii);
@@ -609,17 +622,7 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                             const uint32_t z2 = lds32(slot + kOffZ + tt * 32 + gq * 4);
                             const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
                             const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
-                            if (ONE) {
-                                const uint2 tkw = lds64(slot + kOffE);                   // (sum_k x, 2^(24-S)) of token 0
-                                const float2 tk = make_float2(__uint_as_float(tkw.x), __uint_as_float(tkw.y));
-                                float e0 = d[t][0][0][0] + d[t][1][0][0], e2 = d[t][0][0][2] + d[t][1][0][2];
-                                if (CH == 4) {
-                                    e0 += d[t][2 % CH][0][0] + d[t][3 % CH][0][0];
-                                    e2 += d[t][2 % CH][0][2] + d[t][3 % CH][0][2];
-                                }
-                                acc[t][0][0] = fmaf(sf.x, fmaf(-zf.x, tk.x, e0 * tk.y), acc[t][0][0]);
-                                acc[t][0][2] = fmaf(sf.y, fmaf(-zf.y, tk.x, e2 * tk.y), acc[t][0][2]);
-                            } else {
+                            {
 #pragma unroll
                                 for (int n = 0; n < NT; ++n) {
                                     const float4 tk = *reinterpret_cast<const float4*>(sxe + 8 * n + 2 * c);   // (sx0, e0, sx1, e1)
@@ -648,16 +651,16 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
 #pragma unroll
                     for (int t = 0; t < TPW; ++t) {
                         if (t >= n_act) break;
-                        __half* yrow = ybase + 16 * (tile0 + t) + 2 * gq;
-                        if (ONE) {
-                            // the lane pair c >> 1 holds tile c >> 1 (in acc[0]); its even lane stores
-                            if (c == 2 * t) *reinterpret_cast<__half2*>(yrow) = __floats2half2_rn(acc[0][0][0], acc[0][0][2]);
-                        } else {
+                        const int row = 16 * (tile0 + t) + 2 * gq;
 #pragma unroll
-                            for (int n = 0; n < NT; ++n) {
-                                const int m0 = 8 * n + 2 * c;
-                                if (m0 < M) *reinterpret_cast<__half2*>(yrow + static_cast<size_t>(m0) * N) = __floats2half2_rn(acc[t][n][0], acc[t][n][2]);
-                                if (m0 + 1 < M) *reinterpret_cast<__half2*>(yrow + static_cast<size_t>(m0 + 1) * N) = __floats2half2_rn(acc[t][n][1], acc[t][n][3]);
+                        for (int n = 0; n < NT; ++n) {
+#pragma unroll
+                            for (int q = 0; q < 2; ++q) {                    // tokens 8n + 2c and 8n + 2c + 1
+                                const int m = 8 * n + 2 * c + q;
+                                if (m >= M) continue;
+                                const size_t at = static_cast<size_t>(m) * N + row;
+                                if (partial) *reinterpret_cast<float2*>(reinterpret_cast<float*>(p.ws + yword) + at) = make_float2(acc[t][n][q], acc[t][n][2 + q]);
+                                else *reinterpret_cast<__half2*>(reinterpret_cast<__half*>(yword) + at) = __floats2half2_rn(acc[t][n][q], acc[t][n][2 + q]);
                             }
                         }
                     }
@@ -668,6 +671,27 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
     }
     __syncthreads();
     if (tid == 0 && *abort != 0) atomicOr(reinterpret_cast<unsigned int*>(p.ws), 1u);
+}
+
+// ------------------------------------------------------------------------------------------ split row blocks: the sum of the parts
+// y = fp16(sum over the parts of a layer's fp32 partial outputs, in part order) for the layers whose groups were cut
+// into several items.  Block (bx, l) walks layer l's outputs in steps of the grid's x extent.
+__global__ void __launch_bounds__(256) gemv_set_finish_kernel(const SetLayer* __restrict__ layers, const uint8_t* __restrict__ ws) {
+    const SetLayer& L = layers[blockIdx.y];
+    const int S = L.split;
+    if (S <= 1) return;
+    const size_t pairs = static_cast<size_t>(L.M) * L.N / 2;
+    const float2* part = reinterpret_cast<const float2*>(ws + L.part_off);
+    __half2* y = reinterpret_cast<__half2*>(L.y);
+    for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < pairs; i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        float2 sum = part[i];
+        for (int k = 1; k < S; ++k) {
+            const float2 v = part[static_cast<size_t>(k) * pairs + i];
+            sum.x += v.x;
+            sum.y += v.y;
+        }
+        y[i] = __floats2half2_rn(sum.x, sum.y);
+    }
 }
 
 // ------------------------------------------------------------------------------------------ self-test of the bounded wait
@@ -695,10 +719,18 @@ struct SetGeometry {
     int nt, bmax, mmax, tpw, mpad;     // tpw: tiles per consumer warp; mpad: tokens in the staged layout
     int slot_bytes;
     int n_slots, grid, ctas_per_sm;
+    int split;                         // parts the groups of every row block are cut into (fewer for layers with few groups)
     size_t smem_bytes;
     long long n_items, n_tasks;
     size_t ws_bytes;
 };
+constexpr int kSetMaxSplit = 8;
+constexpr int kSetMinGroupsPerPart = 4;
+// Parts of a layer with G groups when the set asks for `split`.
+static int layer_split(int split, int G) {
+    const int cap = G / kSetMinGroupsPerPart > 1 ? G / kSetMinGroupsPerPart : 1;
+    return split < cap ? split : cap;
+}
 
 static size_t align_to(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // Workspace of one layer: per group the sums and the fragments of its slices.
@@ -711,10 +743,10 @@ static size_t layer_ws_bytes(int M, const GroupTable& gt) {
 // weighs what a consumer warp issues for it: about 70 / 73 / 120 / 80 instructions at 1 / 2 / 3 / 4 bits
 // (counted in the kernel's loops: one AND per operand register, one MMA per four, the fragment loads and
 // the fold).
-static unsigned long long item_cost(int tiles_here, const GroupTable& gt) {
+static unsigned long long item_cost(int tiles_here, const GroupTable& gt, const uint8_t* order, int p0, int p1) {
     static const unsigned kGroupWork[5] = {0, 70, 73, 120, 80};
     unsigned long long w = 0;
-    for (int j = 0; j < gt.G; ++j) w += kGroupWork[gt.bits[j]];
+    for (int q = p0; q < p1; ++q) w += kGroupWork[gt.bits[order[q]]];
     return w * static_cast<unsigned long long>(tiles_here);
 }
 
@@ -749,6 +781,23 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     }
     if (sg->n_items > 0x3fffffff || sg->n_tasks > 0x3fffffff) return SLIM_ERR_UNSUPPORTED;
     sg->nt = sg->mmax <= 8 ? 1 : 2;
+    // A set with fewer row blocks than persistent CTAs cuts the groups of every row block into parts (items of their
+    // own, fp32 partial outputs in the workspace, summed in part order by a small kernel afterwards).
+    const long long want = static_cast<long long>(set_sm_count()) * kSetCtasPerSm;
+    sg->split = 1;
+    if (sg->n_items < want) {
+        long long sp = (want + sg->n_items - 1) / sg->n_items;
+        sg->split = static_cast<int>(sp < kSetMaxSplit ? sp : kSetMaxSplit);
+    }
+    if (sg->split > 1) {
+        sg->n_items = 0;
+        for (int l = 0; l < n_layers; ++l) {
+            const slim_layer& L = layers[l];
+            const int sp = layer_split(sg->split, L.K / SLIM_GROUP);
+            sg->n_items += static_cast<long long>(sp) * (((L.N >> 4) + tpi - 1) / tpi);
+            if (sp > 1) sg->ws_bytes += align_to(static_cast<size_t>(sp) * L.M * L.N * sizeof(float), 128);
+        }
+    }
     sg->slot_bytes = static_cast<int>(align_to(static_cast<size_t>(slot_off_w(tpi, sg->mpad)) + static_cast<size_t>(tpi) * 256 * sg->bmax, 128));
     // as many CTAs per SM (kSetCtasPerSm at most) as still leaves each a ring of 5 slots
     const size_t per_sm = 224 * 1024;
@@ -832,6 +881,22 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
     const int tpi = slim::kSetConsumers * sg.tpw;
     int task = 0;
     size_t ws_off = 256;
+    // workspace: the staged activations of all layers, then the fp32 partial outputs of the layers that are split
+    std::vector<size_t> part_off(static_cast<size_t>(n_layers), 0);
+    {
+        size_t off = 256;
+        for (int l = 0; l < n_layers; ++l) {
+            slim::GroupTable gt;
+            slim::make_group_table(layers_host[l].N, layers_host[l].K, g, layers_host[l].bits_host, &gt);
+            off += slim::layer_ws_bytes(sg.mpad, gt);
+        }
+        for (int l = 0; l < n_layers; ++l) {
+            const slim_layer& L = layers_host[l];
+            const int sp = slim::layer_split(sg.split, L.K / SLIM_GROUP);
+            part_off[l] = off;
+            if (sp > 1) off += slim::align_to(static_cast<size_t>(sp) * L.M * L.N * sizeof(float), 128);
+        }
+    }
     for (int l = 0; l < n_layers; ++l) {
         const slim_layer& L = layers_host[l];
         slim::GroupTable gt;
@@ -848,6 +913,9 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
         d.task0 = task;
         d.x_off = ws_off;
         ws_off += slim::layer_ws_bytes(sg.mpad, gt);
+        const int sp = slim::layer_split(sg.split, gt.G);
+        d.split = static_cast<uint8_t>(sp);
+        d.part_off = part_off[l];
         memcpy(d.prefix, gt.prefix, sizeof d.prefix);
         memcpy(d.bits, gt.bits, sizeof d.bits);
         d.pre3[0] = 0;
@@ -862,12 +930,21 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
         const int n_rb = ((L.N >> 4) + tpi - 1) / tpi;
         for (int rb = 0; rb < n_rb; ++rb) {
             const int th = (L.N >> 4) - tpi * rb;
-            slim::SetItem it;
-            memset(&it, 0, sizeof it);
-            it.layer = l; it.rb = rb; it.N = L.N; it.G = gt.G; it.y = d.y; it.M = L.M;
-            it.counts = d.count[0] | (d.count[1] << 9) | (d.count[2] << 18);
-            items.push_back(it);
-            cost.push_back(slim::item_cost(th < tpi ? th : tpi, gt));
+            for (int part = 0; part < sp; ++part) {
+                const int p0 = gt.G * part / sp, p1 = gt.G * (part + 1) / sp;
+                slim::SetItem it;
+                memset(&it, 0, sizeof it);
+                it.layer = l; it.rb = rb; it.N = L.N; it.range = p0 | (p1 << 16); it.M = L.M;
+                it.counts = d.count[0] | (d.count[1] << 9) | (d.count[2] << 18);
+                if (sp > 1) {      // its fp32 partial output [M][N], as a workspace offset
+                    it.y = reinterpret_cast<__half*>(part_off[l] + static_cast<size_t>(part) * L.M * L.N * sizeof(float));
+                    it.counts |= slim::kItemPartial;
+                } else {
+                    it.y = d.y;
+                }
+                items.push_back(it);
+                cost.push_back(slim::item_cost(th < tpi ? th : tpi, gt, d.order, p0, p1));
+            }
         }
         task += (sg.mpad == 2 ? 1 : sg.mpad) * gt.G;
     }
@@ -910,6 +987,7 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
     info->max_bits = sg.bmax;
     info->max_tokens = sg.mmax;
     info->tiles_per_warp = sg.tpw;
+    info->split = sg.split;
     info->plan_bytes = slim::set_plan_bytes(n_layers, n_items);
     info->workspace_bytes = sg.ws_bytes;
     } catch (const std::exception&) {
@@ -935,7 +1013,8 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
         info->n_slots > slim::kSetMaxSlots || info->slot_bytes < 128 || info->slot_bytes % 128 != 0 ||
         (info->token_tiles != 1 && info->token_tiles != 2) || info->max_tokens < 1 || info->max_tokens > 8 * info->token_tiles ||
         info->tiles_per_warp != (info->max_tokens <= 8 ? 2 : 1) ||
-        info->max_bits < 1 || info->max_bits > 4 || info->stage_tasks < 1)
+        info->max_bits < 1 || info->max_bits > 4 || info->stage_tasks < 1 || info->split < 1 || info->split > slim::kSetMaxSplit ||
+        info->n_layers > 65535)
         return SLIM_ERR_INVALID_ARG;
     const size_t smem = slim::kSetOffRing + static_cast<size_t>(info->n_slots) * info->slot_bytes;
     if (smem > 224 * 1024) return SLIM_ERR_INVALID_ARG;
@@ -964,6 +1043,10 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
                         : info->token_tiles == 1 ? slim::launch_set<1, false, 2>(prm, info->grid, smem, s)
                                                  : slim::launch_set<2, false, 1>(prm, info->grid, smem, s);
     SLIM_CUDA_TRY(e);
+    if (info->split > 1) {
+        slim::gemv_set_finish_kernel<<<dim3(32, static_cast<unsigned>(info->n_layers)), 256, 0, s>>>(prm.layers, prm.ws);
+        SLIM_CUDA_TRY(cudaGetLastError());
+    }
     return SLIM_OK;
 }
 
