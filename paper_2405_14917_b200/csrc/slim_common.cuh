@@ -26,6 +26,12 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // Scratch bytes slim_mpq_gemm wants for (M, N) on the current device (256 when it needs none).
 size_t gemm_workspace_bytes(int M, int N, int G);
 
+// slim_mpq_gemv sends large layers through the layer-set kernels: workspace bytes that takes (0: this shape stays on the
+// per-layer kernel), and the call itself (SLIM_OK, a negative status, or 1 if not taken).
+size_t gemv_route_workspace_bytes(int M, int N, int K, int g, const uint8_t* bits_host, const GroupTable& gt);
+int gemv_route(const void* x, const void* packed, const uint8_t* bits_host, const GroupTable& gt, const void* scales, const void* zeros,
+               void* y, int M, int N, int K, int g, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+
 // Validates shape arguments and fills the table.  Returns SLIM_OK or an error status.
 int make_group_table(int N, int K, int g, const uint8_t* bits_host, GroupTable* out);
 

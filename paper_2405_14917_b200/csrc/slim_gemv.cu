@@ -512,6 +512,10 @@ int slim_workspace_bytes(int M, int N, int K, int g, const uint8_t* bits_host, s
     if (M > SLIM_GEMV_MAX_M && N > 0) *out_bytes = slim::gemm_workspace_bytes(M, N, gt.G);
     else if (M >= slim::kPreStageMinM && N > 0 && K > 0) *out_bytes = slim::prestage_bytes(M, gt);
     else *out_bytes = slim::kWsHeader;
+    if (M >= 1 && M <= SLIM_GEMV_MAX_M && N > 0 && K > 0) {       // large layers go through the layer-set kernels
+        const size_t routed = slim::gemv_route_workspace_bytes(M, N, K, g, bits_host, gt);
+        if (routed > *out_bytes) *out_bytes = routed;
+    }
     return SLIM_OK;
 }
 
@@ -569,6 +573,12 @@ int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host, c
     if (workspace == nullptr || workspace_bytes < slim::kWsHeader) return SLIM_ERR_WORKSPACE;
     if (!slim::aligned16(workspace)) return SLIM_ERR_ALIGNMENT;
 
+    // A layer large enough to feed the persistent ring on its own goes through the layer-set kernels, if the workspace
+    // has room for their plan and staged activations (slim_workspace_bytes asks for it).
+    {
+        const int routed = slim::gemv_route(x, packed, bits_host, gt, scales, zeros, y, M, N, K, g, workspace, workspace_bytes, s);
+        if (routed <= 0) return routed;
+    }
     // From kPreStageMinM tokens on, a small kernel puts x into fragment order once, in the
     // workspace; with a workspace too small for that every CTA stages its own part of x.
     const bool pre = M >= slim::kPreStageMinM && workspace_bytes >= slim::prestage_bytes(M, gt);

@@ -694,6 +694,30 @@ __global__ void __launch_bounds__(256) gemv_set_finish_kernel(const SetLayer* __
     }
 }
 
+// ------------------------------------------------------------------------------------------ one-layer sets planned on the device
+// Plan of a one-layer set, written by a kernel: the descriptor comes by value and the items are (row block, part) pairs
+// dealt to the CTAs in turn, so no host memory is read after the call has returned and the call can be captured in a
+// CUDA graph (slim_mpq_gemv sends its large layers this way).
+__global__ void __launch_bounds__(256) set_single_plan_kernel(const __grid_constant__ SetLayer d, uint8_t* plan, int grid, int n_rb, int sp) {
+    int* item_begin = reinterpret_cast<int*>(plan);
+    SetLayer* dl = reinterpret_cast<SetLayer*>(plan + kSetPlanHeader);
+    SetItem* items = reinterpret_cast<SetItem*>(dl + 1);
+    const int n = n_rb * sp, q = n / grid, r = n % grid;
+    for (int c = threadIdx.x; c <= grid; c += blockDim.x) item_begin[c] = c * q + min(c, r);
+    const uint4* src = reinterpret_cast<const uint4*>(&d);
+    for (int i = threadIdx.x; i < static_cast<int>(sizeof(SetLayer) / 16); i += blockDim.x) reinterpret_cast<uint4*>(dl)[i] = src[i];
+    for (int k = threadIdx.x; k < n; k += blockDim.x) {
+        const int c = k % grid, t = k / grid;                // CTA c takes items c, c + grid, ...
+        const int rb = k / sp, part = k - rb * sp;
+        const int p0 = d.G * part / sp, p1 = d.G * (part + 1) / sp;
+        SetItem it;
+        it.layer = 0; it.rb = rb; it.N = d.N; it.range = p0 | (p1 << 16); it.M = d.M;
+        it.counts = d.count[0] | (d.count[1] << 9) | (d.count[2] << 18) | (sp > 1 ? kItemPartial : 0);
+        it.y = sp > 1 ? reinterpret_cast<__half*>(d.part_off + static_cast<size_t>(part) * d.M * d.N * sizeof(float)) : d.y;
+        items[c * q + min(c, r) + t] = it;
+    }
+}
+
 // ------------------------------------------------------------------------------------------ self-test of the bounded wait
 // One warp waits, with the bounded wait of the persistent kernel, on an mbarrier that nobody arrives on.  When the
 // limit has passed it raises the abort flag and the kernel reports through the workspace status word exactly as
@@ -785,9 +809,20 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     // own, fp32 partial outputs in the workspace, summed in part order by a small kernel afterwards).
     const long long want = static_cast<long long>(set_sm_count()) * kSetCtasPerSm;
     sg->split = 1;
-    if (sg->n_items < want) {
-        long long sp = (want + sg->n_items - 1) / sg->n_items;
-        sg->split = static_cast<int>(sp < kSetMaxSplit ? sp : kSetMaxSplit);
+    if (sg->n_items < 2 * want) {
+        // the number of parts that fills the last wave of CTAs best (the smallest one within 2 % of the best)
+        auto items_at = [&](int split) {
+            long long n = 0;
+            for (int l = 0; l < n_layers; ++l)
+                n += static_cast<long long>(layer_split(split, layers[l].K / SLIM_GROUP)) * (((layers[l].N >> 4) + tpi - 1) / tpi);
+            return n;
+        };
+        auto fill = [&](long long n) { return static_cast<double>(n) / static_cast<double>((n + want - 1) / want * want); };
+        double best = fill(sg->n_items);
+        for (int split = 2; split <= kSetMaxSplit; ++split) {
+            const double f = fill(items_at(split));
+            if (f > best * 1.02) { best = f; sg->split = split; }
+        }
     }
     if (sg->split > 1) {
         sg->n_items = 0;
@@ -818,6 +853,33 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     return SLIM_OK;
 }
 
+// Device-side descriptor of one layer.
+static void fill_descriptor(const slim_layer& L, const GroupTable& gt, int mpad, int task0, size_t x_off, int split, size_t part_off,
+                            SetLayer* out) {
+    SetLayer& d = *out;
+    memset(&d, 0, sizeof d);
+    d.x = static_cast<const __half*>(L.x);
+    d.packed = static_cast<const uint8_t*>(L.packed);
+    d.scales = static_cast<const __half*>(L.scales);
+    d.zeros = static_cast<const __half*>(L.zeros);
+    d.y = static_cast<__half*>(L.y);
+    d.M = L.M; d.N = L.N; d.K = L.K; d.G = gt.G;
+    d.MP = mpad;
+    d.task0 = task0;
+    d.x_off = x_off;
+    d.split = static_cast<uint8_t>(split);
+    d.part_off = part_off;
+    memcpy(d.prefix, gt.prefix, sizeof d.prefix);
+    memcpy(d.bits, gt.bits, sizeof d.bits);
+    d.pre3[0] = 0;
+    for (int j = 0; j < SLIM_MAX_GROUPS; ++j)
+        d.pre3[j + 1] = static_cast<uint16_t>(d.pre3[j] + (j < gt.G && gt.bits[j] == 3 ? 1 : 0));
+    int n_sorted = 0;                       // streaming order: by bit-width, then by index
+    for (int b = 1; b <= 4; ++b)
+        for (int j = 0; j < gt.G; ++j)
+            if (gt.bits[j] == b) { d.order[n_sorted++] = static_cast<uint8_t>(j); ++d.count[b - 1]; }
+}
+
 static size_t set_plan_bytes(int n_layers, long long n_items) {
     return kSetPlanHeader + static_cast<size_t>(n_layers) * sizeof(SetLayer) + static_cast<size_t>(n_items) * sizeof(SetItem);
 }
@@ -835,6 +897,83 @@ static cudaError_t launch_set(const SetParams& prm, int grid, size_t smem, cudaS
     }
     gemv_set_kernel<NT, ONE, TPW><<<grid, kSetThreads, smem, stream>>>(prm);
     return cudaGetLastError();
+}
+
+}  // namespace slim
+
+namespace slim {
+
+// ------------------------------------------------------------------------------------------ large single layers through the ring
+// A layer of kRouteMinBytes or more is enough work for the persistent kernel on its own (its row blocks cut into parts
+// when they are fewer than the CTAs), and a launch per layer of the cluster kernel reaches a third of that rate on it.
+constexpr size_t kRouteMinBytes = 32u << 20;
+
+struct RouteLayout {
+    SetGeometry sg;
+    int n_rb, sp;
+    size_t plan_off, plan_bytes, x_off, part_off, total;
+};
+
+static bool route_layout(int M, int N, int K, int g, const uint8_t* bits_host, const GroupTable& gt, RouteLayout* r) {
+    if (M < 1 || N <= 0 || static_cast<size_t>(16) * N * gt.prefix[gt.G] < kRouteMinBytes) return false;
+    slim_layer L;
+    memset(&L, 0, sizeof L);
+    L.bits_host = bits_host; L.M = M; L.N = N; L.K = K;
+    if (set_geometry(&L, 1, g, &r->sg) != SLIM_OK) return false;
+    const int tpi = kSetConsumers * r->sg.tpw;
+    r->n_rb = ((N >> 4) + tpi - 1) / tpi;
+    r->sp = layer_split(r->sg.split, gt.G);
+    r->plan_off = 256;
+    r->plan_bytes = set_plan_bytes(1, static_cast<long long>(r->n_rb) * r->sp);
+    r->x_off = r->plan_off + align_to(r->plan_bytes, 256);
+    r->part_off = r->x_off + layer_ws_bytes(r->sg.mpad, gt);
+    r->total = r->part_off + (r->sp > 1 ? align_to(static_cast<size_t>(r->sp) * M * N * sizeof(float), 128) : 0);
+    return true;
+}
+
+size_t gemv_route_workspace_bytes(int M, int N, int K, int g, const uint8_t* bits_host, const GroupTable& gt) {
+    RouteLayout r;
+    return route_layout(M, N, K, g, bits_host, gt, &r) ? r.total : 0;
+}
+
+}  // namespace slim
+
+extern "C" int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* workspace, size_t workspace_bytes, void* stream);
+
+namespace slim {
+
+// Returns SLIM_OK after enqueueing the layer through the layer-set kernels, a negative status on failure, or 1 if this
+// shape or workspace is not routed (the caller then takes the per-layer kernel).
+int gemv_route(const void* x, const void* packed, const uint8_t* bits_host, const GroupTable& gt, const void* scales, const void* zeros,
+               void* y, int M, int N, int K, int g, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+    RouteLayout r;
+    if (!route_layout(M, N, K, g, bits_host, gt, &r) || workspace_bytes < r.total) return 1;
+    slim_layer L;
+    memset(&L, 0, sizeof L);
+    L.x = x; L.packed = packed; L.scales = scales; L.zeros = zeros; L.y = y; L.bits_host = bits_host; L.M = M; L.N = N; L.K = K;
+    SetLayer d;
+    fill_descriptor(L, gt, r.sg.mpad, 0, r.x_off, r.sp, r.part_off, &d);
+    uint8_t* plan = static_cast<uint8_t*>(workspace) + r.plan_off;
+    const long long n_items = static_cast<long long>(r.n_rb) * r.sp;
+    const int grid = static_cast<int>(n_items < r.sg.grid ? n_items : r.sg.grid);
+    set_single_plan_kernel<<<1, 256, 0, stream>>>(d, plan, grid, r.n_rb, r.sp);
+    SLIM_CUDA_TRY(cudaGetLastError());
+    slim_gemv_set_info info;
+    memset(&info, 0, sizeof info);
+    info.n_layers = 1;
+    info.grid = grid;
+    info.n_slots = r.sg.n_slots;
+    info.slot_bytes = r.sg.slot_bytes;
+    info.token_tiles = r.sg.nt;
+    info.stage_tasks = (r.sg.mpad == 2 ? 1 : r.sg.mpad) * gt.G;
+    info.n_items = static_cast<int>(n_items);
+    info.max_bits = r.sg.bmax;
+    info.max_tokens = r.sg.mmax;
+    info.tiles_per_warp = r.sg.tpw;
+    info.split = r.sg.split;
+    info.plan_bytes = r.plan_bytes;
+    info.workspace_bytes = r.total;
+    return slim_mpq_gemv_set(&info, plan, workspace, workspace_bytes, stream);
 }
 
 }  // namespace slim
@@ -902,29 +1041,9 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
         slim::GroupTable gt;
         slim::make_group_table(L.N, L.K, g, L.bits_host, &gt);
         slim::SetLayer d;
-        memset(&d, 0, sizeof d);
-        d.x = static_cast<const __half*>(L.x);
-        d.packed = static_cast<const uint8_t*>(L.packed);
-        d.scales = static_cast<const __half*>(L.scales);
-        d.zeros = static_cast<const __half*>(L.zeros);
-        d.y = static_cast<__half*>(L.y);
-        d.M = L.M; d.N = L.N; d.K = L.K; d.G = gt.G;
-        d.MP = sg.mpad;
-        d.task0 = task;
-        d.x_off = ws_off;
-        ws_off += slim::layer_ws_bytes(sg.mpad, gt);
         const int sp = slim::layer_split(sg.split, gt.G);
-        d.split = static_cast<uint8_t>(sp);
-        d.part_off = part_off[l];
-        memcpy(d.prefix, gt.prefix, sizeof d.prefix);
-        memcpy(d.bits, gt.bits, sizeof d.bits);
-        d.pre3[0] = 0;
-        for (int j = 0; j < SLIM_MAX_GROUPS; ++j)
-            d.pre3[j + 1] = static_cast<uint16_t>(d.pre3[j] + (j < gt.G && gt.bits[j] == 3 ? 1 : 0));
-        int n_sorted = 0;                       // streaming order: by bit-width, then by index
-        for (int b = 1; b <= 4; ++b)
-            for (int j = 0; j < gt.G; ++j)
-                if (gt.bits[j] == b) { d.order[n_sorted++] = static_cast<uint8_t>(j); ++d.count[b - 1]; }
+        slim::fill_descriptor(L, gt, sg.mpad, task, ws_off, sp, part_off[l], &d);
+        ws_off += slim::layer_ws_bytes(sg.mpad, gt);
         SLIM_CUDA_TRY(cudaMemcpyAsync(plan_dev + slim::kSetPlanHeader + static_cast<size_t>(l) * sizeof d, &d, sizeof d,
                                       cudaMemcpyHostToDevice, s));
         const int n_rb = ((L.N >> 4) + tpi - 1) / tpi;

@@ -72,6 +72,46 @@ def test_llama70b_shapes_single_layer_entry_point(N, K, M):
     check_output(y[:, rows], orc.linear_rows_f64(x, L["codes"], L["scales"], L["zeros"], rows), f"gemv {N}x{K} M={M}")
 
 
+@pytest.mark.parametrize("M", [1, 4])
+def test_large_layer_takes_the_ring_or_the_per_layer_kernel_by_workspace_size(M):
+    """slim_mpq_gemv sends a layer of 32 MB or more through the layer-set kernels when the workspace has room for their
+    plan (written by a kernel, so the call can sit in a CUDA graph) and staged activations; with a 256-byte workspace
+    the same call takes the per-layer kernel.  Both against the oracle, the routed one also replayed from a graph."""
+    slim = _slim()
+    N, K = 28672, 8192
+    L, dl = _layer(N, K, 2), _device_layer(N, K, 2)
+    rng = np.random.default_rng(2800 + M)
+    x = _x(rng, M, K)
+    xd = torch.from_numpy(x).cuda()
+    rows = _sample_rows(N, rng)
+    y_ref = orc.linear_rows_f64(x, L["codes"], L["scales"], L["zeros"], rows)
+    big = slim.new_workspace(M, N, K, L["bits"])
+    assert big.numel() > 1 << 16                          # room for the plan, the staged x and the partial outputs
+    small = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    for ws, what in ((big, "through the ring"), (small, "per-layer kernel")):
+        y = slim.mpq_gemv(xd, dl.packed, L["bits"], dl.scales, dl.zeros, N, ws)
+        slim.workspace_status(ws)
+        check_output(y.cpu().numpy()[:, rows], y_ref, f"{what}, M={M}")
+    out = torch.empty((M, N), dtype=torch.float16, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        slim.mpq_gemv(xd, dl.packed, L["bits"], dl.scales, dl.zeros, N, big, out)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        slim.mpq_gemv(xd, dl.packed, L["bits"], dl.scales, dl.zeros, N, big, out)
+    first = out.clone()
+    for _ in range(3):
+        out.fill_(float("nan"))
+        graph.replay()
+    torch.cuda.synchronize()
+    slim.workspace_status(big)
+    assert torch.equal(out, first)
+    check_output(out.cpu().numpy()[:, rows], y_ref, f"replayed from a graph, M={M}")
+
+
 @pytest.mark.parametrize("M", [1, 16])
 def test_llama70b_block_as_one_layer_set(M):
     """All seven projections of a LLaMA-2-70B block in one layer-set launch (the benchmark's 70B configuration
