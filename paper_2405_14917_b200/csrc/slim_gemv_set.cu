@@ -195,30 +195,30 @@ __device__ __forceinline__ void stage_group_i8(const __half* xg, uint8_t* rec, i
     Xs[4 * lane + 2] = __float2int_rn(f23.x * up);
     Xs[4 * lane + 3] = __float2int_rn(f23.y * up);
     __syncwarp();
+    // lane = (MMA mi, lane column c, register half h): the four k-slots (bytes bb) of that B register, all four digits
+    const int mi = lane >> 3, c = (lane >> 1) & 3, h = lane & 1;
     for (int sl = 0; sl < slice_count(b); ++sl) {
         const int w = slice_w(b, sl), lo = slice_lo(b, sl);
-        for (int idx = lane; idx < 64; idx += 32) {
-            const int mi = idx >> 4, n = (idx >> 2) & 3, c = idx & 3;
-            uint32_t word[2];
-            for (int h = 0; h < 2; ++h) {
-                uint32_t v4 = 0;
-                // The MMA of a byte's top field position takes the packed word as it is, i.e. every field of the byte
-                // times that position's digit; the other positions subtract it again.
-                const int mi_top = w == 4 ? (mi | 1) : 3, h_top = w == 1 ? 1 : h;
-                const int pos = i8_pos(w, mi, h), pos_top = i8_pos(w, mi_top, h_top);
-                for (int bb = 0; bb < 4; ++bb) {
-                    int V = Xs[i8_column(w, mi, h, bb, c)] << (lo + pc - w * pos);
-                    if (mi != mi_top || h != h_top) V -= Xs[i8_column(w, mi_top, h_top, bb, c)] << (lo + pc - w * pos_top);
-                    const int d0 = static_cast<int8_t>(V & 0xff), V1 = (V - d0) >> 8;      // |V| < 2^30
-                    const int d1 = static_cast<int8_t>(V1 & 0xff), V2 = (V1 - d1) >> 8;
-                    const int d2 = static_cast<int8_t>(V2 & 0xff), d3 = (V2 - d2) >> 8;    // |d3| <= 64
-                    const int dig = n == 0 ? d3 : (n == 1 ? d2 : (n == 2 ? d1 : d0));
-                    v4 |= static_cast<uint32_t>(dig & 0xff) << (8 * bb);
-                }
-                word[h] = v4;
-            }
-            *reinterpret_cast<uint2*>(rec + 128 + sl * 512 + mi * 128 + (n * 4 + c) * 8) = make_uint2(word[0], word[1]);
+        // The MMA of a byte's top field position takes the packed word as it is, i.e. every field of the byte times
+        // that position's digit; the other positions subtract it again.
+        const int mi_top = w == 4 ? (mi | 1) : 3, h_top = w == 1 ? 1 : h;
+        const int sh = lo + pc - w * i8_pos(w, mi, h), sh_top = lo + pc - w * i8_pos(w, mi_top, h_top);
+        const bool is_top = mi == mi_top && h == h_top;
+        uint32_t word[4] = {0u, 0u, 0u, 0u};               // digits 3 (highest) .. 0 of the four k-slots
+        for (int bb = 0; bb < 4; ++bb) {
+            int V = Xs[i8_column(w, mi, h, bb, c)] << sh;
+            if (!is_top) V -= Xs[i8_column(w, mi_top, h_top, bb, c)] << sh_top;
+            const int d0 = static_cast<int8_t>(V & 0xff), V1 = (V - d0) >> 8;      // |V| < 2^30 + 2^24
+            const int d1 = static_cast<int8_t>(V1 & 0xff), V2 = (V1 - d1) >> 8;
+            const int d2 = static_cast<int8_t>(V2 & 0xff), d3 = (V2 - d2) >> 8;    // |d3| <= 65
+            word[0] |= static_cast<uint32_t>(d3 & 0xff) << (8 * bb);
+            word[1] |= static_cast<uint32_t>(d2 & 0xff) << (8 * bb);
+            word[2] |= static_cast<uint32_t>(d1 & 0xff) << (8 * bb);
+            word[3] |= static_cast<uint32_t>(d0 & 0xff) << (8 * bb);
         }
+#pragma unroll
+        for (int n = 0; n < 4; ++n)
+            *reinterpret_cast<uint32_t*>(rec + 128 + sl * 512 + mi * 128 + (n * 4 + c) * 8 + 4 * h) = word[n];
     }
     if (lane == 0) *reinterpret_cast<float2*>(rec) = make_float2(sum, __int_as_float((127 - S - pc) << 23));
 }
