@@ -21,6 +21,11 @@
  *   none synchronises unless it says so, and all work is enqueued on `stream` (a cudaStream_t
  *   passed as void*; NULL is the legacy default stream).  Calls never throw; they return a status.
  *
+ * Threads: the entry points may be called from several host threads.  The per-device set-up that the first launch of a
+ * kernel performs (a function attribute, a device query) is idempotent and published through atomics, so two threads
+ * that make their first calls together repeat it harmlessly.  Calls that share a workspace, or the built-in scratch
+ * of slim_mpq_gemm_static, must still be ordered on one stream.
+ *
  * Limits: g must be 128; K a multiple of 128 with at most 256 groups; N a multiple of 16;
  * N = 0 or M = 0 is a successful no-op.  Anything else returns an error status and enqueues nothing.
  *
@@ -90,7 +95,9 @@ int slim_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
 /* Synchronises `stream`, reads and clears the workspace status word.  Returns SLIM_OK, or
  * SLIM_ERR_TIMEOUT if a kernel using this workspace abandoned a bounded wait (its output is
- * then undefined), or SLIM_ERR_CUDA. */
+ * then undefined), or SLIM_ERR_CUDA.  A kernel that gave up may have left its flags and partial sums
+ * behind: after SLIM_ERR_TIMEOUT pass the workspace through slim_workspace_init before the next call
+ * that uses more than its status word (slim_mpq_gemm on a shape it cuts across CTAs). */
 int slim_workspace_status(void* workspace, void* stream);
 
 /* Self-test of the device-side time-out path.  (No counterpart in the paper: it exercises the status-word
@@ -116,8 +123,16 @@ int slim_dequant(const void* packed, const uint8_t* bits_host, const void* scale
 /* Decode path, 1 <= M <= 16:  y = x * W-hat^T, fp32 accumulation, fp16 output (the paper's
  * inference kernel, App. B.2: group-by-group dequantisation and dot product with the shared
  * activation).  Streams the packed slices once; HBM-bound.  Results are deterministic for a
- * given (shape, device).  x with Inf/NaN gives unspecified y.  `workspace` must be at least 256
- * bytes (the kernel itself keeps its partial sums in shared memory). */
+ * given (shape, device, workspace size).  x with Inf/NaN gives unspecified y.  `workspace` must be at least
+ * 256 bytes (the kernel itself keeps its partial sums in shared memory).
+ * A layer whose packed codes take 32 MB or more is run by the kernels of slim_mpq_gemv_set instead (same result
+ * within the rounding of the accumulation order; at M = 1 with the fixed-point x described there) when the
+ * workspace has the slim_workspace_bytes() that shape asks for; with a smaller workspace it takes the per-layer
+ * kernel.  The call reads no host memory after it returns and can be captured in a CUDA graph either way.
+ * The per-layer kernel is launched with programmatic stream serialisation and fetches packed, scales and zeros
+ * before it waits for the kernel ahead of it on the stream: those three buffers must be complete when the call is
+ * enqueued, or be written by a kernel that does not signal programmatic launch completion early (x and y may be
+ * produced and consumed by the neighbouring kernels as usual). */
 int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host,
                   const void* scales, const void* zeros, void* y,
                   int M, int N, int K, int g,
@@ -153,10 +168,13 @@ int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* bits_host,
  * then runs; two calls whose kernels can overlap on the GPU (different streams, no ordering) race
  * on it and give undefined results, so keep the calls of a device on one stream or order them.
  * The first call on each device looks up the array's device address (a driver query, no
- * allocation); make that first call outside any stream capture.
+ * allocation); make that first call outside any stream capture.  The array is reserved when the
+ * library's device code is loaded on a GPU, which with lazy module loading is the first use of the
+ * library there: make one call (of any entry point) at start-up, before memory gets tight.
  *
  * status_out: optional device pointer to one 32-bit word (4-byte aligned, may be NULL).  After
- * the call's work completes it holds 0, or 1 if a device-side wait gave up (y is then undefined);
+ * the work of a successful call completes (the no-op shapes included) it holds 0, or 1 if a
+ * device-side wait gave up (y is then undefined);
  * it plays the part slim_workspace_status plays for a caller-owned workspace. */
 #define SLIM_STATIC_SCRATCH_MAX (1280 + 148 * 256 * 128 * 4)
 int slim_mpq_gemm_static(const void* x, const void* packed, const uint8_t* bits_host,
@@ -173,7 +191,9 @@ int slim_mpq_gemm_static(const void* x, const void* packed, const uint8_t* bits_
  * may read what another layer of the same set writes.
  *
  * Every layer gets the y = x * W-hat^T of slim_mpq_gemv (same products, fp32 accumulation in a
- * different order, fp16 output); the results are deterministic for a given (set, device).
+ * different order: the groups of a layer are added sorted by bit-width, and a set with fewer row blocks
+ * than persistent CTAs adds them in up to 8 parts; fp16 output); the results are deterministic for a
+ * given (set, device).
  * A set in which EVERY layer has M = 1 runs on integer tensor-core instructions: per group of 128
  * columns x is first rounded to fixed point with 22 bits relative to the group's largest |x_k|, so an
  * fp16 activation within a factor 2^11 of that maximum is taken exactly and a smaller one with an error
