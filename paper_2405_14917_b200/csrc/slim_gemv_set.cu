@@ -431,6 +431,162 @@ __device__ __forceinline__ void consume_one(const SetParams& p, const uint32_t s
     }
 }
 
+
+// Consumer warp of a set with more than one token somewhere: f16 MMAs on raw code fields (one AND per operand
+// register of two codes, see slim_gemv_dev.cuh), NT tiles of 8 tokens, then the fold
+// acc += s (D 2^(24-S) - z sum_x) per (row, token, group).  Same loop structure as consume_one.
+template <int NT, int TPW>
+__device__ __forceinline__ void consume_f16(const SetParams& p, const uint32_t sbase, const uint32_t ring, volatile int* abort,
+                                            const int i0, const int i1, const int warp, const int lane) {
+    auto full = [&](int s) { return sbase + 8u * s; };
+    auto empty = [&](int s) { return sbase + 8u * (kSetMaxSlots + s); };
+    constexpr int TPI = kSetConsumers * TPW, MPK = 8 * NT;
+    constexpr int CH = NT == 1 ? (TPW == 1 ? 4 : 2) : 2;     // interleaved accumulation chains
+    constexpr uint32_t kOffZ = slot_off_z(TPI), kOffE = slot_off_e(TPI), kOffX = slot_off_x(TPI), kOffW = slot_off_w(TPI, MPK);
+    const int gq = lane >> 2, c = lane & 3;
+    const uint32_t lane0 = lane == 0 ? 1u : 0u;
+    const uint32_t slot_bytes = static_cast<uint32_t>(p.slot_bytes);
+    const int n_slots = p.n_slots;
+    const uint32_t sz_lane = static_cast<uint32_t>(TPW * warp * 32 + gq * 4);
+    const uint32_t x_lane = kOffX + (gq * 4 + c) * 8;             // fragment of token gq of the first token tile
+    const uint32_t e_lane = kOffE + 16u * c;                      // (sum_x, scale) of tokens 2c, 2c + 1
+    const uint32_t w_lane = kOffW + 8u * lane;
+    int s = 0;
+    uint32_t ph = 0;
+    bool ok = true;
+    const int4* items4 = reinterpret_cast<const int4*>(p.items);
+    int4 it_a = items4[2 * i0], it_b = items4[2 * i0 + 1];       // (layer, rb, N, range), (y, M, counts)
+    for (int i = i0; i < i1 && ok; ++i) {
+        const int rb = it_a.y, N = it_a.z, p0 = it_a.w & 0xffff, p1 = it_a.w >> 16, M = it_b.z, counts = it_b.w;
+        const unsigned long long yword = (static_cast<unsigned long long>(static_cast<uint32_t>(it_b.y)) << 32) | static_cast<uint32_t>(it_b.x);
+        if (i + 1 < i1) {                                        // the next item arrives during this one's groups
+            it_a = items4[2 * i + 2];
+            it_b = items4[2 * i + 3];
+        }
+        const int tile0 = TPI * rb + TPW * warp;                 // this warp's first tile of the layer
+        const int n_act = min(TPW, (N >> 4) - tile0);            // its tiles that exist (<= 0: none)
+        if (n_act <= 0) {
+            for (int j = p0; j < p1; ++j) {                      // only hands the slots back
+                if (!__all_sync(0xffffffffu, sb::try_wait(full(s), ph)) && !wait_full_slow(full(s), ph, abort)) { ok = false; break; }
+                __syncwarp();
+                sb::arrive_if(empty(s), lane0);
+                if (++s == n_slots) { s = 0; ph ^= 1u; }
+            }
+            continue;
+        }
+        float acc[TPW][NT][4];
+#pragma unroll
+        for (int t = 0; t < TPW; ++t)
+#pragma unroll
+            for (int n = 0; n < NT; ++n)
+#pragma unroll
+                for (int r = 0; r < 4; ++r) acc[t][n][r] = 0.f;
+
+        auto run_groups = [&](auto btag, int n_groups) -> bool {
+            constexpr int B = decltype(btag)::value;
+            for (int k = 0; k < n_groups; ++k) {
+                if (!__all_sync(0xffffffffu, sb::try_wait(full(s), ph)) && !wait_full_slow(full(s), ph, abort)) return false;
+                const uint32_t slot = ring + static_cast<uint32_t>(s) * slot_bytes;
+                // tile t of the warp: its slices follow each other.  For a tile past the end of the layer the slot holds
+                // stale bytes: its accumulators are computed and never stored.
+                const uint32_t item0 = slot + w_lane + static_cast<uint32_t>(TPW * warp) * (256u * B);
+                float d[TPW][CH][NT][4];      // every chain is started by an MMA with a zero accumulator
+                // one slice of width WD starting at unit `unit0`, activations in fragment slot `xs`
+                auto run_slice = [&](auto wtag, auto first_tag, int unit0, uint32_t xs) {
+                    constexpr int WD = decltype(wtag)::value;
+                    constexpr int MPU = 8 / WD;                 // MMAs per unit
+                    constexpr bool FIRST = decltype(first_tag)::value != 0;   // the group's first slice
+#pragma unroll
+                    for (int u = 0; u < WD; ++u) {
+                        uint2 wd[TPW];
+                        uint32_t shx[TPW], shy[TPW];
+#pragma unroll
+                        for (int t = 0; t < TPW; ++t) {
+                            wd[t] = lds64(item0 + t * (256u * B) + 256u * (unit0 + u));
+                            shx[t] = wd[t].x >> pair_shift(WD);
+                            shy[t] = wd[t].y >> pair_shift(WD);
+                        }
+#pragma unroll
+                        for (int ii = 0; ii < MPU; ++ii) {
+                            const int mi = u * MPU + ii;
+#pragma unroll
+                            for (int n = 0; n < NT; ++n) {
+                                // fragment of token 8n + gq (tokens the layer lacks are staged as zeros)
+                                const uint2 bv = lds64(xs + ((mi * MPK + 8 * n) * 4) * 8);
+#pragma unroll
+                                for (int t = 0; t < TPW; ++t) {
+                                    const uint32_t a0 = pair<WD>(wd[t].x, shx[t], 2 * ii), a1 = pair<WD>(wd[t].y, shy[t], 2 * ii);
+                                    const uint32_t a2 = pair<WD>(wd[t].x, shx[t], 2 * ii + 1), a3 = pair<WD>(wd[t].y, shy[t], 2 * ii + 1);
+                                    if (FIRST && mi < CH) mma_f16_first(d[t][mi & (CH - 1)][n], a0, a1, a2, a3, bv);
+                                    else mma_f16(d[t][mi & (CH - 1)][n], a0, a1, a2, a3, bv);
+                                }
+                            }
+                        }
+                    }
+                };
+                const uint32_t xs0 = slot + x_lane;
+                if (B == 1) run_slice(W1{}, WidthTag<1>{}, 0, xs0);
+                if (B == 2) run_slice(W2{}, WidthTag<1>{}, 0, xs0);
+                if (B == 3) { run_slice(W2{}, WidthTag<1>{}, 0, xs0); run_slice(W1{}, WidthTag<0>{}, 2, xs0 + 8 * MPK * 32); }
+                if (B == 4) run_slice(W4{}, WidthTag<1>{}, 0, xs0);
+                // fold the group: rows 2gq, 2gq+1, tokens 8n+2c, 8n+2c+1
+#pragma unroll
+                for (int t = 0; t < TPW; ++t) {
+                    const uint32_t s2 = lds32(slot + kSlotOffS + sz_lane + t * 32);
+                    const uint32_t z2 = lds32(slot + kOffZ + sz_lane + t * 32);
+                    const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
+                    const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
+#pragma unroll
+                    for (int n = 0; n < NT; ++n) {
+                        const uint4 tkw = lds128(slot + e_lane + 64u * n);       // (sx0, e0, sx1, e1)
+                        const float sx0 = __uint_as_float(tkw.x), e0 = __uint_as_float(tkw.y);
+                        const float sx1 = __uint_as_float(tkw.z), e1 = __uint_as_float(tkw.w);
+                        float dd[4];
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) {
+                            dd[r] = d[t][0][n][r] + d[t][1][n][r];
+                            if (CH == 4) dd[r] += d[t][2 % CH][n][r] + d[t][3 % CH][n][r];
+                        }
+                        acc[t][n][0] = fmaf(sf.x, fmaf(-zf.x, sx0, dd[0] * e0), acc[t][n][0]);
+                        acc[t][n][1] = fmaf(sf.x, fmaf(-zf.x, sx1, dd[1] * e1), acc[t][n][1]);
+                        acc[t][n][2] = fmaf(sf.y, fmaf(-zf.y, sx0, dd[2] * e0), acc[t][n][2]);
+                        acc[t][n][3] = fmaf(sf.y, fmaf(-zf.y, sx1, dd[3] * e1), acc[t][n][3]);
+                    }
+                }
+                __syncwarp();
+                sb::arrive_if(empty(s), lane0);
+                if (++s == n_slots) { s = 0; ph ^= 1u; }
+            }
+            return true;
+        };
+        // the widths start at positions 0, e1, e2, e3 of the layer's streaming order; the item covers [p0, p1)
+        const int e1 = counts & 511, e2 = e1 + ((counts >> 9) & 511), e3 = e2 + ((counts >> 18) & 511);
+        auto part = [&](int a, int b) { return max(min(p1, b) - max(p0, a), 0); };
+        ok = run_groups(WidthTag<1>{}, part(0, e1)) && run_groups(WidthTag<2>{}, part(e1, e2)) &&
+             run_groups(WidthTag<3>{}, part(e2, e3)) && run_groups(WidthTag<4>{}, part(e3, 65535));
+        // ---- this warp's rows of the item: rows 2gq, 2gq+1 of tokens 8n+2c, 8n+2c+1 of every tile
+        if (ok) {
+            const bool partial = (counts & kItemPartial) != 0;
+#pragma unroll
+            for (int t = 0; t < TPW; ++t) {
+                if (t >= n_act) break;
+                const int row = 16 * (tile0 + t) + 2 * gq;
+#pragma unroll
+                for (int n = 0; n < NT; ++n) {
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {                    // tokens 8n + 2c and 8n + 2c + 1
+                        const int m = 8 * n + 2 * c + q;
+                        if (m >= M) continue;
+                        const size_t at = static_cast<size_t>(m) * N + row;
+                        if (partial) *reinterpret_cast<float2*>(reinterpret_cast<float*>(p.ws + yword) + at) = make_float2(acc[t][n][q], acc[t][n][2 + q]);
+                        else *reinterpret_cast<__half2*>(reinterpret_cast<__half*>(yword) + at) = __floats2half2_rn(acc[t][n][q], acc[t][n][2 + q]);
+                    }
+                }
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------ the persistent kernel
 constexpr uint32_t kSetOffAbort = 16 * kSetMaxSlots;          // after the full and empty barriers
 constexpr uint32_t kSetOffDesc = 1024;                        // the producer's copy of its layer's descriptor
@@ -450,7 +606,6 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
     volatile int* abort = reinterpret_cast<volatile int*>(smem + kSetOffAbort);
     const uint32_t ring = sbase + kSetOffRing;
     constexpr int TPI = kSetConsumers * TPW;                  // tiles per item
-    constexpr int MPK = ONE ? 1 : 8 * NT;                     // tokens in the staged layout
     constexpr uint32_t kOffZ = slot_off_z(TPI), kOffE = slot_off_e(TPI), kOffX = slot_off_x(TPI);
     constexpr uint32_t kOffW = slot_off_w(TPI, ONE ? 2 : 8 * NT);
 
@@ -532,141 +687,8 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
             }
         } else {
             // -------------------------------------------------------------- consumer: tile `warp` of every item
-            if constexpr (ONE) {
-                consume_one<TPW>(p, sbase, ring, abort, i0, i1, warp, lane);
-            } else {
-            const int gq = lane >> 2, c = lane & 3;
-            int s = 0;                                    // ring position of the next group
-            uint32_t ph = 0;
-            bool ok = true;
-            const int4* items4 = reinterpret_cast<const int4*>(p.items);
-            int4 it_a = items4[2 * i0], it_b = items4[2 * i0 + 1];   // (layer, rb, N, G), (y, M, -)
-            for (int i = i0; i < i1 && ok; ++i) {
-                const int rb = it_a.y, N = it_a.z, G = (it_a.w >> 16) - (it_a.w & 0xffff), M = it_b.z;
-                const bool partial = (it_b.w & kItemPartial) != 0;
-                const unsigned long long yword = (static_cast<unsigned long long>(static_cast<uint32_t>(it_b.y)) << 32) | static_cast<uint32_t>(it_b.x);
-                if (i + 1 < i1) {                                     // the next item arrives during this one's groups
-                    it_a = items4[2 * i + 2];
-                    it_b = items4[2 * i + 3];
-                }
-                const int tile0 = TPI * rb + TPW * warp;                  // this warp's first tile of the layer
-                const int n_act = min(TPW, (N >> 4) - tile0);              // its tiles that exist (<= 0: none)
-                float acc[TPW][NT][4];
-#pragma unroll
-                for (int t = 0; t < TPW; ++t)
-#pragma unroll
-                    for (int n = 0; n < NT; ++n)
-#pragma unroll
-                        for (int r = 0; r < 4; ++r) acc[t][n][r] = 0.f;
-
-                for (int j = 0; j < G; ++j) {
-                    if (!__all_sync(0xffffffffu, sb::wait(full(s), ph, abort))) { ok = false; break; }
-                    const uint32_t slot = ring + static_cast<uint32_t>(s) * p.slot_bytes;
-                    if (n_act > 0) {
-                        const int b = static_cast<int>(lds32(slot));
-                        // tile t of the warp: its slices follow each other.  For a tile past the end of the
-                        // layer the slot holds stale bytes: its accumulators are computed and never stored.
-                        const uint32_t item0 = slot + kOffW + static_cast<uint32_t>(TPW * warp) * 256u * b;
-                        const uint32_t xs_slot0 = slot + kOffX;
-                        {
-                        constexpr int CH = NT == 1 ? (TPW == 1 ? 4 : 2) : 2;     // interleaved accumulation chains
-                        float d[TPW][CH][NT][4];      // every chain is started by an MMA with a zero accumulator
-
-                        // one slice of width WD starting at unit `unit0`, activations in fragment slot `xs_slot`
-                        auto run_slice = [&](auto wtag, auto first_tag, int unit0, uint32_t xs_slot) {
-                            constexpr int WD = decltype(wtag)::value;
-                            constexpr int MPU = 8 / WD;                 // MMAs per unit
-                            constexpr bool FIRST = decltype(first_tag)::value != 0;   // the group's first slice
-#pragma unroll
-                            for (int u = 0; u < WD; ++u) {
-                                uint2 wd[TPW];
-                                uint32_t shx[TPW], shy[TPW];
-#pragma unroll
-                                for (int t = 0; t < TPW; ++t) {
-                                    const uint32_t item = item0 + t * 256u * b;
-                                    wd[t] = lds64(item + 256 * (unit0 + u) + 8 * lane);
-                                    shx[t] = wd[t].x >> pair_shift(WD);
-                                    shy[t] = wd[t].y >> pair_shift(WD);
-                                }
-#pragma unroll
-                                for (int ii = 0; ii < MPU; ++ii) {
-                                    const int mi = u * MPU + ii;
-#pragma unroll
-                                    for (int n = 0; n < NT; ++n) {
-                                        // fragment of token 8n + gq (tokens the layer lacks are staged as zeros)
-                                        const uint2 bv = lds64(xs_slot + ((mi * MPK + 8 * n + gq) * 4 + c) * 8);
-#pragma unroll
-                                        for (int t = 0; t < TPW; ++t) {
-                                            const uint32_t a0 = pair<WD>(wd[t].x, shx[t], 2 * ii), a1 = pair<WD>(wd[t].y, shy[t], 2 * ii);
-                                            const uint32_t a2 = pair<WD>(wd[t].x, shx[t], 2 * ii + 1), a3 = pair<WD>(wd[t].y, shy[t], 2 * ii + 1);
-                                            if (FIRST && mi < CH) mma_f16_first(d[t][mi & (CH - 1)][n], a0, a1, a2, a3, bv);
-                                            else mma_f16(d[t][mi & (CH - 1)][n], a0, a1, a2, a3, bv);
-                                        }
-                                    }
-                                }
-                            }
-                        };
-                        switch (b) {
-                            case 1: run_slice(W1{}, WidthTag<1>{}, 0, xs_slot0); break;
-                            case 2: run_slice(W2{}, WidthTag<1>{}, 0, xs_slot0); break;
-                            case 3: run_slice(W2{}, WidthTag<1>{}, 0, xs_slot0); run_slice(W1{}, WidthTag<0>{}, 2, xs_slot0 + 8 * MPK * 32); break;
-                            default: run_slice(W4{}, WidthTag<1>{}, 0, xs_slot0); break;
-                        }
-
-                        // fold the group: acc += s * (D * 2^(24-S) - z * sum_x); rows 2gq, 2gq+1, tokens 8n+2c, 8n+2c+1
-                        const float2* sxe = reinterpret_cast<const float2*>(smem + (slot - sbase) + kOffE);
-#pragma unroll
-                        for (int t = 0; t < TPW; ++t) {
-                            const int tt = TPW * warp + t;                             // tile inside the item
-                            const uint32_t s2 = lds32(slot + kSlotOffS + tt * 32 + gq * 4);
-                            const uint32_t z2 = lds32(slot + kOffZ + tt * 32 + gq * 4);
-                            const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
-                            const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&z2));
-                            {
-#pragma unroll
-                                for (int n = 0; n < NT; ++n) {
-                                    const float4 tk = *reinterpret_cast<const float4*>(sxe + 8 * n + 2 * c);   // (sx0, e0, sx1, e1)
-                                    float dd[4];
-#pragma unroll
-                                    for (int r = 0; r < 4; ++r) {
-                                        dd[r] = d[t][0][n][r] + d[t][1][n][r];
-                                        if (CH == 4) dd[r] += d[t][2 % CH][n][r] + d[t][3 % CH][n][r];
-                                    }
-                                    const float d0 = dd[0] * tk.y, d1 = dd[1] * tk.w, d2 = dd[2] * tk.y, d3 = dd[3] * tk.w;
-                                    acc[t][n][0] = fmaf(sf.x, fmaf(-zf.x, tk.x, d0), acc[t][n][0]);
-                                    acc[t][n][1] = fmaf(sf.x, fmaf(-zf.x, tk.z, d1), acc[t][n][1]);
-                                    acc[t][n][2] = fmaf(sf.y, fmaf(-zf.y, tk.x, d2), acc[t][n][2]);
-                                    acc[t][n][3] = fmaf(sf.y, fmaf(-zf.y, tk.z, d3), acc[t][n][3]);
-                                }
-                            }
-                        }
-                        }
-                    }
-                    __syncwarp();
-                    if (lane == 0) sb::arrive(empty(s));
-                    if (++s == p.n_slots) { s = 0; ph ^= 1u; }
-                }
-                // ---- this warp's rows of the item: rows 2gq, 2gq+1 of tokens 8n+2c, 8n+2c+1 of every tile
-                if (ok) {
-#pragma unroll
-                    for (int t = 0; t < TPW; ++t) {
-                        if (t >= n_act) break;
-                        const int row = 16 * (tile0 + t) + 2 * gq;
-#pragma unroll
-                        for (int n = 0; n < NT; ++n) {
-#pragma unroll
-                            for (int q = 0; q < 2; ++q) {                    // tokens 8n + 2c and 8n + 2c + 1
-                                const int m = 8 * n + 2 * c + q;
-                                if (m >= M) continue;
-                                const size_t at = static_cast<size_t>(m) * N + row;
-                                if (partial) *reinterpret_cast<float2*>(reinterpret_cast<float*>(p.ws + yword) + at) = make_float2(acc[t][n][q], acc[t][n][2 + q]);
-                                else *reinterpret_cast<__half2*>(reinterpret_cast<__half*>(yword) + at) = __floats2half2_rn(acc[t][n][q], acc[t][n][2 + q]);
-                            }
-                        }
-                    }
-                }
-            }
-            }
+            if constexpr (ONE) consume_one<TPW>(p, sbase, ring, abort, i0, i1, warp, lane);
+            else consume_f16<NT, TPW>(p, sbase, ring, abort, i0, i1, warp, lane);
         }
     }
     __syncthreads();
