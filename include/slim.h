@@ -223,7 +223,7 @@ typedef struct slim_gemv_set_info {
     int n_items;           /* row blocks (work items) of the set */
     int max_bits;          /* widest group of the set */
     int max_tokens;        /* largest M of the set */
-    int tiles_per_warp;    /* 16-row tiles a consumer warp owns: an item is 128 rows times this */
+    int tiles_per_warp;    /* 16-row tiles a consumer warp owns (2): an item is 128 rows times this */
     int split;             /* parts the groups of a row block are cut into when the set has fewer row blocks than
                               persistent CTAs (1 .. 8; layers with few groups get fewer): fp32 partial outputs in the
                               workspace, summed in part order by a second small kernel */

@@ -441,7 +441,9 @@ __device__ __forceinline__ void consume_f16(const SetParams& p, const uint32_t s
     auto full = [&](int s) { return sbase + 8u * s; };
     auto empty = [&](int s) { return sbase + 8u * (kSetMaxSlots + s); };
     constexpr int TPI = kSetConsumers * TPW, MPK = 8 * NT;
-    constexpr int CH = NT == 1 ? (TPW == 1 ? 4 : 2) : 2;     // interleaved accumulation chains
+    // interleaved accumulation chains per (tile, token tile): with four (tile, token tile) pairs the MMAs of one pair are far
+    // enough apart without a second chain
+    constexpr int CH = NT * TPW >= 4 ? 1 : (NT == 1 ? (TPW == 1 ? 4 : 2) : 2);
     constexpr uint32_t kOffZ = slot_off_z(TPI), kOffE = slot_off_e(TPI), kOffX = slot_off_x(TPI), kOffW = slot_off_w(TPI, MPK);
     const int gq = lane >> 2, c = lane & 3;
     const uint32_t lane0 = lane == 0 ? 1u : 0u;
@@ -544,7 +546,7 @@ __device__ __forceinline__ void consume_f16(const SetParams& p, const uint32_t s
                         float dd[4];
 #pragma unroll
                         for (int r = 0; r < 4; ++r) {
-                            dd[r] = d[t][0][n][r] + d[t][1][n][r];
+                            dd[r] = CH == 1 ? d[t][0][n][r] : d[t][0][n][r] + d[t][CH > 1 ? 1 : 0][n][r];
                             if (CH == 4) dd[r] += d[t][2 % CH][n][r] + d[t][3 % CH][n][r];
                         }
                         acc[t][n][0] = fmaf(sf.x, fmaf(-zf.x, sx0, dd[0] * e0), acc[t][n][0]);
@@ -594,8 +596,8 @@ constexpr uint32_t kSetOffRing = (kSetOffDesc + kSetProducers * sizeof(SetLayer)
 
 // NT: 8-token MMA tiles, 1 (every M <= 8) or 2.  ONE: every layer has a single token; then only
 // column 0 of the MMA results is ever used, so every lane feeds token 0's fragment and folds token 0.
-// TPW: 16-row tiles per consumer warp (an item is 8 * TPW tiles); two tiles share the fragment loads and
-// the per-group bookkeeping.
+// TPW: 16-row tiles per consumer warp (an item is 8 * TPW tiles; always 2 today); two tiles share the fragment
+// loads and the per-group bookkeeping.
 template <int NT, bool ONE, int TPW>
 __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(const __grid_constant__ SetParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -809,7 +811,7 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     memset(sg, 0, sizeof *sg);
     sg->ws_bytes = 256;
     for (int l = 0; l < n_layers; ++l) sg->mmax = sg->mmax > layers[l].M ? sg->mmax : layers[l].M;
-    sg->tpw = sg->mmax > 8 ? 1 : 2;
+    sg->tpw = 2;
     sg->mpad = sg->mmax <= 1 ? 2 : (sg->mmax <= 8 ? 8 : 16);    // one token: the 8-bit digit form, 512 bytes per slice
     const int tpi = kSetConsumers * sg->tpw;          // tiles per item
     for (int l = 0; l < n_layers; ++l) {
@@ -856,12 +858,12 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
         }
     }
     sg->slot_bytes = static_cast<int>(align_to(static_cast<size_t>(slot_off_w(tpi, sg->mpad)) + static_cast<size_t>(tpi) * 256 * sg->bmax, 128));
-    // as many CTAs per SM (kSetCtasPerSm at most) as still leaves each a ring of 5 slots
+    // as many CTAs per SM (kSetCtasPerSm at most) as still leaves each a ring of 4 slots
     const size_t per_sm = 224 * 1024;
     size_t budget = 0;
     for (sg->ctas_per_sm = kSetCtasPerSm; sg->ctas_per_sm >= 1; --sg->ctas_per_sm) {
         budget = per_sm / sg->ctas_per_sm - 1024 - kSetOffRing;   // 1 KB per CTA is reserved by the system
-        if (budget / sg->slot_bytes >= 5 || sg->ctas_per_sm == 1) break;
+        if (budget / sg->slot_bytes >= 4 || sg->ctas_per_sm == 1) break;
     }
     size_t slots = budget / sg->slot_bytes;
     if (slots > kSetMaxSlots) slots = kSetMaxSlots;
@@ -1153,7 +1155,7 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     if (info->n_layers < 1 || info->grid < 1 || info->grid > slim::kSetMaxGrid || info->n_slots < 2 ||
         info->n_slots > slim::kSetMaxSlots || info->slot_bytes < 128 || info->slot_bytes % 128 != 0 ||
         (info->token_tiles != 1 && info->token_tiles != 2) || info->max_tokens < 1 || info->max_tokens > 8 * info->token_tiles ||
-        info->tiles_per_warp != (info->max_tokens <= 8 ? 2 : 1) ||
+        info->tiles_per_warp != 2 ||
         info->max_bits < 1 || info->max_bits > 4 || info->stage_tasks < 1 || info->split < 1 || info->split > slim::kSetMaxSplit ||
         info->n_layers > 65535)
         return SLIM_ERR_INVALID_ARG;
@@ -1182,7 +1184,7 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     SLIM_CUDA_TRY(cudaGetLastError());
     const cudaError_t e = info->max_tokens == 1 ? slim::launch_set<1, true, 2>(prm, info->grid, smem, s)
                         : info->token_tiles == 1 ? slim::launch_set<1, false, 2>(prm, info->grid, smem, s)
-                                                 : slim::launch_set<2, false, 1>(prm, info->grid, smem, s);
+                                                 : slim::launch_set<2, false, 2>(prm, info->grid, smem, s);
     SLIM_CUDA_TRY(e);
     if (info->split > 1) {
         slim::gemv_set_finish_kernel<<<dim3(32, static_cast<unsigned>(info->n_layers)), 256, 0, s>>>(prm.layers, prm.ws);
