@@ -265,86 +265,105 @@ def linear_rows_f64(x16, codes, scales, zeros, rows, g: int = GROUP) -> np.ndarr
 
 
 # --------------------------------------------------------------------------- storage format
+GROUP_SIZES = (32, 64, 128, 256, 512)
+
+
+def ktile(g: int) -> int:
+    """Columns of a K-tile of the packed format: the group itself up to 128 columns, else 128."""
+    assert g in GROUP_SIZES
+    return min(g, 128)
+
+
+def ktile_bits(bits, g: int) -> np.ndarray:
+    """Bit-width of every K-tile: a group of more than 128 columns is g/128 consecutive tiles of its width."""
+    bits = np.asarray(bits, dtype=np.uint8)
+    return np.repeat(bits, max(g // 128, 1))
+
+
 def packed_bytes(N: int, K: int, bits, g: int = GROUP) -> int:
     """N*K*b-bar/8: groups are stored back to back without padding (App. B.2)."""
     assert K % g == 0 and len(bits) == K // g
-    return 16 * N * int(np.asarray(bits, dtype=np.int64).sum())
+    return g // 8 * N * int(np.asarray(bits, dtype=np.int64).sum())
 
 
-def _unit_word_index(N, bits_prefix, b, t, unit, lane, half):
-    """Index (in 32-bit words) of one word of the packed buffer.
+def _item_bit_index(N, T, tile_prefix, b, t, unit, lane, half):
+    """Bit offset, in the packed buffer, of bit 0 of one item (the T/4 bits a lane holds for one row).
 
-    Group at byte 16*N*B_j; inside it the 16-row tile t at t*256*b; inside that
-    the 256-byte unit `unit`; inside that lane L at 8*L; word `half` (0: even row,
-    1: odd row) at 4*half.
+    K-tile at byte (T/8)*N*B (B = bits of the K-tiles before it); inside it the 16-row tile t at t*2T*b; inside
+    that the unit `unit` (2T bytes); inside that lane L at L*T/16 bytes; item `half` (0: even row, 1: odd row)
+    at half*T/32 bytes.
     """
-    byte = 16 * N * bits_prefix + t * 256 * b + 256 * unit + 8 * lane + 4 * half
-    return byte // 4
+    byte = T // 8 * N * tile_prefix + t * 2 * T * b + 2 * T * unit
+    return 8 * byte + (T // 2) * lane + (T // 4) * half
 
 
 def pack(codes: np.ndarray, bits, g: int = GROUP) -> np.ndarray:
     """Pack codes [N][K] into the sliced bit-plane format; returns uint8 bytes.
 
-    Format (g = 128, N a multiple of 16).  B_j = sum_{i<j} b_i.  Group j holds,
-    for each 16-row tile t, b_j units of 256 bytes.  The code of group width b is
-    cut into slices (lo, w) listed in CODE_SLICES[b]; a slice of width w owns w
-    consecutive units.  A unit is 32 lanes x 8 bytes; lane L = 4*gq + c
-    (gq = 0..7, c = 0..3) holds two little-endian 32-bit words, word 0 for row
-    16t + 2gq and word 1 for row 16t + 2gq + 1.  Word (row r, slice (lo, w),
-    unit u of the slice, c) has 32/w fields; field f occupies bits [w f, w f + w)
-    and stores slice (lo, w) of q[r, 128 j + 32 c + (32/w) u + f].
+    Format (N a multiple of 16, g in GROUP_SIZES).  K is cut into K-tiles of T = min(g, 128) columns; a group of
+    more than 128 columns is g/128 consecutive K-tiles of its bit-width.  K-tiles are stored back to back; a tile
+    of b bits takes N*T*b/8 bytes and holds, for each 16-row tile t, b units of 2T bytes.  The code is cut into
+    slices (lo, w) listed in CODE_SLICES[b]; a slice of width w owns w consecutive units.  A unit is 32 lanes x
+    T/16 bytes; lane L = 4*gq + c (gq = 0..7, c = 0..3) holds two little-endian items of T/4 bits, item 0 for row
+    16t + 2gq and item 1 for row 16t + 2gq + 1.  Item (row r, slice (lo, w), unit u of the slice, c) has (T/4)/w
+    fields; field f occupies bits [w f, w f + w) and stores slice (lo, w) of
+    q[r, T jt + (T/4) c + ((T/4)/w) u + f]  (jt = index of the K-tile).  For g = 128 an item is a 32-bit word.
     """
     codes = np.asarray(codes, dtype=np.uint8)
     N, K = codes.shape
-    G = K // g
-    assert g == 128 and K % g == 0 and N % 16 == 0 and len(bits) == G
-    out = np.zeros(packed_bytes(N, K, bits, g) // 4, dtype=np.uint32)
+    assert g in GROUP_SIZES and K % g == 0 and N % 16 == 0 and len(bits) == K // g
+    T = ktile(g)
+    tb = ktile_bits(bits, g)
+    n_bits = 8 * packed_bytes(N, K, bits, g)
+    out_bits = np.zeros(n_bits, dtype=np.uint8)
     rows = np.arange(N)
     t, r = rows // 16, rows % 16
     gq, half = r // 2, r % 2
     prefix = 0
-    for j in range(G):
-        b = int(bits[j])
-        q = codes[:, j * g:(j + 1) * g].astype(np.uint32)
+    for jt in range(K // T):
+        b = int(tb[jt])
+        q = codes[:, jt * T:(jt + 1) * T].astype(np.uint32)
         assert int(q.max(initial=0)) < 2**b, "code out of range for its group width"
         unit_base = 0
         for (lo, w) in CODE_SLICES[b]:
-            nf = 32 // w
+            nf = T // 4 // w
             for u in range(w):
                 for c in range(4):
-                    word = np.zeros(N, dtype=np.uint32)
+                    base = _item_bit_index(N, T, prefix, b, t, unit_base + u, 4 * gq + c, half)
                     for f in range(nf):
-                        k = 32 * c + nf * u + f
-                        word |= ((q[:, k] >> np.uint32(lo)) & np.uint32(2**w - 1)) << np.uint32(w * f)
-                    idx = _unit_word_index(N, prefix, b, t, unit_base + u, 4 * gq + c, half)
-                    out[idx] = word
+                        k = T // 4 * c + nf * u + f
+                        v = (q[:, k] >> np.uint32(lo)) & np.uint32(2**w - 1)
+                        for bit in range(w):
+                            out_bits[base + w * f + bit] = (v >> np.uint32(bit)) & 1
             unit_base += w
         prefix += b
-    return out.view(np.uint8)
+    return np.packbits(out_bits, bitorder="little")
 
 
 def unpack(packed: np.ndarray, N: int, K: int, bits, g: int = GROUP) -> np.ndarray:
     """Inverse of pack: bytes -> codes uint8 [N][K]."""
-    G = K // g
-    words = np.ascontiguousarray(packed).view(np.uint32)
-    assert words.size * 4 == packed_bytes(N, K, bits, g)
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    assert packed.size == packed_bytes(N, K, bits, g)
+    in_bits = np.unpackbits(packed, bitorder="little")
+    T = ktile(g)
+    tb = ktile_bits(bits, g)
     codes = np.zeros((N, K), dtype=np.uint8)
     rows = np.arange(N)
     t, r = rows // 16, rows % 16
     gq, half = r // 2, r % 2
     prefix = 0
-    for j in range(G):
-        b = int(bits[j])
+    for jt in range(K // T):
+        b = int(tb[jt])
         unit_base = 0
         for (lo, w) in CODE_SLICES[b]:
-            nf = 32 // w
+            nf = T // 4 // w
             for u in range(w):
                 for c in range(4):
-                    word = words[_unit_word_index(N, prefix, b, t, unit_base + u, 4 * gq + c, half)]
+                    base = _item_bit_index(N, T, prefix, b, t, unit_base + u, 4 * gq + c, half)
                     for f in range(nf):
-                        k = j * g + 32 * c + nf * u + f
-                        v = (word >> np.uint32(w * f)) & np.uint32(2**w - 1)
-                        codes[:, k] |= (v << np.uint32(lo)).astype(np.uint8)
+                        k = jt * T + T // 4 * c + nf * u + f
+                        for bit in range(w):
+                            codes[:, k] |= (in_bits[base + w * f + bit] << (lo + bit)).astype(np.uint8)
             unit_base += w
         prefix += b
     return codes
