@@ -149,35 +149,35 @@ def selftest_wait_timeout(workspace: torch.Tensor, limit_us: int = 1000) -> None
     _check("slim_selftest_wait_timeout", lib().slim_selftest_wait_timeout(p, workspace.numel(), int(limit_us), _stream(workspace)))
 
 
-def new_workspace(M: int, N: int, K: int, bits, device="cuda") -> torch.Tensor:
+def new_workspace(M: int, N: int, K: int, bits, device="cuda", g: int = GROUP) -> torch.Tensor:
     """Allocates (torch) and initialises a workspace large enough for this shape."""
-    ws = torch.empty(workspace_bytes(M, N, K, bits), dtype=torch.uint8, device=device)
+    ws = torch.empty(workspace_bytes(M, N, K, bits, g), dtype=torch.uint8, device=device)
     workspace_init(ws)
     return ws
 
 
-def pack_weights(codes: torch.Tensor, bits, packed: torch.Tensor | None = None) -> torch.Tensor:
+def pack_weights(codes: torch.Tensor, bits, packed: torch.Tensor | None = None, g: int = GROUP) -> torch.Tensor:
     b = _bits(bits)
     N, K = codes.shape
     if packed is None:
-        packed = torch.empty(packed_bytes(N, K, b), dtype=torch.uint8, device=codes.device)
+        packed = torch.empty(packed_bytes(N, K, b, g), dtype=torch.uint8, device=codes.device)
     _check("slim_pack_weights", lib().slim_pack_weights(_dev(codes, torch.uint8, "codes"), _bp(b),
-                                                        _dev(packed, torch.uint8, "packed"), N, K, GROUP, _stream(codes)))
+                                                        _dev(packed, torch.uint8, "packed"), N, K, g, _stream(codes)))
     return packed
 
 
 def dequant(packed: torch.Tensor, bits, scales: torch.Tensor, zeros: torch.Tensor, N: int, K: int,
-            out: torch.Tensor | None = None) -> torch.Tensor:
+            out: torch.Tensor | None = None, g: int = GROUP) -> torch.Tensor:
     b = _bits(bits)
     if out is None:
         out = torch.empty((N, K), dtype=torch.float16, device=packed.device)
     _check("slim_dequant", lib().slim_dequant(_dev(packed, torch.uint8, "packed"), _bp(b),
                                               _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
-                                              _dev(out, torch.float16, "W"), N, K, GROUP, _stream(packed)))
+                                              _dev(out, torch.float16, "W"), N, K, g, _stream(packed)))
     return out
 
 
-def _linear(fn_name: str, x, packed, bits, scales, zeros, N, workspace, out):
+def _linear(fn_name: str, x, packed, bits, scales, zeros, N, workspace, out, g: int = GROUP):
     b = _bits(bits)
     M, K = x.shape
     if out is None:
@@ -187,21 +187,22 @@ def _linear(fn_name: str, x, packed, bits, scales, zeros, N, workspace, out):
     fn = getattr(lib(), fn_name)
     _check(fn_name, fn(_dev(x, torch.float16, "x"), _dev(packed, torch.uint8, "packed"), _bp(b),
                        _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
-                       _dev(out, torch.float16, "y"), M, N, K, GROUP, wp, wb, _stream(x)))
+                       _dev(out, torch.float16, "y"), M, N, K, g, wp, wb, _stream(x)))
     return out
 
 
-def mpq_gemv(x, packed, bits, scales, zeros, N: int, workspace, out=None) -> torch.Tensor:
+def mpq_gemv(x, packed, bits, scales, zeros, N: int, workspace, out=None, g: int = GROUP) -> torch.Tensor:
     """y = x W-hat^T for 1 <= M <= 16 (decode path)."""
-    return _linear("slim_mpq_gemv", x, packed, bits, scales, zeros, N, workspace, out)
+    return _linear("slim_mpq_gemv", x, packed, bits, scales, zeros, N, workspace, out, g)
 
 
-def mpq_gemm(x, packed, bits, scales, zeros, N: int, workspace, out=None) -> torch.Tensor:
+def mpq_gemm(x, packed, bits, scales, zeros, N: int, workspace, out=None, g: int = GROUP) -> torch.Tensor:
     """y = x W-hat^T for M > 16 (batched tensor-core path)."""
-    return _linear("slim_mpq_gemm", x, packed, bits, scales, zeros, N, workspace, out)
+    return _linear("slim_mpq_gemm", x, packed, bits, scales, zeros, N, workspace, out, g)
 
 
-def mpq_gemm_static(x, packed, bits, scales, zeros, N: int, out: torch.Tensor, status: torch.Tensor | None = None) -> torch.Tensor:
+def mpq_gemm_static(x, packed, bits, scales, zeros, N: int, out: torch.Tensor, status: torch.Tensor | None = None,
+                    g: int = GROUP) -> torch.Tensor:
     """slim_mpq_gemm without a caller workspace: the library's built-in scratch array is used.
 
     For callers that may not allocate device memory, so `out` (fp16 [M][N]) and the optional
@@ -213,7 +214,7 @@ def mpq_gemm_static(x, packed, bits, scales, zeros, N: int, out: torch.Tensor, s
     sp = _dev(status, torch.int32, "status") if status is not None else None
     _check("slim_mpq_gemm_static", lib().slim_mpq_gemm_static(
         _dev(x, torch.float16, "x"), _dev(packed, torch.uint8, "packed"), _bp(b), _dev(scales, torch.float16, "scales"),
-        _dev(zeros, torch.float16, "zeros"), _dev(out, torch.float16, "y"), M, N, K, GROUP, sp, _stream(x)))
+        _dev(zeros, torch.float16, "zeros"), _dev(out, torch.float16, "y"), M, N, K, g, sp, _stream(x)))
     return out
 
 
@@ -427,8 +428,8 @@ class LayerSet:
 class QuantLinear:
     """One quantised layer resident on the device: packed codes, scales, zeros, bit map."""
 
-    def __init__(self, packed, bits, scales, zeros, N: int, K: int):
-        self.packed, self.bits, self.scales, self.zeros, self.N, self.K = packed, _bits(bits), scales, zeros, N, K
+    def __init__(self, packed, bits, scales, zeros, N: int, K: int, g: int = GROUP):
+        self.packed, self.bits, self.scales, self.zeros, self.N, self.K, self.g = packed, _bits(bits), scales, zeros, N, K, g
 
     @classmethod
     def from_weight(cls, W: torch.Tensor, act_norm: torch.Tensor, avg_bits: int, p: int = -1) -> "QuantLinear":
@@ -440,12 +441,12 @@ class QuantLinear:
         return cls(pack_weights(codes, bits), bits, scales, zeros, N, K)
 
     def workspace_bytes(self, M: int) -> int:
-        return workspace_bytes(M, self.N, self.K, self.bits)
+        return workspace_bytes(M, self.N, self.K, self.bits, self.g)
 
     def forward(self, x: torch.Tensor, workspace: torch.Tensor, out=None) -> torch.Tensor:
         fn = mpq_gemv if x.shape[0] <= GEMV_MAX_M else mpq_gemm
-        return fn(x, self.packed, self.bits, self.scales, self.zeros, self.N, workspace, out)
+        return fn(x, self.packed, self.bits, self.scales, self.zeros, self.N, workspace, out, self.g)
 
     def algorithmic_bytes(self, M: int) -> int:
-        G = self.K // GROUP
+        G = self.K // self.g
         return self.packed.numel() + 2 * 2 * G * self.N + G + 2 * M * self.K + 2 * M * self.N

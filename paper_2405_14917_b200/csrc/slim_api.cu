@@ -16,14 +16,15 @@ void set_cuda_error(cudaError_t e) {
 
 int make_group_table(int N, int K, int g, const uint8_t* bits_host, GroupTable* out) {
     if (bits_host == nullptr || N < 0 || K < 0) return SLIM_ERR_INVALID_ARG;
-    if (g != SLIM_GROUP) return SLIM_ERR_UNSUPPORTED;
-    if (K % SLIM_GROUP != 0 || N % 16 != 0) return SLIM_ERR_UNSUPPORTED;
-    const int G = K / SLIM_GROUP;
+    if (g != 128 && g != 256 && g != 512) return SLIM_ERR_UNSUPPORTED;
+    if (K % g != 0 || N % 16 != 0) return SLIM_ERR_UNSUPPORTED;
+    const int G = K / SLIM_GROUP;                      // K-tiles
     if (G > SLIM_MAX_GROUPS) return SLIM_ERR_UNSUPPORTED;
     out->G = G;
+    out->gshift = g == 128 ? 0 : (g == 256 ? 1 : 2);
     int acc = 0;
     for (int j = 0; j < G; ++j) {
-        const int b = bits_host[j];
+        const int b = bits_host[j >> out->gshift];
         if (b < 1 || b > 4) return SLIM_ERR_INVALID_ARG;
         out->bits[j] = static_cast<uint8_t>(b);
         out->prefix[j] = static_cast<uint16_t>(acc);
@@ -58,6 +59,7 @@ int slim_last_cuda_error(void) { return slim::g_last_cuda_error.load(); }
 
 int slim_packed_bytes(int N, int K, int g, const uint8_t* bits_host, size_t* out_bytes) {
     if (out_bytes == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (slim::is_small_group(g)) return slim::small_packed_bytes(N, K, g, bits_host, out_bytes);
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;

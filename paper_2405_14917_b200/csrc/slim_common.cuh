@@ -14,9 +14,11 @@ namespace slim {
 // Group table passed by value in kernel parameters (the paper's "additional array" of group
 // bit-widths plus the "cumulative calculations" that give each group's start, App. B.2).
 struct GroupTable {
-    int G;
-    uint16_t prefix[SLIM_MAX_GROUPS + 1];  // prefix[j] = b_0 + ... + b_{j-1}
-    uint8_t bits[SLIM_MAX_GROUPS];
+    int G;                                 // K-tiles of 128 columns
+    int gshift;                            // a group is 2^gshift consecutive K-tiles (g = 128, 256, 512): tile j belongs to
+                                           // group j >> gshift, whose scale and zero-point rows it shares
+    uint16_t prefix[SLIM_MAX_GROUPS + 1];  // prefix[j] = b_0 + ... + b_{j-1} over the K-tiles
+    uint8_t bits[SLIM_MAX_GROUPS];         // bit-width of every K-tile
 };
 
 void set_cuda_error(cudaError_t e);
@@ -32,8 +34,20 @@ size_t gemv_route_workspace_bytes(int M, int N, int K, int g, const uint8_t* bit
 int gemv_route(const void* x, const void* packed, const uint8_t* bits_host, const GroupTable& gt, const void* scales, const void* zeros,
                void* y, int M, int N, int K, int g, void* workspace, size_t workspace_bytes, cudaStream_t stream);
 
-// Validates shape arguments and fills the table.  Returns SLIM_OK or an error status.
+// Validates shape arguments and fills the table, for group sizes of 128, 256 and 512 columns (bits_host has K / g
+// entries).  Returns SLIM_OK or an error status; SLIM_ERR_UNSUPPORTED for the group sizes 32 and 64, which have
+// kernels of their own (is_small_group).
 int make_group_table(int N, int K, int g, const uint8_t* bits_host, GroupTable* out);
+inline bool is_small_group(int g) { return g == 32 || g == 64; }
+
+// Group sizes of 32 and 64 columns (slim_small_group.cu): same contracts as the entry points that call them.
+int small_packed_bytes(int N, int K, int g, const uint8_t* bits_host, size_t* out_bytes);
+int small_workspace_bytes(int M, int N, int K, int g, const uint8_t* bits_host, size_t* out_bytes);
+int small_pack(const uint8_t* codes, const uint8_t* bits_host, void* packed, int N, int K, int g, cudaStream_t s);
+int small_dequant(const void* packed, const uint8_t* bits_host, const void* scales, const void* zeros, void* W, int N, int K, int g,
+                  cudaStream_t s);
+int small_linear(const void* x, const void* packed, const uint8_t* bits_host, const void* scales, const void* zeros, void* y,
+                 int M, int N, int K, int g, void* workspace, size_t workspace_bytes, cudaStream_t s);
 
 #define SLIM_CUDA_TRY(expr)                                    \
     do {                                                       \

@@ -467,7 +467,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
                         if (lane == 0)
                             g::bulk_g2s(dst, p.packed + 16ull * N * p.gt.prefix[j] + static_cast<size_t>(8 * rb) * 256 * b, wbytes, p_full(sp));
                         else
-                            g::bulk_g2s(dst + 8192 + 256 * (lane - 1), sz + static_cast<size_t>(j) * N, sbytes, p_full(sp));
+                            g::bulk_g2s(dst + 8192 + 256 * (lane - 1), sz + static_cast<size_t>(j >> p.gt.gshift) * N, sbytes, p_full(sp));
                     } else if (lane == 0) {
                         g::mbar_arrive(p_full(sp));             // no row of mine exists: nothing to bring
                     }
@@ -851,6 +851,8 @@ extern "C" int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* b
                              void* y, int M, int N, int K, int g, void* workspace, size_t workspace_bytes, void* stream) {
     if (M < 0) return SLIM_ERR_INVALID_ARG;
     if (M > 0 && M <= SLIM_GEMV_MAX_M) return SLIM_ERR_INVALID_ARG;     // the decode path serves these
+    if (slim::is_small_group(g))
+        return slim::small_linear(x, packed, bits_host, scales, zeros, y, M, N, K, g, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;

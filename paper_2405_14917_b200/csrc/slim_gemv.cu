@@ -162,7 +162,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const __grid_const
                 if (lane < 16 * b) cp_async16(dst + 16 * lane, src + 16 * lane);
                 if (lane + 32 < 16 * b) cp_async16(dst + 16 * (lane + 32), src + 16 * (lane + 32));
                 if (lane < 4) {
-                    const __half* sz = (lane < 2 ? p.scales : p.zeros) + static_cast<size_t>(j) * N + 16 * tile + 8 * (lane & 1);
+                    const __half* sz = (lane < 2 ? p.scales : p.zeros) + static_cast<size_t>(j >> p.gt.gshift) * N + 16 * tile + 8 * (lane & 1);
                     cp_async16(dst + 256 * b + 16 * lane, sz);
                 }
             }
@@ -506,6 +506,7 @@ extern "C" {
 
 int slim_workspace_bytes(int M, int N, int K, int g, const uint8_t* bits_host, size_t* out_bytes) {
     if (out_bytes == nullptr || M < 0) return SLIM_ERR_INVALID_ARG;
+    if (slim::is_small_group(g)) return slim::small_workspace_bytes(M, N, K, g, bits_host, out_bytes);
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;
@@ -556,6 +557,8 @@ int slim_workspace_status(void* workspace, void* stream) {
 int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host, const void* scales, const void* zeros,
                   void* y, int M, int N, int K, int g, void* workspace, size_t workspace_bytes, void* stream) {
     if (M < 0 || M > SLIM_GEMV_MAX_M) return SLIM_ERR_INVALID_ARG;
+    if (slim::is_small_group(g))
+        return slim::small_linear(x, packed, bits_host, scales, zeros, y, M, N, K, g, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;

@@ -73,7 +73,8 @@ struct SetLayer {
     uint8_t bits[SLIM_MAX_GROUPS];
     uint8_t order[SLIM_MAX_GROUPS];       // the order in which the groups are streamed: by bit-width, then by index
     uint8_t split;                        // parts the groups of a row block are cut into (1: whole K per item)
-    uint8_t pad2[3];
+    uint8_t gshift;                       // 2^gshift K-tiles of 128 columns share a row of scales and zeros (g = 128 << gshift)
+    uint8_t pad2[2];
 };
 static_assert(sizeof(SetLayer) % 16 == 0, "descriptors are copied and read in 16-byte pieces");
 
@@ -671,7 +672,7 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                     }
                     const size_t off = lane == 0 ? 16ull * N * D->prefix[j] + static_cast<size_t>(TPI * rb) * 256 * b
                                      : lane == 3 ? staged_group_offset(j, D->pre3[j], MP)
-                                                 : 2ull * static_cast<size_t>(j) * N;
+                                                 : 2ull * static_cast<size_t>(j >> D->gshift) * N;
                     const uint32_t bytes = lane == 0 ? wbytes : lane == 3 ? xbytes : szb;
                     __syncwarp();
                     if (lane < 4) sb::bulk_g2s(slot + dst_off, base + off, bytes, full(s));
@@ -892,6 +893,7 @@ static void fill_descriptor(const slim_layer& L, const GroupTable& gt, int mpad,
     d.task0 = task0;
     d.x_off = x_off;
     d.split = static_cast<uint8_t>(split);
+    d.gshift = static_cast<uint8_t>(gt.gshift);
     d.part_off = part_off;
     memcpy(d.prefix, gt.prefix, sizeof d.prefix);
     memcpy(d.bits, gt.bits, sizeof d.bits);

@@ -65,8 +65,8 @@ __global__ void __launch_bounds__(256) dequant_kernel(const uint32_t* __restrict
 #pragma unroll
         for (int i = 0; i < 8; ++i) q[i] |= ((word >> (w * (f0 + i))) & mask) << lo;
     }
-    const float sc = __half2float(scales[static_cast<size_t>(j) * N + row]);
-    const float zp = __half2float(zeros[static_cast<size_t>(j) * N + row]);
+    const float sc = __half2float(scales[static_cast<size_t>(j >> gt.gshift) * N + row]);
+    const float zp = __half2float(zeros[static_cast<size_t>(j >> gt.gshift) * N + row]);
     __align__(16) __half out[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) out[i] = __float2half_rn(__fmul_rn(sc, __fsub_rn(static_cast<float>(q[i]), zp)));
@@ -78,6 +78,7 @@ __global__ void __launch_bounds__(256) dequant_kernel(const uint32_t* __restrict
 extern "C" {
 
 int slim_pack_weights(const uint8_t* codes, const uint8_t* bits_host, void* packed, int N, int K, int g, void* stream) {
+    if (slim::is_small_group(g)) return slim::small_pack(codes, bits_host, packed, N, K, g, static_cast<cudaStream_t>(stream));
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;
@@ -93,6 +94,7 @@ int slim_pack_weights(const uint8_t* codes, const uint8_t* bits_host, void* pack
 
 int slim_dequant(const void* packed, const uint8_t* bits_host, const void* scales, const void* zeros, void* W,
                  int N, int K, int g, void* stream) {
+    if (slim::is_small_group(g)) return slim::small_dequant(packed, bits_host, scales, zeros, W, N, K, g, static_cast<cudaStream_t>(stream));
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;

@@ -164,6 +164,7 @@ int slim_group_salience(const void* W, const float* act_norm, double* salience, 
 
 static int quantize_minmax_impl(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
                                 int N, int K, int g, int sign_alpha, const int* groups_host, int n_groups, void* stream) {
+    if (g != SLIM_GROUP) return SLIM_ERR_UNSUPPORTED;      // the quantizer kernels work on groups of 128 columns
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;
@@ -328,6 +329,7 @@ __global__ void __launch_bounds__(kSqcWarps * 32) quantize_sqc_kernel(const __ha
 
 extern "C" int slim_quantize_sqc(const void* W, const uint8_t* bits_host, uint8_t* codes, void* scales, void* zeros,
                                  int* tau_index, int N, int K, int g, double lambda, int n, void* stream) {
+    if (g != SLIM_GROUP) return SLIM_ERR_UNSUPPORTED;      // the quantizer kernels work on groups of 128 columns
     slim::GroupTable gt;
     const int st = slim::make_group_table(N, K, g, bits_host, &gt);
     if (st != SLIM_OK) return st;

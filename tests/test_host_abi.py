@@ -60,7 +60,12 @@ def test_shape_and_argument_errors(slim):
     out = ctypes.c_size_t(0)
     L = slim.lib()
     bp = bits.ctypes.data_as(ctypes.c_void_p)
-    assert L.slim_packed_bytes(16, 256, 64, bp, ctypes.byref(out)) == -2      # g != 128
+    assert L.slim_packed_bytes(16, 256, 96, bp, ctypes.byref(out)) == -2      # g not in {32, 64, 128, 256, 512}
+    assert L.slim_packed_bytes(16, 256, 1024, bp, ctypes.byref(out)) == -2
+    b4 = np.array([2, 3, 1, 2], np.uint8)
+    assert L.slim_packed_bytes(16, 256, 64, b4.ctypes.data_as(ctypes.c_void_p), ctypes.byref(out)) == 0 and out.value == 16 * 64 * 8 // 8
+    assert L.slim_packed_bytes(16, 256, 256, bp, ctypes.byref(out)) == 0 and out.value == 16 * 256 * 2 // 8
+    assert L.slim_packed_bytes(16, 256, 512, bp, ctypes.byref(out)) == -2     # K % g
     assert L.slim_packed_bytes(16, 200, 128, bp, ctypes.byref(out)) == -2     # K % 128
     assert L.slim_packed_bytes(24, 256, 128, bp, ctypes.byref(out)) == -2     # N % 16
     assert L.slim_packed_bytes(16, 256, 128, None, ctypes.byref(out)) == -1   # no bit map
