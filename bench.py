@@ -781,6 +781,60 @@ def single_layer_entry(layer, device, timer, copies=64):
             "rotating_copies": copies, "rotating_per_layer": per_layer, "rotating_set": as_set}
 
 
+def group_size_entries(device, timer):
+    """One 4096 x 4096 layer, avg 2-bit, M = 1, at the group sizes of the paper's group-size ablation: 64 distinct copies
+    (> L2) per step through slim_mpq_gemv.  Throughput does not depend on the values, so codes, scales and zero points
+    are drawn directly (seeded), with the 25 / 50 / 25 % mix of 1 / 2 / 3-bit groups of the other workloads."""
+    import torch
+    from paper_2405_14917_b200 import binding as slim
+    N = K = 4096
+    copies = 64
+    out = []
+    gen = torch.Generator(device=device)
+    gen.manual_seed(32)
+    for g in (32, 64, 128, 256, 512):
+        G = K // g
+        order = torch.randperm(G, generator=gen, device=device).cpu().numpy()
+        bits = np.full(G, 2, dtype=np.uint8)
+        bits[order[:G // 4]] = 3
+        bits[order[G // 4:2 * (G // 4)]] = 1
+        layers = []
+        for _ in range(copies):
+            codes = torch.cat([torch.randint(0, 2 ** int(b), (N, g), generator=gen, device=device, dtype=torch.uint8) for b in bits], dim=1)
+            scales = (torch.rand((G, N), generator=gen, device=device) * 0.02 + 0.001).half()
+            zeros = torch.cat([torch.randint(0, 2 ** int(b), (1, N), generator=gen, device=device) for b in bits]).half()
+            layers.append(slim.QuantLinear(slim.pack_weights(codes.contiguous(), bits, g=g), bits, scales, zeros, N, K, g))
+            del codes
+        M = 1
+        x = torch.randn(M, K, generator=gen, device=device).half()
+        ys = [torch.empty(M, N, dtype=torch.float16, device=device) for _ in layers]
+        ws = torch.zeros(max(L.workspace_bytes(M) for L in layers), dtype=torch.uint8, device=device)
+        slim.workspace_init(ws)
+
+        def run():
+            for L, y in zip(layers, ys):
+                L.forward(x, ws, out=y)
+        graph = _graph_of(run, device)
+        for _ in range(3):
+            graph.replay()
+        tm = _timing_summary(timer.blocks(graph.replay, 10, 0.3), 10)
+        slim.workspace_status(ws)
+        alg = sum(L.algorithmic_bytes(M) for L in layers)
+        ms = tm["ms_per_step_median"]
+        peak, peak_kind = measured_hbm_peak()
+        achieved = alg / (ms * 1e-3) / 1e9
+        out.append({"name": f"single-4096x4096-avg2-m1-g{g}", "metric": f"one 4096 x 4096 layer per launch, avg 2-bit, M = 1, group size {g} (slim_mpq_gemv, 64 rotating copies)",
+                    "value": achieved, "unit": UNIT, "ms_per_step": ms, "timing": tm,
+                    "kernel": "gemv_small_kernel (CUDA cores)" if g < 128 else "gemv_kernel (tensor cores)",
+                    "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
+                                 "avg_launch_us": 1e3 * ms / copies, "algorithmic_bytes_per_launch": alg / copies},
+                    "config": {"workload": f"single-4096x4096-avg2-m1-g{g}", "g": g, "layers": copies, "algorithmic_bytes_per_step": alg,
+                               "data": "codes, scales and zero points drawn directly (seeded)"}})
+        del layers, graph
+        torch.cuda.empty_cache()
+    return out
+
+
 def cpu_baseline_legs(spec):
     """The oracle as it stands on the host cores: all cores (the reported baseline) and one core."""
     base = cpu_baseline(spec, budget_s=10.0)
@@ -819,6 +873,11 @@ def secondary_entries(args, device, timer, primary_layers, clock_gpu):
     guarded(lambda: decode_entry("llama7b-decode-avg2-m1-per-layer", primary_layers, spec7, device, timer, "per-layer", 50, 0.5, clock_gpu=clock_gpu))
     guarded(lambda: decode_entry("llama7b-decode-avg2-m1-decoder-order", primary_layers, spec7, device, timer, "decoder-order", 50, 0.5, clock_gpu=clock_gpu))
     guarded(lambda: single_layer_entry(primary_layers[0], device, timer))
+    try:
+        out.extend(group_size_entries(device, timer))
+    except Exception as e:
+        out.append({"name": "group sizes", "error": f"{type(e).__name__}: {e}"})
+    torch.cuda.empty_cache()
     for wname in ("llama13b-prefill-avg3-m2048", "llama13b-prefill-avg3-m512"):
         spec = workload_spec(wname)
         layers13 = build_layers(spec, device, 0) if wname.endswith("m2048") else layers13

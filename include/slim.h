@@ -1,7 +1,7 @@
 /* slim.h -- C ABI of the B200 (sm_100a) group-wise mixed-precision weight-only linear layer.
  *
  * The layer is y = x * W^T with W stored quantised: the input dimension K is cut into groups of
- * g = 128 consecutive columns (Algorithm 1 of the SliM-LLM paper slices w[:, b:b+beta]); group j
+ * g consecutive columns, 128 in the paper's main results (Algorithm 1 of the SliM-LLM paper slices w[:, b:b+beta]); group j
  * carries one bit-width b_j in {1,2,3,4} (Salience-Determined Bit Allocation, Sec. 3.2.2) and every
  * (row, group) pair carries an fp16 scale s and an fp16 zero point z.  A stored code q dequantises
  * as w = s * (q - z) (inverse of Eq. 1, written out inside Eq. 5).
@@ -14,7 +14,7 @@
  *     scales  fp16  [G][N]        device   (N contiguous)
  *     zeros   fp16  [G][N]        device   (any fp16 value; integers for Eq. 1, 0.5 for Eq. 2)
  *     codes   uint8 [N][K]        device   (unpacked codes, code < 2^b_j)
- *     bits    uint8 [G]           HOST     (read during the call; values 1..4)
+ *     bits    uint8 [G]           HOST     (read during the call; values 1..4; G = K / g)
  *     packed  bytes               device   (format below, slim_packed_bytes() bytes)
  *   "device" pointers must be 16-byte aligned and are owned by the caller, who keeps them alive
  *   until the work enqueued on `stream` has finished.  No function allocates device memory,
@@ -26,21 +26,29 @@
  * that make their first calls together repeat it harmlessly.  Calls that share a workspace, or the built-in scratch
  * of slim_mpq_gemm_static, must still be ordered on one stream.
  *
- * Limits: g must be 128; K a multiple of 128 with at most 256 groups; N a multiple of 16;
- * N = 0 or M = 0 is a successful no-op.  Anything else returns an error status and enqueues nothing.
+ * Limits: g in {32, 64, 128, 256, 512} (the group sizes of the paper's group-size ablation; bits, scales and zeros
+ * have K / g entries or rows); K a multiple of g and of 128 with at most 256 tiles of 128 columns (1024 groups for
+ * g < 128); N a multiple of 16; N = 0 or M = 0 is a successful no-op.  Anything else returns an error status and
+ * enqueues nothing.  The quantizers, the SBA search, the GPTQ loop and the layer-set launch of groups smaller than
+ * 128 columns take g = 128 only (SLIM_ERR_UNSUPPORTED otherwise); pack, dequant and both linear entry points take
+ * every g.  Groups of 256 and 512 columns run on the tensor-core kernels of the 128-column tiles (a group is 2 or 4
+ * tiles that share a row of scales and zeros); groups of 32 and 64 columns run on plain CUDA-core kernels, and the
+ * batched entry point then wants room for the fp16 weights in its workspace (slim_workspace_bytes says how much).
  *
- * Packed format ("sliced bit planes", version SLIM_FORMAT_VERSION).  Groups are stored back to
- * back without padding, as the paper's deployment format does (App. B.2), so the buffer holds
- * exactly N*K*avg_bits/8 bytes.  With B_j = b_0 + ... + b_{j-1}:
- *   - group j starts at byte 16*N*B_j and holds, for each tile t of 16 consecutive rows, b_j
- *     units of 256 bytes (tile t at offset t*256*b_j inside the group);
+ * Packed format ("sliced bit planes", version SLIM_FORMAT_VERSION).  K is cut into K-tiles of T = min(g, 128)
+ * columns; a group of more than 128 columns is g/128 consecutive K-tiles of its bit-width.  K-tiles are stored back
+ * to back without padding, as the paper's deployment format does (App. B.2), so the buffer holds exactly
+ * N*K*avg_bits/8 bytes.  With B_j = bits of the K-tiles before tile j:
+ *   - K-tile j starts at byte (T/8)*N*B_j and holds, for each tile t of 16 consecutive rows, b_j
+ *     units of 2T bytes (tile t at offset t*2T*b_j inside the K-tile);
  *   - a b-bit code is cut into slices (lo, w): b=1 -> (0,1); b=2 -> (0,2); b=3 -> (0,2),(2,1);
  *     b=4 -> (0,4); slice value = (q >> lo) & (2^w - 1).  A slice of width w owns w consecutive
  *     units, slices in the order listed;
- *   - a unit is 32 lanes x 8 bytes.  Lane L = 4*gq + c (gq = 0..7, c = 0..3) holds two
- *     little-endian 32-bit words: word 0 belongs to row 16t + 2gq, word 1 to row 16t + 2gq + 1;
- *   - the word of (row r, slice (lo,w), unit u of that slice, c) has 32/w fields of w bits; field f
- *     (bits [w*f, w*f + w)) stores the slice of q[r][128*j + 32*c + (32/w)*u + f].
+ *   - a unit is 32 lanes x T/16 bytes.  Lane L = 4*gq + c (gq = 0..7, c = 0..3) holds two
+ *     little-endian items of T/4 bits: item 0 belongs to row 16t + 2gq, item 1 to row 16t + 2gq + 1;
+ *   - the item of (row r, slice (lo,w), unit u of that slice, c) has (T/4)/w fields of w bits; field f
+ *     (bits [w*f, w*f + w)) stores the slice of q[r][T*j + (T/4)*c + ((T/4)/w)*u + f].
+ * For g >= 128 a unit is 256 bytes and an item a 32-bit word.
  */
 #ifndef SLIM_H_
 #define SLIM_H_
@@ -53,14 +61,14 @@ extern "C" {
 #endif
 
 #define SLIM_FORMAT_VERSION 2
-#define SLIM_GROUP 128
-#define SLIM_MAX_GROUPS 256
+#define SLIM_GROUP 128           /* the paper's default group size, and the widest K-tile of the packed format */
+#define SLIM_MAX_GROUPS 256      /* most K-tiles of 128 columns in a layer (K <= 32768) */
 #define SLIM_GEMV_MAX_M 16
 
 enum {
     SLIM_OK = 0,
     SLIM_ERR_INVALID_ARG = -1, /* null pointer, negative size, bit-width outside 1..4, M out of range */
-    SLIM_ERR_UNSUPPORTED = -2, /* g != 128, K % 128 != 0, N % 16 != 0, more than 256 groups */
+    SLIM_ERR_UNSUPPORTED = -2, /* group size not served by this entry point, K % g or K % 128 != 0, N % 16 != 0, too many groups */
     SLIM_ERR_ALIGNMENT = -3,   /* a device pointer is not 16-byte aligned */
     SLIM_ERR_WORKSPACE = -4,   /* workspace missing or smaller than slim_workspace_bytes() */
     SLIM_ERR_CUDA = -5,        /* a CUDA runtime call failed; see slim_last_cuda_error() */
@@ -201,7 +209,8 @@ int slim_mpq_gemm_static(const void* x, const void* packed, const uint8_t* bits_
  * most  sum over groups of 2^-22 max|x_group| sum_{k in group} |w-hat[n][k]|  to the error of the fp16
  * path (slim_mpq_gemv multiplies the fp16 x as it is); x must be finite.  Sets with more tokens multiply
  * the fp16 x as it is.
- * N > 0 a multiple of 16, K > 0 a multiple of 128. */
+ * N > 0 a multiple of 16, K > 0 a multiple of 128; g in {128, 256, 512}, one value for the whole set (for 256 and
+ * 512 "group" in the bound above reads "128 columns of a group"); SLIM_ERR_UNSUPPORTED for 32 and 64. */
 typedef struct slim_layer {
     const void* x;             /* device fp16 [M][K] */
     const void* packed;        /* device, packed codes of the layer */
