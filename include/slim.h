@@ -228,7 +228,7 @@ typedef struct slim_gemv_set_info {
     int n_slots;           /* ring slots per CTA */
     int slot_bytes;
     int token_tiles;       /* 8-token MMA tiles: 1 or 2 */
-    int stage_tasks;       /* (layer, token, group) triples of the set */
+    int stage_tasks;       /* (layer, token, group) triples staged; layers with one x and one bit map count once */
     int n_items;           /* row blocks (work items) of the set */
     int max_bits;          /* widest group of the set */
     int max_tokens;        /* largest M of the set */

@@ -1047,7 +1047,7 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
     int task = 0;
     size_t ws_off = 256;
     // workspace: the staged activations of all layers, then the fp32 partial outputs of the layers that are split
-    std::vector<size_t> part_off(static_cast<size_t>(n_layers), 0);
+    std::vector<size_t> part_off(static_cast<size_t>(n_layers), 0), x_off(static_cast<size_t>(n_layers), 0);
     {
         size_t off = 256;
         for (int l = 0; l < n_layers; ++l) {
@@ -1068,7 +1068,15 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
         slim::make_group_table(L.N, L.K, g, L.bits_host, &gt);
         slim::SetLayer d;
         const int sp = slim::layer_split(sg.split, gt.G);
-        slim::fill_descriptor(L, gt, sg.mpad, task, ws_off, sp, part_off[l], &d);
+        // A layer that reads the activations of an earlier layer through the same bit map (the staged form depends
+        // on the group's bit-width) uses that layer's staged copy and has no staging tasks of its own.
+        int same = -1;
+        for (int e = 0; e < l && same < 0; ++e) {
+            const slim_layer& E = layers_host[e];
+            if (E.x == L.x && E.M == L.M && E.K == L.K && memcmp(E.bits_host, L.bits_host, static_cast<size_t>(L.K / g)) == 0) same = e;
+        }
+        x_off[l] = same >= 0 ? x_off[same] : ws_off;
+        slim::fill_descriptor(L, gt, sg.mpad, task, x_off[l], sp, part_off[l], &d);
         ws_off += slim::layer_ws_bytes(sg.mpad, gt);
         SLIM_CUDA_TRY(cudaMemcpyAsync(plan_dev + slim::kSetPlanHeader + static_cast<size_t>(l) * sizeof d, &d, sizeof d,
                                       cudaMemcpyHostToDevice, s));
@@ -1091,7 +1099,7 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
                 cost.push_back(slim::item_cost(th < tpi ? th : tpi, gt, d.order, p0, p1));
             }
         }
-        task += (sg.mpad == 2 ? 1 : sg.mpad) * gt.G;
+        if (same < 0) task += (sg.mpad == 2 ? 1 : sg.mpad) * gt.G;
     }
     // The deal: items by falling cost (equal costs in the set's order), each to the CTA that has the
     // least so far (the lowest-numbered of equals).  Within a CTA the heavy items come first.

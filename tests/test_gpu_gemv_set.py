@@ -177,6 +177,32 @@ def test_projections_that_share_one_input():
         check_output(y.cpu().numpy(), orc.linear_f64(layers[0]["x"], L["codes"], L["scales"], L["zeros"]), "shared x")
 
 
+@pytest.mark.parametrize("M", [1, 2, 9])
+def test_layers_that_share_input_and_bit_map_are_staged_once(M):
+    """The staged form of x depends on the bit-width of each group, so layers share a staged copy when they share
+    the x tensor AND the bit map.  Two such layers, one with the same x but another map in between, and one with
+    its own x: the staging tasks are those of three layers, and every output still matches."""
+    slim = _slim()
+    K = 1024
+    bits_a = np.array([2, 1, 3, 2, 2, 4, 1, 1], dtype=np.uint8)
+    bits_b = np.array([3, 1, 2, 2, 1, 2, 3, 2], dtype=np.uint8)
+    layers = [oracle_layer(384, K, 2, M, seed_name="share", block=0, bits=bits_a),
+              oracle_layer(256, K, 2, M, seed_name="share", block=1, bits=bits_b),
+              oracle_layer(512, K, 2, M, seed_name="share", block=2, bits=bits_a),
+              oracle_layer(128, K, 2, M, seed_name="share", block=3, bits=bits_a)]
+    x_shared = torch.from_numpy(layers[0]["x"]).cuda()
+    x_own = torch.from_numpy(layers[3]["x"]).cuda()
+    xs = [x_shared, x_shared, x_shared, x_own]
+    entries = [(_device_layer(L), x, torch.empty(M, L["N"], dtype=torch.float16, device="cuda")) for L, x in zip(layers, xs)]
+    s = slim.LayerSet(entries)
+    alone = slim.LayerSet(entries[:1]).info["stage_tasks"]
+    assert s.info["stage_tasks"] == 3 * alone
+    s.run()
+    s.check()
+    for k, (L, (_, x, y)) in enumerate(zip(layers, entries)):
+        check_output(y.cpu().numpy(), orc.linear_f64(x.cpu().numpy(), L["codes"], L["scales"], L["zeros"]), f"layer {k}")
+
+
 def test_single_token_fixed_point_with_outlier_channels():
     """Single-token sets round x per group to fixed point relative to the group's largest |x|.  Outlier channels
     (a few activations 100 x the rest, as in LLM activations) and a group of tiny activations must stay within the
