@@ -235,8 +235,8 @@ typedef struct slim_gemv_set_info {
     int tiles_per_warp;    /* 16-row tiles a consumer warp owns (2): an item is 128 rows times this */
     int split;             /* parts the groups of a row block are cut into when the set has fewer row blocks than
                               persistent CTAs (1 .. 8; layers with few groups get fewer): fp32 partial outputs in the
-                              workspace, summed in part order by a second small kernel */
-    int reserved;
+                              workspace, added in part order by the warp whose part lands last */
+    int n_counters;        /* arrival counters of the split row blocks (workspace, cleared by every launch) */
     size_t plan_bytes;
     size_t workspace_bytes;
 } slim_gemv_set_info;

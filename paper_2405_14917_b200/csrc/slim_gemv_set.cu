@@ -74,7 +74,7 @@ struct SetLayer {
     uint8_t order[SLIM_MAX_GROUPS];       // the order in which the groups are streamed: by bit-width, then by index
     uint8_t split;                        // parts the groups of a row block are cut into (1: whole K per item)
     uint8_t gshift;                       // 2^gshift K-tiles of 128 columns share a row of scales and zeros (g = 128 << gshift)
-    uint8_t pad2[2];
+    uint16_t cnt0;                        // split > 1: the layer's first arrival counter (one per row block and consumer warp)
 };
 static_assert(sizeof(SetLayer) % 16 == 0, "descriptors are copied and read in 16-byte pieces");
 
@@ -102,7 +102,7 @@ struct SetParams {
     const int* item_begin;
     const SetLayer* layers;
     const SetItem* items;
-    uint8_t* ws;                           // workspace: status word, then the layers' fragments and sums
+    uint8_t* ws;                           // workspace: status word, arrival counters, then the layers' fragments and sums
     int n_layers, n_slots, slot_bytes;
     int one;                               // 1: a multiplier the compiler cannot fold, for selects done as integer multiply-adds
 };
@@ -237,18 +237,15 @@ __device__ __forceinline__ void mma_i8_first(int (&d)[4], uint32_t a0, uint32_t 
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b.x), "r"(b.y), "r"(0));
 }
 
-// One warp per (layer, token, group): fragments and sums of the whole set, once.
-__global__ void __launch_bounds__(256) gemv_set_stage_kernel(const SetLayer* __restrict__ layers, uint8_t* ws, int n_layers, int n_tasks) {
-    const int lane = threadIdx.x & 31;
-    const int task = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (task >= n_tasks) return;
-    int lo = 0, hi = n_layers - 1;                       // last layer whose task0 <= task
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (layers[mid].task0 <= task) lo = mid; else hi = mid - 1;
-    }
-    const SetLayer& L = layers[lo];
-    const int pi = task - L.task0;
+// The arrival counters of the split row blocks (workspace offset kSetOffCounters) start every launch at zero.
+constexpr uint32_t kSetOffCounters = 256;
+__device__ __forceinline__ void stage_clear_counters(uint8_t* ws, int n_counters) {
+    unsigned int* cnt = reinterpret_cast<unsigned int*>(ws + kSetOffCounters);
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_counters; i += gridDim.x * blockDim.x) cnt[i] = 0u;
+}
+
+// Staging task `pi` of layer L (one warp): token pi / G, group pi % G.
+__device__ __forceinline__ void stage_task(const SetLayer& L, uint8_t* ws, int pi, int lane) {
     const int m = pi / L.G, j = pi - m * L.G;        // m < MP
     uint8_t* grp = ws + L.x_off + staged_group_offset(j, L.pre3[j], L.MP);
     if (L.MP == 2) {                                     // single-token set: the 8-bit form, one task per group
@@ -269,6 +266,21 @@ __global__ void __launch_bounds__(256) gemv_set_stage_kernel(const SetLayer* __r
     if (m == 0 && lane < 16 && lane >= L.M) sxe[lane] = make_float2(0.f, 1.f);   // absent tokens read 0
 }
 
+// One warp per (layer, token, group): fragments and sums of the whole set, once.
+__global__ void __launch_bounds__(256) gemv_set_stage_kernel(const SetLayer* __restrict__ layers, uint8_t* ws, int n_layers, int n_tasks,
+                                                             int n_counters) {
+    stage_clear_counters(ws, n_counters);
+    const int lane = threadIdx.x & 31;
+    const int task = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (task >= n_tasks) return;
+    int lo = 0, hi = n_layers - 1;                       // last layer whose task0 <= task
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (layers[mid].task0 <= task) lo = mid; else hi = mid - 1;
+    }
+    stage_task(layers[lo], ws, task - layers[lo].task0, lane);
+}
+
 // D = A * B with a zero accumulator input: starts an accumulation chain without clearing registers first.
 __device__ __forceinline__ void mma_f16_first(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint2 b) {
     asm volatile(
@@ -277,6 +289,39 @@ __device__ __forceinline__ void mma_f16_first(float (&d)[4], uint32_t a0, uint32
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b.x), "r"(b.y), "f"(0.f));
 }
 
+
+// A consumer warp that has stored its fp32 partial sums of a split row block (n_act tiles from tile0 on, M tokens)
+// counts itself on the row block's counter of this warp.  The warp that counts last sees the other parts and adds all
+// parts in part order, so the result does not depend on which part came last: y = fp16 of that sum.  Out of line: it
+// runs once per item.
+__device__ __noinline__ void finish_parts(const SetParams& p, int layer, int rb, int warp, int lane, int tile0, int n_act, int M, int N) {
+    const SetLayer* L = p.layers + layer;
+    __threadfence();                                    // this lane's partial sums before the count
+    __syncwarp();
+    unsigned int old = 0;
+    if (lane == 0)
+        old = atomicAdd(reinterpret_cast<unsigned int*>(p.ws + kSetOffCounters) + L->cnt0 + rb * kSetConsumers + warp, 1u);
+    old = __shfl_sync(0xffffffffu, old, 0);
+    const int S = L->split;
+    if (static_cast<int>(old) + 1 != S) return;
+    __threadfence();
+    const float* part = reinterpret_cast<const float*>(p.ws + L->part_off);
+    const size_t MN = static_cast<size_t>(M) * N;
+    __half* y = L->y;
+    // 16 * n_act rows x M tokens as pairs of rows: pair i of token m
+    const int pairs = 8 * n_act;
+    for (int i = lane; i < pairs * M; i += 32) {
+        const int m = i / pairs, r = i - m * pairs;
+        const size_t at = static_cast<size_t>(m) * N + 16 * tile0 + 2 * r;
+        float2 sum = __ldcg(reinterpret_cast<const float2*>(part + at));
+        for (int k = 1; k < S; ++k) {
+            const float2 v = __ldcg(reinterpret_cast<const float2*>(part + k * MN + at));
+            sum.x += v.x;
+            sum.y += v.y;
+        }
+        *reinterpret_cast<__half2*>(y + at) = __floats2half2_rn(sum.x, sum.y);
+    }
+}
 
 // Slow path of a consumer's wait, kept out of line so that the loop around it stays small.
 __device__ __noinline__ bool wait_full_slow(uint32_t bar, uint32_t parity, volatile int* abort) {
@@ -315,7 +360,7 @@ __device__ __forceinline__ void consume_one(const SetParams& p, const uint32_t s
     const int4* items4 = reinterpret_cast<const int4*>(p.items);
     int4 it_a = items4[2 * i0], it_b = items4[2 * i0 + 1];       // (layer, rb, N, G), (y, M, counts)
     for (int i = i0; i < i1 && ok; ++i) {
-        const int rb = it_a.y, N = it_a.z, p0 = it_a.w & 0xffff, p1 = it_a.w >> 16, counts = it_b.w;
+        const int layer = it_a.x, rb = it_a.y, N = it_a.z, p0 = it_a.w & 0xffff, p1 = it_a.w >> 16, counts = it_b.w;
         const int G = p1 - p0;                                   // groups of this item
         const unsigned long long yword = (static_cast<unsigned long long>(static_cast<uint32_t>(it_b.y)) << 32) | static_cast<uint32_t>(it_b.x);
         if (i + 1 < i1) {                                        // the next item arrives during this one's groups
@@ -428,6 +473,7 @@ __device__ __forceinline__ void consume_one(const SetParams& p, const uint32_t s
                     else *reinterpret_cast<__half2*>(reinterpret_cast<__half*>(yword) + row) = __floats2half2_rn(acc0, acc2);
                 }
             }
+            if (counts & kItemPartial) finish_parts(p, layer, rb, warp, lane, tile0, n_act, 1, N);
         }
     }
 }
@@ -460,7 +506,7 @@ __device__ __forceinline__ void consume_f16(const SetParams& p, const uint32_t s
     const int4* items4 = reinterpret_cast<const int4*>(p.items);
     int4 it_a = items4[2 * i0], it_b = items4[2 * i0 + 1];       // (layer, rb, N, range), (y, M, counts)
     for (int i = i0; i < i1 && ok; ++i) {
-        const int rb = it_a.y, N = it_a.z, p0 = it_a.w & 0xffff, p1 = it_a.w >> 16, M = it_b.z, counts = it_b.w;
+        const int layer = it_a.x, rb = it_a.y, N = it_a.z, p0 = it_a.w & 0xffff, p1 = it_a.w >> 16, M = it_b.z, counts = it_b.w;
         const unsigned long long yword = (static_cast<unsigned long long>(static_cast<uint32_t>(it_b.y)) << 32) | static_cast<uint32_t>(it_b.x);
         if (i + 1 < i1) {                                        // the next item arrives during this one's groups
             it_a = items4[2 * i + 2];
@@ -586,6 +632,7 @@ __device__ __forceinline__ void consume_f16(const SetParams& p, const uint32_t s
                     }
                 }
             }
+            if (partial) finish_parts(p, layer, rb, warp, lane, tile0, n_act, M, N);
         }
     }
 }
@@ -698,49 +745,35 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
     if (tid == 0 && *abort != 0) atomicOr(reinterpret_cast<unsigned int*>(p.ws), 1u);
 }
 
-// ------------------------------------------------------------------------------------------ split row blocks: the sum of the parts
-// y = fp16(sum over the parts of a layer's fp32 partial outputs, in part order) for the layers whose groups were cut
-// into several items.  Block (bx, l) walks layer l's outputs in steps of the grid's x extent.
-__global__ void __launch_bounds__(256) gemv_set_finish_kernel(const SetLayer* __restrict__ layers, const uint8_t* __restrict__ ws) {
-    const SetLayer& L = layers[blockIdx.y];
-    const int S = L.split;
-    if (S <= 1) return;
-    const size_t pairs = static_cast<size_t>(L.M) * L.N / 2;
-    const float2* part = reinterpret_cast<const float2*>(ws + L.part_off);
-    __half2* y = reinterpret_cast<__half2*>(L.y);
-    for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < pairs; i += static_cast<size_t>(gridDim.x) * blockDim.x) {
-        float2 sum = part[i];
-        for (int k = 1; k < S; ++k) {
-            const float2 v = part[static_cast<size_t>(k) * pairs + i];
-            sum.x += v.x;
-            sum.y += v.y;
-        }
-        y[i] = __floats2half2_rn(sum.x, sum.y);
-    }
-}
-
 // ------------------------------------------------------------------------------------------ one-layer sets planned on the device
-// Plan of a one-layer set, written by a kernel: the descriptor comes by value and the items are (row block, part) pairs
-// dealt to the CTAs in turn, so no host memory is read after the call has returned and the call can be captured in a
-// CUDA graph (slim_mpq_gemv sends its large layers this way).
-__global__ void __launch_bounds__(256) set_single_plan_kernel(const __grid_constant__ SetLayer d, uint8_t* plan, int grid, int n_rb, int sp) {
-    int* item_begin = reinterpret_cast<int*>(plan);
-    SetLayer* dl = reinterpret_cast<SetLayer*>(plan + kSetPlanHeader);
-    SetItem* items = reinterpret_cast<SetItem*>(dl + 1);
-    const int n = n_rb * sp, q = n / grid, r = n % grid;
-    for (int c = threadIdx.x; c <= grid; c += blockDim.x) item_begin[c] = c * q + min(c, r);
-    const uint4* src = reinterpret_cast<const uint4*>(&d);
-    for (int i = threadIdx.x; i < static_cast<int>(sizeof(SetLayer) / 16); i += blockDim.x) reinterpret_cast<uint4*>(dl)[i] = src[i];
-    for (int k = threadIdx.x; k < n; k += blockDim.x) {
-        const int c = k % grid, t = k / grid;                // CTA c takes items c, c + grid, ...
-        const int rb = k / sp, part = k - rb * sp;
-        const int p0 = d.G * part / sp, p1 = d.G * (part + 1) / sp;
-        SetItem it;
-        it.layer = 0; it.rb = rb; it.N = d.N; it.range = p0 | (p1 << 16); it.M = d.M;
-        it.counts = d.count[0] | (d.count[1] << 9) | (d.count[2] << 18) | (sp > 1 ? kItemPartial : 0);
-        it.y = sp > 1 ? reinterpret_cast<__half*>(d.part_off + static_cast<size_t>(part) * d.M * d.N * sizeof(float)) : d.y;
-        items[c * q + min(c, r) + t] = it;
+// Plan and staging of a one-layer set in one kernel: the descriptor comes by value, every warp stages one (token, group)
+// of x, and block 0 also writes the plan: the items are (row block, part) pairs dealt to the CTAs in turn.  No host
+// memory is read after the call has returned, so the call can be captured in a CUDA graph (slim_mpq_gemv sends its
+// large layers this way).
+__global__ void __launch_bounds__(256) set_single_stage_kernel(const __grid_constant__ SetLayer d, uint8_t* plan, uint8_t* ws, int grid,
+                                                               int n_rb, int sp, int n_tasks, int n_counters) {
+    stage_clear_counters(ws, n_counters);
+    if (blockIdx.x == 0) {
+        int* item_begin = reinterpret_cast<int*>(plan);
+        SetLayer* dl = reinterpret_cast<SetLayer*>(plan + kSetPlanHeader);
+        SetItem* items = reinterpret_cast<SetItem*>(dl + 1);
+        const int n = n_rb * sp, q = n / grid, r = n % grid;
+        for (int c = threadIdx.x; c <= grid; c += blockDim.x) item_begin[c] = c * q + min(c, r);
+        const uint4* src = reinterpret_cast<const uint4*>(&d);
+        for (int i = threadIdx.x; i < static_cast<int>(sizeof(SetLayer) / 16); i += blockDim.x) reinterpret_cast<uint4*>(dl)[i] = src[i];
+        for (int k = threadIdx.x; k < n; k += blockDim.x) {
+            const int c = k % grid, t = k / grid;                // CTA c takes items c, c + grid, ...
+            const int rb = k / sp, part = k - rb * sp;
+            const int p0 = d.G * part / sp, p1 = d.G * (part + 1) / sp;
+            SetItem it;
+            it.layer = 0; it.rb = rb; it.N = d.N; it.range = p0 | (p1 << 16); it.M = d.M;
+            it.counts = d.count[0] | (d.count[1] << 9) | (d.count[2] << 18) | (sp > 1 ? kItemPartial : 0);
+            it.y = sp > 1 ? reinterpret_cast<__half*>(d.part_off + static_cast<size_t>(part) * d.M * d.N * sizeof(float)) : d.y;
+            items[c * q + min(c, r) + t] = it;
+        }
     }
+    const int task = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (task < n_tasks) stage_task(d, ws, task, threadIdx.x & 31);
 }
 
 // ------------------------------------------------------------------------------------------ self-test of the bounded wait
@@ -771,6 +804,8 @@ struct SetGeometry {
     int split;                         // parts the groups of every row block are cut into (fewer for layers with few groups)
     size_t smem_bytes;
     long long n_items, n_tasks;
+    int n_counters;                    // arrival counters of the split row blocks: one per (row block, consumer warp)
+    size_t cnt_bytes;                  // their room in the workspace, right after the 256-byte header
     size_t ws_bytes;
 };
 constexpr int kSetMaxSplit = 8;
@@ -831,7 +866,7 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     if (sg->n_items > 0x3fffffff || sg->n_tasks > 0x3fffffff) return SLIM_ERR_UNSUPPORTED;
     sg->nt = sg->mmax <= 8 ? 1 : 2;
     // A set with fewer row blocks than persistent CTAs cuts the groups of every row block into parts (items of their
-    // own, fp32 partial outputs in the workspace, summed in part order by a small kernel afterwards).
+    // own, fp32 partial outputs in the workspace, added in part order by the consumer warp whose part lands last).
     const long long want = static_cast<long long>(set_sm_count()) * kSetCtasPerSm;
     sg->split = 1;
     if (sg->n_items < 2 * want) {
@@ -851,12 +886,21 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     }
     if (sg->split > 1) {
         sg->n_items = 0;
+        long long counters = 0;
         for (int l = 0; l < n_layers; ++l) {
             const slim_layer& L = layers[l];
             const int sp = layer_split(sg->split, L.K / SLIM_GROUP);
-            sg->n_items += static_cast<long long>(sp) * (((L.N >> 4) + tpi - 1) / tpi);
-            if (sp > 1) sg->ws_bytes += align_to(static_cast<size_t>(sp) * L.M * L.N * sizeof(float), 128);
+            const int n_rb = ((L.N >> 4) + tpi - 1) / tpi;
+            sg->n_items += static_cast<long long>(sp) * n_rb;
+            if (sp > 1) {
+                sg->ws_bytes += align_to(static_cast<size_t>(sp) * L.M * L.N * sizeof(float), 128);
+                counters += static_cast<long long>(n_rb) * kSetConsumers;
+            }
         }
+        if (counters > 65535) return SLIM_ERR_UNSUPPORTED;       // cannot happen: a split set has fewer than 2 x grid row blocks
+        sg->n_counters = static_cast<int>(counters);
+        sg->cnt_bytes = align_to(static_cast<size_t>(counters) * sizeof(unsigned int), 256);
+        sg->ws_bytes += sg->cnt_bytes;
     }
     sg->slot_bytes = static_cast<int>(align_to(static_cast<size_t>(slot_off_w(tpi, sg->mpad)) + static_cast<size_t>(tpi) * 256 * sg->bmax, 128));
     // as many CTAs per SM (kSetCtasPerSm at most) as still leaves each a ring of 4 slots
@@ -880,7 +924,7 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
 
 // Device-side descriptor of one layer.
 static void fill_descriptor(const slim_layer& L, const GroupTable& gt, int mpad, int task0, size_t x_off, int split, size_t part_off,
-                            SetLayer* out) {
+                            int cnt0, SetLayer* out) {
     SetLayer& d = *out;
     memset(&d, 0, sizeof d);
     d.x = static_cast<const __half*>(L.x);
@@ -895,6 +939,7 @@ static void fill_descriptor(const slim_layer& L, const GroupTable& gt, int mpad,
     d.split = static_cast<uint8_t>(split);
     d.gshift = static_cast<uint8_t>(gt.gshift);
     d.part_off = part_off;
+    d.cnt0 = static_cast<uint16_t>(cnt0);
     memcpy(d.prefix, gt.prefix, sizeof d.prefix);
     memcpy(d.bits, gt.bits, sizeof d.bits);
     d.pre3[0] = 0;
@@ -949,7 +994,7 @@ static bool route_layout(int M, int N, int K, int g, const uint8_t* bits_host, c
     const int tpi = kSetConsumers * r->sg.tpw;
     r->n_rb = ((N >> 4) + tpi - 1) / tpi;
     r->sp = layer_split(r->sg.split, gt.G);
-    r->plan_off = 256;
+    r->plan_off = kSetOffCounters + r->sg.cnt_bytes;
     r->plan_bytes = set_plan_bytes(1, static_cast<long long>(r->n_rb) * r->sp);
     r->x_off = r->plan_off + align_to(r->plan_bytes, 256);
     r->part_off = r->x_off + layer_ws_bytes(r->sg.mpad, gt);
@@ -964,9 +1009,50 @@ size_t gemv_route_workspace_bytes(int M, int N, int K, int g, const uint8_t* bit
 
 }  // namespace slim
 
-extern "C" int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* workspace, size_t workspace_bytes, void* stream);
-
 namespace slim {
+
+// Checks a launch record and fills the kernel parameters and the dynamic shared memory of the persistent kernel.
+static int set_params(const slim_gemv_set_info* info, const void* plan, void* workspace, size_t workspace_bytes, SetParams* out, size_t* smem_out) {
+    if (info == nullptr || plan == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (info->n_layers < 1 || info->grid < 1 || info->grid > kSetMaxGrid || info->n_slots < 2 ||
+        info->n_slots > kSetMaxSlots || info->slot_bytes < 128 || info->slot_bytes % 128 != 0 ||
+        (info->token_tiles != 1 && info->token_tiles != 2) || info->max_tokens < 1 || info->max_tokens > 8 * info->token_tiles ||
+        info->tiles_per_warp != 2 ||
+        info->max_bits < 1 || info->max_bits > 4 || info->stage_tasks < 1 || info->split < 1 || info->split > kSetMaxSplit ||
+        info->n_counters < 0 || info->n_counters > 65535 || info->n_layers > 65535)
+        return SLIM_ERR_INVALID_ARG;
+    const size_t smem = kSetOffRing + static_cast<size_t>(info->n_slots) * info->slot_bytes;
+    if (smem > 224 * 1024) return SLIM_ERR_INVALID_ARG;
+    if (!aligned16(plan)) return SLIM_ERR_ALIGNMENT;
+    if (workspace == nullptr || workspace_bytes < info->workspace_bytes || workspace_bytes < 256 ||
+        workspace_bytes < kSetOffCounters + static_cast<size_t>(info->n_counters) * sizeof(unsigned int))
+        return SLIM_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return SLIM_ERR_ALIGNMENT;
+    SetParams& prm = *out;
+    memset(&prm, 0, sizeof prm);
+    prm.item_begin = static_cast<const int*>(plan);
+    prm.layers = reinterpret_cast<const SetLayer*>(static_cast<const uint8_t*>(plan) + kSetPlanHeader);
+    prm.items = reinterpret_cast<const SetItem*>(prm.layers + info->n_layers);
+    prm.ws = static_cast<uint8_t*>(workspace);
+    prm.n_layers = info->n_layers;
+    prm.n_slots = info->n_slots;
+    prm.slot_bytes = info->slot_bytes;
+    prm.one = 1;
+    const int tpi = kSetConsumers * info->tiles_per_warp;
+    const int mp = info->max_tokens == 1 ? 2 : 8 * info->token_tiles;
+    if (slot_off_w(tpi, mp) + tpi * 256 * info->max_bits > info->slot_bytes) return SLIM_ERR_INVALID_ARG;
+    *smem_out = smem;
+    return SLIM_OK;
+}
+
+// The persistent kernel of the set in the form its token count asks for.
+static int launch_set_for(const slim_gemv_set_info* info, const SetParams& prm, size_t smem, cudaStream_t s) {
+    const cudaError_t e = info->max_tokens == 1 ? launch_set<1, true, 2>(prm, info->grid, smem, s)
+                        : info->token_tiles == 1 ? launch_set<1, false, 2>(prm, info->grid, smem, s)
+                                                 : launch_set<2, false, 2>(prm, info->grid, smem, s);
+    SLIM_CUDA_TRY(e);
+    return SLIM_OK;
+}
 
 // Returns SLIM_OK after enqueueing the layer through the layer-set kernels, a negative status on failure, or 1 if this
 // shape or workspace is not routed (the caller then takes the per-layer kernel).
@@ -978,12 +1064,10 @@ int gemv_route(const void* x, const void* packed, const uint8_t* bits_host, cons
     memset(&L, 0, sizeof L);
     L.x = x; L.packed = packed; L.scales = scales; L.zeros = zeros; L.y = y; L.bits_host = bits_host; L.M = M; L.N = N; L.K = K;
     SetLayer d;
-    fill_descriptor(L, gt, r.sg.mpad, 0, r.x_off, r.sp, r.part_off, &d);
+    fill_descriptor(L, gt, r.sg.mpad, 0, r.x_off, r.sp, r.part_off, 0, &d);
     uint8_t* plan = static_cast<uint8_t*>(workspace) + r.plan_off;
     const long long n_items = static_cast<long long>(r.n_rb) * r.sp;
     const int grid = static_cast<int>(n_items < r.sg.grid ? n_items : r.sg.grid);
-    set_single_plan_kernel<<<1, 256, 0, stream>>>(d, plan, grid, r.n_rb, r.sp);
-    SLIM_CUDA_TRY(cudaGetLastError());
     slim_gemv_set_info info;
     memset(&info, 0, sizeof info);
     info.n_layers = 1;
@@ -997,9 +1081,16 @@ int gemv_route(const void* x, const void* packed, const uint8_t* bits_host, cons
     info.max_tokens = r.sg.mmax;
     info.tiles_per_warp = r.sg.tpw;
     info.split = r.sg.split;
+    info.n_counters = r.sg.n_counters;
     info.plan_bytes = r.plan_bytes;
     info.workspace_bytes = r.total;
-    return slim_mpq_gemv_set(&info, plan, workspace, workspace_bytes, stream);
+    SetParams prm;
+    size_t smem = 0;
+    const int st = set_params(&info, plan, workspace, workspace_bytes, &prm, &smem);
+    if (st != SLIM_OK) return st;
+    set_single_stage_kernel<<<(info.stage_tasks + 7) / 8, 256, 0, stream>>>(d, plan, prm.ws, grid, r.n_rb, r.sp, info.stage_tasks, info.n_counters);
+    SLIM_CUDA_TRY(cudaGetLastError());
+    return launch_set_for(&info, prm, smem, stream);
 }
 
 }  // namespace slim
@@ -1044,12 +1135,13 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
     items.reserve(static_cast<size_t>(sg.n_items));
     cost.reserve(static_cast<size_t>(sg.n_items));
     const int tpi = slim::kSetConsumers * sg.tpw;
-    int task = 0;
-    size_t ws_off = 256;
-    // workspace: the staged activations of all layers, then the fp32 partial outputs of the layers that are split
+    int task = 0, cnt0 = 0;
+    size_t ws_off = slim::kSetOffCounters + sg.cnt_bytes;
+    // workspace: header, the arrival counters of the split row blocks, the staged activations of all layers, then the
+    // fp32 partial outputs of the layers that are split
     std::vector<size_t> part_off(static_cast<size_t>(n_layers), 0), x_off(static_cast<size_t>(n_layers), 0);
     {
-        size_t off = 256;
+        size_t off = ws_off;
         for (int l = 0; l < n_layers; ++l) {
             slim::GroupTable gt;
             slim::make_group_table(layers_host[l].N, layers_host[l].K, g, layers_host[l].bits_host, &gt);
@@ -1076,11 +1168,12 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
             if (E.x == L.x && E.M == L.M && E.K == L.K && memcmp(E.bits_host, L.bits_host, static_cast<size_t>(L.K / g)) == 0) same = e;
         }
         x_off[l] = same >= 0 ? x_off[same] : ws_off;
-        slim::fill_descriptor(L, gt, sg.mpad, task, x_off[l], sp, part_off[l], &d);
+        slim::fill_descriptor(L, gt, sg.mpad, task, x_off[l], sp, part_off[l], cnt0, &d);
         ws_off += slim::layer_ws_bytes(sg.mpad, gt);
         SLIM_CUDA_TRY(cudaMemcpyAsync(plan_dev + slim::kSetPlanHeader + static_cast<size_t>(l) * sizeof d, &d, sizeof d,
                                       cudaMemcpyHostToDevice, s));
         const int n_rb = ((L.N >> 4) + tpi - 1) / tpi;
+        if (sp > 1) cnt0 += n_rb * slim::kSetConsumers;
         for (int rb = 0; rb < n_rb; ++rb) {
             const int th = (L.N >> 4) - tpi * rb;
             for (int part = 0; part < sp; ++part) {
@@ -1141,6 +1234,7 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
     info->max_tokens = sg.mmax;
     info->tiles_per_warp = sg.tpw;
     info->split = sg.split;
+    info->n_counters = sg.n_counters;
     info->plan_bytes = slim::set_plan_bytes(n_layers, n_items);
     info->workspace_bytes = sg.ws_bytes;
     } catch (const std::exception&) {
@@ -1161,46 +1255,14 @@ int slim_selftest_wait_timeout(void* workspace, size_t workspace_bytes, unsigned
 }
 
 int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* workspace, size_t workspace_bytes, void* stream) {
-    if (info == nullptr || plan == nullptr) return SLIM_ERR_INVALID_ARG;
-    if (info->n_layers < 1 || info->grid < 1 || info->grid > slim::kSetMaxGrid || info->n_slots < 2 ||
-        info->n_slots > slim::kSetMaxSlots || info->slot_bytes < 128 || info->slot_bytes % 128 != 0 ||
-        (info->token_tiles != 1 && info->token_tiles != 2) || info->max_tokens < 1 || info->max_tokens > 8 * info->token_tiles ||
-        info->tiles_per_warp != 2 ||
-        info->max_bits < 1 || info->max_bits > 4 || info->stage_tasks < 1 || info->split < 1 || info->split > slim::kSetMaxSplit ||
-        info->n_layers > 65535)
-        return SLIM_ERR_INVALID_ARG;
-    const size_t smem = slim::kSetOffRing + static_cast<size_t>(info->n_slots) * info->slot_bytes;
-    if (smem > 224 * 1024) return SLIM_ERR_INVALID_ARG;
-    if (!slim::aligned16(plan)) return SLIM_ERR_ALIGNMENT;
-    if (workspace == nullptr || workspace_bytes < info->workspace_bytes || workspace_bytes < 256) return SLIM_ERR_WORKSPACE;
-    if (!slim::aligned16(workspace)) return SLIM_ERR_ALIGNMENT;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-
     slim::SetParams prm;
-    memset(&prm, 0, sizeof prm);
-    prm.item_begin = static_cast<const int*>(plan);
-    prm.layers = reinterpret_cast<const slim::SetLayer*>(static_cast<const uint8_t*>(plan) + slim::kSetPlanHeader);
-    prm.items = reinterpret_cast<const slim::SetItem*>(prm.layers + info->n_layers);
-    prm.ws = static_cast<uint8_t*>(workspace);
-    prm.n_layers = info->n_layers;
-    prm.n_slots = info->n_slots;
-    prm.slot_bytes = info->slot_bytes;
-    prm.one = 1;
-    const int tpi = slim::kSetConsumers * info->tiles_per_warp;
-    const int mp = info->max_tokens == 1 ? 2 : 8 * info->token_tiles;
-    if (slim::slot_off_w(tpi, mp) + tpi * 256 * info->max_bits > info->slot_bytes) return SLIM_ERR_INVALID_ARG;
-
-    slim::gemv_set_stage_kernel<<<(info->stage_tasks + 7) / 8, 256, 0, s>>>(prm.layers, prm.ws, info->n_layers, info->stage_tasks);
+    size_t smem = 0;
+    const int st = slim::set_params(info, plan, workspace, workspace_bytes, &prm, &smem);
+    if (st != SLIM_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    slim::gemv_set_stage_kernel<<<(info->stage_tasks + 7) / 8, 256, 0, s>>>(prm.layers, prm.ws, info->n_layers, info->stage_tasks, info->n_counters);
     SLIM_CUDA_TRY(cudaGetLastError());
-    const cudaError_t e = info->max_tokens == 1 ? slim::launch_set<1, true, 2>(prm, info->grid, smem, s)
-                        : info->token_tiles == 1 ? slim::launch_set<1, false, 2>(prm, info->grid, smem, s)
-                                                 : slim::launch_set<2, false, 2>(prm, info->grid, smem, s);
-    SLIM_CUDA_TRY(e);
-    if (info->split > 1) {
-        slim::gemv_set_finish_kernel<<<dim3(32, static_cast<unsigned>(info->n_layers)), 256, 0, s>>>(prm.layers, prm.ws);
-        SLIM_CUDA_TRY(cudaGetLastError());
-    }
-    return SLIM_OK;
+    return slim::launch_set_for(info, prm, smem, s);
 }
 
 }  // extern "C"
