@@ -146,3 +146,43 @@ def test_salience_and_bit_budget(g):
     assert np.isclose(S[2], manual, rtol=1e-12)
     bits = orc.allocate_bits(S, 2)
     assert int(bits.astype(np.int64).sum()) * g == 2 * K          # the average-bit budget holds exactly
+
+
+@pytest.mark.parametrize("g", (32, 64, 256))
+def test_sqc_against_the_scalar_restatement_at_other_group_sizes(g):
+    """Function SQC of Algorithm 2 at group size g: the 3-sigma mask, the tau grid and the two-term loss are taken
+    per (row, group of g columns); a scalar restatement of the algorithm must pick the same tau, step, zero point
+    and codes."""
+    from tests.test_oracle_sqc import _brute_sqc_row
+    rng = np.random.default_rng(300 + g)
+    N, K = 2, 2 * g
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float16)
+    W[0, 3] = np.float16(0.25)                       # an outlier for the mask
+    W[1, g:] = -np.abs(W[1, g:])                     # an all-negative group
+    bits = np.array([2, 3], np.uint8)
+    codes, scales, zeros, ti, loss, loss_s = orc.quantize_sqc(W, bits, g, lam=0.1, n=10)
+    for r in range(N):
+        for j in range(2):
+            w = [float(v) for v in W[r, g * j:g * (j + 1)]]
+            L, i, delta, z, q, Ls = _brute_sqc_row(w, int(bits[j]), lam=0.1, n=10)
+            assert ti[j, r] == i and float(scales[j, r]) == delta and float(zeros[j, r]) == z
+            assert list(codes[r, g * j:g * (j + 1)]) == q
+            assert loss[j, r] == L and loss_s[j, r] == Ls
+
+
+@pytest.mark.parametrize("g", SIZES)
+def test_sign_alpha_one_bit_groups_at_every_group_size(g):
+    """Eq. 2 per group of g columns: codes are the signs, s (q - z) = +- mean |w| of the group."""
+    rng = np.random.default_rng(500 + g)
+    N, K = 4, 3 * g
+    W = rng.normal(0, 0.02, (N, K)).astype(np.float16)
+    bits = np.array([1, 2, 1], np.uint8)
+    codes, scales, zeros = orc.quantize_minmax_sign1(W, bits, g)
+    c2, s2, z2 = orc.quantize_minmax(W, bits, g)
+    assert (codes[:, g:2 * g] == c2[:, g:2 * g]).all() and (scales[1] == s2[1]).all()      # the 2-bit group is Eq. 1
+    for j in (0, 2):
+        w = W[:, g * j:g * (j + 1)].astype(np.float64)
+        assert ((codes[:, g * j:g * (j + 1)] == 1) == (w >= 0)).all()
+        alpha = np.abs(w).mean(axis=1)
+        assert (zeros[j] == np.float16(0.5)).all()
+        assert np.array_equal(scales[j], (2 * alpha).astype(np.float16))
