@@ -783,8 +783,8 @@ def single_layer_entry(layer, device, timer, copies=64):
 
 def group_size_entries(device, timer):
     """One 4096 x 4096 layer, avg 2-bit, M = 1, at the group sizes of the paper's group-size ablation: 64 distinct copies
-    (> L2) per step through slim_mpq_gemv.  Throughput does not depend on the values, so codes, scales and zero points
-    are drawn directly (seeded), with the 25 / 50 / 25 % mix of 1 / 2 / 3-bit groups of the other workloads."""
+    (> L2) per step through slim_mpq_gemv, each made on the device from a seeded weight at that group size (salience ->
+    bit allocation -> Eq. 1 -> packing)."""
     import torch
     from paper_2405_14917_b200 import binding as slim
     N = K = 4096
@@ -793,18 +793,11 @@ def group_size_entries(device, timer):
     gen = torch.Generator(device=device)
     gen.manual_seed(32)
     for g in (32, 64, 128, 256, 512):
-        G = K // g
-        order = torch.randperm(G, generator=gen, device=device).cpu().numpy()
-        bits = np.full(G, 2, dtype=np.uint8)
-        bits[order[:G // 4]] = 3
-        bits[order[G // 4:2 * (G // 4)]] = 1
         layers = []
-        for _ in range(copies):
-            codes = torch.cat([torch.randint(0, 2 ** int(b), (N, g), generator=gen, device=device, dtype=torch.uint8) for b in bits], dim=1)
-            scales = (torch.rand((G, N), generator=gen, device=device) * 0.02 + 0.001).half()
-            zeros = torch.cat([torch.randint(0, 2 ** int(b), (1, N), generator=gen, device=device) for b in bits]).half()
-            layers.append(slim.QuantLinear(slim.pack_weights(codes.contiguous(), bits, g=g), bits, scales, zeros, N, K, g))
-            del codes
+        for i in range(copies):
+            W, a = wl.make_weight_and_norms_device((32, g, i), N, K, device)
+            layers.append(slim.QuantLinear.from_weight(W, a, 2, g=g))
+            del W, a
         M = 1
         x = torch.randn(M, K, generator=gen, device=device).half()
         ys = [torch.empty(M, N, dtype=torch.float16, device=device) for _ in layers]
@@ -829,7 +822,7 @@ def group_size_entries(device, timer):
                     "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
                                  "avg_launch_us": 1e3 * ms / copies, "algorithmic_bytes_per_launch": alg / copies},
                     "config": {"workload": f"single-4096x4096-avg2-m1-g{g}", "g": g, "layers": copies, "algorithmic_bytes_per_step": alg,
-                               "data": "codes, scales and zero points drawn directly (seeded)"}})
+                               "data": "synthetic weights quantised on the device at this group size"}})
         del layers, graph
         torch.cuda.empty_cache()
     return out

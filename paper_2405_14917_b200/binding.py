@@ -218,11 +218,11 @@ def mpq_gemm_static(x, packed, bits, scales, zeros, N: int, out: torch.Tensor, s
     return out
 
 
-def group_salience(W: torch.Tensor, act_norm: torch.Tensor) -> torch.Tensor:
+def group_salience(W: torch.Tensor, act_norm: torch.Tensor, g: int = GROUP) -> torch.Tensor:
     N, K = W.shape
-    out = torch.empty(K // GROUP, dtype=torch.float64, device=W.device)
+    out = torch.empty(K // g, dtype=torch.float64, device=W.device)
     _check("slim_group_salience", lib().slim_group_salience(_dev(W, torch.float16, "W"), _dev(act_norm, torch.float32, "act_norm"),
-                                                            _dev(out, torch.float64, "salience"), N, K, GROUP, _stream(W)))
+                                                            _dev(out, torch.float64, "salience"), N, K, g, _stream(W)))
     return out
 
 
@@ -233,45 +233,46 @@ def allocate_bits(salience, avg_bits: int, p: int = -1) -> np.ndarray:
     return out
 
 
-def quantize_minmax(W: torch.Tensor, bits, one_bit: str = "minmax"):
+def quantize_minmax(W: torch.Tensor, bits, one_bit: str = "minmax", g: int = GROUP):
     """Eq. 1 per (row, group); one_bit="sign_alpha" binarises the one-bit groups with Eq. 2 instead."""
     if one_bit not in ("minmax", "sign_alpha"):
         raise ValueError("one_bit must be 'minmax' or 'sign_alpha'")
     fn_name = "slim_quantize_minmax" if one_bit == "minmax" else "slim_quantize_minmax_sign1"
     b = _bits(bits)
     N, K = W.shape
-    G = K // GROUP
+    G = K // g
     codes = torch.empty((N, K), dtype=torch.uint8, device=W.device)
     scales = torch.empty((G, N), dtype=torch.float16, device=W.device)
     zeros = torch.empty((G, N), dtype=torch.float16, device=W.device)
     _check(fn_name, getattr(lib(), fn_name)(_dev(W, torch.float16, "W"), _bp(b), _dev(codes, torch.uint8, "codes"),
                                             _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
-                                            N, K, GROUP, _stream(W)))
+                                            N, K, g, _stream(W)))
     return codes, scales, zeros
 
 
-def quantize_minmax_groups(W: torch.Tensor, bits, groups, codes: torch.Tensor, scales: torch.Tensor, zeros: torch.Tensor) -> None:
+def quantize_minmax_groups(W: torch.Tensor, bits, groups, codes: torch.Tensor, scales: torch.Tensor, zeros: torch.Tensor,
+                           g: int = GROUP) -> None:
     """Re-quantises (Eq. 1) only the listed groups under `bits`, in place in codes / scales / zeros."""
     b = _bits(bits)
     gl = np.ascontiguousarray(np.asarray(groups), dtype=np.int32)
     N, K = W.shape
     _check("slim_quantize_minmax_groups", lib().slim_quantize_minmax_groups(
         _dev(W, torch.float16, "W"), _bp(b), _dev(codes, torch.uint8, "codes"), _dev(scales, torch.float16, "scales"),
-        _dev(zeros, torch.float16, "zeros"), N, K, GROUP, gl.ctypes.data, int(gl.size), _stream(W)))
+        _dev(zeros, torch.float16, "zeros"), N, K, g, gl.ctypes.data, int(gl.size), _stream(W)))
 
 
-def quantize_sqc(W: torch.Tensor, bits, lam: float = 0.1, n: int = 50):
+def quantize_sqc(W: torch.Tensor, bits, lam: float = 0.1, n: int = 50, g: int = GROUP):
     """SQC line search (Algorithm 2) on the device.  Returns codes, scales, zeros, tau index."""
     b = _bits(bits)
     N, K = W.shape
-    G = K // GROUP
+    G = K // g
     codes = torch.empty((N, K), dtype=torch.uint8, device=W.device)
     scales = torch.empty((G, N), dtype=torch.float16, device=W.device)
     zeros = torch.empty((G, N), dtype=torch.float16, device=W.device)
     tau = torch.empty((G, N), dtype=torch.int32, device=W.device)
     _check("slim_quantize_sqc", lib().slim_quantize_sqc(_dev(W, torch.float16, "W"), _bp(b), _dev(codes, torch.uint8, "codes"),
                                                         _dev(scales, torch.float16, "scales"), _dev(zeros, torch.float16, "zeros"),
-                                                        _dev(tau, torch.int32, "tau_index"), N, K, GROUP, float(lam), int(n), _stream(W)))
+                                                        _dev(tau, torch.int32, "tau_index"), N, K, g, float(lam), int(n), _stream(W)))
     return codes, scales, zeros, tau
 
 
@@ -432,13 +433,13 @@ class QuantLinear:
         self.packed, self.bits, self.scales, self.zeros, self.N, self.K, self.g = packed, _bits(bits), scales, zeros, N, K, g
 
     @classmethod
-    def from_weight(cls, W: torch.Tensor, act_norm: torch.Tensor, avg_bits: int, p: int = -1) -> "QuantLinear":
+    def from_weight(cls, W: torch.Tensor, act_norm: torch.Tensor, avg_bits: int, p: int = -1, g: int = GROUP) -> "QuantLinear":
         """Salience -> bit allocation -> Eq. 1 quantizer -> packing, all on the device."""
         N, K = W.shape
-        sal = group_salience(W, act_norm).cpu().numpy()
+        sal = group_salience(W, act_norm, g).cpu().numpy()
         bits = allocate_bits(sal, avg_bits, p)
-        codes, scales, zeros = quantize_minmax(W, bits)
-        return cls(pack_weights(codes, bits), bits, scales, zeros, N, K)
+        codes, scales, zeros = quantize_minmax(W, bits, g=g)
+        return cls(pack_weights(codes, bits, g=g), bits, scales, zeros, N, K, g)
 
     def workspace_bytes(self, M: int) -> int:
         return workspace_bytes(M, self.N, self.K, self.bits, self.g)

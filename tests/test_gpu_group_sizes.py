@@ -147,6 +147,56 @@ def test_full_size_layer_with_large_groups(g):
         check_output(y.cpu().numpy()[:, rows], orc.linear_rows_f64(x, L["codes"], L["scales"], L["zeros"], rows, g), f"g={g} M={M}")
 
 
+def _same_bits(a, b):
+    return (a.cpu().numpy().view(np.uint16) == b.view(np.uint16)).all()
+
+
+@pytest.mark.parametrize("g", ALL)
+@pytest.mark.parametrize("N,K", [(48, 1024), (272, 4096)])
+def test_salience_and_quantizers_match_the_oracle_bit_for_bit(g, N, K):
+    """Group salience, the Eq. 1 quantizer, its Eq. 2 one-bit form and SQC (Algorithm 2) at group size g."""
+    slim = _slim()
+    sd = wl.layer_seed("test", f"quant-group-size-{g}-{N}x{K}", 0)
+    W = wl.make_weight(sd, N, K)
+    a = wl.make_act_norms(sd, K)
+    Wd = torch.from_numpy(W).cuda()
+    sal_ref = orc.group_salience(W, a, g)
+    sal = slim.group_salience(Wd, torch.from_numpy(a).cuda(), g).cpu().numpy()
+    assert sal.shape == (K // g,) and np.allclose(sal, sal_ref, rtol=1e-12, atol=0)
+    rng = np.random.default_rng(g + N)
+    bits = rng.integers(1, 5, K // g).astype(np.uint8)
+    for one_bit, ref in (("minmax", orc.quantize_minmax), ("sign_alpha", orc.quantize_minmax_sign1)):
+        codes, scales, zeros = slim.quantize_minmax(Wd, bits, one_bit=one_bit, g=g)
+        c_ref, s_ref, z_ref = ref(W, bits, g)
+        assert _same_bits(scales, s_ref) and _same_bits(zeros, z_ref), one_bit
+        assert (codes.cpu().numpy() == c_ref).all(), one_bit
+    rows = 16 if K > 1024 else N                  # the oracle's tau search is slow: a slice of the rows
+    codes, scales, zeros, tau = slim.quantize_sqc(Wd[:rows].contiguous(), bits, lam=0.1, n=20, g=g)
+    c_ref, s_ref, z_ref, t_ref, _, _ = orc.quantize_sqc(W[:rows], bits, g, lam=0.1, n=20)
+    assert (tau.cpu().numpy() == t_ref).all()
+    assert _same_bits(scales, s_ref) and _same_bits(zeros, z_ref) and (codes.cpu().numpy() == c_ref).all()
+
+
+@pytest.mark.parametrize("g", ALL)
+def test_layer_built_on_the_device_from_a_weight(g):
+    """Salience -> bit allocation -> Eq. 1 -> packing on the device at group size g, then one decode call: the result
+    is the oracle's layer of the same bit map."""
+    slim = _slim()
+    N, K, M = 256, 2048, 3
+    sd = wl.layer_seed("test", f"from-weight-{g}", 0)
+    W = wl.make_weight(sd, N, K)
+    a = wl.make_act_norms(sd, K)
+    x = wl.make_x(sd, M, K)
+    L = slim.QuantLinear.from_weight(torch.from_numpy(W).cuda(), torch.from_numpy(a).cuda(), 2, g=g)
+    assert L.g == g and int(L.bits.astype(int).sum()) * g == 2 * K
+    codes, scales, zeros = orc.quantize_minmax(W, L.bits, g)
+    assert (L.packed.cpu().numpy() == orc.pack(codes, L.bits, g)).all()
+    ws = slim.new_workspace(M, N, K, L.bits, g=g)
+    y = L.forward(torch.from_numpy(x).cuda(), ws)
+    slim.workspace_status(ws)
+    check_output(y.cpu().numpy(), orc.linear_f64(x, codes, scales, zeros, g), f"g={g}")
+
+
 def test_unsupported_group_sizes_are_statuses():
     slim = _slim()
     bits = np.full(8, 2, dtype=np.uint8)
