@@ -40,17 +40,17 @@ FALLBACK_TENSOR_TFLOPS = 1400.0
 # dram__bytes_write.sum), keyed by the sha256 of the kernel source it was taken from.  A kernel
 # that has changed since reports null.
 NCU_TRAFFIC = {
-    # layer-set kernel, 4 blocks of the LLaMA-7B sweep (28 layers, avg 2-bit, M = 1): 228,637,952 B read +
-    # 4,588,800 B written per launch (algorithmic 228,297,816 B); scaled to the full sweep by the algorithmic bytes
+    # layer-set kernel, 4 blocks of the LLaMA-7B sweep (28 layers, avg 2-bit, M = 1): 228,647,680 B read +
+    # 4,347,392 B written per launch (algorithmic 228,297,816 B); scaled to the full sweep by the algorithmic bytes
     # (the traffic is the packed data read once, so it grows in proportion)
-    "8cfdeff70d76853300d9a46b806c867f18cad01c2b5297166eb10983046d9c5d": {"layer": "4 blocks", "traffic_bytes": 233226752, "algorithmic_bytes": 228297816},
+    "f44ab8781c759ebcbd6e82bd44590508fffc816de54eaf735911b3cd95707a47": {"layer": "4 blocks", "traffic_bytes": 232995072, "algorithmic_bytes": 228297816},
 }
 
 
 # DRAM bytes (read + written) of the 14 gemm_kernel launches of one step of llama13b-prefill-avg3-m2048, from one ncu
 # capture of dram__bytes_read.sum and dram__bytes_write.sum; keyed by the SHA-256 of slim_gemm.cu at capture time
 NCU_TRAFFIC_GEMM = {
-    "1a98f6bdbcf5c7c1c57790e2a1ed836e1474feb538dcafefdc70f951cd97623b": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1119355392 + 232290560},
+    "5fd2ba9fc66a0002d80a79c938e81c8775052fcd9e7b4f9781ec9ffa2f9dccb0": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1054245120 + 218284032},
 }
 
 
