@@ -3,6 +3,7 @@ itself: a library KL, closed forms, invariances, a scalar brute force and constr
 import math
 
 import numpy as np
+import pytest
 import scipy.special
 import scipy.stats
 
@@ -66,14 +67,14 @@ def test_budget_and_double_pointer_shape():
         assert errs[p_star] == min(errs) and all(e > errs[p_star] for e in errs[:p_star])   # first minimum
 
 
-def _scalar_candidate_error(W, x, bits):
+def _scalar_candidate_error(W, x, bits, g=128):
     """Error of one bit map, element by element with Python floats: Eq. 1 per (row, group), output, softmax, KL."""
     N, K = W.shape
     M = x.shape[0]
     What = [[0.0] * K for _ in range(N)]
     for n in range(N):
         for j, b in enumerate(bits):
-            w = [float(W[n, k]) for k in range(128 * j, 128 * j + 128)]
+            w = [float(W[n, k]) for k in range(g * j, g * j + g)]
             lo, hi, levels = min(min(w), 0.0), max(max(w), 0.0), 2 ** int(b) - 1
             s = float(np.float16((hi - lo) / levels))
             if s == 0.0:
@@ -81,7 +82,7 @@ def _scalar_candidate_error(W, x, bits):
             z = min(max(-float(np.rint(lo / s)), 0.0), levels)
             for i, v in enumerate(w):
                 q = min(max(float(np.rint(v / s)) + z, 0.0), levels)
-                What[n][128 * j + i] = s * (q - z)
+                What[n][g * j + i] = s * (q - z)
     total = 0.0
     for t in range(M):
         yf = [sum(float(x[t, k]) * float(W[n, k]) for k in range(K)) for n in range(N)]
@@ -97,6 +98,19 @@ def test_search_against_scalar_brute_force():
     p_star, bits, errs = orc.sba_search(W, x, a, 2)
     S = orc.group_salience(W, a)
     want = [_scalar_candidate_error(W, x, orc.allocate_bits(S, 2, p)) for p in range(3)]
+    for e, w in zip(errs, want):
+        assert abs(e - w) <= 1e-9 * max(w, 1e-12)
+    assert p_star == min(range(3), key=lambda p: (want[p], p))
+
+
+@pytest.mark.parametrize("g", [32, 64, 256])
+def test_search_against_scalar_brute_force_at_other_group_sizes(g):
+    """The search ranks, quantises and scores groups of g columns (the group-size ablation of the appendix)."""
+    W, x, a = _layer(3, 4 * g, 2, name=f"sba-brute-g{g}")
+    p_star, bits, errs = orc.sba_search(W, x, a, 2, g=g)
+    S = orc.group_salience(W, a, g)
+    assert len(bits) == 4 and len(errs) == 3
+    want = [_scalar_candidate_error(W, x, orc.allocate_bits(S, 2, p), g) for p in range(3)]
     for e, w in zip(errs, want):
         assert abs(e - w) <= 1e-9 * max(w, 1e-12)
     assert p_star == min(range(3), key=lambda p: (want[p], p))
