@@ -302,19 +302,19 @@ def sba_workspace_bytes(M: int, N: int, K: int, avg_bits: int, g: int = GROUP) -
 
 
 def sba_search(W: torch.Tensor, x: torch.Tensor, act_norm: torch.Tensor, avg_bits: int, include_uniform: bool = True,
-               workspace: torch.Tensor | None = None):
+               workspace: torch.Tensor | None = None, g: int = GROUP):
     """Salience-Determined Bit Allocation search (func SBA of Algorithm 2) on the device.
     Returns (p_star, bits[G] (numpy), errors (numpy, one per candidate p))."""
     N, K = W.shape
     M = x.shape[0]
-    G = K // GROUP
+    G = K // g
     if workspace is None:
-        workspace = torch.empty(sba_workspace_bytes(M, N, K, avg_bits), dtype=torch.uint8, device=W.device)
+        workspace = torch.empty(sba_workspace_bytes(M, N, K, avg_bits, g), dtype=torch.uint8, device=W.device)
     p_star = ctypes.c_int(-1)
     bits = np.zeros(G, dtype=np.uint8)
     errors = np.zeros(G // 2 + 1 - (0 if include_uniform else 1), dtype=np.float64)
     _check("slim_sba_search", lib().slim_sba_search(_dev(W, torch.float16, "W"), _dev(x, torch.float16, "x"),
-                                                    _dev(act_norm, torch.float32, "act_norm"), M, N, K, GROUP, avg_bits,
+                                                    _dev(act_norm, torch.float32, "act_norm"), M, N, K, g, avg_bits,
                                                     1 if include_uniform else 0, _dev(workspace, torch.uint8, "workspace"),
                                                     workspace.numel(), ctypes.addressof(p_star), bits.ctypes.data,
                                                     errors.ctypes.data, _stream(W)))

@@ -130,7 +130,7 @@ __device__ __forceinline__ unsigned short double_to_half_bits_rn(double v) {
 // Groups a launch of the quantizer is restricted to (n = 0: all groups).
 struct GroupSubset {
     int n;
-    uint8_t idx[SLIM_MAX_GROUPS];
+    uint16_t idx[kQuantMaxGroups];
 };
 
 // rint(w / s) for fp16-exact w and s > 0 without a division per weight: t = w * (1/s) is within a few
@@ -257,12 +257,11 @@ static int quantize_minmax_impl(const void* W, const uint8_t* bits_host, uint8_t
     slim::GroupSubset sub;
     memset(&sub, 0, sizeof sub);
     if (groups_host != nullptr) {
-        if (gb.G > SLIM_MAX_GROUPS) return SLIM_ERR_UNSUPPORTED;     // the subset form lists at most 256 groups
         if (n_groups < 0 || n_groups > gb.G) return SLIM_ERR_INVALID_ARG;
         if (n_groups == 0) return SLIM_OK;
         for (int i = 0; i < n_groups; ++i) {
             if (groups_host[i] < 0 || groups_host[i] >= gb.G) return SLIM_ERR_INVALID_ARG;
-            sub.idx[i] = static_cast<uint8_t>(groups_host[i]);
+            sub.idx[i] = static_cast<uint16_t>(groups_host[i]);
         }
         sub.n = n_groups;
     }

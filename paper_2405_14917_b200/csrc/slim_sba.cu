@@ -126,11 +126,14 @@ struct SbaLayout {
 };
 static size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 
+constexpr int kSbaMaxGroups = 1024;       // K <= 32768 in groups of 32 columns
+
 static int sba_layout(int M, int N, int K, int g, int avg_bits, SbaLayout* lay) {
     if (M < 1 || N < 16 || K < SLIM_GROUP || avg_bits < 2 || avg_bits > 3) return SLIM_ERR_INVALID_ARG;
-    if (g != SLIM_GROUP || K % SLIM_GROUP != 0 || N % 16 != 0 || K / SLIM_GROUP > SLIM_MAX_GROUPS) return SLIM_ERR_UNSUPPORTED;
-    const int G = K / SLIM_GROUP;
-    uint8_t widest[SLIM_MAX_GROUPS];
+    if (g != 32 && g != 64 && g != 128 && g != 256 && g != 512) return SLIM_ERR_UNSUPPORTED;
+    if (K % g != 0 || K % SLIM_GROUP != 0 || N % 16 != 0 || K / SLIM_GROUP > SLIM_MAX_GROUPS) return SLIM_ERR_UNSUPPORTED;
+    const int G = K / g;
+    uint8_t widest[kSbaMaxGroups];
     for (int j = 0; j < G; ++j) widest[j] = 3;      // 3-bit groups have two slices: the largest staging area of any map
     size_t need = 0;
     const int st = slim_workspace_bytes(M, N, K, g, widest, &need);     // every candidate map needs at most this
@@ -198,12 +201,12 @@ int slim_sba_search(const void* W, const void* x, const float* act_norm, int M, 
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SLIM_ERR_ALIGNMENT;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    const int G = K / SLIM_GROUP;
+    const int G = K / g;
     const int first = include_uniform ? 0 : 1;
     if (first > G / 2) return SLIM_ERR_INVALID_ARG;                       // a single group has only the uniform map
 
     // salience and its ranking (host: G numbers)
-    double sal[SLIM_MAX_GROUPS];
+    double sal[slim::kSbaMaxGroups];
     double* sal_dev = reinterpret_cast<double*>(ws + lay.salience);
     st = slim_group_salience(W, act_norm, sal_dev, N, K, g, stream);
     if (st != SLIM_OK) return st;
@@ -223,7 +226,7 @@ int slim_sba_search(const void* W, const void* x, const float* act_norm, int M, 
     void* packed = ws + lay.packed;
     void* y_q = ws + lay.y_q;
     double* kl = reinterpret_cast<double*>(ws + lay.kl);
-    uint8_t bits[SLIM_MAX_GROUPS], prev[SLIM_MAX_GROUPS];
+    uint8_t bits[slim::kSbaMaxGroups], prev[slim::kSbaMaxGroups];
     for (int p = first; p <= G / 2; ++p) {
         st = slim_allocate_bits(sal, G, avg_bits, p, bits);
         if (st != SLIM_OK) return st;
@@ -232,7 +235,7 @@ int slim_sba_search(const void* W, const void* x, const float* act_norm, int M, 
         } else {
             // consecutive candidates differ in the two groups the double pointer has just passed: only those
             // are quantised again, the codes, scales and zeros of all other groups stay
-            int changed[SLIM_MAX_GROUPS], n_changed = 0;
+            int changed[slim::kSbaMaxGroups], n_changed = 0;
             for (int j = 0; j < G; ++j)
                 if (bits[j] != prev[j]) changed[n_changed++] = j;
             st = slim_quantize_minmax_groups(W, bits, codes, scales, zeros, N, K, g, changed, n_changed, stream);

@@ -50,11 +50,11 @@ def test_softmax_kl_against_the_oracle():
     assert np.abs(z).max() <= 1e-15
 
 
-def _check_search(W, x, a, avg, include_uniform=True):
+def _check_search(W, x, a, avg, include_uniform=True, g=128):
     slim = _slim()
     p_star, bits, errs = slim.sba_search(torch.from_numpy(W).cuda(), torch.from_numpy(x).cuda(),
-                                         torch.from_numpy(a.astype(np.float32)).cuda(), avg, include_uniform)
-    p_ref, bits_ref, errs_ref = orc.sba_search(W, x, a.astype(np.float32), avg, include_uniform=include_uniform)
+                                         torch.from_numpy(a.astype(np.float32)).cuda(), avg, include_uniform, g=g)
+    p_ref, bits_ref, errs_ref = orc.sba_search(W, x, a.astype(np.float32), avg, g=g, include_uniform=include_uniform)
     errs_ref = np.asarray(errs_ref)
     assert errs.shape == errs_ref.shape
     assert np.abs(errs - errs_ref).max() <= ERR_RTOL * np.abs(errs_ref).max() + ERR_ATOL, (errs, errs_ref)
@@ -62,7 +62,7 @@ def _check_search(W, x, a, avg, include_uniform=True):
     # the winner is the oracle's, unless the oracle's own errors tie within the tolerance: then any of the tied
     # candidates is a valid answer
     assert errs_ref[p_star - first] <= errs_ref.min() * (1 + 2 * ERR_RTOL) + ERR_ATOL
-    G = W.shape[1] // 128
+    G = W.shape[1] // g
     assert int(bits.sum()) == avg * G and (bits == avg + 1).sum() == (bits == avg - 1).sum() == p_star
     if p_star == p_ref:
         assert (bits == bits_ref).all()
@@ -73,6 +73,19 @@ def _check_search(W, x, a, avg, include_uniform=True):
 def test_search_matches_the_oracle(N, K, M, avg):
     W, x, a = _layer(N, K, M, block=avg)
     _check_search(W, x, a, avg)
+
+
+@pytest.mark.parametrize("g,N,K,M,avg", [(32, 128, 512, 8, 2), (64, 256, 1024, 40, 2), (256, 128, 2048, 4, 2), (512, 64, 4096, 24, 2),
+                                         (32, 64, 9216, 8, 3)])
+def test_search_at_the_other_group_sizes(g, N, K, M, avg):
+    """Groups of 32 to 512 columns (the group-size ablation of the appendix); the last case has 288 groups, more than
+    a layer of 128-column groups can have.  Its weights are scaled by 1/8 (exact in fp16): with 9216 inputs the logits
+    would otherwise be large enough for the fp16 rounding of the device's outputs to show in the errors at first
+    order."""
+    W, x, a = _layer(N, K, M, name=f"sba-gpu-g{g}")
+    if K > 4096:
+        W = (W.astype(np.float32) * 0.125).astype(np.float16)
+    _check_search(W, x, a, avg, g=g)
 
 
 def test_search_without_the_uniform_candidate_and_constructed_optimum():

@@ -158,7 +158,8 @@ def test_sba_workspace_and_quantizer_argument_errors(slim):
     assert L.slim_sba_workspace_bytes(128, 4096, 4096, 128, 4, ctypes.byref(out)) == -1      # average bit-width
     assert L.slim_sba_workspace_bytes(0, 4096, 4096, 128, 2, ctypes.byref(out)) == -1        # no calibration token
     assert L.slim_sba_workspace_bytes(128, 4096, 4000, 128, 2, ctypes.byref(out)) == -2      # K not a multiple of 128
-    assert L.slim_sba_workspace_bytes(128, 4096, 4096, 64, 2, ctypes.byref(out)) == -2       # group size
+    assert L.slim_sba_workspace_bytes(128, 4096, 4096, 96, 2, ctypes.byref(out)) == -2       # group size
+    assert L.slim_sba_workspace_bytes(128, 4096, 4096, 64, 2, ctypes.byref(out)) == 0
     assert L.slim_sba_workspace_bytes(128, 4096, 4096, 128, 2, None) == -1
     # nothing is launched for null pointers
     bits = np.array([2, 2], dtype=np.uint8)
