@@ -2,6 +2,7 @@
 the defining property of the factor, a column-by-column elimination written with scalar loops, the
 constrained least-squares problem the update solves, and special cases with known answers."""
 import numpy as np
+import pytest
 
 from oracle import slim_oracle as orc
 from paper_2405_14917_b200 import workloads as wl
@@ -12,8 +13,8 @@ def _layer(N, K, T, name="gptq", block=0):
     return wl.make_weight(seed, N, K), wl.make_calibration_x(seed, T, K)
 
 
-def _w_hat(codes, scales, zeros):
-    return orc.dequant_f64(codes, scales, zeros)
+def _w_hat(codes, scales, zeros, g=128):
+    return orc.dequant_f64(codes, scales, zeros, g)
 
 
 # ------------------------------------------------------------------------------------------ Hessian and factor
@@ -41,12 +42,12 @@ def test_factor_defining_property_and_damping():
 
 
 # ------------------------------------------------------------------------------------------ the update
-def _columnwise(W16, x16, codes, scales, zeros, lam, upto):
+def _columnwise(W16, x16, codes, scales, zeros, lam, upto, g=128):
     """The published column-by-column elimination with the codes held fixed, scalar loops: after column k is set
     to its quantised value, its error divided by U_kk is pushed onto every later column through row k of U."""
     U, _ = orc.gptq_factor(orc.gptq_hessian(x16), lam)
     w = W16.astype(np.float64).copy()
-    w_hat = _w_hat(codes, scales, zeros)
+    w_hat = _w_hat(codes, scales, zeros, g)
     N, K = w.shape
     for k in range(upto):
         for n in range(N):
@@ -72,6 +73,22 @@ def test_block_update_equals_column_by_column_elimination():
         q_fn = orc.quantize_minmax if quantizer == "minmax" else (lambda a, b: orc.quantize_sqc(a, b)[:3])
         q, s, z = q_fn(w_in.astype(np.float16), bits[2:3])
         assert (q == codes[:, 256:]).all() and (s[0] == scales[2]).all() and (z[0] == zeros[2]).all()
+
+
+@pytest.mark.parametrize("g", [32, 64, 256])
+def test_block_update_equals_column_by_column_elimination_at_other_group_sizes(g):
+    """Algorithm 1 takes blocks of beta columns: with groups of g columns the block update over a group must still
+    equal the column-by-column elimination over its g columns."""
+    K = 3 * g
+    W, x = _layer(2, K, 40 if g < 256 else 900, name=f"gptq-col-g{g}")
+    bits = np.array([2, 3, 1])
+    for quantizer in ("minmax", "sqc"):
+        codes, scales, zeros, w_run = orc.gptq_quantize(W, x, bits, 0.01, quantizer, g)
+        w_in = _columnwise(W, x, codes, scales, zeros, 0.01, 2 * g, g)[:, 2 * g:]
+        assert np.abs(w_run[:, 2 * g:] - w_in).max() <= 1e-9
+        q_fn = orc.quantize_minmax if quantizer == "minmax" else (lambda a, b, gg: orc.quantize_sqc(a, b, gg)[:3])
+        q, s, z = q_fn(w_in.astype(np.float16), bits[2:3], g)
+        assert (q == codes[:, 2 * g:]).all() and (s[0] == scales[2]).all() and (z[0] == zeros[2]).all()
 
 
 def test_update_solves_the_constrained_least_squares_problem():
