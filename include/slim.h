@@ -30,8 +30,9 @@
  * have K / g entries or rows); K a multiple of g and of 128 with at most 256 tiles of 128 columns (1024 groups for
  * g < 128); N a multiple of 16; N = 0 or M = 0 is a successful no-op.  Anything else returns an error status and
  * enqueues nothing.  Pack, dequant, both linear entry points, the group salience and the quantizers
- * (slim_quantize_minmax, _groups, _sign1, _sqc) and the SBA search take every g; the layer-set launch and
- * slim_mpq_gemm_static take 128, 256 and 512; the GPTQ loop takes 128 only (SLIM_ERR_UNSUPPORTED otherwise).  Groups of 256 and 512 columns run on the tensor-core kernels of the 128-column tiles (a group is 2 or 4
+ * (slim_quantize_minmax, _groups, _sign1, _sqc; these also take a K that is any multiple of g), the SBA search and
+ * the GPTQ loop take every g; the layer-set launch and slim_mpq_gemm_static take 128, 256 and 512
+ * (SLIM_ERR_UNSUPPORTED otherwise).  Groups of 256 and 512 columns run on the tensor-core kernels of the 128-column tiles (a group is 2 or 4
  * tiles that share a row of scales and zeros); groups of 32 and 64 columns run on plain CUDA-core kernels, and the
  * batched entry point then wants room for the fp16 weights in its workspace (slim_workspace_bytes says how much).
  *

@@ -342,7 +342,7 @@ def gptq_factor(x: torch.Tensor, lam: float = 0.01, workspace: torch.Tensor | No
 
 
 def gptq_quantize(W: torch.Tensor, x: torch.Tensor, bits, lam: float = 0.01, quantizer: str = "sqc",
-                  workspace: torch.Tensor | None = None, return_running: bool = False):
+                  workspace: torch.Tensor | None = None, return_running: bool = False, g: int = GROUP):
     """Main loop of Algorithm 1 under a given bit map: group by group, quantise the running weights
     (SQC or Eq. 1) and push the group's error onto the columns still to come.  W fp16 [N][K], x fp16
     [T][K] calibration tokens.  Returns (codes uint8 [N][K], scales fp16 [G][N], zeros fp16 [G][N])
@@ -352,9 +352,9 @@ def gptq_quantize(W: torch.Tensor, x: torch.Tensor, bits, lam: float = 0.01, qua
     N, K = W.shape
     T = x.shape[0]
     b = _bits(bits)
-    G = K // GROUP
+    G = K // g
     if workspace is None:
-        workspace = torch.empty(gptq_workspace_bytes(T, N, K), dtype=torch.uint8, device=W.device)
+        workspace = torch.empty(gptq_workspace_bytes(T, N, K, g), dtype=torch.uint8, device=W.device)
     codes = torch.empty(N, K, dtype=torch.uint8, device=W.device)
     scales = torch.empty(G, N, dtype=torch.float16, device=W.device)
     zeros = torch.empty(G, N, dtype=torch.float16, device=W.device)
@@ -362,7 +362,7 @@ def gptq_quantize(W: torch.Tensor, x: torch.Tensor, bits, lam: float = 0.01, qua
     _check("slim_gptq_quantize", lib().slim_gptq_quantize(
         _dev(W, torch.float16, "W"), _dev(x, torch.float16, "x"), _bp(b), float(lam), 1 if quantizer == "sqc" else 0,
         codes.data_ptr(), scales.data_ptr(), zeros.data_ptr(), running.data_ptr() if return_running else None,
-        N, K, T, GROUP, _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(W)))
+        N, K, T, g, _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(W)))
     return (codes, scales, zeros, running) if return_running else (codes, scales, zeros)
 
 

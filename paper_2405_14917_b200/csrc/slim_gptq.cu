@@ -57,13 +57,13 @@ __device__ __forceinline__ void tile_mac(double (&acc)[4][4], int klen, const Op
         __syncthreads();
     }
 }
-// Operand stored with the tile index contiguous: element (k, i) = src[k * ld + i], k < kmax.
+// Operand stored with the tile index contiguous: element (k, i) = src[k * ld + i], k < kmax, i < imax.
 struct OpK {
-    const double* src; size_t ld; int kmax;
+    const double* src; size_t ld; int kmax; int imax = 1 << 30;
     __device__ __forceinline__ void load(int k0, double (&r)[4]) const {
         const int k = k0 + (threadIdx.x >> 4), i = (threadIdx.x & 15) * 4;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) r[e] = k < kmax ? src[static_cast<size_t>(k) * ld + i + e] : 0.0;
+        for (int e = 0; e < 4; ++e) r[e] = (k < kmax && i + e < imax) ? src[static_cast<size_t>(k) * ld + i + e] : 0.0;
     }
     __device__ __forceinline__ static void store(double (*S)[kFPad], const double (&r)[4]) {
         const int k = threadIdx.x >> 4, i = (threadIdx.x & 15) * 4;
@@ -331,27 +331,27 @@ __global__ void __launch_bounds__(256) gptq_init_kernel(const __half* __restrict
     const int k = static_cast<int>(i % static_cast<size_t>(K));
     w[i] = dead[k] ? 0.0 : static_cast<double>(__half2float(W[i]));
 }
-// The group's current weights rounded to fp16 (one rounding), [N][128]: the quantizer's input.
-__global__ void __launch_bounds__(256) gptq_round_kernel(const double* __restrict__ w, __half* __restrict__ wb, int N, int K, int c0) {
+// The group's current weights rounded to fp16 (one rounding), [N][g]: the quantizer's input.
+__global__ void __launch_bounds__(256) gptq_round_kernel(const double* __restrict__ w, __half* __restrict__ wb, int N, int K, int c0, int g) {
     const int i = blockIdx.x * 256 + threadIdx.x;
-    if (i >= N * SLIM_GROUP) return;
-    const int n = i >> 7, c = i & 127;
+    if (i >= N * g) return;
+    const int n = i / g, c = i - n * g;
     wb[i] = __double2half(w[static_cast<size_t>(n) * K + c0 + c]);
 }
-// delta = w_b - s (q - z) for 16 rows per CTA, codes copied into the layer's array,
-// E[n][c] = sum_{c' <= c} delta[n][c'] R[c0 + c'][c0 + c]   (thread c, c' ascending).
-constexpr int kErrRows = 16;
-__global__ void __launch_bounds__(SLIM_GROUP) gptq_error_kernel(const double* __restrict__ w, const uint8_t* __restrict__ qb,
-                                                                const __half* __restrict__ s_row, const __half* __restrict__ z_row,
-                                                                const double* __restrict__ R, uint8_t* __restrict__ codes,
-                                                                double* __restrict__ E, int N, int K, int c0) {
-    __shared__ double delta[kErrRows][SLIM_GROUP];
-    const int c = threadIdx.x, n0 = kErrRows * blockIdx.x;
-    for (int r = 0; r < kErrRows; ++r) {
+// delta = w_b - s (q - z) for ROWS rows per CTA, codes copied into the layer's array,
+// E[n][c] = sum_{c' <= c} delta[n][c'] R[c0 + c'][c0 + c]   (thread c of the group's GS columns, c' ascending).
+template <int GS, int ROWS>
+__global__ void __launch_bounds__(GS) gptq_error_kernel(const double* __restrict__ w, const uint8_t* __restrict__ qb,
+                                                        const __half* __restrict__ s_row, const __half* __restrict__ z_row,
+                                                        const double* __restrict__ R, uint8_t* __restrict__ codes,
+                                                        double* __restrict__ E, int N, int K, int c0) {
+    __shared__ double delta[ROWS][GS];
+    const int c = threadIdx.x, n0 = ROWS * blockIdx.x;
+    for (int r = 0; r < ROWS; ++r) {
         const int n = n0 + r;
         double d = 0.0;
         if (n < N) {
-            const uint8_t q = qb[static_cast<size_t>(n) * SLIM_GROUP + c];
+            const uint8_t q = qb[static_cast<size_t>(n) * GS + c];
             codes[static_cast<size_t>(n) * K + c0 + c] = q;
             const double sc = static_cast<double>(__half2float(s_row[n])), zp = static_cast<double>(__half2float(z_row[n]));
             d = w[static_cast<size_t>(n) * K + c0 + c] - sc * (static_cast<double>(q) - zp);
@@ -359,32 +359,35 @@ __global__ void __launch_bounds__(SLIM_GROUP) gptq_error_kernel(const double* __
         delta[r][c] = d;
     }
     __syncthreads();
-    double acc[kErrRows];
+    double acc[ROWS];
 #pragma unroll
-    for (int r = 0; r < kErrRows; ++r) acc[r] = 0.0;
+    for (int r = 0; r < ROWS; ++r) acc[r] = 0.0;
     for (int c2 = 0; c2 <= c; ++c2) {
         const double rv = R[static_cast<size_t>(c0 + c2) * K + c0 + c];
 #pragma unroll
-        for (int r = 0; r < kErrRows; ++r) acc[r] = fma(delta[r][c2], rv, acc[r]);
+        for (int r = 0; r < ROWS; ++r) acc[r] = fma(delta[r][c2], rv, acc[r]);
     }
-    for (int r = 0; r < kErrRows; ++r)
-        if (n0 + r < N) E[static_cast<size_t>(n0 + r) * SLIM_GROUP + c] = acc[r];
+    for (int r = 0; r < ROWS; ++r)
+        if (n0 + r < N) E[static_cast<size_t>(n0 + r) * GS + c] = acc[r];
 }
-// w[n][k] -= sum_c E[n][c] U[c0 + c][k] for the columns k >= k0 = c0 + 128 (c ascending).
+// w[n][k] -= sum_c E[n][c] U[c0 + c][k] for the columns k >= k0 = c0 + g (c ascending).
 __global__ void __launch_bounds__(256) gptq_update_kernel(double* __restrict__ w, const double* __restrict__ E,
-                                                          const double* __restrict__ U, int N, int K, int c0) {
+                                                          const double* __restrict__ U, int N, int K, int c0, int g) {
     __shared__ __align__(16) double As[kFK][kFPad], Bs[kFK][kFPad];
-    const int n0 = kFB * blockIdx.y, k0 = c0 + SLIM_GROUP + kFB * blockIdx.x;
+    const int n0 = kFB * blockIdx.y, k0 = c0 + g + kFB * blockIdx.x;
     double acc[4][4] = {};
-    tile_mac(acc, SLIM_GROUP, OpI{E + static_cast<size_t>(n0) * SLIM_GROUP, SLIM_GROUP, SLIM_GROUP, N - n0},
-             OpK{U + static_cast<size_t>(c0) * K + k0, static_cast<size_t>(K), SLIM_GROUP}, As, Bs);
+    tile_mac(acc, g, OpI{E + static_cast<size_t>(n0) * g, static_cast<size_t>(g), g, N - n0},
+             OpK{U + static_cast<size_t>(c0) * K + k0, static_cast<size_t>(K), g, K - k0}, As, Bs);
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
         const int n = n0 + tidx(ty, e);
         if (n >= N) continue;
 #pragma unroll
-        for (int f = 0; f < 4; ++f) w[static_cast<size_t>(n) * K + k0 + tidx(tx, f)] -= acc[e][f];
+        for (int f = 0; f < 4; ++f) {
+            const int k = k0 + tidx(tx, f);
+            if (k < K) w[static_cast<size_t>(n) * K + k] -= acc[e][f];      // groups of 32 columns end in the middle of a tile
+        }
     }
 }
 
@@ -395,16 +398,16 @@ struct GptqLayout {
 static size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 static int gptq_layout(int T, int N, int K, int g, GptqLayout* lay) {
     if (lay == nullptr || T < 1 || N < 0 || K < 1) return SLIM_ERR_INVALID_ARG;
-    if (g != SLIM_GROUP) return SLIM_ERR_UNSUPPORTED;
-    if (K % SLIM_GROUP != 0 || K / SLIM_GROUP > SLIM_MAX_GROUPS) return SLIM_ERR_UNSUPPORTED;
+    if (g != 32 && g != 64 && g != 128 && g != 256 && g != 512) return SLIM_ERR_UNSUPPORTED;
+    if (K % g != 0 || K % SLIM_GROUP != 0 || K / SLIM_GROUP > SLIM_MAX_GROUPS) return SLIM_ERR_UNSUPPORTED;
     size_t off = 0;
     lay->dead = off; off += up256(static_cast<size_t>(K));
     lay->R = off; off += up256(static_cast<size_t>(K) * K * sizeof(double));
     lay->U = off; off += up256(static_cast<size_t>(K) * K * sizeof(double));
     lay->w = off; off += up256(static_cast<size_t>(N) * K * sizeof(double));
-    lay->E = off; off += up256(static_cast<size_t>(N) * SLIM_GROUP * sizeof(double));
-    lay->wb = off; off += up256(static_cast<size_t>(N) * SLIM_GROUP * sizeof(__half));
-    lay->qb = off; off += up256(static_cast<size_t>(N) * SLIM_GROUP);
+    lay->E = off; off += up256(static_cast<size_t>(N) * g * sizeof(double));
+    lay->wb = off; off += up256(static_cast<size_t>(N) * g * sizeof(__half));
+    lay->qb = off; off += up256(static_cast<size_t>(N) * g);
     lay->total = off;
     return SLIM_OK;
 }
@@ -473,9 +476,10 @@ int slim_gptq_quantize(const void* W, const void* x, const uint8_t* bits_host, d
     slim::GptqLayout lay;
     int st = slim::gptq_layout(T, N, K, g, &lay);
     if (st != SLIM_OK) return st;
-    slim::GroupTable gt;
-    st = slim::make_group_table(N, K, g, bits_host, &gt);
-    if (st != SLIM_OK) return st;
+    if (bits_host == nullptr || N % 16 != 0) return bits_host == nullptr ? SLIM_ERR_INVALID_ARG : SLIM_ERR_UNSUPPORTED;
+    const int G = K / g;
+    for (int j = 0; j < G; ++j)
+        if (bits_host[j] < 1 || bits_host[j] > 4) return SLIM_ERR_INVALID_ARG;
     if (!(lambda > 0.0)) return SLIM_ERR_INVALID_ARG;
     if (N == 0) return SLIM_OK;
     if (W == nullptr || x == nullptr || codes == nullptr || scales == nullptr || zeros == nullptr) return SLIM_ERR_INVALID_ARG;
@@ -499,20 +503,28 @@ int slim_gptq_quantize(const void* W, const void* x, const uint8_t* bits_host, d
     const size_t total = static_cast<size_t>(N) * K;
     slim::gptq_init_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, s>>>(static_cast<const __half*>(W), ws + lay.dead, w, total, K);
     SLIM_CUDA_TRY(cudaGetLastError());
-    for (int j = 0; j < gt.G; ++j) {
-        const int c0 = SLIM_GROUP * j;
-        slim::gptq_round_kernel<<<(N * SLIM_GROUP + 255) / 256, 256, 0, s>>>(w, wb, N, K, c0);
+    for (int j = 0; j < G; ++j) {
+        const int c0 = g * j;
+        slim::gptq_round_kernel<<<(N * g + 255) / 256, 256, 0, s>>>(w, wb, N, K, c0, g);
         SLIM_CUDA_TRY(cudaGetLastError());
-        const uint8_t b1[1] = {gt.bits[j]};
+        const uint8_t b1[1] = {bits_host[j]};
+        // the group as a one-group layer of g columns
         st = use_sqc ? slim_quantize_sqc(wb, b1, qb, sc + static_cast<size_t>(j) * N, zp + static_cast<size_t>(j) * N, nullptr,
-                                         N, SLIM_GROUP, g, 0.1, 50, stream)
+                                         N, g, g, 0.1, 50, stream)
                      : slim_quantize_minmax(wb, b1, qb, sc + static_cast<size_t>(j) * N, zp + static_cast<size_t>(j) * N,
-                                            N, SLIM_GROUP, g, stream);
+                                            N, g, g, stream);
         if (st != SLIM_OK) return st;
-        slim::gptq_error_kernel<<<(N + slim::kErrRows - 1) / slim::kErrRows, SLIM_GROUP, 0, s>>>(
-            w, qb, sc + static_cast<size_t>(j) * N, zp + static_cast<size_t>(j) * N, R, codes, E, N, K, c0);
-        if (j + 1 < gt.G)
-            slim::gptq_update_kernel<<<dim3((K - c0 - SLIM_GROUP) / slim::kFB, (N + slim::kFB - 1) / slim::kFB), 256, 0, s>>>(w, E, U, N, K, c0);
+        const __half* s_row = sc + static_cast<size_t>(j) * N;
+        const __half* z_row = zp + static_cast<size_t>(j) * N;
+        switch (g) {
+            case 32: slim::gptq_error_kernel<32, 16><<<(N + 15) / 16, 32, 0, s>>>(w, qb, s_row, z_row, R, codes, E, N, K, c0); break;
+            case 64: slim::gptq_error_kernel<64, 16><<<(N + 15) / 16, 64, 0, s>>>(w, qb, s_row, z_row, R, codes, E, N, K, c0); break;
+            case 128: slim::gptq_error_kernel<128, 16><<<(N + 15) / 16, 128, 0, s>>>(w, qb, s_row, z_row, R, codes, E, N, K, c0); break;
+            case 256: slim::gptq_error_kernel<256, 16><<<(N + 15) / 16, 256, 0, s>>>(w, qb, s_row, z_row, R, codes, E, N, K, c0); break;
+            default: slim::gptq_error_kernel<512, 8><<<(N + 7) / 8, 512, 0, s>>>(w, qb, s_row, z_row, R, codes, E, N, K, c0); break;
+        }
+        if (j + 1 < G)
+            slim::gptq_update_kernel<<<dim3((K - c0 - g + slim::kFB - 1) / slim::kFB, (N + slim::kFB - 1) / slim::kFB), 256, 0, s>>>(w, E, U, N, K, c0, g);
         SLIM_CUDA_TRY(cudaGetLastError());
     }
     if (w_running != nullptr) SLIM_CUDA_TRY(cudaMemcpyAsync(w_running, w, total * sizeof(double), cudaMemcpyDeviceToDevice, s));

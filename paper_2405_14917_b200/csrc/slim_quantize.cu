@@ -20,7 +20,8 @@ struct GroupBits {
 static int make_group_bits(int N, int K, int g, const uint8_t* bits_host, GroupBits* out) {
     if (bits_host == nullptr || N < 0 || K < 0) return SLIM_ERR_INVALID_ARG;
     if (g != 32 && g != 64 && g != 128 && g != 256 && g != 512) return SLIM_ERR_UNSUPPORTED;
-    if (K % g != 0 || K % SLIM_GROUP != 0 || N % 16 != 0 || K / SLIM_GROUP > SLIM_MAX_GROUPS) return SLIM_ERR_UNSUPPORTED;
+    // the quantizers work group by group: any K that is a multiple of g (Algorithm 1 hands them one group at a time)
+    if (K % g != 0 || N % 16 != 0 || K / g > kQuantMaxGroups) return SLIM_ERR_UNSUPPORTED;
     memset(out, 0, sizeof *out);
     out->G = K / g;
     for (int j = 0; j < out->G; ++j) {
@@ -233,7 +234,7 @@ extern "C" {
 int slim_group_salience(const void* W, const float* act_norm, double* salience, int N, int K, int g, void* stream) {
     if (N < 0 || K < 0) return SLIM_ERR_INVALID_ARG;
     if (g != 32 && g != 64 && g != 128 && g != 256 && g != 512) return SLIM_ERR_UNSUPPORTED;
-    if (K % g != 0 || K % SLIM_GROUP != 0 || K / SLIM_GROUP > SLIM_MAX_GROUPS) return SLIM_ERR_UNSUPPORTED;
+    if (K % g != 0 || K / g > slim::kQuantMaxGroups) return SLIM_ERR_UNSUPPORTED;
     if (K == 0) return SLIM_OK;
     if (W == nullptr || act_norm == nullptr || salience == nullptr) return SLIM_ERR_INVALID_ARG;
     if (!slim::aligned16(W) || !slim::aligned16(act_norm) || !slim::aligned16(salience)) return SLIM_ERR_ALIGNMENT;

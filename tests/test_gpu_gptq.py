@@ -35,11 +35,11 @@ def test_factor_against_the_library_cholesky_of_the_inverse(K, T):
     assert np.abs(U - U_ref).max() <= 1e-9 * np.abs(U_ref).max()
 
 
-def _check_quantize(W, x, bits, quantizer, lam=0.01):
+def _check_quantize(W, x, bits, quantizer, lam=0.01, g=128):
     slim = _slim()
     codes, scales, zeros, running = slim.gptq_quantize(torch.from_numpy(W).cuda(), torch.from_numpy(x).cuda(), bits, lam, quantizer,
-                                                       return_running=True)
-    c_ref, s_ref, z_ref, w_ref = orc.gptq_quantize(W, x, np.asarray(bits), lam, quantizer)
+                                                       return_running=True, g=g)
+    c_ref, s_ref, z_ref, w_ref = orc.gptq_quantize(W, x, np.asarray(bits), lam, quantizer, g)
     codes, scales, zeros, running = codes.cpu().numpy(), scales.cpu().numpy(), zeros.cpu().numpy(), running.cpu().numpy()
     assert (scales.view(np.uint16) == s_ref.view(np.uint16)).all()
     assert (zeros.view(np.uint16) == z_ref.view(np.uint16)).all()
@@ -57,6 +57,17 @@ def test_quantize_matches_the_oracle(N, K, T, bits, quantizer):
         N = N // 16 * 16 + 16
     W, x = _layer(N, K, T, block=len(bits))
     _check_quantize(W, x, bits, quantizer)
+
+
+@pytest.mark.parametrize("g,N,K,T", [(32, 48, 384, 200), (32, 16, 1152, 300), (64, 80, 512, 128), (256, 64, 1024, 300), (512, 32, 1536, 400)])
+@pytest.mark.parametrize("quantizer", ["minmax", "sqc"])
+def test_quantize_at_the_other_group_sizes(g, N, K, T, quantizer):
+    """Algorithm 1 with blocks of g columns (the group-size ablation of the appendix).  At g = 32 every other
+    trailing region ends in the middle of a 64-column tile of the update."""
+    rng = np.random.default_rng(g + K)
+    bits = rng.integers(1, 5, K // g)
+    W, x = _layer(N, K, T, block=g)
+    _check_quantize(W, x, bits, quantizer, g=g)
 
 
 def test_uncorrelated_inputs_and_dead_channel():

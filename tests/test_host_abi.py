@@ -183,7 +183,9 @@ def test_gptq_workspace_and_argument_errors(slim):
     assert ws_bytes(64, 0, 512)[1] == 512 + 2 * 512 * 512 * 8            # the factor alone
     assert ws_bytes(0, 256, 512)[0] == -1                                 # no calibration token
     assert ws_bytes(64, 256, 500)[0] == -2                                # K not a multiple of 128
-    assert ws_bytes(64, 256, 512, g=64)[0] == -2                          # group size
+    assert ws_bytes(64, 256, 512, g=96)[0] == -2                          # group size
+    st64, b64 = ws_bytes(64, 256, 512, g=64)                              # the per-group buffers follow the group size
+    assert st64 == 0 and b64 == b - 256 * 64 * (8 + 2 + 1)
     bits = np.array([2, 2, 2, 2], dtype=np.uint8)
     L = slim.lib()
     args = lambda lam, wsb: (256, 256, bits.ctypes.data, ctypes.c_double(lam), 1, 256, 256, 256, None, 256, 512, 64, 128, 256, wsb, None)
