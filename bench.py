@@ -656,18 +656,19 @@ def decode_entry(name, layers, spec, device, timer, launch, steps, min_total_s, 
     peak, peak_kind = measured_hbm_peak()
     per_launch_us = 1e3 * ms / n_dom
     achieved = alg_bytes / n_dom / (per_launch_us * 1e-6) / 1e9
-    kernel = {"set": "gemv_set_kernel", "per-layer": "gemv_kernel", "decoder-order": "gemv_set_kernel + gemv_kernel"}[launch]
-    integer_form = M == 1 and launch != "per-layer"
+    one = "gemv_one_kernel" if M == 1 else "gemv_kernel"      # slim_mpq_gemv's single-token kernel, or the general one
+    kernel = {"set": "gemv_set_kernel", "per-layer": one, "decoder-order": "gemv_set_kernel + " + one}[launch]
+    integer_form = M == 1
     out = {"name": name, "metric": f"mixed-precision dequant GEMV GB/s at M={M} ({spec['model']} layers, avg {spec['avg_bits']}-bit, g=128)",
            "value": value, "unit": UNIT, "ms_per_step": ms, "timing": tm,
            "dtype": ("s32 (mma.sync m16n8k32 u8 x s8: byte-masked code words against base-256 digits of fixed-point x; f32 fold)"
                      if integer_form and launch == "set" else
-                     "s32 integer MMAs in the q/k/v and gate/up sets, f16 MMAs in the o and down calls" if integer_form else
+                     "s32 (mma.sync m16n8k32 u8 x s8 on byte-masked code words, f32 fold) in every call" if integer_form else
                      "f16 (mma.sync m16n8k16 on raw code fields, f32 accumulate)"),
            "config": {"workload": name, "layers": len(layers), "M": M, "avg_bits": spec["avg_bits"], "g": wl.GROUP,
                       "algorithmic_bytes_per_step": alg_bytes, "l2": f"distinct layers, {alg_bytes / 1e9:.2f} GB per step > L2",
                       "launch": {"set": "CUDA graph of the layer-set launch: one persistent kernel for the whole sweep (plus one kernel that stages x)",
-                                 "per-layer": "CUDA graph of one slim_mpq_gemv launch per layer, programmatic dependent launch",
+                                 "per-layer": "CUDA graph of one slim_mpq_gemv launch per layer (the launch mode of App. B.2), programmatic dependent launch",
                                  "decoder-order": "CUDA graph; per block: set(q, k, v) on one x, o, set(gate, up) on one x, down: the calls a decoder can issue, in its order"}[launch],
                       "grouped_launch": launch != "per-layer"},
            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
@@ -857,7 +858,7 @@ def group_size_entries(device, timer):
         achieved = alg / (ms * 1e-3) / 1e9
         out.append({"name": f"single-4096x4096-avg2-m1-g{g}", "metric": f"one 4096 x 4096 layer per launch, avg 2-bit, M = 1, group size {g} (slim_mpq_gemv, 64 rotating copies)",
                     "value": achieved, "unit": UNIT, "ms_per_step": ms, "timing": tm,
-                    "kernel": "gemv_small_kernel (CUDA cores)" if g < 128 else "gemv_kernel (tensor cores)",
+                    "kernel": "gemv_small_kernel (CUDA cores)" if g < 128 else "gemv_one_kernel (tensor cores)",
                     "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
                                  "avg_launch_us": 1e3 * ms / copies, "algorithmic_bytes_per_launch": alg / copies},
                     "config": {"workload": f"single-4096x4096-avg2-m1-g{g}", "g": g, "layers": copies, "algorithmic_bytes_per_step": alg,

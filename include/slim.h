@@ -138,7 +138,10 @@ int slim_dequant(const void* packed, const uint8_t* bits_host, const void* scale
  * within the rounding of the accumulation order; at M = 1 with the fixed-point x described there) when the
  * workspace has the slim_workspace_bytes() that shape asks for; with a smaller workspace it takes the per-layer
  * kernel.  The call reads no host memory after it returns and can be captured in a CUDA graph either way.
- * The per-layer kernel is launched with programmatic stream serialisation and fetches packed, scales and zeros
+ * At M = 1 every route takes x in the 22-bit fixed-point form described at slim_mpq_gemv_set (the per-layer
+ * single-token kernel, CTAs that hold the whole K of a few 16-row tiles, serves the layers whose K fits a CTA's
+ * shared memory with all CTAs resident at once; the others, and M > 1, multiply the fp16 x as it is).
+ * The per-layer kernels are launched with programmatic stream serialisation and fetches packed, scales and zeros
  * before it waits for the kernel ahead of it on the stream: those three buffers must be complete when the call is
  * enqueued, or be written by a kernel that does not signal programmatic launch completion early (x and y may be
  * produced and consumed by the neighbouring kernels as usual). */
@@ -208,7 +211,7 @@ int slim_mpq_gemm_static(const void* x, const void* packed, const uint8_t* bits_
  * fp16 activation within a factor 2^11 of that maximum is taken exactly and a smaller one with an error
  * of at most 2^-22 of the maximum; the sums over the group are then exact.  Per output row n this adds at
  * most  sum over groups of 2^-22 max|x_group| sum_{k in group} |w-hat[n][k]|  to the error of the fp16
- * path (slim_mpq_gemv multiplies the fp16 x as it is); x must be finite.  Sets with more tokens multiply
+ * path at more than one token; x must be finite.  Sets with more tokens multiply
  * the fp16 x as it is.
  * N > 0 a multiple of 16, K > 0 a multiple of 128; g in {128, 256, 512}, one value for the whole set (for 256 and
  * 512 "group" in the bound above reads "128 columns of a group"); SLIM_ERR_UNSUPPORTED for 32 and 64. */

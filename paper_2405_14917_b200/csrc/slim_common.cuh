@@ -34,6 +34,11 @@ size_t gemv_route_workspace_bytes(int M, int N, int K, int g, const uint8_t* bit
 int gemv_route(const void* x, const void* packed, const uint8_t* bits_host, const GroupTable& gt, const void* scales, const void* zeros,
                void* y, int M, int N, int K, int g, void* workspace, size_t workspace_bytes, cudaStream_t stream);
 
+// slim_mpq_gemv sends single-token layers whose K fits a CTA's shared memory to a kernel of their own (slim_gemv_one.cu):
+// SLIM_OK, a negative status, or 1 if not taken.
+int gemv_one(const void* x, const void* packed, const GroupTable& gt, const void* scales, const void* zeros, void* y,
+             int M, int N, int K, void* workspace, cudaStream_t stream);
+
 // Validates shape arguments and fills the table, for group sizes of 128, 256 and 512 columns (bits_host has K / g
 // entries).  Returns SLIM_OK or an error status; SLIM_ERR_UNSUPPORTED for the group sizes 32 and 64, which have
 // kernels of their own (is_small_group).

@@ -582,6 +582,11 @@ int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host, c
         const int routed = slim::gemv_route(x, packed, bits_host, gt, scales, zeros, y, M, N, K, g, workspace, workspace_bytes, s);
         if (routed <= 0) return routed;
     }
+    // A single token: the integer form with the whole K of a few tiles per CTA, if the layer fits it.
+    {
+        const int taken = slim::gemv_one(x, packed, gt, scales, zeros, y, M, N, K, workspace, s);
+        if (taken <= 0) return taken;
+    }
     // From kPreStageMinM tokens on, a small kernel puts x into fragment order once, in the
     // workspace; with a workspace too small for that every CTA stages its own part of x.
     const bool pre = M >= slim::kPreStageMinM && workspace_bytes >= slim::prestage_bytes(M, gt);

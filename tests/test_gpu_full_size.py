@@ -225,11 +225,19 @@ def _row_bound(L, x):
     return sum(2.0 ** -22 * xa[128 * j:128 * j + 128].max() * What[:, 128 * j:128 * j + 128].sum(axis=1) for j in range(G))
 
 
-def _run_single_token_set(L, x):
+ROUTES = ("set", "per-layer")         # the layer-set launch, and slim_mpq_gemv's single-token kernel
+
+
+def _run_single_token_set(L, x, route="set"):
     slim = _slim()
     dl = slim.QuantLinear(torch.from_numpy(orc.pack(L["codes"], L["bits"])).cuda(), L["bits"],
                           torch.from_numpy(L["scales"]).cuda(), torch.from_numpy(L["zeros"]).cuda(), L["N"], L["K"])
     y = torch.full((1, L["N"]), float("nan"), dtype=torch.float16, device="cuda")
+    if route == "per-layer":
+        ws = slim.new_workspace(1, L["N"], L["K"], L["bits"])
+        dl.forward(torch.from_numpy(x).cuda(), ws, out=y)
+        slim.workspace_status(ws)
+        return y.cpu().numpy()
     s = slim.LayerSet([(dl, torch.from_numpy(x).cuda(), y)])
     assert s.info["max_tokens"] == 1
     s.run()
@@ -244,8 +252,9 @@ def _check_row_bound(y, y_ref, bound, what):
     assert worst <= 0, f"{what}: a row exceeds the fixed-point bound by {worst:.3e}"
 
 
+@pytest.mark.parametrize("route", ROUTES)
 @pytest.mark.parametrize("ratio", [1e3, 1e4])
-def test_fixed_point_form_one_dominant_activation_in_every_group(ratio):
+def test_fixed_point_form_one_dominant_activation_in_every_group(ratio, route):
     """Every group holds one activation `ratio` times the rest (which then lose their last bits to the fixed-point
     grid), and a quarter of the rows have a weight that dequantises to exactly 0 at the dominant column of every
     group, so that nothing large hides their rounding error."""
@@ -263,13 +272,14 @@ def test_fixed_point_form_one_dominant_activation_in_every_group(ratio):
         codes[zero_rows, k] = zint[j, zero_rows].astype(np.uint8)     # q = z: the weight is exactly 0
     L["codes"] = codes
     assert (orc.dequant_f64(codes, L["scales"], L["zeros"])[np.ix_(zero_rows, dom)] == 0).all()
-    y = _run_single_token_set(L, x)
+    y = _run_single_token_set(L, x, route)
     y_ref = orc.linear_f64(x, codes, L["scales"], L["zeros"])
     check_output(y, y_ref, f"dominant activation x{ratio:g}")
     _check_row_bound(y, y_ref, _row_bound(L, x), f"dominant activation x{ratio:g}")
 
 
-def test_fixed_point_form_largest_and_smallest_fp16_activations():
+@pytest.mark.parametrize("route", ROUTES)
+def test_fixed_point_form_largest_and_smallest_fp16_activations(route):
     """A group whose largest |x| is 65504 (the fixed-point scale 2^S is then below 1), a group of fp16 subnormals
     only (2^S = 2^27), a group with one subnormal among zeros, and ordinary groups in between."""
     N, K = 256, 1024
@@ -282,7 +292,7 @@ def test_fixed_point_form_largest_and_smallest_fp16_activations():
     x[0, 384:512] = sub                                            # subnormals of both signs
     x[0, 640:768] = 0
     x[0, 700] = np.array([1], dtype=np.uint16).view(np.float16)[0]  # the smallest subnormal, alone in its group
-    y = _run_single_token_set(L, x)
+    y = _run_single_token_set(L, x, route)
     y_ref = orc.linear_f64(x, L["codes"], L["scales"], L["zeros"])
     check_output(y, y_ref, "fp16 range")
     _check_row_bound(y, y_ref, _row_bound(L, x), "fp16 range")
@@ -290,6 +300,6 @@ def test_fixed_point_form_largest_and_smallest_fp16_activations():
     x2 = np.zeros_like(x)
     x2[0, 384:512] = sub
     x2[0, 700] = x[0, 700]
-    y2 = _run_single_token_set(L, x2)
+    y2 = _run_single_token_set(L, x2, route)
     y2_ref = orc.linear_f64(x2, L["codes"], L["scales"], L["zeros"])
     assert np.abs(y2.astype(np.float64) - y2_ref).max() <= 2.0 ** -10 * np.abs(y2_ref).max() + 2.0 ** -25
