@@ -37,13 +37,23 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_TENSOR_TFLOPS = 1400.0
 
 # DRAM traffic of the GEMV kernel per launch from one ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), keyed by the sha256 of the kernel source it was taken from.  A kernel
-# that has changed since reports null.
+# dram__bytes_write.sum), keyed by the sha256 of the kernel's sources (slim_gemv_set.cu and the two device headers
+# it includes, concatenated in that order) at the time of the capture.  A kernel that has changed since reports null.
+SET_KERNEL_SOURCES = ("slim_gemv_set.cu", "slim_gemv_i8.cuh", "slim_gemv_dev.cuh")
+
+
+def set_kernel_hash():
+    h = hashlib.sha256()
+    for name in SET_KERNEL_SOURCES:
+        h.update(open(os.path.join(ROOT, "paper_2405_14917_b200", "csrc", name), "rb").read())
+    return h.hexdigest()
+
+
 NCU_TRAFFIC = {
-    # layer-set kernel, 4 blocks of the LLaMA-7B sweep (28 layers, avg 2-bit, M = 1): 228,647,680 B read +
-    # 4,347,392 B written per launch (algorithmic 228,297,816 B); scaled to the full sweep by the algorithmic bytes
+    # layer-set kernel, 4 blocks of the LLaMA-7B sweep (28 layers, avg 2-bit, M = 1): 228,637,696 B read +
+    # 3,888,640 B written per launch (algorithmic 228,297,816 B); scaled to the full sweep by the algorithmic bytes
     # (the traffic is the packed data read once, so it grows in proportion)
-    "f44ab8781c759ebcbd6e82bd44590508fffc816de54eaf735911b3cd95707a47": {"layer": "4 blocks", "traffic_bytes": 232995072, "algorithmic_bytes": 228297816},
+    "d55c23b51182f823ade7b02461006a318690733477b3f74f70d725dccc2b2cb7": {"layer": "4 blocks", "traffic_bytes": 232526336, "algorithmic_bytes": 228297816},
 }
 
 
@@ -974,8 +984,7 @@ def run_ours(args, spec):
             "timing": tm, "roofline": entry["roofline"], "e2e": entry["e2e"],
             "gpu_launches": steps * tm["blocks"] * entry["gpu_launches_per_step"], "clocks": entry["clocks"]}
     if M <= slim.GEMV_MAX_M and launch == "set":
-        sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2405_14917_b200", "csrc", "slim_gemv_set.cu"), "rb").read()).hexdigest()
-        traffic = NCU_TRAFFIC.get(sha)
+        traffic = NCU_TRAFFIC.get(set_kernel_hash())
         line["roofline"]["traffic"] = (traffic["traffic_bytes"] / traffic["algorithmic_bytes"] * entry["roofline"]["algorithmic_bytes_per_launch"]) if traffic else None
     elif "traffic" not in line["roofline"]:
         line["roofline"]["traffic"] = None

@@ -27,7 +27,7 @@ namespace slim {
 
 constexpr int kOneWarps = 16;
 constexpr int kOneThreads = 32 * kOneWarps;
-constexpr int kOneCluster = 8;                          // CTAs that share the staging of x
+constexpr int kOneCluster = 8;                          // CTAs that share the staging of x (4 where eight do not all fit)
 constexpr int kOneMaxPairs = 4;                         // tile pairs per CTA
 constexpr uint32_t kOneOffAbort = 8 * kOneWarps;        // after the warps' barriers
 constexpr uint32_t kOneOffXs = 256;                     // per warp: 128 ints of scratch for the digit staging, later its partial sums
@@ -139,6 +139,8 @@ __global__ void __launch_bounds__(kOneThreads, PAIRS == 1 ? 2 : 1) gemv_one_kern
     const int tiles_here = max(min(TPC, (p.N >> 4) - tile0), 0);  // 0: a CTA that only fills up its cluster
     const int ng = (p.G - warp + kOneWarps - 1) / kOneWarps;      // this warp's K-tiles: warp, warp + 16, ...
     const uint32_t rank = cluster_ctarank();
+    uint32_t nrank;                                        // CTAs of the cluster: 8 or 4
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(nrank));
 
     // ---- requests that do not depend on x
     if (lane == 0) {
@@ -173,15 +175,14 @@ __global__ void __launch_bounds__(kOneThreads, PAIRS == 1 ? 2 : 1) gemv_one_kern
 
     // ---- the activations as digits: this CTA's share of the K-tiles, written into every CTA of the cluster
     int* Xs = reinterpret_cast<int*>(smem + kOneOffXs + 512 * warp);
-    for (int j = static_cast<int>(rank) + kOneCluster * warp; j < p.G; j += kOneCluster * kOneWarps) {
+    for (int j = static_cast<int>(rank + nrank * warp); j < p.G; j += static_cast<int>(nrank) * kOneWarps) {
         const uint32_t off = p.off_x + static_cast<uint32_t>(staged_group_offset(j, p.pre3[j], 2));
         stage_group_i8(p.x + SLIM_GROUP * j, smem + off, p.bits[j], lane, Xs);
         __syncwarp();
         const int pieces = (128 + 512 * slice_count(p.bits[j])) / 16;
         for (int i = lane; i < pieces; i += 32) {
             const uint4 v = lds128(sbase + off + 16u * i);
-#pragma unroll
-            for (uint32_t r = 0; r < kOneCluster; ++r)
+            for (uint32_t r = 0; r < nrank; ++r)
                 if (r != rank) st_cluster_u32x4(sbase + off + 16u * i, r, v);
         }
     }
@@ -237,7 +238,7 @@ __global__ void __launch_bounds__(kOneThreads, PAIRS == 1 ? 2 : 1) gemv_one_kern
 }
 
 template <int PAIRS>
-static cudaError_t launch_one(const OneParams& prm, int grid, size_t smem, cudaStream_t stream) {
+static cudaError_t launch_one(const OneParams& prm, int grid, int cluster, size_t smem, cudaStream_t stream) {
     static std::atomic<bool> attr_set[64];    // zero-initialised; set-up is idempotent, so a race repeats it harmlessly
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -257,7 +258,7 @@ static cudaError_t launch_one(const OneParams& prm, int grid, size_t smem, cudaS
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = kOneCluster;
+    attr[1].val.clusterDim.x = static_cast<unsigned>(cluster);
     attr[1].val.clusterDim.y = 1;
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
@@ -267,16 +268,16 @@ static cudaError_t launch_one(const OneParams& prm, int grid, size_t smem, cudaS
 
 // Clusters of the kernel that can be resident at once with `smem` bytes of dynamic shared memory (0 on failure).
 template <int PAIRS>
-static int one_max_clusters(size_t smem) {
+static int one_max_clusters(size_t smem, int cluster) {
     if (cudaFuncSetAttribute(gemv_one_kernel<PAIRS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024) != cudaSuccess) return 0;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(kOneCluster, 1, 1);
+    cfg.gridDim = dim3(static_cast<unsigned>(cluster), 1, 1);
     cfg.blockDim = dim3(kOneThreads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = kOneCluster;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(cluster);
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
@@ -288,17 +289,17 @@ static int one_max_clusters(size_t smem) {
 
 // The same, asked once per device for the two sizes that matter: a CTA small enough for two per SM, and the largest.
 constexpr size_t kOneHalfSm = 112 * 1024;
-static int one_clusters_cached(int pairs, size_t smem) {
-    static std::atomic<int> cache[64][kOneMaxPairs][2];    // 0: not asked yet; idempotent, so a race repeats the query
+static int one_clusters_cached(int pairs, size_t smem, int cluster) {
+    static std::atomic<int> cache[64][kOneMaxPairs][2][2];  // 0: not asked yet; idempotent, so a race repeats the query
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
-    const int cls = smem <= kOneHalfSm ? 0 : 1;
-    int v = cache[dev][pairs - 1][cls].load();
+    const int cls = smem <= kOneHalfSm ? 0 : 1, ci = cluster == kOneCluster ? 0 : 1;
+    int v = cache[dev][pairs - 1][cls][ci].load();
     if (v == 0) {
         const size_t ask = cls == 0 ? kOneHalfSm : 224 * 1024;
-        v = pairs == 1 ? one_max_clusters<1>(ask) : pairs == 2 ? one_max_clusters<2>(ask)
-          : pairs == 3 ? one_max_clusters<3>(ask) : one_max_clusters<4>(ask);
-        cache[dev][pairs - 1][cls].store(v > 0 ? v : -1);
+        v = pairs == 1 ? one_max_clusters<1>(ask, cluster) : pairs == 2 ? one_max_clusters<2>(ask, cluster)
+          : pairs == 3 ? one_max_clusters<3>(ask, cluster) : one_max_clusters<4>(ask, cluster);
+        cache[dev][pairs - 1][cls][ci].store(v > 0 ? v : -1);
     }
     return v > 0 ? v : 0;
 }
@@ -314,7 +315,7 @@ int gemv_one(const void* x, const void* packed, const GroupTable& gt, const void
     for (int j = 0; j < gt.G; ++j) n3 += gt.bits[j] == 3 ? 1 : 0;
     const size_t x_bytes = staged_group_offset(gt.G, n3, 2);
     const int tiles = N >> 4;
-    int pairs = 0;
+    int pairs = 0, cluster = 0;
     size_t smem = 0;
     uint32_t off_z = 0, off_x = 0, off_w = 0;
     for (int pr = 1; pr <= kOneMaxPairs; ++pr) {
@@ -323,9 +324,11 @@ int gemv_one(const void* x, const void* packed, const GroupTable& gt, const void
         const size_t oz = kOneOffS + sz, ox = (oz + sz + 127) / 128 * 128, ow = (ox + x_bytes + 127) / 128 * 128;
         const size_t total = ow + static_cast<size_t>(tpc) * 256 * gt.prefix[gt.G];
         if (total > 224 * 1024) break;
-        const int clusters = one_clusters_cached(pr, total);
-        const int grid = ((tiles + tpc - 1) / tpc + kOneCluster - 1) / kOneCluster * kOneCluster;
-        if (grid <= clusters * kOneCluster) {
+        for (int cs = kOneCluster; cs >= 4 && cluster == 0; cs /= 2) {        // eight CTAs share the staging, or four
+            const int grid = ((tiles + tpc - 1) / tpc + cs - 1) / cs * cs;
+            if (grid <= one_clusters_cached(pr, total, cs) * cs) cluster = cs;
+        }
+        if (cluster != 0) {
             pairs = pr; smem = total;
             off_z = static_cast<uint32_t>(oz); off_x = static_cast<uint32_t>(ox); off_w = static_cast<uint32_t>(ow);
             break;
@@ -348,11 +351,11 @@ int gemv_one(const void* x, const void* packed, const GroupTable& gt, const void
     prm.pre3[0] = 0;
     for (int j = 0; j < SLIM_MAX_GROUPS; ++j)
         prm.pre3[j + 1] = static_cast<uint16_t>(prm.pre3[j] + (j < gt.G && gt.bits[j] == 3 ? 1 : 0));
-    const int grid = ((tiles + 2 * pairs - 1) / (2 * pairs) + kOneCluster - 1) / kOneCluster * kOneCluster;
-    const cudaError_t e = pairs == 1 ? launch_one<1>(prm, grid, smem, stream)
-                        : pairs == 2 ? launch_one<2>(prm, grid, smem, stream)
-                        : pairs == 3 ? launch_one<3>(prm, grid, smem, stream)
-                                     : launch_one<4>(prm, grid, smem, stream);
+    const int grid = ((tiles + 2 * pairs - 1) / (2 * pairs) + cluster - 1) / cluster * cluster;
+    const cudaError_t e = pairs == 1 ? launch_one<1>(prm, grid, cluster, smem, stream)
+                        : pairs == 2 ? launch_one<2>(prm, grid, cluster, smem, stream)
+                        : pairs == 3 ? launch_one<3>(prm, grid, cluster, smem, stream)
+                                     : launch_one<4>(prm, grid, cluster, smem, stream);
     SLIM_CUDA_TRY(e);
     return SLIM_OK;
 }
