@@ -613,7 +613,7 @@ def decode_sweep(layers, M, device, launch, seed=1234):
     if launch == "set":
         layer_set = slim.LayerSet(list(zip(layers, xs, ys)))
         keep.append(layer_set)
-        run, checks, n_dom, n_kern = layer_set.run, [layer_set.check], 1, 2
+        run, checks, n_dom, n_kern = layer_set.run, [layer_set.check], 1, (1 if layer_set.info["resident_pairs"] > 0 else 2)
     elif launch == "per-layer":
         def run():
             for L, x, y in zip(layers, xs, ys):
@@ -630,7 +630,8 @@ def decode_sweep(layers, M, device, launch, seed=1234):
             checks += [qkv.check, gu.check]
             calls += [qkv.run, (lambda i=o: layers[i].forward(xs[i], ws, out=ys[i])), gu.run,
                       (lambda i=down: layers[i].forward(xs[i], ws, out=ys[i]))]
-            n_kern += 2 + 1 + 2 + 1 if M < 4 else 2 + 2 + 2 + 2
+            one = 1 if M < 4 else 2                                  # slim_mpq_gemv: from four tokens on a kernel stages x first
+            n_kern += sum(1 if st.info["resident_pairs"] > 0 else 2 for st in (qkv, gu)) + 2 * one
 
         def run():
             for c in calls:
@@ -679,7 +680,7 @@ def decode_entry(name, layers, spec, device, timer, launch, steps, min_total_s, 
                       "algorithmic_bytes_per_step": alg_bytes, "l2": f"distinct layers, {alg_bytes / 1e9:.2f} GB per step > L2",
                       "launch": {"set": "CUDA graph of the layer-set launch: one persistent kernel for the whole sweep (plus one kernel that stages x)",
                                  "per-layer": "CUDA graph of one slim_mpq_gemv launch per layer (the launch mode of App. B.2), programmatic dependent launch",
-                                 "decoder-order": "CUDA graph; per block: set(q, k, v) on one x, o, set(gate, up) on one x, down: the calls a decoder can issue, in its order"}[launch],
+                                 "decoder-order": "CUDA graph; per block: set(q, k, v) on one x, o, set(gate, up) on one x, down: the calls a decoder can issue, in its order (at one token the q/k/v set is one resident launch, gate/up the ring)"}[launch],
                       "grouped_launch": launch != "per-layer"},
            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
                         "kernel": kernel, "avg_launch_us": per_launch_us, "algorithmic_bytes_per_launch": alg_bytes / n_dom,

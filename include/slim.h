@@ -241,8 +241,13 @@ typedef struct slim_gemv_set_info {
                               persistent CTAs (1 .. 8; layers with few groups get fewer): fp32 partial outputs in the
                               workspace, added in part order by the warp whose part lands last */
     int n_counters;        /* arrival counters of the split row blocks (workspace, cleared by every launch) */
+    int resident_pairs;    /* > 0: a small single-token set that runs as ONE launch with every CTA resident at once (the
+                              whole K of 2 x resident_pairs row tiles per CTA, no ring, no staging kernel); the ring
+                              fields above are then unused.  0: the persistent ring */
+    int resident_cluster;  /* CTAs that share the staging of x in that launch (8 or 4) */
     size_t plan_bytes;
     size_t workspace_bytes;
+    size_t resident_smem;  /* dynamic shared memory of that launch */
 } slim_gemv_set_info;
 
 /* Host-only.  Sizes of the device plan buffer and of the workspace a set needs on the current
@@ -261,7 +266,8 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g,
                        void* plan, size_t plan_bytes, slim_gemv_set_info* info, void* stream);
 
 /* Runs the set: one small kernel puts every layer's activations into fragment order in the
- * workspace, one persistent kernel computes all layers.  `workspace` as for slim_mpq_gemv
+ * workspace, one persistent kernel computes all layers (a small single-token set whose CTAs are all resident at
+ * once runs as one launch instead: slim_gemv_set_info.resident_pairs).  `workspace` as for slim_mpq_gemv
  * (zeroed once with slim_workspace_init; slim_workspace_status reports a device-side time-out). */
 int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan,
                       void* workspace, size_t workspace_bytes, void* stream);

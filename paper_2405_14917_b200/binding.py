@@ -377,7 +377,8 @@ class _SetInfo(ctypes.Structure):
     _fields_ = [("n_layers", ctypes.c_int), ("grid", ctypes.c_int), ("n_slots", ctypes.c_int), ("slot_bytes", ctypes.c_int),
                 ("token_tiles", ctypes.c_int), ("stage_tasks", ctypes.c_int), ("n_items", ctypes.c_int), ("max_bits", ctypes.c_int),
                 ("max_tokens", ctypes.c_int), ("tiles_per_warp", ctypes.c_int), ("split", ctypes.c_int), ("n_counters", ctypes.c_int),
-                ("plan_bytes", ctypes.c_size_t), ("workspace_bytes", ctypes.c_size_t)]
+                ("resident_pairs", ctypes.c_int), ("resident_cluster", ctypes.c_int),
+                ("plan_bytes", ctypes.c_size_t), ("workspace_bytes", ctypes.c_size_t), ("resident_smem", ctypes.c_size_t)]
 
 
 class LayerSet:

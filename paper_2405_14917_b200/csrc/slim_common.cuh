@@ -39,6 +39,16 @@ int gemv_route(const void* x, const void* packed, const uint8_t* bits_host, cons
 int gemv_one(const void* x, const void* packed, const GroupTable& gt, const void* scales, const void* zeros, void* y,
              int M, int N, int K, void* workspace, cudaStream_t stream);
 
+// A set of single-token layers as one resident launch of that kernel (small sets: q/k/v, gate/up).  one_set_plan decides
+// (SLIM_OK: taken, descriptors written into the plan buffer; 1: not taken; negative: error), one_set_launch runs it.
+struct OneSetPlan {
+    int pairs, cluster, grid;
+    size_t smem;
+};
+constexpr size_t kOneSetPlanHeader = 4096;       // CTA ranges of the layers, then the descriptors
+int one_set_plan(const slim_layer* layers, int n_layers, int g, void* plan, size_t plan_bytes, cudaStream_t stream, OneSetPlan* out);
+int one_set_launch(const OneSetPlan& pl, const void* plan, int n_layers, void* workspace, cudaStream_t stream);
+
 // Validates shape arguments and fills the table, for group sizes of 128, 256 and 512 columns (bits_host has K / g
 // entries).  Returns SLIM_OK or an error status; SLIM_ERR_UNSUPPORTED for the group sizes 32 and 64, which have
 // kernels of their own (is_small_group).

@@ -22,6 +22,7 @@
 
 #include <atomic>
 #include <cstring>
+#include <vector>
 
 namespace slim {
 
@@ -31,7 +32,8 @@ constexpr int kOneCluster = 8;                          // CTAs that share the s
 constexpr int kOneMaxPairs = 4;                         // tile pairs per CTA
 constexpr uint32_t kOneOffAbort = 8 * kOneWarps;        // after the warps' barriers
 constexpr uint32_t kOneOffXs = 256;                     // per warp: 128 ints of scratch for the digit staging, later its partial sums
-constexpr uint32_t kOneOffS = kOneOffXs + kOneWarps * 512;
+constexpr uint32_t kOneOffDesc = kOneOffXs + kOneWarps * 512;   // the layer's descriptor, when it comes from the plan buffer of a set
+constexpr uint32_t kOneOffS = kOneOffDesc + 1408;
 
 struct OneParams {
     const __half* x;
@@ -39,7 +41,7 @@ struct OneParams {
     const __half* scales;
     const __half* zeros;
     __half* y;
-    uint8_t* ws;                            // status word at offset 0
+    uint8_t* ws;                            // status word at offset 0 (single-layer launch; a set passes it to the kernel)
     int N, G, gshift;
     int one;                                // 1: a multiplier the compiler cannot fold (selects done as integer multiply-adds)
     uint32_t off_z, off_x, off_w;           // shared-memory offsets: zeros, activation records, slices (scales at kOneOffS)
@@ -47,6 +49,7 @@ struct OneParams {
     uint16_t pre3[SLIM_MAX_GROUPS + 1];     // 3-bit K-tiles before j (their activation records hold two slices)
     uint8_t bits[SLIM_MAX_GROUPS];
 };
+static_assert(sizeof(OneParams) % 16 == 0 && sizeof(OneParams) <= kOneOffS - kOneOffDesc, "descriptors are copied in 16-byte pieces");
 
 __device__ __forceinline__ void st_cluster_u32x4(uint32_t local_addr, uint32_t rank, uint4 v) {
     uint32_t remote;
@@ -127,15 +130,15 @@ __device__ __forceinline__ void one_group(const OneParams& p, uint32_t wj, uint3
     }
 }
 
+// The work of CTA `bid` of layer p (see the head of the file).
 template <int PAIRS>
-__global__ void __launch_bounds__(kOneThreads, PAIRS == 1 ? 2 : 1) gemv_one_kernel(const __grid_constant__ OneParams p) {
-    extern __shared__ __align__(128) uint8_t smem[];
+__device__ __forceinline__ void one_body(const OneParams& p, int bid, uint8_t* status, uint8_t* smem) {
     constexpr int TPC = 2 * PAIRS;                         // tiles per CTA
     const uint32_t sbase = smem_u32(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     volatile int* abort = reinterpret_cast<volatile int*>(smem + kOneOffAbort);
     const uint32_t bar = sbase + 8u * warp;
-    const int tile0 = TPC * blockIdx.x;
+    const int tile0 = TPC * bid;
     const int tiles_here = max(min(TPC, (p.N >> 4) - tile0), 0);  // 0: a CTA that only fills up its cluster
     const int ng = (p.G - warp + kOneWarps - 1) / kOneWarps;      // this warp's K-tiles: warp, warp + 16, ...
     const uint32_t rank = cluster_ctarank();
@@ -221,7 +224,7 @@ __global__ void __launch_bounds__(kOneThreads, PAIRS == 1 ? 2 : 1) gemv_one_kern
     }
     __syncthreads();
     if (*abort != 0) {
-        if (tid == 0) atomicOr(reinterpret_cast<unsigned int*>(p.ws), 1u);
+        if (tid == 0) atomicOr(reinterpret_cast<unsigned int*>(status), 1u);
         return;
     }
     if (tid < 8 * tiles_here) {                            // a pair of rows per thread
@@ -235,6 +238,28 @@ __global__ void __launch_bounds__(kOneThreads, PAIRS == 1 ? 2 : 1) gemv_one_kern
         }
         *reinterpret_cast<__half2*>(p.y + 16 * tile0 + 2 * tid) = __floats2half2_rn(sum.x, sum.y);
     }
+}
+
+template <int PAIRS>
+__global__ void __launch_bounds__(kOneThreads, PAIRS == 1 ? 2 : 1) gemv_one_kernel(const __grid_constant__ OneParams p) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    one_body<PAIRS>(p, static_cast<int>(blockIdx.x), p.ws, smem);
+}
+
+// Several layers in one launch, every CTA resident at once: layer l owns the CTAs cta0[l] .. cta0[l + 1] (whole
+// clusters).  The descriptors live in the plan buffer of the set; a CTA copies its own into shared memory first.
+template <int PAIRS>
+__global__ void __launch_bounds__(kOneThreads, PAIRS == 1 ? 2 : 1) gemv_one_set_kernel(const OneParams* __restrict__ layers,
+                                                                                     const int* __restrict__ cta0, int n_layers,
+                                                                                     uint8_t* status) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    int l = 0;
+    while (l + 1 < n_layers && cta0[l + 1] <= static_cast<int>(blockIdx.x)) ++l;
+    const uint4* src = reinterpret_cast<const uint4*>(layers + l);
+    uint4* dst = reinterpret_cast<uint4*>(smem + kOneOffDesc);
+    for (int i = threadIdx.x; i < static_cast<int>(sizeof(OneParams) / 16); i += kOneThreads) dst[i] = src[i];
+    __syncthreads();
+    one_body<PAIRS>(*reinterpret_cast<const OneParams*>(smem + kOneOffDesc), static_cast<int>(blockIdx.x) - cta0[l], status, smem);
 }
 
 template <int PAIRS>
@@ -304,38 +329,25 @@ static int one_clusters_cached(int pairs, size_t smem, int cluster) {
     return v > 0 ? v : 0;
 }
 
-// Enqueues the layer on the single-token kernel and returns SLIM_OK, a negative status on failure, or 1 if this shape
-// does not fit it (the caller then takes the general kernel): the whole K of a CTA's tiles, their scales and zeros and
-// the digit form of x must fit the shared memory of a CTA, and all CTAs must be resident at once.
-int gemv_one(const void* x, const void* packed, const GroupTable& gt, const void* scales, const void* zeros, void* y,
-             int M, int N, int K, void* workspace, cudaStream_t stream) {
-    (void)K;
-    if (M != 1 || N <= 0 || gt.G < 1) return 1;
+// Shared-memory layout of a CTA with `pairs` tile pairs of a layer; false if it does not fit.
+struct OneShape {
+    size_t smem;
+    uint32_t off_z, off_x, off_w;
+};
+static bool one_shape(const GroupTable& gt, int pairs, OneShape* o) {
     int n3 = 0;
     for (int j = 0; j < gt.G; ++j) n3 += gt.bits[j] == 3 ? 1 : 0;
     const size_t x_bytes = staged_group_offset(gt.G, n3, 2);
-    const int tiles = N >> 4;
-    int pairs = 0, cluster = 0;
-    size_t smem = 0;
-    uint32_t off_z = 0, off_x = 0, off_w = 0;
-    for (int pr = 1; pr <= kOneMaxPairs; ++pr) {
-        const int tpc = 2 * pr;
-        const size_t sz = static_cast<size_t>(gt.G) * 32 * tpc;
-        const size_t oz = kOneOffS + sz, ox = (oz + sz + 127) / 128 * 128, ow = (ox + x_bytes + 127) / 128 * 128;
-        const size_t total = ow + static_cast<size_t>(tpc) * 256 * gt.prefix[gt.G];
-        if (total > 224 * 1024) break;
-        for (int cs = kOneCluster; cs >= 4 && cluster == 0; cs /= 2) {        // eight CTAs share the staging, or four
-            const int grid = ((tiles + tpc - 1) / tpc + cs - 1) / cs * cs;
-            if (grid <= one_clusters_cached(pr, total, cs) * cs) cluster = cs;
-        }
-        if (cluster != 0) {
-            pairs = pr; smem = total;
-            off_z = static_cast<uint32_t>(oz); off_x = static_cast<uint32_t>(ox); off_w = static_cast<uint32_t>(ow);
-            break;
-        }
-    }
-    if (pairs == 0) return 1;
-    OneParams prm;
+    const int tpc = 2 * pairs;
+    const size_t sz = static_cast<size_t>(gt.G) * 32 * tpc;
+    const size_t oz = kOneOffS + sz, ox = (oz + sz + 127) / 128 * 128, ow = (ox + x_bytes + 127) / 128 * 128;
+    o->smem = ow + static_cast<size_t>(tpc) * 256 * gt.prefix[gt.G];
+    o->off_z = static_cast<uint32_t>(oz); o->off_x = static_cast<uint32_t>(ox); o->off_w = static_cast<uint32_t>(ow);
+    return o->smem <= 224 * 1024;
+}
+static void one_fill(OneParams* out, const void* x, const void* packed, const void* scales, const void* zeros, void* y, void* workspace,
+                     int N, const GroupTable& gt, const OneShape& sh) {
+    OneParams& prm = *out;
     memset(&prm, 0, sizeof prm);
     prm.x = static_cast<const __half*>(x);
     prm.packed = static_cast<const uint8_t*>(packed);
@@ -345,17 +357,130 @@ int gemv_one(const void* x, const void* packed, const GroupTable& gt, const void
     prm.ws = static_cast<uint8_t*>(workspace);
     prm.N = N; prm.G = gt.G; prm.gshift = gt.gshift;
     prm.one = 1;
-    prm.off_z = off_z; prm.off_x = off_x; prm.off_w = off_w;
+    prm.off_z = sh.off_z; prm.off_x = sh.off_x; prm.off_w = sh.off_w;
     memcpy(prm.prefix, gt.prefix, sizeof prm.prefix);
     memcpy(prm.bits, gt.bits, sizeof prm.bits);
     prm.pre3[0] = 0;
     for (int j = 0; j < SLIM_MAX_GROUPS; ++j)
         prm.pre3[j + 1] = static_cast<uint16_t>(prm.pre3[j] + (j < gt.G && gt.bits[j] == 3 ? 1 : 0));
-    const int grid = ((tiles + 2 * pairs - 1) / (2 * pairs) + cluster - 1) / cluster * cluster;
-    const cudaError_t e = pairs == 1 ? launch_one<1>(prm, grid, cluster, smem, stream)
-                        : pairs == 2 ? launch_one<2>(prm, grid, cluster, smem, stream)
-                        : pairs == 3 ? launch_one<3>(prm, grid, cluster, smem, stream)
-                                     : launch_one<4>(prm, grid, cluster, smem, stream);
+}
+static int pad_to(int v, int m) { return (v + m - 1) / m * m; }
+
+// Enqueues the layer on the single-token kernel and returns SLIM_OK, a negative status on failure, or 1 if this shape
+// does not fit it (the caller then takes the general kernel): the whole K of a CTA's tiles, their scales and zeros and
+// the digit form of x must fit the shared memory of a CTA.  Among the tile counts that fit, the one that needs the
+// fewest waves of resident CTAs is taken (one wave for the decode shapes of 7B and 13B models), the smallest of equals.
+int gemv_one(const void* x, const void* packed, const GroupTable& gt, const void* scales, const void* zeros, void* y,
+             int M, int N, int K, void* workspace, cudaStream_t stream) {
+    (void)K;
+    if (M != 1 || N <= 0 || gt.G < 1) return 1;
+    const int tiles = N >> 4;
+    int pairs = 0, cluster = 0, best_waves = 1 << 30;
+    OneShape shape;
+    for (int pr = 1; pr <= kOneMaxPairs; ++pr) {
+        OneShape sh;
+        if (!one_shape(gt, pr, &sh)) break;
+        for (int cs = kOneCluster; cs >= 4; cs /= 2) {                         // eight CTAs share the staging, or four
+            const int grid = pad_to((tiles + 2 * pr - 1) / (2 * pr), cs), resident = one_clusters_cached(pr, sh.smem, cs) * cs;
+            if (resident <= 0) continue;
+            const int waves = (grid + resident - 1) / resident;
+            if (waves < best_waves) { best_waves = waves; pairs = pr; cluster = cs; shape = sh; }
+        }
+        if (best_waves == 1) break;
+    }
+    if (pairs == 0) return 1;
+    OneParams prm;
+    one_fill(&prm, x, packed, scales, zeros, y, workspace, N, gt, shape);
+    const int grid = pad_to((tiles + 2 * pairs - 1) / (2 * pairs), cluster);
+    const cudaError_t e = pairs == 1 ? launch_one<1>(prm, grid, cluster, shape.smem, stream)
+                        : pairs == 2 ? launch_one<2>(prm, grid, cluster, shape.smem, stream)
+                        : pairs == 3 ? launch_one<3>(prm, grid, cluster, shape.smem, stream)
+                                     : launch_one<4>(prm, grid, cluster, shape.smem, stream);
+    SLIM_CUDA_TRY(e);
+    return SLIM_OK;
+}
+
+// ------------------------------------------------------------------------------------------ small single-token sets, resident
+// A set of single-token layers whose CTAs are all resident at once (q/k/v, gate/up: a few layers) runs as ONE launch of
+// the kernel above instead of the staging kernel plus the persistent ring: no ring to fill and drain, no second kernel.
+constexpr int kOneSetMaxLayers = 64;
+
+template <int PAIRS>
+static cudaError_t launch_one_set(const OneSetPlan& pl, const void* plan, int n_layers, void* workspace, cudaStream_t stream) {
+    static std::atomic<bool> attr_set[64];    // zero-initialised; set-up is idempotent, so a race repeats it harmlessly
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        e = cudaFuncSetAttribute(gemv_one_set_kernel<PAIRS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(static_cast<unsigned>(pl.grid), 1, 1);
+    cfg.blockDim = dim3(kOneThreads, 1, 1);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = static_cast<unsigned>(pl.cluster);
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    const uint8_t* base = static_cast<const uint8_t*>(plan);
+    return cudaLaunchKernelEx(&cfg, gemv_one_set_kernel<PAIRS>, reinterpret_cast<const OneParams*>(base + kOneSetPlanHeader),
+                              reinterpret_cast<const int*>(base), n_layers, static_cast<uint8_t*>(workspace));
+}
+
+int one_set_plan(const slim_layer* layers, int n_layers, int g, void* plan, size_t plan_bytes, cudaStream_t stream, OneSetPlan* out) {
+    if (n_layers < 1 || n_layers > kOneSetMaxLayers || g < SLIM_GROUP) return 1;
+    if (plan_bytes < kOneSetPlanHeader + static_cast<size_t>(n_layers) * sizeof(OneParams)) return 1;
+    std::vector<GroupTable> gt(static_cast<size_t>(n_layers));
+    for (int l = 0; l < n_layers; ++l) {
+        if (layers[l].M != 1) return 1;
+        const int st = make_group_table(layers[l].N, layers[l].K, g, layers[l].bits_host, &gt[l]);
+        if (st != SLIM_OK) return st;
+    }
+    for (int pr = 1; pr <= kOneMaxPairs; ++pr) {
+        OneShape sh[kOneSetMaxLayers];
+        size_t smem = 0;
+        bool fits = true;
+        for (int l = 0; l < n_layers && fits; ++l) {
+            fits = one_shape(gt[l], pr, &sh[l]);
+            smem = smem > sh[l].smem ? smem : sh[l].smem;
+        }
+        if (!fits) break;
+        for (int cs = kOneCluster; cs >= 4; cs /= 2) {
+            int cta0[kOneSetMaxLayers + 1];
+            cta0[0] = 0;
+            for (int l = 0; l < n_layers; ++l) cta0[l + 1] = cta0[l] + pad_to(((layers[l].N >> 4) + 2 * pr - 1) / (2 * pr), cs);
+            if (cta0[n_layers] > one_clusters_cached(pr, smem, cs) * cs) continue;
+            // taken: descriptors and CTA ranges into the plan buffer (pageable sources are staged before the copies return)
+            std::vector<OneParams> prm(static_cast<size_t>(n_layers));
+            for (int l = 0; l < n_layers; ++l)
+                one_fill(&prm[l], layers[l].x, layers[l].packed, layers[l].scales, layers[l].zeros, layers[l].y, nullptr, layers[l].N, gt[l], sh[l]);
+            uint8_t* base = static_cast<uint8_t*>(plan);
+            SLIM_CUDA_TRY(cudaMemcpyAsync(base, cta0, static_cast<size_t>(n_layers + 1) * sizeof(int), cudaMemcpyHostToDevice, stream));
+            SLIM_CUDA_TRY(cudaMemcpyAsync(base + kOneSetPlanHeader, prm.data(), static_cast<size_t>(n_layers) * sizeof(OneParams), cudaMemcpyHostToDevice, stream));
+            out->pairs = pr; out->cluster = cs; out->grid = cta0[n_layers]; out->smem = smem;
+            return SLIM_OK;
+        }
+    }
+    return 1;
+}
+
+int one_set_launch(const OneSetPlan& pl, const void* plan, int n_layers, void* workspace, cudaStream_t stream) {
+    if (pl.pairs < 1 || pl.pairs > kOneMaxPairs || (pl.cluster != 4 && pl.cluster != kOneCluster) || pl.grid < pl.cluster ||
+        pl.grid % pl.cluster != 0 || pl.smem > 224 * 1024 || n_layers < 1 || n_layers > kOneSetMaxLayers)
+        return SLIM_ERR_INVALID_ARG;
+    const cudaError_t e = pl.pairs == 1 ? launch_one_set<1>(pl, plan, n_layers, workspace, stream)
+                        : pl.pairs == 2 ? launch_one_set<2>(pl, plan, n_layers, workspace, stream)
+                        : pl.pairs == 3 ? launch_one_set<3>(pl, plan, n_layers, workspace, stream)
+                                        : launch_one_set<4>(pl, plan, n_layers, workspace, stream);
     SLIM_CUDA_TRY(e);
     return SLIM_OK;
 }

@@ -997,6 +997,29 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g, void*
     uint8_t* plan_dev = static_cast<uint8_t*>(plan);
 
     try {                       // the host-side lists may fail to allocate: reported as a status
+    // A single-token set small enough for all its CTAs to be resident at once runs as one launch without a ring.
+    if (sg.mmax == 1) {
+        slim::OneSetPlan op;
+        const int taken = slim::one_set_plan(layers_host, n_layers, g, plan, plan_bytes, s, &op);
+        if (taken < 0) return taken;
+        if (taken == SLIM_OK) {
+            memset(info, 0, sizeof *info);
+            info->n_layers = n_layers;
+            info->grid = op.grid;
+            info->token_tiles = 1;
+            info->max_bits = sg.bmax;
+            info->max_tokens = 1;
+            info->tiles_per_warp = 2;
+            info->split = 1;
+            info->n_items = op.grid;
+            info->resident_pairs = op.pairs;
+            info->resident_cluster = op.cluster;
+            info->resident_smem = op.smem;
+            info->plan_bytes = slim::set_plan_bytes(n_layers, sg.n_items);
+            info->workspace_bytes = 256;
+            return SLIM_OK;
+        }
+    }
     // Second pass: descriptors and items.  The copies below read host memory that goes out of scope:
     // pageable sources are staged before cudaMemcpyAsync returns.
     static_assert((slim::kSetMaxGrid + 1) * sizeof(int) <= slim::kSetPlanHeader, "item ranges fit the plan header");
@@ -1125,6 +1148,15 @@ int slim_selftest_wait_timeout(void* workspace, size_t workspace_bytes, unsigned
 }
 
 int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* workspace, size_t workspace_bytes, void* stream) {
+    if (info != nullptr && info->resident_pairs > 0) {
+        if (plan == nullptr) return SLIM_ERR_INVALID_ARG;
+        if (!slim::aligned16(plan)) return SLIM_ERR_ALIGNMENT;
+        if (workspace == nullptr || workspace_bytes < 256) return SLIM_ERR_WORKSPACE;
+        if (!slim::aligned16(workspace)) return SLIM_ERR_ALIGNMENT;
+        slim::OneSetPlan op;
+        op.pairs = info->resident_pairs; op.cluster = info->resident_cluster; op.grid = info->grid; op.smem = info->resident_smem;
+        return slim::one_set_launch(op, plan, info->n_layers, workspace, static_cast<cudaStream_t>(stream));
+    }
     slim::SetParams prm;
     size_t smem = 0;
     const int st = slim::set_params(info, plan, workspace, workspace_bytes, &prm, &smem);

@@ -138,6 +138,35 @@ def test_llama70b_block_as_one_layer_set(M):
                      f"set, 70B {name} {L['N']}x{L['K']} M={M}")
 
 
+def test_projections_of_a_block_as_small_single_token_sets():
+    """The small sets a decoder issues at one token.  q/k/v (three 4096 x 4096 layers on one x) fit the GPU as one
+    wave of resident CTAs and run as a single launch; gate/up (two 11008 x 4096 layers) are too many CTAs for that
+    and take the persistent ring with their row blocks cut into parts, which the last-arriving part adds up."""
+    slim = _slim()
+    rng = np.random.default_rng(404)
+    for shapes, resident in (([(4096, 4096)] * 3, True), ([(11008, 4096)] * 2, False)):
+        x = _x(rng, 1, 4096)
+        xd = torch.from_numpy(x).cuda()
+        entries = []
+        for i, (N, K) in enumerate(shapes):
+            entries.append((_device_layer(N, K, 2 + (i & 1)), xd, torch.full((1, N), float("nan"), dtype=torch.float16, device="cuda")))
+        s = slim.LayerSet(entries)
+        assert (s.info["resident_pairs"] > 0) == resident
+        if not resident:
+            assert s.info["split"] > 1 and s.info["n_counters"] > 0
+        for _ in range(2):                       # twice: the arrival counters start every launch at zero
+            for (_, _, y) in entries:
+                y.fill_(float("nan"))
+            s.run()
+            s.check()
+            for i, ((N, K), (_, _, y)) in enumerate(zip(shapes, entries)):
+                L = _layer(N, K, 2 + (i & 1))
+                y = y.cpu().numpy()
+                assert np.isfinite(y.astype(np.float64)).all()
+                rows = _sample_rows(N, rng, 120)
+                check_output(y[:, rows], orc.linear_rows_f64(x, L["codes"], L["scales"], L["zeros"], rows), f"{N}x{K} layer {i}")
+
+
 @pytest.mark.parametrize("M", [1, 4, 8, 16])
 def test_llama7b_avg3_layer_set_all_token_counts(M):
     """LLaMA-7B shapes at avg 3 bits (bit-widths 2, 3, 4) through the layer-set launch, for every token count of

@@ -48,9 +48,24 @@ def test_mixed_shapes_one_token():
               oracle_layer(1040, 512, 2, 1, block=4)]
     ys, s = _run_set(layers)
     _check_all(layers, ys, "one token")
+    # a single-token set this small runs as one launch with every CTA resident at once: whole clusters per layer,
+    # 2 x resident_pairs tiles of 16 rows per CTA
+    assert s.info["resident_pairs"] > 0 and s.info["resident_cluster"] in (4, 8)
+    rows = 32 * s.info["resident_pairs"]
+    cs = s.info["resident_cluster"]
+    assert s.info["grid"] == sum(-(-(-(-L["N"] // rows)) // cs) * cs for L in layers)
+
+
+def test_small_set_of_several_tokens_cuts_its_row_blocks_into_parts():
+    # the same shapes with two tokens somewhere: the persistent ring, and a set this small cuts the groups of its row
+    # blocks into parts (fewer for the layers with few groups)
+    layers = [oracle_layer(512, 1024, 2, 2, block=0), oracle_layer(272, 1408, 3, 1, block=1),
+              oracle_layer(128, 128, 2, 1, block=2), oracle_layer(16, 256, 3, 2, block=3),
+              oracle_layer(1040, 512, 2, 1, block=4)]
+    ys, s = _run_set(layers)
+    _check_all(layers, ys, "two tokens")
     rows = 128 * s.info["tiles_per_warp"]           # rows of a work item
-    # a set this small cuts the groups of its row blocks into parts (fewer for the layers with few groups)
-    assert s.info["split"] > 1
+    assert s.info["resident_pairs"] == 0 and s.info["split"] > 1
     parts = [min(s.info["split"], max(L["K"] // 128 // 4, 1)) for L in layers]
     assert s.info["n_items"] == sum(k * -(-L["N"] // rows) for k, L in zip(parts, layers))
 
