@@ -445,7 +445,11 @@ int one_set_plan(const slim_layer* layers, int n_layers, int g, void* plan, size
         const int st = make_group_table(layers[l].N, layers[l].K, g, layers[l].bits_host, &gt[l]);
         if (st != SLIM_OK) return st;
     }
-    for (int pr = 1; pr <= kOneMaxPairs; ++pr) {
+    // one wave of resident CTAs; a set of at most four layers may take two (it is still ahead of filling and draining a ring)
+    // (then with the largest tile count that fits, which needs the fewest CTAs)
+    for (int waves = 1; waves <= (n_layers <= 4 ? 2 : 1); ++waves)
+    for (int step = 1; step <= kOneMaxPairs; ++step) {
+        const int pr = waves == 1 ? step : kOneMaxPairs + 1 - step;
         OneShape sh[kOneSetMaxLayers];
         size_t smem = 0;
         bool fits = true;
@@ -453,12 +457,12 @@ int one_set_plan(const slim_layer* layers, int n_layers, int g, void* plan, size
             fits = one_shape(gt[l], pr, &sh[l]);
             smem = smem > sh[l].smem ? smem : sh[l].smem;
         }
-        if (!fits) break;
+        if (!fits) { if (waves == 1) break; else continue; }
         for (int cs = kOneCluster; cs >= 4; cs /= 2) {
             int cta0[kOneSetMaxLayers + 1];
             cta0[0] = 0;
             for (int l = 0; l < n_layers; ++l) cta0[l + 1] = cta0[l] + pad_to(((layers[l].N >> 4) + 2 * pr - 1) / (2 * pr), cs);
-            if (cta0[n_layers] > one_clusters_cached(pr, smem, cs) * cs) continue;
+            if (cta0[n_layers] > waves * one_clusters_cached(pr, smem, cs) * cs) continue;
             // taken: descriptors and CTA ranges into the plan buffer (pageable sources are staged before the copies return)
             std::vector<OneParams> prm(static_cast<size_t>(n_layers));
             for (int l = 0; l < n_layers; ++l)

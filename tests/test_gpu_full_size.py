@@ -140,16 +140,18 @@ def test_llama70b_block_as_one_layer_set(M):
 
 def test_projections_of_a_block_as_small_single_token_sets():
     """The small sets a decoder issues at one token.  q/k/v (three 4096 x 4096 layers on one x) fit the GPU as one
-    wave of resident CTAs and run as a single launch; gate/up (two 11008 x 4096 layers) are too many CTAs for that
-    and take the persistent ring with their row blocks cut into parts, which the last-arriving part adds up."""
+    wave of resident CTAs and run as a single launch; gate/up (two 11008 x 4096 layers) take two waves of it; six
+    11008 x 4096 layers are too many CTAs for that and too few row blocks for the persistent ring as it is, so their
+    row blocks are cut into parts, which the last-arriving part adds up."""
     slim = _slim()
     rng = np.random.default_rng(404)
-    for shapes, resident in (([(4096, 4096)] * 3, True), ([(11008, 4096)] * 2, False)):
-        x = _x(rng, 1, 4096)
-        xd = torch.from_numpy(x).cuda()
-        entries = []
+    for shapes, resident in (([(4096, 4096)] * 3, True), ([(11008, 4096)] * 2, True), ([(11008, 4096)] * 6, False)):
+        entries, xs = [], []
         for i, (N, K) in enumerate(shapes):
-            entries.append((_device_layer(N, K, 2 + (i & 1)), xd, torch.full((1, N), float("nan"), dtype=torch.float16, device="cuda")))
+            x = _x(rng, 1, K) if (i == 0 or len(shapes) > 3) else xs[0]          # q/k/v and gate/up share their input
+            xs.append(x)
+            entries.append((_device_layer(N, K, 2 + (i & 1)), torch.from_numpy(x).cuda(),
+                            torch.full((1, N), float("nan"), dtype=torch.float16, device="cuda")))
         s = slim.LayerSet(entries)
         assert (s.info["resident_pairs"] > 0) == resident
         if not resident:
@@ -164,7 +166,7 @@ def test_projections_of_a_block_as_small_single_token_sets():
                 y = y.cpu().numpy()
                 assert np.isfinite(y.astype(np.float64)).all()
                 rows = _sample_rows(N, rng, 120)
-                check_output(y[:, rows], orc.linear_rows_f64(x, L["codes"], L["scales"], L["zeros"], rows), f"{N}x{K} layer {i}")
+                check_output(y[:, rows], orc.linear_rows_f64(xs[i], L["codes"], L["scales"], L["zeros"], rows), f"{N}x{K} layer {i}")
 
 
 @pytest.mark.parametrize("M", [1, 4, 8, 16])
