@@ -9,7 +9,7 @@
 // These group sizes trade a fifth to a half more scale and zero-point bytes for accuracy; they are served by plain
 // CUDA-core kernels (one FMA per weight and token), not by the tensor-core kernels of the 128-column tiles:
 //   pack_small_kernel, dequant_small_kernel   one thread per item / per 8 outputs, bit-exact
-//   gemv_small_kernel (1 <= M <= 16)          a block per 16-row tile, the groups dealt to its 8 warps, fp32 accumulation
+//   gemv_small_kernel (1 <= M <= 16)          a block per 16-row tile, the groups dealt to its 16 warps, fp32 accumulation
 //   M > 16                                    the weights are materialised as fp16 in the workspace (dequant_small_kernel)
 //                                             and multiplied by dense_f16_kernel (mma.sync, fp32 accumulation)
 #include "slim_common.cuh"
@@ -114,16 +114,50 @@ __global__ void __launch_bounds__(256) dequant_small_kernel(const uint8_t* __res
     *reinterpret_cast<uint4*>(W + static_cast<size_t>(row) * K + k0) = *reinterpret_cast<const uint4*>(out);
 }
 
-// The codes of one lane (rows 2gq, 2gq + 1, its T/4 columns) from the W units of a width-W slice that start at `unit0`.
-template <int T, int W>
-__device__ __forceinline__ void small_decode(const uint8_t* __restrict__ unit0, int lo, uint32_t (&q)[2][T / 4]) {
+// ------------------------------------------------------------------------------------------ decode path, 1 <= M <= 16
+// A block of 16 warps per 16-row tile; warp w takes the groups w, w + 16, ...; lane 4*gq + c holds the items of rows
+// 2gq, 2gq + 1 for the column range c of the group, decodes its T/4 codes per row and multiplies them with the
+// tokens' activations (fp32 FMAs); per (row, group) acc += s * (sum_k q x - z * sum_k x).  The four lanes of a row
+// pair are added by shuffles, the sixteen warps through shared memory, in a fixed order.
+// The kernel is a chain of small loads, so a group's bytes (its b units, both rows of a lane in one load, and the
+// scale and zero-point pairs) are requested one group ahead of their use.
+constexpr int kSmallWarps = 16;
+
+template <int T>
+struct SmallRaw {
+    uint32_t unit[4];      // the lane's items of rows 2gq (low part) and 2gq + 1 of up to four units
+    uint32_t s2, z2;       // scales and zero points of the two rows (half2)
+    int b;
+};
+template <int T>
+__device__ __forceinline__ SmallRaw<T> small_load(const uint8_t* __restrict__ packed, const __half* __restrict__ scales,
+                                                  const __half* __restrict__ zeros, int N, const SmallTable& st, int j, int t, int lane,
+                                                  int row0) {
     typedef typename SmallItem<T>::type item_t;
-    constexpr int NF = T / 4 / W;
+    SmallRaw<T> r;
+    r.b = st.bits[j];
+    const uint8_t* base = packed + small_item_offset<T>(N, st, j, t, 0, lane, 0);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        r.unit[u] = 0u;
+        if (u < r.b) {
+            if (sizeof(item_t) == 1) r.unit[u] = *reinterpret_cast<const uint16_t*>(base + 2 * T * u);
+            else r.unit[u] = *reinterpret_cast<const uint32_t*>(base + 2 * T * u);
+        }
+    }
+    r.s2 = *reinterpret_cast<const uint32_t*>(scales + static_cast<size_t>(j) * N + row0);
+    r.z2 = *reinterpret_cast<const uint32_t*>(zeros + static_cast<size_t>(j) * N + row0);
+    return r;
+}
+// The codes of one lane (rows 2gq, 2gq + 1, its T/4 columns) from the W units of a width-W slice that start at unit `u0`.
+template <int T, int W>
+__device__ __forceinline__ void small_decode(const SmallRaw<T>& raw, int u0, int lo, uint32_t (&q)[2][T / 4]) {
+    typedef typename SmallItem<T>::type item_t;
+    constexpr int NF = T / 4 / W, IB = 8 * sizeof(item_t);
     constexpr uint32_t kMask = (1u << W) - 1u;
 #pragma unroll
     for (int u = 0; u < W; ++u) {
-        const uint32_t i0 = *reinterpret_cast<const item_t*>(unit0 + 2 * T * u);
-        const uint32_t i1 = *reinterpret_cast<const item_t*>(unit0 + 2 * T * u + T / 32);
+        const uint32_t i0 = raw.unit[u0 + u] & ((1u << IB) - 1u), i1 = raw.unit[u0 + u] >> IB;
 #pragma unroll
         for (int f = 0; f < NF; ++f) {
             q[0][NF * u + f] |= ((i0 >> (W * f)) & kMask) << lo;
@@ -132,17 +166,13 @@ __device__ __forceinline__ void small_decode(const uint8_t* __restrict__ unit0, 
     }
 }
 
-// ------------------------------------------------------------------------------------------ decode path, 1 <= M <= 16
-// A block of 8 warps per 16-row tile; warp w takes the groups w, w + 8, ...; lane 4*gq + c holds the items of rows
-// 2gq, 2gq + 1 for the column range c of the group, decodes its T/4 codes per row and multiplies them with the
-// tokens' activations (fp32 FMAs); per (row, group) acc += s * (sum_k q x - z * sum_k x).  The four lanes of a row
-// pair are added by shuffles, the eight warps through shared memory, in a fixed order.
 template <int T, int MT>     // MT: tokens handled per pass (the block loops over the token tiles)
-__global__ void __launch_bounds__(256) gemv_small_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ packed,
-                                                         const __half* __restrict__ scales, const __half* __restrict__ zeros,
-                                                         __half* __restrict__ y, int M, int N, int K, const __grid_constant__ SmallTable st) {
+__global__ void __launch_bounds__(32 * kSmallWarps, MT == 1 ? 2 : 1) gemv_small_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ packed,
+                                                                      const __half* __restrict__ scales, const __half* __restrict__ zeros,
+                                                                      __half* __restrict__ y, int M, int N, int K,
+                                                                      const __grid_constant__ SmallTable st) {
     constexpr int C = T / 4;                               // columns per lane
-    __shared__ float red[8][MT][16];
+    __shared__ float red[kSmallWarps][MT][16];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gq = lane >> 2, c = lane & 3;
     const int t = blockIdx.x;
@@ -151,34 +181,44 @@ __global__ void __launch_bounds__(256) gemv_small_kernel(const __half* __restric
         float acc[MT][2];
 #pragma unroll
         for (int m = 0; m < MT; ++m) acc[m][0] = acc[m][1] = 0.f;
-        for (int j = warp; j < st.G; j += 8) {
-            const int b = st.bits[j];
+        SmallRaw<T> next;
+        if (warp < st.G) next = small_load<T>(packed, scales, zeros, N, st, warp, t, lane, row0);
+        for (int j = warp; j < st.G; j += kSmallWarps) {
+            const SmallRaw<T> raw = next;
+            if (j + kSmallWarps < st.G) next = small_load<T>(packed, scales, zeros, N, st, j + kSmallWarps, t, lane, row0);
             uint32_t q[2][C];
 #pragma unroll
             for (int i = 0; i < C; ++i) q[0][i] = q[1][i] = 0u;
-            const uint8_t* tile = packed + small_item_offset<T>(N, st, j, t, 0, lane, 0);
-            switch (b) {
-                case 1: small_decode<T, 1>(tile, 0, q); break;
-                case 2: small_decode<T, 2>(tile, 0, q); break;
-                case 3: small_decode<T, 2>(tile, 0, q); small_decode<T, 1>(tile + 2 * (2 * T), 2, q); break;
-                default: small_decode<T, 4>(tile, 0, q); break;
+            switch (raw.b) {
+                case 1: small_decode<T, 1>(raw, 0, 0, q); break;
+                case 2: small_decode<T, 2>(raw, 0, 0, q); break;
+                case 3: small_decode<T, 2>(raw, 0, 0, q); small_decode<T, 1>(raw, 2, 2, q); break;
+                default: small_decode<T, 4>(raw, 0, 0, q); break;
             }
-            const float s0 = __half2float(scales[static_cast<size_t>(j) * N + row0]), s1 = __half2float(scales[static_cast<size_t>(j) * N + row0 + 1]);
-            const float z0 = __half2float(zeros[static_cast<size_t>(j) * N + row0]), z1 = __half2float(zeros[static_cast<size_t>(j) * N + row0 + 1]);
+            const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&raw.s2));
+            const float2 zf = __half22float2(*reinterpret_cast<const __half2*>(&raw.z2));
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
                 if (m0 + m >= M) break;
-                const __half* xp = x + static_cast<size_t>(m0 + m) * K + T * j + C * c;
+                const uint4* xp = reinterpret_cast<const uint4*>(x + static_cast<size_t>(m0 + m) * K + T * j + C * c);
                 float d0 = 0.f, d1 = 0.f, sx = 0.f;
 #pragma unroll
-                for (int i = 0; i < C; ++i) {
-                    const float xv = __half2float(xp[i]);
-                    d0 = fmaf(static_cast<float>(q[0][i]), xv, d0);
-                    d1 = fmaf(static_cast<float>(q[1][i]), xv, d1);
-                    sx += xv;
+                for (int v = 0; v < C / 8; ++v) {
+                    const uint4 xv4 = xp[v];
+                    const uint32_t w4[4] = {xv4.x, xv4.y, xv4.z, xv4.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float2 xv = __half22float2(*reinterpret_cast<const __half2*>(&w4[i]));
+                        d0 = fmaf(static_cast<float>(q[0][8 * v + 2 * i]), xv.x, d0);
+                        d1 = fmaf(static_cast<float>(q[1][8 * v + 2 * i]), xv.x, d1);
+                        d0 = fmaf(static_cast<float>(q[0][8 * v + 2 * i + 1]), xv.y, d0);
+                        d1 = fmaf(static_cast<float>(q[1][8 * v + 2 * i + 1]), xv.y, d1);
+                        sx += xv.x;
+                        sx += xv.y;
+                    }
                 }
-                acc[m][0] = fmaf(s0, fmaf(-z0, sx, d0), acc[m][0]);
-                acc[m][1] = fmaf(s1, fmaf(-z1, sx, d1), acc[m][1]);
+                acc[m][0] = fmaf(sf.x, fmaf(-zf.x, sx, d0), acc[m][0]);
+                acc[m][1] = fmaf(sf.y, fmaf(-zf.y, sx, d1), acc[m][1]);
             }
         }
 #pragma unroll
@@ -197,7 +237,7 @@ __global__ void __launch_bounds__(256) gemv_small_kernel(const __half* __restric
             if (m0 + m < M) {
                 float v = 0.f;
 #pragma unroll
-                for (int k = 0; k < 8; ++k) v += red[k][m][r];
+                for (int k = 0; k < kSmallWarps; ++k) v += red[k][m][r];
                 y[static_cast<size_t>(m0 + m) * N + 16 * t + r] = __float2half_rn(v);
             }
         }
@@ -326,11 +366,13 @@ int small_linear(const void* x, const void* packed, const uint8_t* bits_host, co
     if (M <= SLIM_GEMV_MAX_M) {
         const unsigned grid = static_cast<unsigned>(N / 16);
         if (g == 32) {
-            if (M <= 4) gemv_small_kernel<32, 4><<<grid, 256, 0, s>>>(xh, pk, sc, zp, yh, M, N, K, st);
-            else gemv_small_kernel<32, 8><<<grid, 256, 0, s>>>(xh, pk, sc, zp, yh, M, N, K, st);
+            if (M == 1) gemv_small_kernel<32, 1><<<grid, 32 * kSmallWarps, 0, s>>>(xh, pk, sc, zp, yh, M, N, K, st);
+            else if (M <= 4) gemv_small_kernel<32, 4><<<grid, 32 * kSmallWarps, 0, s>>>(xh, pk, sc, zp, yh, M, N, K, st);
+            else gemv_small_kernel<32, 8><<<grid, 32 * kSmallWarps, 0, s>>>(xh, pk, sc, zp, yh, M, N, K, st);
         } else {
-            if (M <= 4) gemv_small_kernel<64, 4><<<grid, 256, 0, s>>>(xh, pk, sc, zp, yh, M, N, K, st);
-            else gemv_small_kernel<64, 8><<<grid, 256, 0, s>>>(xh, pk, sc, zp, yh, M, N, K, st);
+            if (M == 1) gemv_small_kernel<64, 1><<<grid, 32 * kSmallWarps, 0, s>>>(xh, pk, sc, zp, yh, M, N, K, st);
+            else if (M <= 4) gemv_small_kernel<64, 4><<<grid, 32 * kSmallWarps, 0, s>>>(xh, pk, sc, zp, yh, M, N, K, st);
+            else gemv_small_kernel<64, 8><<<grid, 32 * kSmallWarps, 0, s>>>(xh, pk, sc, zp, yh, M, N, K, st);
         }
         SLIM_CUDA_TRY(cudaGetLastError());
         return SLIM_OK;
