@@ -150,7 +150,8 @@ int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host,
                   int M, int N, int K, int g,
                   void* workspace, size_t workspace_bytes, void* stream);
 
-/* Host-only introspection: the launch plan slim_mpq_gemv uses for this shape on the current device
+/* Host-only introspection: the launch plan of slim_mpq_gemv's general kernel (M >= 2, and the single-token layers whose
+ * K does not fit the single-token kernel) for this shape on the current device
  * (148 SMs assumed when no device is present).  out6 = {16-row tiles per CTA, k-slices =
  * cluster size, row blocks, dynamic shared memory bytes, 8-token MMA tiles, groups per chunk}.
  * grid = k-slices x row blocks, 8 warps per CTA. */
