@@ -36,6 +36,16 @@ def test_small_layers_all_token_counts(N, K, avg, M):
     check_output(y, y_ref, f"{N}x{K} avg{avg} M={M}")
 
 
+@pytest.mark.parametrize("N,K", [(16, 128), (16, 2048), (48, 32768), (2064, 256), (4736, 1024)])
+def test_single_token_edge_shapes(N, K):
+    """One token at the edges of the single-token kernel: a single tile and a single group; a K of 256 groups whose
+    digit form does not fit a CTA (the general kernel takes it); row counts that leave a CTA with one tile of its pair
+    and pad the grid to whole clusters; more CTAs than one tile pair each lets be resident (several pairs per CTA)."""
+    L = oracle_layer(N, K, 2, 1, seed_name="one-token-edges")
+    y = _run(L)
+    check_output(y, orc.linear_f64(L["x"], L["codes"], L["scales"], L["zeros"]), f"{N}x{K}")
+
+
 @pytest.mark.parametrize("bits", [[1] * 8, [2] * 8, [3] * 8, [4] * 8, [1, 4, 2, 3, 3, 1, 4, 2], [3], [2, 1]])
 @pytest.mark.parametrize("M", [1, 4])
 def test_adversarial_bit_maps(bits, M):
