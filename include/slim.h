@@ -268,7 +268,9 @@ int slim_gemv_set_plan(const slim_layer* layers_host, int n_layers, int g,
 
 /* Runs the set: one small kernel puts every layer's activations into fragment order in the
  * workspace, one persistent kernel computes all layers (a small single-token set whose CTAs are all resident at
- * once runs as one launch instead: slim_gemv_set_info.resident_pairs).  `workspace` as for slim_mpq_gemv
+ * once runs as one launch instead: slim_gemv_set_info.resident_pairs; that launch uses programmatic stream
+ * serialisation and requests packed, scales and zeros before it waits for the kernel ahead of it on the stream, under
+ * the rule stated at slim_mpq_gemv).  `workspace` as for slim_mpq_gemv
  * (zeroed once with slim_workspace_init; slim_workspace_status reports a device-side time-out). */
 int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan,
                       void* workspace, size_t workspace_bytes, void* stream);
