@@ -46,6 +46,49 @@ def test_single_token_edge_shapes(N, K):
     check_output(y, orc.linear_f64(L["x"], L["codes"], L["scales"], L["zeros"]), f"{N}x{K}")
 
 
+@pytest.mark.parametrize("M", [1, 4])
+@pytest.mark.parametrize("as_graph", [False, True])
+def test_chain_of_layers_each_reading_the_output_of_the_one_before(M, as_graph):
+    """Six layers launched back to back, each taking the y of the one before as its x.  The kernels are launched with
+    programmatic stream serialisation and request their weights before they wait for the kernel ahead; what they read of
+    x must still be that kernel's finished output.  Checked layer by layer against the oracle fed with the device's own
+    (fp16) inputs, eagerly and as a replayed CUDA graph."""
+    from paper_2405_14917_b200 import binding as slim
+    dims = [1024, 512, 2048, 512, 1024, 256, 768]
+    layers = [oracle_layer(dims[i + 1], dims[i], 3, M, seed_name="chain", block=i) for i in range(6)]
+    dev = []
+    for L in layers:
+        dev.append(slim.QuantLinear(torch.from_numpy(orc.pack(L["codes"], L["bits"])).cuda(), L["bits"],
+                                    torch.from_numpy(L["scales"]).cuda(), torch.from_numpy(L["zeros"]).cuda(), L["N"], L["K"]))
+    acts = [torch.from_numpy(layers[0]["x"]).cuda()] + [torch.zeros(M, d, dtype=torch.float16, device="cuda") for d in dims[1:]]
+    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    slim.workspace_init(ws)
+
+    def run():
+        for i, dl in enumerate(dev):
+            dl.forward(acts[i], ws, out=acts[i + 1])
+    run()
+    torch.cuda.synchronize()
+    if as_graph:
+        for a in acts[1:]:
+            a.zero_()
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g):
+                run()
+        torch.cuda.current_stream().wait_stream(side)
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+    slim.workspace_status(ws)
+    for i, L in enumerate(layers):
+        x_in = acts[i].cpu().numpy()
+        y_ref = orc.linear_f64(x_in, L["codes"], L["scales"], L["zeros"])
+        check_output(acts[i + 1].cpu().numpy(), y_ref, f"layer {i} of the chain")
+
+
 @pytest.mark.parametrize("bits", [[1] * 8, [2] * 8, [3] * 8, [4] * 8, [1, 4, 2, 3, 3, 1, 4, 2], [3], [2, 1]])
 @pytest.mark.parametrize("M", [1, 4])
 def test_adversarial_bit_maps(bits, M):

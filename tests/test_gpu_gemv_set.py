@@ -218,6 +218,31 @@ def test_layers_that_share_input_and_bit_map_are_staged_once(M):
         check_output(y.cpu().numpy(), orc.linear_f64(x.cpu().numpy(), L["codes"], L["scales"], L["zeros"]), f"layer {k}")
 
 
+@pytest.mark.parametrize("M", [1, 3])
+def test_a_set_that_reads_the_outputs_of_the_set_before(M):
+    """Two small sets launched back to back on one stream; the layers of the second read what the first wrote.  At
+    one token both are single resident launches that fetch their weights before they wait for the launch ahead."""
+    slim = _slim()
+    first = [oracle_layer(512, 1024, 2, M, seed_name="set-chain", block=0), oracle_layer(768, 1024, 3, M, seed_name="set-chain", block=1)]
+    second = [oracle_layer(256, 512, 2, M, seed_name="set-chain", block=2), oracle_layer(384, 768, 2, M, seed_name="set-chain", block=3)]
+    x0 = torch.from_numpy(first[0]["x"]).cuda()
+    mid = [torch.zeros(M, L["N"], dtype=torch.float16, device="cuda") for L in first]
+    out = [torch.zeros(M, L["N"], dtype=torch.float16, device="cuda") for L in second]
+    s1 = slim.LayerSet([(_device_layer(L), x0, y) for L, y in zip(first, mid)])
+    s2 = slim.LayerSet([(_device_layer(L), x, y) for L, x, y in zip(second, mid, out)])
+    assert (s1.info["resident_pairs"] > 0) == (M == 1)
+    for _ in range(3):
+        s1.run()
+        s2.run()
+    s1.check()
+    s2.check()
+    x0h = first[0]["x"]
+    for L, y in zip(first, mid):
+        check_output(y.cpu().numpy(), orc.linear_f64(x0h, L["codes"], L["scales"], L["zeros"]), "first set")
+    for L, x, y in zip(second, mid, out):
+        check_output(y.cpu().numpy(), orc.linear_f64(x.cpu().numpy(), L["codes"], L["scales"], L["zeros"]), "second set")
+
+
 def test_single_token_fixed_point_with_outlier_channels():
     """Single-token sets round x per group to fixed point relative to the group's largest |x|.  Outlier channels
     (a few activations 100 x the rest, as in LLM activations) and a group of tiny activations must stay within the
