@@ -4,8 +4,9 @@
 // A decode-sized layer is a few megabytes, so the launch is over in a few microseconds and what counts is the
 // length of the dependent chain inside a CTA, not the instruction count.  Hence:
 //
-//  * a CTA owns 2, 4, 6 or 8 tiles of 16 rows and the WHOLE K: no partial sums leave the CTA, no cluster, no second
-//    pass.  The tile count is the smallest for which all CTAs of the layer are resident at once.
+//  * a CTA owns 2, 4, 6 or 8 tiles of 16 rows and the WHOLE K: no partial sums leave the CTA and there is no second
+//    pass.  The tile count is the smallest for which all CTAs of the layer are resident at once (else the one that
+//    needs the fewest waves).
 //  * warp w owns the groups w, w + 16, ... of the CTA's tiles: it brings their slices with one cp.async.bulk per
 //    group onto a barrier of its own, their scales and zeros with 16-byte cp.async, multiplies and folds.  Warps
 //    meet at the end to add their sixteen partial sums per row in warp order (deterministic).
@@ -15,8 +16,10 @@
 //  * everything that does not depend on x (the slices, scales, zeros) is requested BEFORE griddepcontrol.wait, and
 //    the dependents are released right after, so with programmatic dependent launch the loads of layer l + 1 are in
 //    flight while layer l computes.
+//  * a set of a few single-token layers (q/k/v, gate/up) whose CTAs are all resident at once is ONE launch of the
+//    same body: every layer owns whole clusters, a CTA reads its layer's descriptor from the plan buffer first.
 //
-// Every wait is bounded and reports through the workspace status word.
+// Every wait on a barrier in memory is bounded and reports through the workspace status word.
 #include "slim_common.cuh"
 #include "slim_gemv_i8.cuh"
 
