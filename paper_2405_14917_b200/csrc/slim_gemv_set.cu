@@ -142,13 +142,23 @@ __global__ void __launch_bounds__(256) gemv_set_stage_kernel(const SetLayer* __r
     stage_clear_counters(ws, n_counters);
     const int lane = threadIdx.x & 31;
     const int task = blockIdx.x * 8 + (threadIdx.x >> 5);
+    // The layer of a task is the last one whose first task is not above it.  A search through the descriptors is a
+    // chain of dependent loads from global memory (eight for the 224 layers of a 7B sweep, most of this kernel's time),
+    // so a set of up to kStageTable layers first puts their first tasks into shared memory, all loads in flight at once.
+    constexpr int kStageTable = 2048;
+    __shared__ int first_task[kStageTable];
+    const bool table = n_layers <= kStageTable;
+    if (table) {
+        for (int l = threadIdx.x; l < n_layers; l += blockDim.x) first_task[l] = layers[l].task0;
+        __syncthreads();
+    }
     if (task >= n_tasks) return;
-    int lo = 0, hi = n_layers - 1;                       // last layer whose task0 <= task
+    int lo = 0, hi = n_layers - 1;
     while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
-        if (layers[mid].task0 <= task) lo = mid; else hi = mid - 1;
+        if ((table ? first_task[mid] : layers[mid].task0) <= task) lo = mid; else hi = mid - 1;
     }
-    stage_task(layers[lo], ws, task - layers[lo].task0, lane);
+    stage_task(layers[lo], ws, task - (table ? first_task[lo] : layers[lo].task0), lane);
 }
 
 // D = A * B with a zero accumulator input: starts an accumulation chain without clearing registers first.
