@@ -50,10 +50,10 @@ def set_kernel_hash():
 
 
 NCU_TRAFFIC = {
-    # layer-set kernel, 4 blocks of the LLaMA-7B sweep (28 layers, avg 2-bit, M = 1): 228,645,632 B read +
-    # 4,398,336 B written per launch (algorithmic 228,297,816 B); scaled to the full sweep by the algorithmic bytes
+    # layer-set kernel, 4 blocks of the LLaMA-7B sweep (28 layers, avg 2-bit, M = 1): 228,641,280 B read +
+    # 5,452,544 B written per launch (algorithmic 228,297,816 B); scaled to the full sweep by the algorithmic bytes
     # (the traffic is the packed data read once, so it grows in proportion)
-    "cb1abb0f9791d151c1d18d89807f0df61e5dc627fab0d9a2d5342caf3b2d8131": {"layer": "4 blocks", "traffic_bytes": 233043968, "algorithmic_bytes": 228297816},
+    "07e9a7071019a32d39d424c0ce137b71d58c425a00b8a87620fa5ace5a4ffa36": {"layer": "4 blocks", "traffic_bytes": 234093824, "algorithmic_bytes": 228297816},
 }
 
 
@@ -930,7 +930,7 @@ def secondary_entries(args, device, timer, primary_layers, clock_gpu):
     torch.cuda.empty_cache()
     spec3 = workload_spec("llama7b-decode-avg3-m1-blocks8")
     layers3 = build_layers(spec3, device, 0)
-    for M in (1, 4, 8, 16):
+    for M in (1, 4, 8, 16, 32, 64):
         sp = dict(spec3, M=M)
         guarded(lambda: decode_entry(f"llama7b-decode-avg3-m{M}-blocks8", layers3, sp, device, timer, "set", 50, 0.6, clock_gpu=clock_gpu))
     del layers3

@@ -65,6 +65,7 @@ extern "C" {
 #define SLIM_GROUP 128           /* the paper's default group size, and the widest K-tile of the packed format */
 #define SLIM_MAX_GROUPS 256      /* most K-tiles of 128 columns in a layer (K <= 32768) */
 #define SLIM_GEMV_MAX_M 16
+#define SLIM_GEMV_SET_MAX_M 64   /* tokens of a layer in a layer set */
 
 enum {
     SLIM_OK = 0,
@@ -196,7 +197,7 @@ int slim_mpq_gemm_static(const void* x, const void* packed, const uint8_t* bits_
 
 /* ---- layer-set launch of the decode path --------------------------------------------------- */
 
-/* Several INDEPENDENT layers of the decode path (1 <= M <= 16 each) in one launch: the q/k/v or
+/* Several INDEPENDENT layers of the decode path (1 <= M <= SLIM_GEMV_SET_MAX_M = 64 tokens each) in one launch: the q/k/v or
  * gate/up projections that share an input, or a sweep over a model's layers.  (The paper launches
  * its kernel per layer, App. B.2; a decode-sized layer is too small to keep HBM busy on its own,
  * so the set is walked by persistent CTAs that stream the packed slices of one 128-row block after
@@ -213,7 +214,10 @@ int slim_mpq_gemm_static(const void* x, const void* packed, const uint8_t* bits_
  * of at most 2^-22 of the maximum; the sums over the group are then exact.  Per output row n this adds at
  * most  sum over groups of 2^-22 max|x_group| sum_{k in group} |w-hat[n][k]|  to the error of the fp16
  * path at more than one token; x must be finite.  Sets with more tokens multiply
- * the fp16 x as it is.
+ * the fp16 x as it is, in MMA tiles of 8 tokens: the set's widest layer, rounded up to 8, 16, 32 or 64 tokens, fixes
+ * how many tiles every layer computes, so a set is fastest when its layers have about the same token count.  (Between
+ * 17 and about 100 tokens a layer set streams several times the weights per second that slim_mpq_gemm dequantises,
+ * which is built for hundreds of tokens and more.)
  * N > 0 a multiple of 16, K > 0 a multiple of 128; g in {128, 256, 512}, one value for the whole set (for 256 and
  * 512 "group" in the bound above reads "128 columns of a group"); SLIM_ERR_UNSUPPORTED for 32 and 64. */
 typedef struct slim_layer {
@@ -232,7 +236,7 @@ typedef struct slim_gemv_set_info {
     int grid;              /* persistent CTAs */
     int n_slots;           /* ring slots per CTA */
     int slot_bytes;
-    int token_tiles;       /* 8-token MMA tiles: 1 or 2 */
+    int token_tiles;       /* 8-token MMA tiles: 1, 2, 4 or 8 */
     int stage_tasks;       /* (layer, token, group) triples staged; layers with one x and one bit map count once */
     int n_items;           /* row blocks (work items) of the set */
     int max_bits;          /* widest group of the set */

@@ -59,8 +59,10 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 
 // ------------------------------------------------------------------------------------------ activation staging
 // Byte offset of group j inside a layer's staged activations (pre3 = 3-bit groups before j).
+// A record starts with (sum_k x, scale) per token, 8 bytes each: 128 bytes for up to 16 tokens, 8 M beyond.
+__host__ __device__ constexpr int staged_header_bytes(int M) { return M > 16 ? 8 * M : 128; }
 __host__ __device__ inline size_t staged_group_offset(int j, int pre3, int M) {
-    return 128u * static_cast<size_t>(j) + 256u * static_cast<size_t>(M) * static_cast<size_t>(j + pre3);
+    return static_cast<size_t>(staged_header_bytes(M)) * static_cast<size_t>(j) + 256u * static_cast<size_t>(M) * static_cast<size_t>(j + pre3);
 }
 // ---- single-token sets: activations as signed 8-bit digits, the packed words as unsigned bytes ----------
 // With one token seven of the eight MMA columns are free, and an integer MMA takes four codes per

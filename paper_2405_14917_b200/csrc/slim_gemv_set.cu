@@ -40,7 +40,8 @@ constexpr int kSetConsumers = 8;                       // consumer warps; each o
 constexpr int kSetProducers = 2;                       // producer warps: they take the groups in turn
 constexpr int kSetThreads = 32 * (kSetConsumers + kSetProducers);
 constexpr int kSetMaxSlots = 32;
-constexpr int kSetCtasPerSm = 2;                       // resident CTAs per SM the plan aims at
+constexpr int kSetCtasPerSm = 2;                       // resident CTAs per SM the plan aims at (one from 17 tokens on: registers)
+constexpr int kSetMaxTokens = 64;                      // tokens of a layer in a set: up to eight MMA tiles of 8
 
 // Layout of a ring slot (tpi = 16-row tiles of a work item, mp = 256-byte pieces per slice of the staged
 // activations: 2 for single-token sets, else the 8 or 16 tokens of the set).  Everything but the packed slices has
@@ -49,8 +50,8 @@ constexpr int kSetCtasPerSm = 2;                       // resident CTAs per SM t
 constexpr int kSlotOffS = 16;
 __host__ __device__ constexpr int slot_off_z(int tpi) { return kSlotOffS + 32 * tpi; }
 __host__ __device__ constexpr int slot_off_e(int tpi) { return kSlotOffS + 64 * tpi; }
-__host__ __device__ constexpr int slot_off_x(int tpi) { return slot_off_e(tpi) + 128; }
-__host__ __device__ constexpr int slot_off_w(int tpi, int mp) { return slot_off_x(tpi) + 2 * 256 * mp; }
+__host__ __device__ constexpr int slot_off_x(int tpi, int mp) { return slot_off_e(tpi) + (mp > 16 ? 8 * mp : 128); }
+__host__ __device__ constexpr int slot_off_w(int tpi, int mp) { return slot_off_x(tpi, mp) + 2 * 256 * mp; }
 
 // Device-side description of one layer (lives in the plan buffer).
 struct SetLayer {
@@ -125,15 +126,17 @@ __device__ __forceinline__ void stage_task(const SetLayer& L, uint8_t* ws, int p
     }
     float2* sxe = reinterpret_cast<float2*>(grp);
     if (m < L.M) {
-        const float2 r = stage_group(L.x + static_cast<size_t>(m) * L.K + j * SLIM_GROUP, grp + 128, L.bits[j], m, L.MP, lane);
+        const float2 r = stage_group(L.x + static_cast<size_t>(m) * L.K + j * SLIM_GROUP, grp + staged_header_bytes(L.MP), L.bits[j], m, L.MP, lane);
         if (lane == 0) sxe[m] = r;
     } else {
         // a token the layer does not have: zero fragments in every slice of the group
         const int cc = lane & 3, mi = lane >> 2;
         for (int sl = 0; sl < slice_count(L.bits[j]); ++sl)
-            *reinterpret_cast<uint2*>(grp + 128 + (((static_cast<size_t>(sl) * 8 + mi) * L.MP + m) * 4 + cc) * 8) = make_uint2(0u, 0u);
+            *reinterpret_cast<uint2*>(grp + staged_header_bytes(L.MP) + (((static_cast<size_t>(sl) * 8 + mi) * L.MP + m) * 4 + cc) * 8) = make_uint2(0u, 0u);
     }
-    if (m == 0 && lane < 16 && lane >= L.M) sxe[lane] = make_float2(0.f, 1.f);   // absent tokens read 0
+    if (m == 0)
+        for (int t = lane; t < max(L.MP, 16); t += 32)
+            if (t >= L.M) sxe[t] = make_float2(0.f, 1.f);                          // absent tokens read 0
 }
 
 // One warp per (layer, token, group): fragments and sums of the whole set, once.
@@ -219,7 +222,7 @@ __device__ __forceinline__ void consume_one(const SetParams& p, const uint32_t s
     auto full = [&](int s) { return sbase + 8u * s; };
     auto empty = [&](int s) { return sbase + 8u * (kSetMaxSlots + s); };
     constexpr int TPI = kSetConsumers * TPW, CHI = 2;
-    constexpr uint32_t kOffZ = slot_off_z(TPI), kOffE = slot_off_e(TPI), kOffX = slot_off_x(TPI), kOffW = slot_off_w(TPI, 2);
+    constexpr uint32_t kOffZ = slot_off_z(TPI), kOffE = slot_off_e(TPI), kOffX = slot_off_x(TPI, 2), kOffW = slot_off_w(TPI, 2);
     static_assert(TPW <= 2, "one lane pair per tile");
     const int gq = lane >> 2, c = lane & 3;
     const int tsel = TPW == 2 ? (c >> 1) : 0;
@@ -371,7 +374,7 @@ __device__ __forceinline__ void consume_f16(const SetParams& p, const uint32_t s
     // interleaved accumulation chains per (tile, token tile): with four (tile, token tile) pairs the MMAs of one pair are far
     // enough apart without a second chain
     constexpr int CH = NT * TPW >= 4 ? 1 : (NT == 1 ? (TPW == 1 ? 4 : 2) : 2);
-    constexpr uint32_t kOffZ = slot_off_z(TPI), kOffE = slot_off_e(TPI), kOffX = slot_off_x(TPI), kOffW = slot_off_w(TPI, MPK);
+    constexpr uint32_t kOffZ = slot_off_z(TPI), kOffE = slot_off_e(TPI), kOffX = slot_off_x(TPI, MPK), kOffW = slot_off_w(TPI, MPK);
     const int gq = lane >> 2, c = lane & 3;
     const uint32_t lane0 = lane == 0 ? 1u : 0u;
     const uint32_t slot_bytes = static_cast<uint32_t>(p.slot_bytes);
@@ -527,7 +530,7 @@ constexpr uint32_t kSetOffRing = (kSetOffDesc + kSetProducers * sizeof(SetLayer)
 // TPW: 16-row tiles per consumer warp (an item is 8 * TPW tiles; always 2 today); two tiles share the fragment
 // loads and the per-group bookkeeping.
 template <int NT, bool ONE, int TPW>
-__global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(const __grid_constant__ SetParams p) {
+__global__ void __launch_bounds__(kSetThreads, NT >= 4 ? 1 : kSetCtasPerSm) gemv_set_kernel(const __grid_constant__ SetParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -536,7 +539,7 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
     volatile int* abort = reinterpret_cast<volatile int*>(smem + kSetOffAbort);
     const uint32_t ring = sbase + kSetOffRing;
     constexpr int TPI = kSetConsumers * TPW;                  // tiles per item
-    constexpr uint32_t kOffZ = slot_off_z(TPI), kOffE = slot_off_e(TPI), kOffX = slot_off_x(TPI);
+    constexpr uint32_t kOffZ = slot_off_z(TPI), kOffE = slot_off_e(TPI), kOffX = slot_off_x(TPI, ONE ? 2 : 8 * NT);
     constexpr uint32_t kOffW = slot_off_w(TPI, ONE ? 2 : 8 * NT);
 
     if (tid == 0) {
@@ -591,7 +594,7 @@ __global__ void __launch_bounds__(kSetThreads, kSetCtasPerSm) gemv_set_kernel(co
                     const int j = D->order[jj];            // the groups are streamed sorted by bit-width
                     const uint32_t b = D->bits[j];
                     const uint32_t wbytes = static_cast<uint32_t>(tiles_here) * 256u * b;
-                    const uint32_t xbytes = 128u + static_cast<uint32_t>(slice_count(b)) * 256u * MP;
+                    const uint32_t xbytes = static_cast<uint32_t>(staged_header_bytes(MP)) + static_cast<uint32_t>(slice_count(b)) * 256u * MP;
                     const uint32_t slot = ring + static_cast<uint32_t>(s) * p.slot_bytes;
                     if (lane == 0) {
                         asm volatile("st.shared.u32 [%0], %1;" ::"r"(slot), "r"(b) : "memory");
@@ -701,7 +704,7 @@ static size_t align_to(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static size_t layer_ws_bytes(int M, const GroupTable& gt) {
     int slots = gt.G;
     for (int j = 0; j < gt.G; ++j) slots += gt.bits[j] == 3 ? 1 : 0;
-    return align_to(static_cast<size_t>(gt.G) * 128 + static_cast<size_t>(slots) * 256 * M, 128);
+    return align_to(static_cast<size_t>(gt.G) * staged_header_bytes(M) + static_cast<size_t>(slots) * 256 * M, 128);
 }
 // Work of an item for the deal.  The kernel is bound by the instructions it issues, so a (tile, group)
 // weighs what a consumer warp issues for it: about 70 / 73 / 120 / 80 instructions at 1 / 2 / 3 / 4 bits
@@ -728,11 +731,12 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     sg->ws_bytes = 256;
     for (int l = 0; l < n_layers; ++l) sg->mmax = sg->mmax > layers[l].M ? sg->mmax : layers[l].M;
     sg->tpw = 2;
-    sg->mpad = sg->mmax <= 1 ? 2 : (sg->mmax <= 8 ? 8 : 16);    // one token: the 8-bit digit form, 512 bytes per slice
+    // one token: the 8-bit digit form, 512 bytes per slice; else the tokens of the widest layer rounded up to 8, 16, 32, 64
+    sg->mpad = sg->mmax <= 1 ? 2 : (sg->mmax <= 8 ? 8 : (sg->mmax <= 16 ? 16 : (sg->mmax <= 32 ? 32 : 64)));
     const int tpi = kSetConsumers * sg->tpw;          // tiles per item
     for (int l = 0; l < n_layers; ++l) {
         const slim_layer& L = layers[l];
-        if (L.M < 1 || L.M > SLIM_GEMV_MAX_M) return SLIM_ERR_INVALID_ARG;
+        if (L.M < 1 || L.M > kSetMaxTokens) return SLIM_ERR_INVALID_ARG;
         GroupTable gt;
         const int st = make_group_table(L.N, L.K, g, L.bits_host, &gt);
         if (st != SLIM_OK) return st;
@@ -744,10 +748,10 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
         sg->ws_bytes += layer_ws_bytes(sg->mpad, gt);
     }
     if (sg->n_items > 0x3fffffff || sg->n_tasks > 0x3fffffff) return SLIM_ERR_UNSUPPORTED;
-    sg->nt = sg->mmax <= 8 ? 1 : 2;
+    sg->nt = sg->mmax <= 1 ? 1 : sg->mpad / 8;
     // A set with fewer row blocks than persistent CTAs cuts the groups of every row block into parts (items of their
     // own, fp32 partial outputs in the workspace, added in part order by the consumer warp whose part lands last).
-    const long long want = static_cast<long long>(set_sm_count()) * kSetCtasPerSm;
+    const long long want = static_cast<long long>(set_sm_count()) * (sg->nt >= 4 ? 1 : kSetCtasPerSm);
     sg->split = 1;
     if (sg->n_items < 2 * want) {
         // the number of parts that fills the last wave of CTAs best (the smallest one within 2 % of the best)
@@ -786,7 +790,7 @@ static int set_geometry(const slim_layer* layers, int n_layers, int g, SetGeomet
     // as many CTAs per SM (kSetCtasPerSm at most) as still leaves each a ring of 4 slots
     const size_t per_sm = 224 * 1024;
     size_t budget = 0;
-    for (sg->ctas_per_sm = kSetCtasPerSm; sg->ctas_per_sm >= 1; --sg->ctas_per_sm) {
+    for (sg->ctas_per_sm = sg->nt >= 4 ? 1 : kSetCtasPerSm; sg->ctas_per_sm >= 1; --sg->ctas_per_sm) {
         budget = per_sm / sg->ctas_per_sm - 1024 - kSetOffRing;   // 1 KB per CTA is reserved by the system
         if (budget / sg->slot_bytes >= 4 || sg->ctas_per_sm == 1) break;
     }
@@ -896,7 +900,8 @@ static int set_params(const slim_gemv_set_info* info, const void* plan, void* wo
     if (info == nullptr || plan == nullptr) return SLIM_ERR_INVALID_ARG;
     if (info->n_layers < 1 || info->grid < 1 || info->grid > kSetMaxGrid || info->n_slots < 2 ||
         info->n_slots > kSetMaxSlots || info->slot_bytes < 128 || info->slot_bytes % 128 != 0 ||
-        (info->token_tiles != 1 && info->token_tiles != 2) || info->max_tokens < 1 || info->max_tokens > 8 * info->token_tiles ||
+        (info->token_tiles != 1 && info->token_tiles != 2 && info->token_tiles != 4 && info->token_tiles != 8) ||
+        info->max_tokens < 1 || info->max_tokens > 8 * info->token_tiles ||
         info->tiles_per_warp != 2 ||
         info->max_bits < 1 || info->max_bits > 4 || info->stage_tasks < 1 || info->split < 1 || info->split > kSetMaxSplit ||
         info->n_counters < 0 || info->n_counters > 65535 || info->n_layers > 65535)
@@ -928,6 +933,8 @@ static int set_params(const slim_gemv_set_info* info, const void* plan, void* wo
 // The persistent kernel of the set in the form its token count asks for.
 static int launch_set_for(const slim_gemv_set_info* info, const SetParams& prm, size_t smem, cudaStream_t s) {
     const cudaError_t e = info->max_tokens == 1 ? launch_set<1, true, 2>(prm, info->grid, smem, s)
+                        : info->token_tiles == 8 ? launch_set<8, false, 2>(prm, info->grid, smem, s)
+                        : info->token_tiles == 4 ? launch_set<4, false, 2>(prm, info->grid, smem, s)
                         : info->token_tiles == 1 ? launch_set<1, false, 2>(prm, info->grid, smem, s)
                                                  : launch_set<2, false, 2>(prm, info->grid, smem, s);
     SLIM_CUDA_TRY(e);

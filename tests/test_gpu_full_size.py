@@ -169,11 +169,12 @@ def test_projections_of_a_block_as_small_single_token_sets():
                 check_output(y[:, rows], orc.linear_rows_f64(xs[i], L["codes"], L["scales"], L["zeros"], rows), f"{N}x{K} layer {i}")
 
 
-@pytest.mark.parametrize("M", [1, 4, 8, 16])
+@pytest.mark.parametrize("M", [1, 4, 8, 16, 32, 64])
 def test_llama7b_avg3_layer_set_all_token_counts(M):
     """LLaMA-7B shapes at avg 3 bits (bit-widths 2, 3, 4) through the layer-set launch, for every token count of
-    that configuration: the single-token integer form, the one-token-tile and the two-token-tile f16 forms, each
-    with more work items than persistent CTAs so that CTAs cross item and layer boundaries."""
+    that configuration and for the 32 and 64 tokens a set also takes: the single-token integer form and the f16 forms
+    of one, two, four and eight token tiles, each with more work items than persistent CTAs so that CTAs cross item and
+    layer boundaries."""
     slim = _slim()
     rng = np.random.default_rng(300 + M)
     entries, meta = [], []

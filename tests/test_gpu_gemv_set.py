@@ -70,7 +70,7 @@ def test_small_set_of_several_tokens_cuts_its_row_blocks_into_parts():
     assert s.info["n_items"] == sum(k * -(-L["N"] // rows) for k, L in zip(parts, layers))
 
 
-@pytest.mark.parametrize("Ms", [(1, 2, 3), (4, 8, 5), (16, 9, 1), (16, 16, 16)])
+@pytest.mark.parametrize("Ms", [(1, 2, 3), (4, 8, 5), (16, 9, 1), (16, 16, 16), (17, 3, 1), (32, 32, 32), (5, 40, 64), (64, 64, 64), (33, 1, 24)])
 def test_mixed_token_counts(Ms):
     layers = [oracle_layer(384, 768, 2, Ms[0], block=0), oracle_layer(144, 1280, 3, Ms[1], block=1),
               oracle_layer(256, 256, 2, Ms[2], block=2)]
@@ -146,9 +146,9 @@ def test_rejects_bad_sets():
         slim.LayerSet([])
     with pytest.raises(ValueError):
         slim.LayerSet([(dl, x, torch.empty(1, 64, dtype=torch.float16, device="cuda"))])
-    x17 = torch.zeros(17, 256, dtype=torch.float16, device="cuda")
+    x65 = torch.zeros(65, 256, dtype=torch.float16, device="cuda")          # a set takes up to 64 tokens per layer
     with pytest.raises(slim.SlimError):
-        slim.LayerSet([(dl, x17, torch.empty(17, 128, dtype=torch.float16, device="cuda"))])
+        slim.LayerSet([(dl, x65, torch.empty(65, 128, dtype=torch.float16, device="cuda"))])
 
 
 def test_llama7b_shapes_full_size_in_the_benchmark_configuration():
