@@ -139,7 +139,8 @@ def test_layer_set_sizes_and_argument_errors(slim):
     assert _set_bytes(slim, [(9, 256, 512, [2, 3, 1, 2])])[2] == 256 + (4 * 128 + (4 + 1) * 8 * 16 * 32)     # sixteen wide
     assert _set_bytes(slim, [])[0] == -1                                  # empty set
     assert _set_bytes(slim, [(0, 256, 512, [2] * 4)])[0] == -1            # no token
-    assert _set_bytes(slim, [(17, 256, 512, [2] * 4)])[0] == -1           # the batched path serves these
+    assert _set_bytes(slim, [(40, 256, 512, [2, 3, 1, 2])])[2] == 256 + (4 * 512 + (4 + 1) * 256 * 64)        # 64 wide: 8 bytes of sums per token
+    assert _set_bytes(slim, [(65, 256, 512, [2] * 4)])[0] == -1           # more than 64 tokens: the batched path
     assert _set_bytes(slim, [(1, 256, 512, [2, 5, 2, 2])])[0] == -1       # bit-width out of range
     assert _set_bytes(slim, [(1, 250, 512, [2] * 4)])[0] == -2            # N not a multiple of 16
     assert _set_bytes(slim, [(1, 256, 500, [2] * 4)])[0] == -2            # K not a multiple of 128
