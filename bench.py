@@ -60,7 +60,7 @@ NCU_TRAFFIC = {
 # DRAM bytes (read + written) of the 14 gemm_kernel launches of one step of llama13b-prefill-avg3-m2048, from one ncu
 # capture of dram__bytes_read.sum and dram__bytes_write.sum; keyed by the SHA-256 of slim_gemm.cu at capture time
 NCU_TRAFFIC_GEMM = {
-    "5fd2ba9fc66a0002d80a79c938e81c8775052fcd9e7b4f9781ec9ffa2f9dccb0": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1054245120 + 218284032},
+    "7082f3a4c2b0494e1fc5b0a677a09ca71f4b833ea04442557984c259de1928ef": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1081612800 + 227610112},
 }
 
 

@@ -15,7 +15,10 @@
 //  * D = fp32 accumulator in tensor memory, 128 lanes x TOK columns per CTA; tcgen05.mma
 //    cta_group::2 kind::f16 is issued by one thread of the leader CTA (cluster rank 0), eight
 //    K=16 steps per group, and a multicast tcgen05.commit hands the stages back to both CTAs.
-//  * Epilogue warps of each CTA read their D with tcgen05.ld and store y as fp16.
+//  * Epilogue warps of each CTA read their D with tcgen05.ld and store y as fp16: a whole tile goes
+//    through shared memory, 32 tokens x 32 rows per warp at a time, and out with one tensor store per
+//    chunk (two buffers per warp: a chunk is written while the store of the one before reads its
+//    buffer); the tensor map clips rows past N and tokens past M.
 //
 // Dequantisation: a code field is left in mantissa bits [6,10) of the half 1024; one HFMA2 with
 // constants that hold the zero point turns it into q - z exactly for every zero point that is a
@@ -36,6 +39,7 @@
 
 #include <cuda.h>
 #include <cstring>
+#include <cmath>
 
 namespace slim {
 
@@ -50,6 +54,8 @@ constexpr int kNS = 4 / kGPS;               // pipeline stages: a shared-memory 
 constexpr int kPStageBytes = 8192 + 512;    // 128 rows x 128 k x 4 bits, + scales + zeros
 constexpr int kTmemCols = 512;
 constexpr int kEpiCols = 16;                // accumulator columns (tokens) the epilogue handles at a time
+constexpr int kYBox = 32;                   // tokens, and rows, of one output store
+constexpr int kYBoxBytes = kYBox * kYBox * 2;
 constexpr int kTmemAcol = 256;              // A stages start here; D occupies [0, TOK)
 constexpr unsigned long long kGemmWaitNs = 2000000000ull;
 
@@ -60,7 +66,7 @@ struct GemmParams {
     __half* y;
     unsigned int* status;
     unsigned int* flags;     // [grid]: "partial of this CTA is ready" (stream-K only; zero between launches)
-    float* partials;         // [grid][TOK][128] fp32 (stream-K only)
+    float* partials;         // [grid][4 epilogue warps][TOK][32 rows] fp32 (stream-K only)
     int M, N, K;
     int row_blocks, tok_tiles;   // 256-row blocks, TOK-token tiles
     int stream_k;            // 1: clusters take equal shares of (tile, group) units; 0: whole tiles
@@ -228,6 +234,23 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
           "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr) : "memory");
 }
+// Shared memory -> global, tile of a tensor map (rows and columns past the tensor's extent are clipped).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all but the newest `N` stores of this thread have read their shared memory
+template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void sts_u16(uint32_t addr, uint16_t v) { asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory"); }
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+// orders what this thread has observed through ordinary loads before the bulk copies it issues next
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
@@ -341,8 +364,10 @@ template <int TOK> struct GemmCfg {
     static constexpr int XBOX = HALF * 128;                  // bytes of one TMA box: HALF rows x 64 k
     static constexpr int XSTAGE = 2 * XBOX;                  // one group: 128 k
     static constexpr int OFF_P = kNS * kGPS * XSTAGE;
-    static constexpr int OFF_BAR = OFF_P + NP * kPStageBytes;
-    static constexpr int NBAR = 3 * kNS + 2 * NP + 2;
+    static constexpr int OFF_STAGE = OFF_P + NP * kPStageBytes;   // output staging: per epilogue warp two tiles of 32 tokens x 32 rows, fp16
+    static constexpr int OFF_BAR = OFF_STAGE + 4 * 2 * kYBoxBytes;
+    static constexpr int NPEERBAR = TOK / kEpiCols;         // per epilogue warp: one per 16-token piece of a peer's partial tile
+    static constexpr int NBAR = 3 * kNS + 2 * NP + 2 + 4 * NPEERBAR;
     static constexpr int OFF_MISC = OFF_BAR + 8 * NBAR;      // tensor-memory base, abort flag
     static constexpr int SMEM = OFF_MISC + 16 + 1024;        // + slack to align the base to 1024
 };
@@ -355,7 +380,7 @@ __device__ __forceinline__ uint64_t sw128_kmajor_desc(uint32_t smem_addr) {
 
 template <int TOK>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ GemmParams p) {
+gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap y_map, const __grid_constant__ GemmParams p) {
     using C = GemmCfg<TOK>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (g::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -376,6 +401,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
     auto p_empty = [&](int s) { return bar0 + 8 * (3 * kNS + C::NP + s); };
     const uint32_t d_full = bar0 + 8 * (3 * kNS + 2 * C::NP);
     const uint32_t d_empty = d_full + 8;                 // leader's: 8 epilogue warps of the pair
+    auto peer_full = [&](int q, int s) { return d_empty + 8 + 8 * (C::NPEERBAR * q + s); };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OFF_MISC);
     volatile int* abort = reinterpret_cast<volatile int*>(smem + C::OFF_MISC + 4);
 
@@ -384,6 +410,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
         for (int s = 0; s < C::NP; ++s) { g::mbar_init(p_full(s), 1); g::mbar_init(p_empty(s), 8); }
         g::mbar_init(d_full, 1);
         g::mbar_init(d_empty, 8);
+        for (int s = 0; s < 4 * C::NPEERBAR; ++s) g::mbar_init(peer_full(0, s), 1);
         *abort = 0;
         g::fence_barrier_init();
         g::fence_proxy_async();
@@ -643,67 +670,140 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
                     if (range_begin(pc + 1) >= static_cast<long long>(tile + 1) * G) break;
                 }
             }
-            auto peer_active = [&](int k) { return range_begin(cl + k) < range_begin(cl + k + 1); };
+            // bit k-1: peer k has a segment (a cut leaves every pair at least eight groups and a tile has at most
+            // SLIM_MAX_GROUPS of them, so there are fewer than 64 peers)
+            unsigned long long act = 0ull;
+            for (int k = 1; k <= npeer && k <= 64; ++k)
+                if (range_begin(cl + k) < range_begin(cl + k + 1)) act |= 1ull << (k - 1);
+            auto peer_active = [&](int k) { return ((act >> (k - 1)) & 1ull) != 0ull; };
             bool gave_up = !g::mbar_wait_long(d_full, phd, abort);
             gave_up = epi_any(gave_up);          // named barriers may follow, now or in a later unit: decide once for all
             if (gave_up) { ok = false; break; }
             g::tc_fence_after();
             if (npeer > 0) {
-                if (et == 0) {
+                // thread k-1 waits for peer k's flag; the barrier passes what each of them acquired on to everyone
+                bool late = false;
+                if (et < npeer && peer_active(et + 1)) {
+                    volatile unsigned int* f = p.flags + blockIdx.x + 2 * (et + 1);
                     const unsigned long long t0 = g::global_timer_ns();
-                    for (int k = 1; k <= npeer; ++k) {
-                        if (!peer_active(k)) continue;
-                        volatile unsigned int* f = p.flags + blockIdx.x + 2 * k;
-                        while (*f == 0u) {
-                            if (*abort != 0 || g::global_timer_ns() - t0 > kGemmWaitNs) { *abort = 1; break; }
-                        }
+                    while (*f == 0u) {
+                        if (*abort != 0 || g::global_timer_ns() - t0 > kGemmWaitNs) { *abort = 1; late = true; break; }
                     }
                     __threadfence();
                 }
-                if (epi_any(et == 0 && *abort != 0)) { ok = false; break; }   // thread 0's view of the flag, for everyone
+                if (epi_any(late)) { ok = false; break; }
             }
-            // slot layout [token][row]: a warp touches 32 consecutive floats per access
-            float* my_slot = p.partials + static_cast<size_t>(blockIdx.x) * (TOK * kRowsPerCta) + 32 * q + lane;
-            if (is_partial) {
+            // slot layout [epilogue warp][token][row of the warp]: the 16-token pieces of a warp are contiguous 2 KB
+            float* my_slot = p.partials + static_cast<size_t>(blockIdx.x) * (TOK * kRowsPerCta) + q * (TOK * 32) + lane;
+            const uint32_t stg = sbase + C::OFF_STAGE + q * 2 * kYBoxBytes + 2 * lane;    // my output staging, at my row
+            const int n0 = kRowsPerCta * rb + 32 * q;
+            bool bad = false;                    // a wait inside the owner's loop gave up
+            if (!is_partial && npeer == 0) {
+                // whole tile: 32 tokens at a time through shared memory, one tensor store per chunk; the
+                // store of a chunk reads its buffer while the next chunk is written into the other one
+#pragma unroll 1
+                for (int cc = 0; cc < TOK / kYBox; ++cc) {
+                    const uint32_t buf = stg + (cc & 1) * kYBoxBytes;
+                    if (lane == 0) g::bulk_wait_read<1>();
+                    __syncwarp();
+                    uint32_t v[32];
+                    g::tmem_ld32(tmem + (static_cast<uint32_t>(32 * q) << 16) + kYBox * cc, v);
+                    g::tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const __half2 h = __floats2half2_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+                        g::sts_u16(buf + (2 * i) * 2 * kYBox, __half_as_ushort(__low2half(h)));
+                        g::sts_u16(buf + (2 * i + 1) * 2 * kYBox, __half_as_ushort(__high2half(h)));
+                    }
+                    g::fence_proxy_async();
+                    __syncwarp();
+                    const int m0 = mt * TOK + kYBox * cc;
+                    if (lane == 0 && n0 < N && m0 < p.M) {
+                        g::tma_store_2d(&y_map, n0, m0, buf - 2 * lane);
+                        g::bulk_commit();
+                    }
+                }
+            } else if (is_partial) {
 #pragma unroll 1
                 for (int cc = 0; cc < TOK / kEpiCols; ++cc) {
                     uint32_t v[kEpiCols];
                     g::tmem_ld16(tmem + (static_cast<uint32_t>(32 * q) << 16) + kEpiCols * cc, v);
                     g::tc_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < kEpiCols; ++i) my_slot[(kEpiCols * cc + i) * kRowsPerCta] = __uint_as_float(v[i]);
+                    for (int i = 0; i < kEpiCols; ++i) my_slot[(kEpiCols * cc + i) * 32] = __uint_as_float(v[i]);
                 }
             } else {
-                // sum of the peers' partials for one chunk of tokens, in CTA order
-                auto peer_sum = [&](int cc, float (&t)[kEpiCols]) {
+                // Owner of a cut tile.  This is the last segment of my range, so the activation stages are free (every
+                // MMA that read them has completed): my quarter of them is a ring of 2 KB sub-slots into which lane 0
+                // brings the peers' partials by bulk copies, one per (16-token piece, peer), a ring's worth ahead.
+                // Piece by piece the peers are added in pair order, then the accumulator; two pieces make one
+                // tensor store.
+                constexpr int S = C::NPEERBAR;
+                static_assert((S & (S - 1)) == 0 && S * 2048 * 4 <= C::OFF_P, "ring of the peers' partials");
+                const int np_act = __popcll(act);
+                const int J = S * np_act;
+                // the active peer after peer k, going round
+                auto next_peer = [&](int k) {
+                    const unsigned long long above = k < 64 ? act >> k : 0ull;
+                    return above != 0ull ? k + __ffsll(static_cast<long long>(above)) : __ffsll(static_cast<long long>(act));
+                };
+                const uint32_t ring = sbase + q * (S * 2048);
+                const float* peer0 = p.partials + static_cast<size_t>(blockIdx.x) * (TOK * kRowsPerCta) + q * (TOK * 32);
+                int j_iss = 0, k_iss = np_act > 0 ? next_peer(64) : 0, cc_iss = 0, a_iss = 0, j_con = 0;
+                auto issue_next = [&]() {                        // job j_iss = (piece cc_iss, peer k_iss)
+                    if (lane == 0) {
+                        const uint32_t slot = j_iss & (S - 1);
+                        g::mbar_expect_tx(peer_full(q, slot), 2048);
+                        g::bulk_g2s(ring + slot * 2048, peer0 + static_cast<size_t>(2 * k_iss) * (TOK * kRowsPerCta) + cc_iss * 512, 2048,
+                                    peer_full(q, slot));
+                    }
+                    ++j_iss;
+                    k_iss = next_peer(k_iss);
+                    if (++a_iss == np_act) { a_iss = 0; ++cc_iss; }
+                };
+                g::fence_proxy_async_all();                      // the flags were seen through ordinary loads
+                while (j_iss < min(S, J)) issue_next();
+#pragma unroll 1
+                for (int cc = 0; cc < S && !bad; ++cc) {
+                    float t[kEpiCols];
 #pragma unroll
                     for (int i = 0; i < kEpiCols; ++i) t[i] = 0.f;
-                    for (int k = 1; k <= npeer; ++k) {
-                        if (!peer_active(k)) continue;
-                        const float* slot = p.partials + static_cast<size_t>(blockIdx.x + 2 * k) * (TOK * kRowsPerCta) + 32 * q + lane;
+                    for (int a = 0; a < np_act; ++a) {
+                        const uint32_t slot = j_con & (S - 1);
+                        if (!g::mbar_wait_warp(peer_full(q, slot), (j_con / S) & 1, abort)) { bad = true; break; }
+                        ++j_con;
 #pragma unroll
-                        for (int i = 0; i < kEpiCols; ++i) t[i] += __ldcg(slot + (kEpiCols * cc + i) * kRowsPerCta);
+                        for (int i = 0; i < kEpiCols; ++i) t[i] += g::lds_f32(ring + slot * 2048 + 128 * i + 4 * lane);
+                        __syncwarp();
+                        if (j_iss < J) issue_next();
                     }
-                };
-                float t[kEpiCols];
-                if (npeer > 0) peer_sum(0, t);
-#pragma unroll 1
-                for (int cc = 0; cc < TOK / kEpiCols; ++cc) {
+                    if (bad) break;
                     uint32_t v[kEpiCols];
                     g::tmem_ld16(tmem + (static_cast<uint32_t>(32 * q) << 16) + kEpiCols * cc, v);
                     g::tc_wait_ld();
-                    if (npeer > 0) {
-#pragma unroll
-                        for (int i = 0; i < kEpiCols; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + t[i]);
-                        if (cc + 1 < TOK / kEpiCols) peer_sum(cc + 1, t);     // in flight while this chunk is stored
+                    const uint32_t buf = stg + ((cc >> 1) & 1) * kYBoxBytes + (cc & 1) * (kEpiCols * 2 * kYBox);
+                    if ((cc & 1) == 0) {
+                        if (lane == 0) g::bulk_wait_read<1>();
+                        __syncwarp();
                     }
-                    const int m0 = mt * TOK + kEpiCols * cc;
-                    if (n < N) {
 #pragma unroll
-                        for (int i = 0; i < kEpiCols; ++i)
-                            if (m0 + i < p.M) p.y[static_cast<size_t>(m0 + i) * N + n] = __float2half_rn(__uint_as_float(v[i]));
+                    for (int i = 0; i < kEpiCols / 2; ++i) {
+                        const __half2 h = __floats2half2_rn(__uint_as_float(v[2 * i]) + t[2 * i], __uint_as_float(v[2 * i + 1]) + t[2 * i + 1]);
+                        g::sts_u16(buf + (2 * i) * 2 * kYBox, __half_as_ushort(__low2half(h)));
+                        g::sts_u16(buf + (2 * i + 1) * 2 * kYBox, __half_as_ushort(__high2half(h)));
+                    }
+                    if (cc & 1) {
+                        g::fence_proxy_async();
+                        __syncwarp();
+                        const int m0 = mt * TOK + kEpiCols * (cc - 1);
+                        if (lane == 0 && n0 < N && m0 < p.M) {
+                            g::tma_store_2d(&y_map, n0, m0, stg - 2 * lane + ((cc >> 1) & 1) * kYBoxBytes);
+                            g::bulk_commit();
+                        }
                     }
                 }
+                if (bad)                                         // leave no copy in flight
+                    for (int j = j_con; j < j_iss; ++j) g::mbar_drain(peer_full(q, j & (S - 1)), (j / S) & 1);
             }
             g::tc_fence_before();
             __syncwarp();
@@ -714,10 +814,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ G
                 epi_sync();
                 if (et == 0) { __threadfence(); *(volatile unsigned int*)(p.flags + blockIdx.x) = 1u; }
             } else if (npeer > 0) {
-                epi_sync();                                     // everyone has read the peers' slots
+                if (epi_any(bad)) { ok = false; break; }        // everyone has read the peers' slots
                 if (et < npeer) p.flags[blockIdx.x + 2 * (1 + et)] = 0u;   // ready for the next launch (unused ones are 0 already)
             }
         }
+        if (lane == 0) g::bulk_wait_all();                      // my stores have been written
     }
 
     // nobody leaves, and the pair's tensor memory stays, until both CTAs are through
@@ -757,6 +858,19 @@ static bool make_x_map(CUtensorMap* map, const void* x, int M, int K, int rows) 
     const cuuint32_t estr[2] = {1u, 1u};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Tensor map of y [M][N] fp16 for the epilogue's stores: boxes of 32 rows of W x 32 tokens, no swizzle.
+static bool make_y_map(CUtensorMap* map, void* y, int M, int N) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (enc == nullptr) return false;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(M)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(N) * sizeof(__half)};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kYBox), static_cast<cuuint32_t>(kYBox)};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -817,11 +931,13 @@ static GemmPlan plan_gemm(int M, int N, int G) {
     const int waves = (tiles + pairs - 1) / pairs;
     pl.grid = 2 * npairs;
     pl.stream_k = 0;
-    // time in units of one group: whole tiles take waves * G; equal shares take units / pairs plus
-    // about two dozen groups' worth of draining, storing and re-reading a partial tile (measured)
+    // time in units of one group: whole tiles take waves * G; equal shares take units / pairs plus the
+    // hand-over of the cut tiles, a dozen groups' worth for the drains and flags and seven (256 tokens) or
+    // three and a half (128) per peer whose partial tile the owner of a tile brings in and adds (measured)
     const long long units = static_cast<long long>(tiles) * G;
-    if (resident > 0 && units >= 8ll * pairs &&
-        static_cast<double>(units) / pairs + 24.0 < 0.95 * static_cast<double>(waves) * G) {
+    const double share = static_cast<double>(units) / pairs;
+    const double handover = 12.0 + (pl.tok == 256 ? 7.0 : 3.5) * ceil(static_cast<double>(G) / (share > 1.0 ? share : 1.0));
+    if (resident > 0 && units >= 8ll * pairs && share + handover < 0.93 * static_cast<double>(waves) * G) {
         pl.stream_k = 1;
         pl.grid = 2 * pairs;
     }
@@ -831,7 +947,7 @@ static GemmPlan plan_gemm(int M, int N, int G) {
 size_t gemm_workspace_bytes(int M, int N, int G) { return plan_gemm(M, N, G).workspace_bytes; }
 
 template <int TOK>
-static cudaError_t launch_gemm(const CUtensorMap& map, const GemmParams& prm, int grid, cudaStream_t stream) {
+static cudaError_t launch_gemm(const CUtensorMap& map, const CUtensorMap& ymap, const GemmParams& prm, int grid, cudaStream_t stream) {
     static std::atomic<bool> attr_set[64];    // zero-initialised; set-up is idempotent, so a race repeats it harmlessly
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -841,7 +957,7 @@ static cudaError_t launch_gemm(const CUtensorMap& map, const GemmParams& prm, in
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    gemm_kernel<TOK><<<grid, kGemmThreads, GemmCfg<TOK>::SMEM, stream>>>(map, prm);   // clusters of 2: see the kernel
+    gemm_kernel<TOK><<<grid, kGemmThreads, GemmCfg<TOK>::SMEM, stream>>>(map, ymap, prm);   // clusters of 2: see the kernel
     return cudaGetLastError();
 }
 
@@ -878,7 +994,8 @@ extern "C" int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* b
     }
     const int tok = pl.tok;
     CUtensorMap map;
-    if (!slim::make_x_map(&map, x, M, K, tok / 2)) {
+    CUtensorMap ymap;
+    if (!slim::make_x_map(&map, x, M, K, tok / 2) || !slim::make_y_map(&ymap, y, M, N)) {
         slim::set_cuda_error(cudaErrorUnknown);
         return SLIM_ERR_CUDA;
     }
@@ -896,7 +1013,7 @@ extern "C" int slim_mpq_gemm(const void* x, const void* packed, const uint8_t* b
     prm.tok_tiles = pl.tok_tiles;
     prm.stream_k = pl.stream_k;
     prm.gt = gt;
-    const cudaError_t e = tok == 128 ? slim::launch_gemm<128>(map, prm, pl.grid, s) : slim::launch_gemm<256>(map, prm, pl.grid, s);
+    const cudaError_t e = tok == 128 ? slim::launch_gemm<128>(map, ymap, prm, pl.grid, s) : slim::launch_gemm<256>(map, ymap, prm, pl.grid, s);
     SLIM_CUDA_TRY(e);
     return SLIM_OK;
 }
