@@ -60,7 +60,7 @@ NCU_TRAFFIC = {
 # DRAM bytes (read + written) of the 14 gemm_kernel launches of one step of llama13b-prefill-avg3-m2048, from one ncu
 # capture of dram__bytes_read.sum and dram__bytes_write.sum; keyed by the SHA-256 of slim_gemm.cu at capture time
 NCU_TRAFFIC_GEMM = {
-    "7082f3a4c2b0494e1fc5b0a677a09ca71f4b833ea04442557984c259de1928ef": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1081612800 + 227610112},
+    "dbc3193e73bdb7e948ea7dbf80ad45e9062ae8502ba37a68ba3fc72e6b14adae": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1089319424 + 227502336},
 }
 
 
