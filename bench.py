@@ -60,7 +60,7 @@ NCU_TRAFFIC = {
 # DRAM bytes (read + written) of the 14 gemm_kernel launches of one step of llama13b-prefill-avg3-m2048, from one ncu
 # capture of dram__bytes_read.sum and dram__bytes_write.sum; keyed by the SHA-256 of slim_gemm.cu at capture time
 NCU_TRAFFIC_GEMM = {
-    "dbc3193e73bdb7e948ea7dbf80ad45e9062ae8502ba37a68ba3fc72e6b14adae": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1089319424 + 227502336},
+    "6f5c4d2ed60f5eb666f3c4ef50c259260639ac2a29d416275f184f177415e16e": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1092798464 + 225962240},
 }
 
 

