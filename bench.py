@@ -60,7 +60,7 @@ NCU_TRAFFIC = {
 # DRAM bytes (read + written) of the 14 gemm_kernel launches of one step of llama13b-prefill-avg3-m2048, from one ncu
 # capture of dram__bytes_read.sum and dram__bytes_write.sum; keyed by the SHA-256 of slim_gemm.cu at capture time
 NCU_TRAFFIC_GEMM = {
-    "6f5c4d2ed60f5eb666f3c4ef50c259260639ac2a29d416275f184f177415e16e": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1092798464 + 225962240},
+    "ad7945290f038e77cbf6c6d2a50d2968e912f1a5cf48c971f87e17eb864f8f57": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1082789120 + 227386112},
 }
 
 

@@ -935,12 +935,14 @@ static GemmPlan plan_gemm(int M, int N, int G) {
     pl.grid = 2 * npairs;
     pl.stream_k = 0;
     // time in units of one group: whole tiles take waves * G; equal shares take units / pairs plus the
-    // hand-over of the cut tiles, a dozen groups' worth for the drains and flags and seven (256 tokens) or
-    // three and a half (128) per peer whose partial tile the owner of a tile brings in and adds (measured)
+    // hand-over of the cut tiles: a dozen groups' worth when a tile has one peer (drains, flags, one partial
+    // tile brought in and added), with more peers seven more per peer at 256 tokens and three and a half at
+    // 128 (measured: graph-replayed timings of nine layer shapes at M = 32 ... 2048 with either schedule)
     const long long units = static_cast<long long>(tiles) * G;
     const double share = static_cast<double>(units) / pairs;
-    const double handover = 12.0 + (pl.tok == 256 ? 7.0 : 3.5) * ceil(static_cast<double>(G) / (share > 1.0 ? share : 1.0));
-    if (resident > 0 && units >= 8ll * pairs && share + handover < 0.93 * static_cast<double>(waves) * G) {
+    const double peers = ceil(static_cast<double>(G) / (share > 1.0 ? share : 1.0));
+    const double handover = 12.0 + (peers > 1.0 ? (pl.tok == 256 ? 7.0 : 3.5) * peers : 0.0);
+    if (resident > 0 && units >= 8ll * pairs && share + handover < 0.95 * static_cast<double>(waves) * G) {
         pl.stream_k = 1;
         pl.grid = 2 * pairs;
     }
