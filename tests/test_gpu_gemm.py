@@ -101,6 +101,22 @@ def test_stream_k_and_whole_tile_paths_agree():
     assert np.abs(ys[0].astype(np.float64) - ys[1].astype(np.float64)).max() <= 2e-3 * np.abs(ys[1].astype(np.float64)).max()
 
 
+@pytest.mark.parametrize("M", [100, 300])
+def test_cut_tiles_with_many_peers(M):
+    """Few tiles and a long K: the plan cuts every tile into many segments, so the pair that starts a tile adds the
+    partial tiles of five to nine peers (its shared-memory ring goes round several times), with a ragged last row
+    block and a ragged token tile, at 128 and at 256 tokens per tile."""
+    slim = _slim()
+    N, K = 2064, 13824
+    L = oracle_layer(N, K, 3, M)
+    assert slim.workspace_bytes(M, N, K, L["bits"]) > 1 << 20          # the tiles are cut
+    y1 = _run(L)
+    y2 = _run(L)
+    assert (y1.view(np.uint16) == y2.view(np.uint16)).all()
+    rows = np.unique(np.concatenate([[0, 127, 128, 2047, 2048, 2063], np.random.default_rng(M).integers(0, N, 100)]))
+    check_output(y1[:, rows], orc.linear_rows_f64(L["x"], L["codes"], L["scales"], L["zeros"], rows), f"{N}x{K} M={M}")
+
+
 def test_argument_errors_are_statuses():
     slim = _slim()
     L = oracle_layer(128, 256, 2, 1)
