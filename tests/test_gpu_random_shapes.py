@@ -1,6 +1,7 @@
 """GPU parity on seeded random shapes: the decode path through both of its entry points (slim_mpq_gemv and the
-layer-set launch) against the fp64 oracle, over row counts, K, group sizes, bit maps, token counts, activation
-scales and half-integer zero points that the hand-picked cases of the other files do not enumerate."""
+layer-set launch) and the batched path (slim_mpq_gemm) against the fp64 oracle, over row counts, K, group sizes,
+bit maps, token counts, activation scales and half-integer zero points that the hand-picked cases of the other
+files do not enumerate."""
 import numpy as np
 import pytest
 import torch
@@ -74,3 +75,23 @@ def test_sets_of_several_layers(seed):
         for i, ((L, _, y), ref) in enumerate(zip(entries, refs)):
             check_output(y.cpu().numpy(), ref, f"seed {seed} case {case} layer {i}: {L.N}x{L.K} g={g}")
     assert modes          # which routes a seed reaches depends on its draws; the union over the seeds is all three
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_batched_path_on_random_shapes(seed):
+    """slim_mpq_gemm on random row counts, K, group sizes, bit maps and 17 to 700 tokens: ragged row blocks and token
+    tiles (the output leaves through clipped tensor stores), whole tiles and cut ones (a long K on few tiles)."""
+    from paper_2405_14917_b200 import binding as slim
+    rng = np.random.default_rng(3000 + seed)
+    for case in range(6):
+        g = int(rng.choice([128, 128, 256, 512]))
+        M = int(rng.integers(17, 701))
+        long_k = case % 2 == 1                       # every other case: few row blocks, many groups
+        L, x, ref = _random_layer(rng, g, M, max_k=16384 if long_k else 4096, max_tiles=24 if long_k else 160)
+        ws = torch.zeros(L.workspace_bytes(M), dtype=torch.uint8, device="cuda")
+        slim.workspace_init(ws)
+        y = torch.full((M, L.N), float("nan"), dtype=torch.float16, device="cuda")
+        for _ in range(2):                           # twice into the same workspace: its flags must come back to zero
+            L.forward(torch.from_numpy(x).cuda(), ws, out=y)
+        slim.workspace_status(ws)
+        check_output(y.cpu().numpy(), ref, f"gemm seed {seed} case {case}: {L.N}x{L.K} g={g} M={M}")
