@@ -60,7 +60,7 @@ NCU_TRAFFIC = {
 # DRAM bytes (read + written) of the 14 gemm_kernel launches of one step of llama13b-prefill-avg3-m2048, from one ncu
 # capture of dram__bytes_read.sum and dram__bytes_write.sum; keyed by the SHA-256 of slim_gemm.cu at capture time
 NCU_TRAFFIC_GEMM = {
-    "ad7945290f038e77cbf6c6d2a50d2968e912f1a5cf48c971f87e17eb864f8f57": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1082789120 + 227386112},
+    "a9b998b7a42c63bfc7bf8985dc1e3ee6b8be9ec1e3e35774be2538fadf174e9b": {"workload": "llama13b-prefill-avg3-m2048", "launches": 14, "traffic_bytes": 1049365760 + 218744064},
 }
 
 

@@ -934,17 +934,27 @@ static GemmPlan plan_gemm(int M, int N, int G) {
     const int waves = (tiles + pairs - 1) / pairs;
     pl.grid = 2 * npairs;
     pl.stream_k = 0;
-    // time in units of one group: whole tiles take waves * G; equal shares take units / pairs plus the
-    // hand-over of the cut tiles: a dozen groups' worth when a tile has one peer (drains, flags, one partial
-    // tile brought in and added), with more peers seven more per peer at 256 tokens and three and a half at
-    // 128 (measured: graph-replayed timings of nine layer shapes at M = 32 ... 2048 with either schedule)
+    // Time in units of one group.  Whole tiles take waves * G.  Equal shares of the (tile, group) units over P
+    // pairs take units / P plus the hand-over of the cut tiles: a dozen groups' worth when a tile has one peer
+    // (drains, flags, one partial tile brought in and added), with more peers seven more per peer at 256 tokens
+    // and three and a half at 128 (measured: graph-replayed timings of nine layer shapes at M = 32 ... 2048 with
+    // either schedule).  P is every resident pair, or, for a layer with few tiles, two, three or four pairs per
+    // tile: the cuts then fall on the same groups in every tile and a tile has one, two or three peers, where
+    // equal shares over all pairs would give it more.
     const long long units = static_cast<long long>(tiles) * G;
-    const double share = static_cast<double>(units) / pairs;
-    const double peers = ceil(static_cast<double>(G) / (share > 1.0 ? share : 1.0));
-    const double handover = 12.0 + (peers > 1.0 ? (pl.tok == 256 ? 7.0 : 3.5) * peers : 0.0);
-    if (resident > 0 && units >= 8ll * pairs && share + handover < 0.95 * static_cast<double>(waves) * G) {
-        pl.stream_k = 1;
-        pl.grid = 2 * pairs;
+    const double per_peer = pl.tok == 256 ? 7.0 : 3.5;
+    double best = 0.95 * static_cast<double>(waves) * G;
+    for (int k = 1; k <= 4 && resident > 0; ++k) {
+        const int P = k == 1 ? pairs : k * tiles;
+        if (P > pairs || units < 8ll * P) continue;
+        const double share = static_cast<double>(units) / P;
+        const double peers = k == 1 ? ceil(static_cast<double>(G) / share) : static_cast<double>(k - 1);
+        const double cost = share + 12.0 + (peers > 1.0 ? per_peer * peers : 0.0);
+        if (cost < best) {
+            best = cost;
+            pl.stream_k = 1;
+            pl.grid = 2 * P;
+        }
     }
     pl.workspace_bytes = pl.stream_k ? kGemmWsPartials + static_cast<size_t>(pl.grid) * pl.tok * kRowsPerCta * sizeof(float) : 256;
     return pl;
