@@ -922,10 +922,10 @@ def secondary_entries(args, device, timer, primary_layers, clock_gpu):
     except Exception as e:
         out.append({"name": "group sizes", "error": f"{type(e).__name__}: {e}"})
     torch.cuda.empty_cache()
-    for wname in ("llama13b-prefill-avg3-m2048", "llama13b-prefill-avg3-m512"):
+    for wname in ("llama13b-prefill-avg3-m2048", "llama13b-prefill-avg3-m512", "llama13b-prefill-avg3-m128"):
         spec = workload_spec(wname)
         layers13 = build_layers(spec, device, 0) if wname.endswith("m2048") else layers13
-        guarded(lambda: gemm_entry(wname, layers13, spec, device, timer, 20, 1.0, clock_gpu=clock_gpu))
+        guarded(lambda: gemm_entry(wname, layers13, spec, device, timer, 20, 1.0 if spec["M"] >= 512 else 0.5, clock_gpu=clock_gpu))
     del layers13
     torch.cuda.empty_cache()
     spec3 = workload_spec("llama7b-decode-avg3-m1-blocks8")
