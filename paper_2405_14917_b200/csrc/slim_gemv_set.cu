@@ -142,6 +142,8 @@ __device__ __forceinline__ void stage_task(const SetLayer& L, uint8_t* ws, int p
 // One warp per (layer, token, group): fragments and sums of the whole set, once.
 __global__ void __launch_bounds__(256) gemv_set_stage_kernel(const SetLayer* __restrict__ layers, uint8_t* ws, int n_layers, int n_tasks,
                                                              int n_counters) {
+    pdl_wait();                       // x may be the output of the kernel before; the workspace may still be read by it
+    pdl_launch_dependents();
     stage_clear_counters(ws, n_counters);
     const int lane = threadIdx.x & 31;
     const int task = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -549,6 +551,11 @@ __global__ void __launch_bounds__(kSetThreads, NT >= 4 ? 1 : kSetCtasPerSm) gemv
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
+    // Launched with programmatic stream serialization: everything above ran while the kernel before (the staging
+    // kernel of this set) was still finishing; nothing of the plan or the workspace is read before it has completed.
+    // The kernel after this one may be set up early in turn (ours wait in the same way before they touch memory).
+    pdl_wait();
+    pdl_launch_dependents();
 
     const int i0 = p.item_begin[blockIdx.x], i1 = p.item_begin[blockIdx.x + 1];
     if (i0 < i1) {
@@ -635,6 +642,8 @@ __global__ void __launch_bounds__(kSetThreads, NT >= 4 ? 1 : kSetCtasPerSm) gemv
 // large layers this way).
 __global__ void __launch_bounds__(256) set_single_stage_kernel(const __grid_constant__ SetLayer d, uint8_t* plan, uint8_t* ws, int grid,
                                                                int n_rb, int sp, int n_tasks, int n_counters) {
+    pdl_wait();                       // x may be the output of the kernel before; the workspace may still be read by it
+    pdl_launch_dependents();
     stage_clear_counters(ws, n_counters);
     if (blockIdx.x == 0) {
         int* item_begin = reinterpret_cast<int*>(plan);
@@ -839,8 +848,26 @@ static size_t set_plan_bytes(int n_layers, long long n_items) {
     return kSetPlanHeader + static_cast<size_t>(n_layers) * sizeof(SetLayer) + static_cast<size_t>(n_items) * sizeof(SetItem);
 }
 
+// Launch configuration with programmatic stream serialization: the kernel may be set up while the one before it in
+// the stream is still running; it waits (griddepcontrol.wait) before it touches what that kernel reads or writes.
+struct PdlLaunch {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    PdlLaunch(unsigned grid, unsigned block, size_t smem, cudaStream_t stream, bool early = true) {
+        memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3(grid, 1, 1);
+        cfg.blockDim = dim3(block, 1, 1);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = early ? 1 : 0;
+    }
+};
+
 template <int NT, bool ONE, int TPW>
-static cudaError_t launch_set(const SetParams& prm, int grid, size_t smem, cudaStream_t stream) {
+static cudaError_t launch_set(const SetParams& prm, int grid, size_t smem, cudaStream_t stream, bool early) {
     static std::atomic<bool> attr_set[64];    // zero-initialised; set-up is idempotent, so a race repeats it harmlessly
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -850,8 +877,8 @@ static cudaError_t launch_set(const SetParams& prm, int grid, size_t smem, cudaS
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    gemv_set_kernel<NT, ONE, TPW><<<grid, kSetThreads, smem, stream>>>(prm);
-    return cudaGetLastError();
+    PdlLaunch l(static_cast<unsigned>(grid), kSetThreads, smem, stream, early);
+    return cudaLaunchKernelEx(&l.cfg, gemv_set_kernel<NT, ONE, TPW>, prm);
 }
 
 }  // namespace slim
@@ -931,12 +958,12 @@ static int set_params(const slim_gemv_set_info* info, const void* plan, void* wo
 }
 
 // The persistent kernel of the set in the form its token count asks for.
-static int launch_set_for(const slim_gemv_set_info* info, const SetParams& prm, size_t smem, cudaStream_t s) {
-    const cudaError_t e = info->max_tokens == 1 ? launch_set<1, true, 2>(prm, info->grid, smem, s)
-                        : info->token_tiles == 8 ? launch_set<8, false, 2>(prm, info->grid, smem, s)
-                        : info->token_tiles == 4 ? launch_set<4, false, 2>(prm, info->grid, smem, s)
-                        : info->token_tiles == 1 ? launch_set<1, false, 2>(prm, info->grid, smem, s)
-                                                 : launch_set<2, false, 2>(prm, info->grid, smem, s);
+static int launch_set_for(const slim_gemv_set_info* info, const SetParams& prm, size_t smem, cudaStream_t s, bool early) {
+    const cudaError_t e = info->max_tokens == 1 ? launch_set<1, true, 2>(prm, info->grid, smem, s, early)
+                        : info->token_tiles == 8 ? launch_set<8, false, 2>(prm, info->grid, smem, s, early)
+                        : info->token_tiles == 4 ? launch_set<4, false, 2>(prm, info->grid, smem, s, early)
+                        : info->token_tiles == 1 ? launch_set<1, false, 2>(prm, info->grid, smem, s, early)
+                                                 : launch_set<2, false, 2>(prm, info->grid, smem, s, early);
     SLIM_CUDA_TRY(e);
     return SLIM_OK;
 }
@@ -975,9 +1002,11 @@ int gemv_route(const void* x, const void* packed, const uint8_t* bits_host, cons
     size_t smem = 0;
     const int st = set_params(&info, plan, workspace, workspace_bytes, &prm, &smem);
     if (st != SLIM_OK) return st;
-    set_single_stage_kernel<<<(info.stage_tasks + 7) / 8, 256, 0, stream>>>(d, plan, prm.ws, grid, r.n_rb, r.sp, info.stage_tasks, info.n_counters);
-    SLIM_CUDA_TRY(cudaGetLastError());
-    return launch_set_for(&info, prm, smem, stream);
+    {
+        PdlLaunch l(static_cast<unsigned>((info.stage_tasks + 7) / 8), 256, 0, stream);
+        SLIM_CUDA_TRY(cudaLaunchKernelEx(&l.cfg, set_single_stage_kernel, d, plan, prm.ws, grid, r.n_rb, r.sp, info.stage_tasks, info.n_counters));
+    }
+    return launch_set_for(&info, prm, smem, stream, true);
 }
 
 }  // namespace slim
@@ -1179,9 +1208,11 @@ int slim_mpq_gemv_set(const slim_gemv_set_info* info, const void* plan, void* wo
     const int st = slim::set_params(info, plan, workspace, workspace_bytes, &prm, &smem);
     if (st != SLIM_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    slim::gemv_set_stage_kernel<<<(info->stage_tasks + 7) / 8, 256, 0, s>>>(prm.layers, prm.ws, info->n_layers, info->stage_tasks, info->n_counters);
-    SLIM_CUDA_TRY(cudaGetLastError());
-    return slim::launch_set_for(info, prm, smem, s);
+    {
+        slim::PdlLaunch l(static_cast<unsigned>((info->stage_tasks + 7) / 8), 256, 0, s, false);
+        SLIM_CUDA_TRY(cudaLaunchKernelEx(&l.cfg, slim::gemv_set_stage_kernel, prm.layers, prm.ws, info->n_layers, info->stage_tasks, info->n_counters));
+    }
+    return slim::launch_set_for(info, prm, smem, s, false);
 }
 
 }  // extern "C"
