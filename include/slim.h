@@ -145,8 +145,8 @@ int slim_dequant(const void* packed, const uint8_t* bits_host, const void* scale
  * The per-layer kernels are launched with programmatic stream serialisation and fetches packed, scales and zeros
  * before it waits for the kernel ahead of it on the stream: those three buffers must be complete when the call is
  * enqueued, or be written by a kernel that does not signal programmatic launch completion early (x and y may be
- * produced and consumed by the neighbouring kernels as usual).  The two kernels of the 32 MB route are launched the
- * same way, but touch no buffer before they have waited for the kernel ahead of them. */
+ * produced and consumed by the neighbouring kernels as usual).  At M = 1 the two kernels of the 32 MB route are launched
+ * the same way, but touch no buffer before they have waited for the kernel ahead of them. */
 int slim_mpq_gemv(const void* x, const void* packed, const uint8_t* bits_host,
                   const void* scales, const void* zeros, void* y,
                   int M, int N, int K, int g,
